@@ -1,0 +1,157 @@
+/*
+ * hyq.h - C ABI of the B200 (sm_100a) HyQuant prefill path.
+ *
+ * Three operations, in the order the paper's prefill operator runs them
+ * (Algorithm 2: Stage 1 -> Stage 2 -> Stage 3):
+ *
+ *   hyq_select_vertical            Algorithm 1 (vertical token identification)
+ *   hyq_quantize_blocks            Algorithm 2, Stage 2 (per-tile quantization)
+ *   hyq_hybrid_attention_prefill   Eq. 6-7 / Algorithm 2, Stage 3 (fused hybrid softmax attention)
+ *
+ * Common rules
+ *   - Every tensor pointer is a DEVICE pointer to a contiguous row-major array.
+ *     Q is [B, Hq, L, D]; K and V are [B, Hkv, L, D]; bf16 unless stated.
+ *     Hq % Hkv == 0; query head h reads kv head h / (Hq / Hkv) (Algorithm 1's
+ *     reshape Hq -> Hkv x g).  D must be 128.  L >= 1 is arbitrary (ragged tails
+ *     are handled); Lq == Lk == L.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Calls
+ *     enqueue work and return; they never synchronise.
+ *   - The caller owns every buffer, including `workspace`; the library allocates
+ *     no device memory and keeps no pointer once the enqueued work has completed.
+ *     Workspace sizes come from the *_workspace queries (host-only, no launches).
+ *     Workspace and tensor pointers must be 16-byte aligned.
+ *   - Return value: HYQ_OK or an error code.  Arguments are checked on the host
+ *     before anything is launched; on error nothing has been enqueued.  Device-side
+ *     anomalies (a bounded wait that ran out) are written to `status_word` and
+ *     the kernel exits normally - no trap, no hang.
+ *   - NaN / Inf inputs are undefined behaviour.
+ */
+#ifndef HYQ_H_
+#define HYQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+  HYQ_OK = 0,
+  HYQ_ERR_INVALID_ARG = 1,   /* null pointer, non-positive size, k > P, Hq % Hkv != 0 ... */
+  HYQ_ERR_UNSUPPORTED = 2,   /* D != 128, block_tokens != 64, format combination not built */
+  HYQ_ERR_WORKSPACE = 3,     /* workspace_bytes smaller than the matching *_workspace query */
+  HYQ_ERR_ALIGNMENT = 4,     /* a pointer is not 16-byte aligned */
+  HYQ_ERR_CUDA = 5,          /* a CUDA runtime / driver call failed (launch, tensor map) */
+  HYQ_ERR_TIMEOUT = 6        /* value written to status_word by a kernel whose bounded wait expired */
+};
+
+/* low-bit formats of Algorithm 2 Stage 2 (c_B = 127 / 448; 7 for INT4) */
+enum { HYQ_FMT_INT8 = 0, HYQ_FMT_FP8_E4M3 = 1, HYQ_FMT_INT4 = 2 };
+
+/* attention kernel choice */
+enum {
+  HYQ_IMPL_AUTO = 0,      /* the tensor-core kernel */
+  HYQ_IMPL_TCGEN05 = 1,   /* TMA + tcgen05.mma + TMEM kernel */
+  HYQ_IMPL_SIMT = 2       /* plain fp32 CUDA-core kernel: slow, used to cross-check at sizes the CPU cannot */
+};
+
+/* Static string for a status code. */
+const char* hyq_status_string(int status);
+
+/* Library ABI version (bumped when a signature or struct changes). */
+int hyq_version(void);
+
+/* Algorithm 1's count: k = min(P, max(1, ceil(P * ratio))) with P = max(0, Lk - window); 0 when P == 0. */
+int hyq_paper_k(int Lk, int window, double ratio);
+
+/* ---------------------------------------------------------------------------------------------
+ * hyq_select_vertical - Algorithm 1 (vertical token identification).
+ *
+ *   P    = max(0, Lk - window)                      candidate keys: the non-window prefix [0, P)
+ *   t    = n_tail, or min(window, Lq) if n_tail == 0
+ *   qbar = mean of the last t query rows of head (b, h)           (fp64)
+ *   S[p] = qbar . K[b, h / g, p, :]                               (fp64 fma chain over channels 0..D-1)
+ *   idx_out[b, h, :] = positions of the k largest S, equal scores resolved towards the
+ *                      lower position, written in ASCENDING position order.
+ *
+ *   q [B,Hq,Lq,D] bf16, k_ [B,Hkv,Lk,D] bf16 (device, read-only).
+ *   idx_out [B,Hq,k] int32 (device, written).  k == 0 or P == 0: nothing is written, HYQ_OK.
+ *   Errors: k > P or k < 0, n_tail > Lq, window == 0 with n_tail == 0 and k > 0 -> INVALID_ARG.
+ *   workspace: hyq_select_vertical_workspace bytes (tail means + one fp64 score per (b,h,p)).
+ * ------------------------------------------------------------------------------------------- */
+int hyq_select_vertical_workspace(int B, int Hq, int Hkv, int Lq, int Lk, int D, int window, int k,
+                                  size_t* bytes /* host, out */);
+int hyq_select_vertical(const void* q, const void* k_, int B, int Hq, int Hkv, int Lq, int Lk, int D,
+                        int window, int n_tail, int k, int32_t* idx_out, void* workspace,
+                        size_t workspace_bytes, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * hyq_quantize_blocks - Algorithm 2, Stage 2 (per-tile symmetric quantization).
+ *
+ *   One tile = block_tokens (64) consecutive tokens x all D channels of one (b, head), cut by
+ *   original position; the last tile of a head may be ragged.
+ *     absmax = max |x| over the tile
+ *     scale  = absmax / c          c = 127 (INT8), 448 (FP8 e4m3), 7 (INT4)
+ *     code   = round_half_even(x * (c / absmax))     INT8 / INT4: integer, clamped to [-c, c]
+ *                                                    FP8: e4m3 (RNE, saturating at +-448)
+ *   All in fp32 with one rounding per operation.  absmax < 2^-100 (all-zero tile): scale 0, codes 0.
+ *
+ *   x [B,H,L,D] bf16 (device, read-only).
+ *   codes_out (device, written): INT8 / FP8: [B,H,L,D] bytes; INT4: [B,H,L,D/2] bytes, channel 2m
+ *       in the low nibble and 2m+1 in the high nibble of byte m, two's complement.
+ *   scales_out [B,H,ceil(L/block_tokens)] fp32 (device, written).
+ * ------------------------------------------------------------------------------------------- */
+int hyq_quantize_blocks(const void* x, int B, int H, int L, int D, int block_tokens, int format,
+                        void* codes_out, float* scales_out, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * hyq_hybrid_attention_prefill - Eq. 6-7 / Algorithm 2 Stage 3: causal attention forward in which,
+ * for query row i of head (b,h) and every key j <= i,
+ *     the pair is FULL PRECISION when j is in vl_idx[b,h,:] or i - j < window,
+ *         score = softmax_scale * <Q[i], K[j]>  (bf16 originals),   value row = V[j]
+ *     and LOW-BIT otherwise,
+ *         score = softmax_scale * q_scale * k_scale * <q_code[i], k_code[j]>,
+ *         value row = v_scale * v_code[j]
+ * and one softmax runs over all keys of the row:  out[i] = sum_j p_ij value_j / sum_j p_ij.
+ *
+ *   struct_size must be sizeof(hyq_attn_args).  Supported format triples (q,k,v):
+ *   (INT8,INT8,INT8) and (INT4,INT4,FP8_E4M3); anything else -> HYQ_ERR_UNSUPPORTED.
+ *   vl_idx [B,Hq,k] int32, each row strictly ascending, values in [0, L); NULL iff k == 0.
+ *   out [B,Hq,L,D]: fp32 (out_dtype 1) or bf16 (out_dtype 0, RNE of the fp32 result).
+ *   lse: optional [B,Hq,L] fp32 natural-log-sum-exp of the scaled scores (NULL to skip).
+ *   status_word: optional device int32; the kernel stores HYQ_ERR_TIMEOUT there if one of its
+ *   bounded waits expires (the output is then undefined); untouched otherwise.
+ * ------------------------------------------------------------------------------------------- */
+typedef struct {
+  uint32_t struct_size;
+  int32_t B, Hq, Hkv, L, D;
+  int32_t window, k, block_tokens;
+  int32_t q_format, k_format, v_format;
+  int32_t out_dtype;                 /* 0 = bf16, 1 = fp32 */
+  int32_t impl;                      /* HYQ_IMPL_* */
+  float softmax_scale;               /* 0 => 1/sqrt(D) */
+  const void* q;                     /* bf16 originals */
+  const void* k_;
+  const void* v;
+  const void* q_codes;               /* as written by hyq_quantize_blocks */
+  const void* k_codes;
+  const void* v_codes;
+  const float* q_scales;
+  const float* k_scales;
+  const float* v_scales;
+  const int32_t* vl_idx;
+  void* out;
+  float* lse;
+  int32_t* status_word;
+  void* workspace;
+  size_t workspace_bytes;
+} hyq_attn_args;
+
+int hyq_hybrid_attention_prefill_workspace(const hyq_attn_args* args, size_t* bytes /* host, out */);
+int hyq_hybrid_attention_prefill(const hyq_attn_args* args, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HYQ_H_ */

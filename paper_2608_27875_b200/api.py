@@ -1,0 +1,201 @@
+"""Thin Python binding of the C-ABI library (``include/hyq.h``): argument
+marshalling only.  torch supplies device memory and the current stream; every
+step of the path runs in the library's kernels.  There is no CPU fallback: the
+first call raises if ``libhyq.so`` has not been built."""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+from .workloads import FMT_FP8_E4M3, FMT_INT4, FMT_INT8  # noqa: F401
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libhyq.so")
+
+HYQ_OK = 0
+IMPL_AUTO, IMPL_TCGEN05, IMPL_SIMT = 0, 1, 2
+EXPORTS = ("hyq_status_string", "hyq_version", "hyq_paper_k", "hyq_select_vertical_workspace",
+           "hyq_select_vertical", "hyq_quantize_blocks", "hyq_hybrid_attention_prefill_workspace",
+           "hyq_hybrid_attention_prefill")
+
+
+class HyqError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {status_string(code)} (status {code})")
+
+
+class AttnArgs(ctypes.Structure):
+    """Mirror of ``hyq_attn_args``."""
+    _fields_ = ([("struct_size", ctypes.c_uint32)] +
+                [(n, ctypes.c_int32) for n in ("B", "Hq", "Hkv", "L", "D", "window", "k", "block_tokens",
+                                               "q_format", "k_format", "v_format", "out_dtype", "impl")] +
+                [("softmax_scale", ctypes.c_float)] +
+                [(n, ctypes.c_void_p) for n in ("q", "k_", "v", "q_codes", "k_codes", "v_codes", "q_scales",
+                                                "k_scales", "v_scales", "vl_idx", "out", "lse", "status_word",
+                                                "workspace")] +
+                [("workspace_bytes", ctypes.c_size_t)])
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded shared library; raises if it is missing (no fallback)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: run `python -m paper_2608_27875_b200.build`")
+        L = ctypes.CDLL(LIB_PATH)
+        L.hyq_status_string.restype = ctypes.c_char_p
+        L.hyq_status_string.argtypes = [ctypes.c_int]
+        L.hyq_version.restype = ctypes.c_int
+        L.hyq_paper_k.restype = ctypes.c_int
+        L.hyq_paper_k.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_double]
+        L.hyq_select_vertical_workspace.argtypes = [ctypes.c_int] * 8 + [ctypes.POINTER(ctypes.c_size_t)]
+        L.hyq_select_vertical.argtypes = ([ctypes.c_void_p] * 2 + [ctypes.c_int] * 9 +
+                                          [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p])
+        L.hyq_quantize_blocks.argtypes = ([ctypes.c_void_p] + [ctypes.c_int] * 6 +
+                                          [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p])
+        L.hyq_hybrid_attention_prefill_workspace.argtypes = [ctypes.POINTER(AttnArgs), ctypes.POINTER(ctypes.c_size_t)]
+        L.hyq_hybrid_attention_prefill.argtypes = [ctypes.POINTER(AttnArgs), ctypes.c_void_p]
+        _lib = L
+    return _lib
+
+
+def status_string(code: int) -> str:
+    return lib().hyq_status_string(int(code)).decode()
+
+
+def _check(code: int, where: str):
+    if code != HYQ_OK:
+        raise HyqError(code, where)
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _dev(t: torch.Tensor, dtype, name: str) -> torch.Tensor:
+    if not (t.is_cuda and t.dtype == dtype and t.is_contiguous()):
+        raise ValueError(f"{name}: expected a contiguous CUDA tensor of {dtype}, got {t.dtype} on {t.device}")
+    return t
+
+
+def hyq_paper_k(Lk: int, window: int, ratio: float) -> int:
+    return int(lib().hyq_paper_k(Lk, window, ratio))
+
+
+def hyq_select_vertical_workspace(B, Hq, Hkv, Lq, Lk, D, window, k) -> int:
+    n = ctypes.c_size_t(0)
+    _check(lib().hyq_select_vertical_workspace(B, Hq, Hkv, Lq, Lk, D, window, k, ctypes.byref(n)),
+           "hyq_select_vertical_workspace")
+    return int(n.value)
+
+
+def hyq_select_vertical(q: torch.Tensor, k: torch.Tensor, window: int, k_sel: int, n_tail: int = 0,
+                        workspace: torch.Tensor | None = None, out: torch.Tensor | None = None) -> torch.Tensor:
+    """Algorithm 1.  q [B,Hq,L,D], k [B,Hkv,L,D] bf16 CUDA -> int32 [B,Hq,k_sel] ascending."""
+    _dev(q, torch.bfloat16, "q"), _dev(k, torch.bfloat16, "k")
+    B, Hq, Lq, D = q.shape
+    _, Hkv, Lk, _ = k.shape
+    P = max(0, Lk - window)
+    k_eff = k_sel if P > 0 else 0
+    if out is None:
+        out = torch.empty(B, Hq, k_eff, dtype=torch.int32, device=q.device)
+    need = hyq_select_vertical_workspace(B, Hq, Hkv, Lq, Lk, D, window, k_eff)
+    if workspace is None:
+        workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=q.device)
+    _check(lib().hyq_select_vertical(q.data_ptr(), k.data_ptr(), B, Hq, Hkv, Lq, Lk, D, window, n_tail, k_eff,
+                                     out.data_ptr(), workspace.data_ptr(), workspace.numel(), _stream()),
+           "hyq_select_vertical")
+    return out
+
+
+def code_row_bytes(fmt: int, D: int) -> int:
+    return D // 2 if fmt == FMT_INT4 else D
+
+
+def hyq_quantize_blocks(x: torch.Tensor, fmt: int, block_tokens: int = 64, codes: torch.Tensor | None = None,
+                        scales: torch.Tensor | None = None):
+    """Algorithm 2 Stage 2.  x [B,H,L,D] bf16 CUDA -> (codes uint8 [B,H,L,D or D/2], scales fp32 [B,H,nb])."""
+    _dev(x, torch.bfloat16, "x")
+    B, H, L, D = x.shape
+    nb = -(-L // block_tokens)
+    if codes is None:
+        codes = torch.empty(B, H, L, code_row_bytes(fmt, D), dtype=torch.uint8, device=x.device)
+    if scales is None:
+        scales = torch.empty(B, H, nb, dtype=torch.float32, device=x.device)
+    _check(lib().hyq_quantize_blocks(x.data_ptr(), B, H, L, D, block_tokens, fmt, codes.data_ptr(),
+                                     scales.data_ptr(), _stream()), "hyq_quantize_blocks")
+    return codes, scales
+
+
+def make_attn_args(q, k, v, q_codes, k_codes, v_codes, q_scales, k_scales, v_scales, fmts, vl_idx, window,
+                   out, lse=None, status_word=None, workspace=None, impl=IMPL_AUTO, softmax_scale=0.0,
+                   block_tokens=64) -> AttnArgs:
+    B, Hq, L, D = q.shape
+    a = AttnArgs()
+    a.struct_size = ctypes.sizeof(AttnArgs)
+    a.B, a.Hq, a.Hkv, a.L, a.D = B, Hq, k.shape[1], L, D
+    a.window, a.k, a.block_tokens = window, (0 if vl_idx is None else vl_idx.shape[2]), block_tokens
+    a.q_format, a.k_format, a.v_format = fmts
+    a.out_dtype = 1 if out.dtype == torch.float32 else 0
+    a.impl = impl
+    a.softmax_scale = softmax_scale
+    a.q, a.k_, a.v = q.data_ptr(), k.data_ptr(), v.data_ptr()
+    a.q_codes, a.k_codes, a.v_codes = q_codes.data_ptr(), k_codes.data_ptr(), v_codes.data_ptr()
+    a.q_scales, a.k_scales, a.v_scales = q_scales.data_ptr(), k_scales.data_ptr(), v_scales.data_ptr()
+    a.vl_idx = None if (vl_idx is None or vl_idx.numel() == 0) else vl_idx.data_ptr()
+    a.out = out.data_ptr()
+    a.lse = None if lse is None else lse.data_ptr()
+    a.status_word = None if status_word is None else status_word.data_ptr()
+    a.workspace = None if workspace is None else workspace.data_ptr()
+    a.workspace_bytes = 0 if workspace is None else workspace.numel()
+    return a
+
+
+def hyq_hybrid_attention_prefill_workspace(args: AttnArgs) -> int:
+    n = ctypes.c_size_t(0)
+    _check(lib().hyq_hybrid_attention_prefill_workspace(ctypes.byref(args), ctypes.byref(n)),
+           "hyq_hybrid_attention_prefill_workspace")
+    return int(n.value)
+
+
+def hyq_hybrid_attention_prefill(q, k, v, q_codes, k_codes, v_codes, q_scales, k_scales, v_scales, fmts,
+                                 vl_idx, window: int, out: torch.Tensor | None = None, out_dtype=torch.float32,
+                                 lse: torch.Tensor | None = None, status_word: torch.Tensor | None = None,
+                                 workspace: torch.Tensor | None = None, impl: int = IMPL_AUTO,
+                                 softmax_scale: float = 0.0) -> torch.Tensor:
+    """Eq. 6-7 / Algorithm 2 Stage 3.  Returns out [B,Hq,L,D] (fp32 by default)."""
+    for t, dt, n in ((q, torch.bfloat16, "q"), (k, torch.bfloat16, "k"), (v, torch.bfloat16, "v"),
+                     (q_codes, torch.uint8, "q_codes"), (k_codes, torch.uint8, "k_codes"),
+                     (v_codes, torch.uint8, "v_codes"), (q_scales, torch.float32, "q_scales"),
+                     (k_scales, torch.float32, "k_scales"), (v_scales, torch.float32, "v_scales")):
+        _dev(t, dt, n)
+    if vl_idx is not None:
+        _dev(vl_idx, torch.int32, "vl_idx")
+    if out is None:
+        out = torch.empty(q.shape, dtype=out_dtype, device=q.device)
+    args = make_attn_args(q, k, v, q_codes, k_codes, v_codes, q_scales, k_scales, v_scales, fmts, vl_idx, window,
+                          out, lse, status_word, workspace, impl, softmax_scale)
+    if workspace is None:
+        need = hyq_hybrid_attention_prefill_workspace(args)
+        workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=q.device)
+        args.workspace, args.workspace_bytes = workspace.data_ptr(), workspace.numel()
+    _check(lib().hyq_hybrid_attention_prefill(ctypes.byref(args), _stream()), "hyq_hybrid_attention_prefill")
+    return out
+
+
+def hybrid_prefill(q, k, v, window: int, k_sel: int, fmts=(FMT_INT8, FMT_INT8, FMT_INT8), impl: int = IMPL_AUTO,
+                   out_dtype=torch.float32):
+    """The whole path on device tensors: select -> quantize Q, K, V -> fused attention."""
+    idx = hyq_select_vertical(q, k, window, k_sel)
+    qc, qs = hyq_quantize_blocks(q, fmts[0])
+    kc, ks = hyq_quantize_blocks(k, fmts[1])
+    vc, vs = hyq_quantize_blocks(v, fmts[2])
+    out = hyq_hybrid_attention_prefill(q, k, v, qc, kc, vc, qs, ks, vs, fmts, idx, window, impl=impl,
+                                       out_dtype=out_dtype)
+    return dict(idx=idx, q_codes=qc, k_codes=kc, v_codes=vc, q_scales=qs, k_scales=ks, v_scales=vs, out=out)

@@ -1,0 +1,126 @@
+// C-ABI entry points of the hyq library: argument checks on the host, then kernel launches.
+#include <cmath>
+
+#include "common.cuh"
+
+namespace hyq {
+size_t attn_simt_workspace_bytes(const hyq_attn_args& a);
+int launch_attn_simt(const hyq_attn_args& a, float alpha, cudaStream_t st);
+size_t attn_tc_workspace_bytes(const hyq_attn_args& a);
+int launch_attn_tc(const hyq_attn_args& a, float alpha, cudaStream_t st);
+}  // namespace hyq
+
+using namespace hyq;
+
+extern "C" {
+
+const char* hyq_status_string(int status) {
+    switch (status) {
+        case HYQ_OK: return "ok";
+        case HYQ_ERR_INVALID_ARG: return "invalid argument";
+        case HYQ_ERR_UNSUPPORTED: return "unsupported shape or format";
+        case HYQ_ERR_WORKSPACE: return "workspace too small";
+        case HYQ_ERR_ALIGNMENT: return "pointer not 16-byte aligned";
+        case HYQ_ERR_CUDA: return "CUDA call failed";
+        case HYQ_ERR_TIMEOUT: return "bounded device wait expired";
+        default: return "unknown status";
+    }
+}
+
+int hyq_version(void) { return 1; }
+
+int hyq_paper_k(int Lk, int window, double ratio) {
+    const long P = (Lk - window > 0) ? (long)Lk - window : 0;
+    if (P == 0) return 0;
+    long k = (long)std::ceil((double)P * ratio);
+    if (k < 1) k = 1;
+    if (k > P) k = P;
+    return (int)k;
+}
+
+static int check_select(const void* q, const void* k_, int B, int Hq, int Hkv, int Lq, int Lk, int D, int window,
+                        int n_tail, int k) {
+    if (B <= 0 || Hq <= 0 || Hkv <= 0 || Lq <= 0 || Lk <= 0 || window < 0 || k < 0 || n_tail < 0) return HYQ_ERR_INVALID_ARG;
+    if (Hq % Hkv) return HYQ_ERR_INVALID_ARG;
+    if (D != HYQ_D) return HYQ_ERR_UNSUPPORTED;
+    const long P = (Lk - window > 0) ? (long)Lk - window : 0;
+    if (P == 0 || k == 0) return HYQ_OK;
+    if (k > P || n_tail > Lq) return HYQ_ERR_INVALID_ARG;
+    if (n_tail == 0 && window == 0) return HYQ_ERR_INVALID_ARG;    // mean of zero rows
+    (void)q; (void)k_;
+    return HYQ_OK;
+}
+
+int hyq_select_vertical_workspace(int B, int Hq, int Hkv, int Lq, int Lk, int D, int window, int k, size_t* bytes) {
+    if (!bytes) return HYQ_ERR_INVALID_ARG;
+    const int rc = check_select(nullptr, nullptr, B, Hq, Hkv, Lq, Lk, D, window, 1, k);
+    if (rc != HYQ_OK) return rc;
+    *bytes = select_workspace_bytes(B, Hq, Lk, window);
+    return HYQ_OK;
+}
+
+int hyq_select_vertical(const void* q, const void* k_, int B, int Hq, int Hkv, int Lq, int Lk, int D, int window,
+                        int n_tail, int k, int32_t* idx_out, void* workspace, size_t workspace_bytes, void* stream) {
+    const int rc = check_select(q, k_, B, Hq, Hkv, Lq, Lk, D, window, n_tail, k);
+    if (rc != HYQ_OK) return rc;
+    const long P = (Lk - window > 0) ? (long)Lk - window : 0;
+    if (P == 0 || k == 0) return HYQ_OK;
+    if (!q || !k_ || !idx_out || !workspace) return HYQ_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k_) || !aligned16(workspace) || (reinterpret_cast<uintptr_t>(idx_out) & 3u))
+        return HYQ_ERR_ALIGNMENT;
+    if (workspace_bytes < select_workspace_bytes(B, Hq, Lk, window)) return HYQ_ERR_WORKSPACE;
+    return launch_select(q, k_, B, Hq, Hkv, Lq, Lk, window, n_tail, k, idx_out, workspace, static_cast<cudaStream_t>(stream));
+}
+
+int hyq_quantize_blocks(const void* x, int B, int H, int L, int D, int block_tokens, int format, void* codes_out,
+                        float* scales_out, void* stream) {
+    if (B <= 0 || H <= 0 || L <= 0) return HYQ_ERR_INVALID_ARG;
+    if (!x || !codes_out || !scales_out) return HYQ_ERR_INVALID_ARG;
+    if (D != HYQ_D || block_tokens != HYQ_BLOCK_TOKENS) return HYQ_ERR_UNSUPPORTED;
+    if (format != HYQ_FMT_INT8 && format != HYQ_FMT_FP8_E4M3 && format != HYQ_FMT_INT4) return HYQ_ERR_UNSUPPORTED;
+    if (!aligned16(x) || !aligned16(codes_out) || (reinterpret_cast<uintptr_t>(scales_out) & 3u)) return HYQ_ERR_ALIGNMENT;
+    return launch_quantize(x, (long)B * H, L, format, codes_out, scales_out, static_cast<cudaStream_t>(stream));
+}
+
+static int check_attn(const hyq_attn_args* a, bool need_pointers) {
+    if (!a || a->struct_size != sizeof(hyq_attn_args)) return HYQ_ERR_INVALID_ARG;
+    if (a->B <= 0 || a->Hq <= 0 || a->Hkv <= 0 || a->L <= 0 || a->window < 0 || a->k < 0) return HYQ_ERR_INVALID_ARG;
+    if (a->Hq % a->Hkv || a->k > a->L) return HYQ_ERR_INVALID_ARG;
+    if (a->out_dtype != 0 && a->out_dtype != 1) return HYQ_ERR_INVALID_ARG;
+    if (a->impl < HYQ_IMPL_AUTO || a->impl > HYQ_IMPL_SIMT) return HYQ_ERR_INVALID_ARG;
+    if (a->D != HYQ_D || a->block_tokens != HYQ_BLOCK_TOKENS) return HYQ_ERR_UNSUPPORTED;
+    const bool int8 = a->q_format == HYQ_FMT_INT8 && a->k_format == HYQ_FMT_INT8 && a->v_format == HYQ_FMT_INT8;
+    const bool int4 = a->q_format == HYQ_FMT_INT4 && a->k_format == HYQ_FMT_INT4 && a->v_format == HYQ_FMT_FP8_E4M3;
+    if (!int8 && !int4) return HYQ_ERR_UNSUPPORTED;
+    if (!need_pointers) return HYQ_OK;
+    const void* ptrs[] = {a->q, a->k_, a->v, a->q_codes, a->k_codes, a->v_codes, a->q_scales, a->k_scales, a->v_scales, a->out};
+    for (const void* p : ptrs)
+        if (!p) return HYQ_ERR_INVALID_ARG;
+    if (a->k > 0 && !a->vl_idx) return HYQ_ERR_INVALID_ARG;
+    const void* al[] = {a->q, a->k_, a->v, a->q_codes, a->k_codes, a->v_codes, a->out, a->workspace};
+    for (const void* p : al)
+        if (!aligned16(p)) return HYQ_ERR_ALIGNMENT;
+    return HYQ_OK;
+}
+
+static bool use_simt(const hyq_attn_args* a) { return a->impl == HYQ_IMPL_SIMT; }
+
+int hyq_hybrid_attention_prefill_workspace(const hyq_attn_args* args, size_t* bytes) {
+    if (!bytes) return HYQ_ERR_INVALID_ARG;
+    const int rc = check_attn(args, false);
+    if (rc != HYQ_OK) return rc;
+    *bytes = use_simt(args) ? attn_simt_workspace_bytes(*args) : attn_tc_workspace_bytes(*args);
+    return HYQ_OK;
+}
+
+int hyq_hybrid_attention_prefill(const hyq_attn_args* args, void* stream) {
+    const int rc = check_attn(args, true);
+    if (rc != HYQ_OK) return rc;
+    const size_t need = use_simt(args) ? attn_simt_workspace_bytes(*args) : attn_tc_workspace_bytes(*args);
+    if (need > 0 && (!args->workspace || args->workspace_bytes < need)) return HYQ_ERR_WORKSPACE;
+    const float alpha = args->softmax_scale != 0.0f ? args->softmax_scale : 1.0f / sqrtf((float)args->D);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    return use_simt(args) ? launch_attn_simt(*args, alpha, st) : launch_attn_tc(*args, alpha, st);
+}
+
+}  // extern "C"

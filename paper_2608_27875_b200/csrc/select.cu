@@ -1,0 +1,209 @@
+// Vertical token identification (Algorithm 1): tail-query mean -> GQA-native dot-product
+// scores over the non-window prefix -> exact top-k per query head.
+//
+// Three kernels, all bound by memory traffic:
+//   tail_mean_kernel   qbar[b,h,:] = (1/t) sum of the last t query rows, fp64
+//   vscore_kernel      S[b,h,p] = qbar[b,h,:] . K[b,h/g,p,:], an fp64 fma chain in channel
+//                      order; each K row is read once per KV head and scored for its g query heads
+//   topk_kernel        per (b,h): MSB-first radix select of the k-th largest score on an
+//                      order-preserving 64-bit key, then an ordered compaction that emits the
+//                      selected positions ascending; equal scores go to the lower position.
+// The fp64 chain is what makes the selected set reproducible bit for bit: ranking in lower
+// precision flips pairs whose scores differ by less than its rounding error.
+#include "common.cuh"
+
+namespace hyq {
+
+constexpr int MEAN_GROUPS = 8;       // row groups summed independently, combined in fixed order
+constexpr int SCORE_KEYS = 128;      // keys per CTA in vscore_kernel
+constexpr int SCORE_GC = 4;          // query heads scored per pass over the staged K tile
+constexpr int TOPK_THREADS = 1024;
+
+// -------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(HYQ_D * MEAN_GROUPS)
+tail_mean_kernel(const __nv_bfloat16* __restrict__ q, int Lq, int t, double* __restrict__ qbar) {
+    const long bh = blockIdx.x;
+    const int d = threadIdx.x % HYQ_D, grp = threadIdx.x / HYQ_D;
+    const __nv_bfloat16* base = q + (bh * Lq + (Lq - t)) * (long)HYQ_D + d;
+    // rows are split into MEAN_GROUPS contiguous ranges; every partial sum and their combination
+    // are exact in fp64 for bf16 inputs of bounded exponent spread, so the order does not matter
+    const int per = (t + MEAN_GROUPS - 1) / MEAN_GROUPS;
+    const int r0 = grp * per, r1 = min(t, r0 + per);
+    double s = 0.0;
+#pragma unroll 8
+    for (int r = r0; r < r1; ++r) s += (double)__bfloat162float(base[(long)r * HYQ_D]);
+    __shared__ double part[MEAN_GROUPS][HYQ_D];
+    part[grp][d] = s;
+    __syncthreads();
+    if (grp == 0) {
+        double tot = 0.0;
+#pragma unroll
+        for (int gi = 0; gi < MEAN_GROUPS; ++gi) tot += part[gi][d];
+        qbar[bh * HYQ_D + d] = tot / (double)t;
+    }
+}
+
+// -------------------------------------------------------------------------------------------
+constexpr int KROW_WORDS = HYQ_D / 2 + 1;    // 65 words per staged key row: conflict-free column reads
+
+__global__ void __launch_bounds__(SCORE_KEYS)
+vscore_kernel(const __nv_bfloat16* __restrict__ kmat, const double* __restrict__ qbar, int Hq, int Hkv, int Lk,
+              int P, double* __restrict__ scores) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const int g = Hq / Hkv;
+    uint32_t* ktile = reinterpret_cast<uint32_t*>(smem_raw);                          // [SCORE_KEYS][KROW_WORDS]
+    double* qs = reinterpret_cast<double*>(smem_raw + align_up(SCORE_KEYS * KROW_WORDS * 4, 16));  // [g][D]
+
+    const int p0 = blockIdx.x * SCORE_KEYS;
+    const int kvh = blockIdx.y, b = blockIdx.z;
+    const int n_keys = min(SCORE_KEYS, P - p0);
+
+    // stage the K rows (coalesced 16-byte reads, 4-byte shared stores)
+    const uint4* src = reinterpret_cast<const uint4*>(kmat + (((long)b * Hkv + kvh) * Lk + p0) * HYQ_D);
+    for (int v = threadIdx.x; v < n_keys * (HYQ_D / 8); v += SCORE_KEYS) {
+        const uint4 w = __ldg(src + v);
+        const int row = v / (HYQ_D / 8), c4 = (v % (HYQ_D / 8)) * 4;
+        uint32_t* dst = ktile + row * KROW_WORDS + c4;
+        dst[0] = w.x; dst[1] = w.y; dst[2] = w.z; dst[3] = w.w;
+    }
+    for (int e = threadIdx.x; e < g * HYQ_D; e += SCORE_KEYS)
+        qs[e] = qbar[((long)b * Hq + (long)kvh * g) * HYQ_D + e];
+    __syncthreads();
+    if ((int)threadIdx.x >= n_keys) return;
+
+    const uint32_t* krow = ktile + threadIdx.x * KROW_WORDS;
+    for (int r0 = 0; r0 < g; r0 += SCORE_GC) {
+        double s[SCORE_GC];
+        const double* qr[SCORE_GC];
+#pragma unroll
+        for (int c = 0; c < SCORE_GC; ++c) { s[c] = 0.0; qr[c] = qs + min(r0 + c, g - 1) * HYQ_D; }
+#pragma unroll 4
+        for (int w = 0; w < HYQ_D / 2; ++w) {
+            const uint32_t kw = krow[w];
+            const double k0 = (double)bf16_lo(kw), k1 = (double)bf16_hi(kw);
+#pragma unroll
+            for (int c = 0; c < SCORE_GC; ++c) {
+                s[c] = fma(qr[c][2 * w], k0, s[c]);
+                s[c] = fma(qr[c][2 * w + 1], k1, s[c]);
+            }
+        }
+#pragma unroll
+        for (int c = 0; c < SCORE_GC; ++c)
+            if (r0 + c < g) scores[(((long)b * Hq + (long)kvh * g + r0 + c)) * P + p0 + threadIdx.x] = s[c];
+    }
+}
+
+// -------------------------------------------------------------------------------------------
+// larger score <=> larger key; -0 and +0 map to the same key
+__device__ __forceinline__ unsigned long long order_key(double s) {
+    unsigned long long u = (s == 0.0) ? 0ull : (unsigned long long)__double_as_longlong(s);
+    return (u >> 63) ? ~u : (u | 0x8000000000000000ull);
+}
+
+// exclusive prefix of a 0/1 flag over the CTA, plus the CTA total
+__device__ __forceinline__ int block_exclusive_scan(bool flag, int* warp_tot, int& total) {
+    const unsigned ball = __ballot_sync(0xffffffffu, flag);
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    const int in_warp = __popc(ball & ((1u << lane) - 1u));
+    __syncthreads();                                  // warp_tot is reused by consecutive scans
+    if (lane == 0) warp_tot[wid] = __popc(ball);
+    __syncthreads();
+    int before = 0, tot = 0;
+#pragma unroll
+    for (int w = 0; w < TOPK_THREADS / 32; ++w) {
+        const int c = warp_tot[w];
+        before += (w < wid) ? c : 0;
+        tot += c;
+    }
+    total = tot;
+    return before + in_warp;
+}
+
+__global__ void __launch_bounds__(TOPK_THREADS)
+topk_kernel(const double* __restrict__ scores, int P, int k, int32_t* __restrict__ idx_out) {
+    __shared__ int hist[256];
+    __shared__ int warp_tot[TOPK_THREADS / 32];
+    __shared__ unsigned long long sh_prefix;
+    __shared__ int sh_krem;
+    const double* row = scores + (long)blockIdx.x * P;
+    int32_t* out = idx_out + (long)blockIdx.x * k;
+
+    // radix select: after the loop `prefix` is the key of the k-th largest score and k_rem how
+    // many positions holding exactly that key are still to be taken
+    unsigned long long prefix = 0ull;
+    int k_rem = k;
+    for (int pass = 0; pass < 8; ++pass) {
+        const int shift = 56 - 8 * pass;
+        for (int e = threadIdx.x; e < 256; e += TOPK_THREADS) hist[e] = 0;
+        __syncthreads();
+        for (int p = threadIdx.x; p < P; p += TOPK_THREADS) {
+            const unsigned long long key = order_key(row[p]);
+            if (pass == 0 || (key >> (shift + 8)) == (prefix >> (shift + 8)))
+                atomicAdd(&hist[(int)((key >> shift) & 0xFF)], 1);
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            int cum = 0, d = 255;
+            for (; d > 0; --d) {
+                if (cum + hist[d] >= k_rem) break;
+                cum += hist[d];
+            }
+            sh_prefix = prefix | ((unsigned long long)d << shift);
+            sh_krem = k_rem - cum;
+        }
+        __syncthreads();
+        prefix = sh_prefix;
+        k_rem = sh_krem;
+        __syncthreads();
+    }
+
+    // ordered compaction: positions ascending; among keys equal to the threshold the first k_rem
+    int taken = 0, eq_seen = 0;
+    for (int base = 0; base < P; base += TOPK_THREADS) {
+        const int p = base + threadIdx.x;
+        unsigned long long key = 0ull;
+        const bool live = p < P;
+        if (live) key = order_key(row[p]);
+        const bool eq = live && key == prefix;
+        int eq_tot, sel_tot;
+        const int eq_rank = eq_seen + block_exclusive_scan(eq, warp_tot, eq_tot);
+        const bool sel = live && (key > prefix || (eq && eq_rank < k_rem));
+        const int pos = taken + block_exclusive_scan(sel, warp_tot, sel_tot);
+        if (sel && pos < k) out[pos] = p;
+        eq_seen += eq_tot;
+        taken += sel_tot;
+        if (taken >= k) break;
+    }
+}
+
+// -------------------------------------------------------------------------------------------
+size_t select_workspace_bytes(int B, int Hq, int Lk, int window) {
+    const long P = (Lk - window > 0) ? Lk - window : 0;
+    return align_up((size_t)B * Hq * HYQ_D * sizeof(double), 256) + align_up((size_t)B * Hq * P * sizeof(double), 256);
+}
+
+int launch_select(const void* q, const void* k, int B, int Hq, int Hkv, int Lq, int Lk, int window, int n_tail,
+                  int k_sel, int32_t* idx_out, void* ws, cudaStream_t st) {
+    const int P = (Lk - window > 0) ? Lk - window : 0;
+    const int t = n_tail ? n_tail : (window < Lq ? window : Lq);
+    const int g = Hq / Hkv;
+    double* qbar = static_cast<double*>(ws);
+    double* scores = reinterpret_cast<double*>(static_cast<char*>(ws) + align_up((size_t)B * Hq * HYQ_D * sizeof(double), 256));
+
+    tail_mean_kernel<<<B * Hq, HYQ_D * MEAN_GROUPS, 0, st>>>(static_cast<const __nv_bfloat16*>(q), Lq, t, qbar);
+    if (launch_status() != HYQ_OK) return HYQ_ERR_CUDA;
+
+    const size_t smem = align_up(SCORE_KEYS * KROW_WORDS * 4, 16) + (size_t)g * HYQ_D * sizeof(double);
+    if (smem > 200 * 1024) return HYQ_ERR_UNSUPPORTED;
+    if (smem > 48 * 1024 &&
+        cudaFuncSetAttribute(vscore_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return HYQ_ERR_CUDA;
+    const dim3 grid((P + SCORE_KEYS - 1) / SCORE_KEYS, Hkv, B);
+    vscore_kernel<<<grid, SCORE_KEYS, smem, st>>>(static_cast<const __nv_bfloat16*>(k), qbar, Hq, Hkv, Lk, P, scores);
+    if (launch_status() != HYQ_OK) return HYQ_ERR_CUDA;
+
+    topk_kernel<<<B * Hq, TOPK_THREADS, 0, st>>>(scores, P, k_sel, idx_out);
+    return launch_status();
+}
+
+}  // namespace hyq

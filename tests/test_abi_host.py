@@ -1,0 +1,112 @@
+"""Host-side checks of the C-ABI library that need no GPU: it loads, exports every symbol the
+header declares, and rejects bad arguments before launching anything."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2608_27875_b200 import api, build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build()
+    return api.lib()
+
+
+def test_every_declared_symbol_is_exported(lib):
+    header = open(os.path.join(ROOT, "include", "hyq.h")).read()
+    declared = set(re.findall(r"\b(hyq_[a-z_0-9]+)\s*\(", header))
+    assert declared == set(api.EXPORTS)
+    for name in declared:
+        assert hasattr(lib, name), name
+
+
+def test_status_strings_and_version(lib):
+    assert lib.hyq_version() >= 1
+    seen = {api.status_string(c) for c in range(7)}
+    assert len(seen) == 7 and "ok" in seen
+    assert api.status_string(99) == "unknown status"
+
+
+def test_paper_k_formula(lib):
+    # k = min(P, max(1, ceil(P r))), P = max(0, L - W)   (Algorithm 1)
+    assert api.hyq_paper_k(8192, 512, 0.02) == 154
+    assert api.hyq_paper_k(32768, 1024, 0.02) == 635
+    assert api.hyq_paper_k(131072, 1024, 0.01) == 1301
+    assert api.hyq_paper_k(16384, 512, 0.03) == 477
+    assert api.hyq_paper_k(100, 100, 0.5) == 0          # P = 0
+    assert api.hyq_paper_k(101, 100, 1e-9) == 1         # at least one
+    assert api.hyq_paper_k(110, 100, 1.0) == 10         # at most P
+
+
+def test_select_argument_checks(lib):
+    n = ctypes.c_size_t(0)
+    assert lib.hyq_select_vertical_workspace(1, 4, 2, 256, 256, 128, 64, 8, ctypes.byref(n)) == 0
+    assert n.value >= 4 * 128 * 8 + 4 * 192 * 8
+    assert lib.hyq_select_vertical_workspace(1, 4, 3, 256, 256, 128, 64, 8, ctypes.byref(n)) == 1   # Hq % Hkv
+    assert lib.hyq_select_vertical_workspace(1, 4, 2, 256, 256, 64, 64, 8, ctypes.byref(n)) == 2    # D != 128
+    assert lib.hyq_select_vertical_workspace(1, 4, 2, 256, 256, 128, 64, 193, ctypes.byref(n)) == 1  # k > P
+    # k > P, bad tail, zero window with default tail: rejected before any pointer is touched
+    assert lib.hyq_select_vertical(None, None, 1, 4, 2, 256, 256, 128, 64, 0, 193, None, None, 0, None) == 1
+    assert lib.hyq_select_vertical(None, None, 1, 4, 2, 256, 256, 128, 64, 300, 8, None, None, 0, None) == 1
+    assert lib.hyq_select_vertical(None, None, 1, 4, 2, 256, 256, 128, 0, 0, 8, None, None, 0, None) == 1
+    # empty problems succeed without pointers
+    assert lib.hyq_select_vertical(None, None, 1, 4, 2, 256, 256, 128, 256, 0, 8, None, None, 0, None) == 0
+    assert lib.hyq_select_vertical(None, None, 1, 4, 2, 256, 256, 128, 64, 0, 0, None, None, 0, None) == 0
+    # null pointers with real work
+    assert lib.hyq_select_vertical(None, None, 1, 4, 2, 256, 256, 128, 64, 0, 8, None, None, 0, None) == 1
+    # misaligned pointer / short workspace (fake addresses: checks come before any launch)
+    assert lib.hyq_select_vertical(0x1008, 0x2000, 1, 4, 2, 256, 256, 128, 64, 0, 8, 0x3000, 0x4000, 1 << 30, None) == 4
+    assert lib.hyq_select_vertical(0x1000, 0x2000, 1, 4, 2, 256, 256, 128, 64, 0, 8, 0x3000, 0x4000, 16, None) == 3
+
+
+def test_quantize_argument_checks(lib):
+    assert lib.hyq_quantize_blocks(None, 1, 1, 64, 128, 64, 0, None, None, None) == 1
+    assert lib.hyq_quantize_blocks(0x1000, 1, 1, 64, 64, 64, 0, 0x2000, 0x3000, None) == 2      # D
+    assert lib.hyq_quantize_blocks(0x1000, 1, 1, 64, 128, 32, 0, 0x2000, 0x3000, None) == 2     # block size
+    assert lib.hyq_quantize_blocks(0x1000, 1, 1, 64, 128, 64, 7, 0x2000, 0x3000, None) == 2     # format
+    assert lib.hyq_quantize_blocks(0x1004, 1, 1, 64, 128, 64, 0, 0x2000, 0x3000, None) == 4
+    assert lib.hyq_quantize_blocks(0x1000, 0, 1, 64, 128, 64, 0, 0x2000, 0x3000, None) == 1
+
+
+def _args(**kw):
+    a = api.AttnArgs()
+    a.struct_size = ctypes.sizeof(api.AttnArgs)
+    a.B, a.Hq, a.Hkv, a.L, a.D, a.window, a.k, a.block_tokens = 1, 4, 2, 256, 128, 64, 8, 64
+    a.q_format = a.k_format = a.v_format = 0
+    a.out_dtype, a.impl = 1, api.IMPL_SIMT
+    for f in ("q", "k_", "v", "q_codes", "k_codes", "v_codes", "q_scales", "k_scales", "v_scales", "vl_idx", "out"):
+        setattr(a, f, 0x10000)
+    a.workspace, a.workspace_bytes = 0x20000, 1 << 30
+    for key, val in kw.items():
+        setattr(a, key, val)
+    return a
+
+
+def test_attention_argument_checks(lib):
+    n = ctypes.c_size_t(0)
+    for impl in (api.IMPL_SIMT, api.IMPL_AUTO):
+        assert lib.hyq_hybrid_attention_prefill_workspace(ctypes.byref(_args(impl=impl)), ctypes.byref(n)) == 0
+    call = lambda a: lib.hyq_hybrid_attention_prefill(ctypes.byref(a), None)   # noqa: E731
+    assert call(_args(struct_size=8)) == 1
+    assert call(_args(Hkv=3)) == 1
+    assert call(_args(D=64)) == 2
+    assert call(_args(block_tokens=32)) == 2
+    assert call(_args(q_format=1, k_format=1, v_format=1)) == 2       # FP8 Q/K not built
+    assert call(_args(q_format=2, k_format=2, v_format=0)) == 2       # INT4 with INT8 V not built
+    assert call(_args(out=None)) == 1
+    assert call(_args(vl_idx=None)) == 1                              # k > 0 needs indices
+    assert call(_args(q=0x10008)) == 4
+    assert call(_args(workspace_bytes=0)) == 3
+    assert call(_args(out_dtype=5)) == 1
+
+
+def test_binding_fails_loudly_without_the_library(monkeypatch, tmp_path):
+    monkeypatch.setattr(api, "_lib", None)
+    monkeypatch.setattr(api, "LIB_PATH", str(tmp_path / "missing.so"))
+    with pytest.raises(RuntimeError, match="missing"):
+        api.lib()

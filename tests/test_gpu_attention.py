@@ -1,0 +1,101 @@
+"""GPU parity: hyq_hybrid_attention_prefill against the fp64 oracle (Eq. 6-7), element by element
+at small sizes and on sampled rows at the benchmark sizes.  Tolerance: max-abs 1e-2 and
+sum|err|/sum|ref| 2e-3 on the fp32 output."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from gpu_util import MAX_ABS_TOL, MEAN_REL_TOL, ensure_built, errors, gpu_attention, oracle_quant_all, rand_bf16
+from paper_2608_27875_b200 import api, workloads as wl
+
+pytestmark = pytest.mark.gpu
+INT8 = (wl.FMT_INT8,) * 3
+INT4FP8 = (wl.FMT_INT4, wl.FMT_INT4, wl.FMT_FP8_E4M3)
+IMPLS = [pytest.param(api.IMPL_SIMT, id="simt"), pytest.param(api.IMPL_TCGEN05, id="umma")]
+
+
+def _rand_idx(B, Hq, P, k, seed):
+    rng = np.random.default_rng(seed)
+    return np.stack([np.stack([np.sort(rng.choice(P, k, replace=False)) for _ in range(Hq)])
+                     for _ in range(B)]).astype(np.int32)
+
+
+def _ref(Q, K, V, qz, fmts, idx, window, rows=None, **kw):
+    (qc, qs), (kc, ks), (vc, vs) = qz
+    return oracle.attention_rows(wl.bits(Q), wl.bits(K), wl.bits(V), qc, kc, vc, qs, ks, vs, fmts, idx, window, rows, **kw)
+
+
+def _check(Q, K, V, fmts, idx, window, impl, rows=None):
+    ensure_built()
+    qz = oracle_quant_all(Q, K, V, fmts)
+    got = gpu_attention(Q, K, V, qz, fmts, idx, window, impl).numpy()
+    ref = _ref(Q, K, V, qz, fmts, idx, window, rows)
+    if rows is not None:
+        got = got[:, :, rows]
+    assert np.isfinite(got).all()
+    max_abs, mean_rel = errors(got, ref)
+    assert max_abs <= MAX_ABS_TOL and mean_rel <= MEAN_REL_TOL, (max_abs, mean_rel)
+    return max_abs, mean_rel
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("fmts", [INT8, INT4FP8])
+@pytest.mark.parametrize("B,Hq,Hkv,L,W,k", [
+    (1, 2, 2, 512, 128, 16),      # several tiles
+    (2, 4, 2, 333, 40, 9),        # ragged tail, window not a tile multiple
+    (1, 4, 1, 130, 128, 2),       # window ~ L
+    (1, 2, 2, 200, 0, 12),        # no window: the diagonal itself is low-bit
+    (1, 2, 1, 257, 64, 0),        # no vertical keys
+    (1, 1, 1, 1, 1, 0),           # a single token
+    (1, 2, 2, 64, 200, 0),        # window >= L: exact attention
+    (1, 2, 2, 640, 1, 639),       # every prefix key vertical
+])
+def test_small_shapes_match_oracle(impl, fmts, B, Hq, Hkv, L, W, k):
+    Q, K, V = (rand_bf16((B, h, L, 128), seed=L + n) for n, h in enumerate((Hq, Hkv, Hkv)))
+    P = max(0, L - W)
+    idx = _rand_idx(B, Hq, P, k, seed=L) if k else None
+    _check(Q, K, V, fmts, idx, W, impl)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_vertical_keys_inside_the_window_and_beyond_the_diagonal(impl):
+    """Index sets are free to name keys that a given row sees through its window or not at all."""
+    L, W = 300, 50
+    Q, K, V = (rand_bf16((1, 2, L, 128), seed=40 + n) for n in range(3))
+    idx = np.array([[[0, 1, 2, 100, 101, 249], [5, 64, 127, 128, 200, 249]]], dtype=np.int32)
+    _check(Q, K, V, INT8, idx, W, impl)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_config0_full_output(impl):
+    w = wl.CONFIGS["c0"]
+    Q, K, V = wl.make_inputs(w)
+    idx = oracle.select_vertical(wl.bits(Q), wl.bits(K), w.window, w.k)
+    _check(Q, K, V, w.fmts, idx, w.window, impl)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_bf16_output_is_the_rounded_fp32_output_and_lse(impl):
+    ensure_built()
+    w = wl.CONFIGS["c0"].scaled(L=700)
+    Q, K, V = wl.make_inputs(w)
+    qz = oracle_quant_all(Q, K, V, w.fmts)
+    idx = oracle.select_vertical(wl.bits(Q), wl.bits(K), w.window, w.k)
+    o32, lse = gpu_attention(Q, K, V, qz, w.fmts, idx, w.window, impl, lse=True)
+    o16 = gpu_attention(Q, K, V, qz, w.fmts, idx, w.window, impl, out_dtype=torch.bfloat16)
+    assert torch.equal(o16, o32.to(torch.bfloat16))
+    _, ref_lse = _ref(Q, K, V, qz, w.fmts, idx, w.window, return_lse=True)
+    np.testing.assert_allclose(lse.numpy(), ref_lse, rtol=0, atol=2e-3)
+
+
+@pytest.mark.parametrize("name", ["c1", "c2", "c4"])
+def test_benchmark_configs_on_sampled_rows(name):
+    """Benchmark-size heads, tensor-core kernel, checked on rows the oracle can do one by one."""
+    w = wl.CONFIGS[name]
+    if w.B > 1:
+        w = w.scaled(B=1)
+    Q, K, V = wl.make_inputs(w, heads=[w.Hkv - 1])
+    idx = oracle.select_vertical(wl.bits(Q), wl.bits(K), w.window, w.k)
+    rows = wl.sample_rows(w.L, w.window, n_random=24)
+    _check(Q, K, V, w.fmts, idx, w.window, api.IMPL_TCGEN05, rows)
