@@ -1,0 +1,171 @@
+// Pre-pass of the fused attention: lays out in the caller's workspace what the tensor-core kernel
+// streams with TMA.  All kernels are simple, coalesced and bound by memory traffic.
+//   - vertical-line bitmask per (b, h) over key positions
+//   - gathered vertical-line K rows (bf16) and V rows (fp16) per query head, in ascending position
+//     order (the physical "reorder" of Algorithm 2 Stage 1, done per query head because under
+//     GQA the heads that share a KV head select different keys)
+//   - V in fp16 (full-precision class) and dequantized V^ = code * scale in fp16 (low-bit class):
+//     the P.V products run as fp16 x fp16 MMAs
+//   - INT4 codes widened to one e4m3 byte each (-7..7 are exact in e4m3), so that the score MMA
+//     returns fp32 sums that are exact integers
+#include <cuda_fp16.h>
+#include <cuda_fp8.h>
+
+#include "attn_common.cuh"
+
+namespace hyq {
+
+__global__ void vl_bitmask_kernel(const int32_t* __restrict__ idx, long n_heads, int k, int L, int mask_words,
+                                  uint32_t* __restrict__ bits) {
+    const long e = (long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= n_heads * k) return;
+    const long head = e / k;
+    const int j = idx[e];
+    if (j >= 0 && j < L) atomicOr(&bits[head * mask_words + (j >> 5)], 1u << (j & 31));
+}
+
+// one warp per gathered row: lane copies 4 channels
+__global__ void gather_vl_kernel(const __nv_bfloat16* __restrict__ kmat, const __nv_bfloat16* __restrict__ vmat,
+                                 const int32_t* __restrict__ idx, int Hq, int Hkv, int L, int k, long n_rows,
+                                 __nv_bfloat16* __restrict__ kvl, __half* __restrict__ vvl) {
+    const long row = ((long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (row >= n_rows) return;
+    const long head = row / k;                       // b * Hq + h
+    const int b = (int)(head / Hq), h = (int)(head % Hq), g = Hq / Hkv;
+    int j = idx[row];
+    j = min(max(j, 0), L - 1);
+    const long src = (((long)b * Hkv + h / g) * L + j) * HYQ_D + lane * 4;
+    const uint2 kw = *reinterpret_cast<const uint2*>(kmat + src);
+    const uint2 vw = *reinterpret_cast<const uint2*>(vmat + src);
+    *reinterpret_cast<uint2*>(kvl + row * HYQ_D + lane * 4) = kw;
+    const __half2 v01 = __floats2half2_rn(bf16_lo(vw.x), bf16_hi(vw.x));
+    const __half2 v23 = __floats2half2_rn(bf16_lo(vw.y), bf16_hi(vw.y));
+    uint2 o;
+    o.x = *reinterpret_cast<const uint32_t*>(&v01);
+    o.y = *reinterpret_cast<const uint32_t*>(&v23);
+    *reinterpret_cast<uint2*>(vvl + row * HYQ_D + lane * 4) = o;
+}
+
+// V (bf16) -> fp16 and V^ = code * scale -> fp16; one thread per 8 channels
+template <int V_FMT>
+__global__ void v_to_fp16_kernel(const uint4* __restrict__ v, const uint2* __restrict__ v_codes,
+                                 const float* __restrict__ v_scales, int L, int nb, long n_vec,
+                                 uint4* __restrict__ v16, uint4* __restrict__ vh16) {
+    const long e = (long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= n_vec) return;
+    const long row = e / (HYQ_D / 8);                // global token row over all (b, kv head)
+    const long head = row / L;
+    const int tok = (int)(row - head * L);
+    const float sc = v_scales[head * nb + tok / HYQ_BLOCK_TOKENS];
+    const uint4 w = __ldg(v + e);
+    const uint32_t ws[4] = {w.x, w.y, w.z, w.w};
+    uint32_t o[4], oh[4];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        const __half2 h2 = __floats2half2_rn(bf16_lo(ws[c]), bf16_hi(ws[c]));
+        o[c] = *reinterpret_cast<const uint32_t*>(&h2);
+    }
+    const uint2 cw = __ldg(v_codes + e);
+    const uint32_t cs[2] = {cw.x, cw.y};
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        const uint32_t two = (cs[c >> 1] >> ((c & 1) * 16)) & 0xFFFFu;
+        float f0, f1;
+        if (V_FMT == HYQ_FMT_INT8) {
+            f0 = (float)(int8_t)(two & 0xFF);
+            f1 = (float)(int8_t)(two >> 8);
+        } else {
+            const __half2_raw hr = __nv_cvt_fp8x2_to_halfraw2((__nv_fp8x2_storage_t)two, __NV_E4M3);
+            const float2 ff = __half22float2(__half2(hr));
+            f0 = ff.x;
+            f1 = ff.y;
+        }
+        const __half2 h2 = __floats2half2_rn(f0 * sc, f1 * sc);
+        oh[c] = *reinterpret_cast<const uint32_t*>(&h2);
+    }
+    v16[e] = make_uint4(o[0], o[1], o[2], o[3]);
+    vh16[e] = make_uint4(oh[0], oh[1], oh[2], oh[3]);
+}
+
+// packed INT4 codes -> one e4m3 byte per code; one thread per 8 codes
+__global__ void int4_to_e4m3_kernel(const uint32_t* __restrict__ packed, long n_words, uint2* __restrict__ out) {
+    const long e = (long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= n_words) return;
+    // e4m3 encodings of 0..8 (1 = 0x38, 2 = 0x40, 3 = 0x44, ...); sign goes to bit 7
+    const uint32_t w = __ldg(packed + e);
+    uint32_t o[2] = {0u, 0u};
+#pragma unroll
+    for (int n = 0; n < 8; ++n) {
+        const int v = ((int)(w << (28 - 4 * n))) >> 28;
+        const int a = abs(v);
+        // magnitudes 0..8 -> 0x00,0x38,0x40,0x44,0x48,0x4A,0x4C,0x4E,0x50
+        const uint64_t lut = 0x4E4C4A4844403800ull;
+        uint32_t code = (a == 8) ? 0x50u : (uint32_t)((lut >> (8 * a)) & 0xFF);
+        code |= (v < 0) ? 0x80u : 0u;
+        o[n >> 2] |= code << ((n & 3) * 8);
+    }
+    out[e] = make_uint2(o[0], o[1]);
+}
+
+int launch_vl_bitmask(const int32_t* idx, long n_heads, int k, int L, int mask_words, uint32_t* bits, cudaStream_t st) {
+    if (cudaMemsetAsync(bits, 0, (size_t)n_heads * mask_words * 4, st) != cudaSuccess) return HYQ_ERR_CUDA;
+    if (k <= 0) return HYQ_OK;
+    const long n = n_heads * k;
+    vl_bitmask_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(idx, n_heads, k, L, mask_words, bits);
+    return launch_status();
+}
+
+// ---------------------------------------------------------------------------------------------
+TcWorkspace tc_workspace_layout(const hyq_attn_args& a) {
+    TcWorkspace w{};
+    size_t off = 0;
+    auto take = [&](size_t bytes) { const size_t o = off; off += align_up(bytes, 1024); return o; };
+    const size_t kv_elems = (size_t)a.B * a.Hkv * a.L * HYQ_D, q_elems = (size_t)a.B * a.Hq * a.L * HYQ_D;
+    w.mask_words = (a.L + 31) / 32;
+    w.vl_bits = take((size_t)a.B * a.Hq * w.mask_words * 4);
+    w.v16 = take(kv_elems * 2);
+    w.vh16 = take(kv_elems * 2);
+    w.kvl = take((size_t)a.B * a.Hq * (a.k > 0 ? a.k : 1) * HYQ_D * 2);
+    w.vvl = take((size_t)a.B * a.Hq * (a.k > 0 ? a.k : 1) * HYQ_D * 2);
+    const bool int4 = a.q_format == HYQ_FMT_INT4;
+    w.q8 = int4 ? take(q_elems) : 0;
+    w.k8 = int4 ? take(kv_elems) : 0;
+    w.total = off;
+    return w;
+}
+
+int launch_tc_prepass(const hyq_attn_args& a, const TcWorkspace& w, cudaStream_t st) {
+    char* base = static_cast<char*>(a.workspace);
+    const long n_heads = (long)a.B * a.Hq;
+    uint32_t* bits = reinterpret_cast<uint32_t*>(base + w.vl_bits);
+    if (launch_vl_bitmask(a.vl_idx, n_heads, a.k, a.L, w.mask_words, bits, st) != HYQ_OK) return HYQ_ERR_CUDA;
+    if (a.k > 0) {
+        const long n = n_heads * a.k;
+        gather_vl_kernel<<<(unsigned)((n * 32 + 255) / 256), 256, 0, st>>>(
+            static_cast<const __nv_bfloat16*>(a.k_), static_cast<const __nv_bfloat16*>(a.v), a.vl_idx, a.Hq, a.Hkv, a.L,
+            a.k, n, reinterpret_cast<__nv_bfloat16*>(base + w.kvl), reinterpret_cast<__half*>(base + w.vvl));
+        if (launch_status() != HYQ_OK) return HYQ_ERR_CUDA;
+    }
+    const int nb = (a.L + HYQ_BLOCK_TOKENS - 1) / HYQ_BLOCK_TOKENS;
+    const long n_vec = (long)a.B * a.Hkv * a.L * (HYQ_D / 8);
+    const unsigned vgrid = (unsigned)((n_vec + 255) / 256);
+    if (a.v_format == HYQ_FMT_INT8)
+        v_to_fp16_kernel<HYQ_FMT_INT8><<<vgrid, 256, 0, st>>>(static_cast<const uint4*>(a.v), static_cast<const uint2*>(a.v_codes),
+            a.v_scales, a.L, nb, n_vec, reinterpret_cast<uint4*>(base + w.v16), reinterpret_cast<uint4*>(base + w.vh16));
+    else
+        v_to_fp16_kernel<HYQ_FMT_FP8_E4M3><<<vgrid, 256, 0, st>>>(static_cast<const uint4*>(a.v), static_cast<const uint2*>(a.v_codes),
+            a.v_scales, a.L, nb, n_vec, reinterpret_cast<uint4*>(base + w.v16), reinterpret_cast<uint4*>(base + w.vh16));
+    if (launch_status() != HYQ_OK) return HYQ_ERR_CUDA;
+    if (a.q_format == HYQ_FMT_INT4) {
+        const long qw = (long)a.B * a.Hq * a.L * (HYQ_D / 8), kw = (long)a.B * a.Hkv * a.L * (HYQ_D / 8);
+        int4_to_e4m3_kernel<<<(unsigned)((qw + 255) / 256), 256, 0, st>>>(static_cast<const uint32_t*>(a.q_codes), qw,
+                                                                        reinterpret_cast<uint2*>(base + w.q8));
+        int4_to_e4m3_kernel<<<(unsigned)((kw + 255) / 256), 256, 0, st>>>(static_cast<const uint32_t*>(a.k_codes), kw,
+                                                                        reinterpret_cast<uint2*>(base + w.k8));
+        if (launch_status() != HYQ_OK) return HYQ_ERR_CUDA;
+    }
+    return HYQ_OK;
+}
+
+}  // namespace hyq

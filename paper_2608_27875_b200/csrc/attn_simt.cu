@@ -8,7 +8,7 @@
 // full precision when the key is a vertical-line key of the head or i - j < window.
 #include <cuda_fp8.h>
 
-#include "common.cuh"
+#include "attn_common.cuh"
 
 namespace hyq {
 
@@ -220,16 +220,6 @@ attn_simt_kernel(hyq_attn_args a, float alpha, const uint32_t* __restrict__ vl_b
     }
 }
 
-// one bit per (b, h, key position): set for vertical-line keys
-__global__ void vl_bitmask_kernel(const int32_t* __restrict__ idx, long n_heads, int k, int L, int mask_words,
-                                  uint32_t* __restrict__ bits) {
-    const long e = (long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (e >= n_heads * k) return;
-    const long head = e / k;
-    const int j = idx[e];
-    if (j >= 0 && j < L) atomicOr(&bits[head * mask_words + (j >> 5)], 1u << (j & 31));
-}
-
 size_t attn_simt_workspace_bytes(const hyq_attn_args& a) {
     return align_up((size_t)a.B * a.Hq * ((a.L + 31) / 32) * 4, 256);
 }
@@ -238,12 +228,7 @@ int launch_attn_simt(const hyq_attn_args& a, float alpha, cudaStream_t st) {
     const int mask_words = (a.L + 31) / 32;
     const long n_heads = (long)a.B * a.Hq;
     uint32_t* bits = static_cast<uint32_t*>(a.workspace);
-    if (cudaMemsetAsync(bits, 0, (size_t)n_heads * mask_words * 4, st) != cudaSuccess) return HYQ_ERR_CUDA;
-    if (a.k > 0) {
-        const long n = n_heads * a.k;
-        vl_bitmask_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(a.vl_idx, n_heads, a.k, a.L, mask_words, bits);
-        if (launch_status() != HYQ_OK) return HYQ_ERR_CUDA;
-    }
+    if (launch_vl_bitmask(a.vl_idx, n_heads, a.k, a.L, mask_words, bits, st) != HYQ_OK) return HYQ_ERR_CUDA;
     const dim3 grid((a.L + ST - 1) / ST, a.Hq, a.B);
     const size_t smem = sizeof(SimtSmem);
     auto run = [&](auto kern) -> int {
