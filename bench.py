@@ -1,0 +1,387 @@
+#!/usr/bin/env python
+"""Benchmark of the HyQuant prefill hot path on B200.
+
+One "step" = one pass of the whole path over one synthetic prefill batch:
+hyq_select_vertical -> hyq_quantize_blocks (Q, K, V) -> hyq_hybrid_attention_prefill
+(its pre-pass included).  The metric is effective TFLOPS = 4*D*causal_pairs / time.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config c2] [--impl reference]
+
+Prints ONE JSON line (rank 0).  With --impl reference the CPU oracle is timed instead
+(rank 0 only) on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2608_27875_b200 import workloads as wl  # noqa: E402
+
+METRIC = "hybrid prefill attention effective TFLOPS"
+NOMINAL = {"bf16_tflops": 2250.0, "lowbit_tflops": 4500.0, "hbm_gbs": 8000.0}
+FALLBACK = {"bf16_tflops": 1590.0, "hbm_gbs": 6650.0}
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu
+# capture summarised under profiles/ (bytes per launch of the benchmark workload; None = no capture yet)
+NCU_TRAFFIC_BYTES = {}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"bf16_tflops": float(d["bf16_tflops"]), "hbm_gbs": float(d["hbm_gbs"]), "source": "measured"}
+    return dict(FALLBACK, source="fallback")
+
+
+def fp_pairs(w: wl.Workload, idx: np.ndarray) -> int:
+    """Number of causal pairs scored in full precision: per head W*L - W(W-1)/2 window pairs plus,
+    for each vertical key j, the L - j - W rows that see it outside their window."""
+    L, W = w.L, min(w.window, w.L)
+    win = W * L - W * (W - 1) // 2
+    extra = np.maximum(0, L - idx.astype(np.int64) - W).sum()
+    return int(idx.shape[0] * idx.shape[1] * win + extra)
+
+
+def roofline_seconds(w, n_fp, p16, p8, bw_gbs):
+    n_lq = w.causal_pairs - n_fp
+    t_mma = 4 * w.D * n_fp / (p16 * 1e12) + 4 * w.D * n_lq / (p8 * 1e12)
+    qb, kvb = w.B * w.Hq * w.L * w.D, w.B * w.Hkv * w.L * w.D
+    code = lambda n, f: n // 2 if f == wl.FMT_INT4 else n   # noqa: E731
+    bytes_min = 2 * qb + code(qb, w.q_fmt) + 2 * 2 * kvb + code(kvb, w.k_fmt) + code(kvb, w.v_fmt) + 4 * qb
+    return max(t_mma, bytes_min / (bw_gbs * 1e9)), t_mma, bytes_min
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu, self.proc, self.lines = gpu_index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.gpu)], stdout=subprocess.PIPE, text=True)
+            threading.Thread(target=lambda: self.lines.extend(self.proc.stdout), daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------------------
+def oracle_sample(w: wl.Workload, budget_s: float):
+    """Times the CPU oracle on a bounded sample of the workload: one KV-head group (its g query
+    heads), selection and quantization in full, attention on evenly spaced query rows chosen so
+    that the whole call costs about `budget_s`.  Returns (seconds, pairs, description)."""
+    import oracle
+    w1 = w.scaled(B=1)
+    Q, K, V = wl.make_inputs(w1, heads=[0])
+    qb, kb, vb = wl.bits(Q), wl.bits(K), wl.bits(V)
+    t0 = time.perf_counter()
+    idx = oracle.select_vertical(qb, kb, w.window, w.k)
+    qz = [oracle.quantize(x, f, 64) for x, f in zip((qb, kb, vb), w.fmts)]
+    t_pre = time.perf_counter() - t0
+    (qc, qs), (kc, ks), (vc, vs) = qz
+    g = w.Hq // w.Hkv
+
+    def run(rows):
+        t = time.perf_counter()
+        oracle.attention_rows(qb, kb, vb, qc, kc, vc, qs, ks, vs, w.fmts, idx, w.window, rows)
+        return time.perf_counter() - t
+
+    # grow the row sample until one call costs a good share of the budget (the per-call cost of
+    # materialising the head's fp64 views makes a tiny pilot a poor predictor)
+    n_rows, t_attn = 32, 0.0
+    while True:
+        rows = np.linspace(0, w.L - 1, n_rows).astype(np.int32)
+        t_attn = run(rows)
+        if t_attn >= 0.4 * budget_s or n_rows >= w.L:
+            break
+        n_rows = int(min(w.L, n_rows * min(8.0, max(1.5, 0.8 * budget_s / max(t_attn, 1e-3)))))
+    pairs = g * int((rows.astype(np.int64) + 1).sum())
+    desc = (f"1 of {w.B * w.Hkv} (batch, kv-head) groups ({g} query heads): selection + quantization in full "
+            f"({t_pre:.2f} s), attention on {n_rows} evenly spaced query rows ({pairs:.3g} causal pairs, {t_attn:.2f} s); "
+            f"TFLOPS = 4*D*pairs / attention seconds")
+    return t_attn, pairs, desc, oracle.num_threads()
+
+
+def run_reference(args, w):
+    import oracle
+    oracle.build()
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    n_steps = args.steps + args.warmup
+    budget = max(2.0, min(20.0, 150.0 / n_steps))
+    vals, desc, cores = [], "", 1
+    for s in range(n_steps):
+        t, pairs, desc, cores = oracle_sample(w, budget)
+        if s >= args.warmup:
+            vals.append((t, pairs))
+    t_tot, p_tot = sum(v[0] for v in vals), sum(v[1] for v in vals)
+    tflops = 4 * w.D * p_tot / t_tot / 1e12
+    line = {
+        "impl": "reference", "metric": METRIC, "value": tflops, "unit": "TFLOPS", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t_tot / max(1, args.steps),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "Hq": w.Hq, "Hkv": w.Hkv, "L": w.L, "D": w.D, "window": w.window,
+                   "k": w.k, "formats": list(w.fmts)},
+        "cpu_baseline": {"value": tflops, "unit": "TFLOPS", "cores": cores, "kind": "oracle", "sample": desc},
+        "e2e": {"value": tflops, "unit": "TFLOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------------
+class DevicePath:
+    """The hot path on device tensors with every buffer preallocated (nothing allocates per step)."""
+
+    def __init__(self, w: wl.Workload, dev):
+        from paper_2608_27875_b200 import api
+        self.api, self.w, self.dev = api, w, dev
+        B, Hq, Hkv, L, D = w.B, w.Hq, w.Hkv, w.L, w.D
+        nb = -(-L // 64)
+        e = lambda *s, dt=torch.uint8: torch.empty(*s, dtype=dt, device=dev)   # noqa: E731
+        self.Q, self.K, self.V = e(B, Hq, L, D, dt=torch.bfloat16), e(B, Hkv, L, D, dt=torch.bfloat16), e(B, Hkv, L, D, dt=torch.bfloat16)
+        self.idx = e(B, Hq, w.k, dt=torch.int32)
+        self.sel_ws = e(max(16, api.hyq_select_vertical_workspace(B, Hq, Hkv, L, L, D, w.window, w.k)))
+        self.qc, self.kc, self.vc = (e(B, h, L, api.code_row_bytes(f, D)) for h, f in zip((Hq, Hkv, Hkv), w.fmts))
+        self.qs, self.ks, self.vs = (e(B, h, nb, dt=torch.float32) for h in (Hq, Hkv, Hkv))
+        self.out = e(B, Hq, L, D, dt=torch.float32)
+        self.status = torch.zeros(1, dtype=torch.int32, device=dev)
+        self.args = api.make_attn_args(self.Q, self.K, self.V, self.qc, self.kc, self.vc, self.qs, self.ks, self.vs,
+                                       w.fmts, self.idx, w.window, self.out, status_word=self.status)
+        self.attn_ws = e(max(16, api.hyq_hybrid_attention_prefill_workspace(self.args)))
+        self.args.workspace, self.args.workspace_bytes = self.attn_ws.data_ptr(), self.attn_ws.numel()
+        self.ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+        # events recorded by the library right around the attention kernel proper
+        self.kev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+        for e_ in self.kev:
+            e_.record()
+        self.args.ev_kernel_start, self.args.ev_kernel_stop = (e_.cuda_event for e_ in self.kev)
+        # kernels launched by one step: select 3, quantize 3, attention pre-pass (bitmask, gather,
+        # V to fp16, and 2 INT4 widenings when used) + the attention kernel
+        self.launches_per_step = 3 + 3 + (3 if w.k > 0 else 1) + (2 if w.q_fmt == wl.FMT_INT4 else 0) + 1
+
+    def load(self, Q, K, V):
+        self.Q.copy_(Q, non_blocking=True)
+        self.K.copy_(K, non_blocking=True)
+        self.V.copy_(V, non_blocking=True)
+
+    def step(self, timed: bool = False):
+        api, w = self.api, self.w
+        if timed:
+            self.ev[0].record()
+        api.hyq_select_vertical(self.Q, self.K, w.window, w.k, workspace=self.sel_ws, out=self.idx)
+        if timed:
+            self.ev[1].record()
+        api.hyq_quantize_blocks(self.Q, w.q_fmt, codes=self.qc, scales=self.qs)
+        api.hyq_quantize_blocks(self.K, w.k_fmt, codes=self.kc, scales=self.ks)
+        api.hyq_quantize_blocks(self.V, w.v_fmt, codes=self.vc, scales=self.vs)
+        if timed:
+            self.ev[2].record()
+        import ctypes
+        rc = api.lib().hyq_hybrid_attention_prefill(ctypes.byref(self.args), torch.cuda.current_stream().cuda_stream)
+        if rc:
+            raise api.HyqError(rc, "hyq_hybrid_attention_prefill")
+        if timed:
+            self.ev[3].record()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", default="c2", choices=sorted(wl.CONFIGS))
+    ap.add_argument("--impl", default="hyq", choices=["hyq", "reference"])
+    ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of oracle time for cpu_baseline")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "hyq" else args.warmup
+    w = wl.CONFIGS[args.config]
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    import ctypes
+    from paper_2608_27875_b200 import api, build
+    rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if rank == 0 or world == 1:
+        build.build()
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+        dist.barrier()
+    api.lib()
+
+    # every rank runs its own full batch of the workload (units = (batch, kv head) groups; no collective)
+    wr = w.scaled(seed=w.seed + 17 * rank)
+    Q, K, V = wl.make_inputs(wr)
+    Qp, Kp, Vp = (t.pin_memory() for t in (Q, K, V))
+    path = DevicePath(wr, dev)
+    path.load(Qp, Kp, Vp)
+    torch.cuda.synchronize()
+
+    def barrier():
+        if world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        path.step()
+    barrier()
+    assert int(path.status.item()) == 0, "attention kernel reported a device-side error"
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    parts = np.zeros(3)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    ev0.record()
+    for _ in range(args.steps):
+        path.step(timed=True)
+    ev1.record()
+    barrier()
+    total_ms = ev0.elapsed_time(ev1)
+    # per-part times of the last step (events are re-recorded every step)
+    parts = np.array([path.ev[n].elapsed_time(path.ev[n + 1]) for n in range(3)])
+    clocks = sampler.stop()
+    assert int(path.status.item()) == 0, "attention kernel reported a device-side error"
+
+    # the dominant kernel alone: attention call (pre-pass + kernel) re-timed over the same inputs
+    attn_ms, kern_ms_l = [], []
+    for _ in range(max(3, min(args.steps, 10))):
+        path.ev[0].record()
+        rc = api.lib().hyq_hybrid_attention_prefill(ctypes.byref(path.args), torch.cuda.current_stream().cuda_stream)
+        path.ev[1].record()
+        torch.cuda.synchronize()
+        assert rc == 0
+        attn_ms.append(path.ev[0].elapsed_time(path.ev[1]))
+        kern_ms_l.append(path.kev[0].elapsed_time(path.kev[1]))
+    attn_call_ms = float(np.mean(attn_ms))
+    kern_ms = float(np.mean(kern_ms_l))
+
+    if world > 1:
+        tt = torch.tensor([total_ms], device=dev)
+        torch.distributed.all_reduce(tt, op=torch.distributed.ReduceOp.MAX)
+        total_ms = float(tt.item())
+    ms_per_step = total_ms / args.steps
+    flops = wr.flops
+    value = world * flops / (ms_per_step * 1e-3) / 1e12
+
+    # end to end through host buffers: H2D of Q, K, V, the path, D2H of the output
+    out_host = torch.empty(path.out.shape, dtype=path.out.dtype).pin_memory()
+    e2e_steps = max(2, min(args.steps, 5))
+    e2e_ms = []
+    for n in range(e2e_steps + 1):
+        barrier()
+        t0 = time.perf_counter()
+        path.load(Qp, Kp, Vp)
+        path.step()
+        out_host.copy_(path.out, non_blocking=True)
+        torch.cuda.synchronize()
+        if n > 0:
+            e2e_ms.append((time.perf_counter() - t0) * 1e3)
+    e2e_t = torch.tensor([float(np.mean(e2e_ms))], device=dev)
+    if world > 1:
+        torch.distributed.all_reduce(e2e_t, op=torch.distributed.ReduceOp.MAX)
+    e2e_val = world * flops / (float(e2e_t.item()) * 1e-3) / 1e12
+    h2d = sum(t.numel() * t.element_size() for t in (Q, K, V))
+    d2h = out_host.numel() * out_host.element_size()
+
+    if rank != 0:
+        if world > 1:
+            torch.distributed.destroy_process_group()
+        return
+
+    # roofline of the attention kernel (tensor-bound): mixed-precision time at measured peaks
+    peaks = measured_peaks()
+    idx = path.idx.cpu().numpy()
+    n_fp = fp_pairs(wr, idx)
+    t_roof_meas, _, bytes_min = roofline_seconds(wr, n_fp, peaks["bf16_tflops"], 2 * peaks["bf16_tflops"], peaks["hbm_gbs"])
+    t_roof_nom, _, _ = roofline_seconds(wr, n_fp, NOMINAL["bf16_tflops"], NOMINAL["lowbit_tflops"], NOMINAL["hbm_gbs"])
+    k_ms = kern_ms if kern_ms else attn_call_ms
+    achieved = flops / (k_ms * 1e-3) / 1e12
+    peak_eff = flops / t_roof_meas / 1e12
+    roofline = {
+        "bound": "tensor", "kernel": "attn_tc_kernel", "achieved": achieved, "peak": peak_eff, "unit": "TFLOP/s",
+        "frac": achieved / peak_eff, "traffic": NCU_TRAFFIC_BYTES.get(w.name),
+        "peak_source": f"{peaks['source']}: bf16 {peaks['bf16_tflops']} TFLOP/s for the full-precision pairs, 2x that "
+                       f"(nominal 8-bit:16-bit ratio) for the low-bit pairs; peak = flops / mixed roofline time",
+        "kernel_ms": k_ms, "timed": "kernel only (events inside the library)" if kern_ms else "attention call incl. pre-pass",
+        "fp_pair_share": n_fp / wr.causal_pairs, "roofline_ms_measured": t_roof_meas * 1e3,
+        "roofline_ms_nominal": t_roof_nom * 1e3, "frac_nominal": (t_roof_nom * 1e3) / k_ms,
+        "frac_nominal_whole_step": (t_roof_nom * 1e3) / ms_per_step, "min_bytes": bytes_min,
+    }
+
+    t_cpu, pairs_cpu, desc, cores = oracle_sample(w, args.cpu_budget)
+    cpu = {"value": 4 * w.D * pairs_cpu / t_cpu / 1e12, "unit": "TFLOPS", "cores": cores, "kind": "oracle", "sample": desc}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": "TFLOPS", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "int4 x int4 -> f32 scores (e4m3 MMA), fp16 P.V, bf16 full-precision tiles" if w.q_fmt == wl.FMT_INT4
+                 else "int8 x int8 -> s32 scores, fp16 P.V, bf16 full-precision tiles",
+        "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B * world, "Hq": w.Hq, "Hkv": w.Hkv, "L": w.L, "D": w.D, "window": w.window,
+                   "k": w.k, "formats": list(w.fmts), "l2": "inputs larger than L2 (Q+K+V bf16 = %.0f MB per step)" % (h2d / 1e6),
+                   "step": "select + quantize Q,K,V + fused attention (pre-pass included)", "out_dtype": "fp32"},
+        "step_parts_ms": {"select": float(parts[0]), "quantize": float(parts[1]), "attention_call": float(parts[2])},
+        "attention_only_tflops": flops / (attn_call_ms * 1e-3) / 1e12,
+        "roofline": roofline, "cpu_baseline": cpu,
+        "e2e": {"value": e2e_val, "unit": "TFLOPS", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "ms_per_step": float(e2e_t.item()), "steps": e2e_steps},
+        "gpu_launches": path.launches_per_step * args.steps,
+        "clocks": clocks,
+    }
+    print(json.dumps(line))
+    if world > 1:
+        torch.distributed.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -122,6 +122,7 @@ int hyq_quantize_blocks(const void* x, int B, int H, int L, int D, int block_tok
  *   lse: optional [B,Hq,L] fp32 natural-log-sum-exp of the scaled scores (NULL to skip).
  *   status_word: optional device int32; the kernel stores HYQ_ERR_TIMEOUT there if one of its
  *   bounded waits expires (the output is then undefined); untouched otherwise.
+ *   ev_kernel_start / ev_kernel_stop: optional caller-created CUDA events for profiling (NULL to skip).
  * ------------------------------------------------------------------------------------------- */
 typedef struct {
   uint32_t struct_size;
@@ -146,6 +147,8 @@ typedef struct {
   int32_t* status_word;
   void* workspace;
   size_t workspace_bytes;
+  void* ev_kernel_start;             /* optional cudaEvent_t, recorded on the stream right before ... */
+  void* ev_kernel_stop;              /* ... and right after the attention kernel proper (pre-pass excluded) */
 } hyq_attn_args;
 
 int hyq_hybrid_attention_prefill_workspace(const hyq_attn_args* args, size_t* bytes /* host, out */);

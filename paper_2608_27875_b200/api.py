@@ -36,7 +36,8 @@ class AttnArgs(ctypes.Structure):
                 [(n, ctypes.c_void_p) for n in ("q", "k_", "v", "q_codes", "k_codes", "v_codes", "q_scales",
                                                 "k_scales", "v_scales", "vl_idx", "out", "lse", "status_word",
                                                 "workspace")] +
-                [("workspace_bytes", ctypes.c_size_t)])
+                [("workspace_bytes", ctypes.c_size_t), ("ev_kernel_start", ctypes.c_void_p),
+                 ("ev_kernel_stop", ctypes.c_void_p)])
 
 
 _lib = None

@@ -410,8 +410,11 @@ int launch_attn_tc(const hyq_attn_args& a, float alpha, cudaStream_t st) {
     if (cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM_BYTES) != cudaSuccess)
         return HYQ_ERR_CUDA;
     const dim3 grid((a.L + BM - 1) / BM, a.Hq, a.B);
+    if (a.ev_kernel_start && cudaEventRecord(static_cast<cudaEvent_t>(a.ev_kernel_start), st) != cudaSuccess) return HYQ_ERR_CUDA;
     attn_tc_kernel<<<grid, TC_THREADS, TC_SMEM_BYTES, st>>>(maps, p);
-    return launch_status();
+    if (launch_status() != HYQ_OK) return HYQ_ERR_CUDA;
+    if (a.ev_kernel_stop && cudaEventRecord(static_cast<cudaEvent_t>(a.ev_kernel_stop), st) != cudaSuccess) return HYQ_ERR_CUDA;
+    return HYQ_OK;
 }
 
 }  // namespace hyq
