@@ -1,18 +1,22 @@
 // Fused hybrid-precision causal attention (Eq. 6-7; Algorithm 2, Stage 3) on the 5th-generation
 // tensor cores: TMA -> shared memory -> tcgen05.mma -> TMEM, one online softmax over three passes.
 //
-// One CTA owns 128 query rows of one (b, query head) and walks key tiles of 128:
+// One CTA owns 256 query rows (two 128-row tiles) of one (b, query head) and walks key tiles of 128:
 //   pass A  low-bit keys   j <= i - W, j not vertical   S = Qc.Kc^T  (kind::i8, or kind::f8f6f4 on
 //                                                       INT4 codes widened to e4m3), V^ in fp16
 //   pass B  vertical keys  gathered per query head, ascending, idx <= i - W   S = Q.Kvl^T (bf16)
 //   pass C  window keys    i - W < j <= i                                     S = Q.K^T   (bf16)
-// All passes feed one running (m, l) per row and one fp32 O accumulator in TMEM; P goes back to
-// TMEM as fp16 and is the A operand of the P.V MMA (fp16 x fp16).
+// All passes feed one running (m, l) per row and one fp32 O accumulator per query tile in TMEM; P goes
+// back to TMEM as fp16 (over the S columns it was computed from) and is the A operand of the P.V
+// MMA (fp16 x fp16).  K/V tiles are loaded once and used by both query tiles.
 //
-// Warp roles (192 threads): warps 0-3 softmax (thread r owns query row r = TMEM lane r),
-// warp 4 lane 0 issues TMA loads, warp 5 lane 0 issues MMAs.  S is double-buffered in TMEM so that
-// Q.K^T of tile t+1 runs under the softmax of tile t.  Every mbarrier wait is bounded; when one
-// expires the CTA records HYQ_ERR_TIMEOUT in the status word and unwinds.
+// Warp roles (320 threads): warps 0-3 and 4-7 are the softmax groups of query tile 0 and 1 (thread r
+// owns query row r = TMEM lane r), warp 8 lane 0 issues TMA loads, warp 9 lane 0 issues MMAs in the
+// order P0.V, Q0.K', P1.V, Q1.K' so that each group's softmax runs under the other group's MMAs.
+// The running maximum is only raised when a tile exceeds it by more than 2^8 (the rescale of O is
+// then rare); vertical-line columns inside low-bit tiles are knocked out by storing -inf into
+// their S columns in TMEM.  Every mbarrier wait is bounded; when one expires the CTA records
+// HYQ_ERR_TIMEOUT in the status word and unwinds.
 #include <cuda_fp16.h>
 
 #include "attn_common.cuh"
@@ -21,15 +25,23 @@
 namespace hyq {
 using namespace sm100;
 
-constexpr int BM = 128, BN = 128;
-constexpr int TC_THREADS = 192;
+constexpr int BM = 128, BN = 128, QT = 2;
+constexpr int TC_THREADS = 320;
 constexpr long long WAIT_LIMIT = 4000000000LL;      // SM clocks (~2 s): far beyond any legitimate wait
+constexpr float RESCALE_THRESHOLD = 8.0f;           // log2 units
 
-constexpr uint32_t SQ_OFF = 0, SQC_OFF = 32768, SK_OFF = 49152, SV_OFF = SK_OFF + 2 * 32768;
-constexpr uint32_t TILE_SMEM = SV_OFF + 2 * 32768;                  // 180224
+constexpr uint32_t SQ_OFF = 0, SQC_OFF = QT * 32768, SK_OFF = SQC_OFF + QT * 16384, SV_OFF = SK_OFF + 2 * 32768;
+constexpr uint32_t TILE_SMEM = SV_OFF + 2 * 32768;                  // 229376
 constexpr uint32_t TC_SMEM_BYTES = TILE_SMEM + 1024;                // + slack for 1024-byte alignment
 
-constexpr uint32_t TM_S0 = 0, TM_S1 = 128, TM_O = 256, TM_COLS = 512;
+constexpr uint32_t TM_COLS = 512;
+__device__ __forceinline__ uint32_t tm_s(int q) { return q * 128; }
+__device__ __forceinline__ uint32_t tm_o(int q) { return 256 + q * 128; }
+
+constexpr uint32_t INT_MAGIC = 0x4B400000u;          // float(2^23 + 2^22): int -> float by integer add
+constexpr float INT_MAGIC_F = 12582912.0f;
+constexpr uint32_t KNOCKOUT_F32 = 0xFF800000u;       // -inf
+constexpr uint32_t KNOCKOUT_S32 = KNOCKOUT_F32 - INT_MAGIC;   // becomes -inf after the magic add
 
 struct TcMaps {
     CUtensorMap q, k, qc, kc, v16, vh16, kvl, vvl;
@@ -50,7 +62,12 @@ struct TcParams {
 };
 
 struct TcBarriers {
-    uint64_t q_full, k_full[2], k_free[2], v_full[2], v_free[2], s_full[2], p_full[2], o_done;
+    uint64_t q_full, k_full[2], k_free[2], v_full[2], v_free[2], s_full[QT], p_full[QT], o_done[QT];
+};
+
+// which key tiles a 128-row query tile visits in each pass
+struct QSched {
+    int live, i0, i1, nA, nB, tC0, tC1;
 };
 
 __device__ __forceinline__ float ex2f(float x) {
@@ -69,20 +86,58 @@ __device__ __forceinline__ int count_le(const int32_t* __restrict__ idx, int k, 
     return lo;
 }
 
+// ---- softmax building blocks: one thread = one query row, 32 score columns per TMEM load ---------
+// running maximum of the raw scores of one 32-column chunk (integers stay integers)
+template <bool INT, bool MASKED>
+__device__ __forceinline__ void chunk_max(const uint32_t (&raw)[32], int col0, int lo_eff, unsigned span, float& fmx, int& imx) {
+#pragma unroll
+    for (int e = 0; e < 32; ++e) {
+        const bool valid = !MASKED || (unsigned)(col0 + e - lo_eff) <= span;
+        if (INT) {
+            const int v = (int)raw[e];
+            imx = max(imx, valid ? v : (int)0x80000000);
+        } else {
+            fmx = fmaxf(fmx, valid ? __uint_as_float(raw[e]) : -INFINITY);
+        }
+    }
+}
+
+// p = 2^(raw * c + bias) for one 32-column chunk, packed to fp16 pairs; returns the fp32 row-sum share
+template <bool INT, bool MASKED>
+__device__ __forceinline__ float chunk_exp(const uint32_t (&raw)[32], int col0, int lo_eff, unsigned span, float c, float bias,
+                                           uint32_t (&pk)[16]) {
+    float s0 = 0.0f, s1 = 0.0f;
+#pragma unroll
+    for (int e = 0; e < 32; e += 2) {
+        float y[2];
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const float x = INT ? __uint_as_float(raw[e + u] + INT_MAGIC) : __uint_as_float(raw[e + u]);
+            y[u] = fmaf(x, c, bias);
+            if (MASKED) y[u] = ((unsigned)(col0 + e + u - lo_eff) <= span) ? y[u] : -INFINITY;
+        }
+        const float p0 = ex2f(y[0]), p1 = ex2f(y[1]);
+        s0 += p0;
+        s1 += p1;
+        const __half2 h2 = __floats2half2_rn(p0, p1);
+        pk[e >> 1] = *reinterpret_cast<const uint32_t*>(&h2);
+    }
+    return s0 + s1;
+}
+
 __global__ void __launch_bounds__(TC_THREADS, 1)
 attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     __shared__ TcBarriers bars;
     __shared__ uint32_t tmem_base_s;
-    __shared__ int abort_s, cnt_b_s;
+    __shared__ int abort_s, cnt_b_s[QT];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int qt = gridDim.x - 1 - blockIdx.x;               // longest rows first
+    const int pt = gridDim.x - 1 - blockIdx.x;               // pair of query tiles; longest rows first
     const int h = blockIdx.y, b = blockIdx.z;
     const int L = p.L, W = p.window, g = p.Hq / p.Hkv;
     const int qhead = b * p.Hq + h, kvhead = b * p.Hkv + h / g;
-    const int i0 = qt * BM, i1 = min(i0 + BM - 1, L - 1);
     const int32_t* idx_row = p.vl_idx + (long)qhead * p.k;
 
     if (threadIdx.x == 0) {
@@ -92,15 +147,20 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
             mbar_init(&bars.k_free[s], 1);
             mbar_init(&bars.v_full[s], 1);
             mbar_init(&bars.v_free[s], 1);
-            mbar_init(&bars.s_full[s], 1);
-            mbar_init(&bars.p_full[s], 128);
         }
-        mbar_init(&bars.o_done, 1);
+        for (int q = 0; q < QT; ++q) {
+            mbar_init(&bars.s_full[q], 1);
+            mbar_init(&bars.p_full[q], 128);
+            mbar_init(&bars.o_done[q], 1);
+        }
         fence_mbar_init();
         abort_s = 0;
-        cnt_b_s = (p.k > 0 && i1 - W >= 0) ? count_le(idx_row, p.k, i1 - W) : 0;
     }
-    if (warp == 4) {
+    if (threadIdx.x < QT) {
+        const int i1 = min(pt * QT * BM + threadIdx.x * BM + BM - 1, L - 1);
+        cnt_b_s[threadIdx.x] = (p.k > 0 && i1 - W >= 0) ? count_le(idx_row, p.k, i1 - W) : 0;
+    }
+    if (warp == 8) {
         tmem_alloc(&tmem_base_s, TM_COLS);
         tmem_relinquish();
     }
@@ -109,12 +169,32 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
     tc_fence_after();
     const uint32_t tmem = tmem_base_s;
 
-    // tile schedule: nA low-bit tiles, nB gathered vertical-line tiles, nC window tiles
-    const int nA = (i1 - W >= 0) ? (i1 - W) / BN + 1 : 0;
-    const int nB = (cnt_b_s + BN - 1) / BN;
-    const int tC0 = (W > 0) ? max(0, i0 - W + 1) / BN : 0;
-    const int nC = (W > 0) ? i1 / BN - tC0 + 1 : 0;
+    // per query tile: nA low-bit tiles, nB gathered vertical-line tiles, window tiles tC0..tC1
+    QSched qs[QT];
+#pragma unroll
+    for (int q = 0; q < QT; ++q) {
+        QSched& s = qs[q];
+        s.i0 = (pt * QT + q) * BM;
+        s.live = s.i0 < L;
+        s.i1 = min(s.i0 + BM - 1, L - 1);
+        s.nA = (s.live && s.i1 - W >= 0) ? (s.i1 - W) / BN + 1 : 0;
+        s.nB = s.live ? (cnt_b_s[q] + BN - 1) / BN : 0;
+        s.tC0 = max(0, s.i0 - W + 1) / BN;
+        s.tC1 = (s.live && W > 0) ? s.i1 / BN : -1;
+    }
+    // the CTA walks the union of both lists (tile 1 holds the later rows, so its lists are the longer ones)
+    const int nA = max(qs[0].nA, qs[1].nA), nB = max(qs[0].nB, qs[1].nB);
+    const int tC0 = qs[0].tC0, tC1 = max(qs[0].tC1, qs[1].tC1);
+    const int nC = (W > 0) ? tC1 - tC0 + 1 : 0;
     const int T = nA + nB + nC;
+    auto active = [&](int q, int t) -> bool {
+        const QSched& s = qs[q];
+        if (!s.live) return false;
+        if (t < nA) return t < s.nA;
+        if (t < nA + nB) return t - nA < s.nB;
+        const int tile = tC0 + t - nA - nB;
+        return tile >= s.tC0 && tile <= s.tC1;
+    };
 
     volatile int* abort_flag = &abort_s;
     auto fail = [&]() {
@@ -122,60 +202,65 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
         if (p.status) atomicExch(p.status, HYQ_ERR_TIMEOUT);
     };
 
-    if (warp == 4) {
+    if (warp == 8) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
             prefetch_tmap(&maps.q);
             prefetch_tmap(&maps.k);
-            mbar_arrive_expect_tx(&bars.q_full, 32768 + (nA > 0 ? 16384 : 0));
-            tma_load_3d(smem + SQ_OFF, &maps.q, &bars.q_full, 0, i0, qhead);
-            tma_load_3d(smem + SQ_OFF + 16384, &maps.q, &bars.q_full, 64, i0, qhead);
-            if (nA > 0) tma_load_3d(smem + SQC_OFF, &maps.qc, &bars.q_full, 0, i0, qhead);
+            prefetch_tmap(&maps.kc);
+            prefetch_tmap(&maps.vh16);
+            uint32_t qbytes = 0;
+            for (int q = 0; q < QT; ++q)
+                if (qs[q].live) qbytes += 32768 + (nA > 0 ? 16384 : 0);
+            mbar_arrive_expect_tx(&bars.q_full, qbytes);
+            for (int q = 0; q < QT; ++q) {
+                if (!qs[q].live) continue;
+                tma_load_3d(smem + SQ_OFF + q * 32768, &maps.q, &bars.q_full, 0, qs[q].i0, qhead);
+                tma_load_3d(smem + SQ_OFF + q * 32768 + 16384, &maps.q, &bars.q_full, 64, qs[q].i0, qhead);
+                if (nA > 0) tma_load_3d(smem + SQC_OFF + q * 16384, &maps.qc, &bars.q_full, 0, qs[q].i0, qhead);
+            }
             for (int t = 0; t < T && !*abort_flag; ++t) {
                 const int s = t & 1, u = t >> 1;
                 unsigned char* sk = smem + SK_OFF + s * 32768;
                 unsigned char* sv = smem + SV_OFF + s * 32768;
+                const bool lowbit = t < nA, vl = !lowbit && t < nA + nB;
+                const int row = lowbit ? t * BN : (vl ? (t - nA) * BN : (tC0 + t - nA - nB) * BN);
+                const int hd = vl ? qhead : kvhead;
                 if (u > 0 && !mbar_wait(&bars.k_free[s], (u - 1) & 1, WAIT_LIMIT)) { fail(); break; }
-                if (t < nA) {
+                if (lowbit) {
                     mbar_arrive_expect_tx(&bars.k_full[s], 16384);
-                    tma_load_3d(sk, &maps.kc, &bars.k_full[s], 0, t * BN, kvhead);
+                    tma_load_3d(sk, &maps.kc, &bars.k_full[s], 0, row, hd);
                 } else {
-                    const bool vl = t < nA + nB;
                     const CUtensorMap* m = vl ? &maps.kvl : &maps.k;
-                    const int row = vl ? (t - nA) * BN : (tC0 + t - nA - nB) * BN;
-                    const int hd = vl ? qhead : kvhead;
                     mbar_arrive_expect_tx(&bars.k_full[s], 32768);
                     tma_load_3d(sk, m, &bars.k_full[s], 0, row, hd);
                     tma_load_3d(sk + 16384, m, &bars.k_full[s], 64, row, hd);
                 }
                 if (u > 0 && !mbar_wait(&bars.v_free[s], (u - 1) & 1, WAIT_LIMIT)) { fail(); break; }
                 {
-                    const bool lowbit = t < nA, vl = !lowbit && t < nA + nB;
                     const CUtensorMap* m = lowbit ? &maps.vh16 : (vl ? &maps.vvl : &maps.v16);
-                    const int row = lowbit ? t * BN : (vl ? (t - nA) * BN : (tC0 + t - nA - nB) * BN);
-                    const int hd = vl ? qhead : kvhead;
                     mbar_arrive_expect_tx(&bars.v_full[s], 32768);
                     tma_load_3d(sv, m, &bars.v_full[s], 0, row, hd);
                     tma_load_3d(sv + 16384, m, &bars.v_full[s], 64, row, hd);
                 }
             }
         }
-    } else if (warp == 5) {
+    } else if (warp == 9) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
-            const uint32_t sq = smem_u32(smem + SQ_OFF), sqc = smem_u32(smem + SQC_OFF);
             const uint32_t idesc_lq = p.lowbit_fp8 ? make_idesc(ACC_F32, FMT_E4M3, FMT_E4M3, 0, 0, BM, BN)
                                                    : make_idesc(ACC_S32, FMT_S8, FMT_S8, 0, 0, BM, BN);
             const uint32_t idesc_qk = make_idesc(ACC_F32, FMT_BF16, FMT_BF16, 0, 0, BM, BN);
             const uint32_t idesc_pv = make_idesc(ACC_F32, FMT_F16, FMT_F16, 0, 1, BM, HYQ_D);
+            int n_pv[QT] = {0, 0};
             bool ok = mbar_wait(&bars.q_full, 0, WAIT_LIMIT);
-            auto issue_qk = [&](int t) -> bool {
-                const int s = t & 1;
-                if (!mbar_wait(&bars.k_full[s], (t >> 1) & 1, WAIT_LIMIT)) return false;
-                tc_fence_after();
-                const uint32_t sk = smem_u32(smem + SK_OFF + s * 32768);
-                const uint32_t d = tmem + (s ? TM_S1 : TM_S0);
+            auto wait_k = [&](int t) { return mbar_wait(&bars.k_full[t & 1], (t >> 1) & 1, WAIT_LIMIT); };
+            auto issue_qk = [&](int q, int t) {
+                if (!active(q, t)) return;
+                const uint32_t sk = smem_u32(smem + SK_OFF + (t & 1) * 32768);
+                const uint32_t d = tmem + tm_s(q);
                 if (t < nA) {
+                    const uint32_t sqc = smem_u32(smem + SQC_OFF + q * 16384);
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk) {
                         const uint64_t da = make_smem_desc(sqc + kk * 32, 0, 1024), db = make_smem_desc(sk + kk * 32, 0, 1024);
@@ -183,60 +268,92 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                         else umma_ss_i8(d, da, db, idesc_lq, kk > 0);
                     }
                 } else {
+                    const uint32_t sq = smem_u32(smem + SQ_OFF + q * 32768);
 #pragma unroll
                     for (int kk = 0; kk < 8; ++kk) {
                         const uint32_t off = (kk >> 2) * 16384 + (kk & 3) * 32;
                         umma_ss_f16(d, make_smem_desc(sq + off, 0, 1024), make_smem_desc(sk + off, 0, 1024), idesc_qk, kk > 0);
                     }
                 }
-                umma_commit(&bars.s_full[s]);
-                umma_commit(&bars.k_free[s]);
-                return true;
+                umma_commit(&bars.s_full[q]);
             };
-            if (ok && T > 0) ok = issue_qk(0);
-            for (int t = 0; t < T && ok && !*abort_flag; ++t) {
-                if (t + 1 < T) ok = issue_qk(t + 1);
-                if (!ok) break;
-                const int s = t & 1, par = (t >> 1) & 1;
-                if (!mbar_wait(&bars.p_full[s], par, WAIT_LIMIT) || !mbar_wait(&bars.v_full[s], par, WAIT_LIMIT)) { ok = false; break; }
+            auto issue_pv = [&](int q, int t) -> bool {
+                if (!active(q, t)) return true;
+                if (!mbar_wait(&bars.p_full[q], n_pv[q] & 1, WAIT_LIMIT)) return false;
                 tc_fence_after();
-                const uint32_t sv = smem_u32(smem + SV_OFF + s * 32768);
-                const uint32_t pa = tmem + (s ? TM_S1 : TM_S0);
+                const uint32_t sv = smem_u32(smem + SV_OFF + (t & 1) * 32768);
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk)
-                    umma_ts_f16(tmem + TM_O, pa + kk * 8, make_smem_desc(sv + kk * 2048, 16384, 1024), idesc_pv, (t > 0 || kk > 0));
-                umma_commit(&bars.o_done);
-                umma_commit(&bars.v_free[s]);
+                    umma_ts_f16(tmem + tm_o(q), tmem + tm_s(q) + kk * 8, make_smem_desc(sv + kk * 2048, 16384, 1024), idesc_pv,
+                                (n_pv[q] > 0 || kk > 0));
+                umma_commit(&bars.o_done[q]);
+                ++n_pv[q];
+                return true;
+            };
+            if (ok && T > 0) {
+                ok = wait_k(0);
+                if (ok) {
+                    tc_fence_after();
+                    issue_qk(0, 0);
+                    issue_qk(1, 0);
+                    umma_commit(&bars.k_free[0]);
+                }
+            }
+            for (int t = 0; t < T && ok && !*abort_flag; ++t) {
+                ok = mbar_wait(&bars.v_full[t & 1], (t >> 1) & 1, WAIT_LIMIT);
+                if (!ok) break;
+                ok = issue_pv(0, t);
+                if (!ok) break;
+                if (t + 1 < T) {
+                    ok = wait_k(t + 1);
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_qk(0, t + 1);
+                }
+                ok = issue_pv(1, t);
+                if (!ok) break;
+                umma_commit(&bars.v_free[t & 1]);
+                if (t + 1 < T) {
+                    issue_qk(1, t + 1);
+                    umma_commit(&bars.k_free[(t + 1) & 1]);
+                }
             }
             if (!ok) fail();
         }
     } else {
-        // ------------------------------------------------------------------ softmax warps
-        const int r = threadIdx.x;                      // query row inside the tile = TMEM lane
-        const int i = i0 + r;
+        // ------------------------------------------------------------------ softmax groups
+        const int q = warp >> 2;
+        const QSched sq = qs[q];
+        const int r = threadIdx.x & 127;                // query row inside the tile = TMEM lane
+        const int i = sq.i0 + r;
         const bool row_live = i < L;
-        const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
+        const bool ragged = sq.i0 + BM > L;
+        const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t ts = tmem + tm_s(q) + lane_addr, to = tmem + tm_o(q) + lane_addr;
         const float q_scale = row_live ? __ldg(p.q_scales + (long)qhead * p.nb + i / HYQ_BLOCK_TOKENS) : 0.0f;
-        const int cnt_r = (nB > 0 && row_live && i - W >= 0) ? count_le(idx_row, p.k, i - W) : 0;
+        const int cnt_r = (sq.nB > 0 && row_live && i - W >= 0) ? count_le(idx_row, p.k, i - W) : 0;
         const uint32_t* bits_row = p.vl_bits + (long)qhead * p.mask_words;
-        float m_run = -INFINITY, l_run = 0.0f;
+        float m_used = -INFINITY, l_run = 0.0f;
+        int n_act = 0;
         bool ok = true;
 
         for (int t = 0; t < T; ++t) {
-            const int s = t & 1;
+            if (!active(q, t)) continue;
             // ---- per-tile column bounds and scales
             int lo = 0, hi = -1;
             bool need_range;
             float cs0, cs1;
             uint32_t vlw[4] = {0u, 0u, 0u, 0u};
-            if (t < nA) {
+            const bool lowbit = t < nA;
+            if (lowbit) {
                 const int j0 = t * BN;
                 hi = row_live ? min(i - W - j0, BN - 1) : -1;
-                need_range = (j0 + BN - 1 > i0 - W) || (i0 + BM > L);
+                need_range = (j0 + BN - 1 > sq.i0 - W) || ragged;
                 const float k0 = __ldg(p.k_scales + (long)kvhead * p.nb + min(2 * t, p.nb - 1));
                 const float k1 = __ldg(p.k_scales + (long)kvhead * p.nb + min(2 * t + 1, p.nb - 1));
-                cs0 = q_scale * k0 * p.scale_log2;
-                cs1 = q_scale * k1 * p.scale_log2;
+                // a zero scale (all-zero tile) still has to let -inf pass through the multiply
+                cs0 = fmaxf(q_scale * k0 * p.scale_log2, 1e-37f);
+                cs1 = fmaxf(q_scale * k1 * p.scale_log2, 1e-37f);
 #pragma unroll
                 for (int w = 0; w < 4; ++w)
                     if (j0 / 32 + w < p.mask_words) vlw[w] = __ldg(bits_row + j0 / 32 + w);
@@ -249,91 +366,118 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                 const int j0 = (tC0 + t - nA - nB) * BN;
                 lo = max(0, i - W + 1 - j0);
                 hi = row_live ? min(i - j0, BN - 1) : -1;
-                need_range = (j0 + BN - 1 > i0) || (j0 <= i1 - W) || (i0 + BM > L);
+                need_range = (j0 + BN - 1 > sq.i0) || (j0 <= sq.i1 - W) || ragged;
                 cs0 = cs1 = p.scale_log2;
             }
-            const bool any_vl = (vlw[0] | vlw[1] | vlw[2] | vlw[3]) != 0u;
-            const bool int_scores = (t < nA) && !p.lowbit_fp8;
+            const int lo_eff = (hi >= lo) ? lo : 4096;
+            const unsigned span = (hi >= lo) ? (unsigned)(hi - lo) : 0u;
+            const bool int_scores = lowbit && !p.lowbit_fp8;
 
-            if (!mbar_wait(&bars.s_full[s], (t >> 1) & 1, WAIT_LIMIT)) { ok = false; break; }
+            if (!mbar_wait(&bars.s_full[q], n_act & 1, WAIT_LIMIT)) { ok = false; break; }
             __syncwarp();
             tc_fence_after();
-            const uint32_t ts = tmem + (s ? TM_S1 : TM_S0) + lane_addr;
 
-            float x[BN];
+            // ---- vertical-line keys inside a low-bit tile: their S columns become -inf
+            if ((vlw[0] | vlw[1] | vlw[2] | vlw[3]) != 0u) {
+                const uint32_t knock = int_scores ? KNOCKOUT_S32 : KNOCKOUT_F32;
+#pragma unroll
+                for (int w = 0; w < 4; ++w) {
+                    uint32_t bits = vlw[w];
+                    while (bits) {
+                        const int c = __ffs(bits) - 1;
+                        bits &= bits - 1;
+                        tmem_st1(ts + w * 32 + c, knock);
+                    }
+                }
+                tmem_wait_st();
+            }
+
+            // ---- pass 1: row maximum of the tile
+            float fm0 = -INFINITY, fm1 = -INFINITY;
+            int im0 = (int)0x80000000, im1 = (int)0x80000000;
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 uint32_t raw[32];
                 tmem_ld32(ts + c * 32, raw);
                 tmem_wait_ld();
-                const float cs = (c < 2) ? cs0 : cs1;
-#pragma unroll
-                for (int e = 0; e < 32; ++e)
-                    x[c * 32 + e] = (int_scores ? (float)(int)raw[e] : __uint_as_float(raw[e])) * cs;
+                float& fm = (c < 2) ? fm0 : fm1;
+                int& im = (c < 2) ? im0 : im1;
+                if (int_scores) {
+                    if (need_range) chunk_max<true, true>(raw, c * 32, lo_eff, span, fm, im);
+                    else chunk_max<true, false>(raw, c * 32, lo_eff, span, fm, im);
+                } else {
+                    if (need_range) chunk_max<false, true>(raw, c * 32, lo_eff, span, fm, im);
+                    else chunk_max<false, false>(raw, c * 32, lo_eff, span, fm, im);
+                }
             }
-            if (need_range) {
-#pragma unroll
-                for (int c = 0; c < BN; ++c) x[c] = (c >= lo && c <= hi) ? x[c] : -INFINITY;
+            if (int_scores) {
+                // knocked-out and masked entries sit far below any real score (|score| < 2^22)
+                fm0 = (im0 < -(1 << 23)) ? -INFINITY : (float)im0;
+                fm1 = (im1 < -(1 << 23)) ? -INFINITY : (float)im1;
             }
-            if (any_vl) {
-#pragma unroll
-                for (int c = 0; c < BN; ++c) x[c] = ((vlw[c >> 5] >> (c & 31)) & 1u) ? -INFINITY : x[c];
-            }
-            float mx = x[0];
-#pragma unroll
-            for (int c = 1; c < BN; ++c) mx = fmaxf(mx, x[c]);
-            const float m_new = fmaxf(m_run, mx);
-            const float m_use = (m_new == -INFINITY) ? 0.0f : m_new;
-            const float alpha = (m_new == m_run) ? 1.0f : ex2f(m_run - m_use);   // m_run = -inf -> 0
+            const float mt = fmaxf(fm0 == -INFINITY ? -INFINITY : fm0 * cs0, fm1 == -INFINITY ? -INFINITY : fm1 * cs1);
 
-            // ---- the previous P.V must have landed before O is rescaled and before P[s] is rewritten
-            if (t > 0) {
-                if (!mbar_wait(&bars.o_done, (t - 1) & 1, WAIT_LIMIT)) { ok = false; break; }
+            // ---- raise the running maximum only when the tile exceeds it by the threshold
+            float alpha = 1.0f;
+            const bool raise = mt > m_used + RESCALE_THRESHOLD;      // also true for the first finite maximum
+            if (raise) {
+                alpha = ex2f(m_used - mt);                           // m_used = -inf -> 0
+                l_run *= alpha;
+                m_used = mt;
+            }
+            if (n_act > 0 && __any_sync(0xffffffffu, raise)) {
+                // the previous P.V of this query tile must have landed before O is rescaled
+                if (!mbar_wait(&bars.o_done[q], (n_act - 1) & 1, WAIT_LIMIT)) { ok = false; break; }
                 __syncwarp();
                 tc_fence_after();
-                if (__any_sync(0xffffffffu, alpha != 1.0f)) {
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        uint32_t o[32];
-                        tmem_ld32(tmem + TM_O + lane_addr + c * 32, o);
-                        tmem_wait_ld();
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t o[32];
+                    tmem_ld32(to + c * 32, o);
+                    tmem_wait_ld();
 #pragma unroll
-                        for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-                        tmem_st32(tmem + TM_O + lane_addr + c * 32, o);
-                    }
+                    for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+                    tmem_st32(to + c * 32, o);
                 }
             }
+            const float m_eff = (m_used == -INFINITY) ? 0.0f : m_used;
+            const float b0 = int_scores ? fmaf(-INT_MAGIC_F, cs0, -m_eff) : -m_eff;
+            const float b1 = int_scores ? fmaf(-INT_MAGIC_F, cs1, -m_eff) : -m_eff;
 
+            // ---- pass 2: P = 2^(s - m) as fp16 over the first 64 columns of S; row sum
             float rs = 0.0f;
 #pragma unroll
-            for (int hlf = 0; hlf < 2; ++hlf) {
-                uint32_t pk[32];
-#pragma unroll
-                for (int e = 0; e < 32; ++e) {
-                    const float p0 = ex2f(x[hlf * 64 + 2 * e] - m_use), p1 = ex2f(x[hlf * 64 + 2 * e + 1] - m_use);
-                    rs += p0 + p1;
-                    const __half2 h2 = __floats2half2_rn(p0, p1);
-                    pk[e] = *reinterpret_cast<const uint32_t*>(&h2);
+            for (int c = 0; c < 4; ++c) {
+                uint32_t raw[32], pk[16];
+                tmem_ld32(ts + c * 32, raw);
+                tmem_wait_ld();
+                const float cs = (c < 2) ? cs0 : cs1, bias = (c < 2) ? b0 : b1;
+                if (int_scores) {
+                    rs += need_range ? chunk_exp<true, true>(raw, c * 32, lo_eff, span, cs, bias, pk)
+                                     : chunk_exp<true, false>(raw, c * 32, lo_eff, span, cs, bias, pk);
+                } else {
+                    rs += need_range ? chunk_exp<false, true>(raw, c * 32, lo_eff, span, cs, bias, pk)
+                                     : chunk_exp<false, false>(raw, c * 32, lo_eff, span, cs, bias, pk);
                 }
-                tmem_st32(ts + hlf * 32, pk);
+                tmem_st16(ts + c * 16, pk);
             }
-            l_run = l_run * alpha + rs;
-            m_run = m_new;
+            l_run += rs;
             tmem_wait_st();
             tc_fence_before();
-            mbar_arrive(&bars.p_full[s]);
+            mbar_arrive(&bars.p_full[q]);
+            ++n_act;
         }
 
         // ---- epilogue: O / l
-        if (ok && T > 0) ok = mbar_wait(&bars.o_done, (T - 1) & 1, WAIT_LIMIT);
+        if (ok && n_act > 0) ok = mbar_wait(&bars.o_done[q], (n_act - 1) & 1, WAIT_LIMIT);
         __syncwarp();
-        if (ok) {
+        if (ok && n_act > 0) {
             tc_fence_after();
             const float inv = (l_run > 0.0f) ? 1.0f / l_run : 0.0f;
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 uint32_t o[32];
-                tmem_ld32(tmem + TM_O + lane_addr + c * 32, o);
+                tmem_ld32(to + c * 32, o);
                 tmem_wait_ld();
                 if (row_live) {
                     if (p.out_fp32) {
@@ -358,15 +502,15 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                     }
                 }
             }
-            if (p.lse && row_live) p.lse[(long)qhead * L + i] = (m_run + log2f(l_run)) * 0.6931471805599453f;
-        } else {
+            if (p.lse && row_live) p.lse[(long)qhead * L + i] = (m_used + log2f(l_run)) * 0.6931471805599453f;
+        } else if (!ok) {
             fail();
         }
     }
 
     tc_fence_before();
     __syncthreads();
-    if (warp == 4) {
+    if (warp == 8) {
         __syncwarp();
         tmem_dealloc(tmem, TM_COLS);
     }
@@ -409,7 +553,7 @@ int launch_attn_tc(const hyq_attn_args& a, float alpha, cudaStream_t st) {
 
     if (cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM_BYTES) != cudaSuccess)
         return HYQ_ERR_CUDA;
-    const dim3 grid((a.L + BM - 1) / BM, a.Hq, a.B);
+    const dim3 grid((a.L + QT * BM - 1) / (QT * BM), a.Hq, a.B);
     if (a.ev_kernel_start && cudaEventRecord(static_cast<cudaEvent_t>(a.ev_kernel_start), st) != cudaSuccess) return HYQ_ERR_CUDA;
     attn_tc_kernel<<<grid, TC_THREADS, TC_SMEM_BYTES, st>>>(maps, p);
     if (launch_status() != HYQ_OK) return HYQ_ERR_CUDA;
