@@ -236,10 +236,13 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", default="c2", choices=sorted(wl.CONFIGS))
     ap.add_argument("--impl", default="hyq", choices=["hyq", "reference"])
+    ap.add_argument("--seq", type=int, default=0, help="override the sequence length (profiling on a smaller case)")
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of oracle time for cpu_baseline")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "hyq" else args.warmup
     w = wl.CONFIGS[args.config]
+    if args.seq:
+        w = w.scaled(L=args.seq, k=max(1, w.k * args.seq // w.L), n_plant=max(1, w.n_plant * args.seq // w.L))
     if args.impl == "reference":
         run_reference(args, w)
         return

@@ -59,6 +59,7 @@ struct TcParams {
     void* out;
     float* lse;
     int32_t* status;
+    long long* timing;           // profiling builds only (HYQ_TC_TIMING): per-section cycle sums of CTA 0
 };
 
 struct TcBarriers {
@@ -69,6 +70,14 @@ struct TcBarriers {
 struct QSched {
     int live, i0, i1, nA, nB, tC0, tC1;
 };
+
+#ifdef HYQ_TC_TIMING
+#define TSTAMP(var) const long long var = clock64()
+#define TACC(slot, a, b) tacc[slot] += (b) - (a)
+#else
+#define TSTAMP(var)
+#define TACC(slot, a, b)
+#endif
 
 __device__ __forceinline__ float ex2f(float x) {
     float y;
@@ -86,45 +95,121 @@ __device__ __forceinline__ int count_le(const int32_t* __restrict__ idx, int k, 
     return lo;
 }
 
-// ---- softmax building blocks: one thread = one query row, 32 score columns per TMEM load ---------
-// running maximum of the raw scores of one 32-column chunk (integers stay integers)
-template <bool INT, bool MASKED>
-__device__ __forceinline__ void chunk_max(const uint32_t (&raw)[32], int col0, int lo_eff, unsigned span, float& fmx, int& imx) {
+// ---- softmax building blocks: one thread = one query row of 128 scores held in registers ---------
+// row maximum of the raw scores of one 64-column half (integer scores are compared as integers)
+template <bool INT>
+__device__ __forceinline__ float half_max(const uint32_t (&raw)[BN], int h) {
+    if (INT) {
+        int m0 = (int)raw[h * 64], m1 = (int)raw[h * 64 + 1];
 #pragma unroll
-    for (int e = 0; e < 32; ++e) {
-        const bool valid = !MASKED || (unsigned)(col0 + e - lo_eff) <= span;
-        if (INT) {
-            const int v = (int)raw[e];
-            imx = max(imx, valid ? v : (int)0x80000000);
-        } else {
-            fmx = fmaxf(fmx, valid ? __uint_as_float(raw[e]) : -INFINITY);
+        for (int e = 2; e < 64; e += 2) {
+            m0 = max(m0, (int)raw[h * 64 + e]);
+            m1 = max(m1, (int)raw[h * 64 + e + 1]);
         }
+        const int m = max(m0, m1);
+        return (m < -(1 << 23)) ? -INFINITY : (float)m;      // knocked-out entries sit far below any score
+    } else {
+        float m0 = __uint_as_float(raw[h * 64]), m1 = __uint_as_float(raw[h * 64 + 1]);
+#pragma unroll
+        for (int e = 2; e < 64; e += 2) {
+            m0 = fmaxf(m0, __uint_as_float(raw[h * 64 + e]));
+            m1 = fmaxf(m1, __uint_as_float(raw[h * 64 + e + 1]));
+        }
+        return fmaxf(m0, m1);
     }
 }
 
-// p = 2^(raw * c + bias) for one 32-column chunk, packed to fp16 pairs; returns the fp32 row-sum share
-template <bool INT, bool MASKED>
-__device__ __forceinline__ float chunk_exp(const uint32_t (&raw)[32], int col0, int lo_eff, unsigned span, float c, float bias,
-                                           uint32_t (&pk)[16]) {
-    float s0 = 0.0f, s1 = 0.0f;
+// p = 2^(raw * c + bias) for 32 columns starting at `col0`, packed to fp16 pairs; returns their fp32 sum
+template <bool INT>
+__device__ __forceinline__ float exp_chunk(const uint32_t (&raw)[BN], int col0, float c, float bias, uint32_t (&pk)[16]) {
+    float s0 = 0.0f, s1 = 0.0f, s2 = 0.0f, s3 = 0.0f;
 #pragma unroll
-    for (int e = 0; e < 32; e += 2) {
-        float y[2];
+    for (int e = 0; e < 32; e += 4) {
+        float pv[4];
 #pragma unroll
-        for (int u = 0; u < 2; ++u) {
-            const float x = INT ? __uint_as_float(raw[e + u] + INT_MAGIC) : __uint_as_float(raw[e + u]);
-            y[u] = fmaf(x, c, bias);
-            if (MASKED) y[u] = ((unsigned)(col0 + e + u - lo_eff) <= span) ? y[u] : -INFINITY;
+        for (int u = 0; u < 4; ++u) {
+            const uint32_t rv = raw[col0 + e + u];
+            const float x = INT ? __uint_as_float(rv + INT_MAGIC) : __uint_as_float(rv);
+            pv[u] = ex2f(fmaf(x, c, bias));
         }
-        const float p0 = ex2f(y[0]), p1 = ex2f(y[1]);
-        s0 += p0;
-        s1 += p1;
-        const __half2 h2 = __floats2half2_rn(p0, p1);
-        pk[e >> 1] = *reinterpret_cast<const uint32_t*>(&h2);
+        s0 += pv[0]; s1 += pv[1]; s2 += pv[2]; s3 += pv[3];
+        const __half2 h01 = __floats2half2_rn(pv[0], pv[1]), h23 = __floats2half2_rn(pv[2], pv[3]);
+        pk[e >> 1] = *reinterpret_cast<const uint32_t*>(&h01);
+        pk[(e >> 1) + 1] = *reinterpret_cast<const uint32_t*>(&h23);
     }
-    return s0 + s1;
+    return (s0 + s1) + (s2 + s3);
 }
 
+// one tile of the online softmax for one query row: S (TMEM) -> running (m, l) -> P (TMEM, fp16)
+// returns false when a bounded wait expired
+template <bool INT>
+__device__ __forceinline__ bool softmax_tile(uint32_t ts, uint32_t to, float cs0, float cs1, bool first, uint64_t* o_done,
+                                             uint32_t o_parity, float& m_used, float& l_run) {
+    uint32_t raw[BN];
+    {
+        uint32_t (*r4)[32] = reinterpret_cast<uint32_t (*)[32]>(raw);
+        tmem_ld32(ts, r4[0]);
+        tmem_ld32(ts + 32, r4[1]);
+        tmem_ld32(ts + 64, r4[2]);
+        tmem_ld32(ts + 96, r4[3]);
+        tmem_wait_ld();
+    }
+    const float f0 = half_max<INT>(raw, 0), f1 = half_max<INT>(raw, 1);
+    const float mt = fmaxf(f0 == -INFINITY ? -INFINITY : f0 * cs0, f1 == -INFINITY ? -INFINITY : f1 * cs1);
+
+    // raise the running maximum only when the tile exceeds it by the threshold
+    float alpha = 1.0f;
+    const bool raise = mt > m_used + RESCALE_THRESHOLD;          // also true for the first finite maximum
+    if (raise) {
+        alpha = ex2f(m_used - mt);                               // m_used = -inf -> 0
+        l_run *= alpha;
+        m_used = mt;
+    }
+    if (!first && __any_sync(0xffffffffu, raise)) {
+        // the previous P.V of this query tile must have landed before O is rescaled
+        if (!mbar_wait(o_done, o_parity, WAIT_LIMIT)) return false;
+        __syncwarp();
+        tc_fence_after();
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+            uint32_t o[32];
+            tmem_ld32(to + c * 32, o);
+            tmem_wait_ld();
+#pragma unroll
+            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+            tmem_st32(to + c * 32, o);
+        }
+    }
+    const float m_eff = (m_used == -INFINITY) ? 0.0f : m_used;
+    const float b0 = INT ? fmaf(-INT_MAGIC_F, cs0, -m_eff) : -m_eff;
+    const float b1 = INT ? fmaf(-INT_MAGIC_F, cs1, -m_eff) : -m_eff;
+    float rs = 0.0f;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        uint32_t pk[16];
+        rs += exp_chunk<INT>(raw, c * 32, (c < 2) ? cs0 : cs1, (c < 2) ? b0 : b1, pk);
+        tmem_st16(ts + c * 16, pk);
+    }
+    l_run += rs;
+    tmem_wait_st();
+    return true;
+}
+
+// boundary tiles: columns outside [lo_eff, lo_eff + span] of this row are set to -inf in TMEM
+__device__ __forceinline__ void mask_tile_in_tmem(uint32_t ts, int lo_eff, unsigned span, uint32_t knock) {
+#pragma unroll 1
+    for (int c = 0; c < 4; ++c) {
+        uint32_t raw[32];
+        tmem_ld32(ts + c * 32, raw);
+        tmem_wait_ld();
+#pragma unroll
+        for (int e = 0; e < 32; ++e) raw[e] = ((unsigned)(c * 32 + e - lo_eff) <= span) ? raw[e] : knock;
+        tmem_st32(ts + c * 32, raw);
+    }
+    tmem_wait_st();
+}
+
+template <bool LOWBIT_FP8>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
     extern __shared__ unsigned char smem_raw[];
@@ -248,7 +333,7 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
     } else if (warp == 9) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
-            const uint32_t idesc_lq = p.lowbit_fp8 ? make_idesc(ACC_F32, FMT_E4M3, FMT_E4M3, 0, 0, BM, BN)
+            const uint32_t idesc_lq = LOWBIT_FP8 ? make_idesc(ACC_F32, FMT_E4M3, FMT_E4M3, 0, 0, BM, BN)
                                                    : make_idesc(ACC_S32, FMT_S8, FMT_S8, 0, 0, BM, BN);
             const uint32_t idesc_qk = make_idesc(ACC_F32, FMT_BF16, FMT_BF16, 0, 0, BM, BN);
             const uint32_t idesc_pv = make_idesc(ACC_F32, FMT_F16, FMT_F16, 0, 1, BM, HYQ_D);
@@ -264,7 +349,7 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk) {
                         const uint64_t da = make_smem_desc(sqc + kk * 32, 0, 1024), db = make_smem_desc(sk + kk * 32, 0, 1024);
-                        if (p.lowbit_fp8) umma_ss_f8f6f4(d, da, db, idesc_lq, kk > 0);
+                        if (LOWBIT_FP8) umma_ss_f8f6f4(d, da, db, idesc_lq, kk > 0);
                         else umma_ss_i8(d, da, db, idesc_lq, kk > 0);
                     }
                 } else {
@@ -337,49 +422,67 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
         int n_act = 0;
         bool ok = true;
 
+        // scales and vertical-line bitmask words of a low-bit tile, fetched one tile ahead of their use
+        float nk0 = 0.0f, nk1 = 0.0f;
+        uint32_t nvl[4] = {0u, 0u, 0u, 0u};
+        auto prefetch_tile = [&](int t) {
+            if (t >= nA) return;
+            nk0 = __ldg(p.k_scales + (long)kvhead * p.nb + min(2 * t, p.nb - 1));
+            nk1 = __ldg(p.k_scales + (long)kvhead * p.nb + min(2 * t + 1, p.nb - 1));
+#pragma unroll
+            for (int w = 0; w < 4; ++w) nvl[w] = (t * 4 + w < p.mask_words) ? __ldg(bits_row + t * 4 + w) : 0u;
+        };
+        prefetch_tile(0);
+#ifdef HYQ_TC_TIMING
+        long long tacc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+#endif
+
         for (int t = 0; t < T; ++t) {
+            const float k0 = nk0, k1 = nk1;
+            uint32_t vlw[4] = {nvl[0], nvl[1], nvl[2], nvl[3]};
+            prefetch_tile(t + 1);
             if (!active(q, t)) continue;
             // ---- per-tile column bounds and scales
             int lo = 0, hi = -1;
             bool need_range;
             float cs0, cs1;
-            uint32_t vlw[4] = {0u, 0u, 0u, 0u};
             const bool lowbit = t < nA;
             if (lowbit) {
                 const int j0 = t * BN;
                 hi = row_live ? min(i - W - j0, BN - 1) : -1;
                 need_range = (j0 + BN - 1 > sq.i0 - W) || ragged;
-                const float k0 = __ldg(p.k_scales + (long)kvhead * p.nb + min(2 * t, p.nb - 1));
-                const float k1 = __ldg(p.k_scales + (long)kvhead * p.nb + min(2 * t + 1, p.nb - 1));
                 // a zero scale (all-zero tile) still has to let -inf pass through the multiply
                 cs0 = fmaxf(q_scale * k0 * p.scale_log2, 1e-37f);
                 cs1 = fmaxf(q_scale * k1 * p.scale_log2, 1e-37f);
-#pragma unroll
-                for (int w = 0; w < 4; ++w)
-                    if (j0 / 32 + w < p.mask_words) vlw[w] = __ldg(bits_row + j0 / 32 + w);
             } else if (t < nA + nB) {
                 const int c0 = (t - nA) * BN;
                 hi = min(cnt_r - c0 - 1, BN - 1);
                 need_range = true;
                 cs0 = cs1 = p.scale_log2;
+                vlw[0] = vlw[1] = vlw[2] = vlw[3] = 0u;
             } else {
                 const int j0 = (tC0 + t - nA - nB) * BN;
                 lo = max(0, i - W + 1 - j0);
                 hi = row_live ? min(i - j0, BN - 1) : -1;
                 need_range = (j0 + BN - 1 > sq.i0) || (j0 <= sq.i1 - W) || ragged;
                 cs0 = cs1 = p.scale_log2;
+                vlw[0] = vlw[1] = vlw[2] = vlw[3] = 0u;
             }
             const int lo_eff = (hi >= lo) ? lo : 4096;
             const unsigned span = (hi >= lo) ? (unsigned)(hi - lo) : 0u;
-            const bool int_scores = lowbit && !p.lowbit_fp8;
+            const bool int_scores = lowbit && !LOWBIT_FP8;
 
+            TSTAMP(c0_);
             if (!mbar_wait(&bars.s_full[q], n_act & 1, WAIT_LIMIT)) { ok = false; break; }
             __syncwarp();
             tc_fence_after();
+            TSTAMP(c1_);
 
+            const uint32_t knock = int_scores ? KNOCKOUT_S32 : KNOCKOUT_F32;
+            // ---- boundary tiles: causal / window / validity limits of this row, applied in TMEM
+            if (need_range) mask_tile_in_tmem(ts, lo_eff, span, knock);
             // ---- vertical-line keys inside a low-bit tile: their S columns become -inf
             if ((vlw[0] | vlw[1] | vlw[2] | vlw[3]) != 0u) {
-                const uint32_t knock = int_scores ? KNOCKOUT_S32 : KNOCKOUT_F32;
 #pragma unroll
                 for (int w = 0; w < 4; ++w) {
                     uint32_t bits = vlw[w];
@@ -391,82 +494,24 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                 }
                 tmem_wait_st();
             }
-
-            // ---- pass 1: row maximum of the tile
-            float fm0 = -INFINITY, fm1 = -INFINITY;
-            int im0 = (int)0x80000000, im1 = (int)0x80000000;
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint32_t raw[32];
-                tmem_ld32(ts + c * 32, raw);
-                tmem_wait_ld();
-                float& fm = (c < 2) ? fm0 : fm1;
-                int& im = (c < 2) ? im0 : im1;
-                if (int_scores) {
-                    if (need_range) chunk_max<true, true>(raw, c * 32, lo_eff, span, fm, im);
-                    else chunk_max<true, false>(raw, c * 32, lo_eff, span, fm, im);
-                } else {
-                    if (need_range) chunk_max<false, true>(raw, c * 32, lo_eff, span, fm, im);
-                    else chunk_max<false, false>(raw, c * 32, lo_eff, span, fm, im);
-                }
-            }
-            if (int_scores) {
-                // knocked-out and masked entries sit far below any real score (|score| < 2^22)
-                fm0 = (im0 < -(1 << 23)) ? -INFINITY : (float)im0;
-                fm1 = (im1 < -(1 << 23)) ? -INFINITY : (float)im1;
-            }
-            const float mt = fmaxf(fm0 == -INFINITY ? -INFINITY : fm0 * cs0, fm1 == -INFINITY ? -INFINITY : fm1 * cs1);
-
-            // ---- raise the running maximum only when the tile exceeds it by the threshold
-            float alpha = 1.0f;
-            const bool raise = mt > m_used + RESCALE_THRESHOLD;      // also true for the first finite maximum
-            if (raise) {
-                alpha = ex2f(m_used - mt);                           // m_used = -inf -> 0
-                l_run *= alpha;
-                m_used = mt;
-            }
-            if (n_act > 0 && __any_sync(0xffffffffu, raise)) {
-                // the previous P.V of this query tile must have landed before O is rescaled
-                if (!mbar_wait(&bars.o_done[q], (n_act - 1) & 1, WAIT_LIMIT)) { ok = false; break; }
-                __syncwarp();
-                tc_fence_after();
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t o[32];
-                    tmem_ld32(to + c * 32, o);
-                    tmem_wait_ld();
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-                    tmem_st32(to + c * 32, o);
-                }
-            }
-            const float m_eff = (m_used == -INFINITY) ? 0.0f : m_used;
-            const float b0 = int_scores ? fmaf(-INT_MAGIC_F, cs0, -m_eff) : -m_eff;
-            const float b1 = int_scores ? fmaf(-INT_MAGIC_F, cs1, -m_eff) : -m_eff;
-
-            // ---- pass 2: P = 2^(s - m) as fp16 over the first 64 columns of S; row sum
-            float rs = 0.0f;
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint32_t raw[32], pk[16];
-                tmem_ld32(ts + c * 32, raw);
-                tmem_wait_ld();
-                const float cs = (c < 2) ? cs0 : cs1, bias = (c < 2) ? b0 : b1;
-                if (int_scores) {
-                    rs += need_range ? chunk_exp<true, true>(raw, c * 32, lo_eff, span, cs, bias, pk)
-                                     : chunk_exp<true, false>(raw, c * 32, lo_eff, span, cs, bias, pk);
-                } else {
-                    rs += need_range ? chunk_exp<false, true>(raw, c * 32, lo_eff, span, cs, bias, pk)
-                                     : chunk_exp<false, false>(raw, c * 32, lo_eff, span, cs, bias, pk);
-                }
-                tmem_st16(ts + c * 16, pk);
-            }
-            l_run += rs;
-            tmem_wait_st();
+            TSTAMP(c2_);
+            if (int_scores) ok = softmax_tile<true>(ts, to, cs0, cs1, n_act == 0, &bars.o_done[q], (n_act - 1) & 1, m_used, l_run);
+            else ok = softmax_tile<false>(ts, to, cs0, cs1, n_act == 0, &bars.o_done[q], (n_act - 1) & 1, m_used, l_run);
+            if (!ok) break;
+            TSTAMP(c3_);
             tc_fence_before();
             mbar_arrive(&bars.p_full[q]);
+            TSTAMP(c4_);
+            TACC(0, c0_, c1_); TACC(1, c1_, c2_); TACC(2, c2_, c3_); TACC(3, c3_, c4_);
+#ifdef HYQ_TC_TIMING
+            tacc[4] += 1;
+#endif
             ++n_act;
         }
+#ifdef HYQ_TC_TIMING
+        if (p.timing && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && (threadIdx.x & 127) == 0)
+            for (int e = 0; e < 5; ++e) p.timing[q * 8 + e] = tacc[e];
+#endif
 
         // ---- epilogue: O / l
         if (ok && n_act > 0) ok = mbar_wait(&bars.o_done[q], (n_act - 1) & 1, WAIT_LIMIT);
@@ -517,6 +562,13 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
 }
 
 // ---------------------------------------------------------------------------------------------
+#ifdef HYQ_TC_TIMING
+static __device__ long long g_timing[16];
+extern "C" int hyq_debug_read_timing(long long* host16) {
+    return cudaMemcpyFromSymbol(host16, g_timing, sizeof(long long) * 16) == cudaSuccess ? 0 : 5;
+}
+#endif
+
 size_t attn_tc_workspace_bytes(const hyq_attn_args& a) { return tc_workspace_layout(a).total; }
 
 int launch_attn_tc(const hyq_attn_args& a, float alpha, cudaStream_t st) {
@@ -550,12 +602,17 @@ int launch_attn_tc(const hyq_attn_args& a, float alpha, cudaStream_t st) {
     p.q_scales = a.q_scales; p.k_scales = a.k_scales; p.vl_idx = a.vl_idx;
     p.vl_bits = reinterpret_cast<const uint32_t*>(base + w.vl_bits);
     p.out = a.out; p.lse = a.lse; p.status = a.status_word;
+    p.timing = nullptr;
+#ifdef HYQ_TC_TIMING
+    cudaGetSymbolAddress(reinterpret_cast<void**>(&p.timing), g_timing);
+#endif
 
-    if (cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM_BYTES) != cudaSuccess)
+    auto kern = int4 ? attn_tc_kernel<true> : attn_tc_kernel<false>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM_BYTES) != cudaSuccess)
         return HYQ_ERR_CUDA;
     const dim3 grid((a.L + QT * BM - 1) / (QT * BM), a.Hq, a.B);
     if (a.ev_kernel_start && cudaEventRecord(static_cast<cudaEvent_t>(a.ev_kernel_start), st) != cudaSuccess) return HYQ_ERR_CUDA;
-    attn_tc_kernel<<<grid, TC_THREADS, TC_SMEM_BYTES, st>>>(maps, p);
+    kern<<<grid, TC_THREADS, TC_SMEM_BYTES, st>>>(maps, p);
     if (launch_status() != HYQ_OK) return HYQ_ERR_CUDA;
     if (a.ev_kernel_stop && cudaEventRecord(static_cast<cudaEvent_t>(a.ev_kernel_stop), st) != cudaSuccess) return HYQ_ERR_CUDA;
     return HYQ_OK;
