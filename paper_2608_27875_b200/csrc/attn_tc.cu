@@ -1,22 +1,24 @@
 // Fused hybrid-precision causal attention (Eq. 6-7; Algorithm 2, Stage 3) on the 5th-generation
 // tensor cores: TMA -> shared memory -> tcgen05.mma -> TMEM, one online softmax over three passes.
 //
-// One CTA owns 256 query rows (two 128-row tiles) of one (b, query head) and walks key tiles of 128:
+// One CTA owns 256 query rows (two 128-row tiles) of one (b, query head) and walks key tiles of 64
+// (one quantization block, so one K scale per tile):
 //   pass A  low-bit keys   j <= i - W, j not vertical   S = Qc.Kc^T  (kind::i8, or kind::f8f6f4 on
 //                                                       INT4 codes widened to e4m3), V^ in fp16
 //   pass B  vertical keys  gathered per query head, ascending, idx <= i - W   S = Q.Kvl^T (bf16)
 //   pass C  window keys    i - W < j <= i                                     S = Q.K^T   (bf16)
-// All passes feed one running (m, l) per row and one fp32 O accumulator per query tile in TMEM; P goes
-// back to TMEM as fp16 (over the S columns it was computed from) and is the A operand of the P.V
-// MMA (fp16 x fp16).  K/V tiles are loaded once and used by both query tiles.
+// All passes feed one running (m, l) per row and one fp32 O accumulator per query tile in TMEM.
+// S is double-buffered per query tile (4 x 64 TMEM columns), so Q.K^T of the next tile is done
+// before the softmax of the current one ends; P goes back to TMEM as fp16 over the S columns it
+// was computed from and is the A operand of the P.V MMA (fp16 x fp16).  K/V tiles are loaded once
+// (4-stage rings) and used by both query tiles.
 //
 // Warp roles (320 threads): warps 0-3 and 4-7 are the softmax groups of query tile 0 and 1 (thread r
-// owns query row r = TMEM lane r), warp 8 lane 0 issues TMA loads, warp 9 lane 0 issues MMAs in the
-// order P0.V, Q0.K', P1.V, Q1.K' so that each group's softmax runs under the other group's MMAs.
+// owns query row r = TMEM lane r), warp 8 lane 0 issues TMA loads, warp 9 lane 0 issues MMAs.
 // The running maximum is only raised when a tile exceeds it by more than 2^8 (the rescale of O is
-// then rare); vertical-line columns inside low-bit tiles are knocked out by storing -inf into
-// their S columns in TMEM.  Every mbarrier wait is bounded; when one expires the CTA records
-// HYQ_ERR_TIMEOUT in the status word and unwinds.
+// then rare); integer scores become floats through a magic-number add folded into the exponent
+// FFMA.  Every mbarrier wait is bounded; when one expires the CTA records HYQ_ERR_TIMEOUT in the
+// status word and unwinds.
 #include <cuda_fp16.h>
 
 #include "attn_common.cuh"
@@ -25,17 +27,22 @@
 namespace hyq {
 using namespace sm100;
 
-constexpr int BM = 128, BN = 128, QT = 2;
+constexpr int BM = 128, BN = 64, QT = 2;
+constexpr int NK = 4, NV = 4;                       // K and V ring depths
 constexpr int TC_THREADS = 320;
 constexpr long long WAIT_LIMIT = 4000000000LL;      // SM clocks (~2 s): far beyond any legitimate wait
 constexpr float RESCALE_THRESHOLD = 8.0f;           // log2 units
 
-constexpr uint32_t SQ_OFF = 0, SQC_OFF = QT * 32768, SK_OFF = SQC_OFF + QT * 16384, SV_OFF = SK_OFF + 2 * 32768;
-constexpr uint32_t TILE_SMEM = SV_OFF + 2 * 32768;                  // 229376
+constexpr uint32_t Q_TILE_BYTES = BM * HYQ_D * 2, QC_TILE_BYTES = BM * HYQ_D;        // 32768, 16384
+constexpr uint32_t K_STAGE_BYTES = BN * HYQ_D * 2, V_STAGE_BYTES = BN * HYQ_D * 2;   // 16384, 16384
+constexpr uint32_t KC_TILE_BYTES = BN * HYQ_D;                                       // 8192
+constexpr uint32_t SQ_OFF = 0, SQC_OFF = QT * Q_TILE_BYTES, SK_OFF = SQC_OFF + QT * QC_TILE_BYTES;
+constexpr uint32_t SV_OFF = SK_OFF + NK * K_STAGE_BYTES;
+constexpr uint32_t TILE_SMEM = SV_OFF + NV * V_STAGE_BYTES;         // 229376
 constexpr uint32_t TC_SMEM_BYTES = TILE_SMEM + 1024;                // + slack for 1024-byte alignment
 
 constexpr uint32_t TM_COLS = 512;
-__device__ __forceinline__ uint32_t tm_s(int q) { return q * 128; }
+__device__ __forceinline__ uint32_t tm_s(int q, int buf) { return (q * 2 + buf) * BN; }
 __device__ __forceinline__ uint32_t tm_o(int q) { return 256 + q * 128; }
 
 constexpr uint32_t INT_MAGIC = 0x4B400000u;          // float(2^23 + 2^22): int -> float by integer add
@@ -49,7 +56,6 @@ struct TcMaps {
 
 struct TcParams {
     int B, Hq, Hkv, L, window, k, nb, mask_words;
-    int lowbit_fp8;              // 1: low-bit codes are e4m3 bytes (kind::f8f6f4), 0: int8 (kind::i8)
     int out_fp32;
     float scale_log2;            // softmax_scale * log2(e)
     const float* q_scales;
@@ -59,11 +65,13 @@ struct TcParams {
     void* out;
     float* lse;
     int32_t* status;
-    long long* timing;           // profiling builds only (HYQ_TC_TIMING): per-section cycle sums of CTA 0
+#ifdef HYQ_TC_TIMING
+    long long* timing;
+#endif
 };
 
 struct TcBarriers {
-    uint64_t q_full, k_full[2], k_free[2], v_full[2], v_free[2], s_full[QT], p_full[QT], o_done[QT];
+    uint64_t q_full, k_full[NK], k_free[NK], v_full[NV], v_free[NV], s_full[QT][2], p_full[QT][2], o_done[QT][2];
 };
 
 // which key tiles a 128-row query tile visits in each pass
@@ -74,9 +82,13 @@ struct QSched {
 #ifdef HYQ_TC_TIMING
 #define TSTAMP(var) const long long var = clock64()
 #define TACC(slot, a, b) tacc[slot] += (b) - (a)
+#define TARGS , long long* tacc
+#define TPASS , tacc
 #else
 #define TSTAMP(var)
 #define TACC(slot, a, b)
+#define TARGS
+#define TPASS
 #endif
 
 __device__ __forceinline__ float ex2f(float x) {
@@ -95,27 +107,31 @@ __device__ __forceinline__ int count_le(const int32_t* __restrict__ idx, int k, 
     return lo;
 }
 
-// ---- softmax building blocks: one thread = one query row of 128 scores held in registers ---------
-// row maximum of the raw scores of one 64-column half (integer scores are compared as integers)
+// ---- softmax building blocks: one thread = one query row of 64 scores held in registers -----------
+// row maximum of the raw scores (integer scores are compared as integers)
 template <bool INT>
-__device__ __forceinline__ float half_max(const uint32_t (&raw)[BN], int h) {
+__device__ __forceinline__ float row_max(const uint32_t (&raw)[BN]) {
     if (INT) {
-        int m0 = (int)raw[h * 64], m1 = (int)raw[h * 64 + 1];
+        int m0 = (int)raw[0], m1 = (int)raw[1], m2 = (int)raw[2], m3 = (int)raw[3];
 #pragma unroll
-        for (int e = 2; e < 64; e += 2) {
-            m0 = max(m0, (int)raw[h * 64 + e]);
-            m1 = max(m1, (int)raw[h * 64 + e + 1]);
+        for (int e = 4; e < BN; e += 4) {
+            m0 = max(m0, (int)raw[e]);
+            m1 = max(m1, (int)raw[e + 1]);
+            m2 = max(m2, (int)raw[e + 2]);
+            m3 = max(m3, (int)raw[e + 3]);
         }
-        const int m = max(m0, m1);
+        const int m = max(max(m0, m1), max(m2, m3));
         return (m < -(1 << 23)) ? -INFINITY : (float)m;      // knocked-out entries sit far below any score
     } else {
-        float m0 = __uint_as_float(raw[h * 64]), m1 = __uint_as_float(raw[h * 64 + 1]);
+        float m0 = __uint_as_float(raw[0]), m1 = __uint_as_float(raw[1]), m2 = __uint_as_float(raw[2]), m3 = __uint_as_float(raw[3]);
 #pragma unroll
-        for (int e = 2; e < 64; e += 2) {
-            m0 = fmaxf(m0, __uint_as_float(raw[h * 64 + e]));
-            m1 = fmaxf(m1, __uint_as_float(raw[h * 64 + e + 1]));
+        for (int e = 4; e < BN; e += 4) {
+            m0 = fmaxf(m0, __uint_as_float(raw[e]));
+            m1 = fmaxf(m1, __uint_as_float(raw[e + 1]));
+            m2 = fmaxf(m2, __uint_as_float(raw[e + 2]));
+            m3 = fmaxf(m3, __uint_as_float(raw[e + 3]));
         }
-        return fmaxf(m0, m1);
+        return fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
     }
 }
 
@@ -140,22 +156,33 @@ __device__ __forceinline__ float exp_chunk(const uint32_t (&raw)[BN], int col0, 
     return (s0 + s1) + (s2 + s3);
 }
 
-// one tile of the online softmax for one query row: S (TMEM) -> running (m, l) -> P (TMEM, fp16)
+// one tile of the online softmax for one query row: S (TMEM) -> running (m, l) -> P (TMEM, fp16).
+// vl0 / vl1: bitmask of vertical-line keys among the 64 columns (they are skipped).
 // returns false when a bounded wait expired
 template <bool INT>
-__device__ __forceinline__ bool softmax_tile(uint32_t ts, uint32_t to, float cs0, float cs1, bool first, uint64_t* o_done,
-                                             uint32_t o_parity, float& m_used, float& l_run) {
+__device__ __forceinline__ bool softmax_tile(uint32_t ts, uint32_t to, float cs, uint32_t vl0, uint32_t vl1, bool first,
+                                             uint64_t* o_done, uint32_t o_parity, float& m_used, float& l_run TARGS) {
     uint32_t raw[BN];
+    TSTAMP(s0_);
     {
-        uint32_t (*r4)[32] = reinterpret_cast<uint32_t (*)[32]>(raw);
-        tmem_ld32(ts, r4[0]);
-        tmem_ld32(ts + 32, r4[1]);
-        tmem_ld32(ts + 64, r4[2]);
-        tmem_ld32(ts + 96, r4[3]);
+        uint32_t (*r2)[32] = reinterpret_cast<uint32_t (*)[32]>(raw);
+        tmem_ld32(ts, r2[0]);
+        tmem_ld32(ts + 32, r2[1]);
         tmem_wait_ld();
     }
-    const float f0 = half_max<INT>(raw, 0), f1 = half_max<INT>(raw, 1);
-    const float mt = fmaxf(f0 == -INFINITY ? -INFINITY : f0 * cs0, f1 == -INFINITY ? -INFINITY : f1 * cs1);
+    TSTAMP(s1_);
+    constexpr uint32_t knock = INT ? KNOCKOUT_S32 : KNOCKOUT_F32;
+    if (vl0 != 0u) {                  // uniform over the warp
+#pragma unroll
+        for (int e = 0; e < 32; ++e) raw[e] = ((vl0 >> e) & 1u) ? knock : raw[e];
+    }
+    if (vl1 != 0u) {
+#pragma unroll
+        for (int e = 0; e < 32; ++e) raw[32 + e] = ((vl1 >> e) & 1u) ? knock : raw[32 + e];
+    }
+    TSTAMP(s2_);
+    const float f = row_max<INT>(raw);
+    const float mt = (f == -INFINITY) ? -INFINITY : f * cs;
 
     // raise the running maximum only when the tile exceeds it by the threshold
     float alpha = 1.0f;
@@ -166,7 +193,9 @@ __device__ __forceinline__ bool softmax_tile(uint32_t ts, uint32_t to, float cs0
         m_used = mt;
     }
     if (!first && __any_sync(0xffffffffu, raise)) {
-        // the previous P.V of this query tile must have landed before O is rescaled
+        // the previous P.V of this query tile must have landed before O is rescaled.  P.V number n
+        // signals barrier n & 1; the one before the previous is known to be complete (the S tile
+        // just read was issued after it), so the parity wait cannot alias.
         if (!mbar_wait(o_done, o_parity, WAIT_LIMIT)) return false;
         __syncwarp();
         tc_fence_after();
@@ -180,25 +209,28 @@ __device__ __forceinline__ bool softmax_tile(uint32_t ts, uint32_t to, float cs0
             tmem_st32(to + c * 32, o);
         }
     }
+    TSTAMP(s3_);
     const float m_eff = (m_used == -INFINITY) ? 0.0f : m_used;
-    const float b0 = INT ? fmaf(-INT_MAGIC_F, cs0, -m_eff) : -m_eff;
-    const float b1 = INT ? fmaf(-INT_MAGIC_F, cs1, -m_eff) : -m_eff;
+    const float bias = INT ? fmaf(-INT_MAGIC_F, cs, -m_eff) : -m_eff;
     float rs = 0.0f;
 #pragma unroll
-    for (int c = 0; c < 4; ++c) {
+    for (int c = 0; c < 2; ++c) {
         uint32_t pk[16];
-        rs += exp_chunk<INT>(raw, c * 32, (c < 2) ? cs0 : cs1, (c < 2) ? b0 : b1, pk);
+        rs += exp_chunk<INT>(raw, c * 32, cs, bias, pk);
         tmem_st16(ts + c * 16, pk);
     }
     l_run += rs;
+    TSTAMP(s4_);
     tmem_wait_st();
+    TSTAMP(s5_);
+    TACC(2, s0_, s1_); TACC(3, s1_, s2_); TACC(4, s2_, s3_); TACC(5, s3_, s4_); TACC(6, s4_, s5_);
     return true;
 }
 
 // boundary tiles: columns outside [lo_eff, lo_eff + span] of this row are set to -inf in TMEM
 __device__ __forceinline__ void mask_tile_in_tmem(uint32_t ts, int lo_eff, unsigned span, uint32_t knock) {
 #pragma unroll 1
-    for (int c = 0; c < 4; ++c) {
+    for (int c = 0; c < BN / 32; ++c) {
         uint32_t raw[32];
         tmem_ld32(ts + c * 32, raw);
         tmem_wait_ld();
@@ -209,7 +241,7 @@ __device__ __forceinline__ void mask_tile_in_tmem(uint32_t ts, int lo_eff, unsig
     tmem_wait_st();
 }
 
-template <bool LOWBIT_FP8>
+template <bool LOWBIT_FP8>       // true: low-bit codes are e4m3 bytes (kind::f8f6f4); false: int8 (kind::i8)
 __global__ void __launch_bounds__(TC_THREADS, 1)
 attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
     extern __shared__ unsigned char smem_raw[];
@@ -227,22 +259,26 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
 
     if (threadIdx.x == 0) {
         mbar_init(&bars.q_full, 1);
-        for (int s = 0; s < 2; ++s) {
+        for (int s = 0; s < NK; ++s) {
             mbar_init(&bars.k_full[s], 1);
             mbar_init(&bars.k_free[s], 1);
+        }
+        for (int s = 0; s < NV; ++s) {
             mbar_init(&bars.v_full[s], 1);
             mbar_init(&bars.v_free[s], 1);
         }
         for (int q = 0; q < QT; ++q) {
-            mbar_init(&bars.s_full[q], 1);
-            mbar_init(&bars.p_full[q], 128);
-            mbar_init(&bars.o_done[q], 1);
+            for (int bf = 0; bf < 2; ++bf) {
+                mbar_init(&bars.s_full[q][bf], 1);
+                mbar_init(&bars.p_full[q][bf], 128);
+                mbar_init(&bars.o_done[q][bf], 1);
+            }
         }
         fence_mbar_init();
         abort_s = 0;
     }
     if (threadIdx.x < QT) {
-        const int i1 = min(pt * QT * BM + threadIdx.x * BM + BM - 1, L - 1);
+        const int i1 = min(pt * QT * BM + (int)threadIdx.x * BM + BM - 1, L - 1);
         cnt_b_s[threadIdx.x] = (p.k > 0 && i1 - W >= 0) ? count_le(idx_row, p.k, i1 - W) : 0;
     }
     if (warp == 8) {
@@ -296,37 +332,37 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
             prefetch_tmap(&maps.vh16);
             uint32_t qbytes = 0;
             for (int q = 0; q < QT; ++q)
-                if (qs[q].live) qbytes += 32768 + (nA > 0 ? 16384 : 0);
+                if (qs[q].live) qbytes += Q_TILE_BYTES + (nA > 0 ? QC_TILE_BYTES : 0);
             mbar_arrive_expect_tx(&bars.q_full, qbytes);
             for (int q = 0; q < QT; ++q) {
                 if (!qs[q].live) continue;
-                tma_load_3d(smem + SQ_OFF + q * 32768, &maps.q, &bars.q_full, 0, qs[q].i0, qhead);
-                tma_load_3d(smem + SQ_OFF + q * 32768 + 16384, &maps.q, &bars.q_full, 64, qs[q].i0, qhead);
-                if (nA > 0) tma_load_3d(smem + SQC_OFF + q * 16384, &maps.qc, &bars.q_full, 0, qs[q].i0, qhead);
+                tma_load_3d(smem + SQ_OFF + q * Q_TILE_BYTES, &maps.q, &bars.q_full, 0, qs[q].i0, qhead);
+                tma_load_3d(smem + SQ_OFF + q * Q_TILE_BYTES + Q_TILE_BYTES / 2, &maps.q, &bars.q_full, 64, qs[q].i0, qhead);
+                if (nA > 0) tma_load_3d(smem + SQC_OFF + q * QC_TILE_BYTES, &maps.qc, &bars.q_full, 0, qs[q].i0, qhead);
             }
             for (int t = 0; t < T && !*abort_flag; ++t) {
-                const int s = t & 1, u = t >> 1;
-                unsigned char* sk = smem + SK_OFF + s * 32768;
-                unsigned char* sv = smem + SV_OFF + s * 32768;
+                const int sk_i = t % NK, uk = t / NK, sv_i = t % NV, uv = t / NV;
+                unsigned char* sk = smem + SK_OFF + sk_i * K_STAGE_BYTES;
+                unsigned char* sv = smem + SV_OFF + sv_i * V_STAGE_BYTES;
                 const bool lowbit = t < nA, vl = !lowbit && t < nA + nB;
                 const int row = lowbit ? t * BN : (vl ? (t - nA) * BN : (tC0 + t - nA - nB) * BN);
                 const int hd = vl ? qhead : kvhead;
-                if (u > 0 && !mbar_wait(&bars.k_free[s], (u - 1) & 1, WAIT_LIMIT)) { fail(); break; }
+                if (uk > 0 && !mbar_wait(&bars.k_free[sk_i], (uk - 1) & 1, WAIT_LIMIT)) { fail(); break; }
                 if (lowbit) {
-                    mbar_arrive_expect_tx(&bars.k_full[s], 16384);
-                    tma_load_3d(sk, &maps.kc, &bars.k_full[s], 0, row, hd);
+                    mbar_arrive_expect_tx(&bars.k_full[sk_i], KC_TILE_BYTES);
+                    tma_load_3d(sk, &maps.kc, &bars.k_full[sk_i], 0, row, hd);
                 } else {
                     const CUtensorMap* m = vl ? &maps.kvl : &maps.k;
-                    mbar_arrive_expect_tx(&bars.k_full[s], 32768);
-                    tma_load_3d(sk, m, &bars.k_full[s], 0, row, hd);
-                    tma_load_3d(sk + 16384, m, &bars.k_full[s], 64, row, hd);
+                    mbar_arrive_expect_tx(&bars.k_full[sk_i], K_STAGE_BYTES);
+                    tma_load_3d(sk, m, &bars.k_full[sk_i], 0, row, hd);
+                    tma_load_3d(sk + K_STAGE_BYTES / 2, m, &bars.k_full[sk_i], 64, row, hd);
                 }
-                if (u > 0 && !mbar_wait(&bars.v_free[s], (u - 1) & 1, WAIT_LIMIT)) { fail(); break; }
+                if (uv > 0 && !mbar_wait(&bars.v_free[sv_i], (uv - 1) & 1, WAIT_LIMIT)) { fail(); break; }
                 {
                     const CUtensorMap* m = lowbit ? &maps.vh16 : (vl ? &maps.vvl : &maps.v16);
-                    mbar_arrive_expect_tx(&bars.v_full[s], 32768);
-                    tma_load_3d(sv, m, &bars.v_full[s], 0, row, hd);
-                    tma_load_3d(sv + 16384, m, &bars.v_full[s], 64, row, hd);
+                    mbar_arrive_expect_tx(&bars.v_full[sv_i], V_STAGE_BYTES);
+                    tma_load_3d(sv, m, &bars.v_full[sv_i], 0, row, hd);
+                    tma_load_3d(sv + V_STAGE_BYTES / 2, m, &bars.v_full[sv_i], 64, row, hd);
                 }
             }
         }
@@ -334,18 +370,23 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             const uint32_t idesc_lq = LOWBIT_FP8 ? make_idesc(ACC_F32, FMT_E4M3, FMT_E4M3, 0, 0, BM, BN)
-                                                   : make_idesc(ACC_S32, FMT_S8, FMT_S8, 0, 0, BM, BN);
+                                                 : make_idesc(ACC_S32, FMT_S8, FMT_S8, 0, 0, BM, BN);
             const uint32_t idesc_qk = make_idesc(ACC_F32, FMT_BF16, FMT_BF16, 0, 0, BM, BN);
             const uint32_t idesc_pv = make_idesc(ACC_F32, FMT_F16, FMT_F16, 0, 1, BM, HYQ_D);
-            int n_pv[QT] = {0, 0};
+            int n_qk[QT] = {0, 0}, n_pv[QT] = {0, 0};      // active tiles issued so far, per query tile
             bool ok = mbar_wait(&bars.q_full, 0, WAIT_LIMIT);
-            auto wait_k = [&](int t) { return mbar_wait(&bars.k_full[t & 1], (t >> 1) & 1, WAIT_LIMIT); };
+            auto wait_k = [&](int t) {
+                const bool r = mbar_wait(&bars.k_full[t % NK], (t / NK) & 1, WAIT_LIMIT);
+                tc_fence_after();
+                return r;
+            };
             auto issue_qk = [&](int q, int t) {
                 if (!active(q, t)) return;
-                const uint32_t sk = smem_u32(smem + SK_OFF + (t & 1) * 32768);
-                const uint32_t d = tmem + tm_s(q);
+                const uint32_t sk = smem_u32(smem + SK_OFF + (t % NK) * K_STAGE_BYTES);
+                const int buf = n_qk[q] & 1;
+                const uint32_t d = tmem + tm_s(q, buf);
                 if (t < nA) {
-                    const uint32_t sqc = smem_u32(smem + SQC_OFF + q * 16384);
+                    const uint32_t sqc = smem_u32(smem + SQC_OFF + q * QC_TILE_BYTES);
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk) {
                         const uint64_t da = make_smem_desc(sqc + kk * 32, 0, 1024), db = make_smem_desc(sk + kk * 32, 0, 1024);
@@ -353,56 +394,76 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                         else umma_ss_i8(d, da, db, idesc_lq, kk > 0);
                     }
                 } else {
-                    const uint32_t sq = smem_u32(smem + SQ_OFF + q * 32768);
+                    const uint32_t sq = smem_u32(smem + SQ_OFF + q * Q_TILE_BYTES);
 #pragma unroll
                     for (int kk = 0; kk < 8; ++kk) {
-                        const uint32_t off = (kk >> 2) * 16384 + (kk & 3) * 32;
-                        umma_ss_f16(d, make_smem_desc(sq + off, 0, 1024), make_smem_desc(sk + off, 0, 1024), idesc_qk, kk > 0);
+                        const uint32_t offq = (kk >> 2) * (Q_TILE_BYTES / 2) + (kk & 3) * 32;
+                        const uint32_t offk = (kk >> 2) * (K_STAGE_BYTES / 2) + (kk & 3) * 32;
+                        umma_ss_f16(d, make_smem_desc(sq + offq, 0, 1024), make_smem_desc(sk + offk, 0, 1024), idesc_qk, kk > 0);
                     }
                 }
-                umma_commit(&bars.s_full[q]);
+                umma_commit(&bars.s_full[q][buf]);
+                ++n_qk[q];
             };
             auto issue_pv = [&](int q, int t) -> bool {
                 if (!active(q, t)) return true;
-                if (!mbar_wait(&bars.p_full[q], n_pv[q] & 1, WAIT_LIMIT)) return false;
+                const int buf = n_pv[q] & 1;
+                if (!mbar_wait(&bars.p_full[q][buf], (n_pv[q] >> 1) & 1, WAIT_LIMIT)) return false;
                 tc_fence_after();
-                const uint32_t sv = smem_u32(smem + SV_OFF + (t & 1) * 32768);
+                const uint32_t sv = smem_u32(smem + SV_OFF + (t % NV) * V_STAGE_BYTES);
 #pragma unroll
-                for (int kk = 0; kk < 8; ++kk)
-                    umma_ts_f16(tmem + tm_o(q), tmem + tm_s(q) + kk * 8, make_smem_desc(sv + kk * 2048, 16384, 1024), idesc_pv,
-                                (n_pv[q] > 0 || kk > 0));
-                umma_commit(&bars.o_done[q]);
+                for (int kk = 0; kk < BN / 16; ++kk)
+                    umma_ts_f16(tmem + tm_o(q), tmem + tm_s(q, buf) + kk * 8,
+                                make_smem_desc(sv + kk * 2048, V_STAGE_BYTES / 2, 1024), idesc_pv, (n_pv[q] > 0 || kk > 0));
+                umma_commit(&bars.o_done[q][buf]);       // P.V number n of this query tile -> barrier n & 1
                 ++n_pv[q];
                 return true;
             };
-            if (ok && T > 0) {
-                ok = wait_k(0);
-                if (ok) {
-                    tc_fence_after();
-                    issue_qk(0, 0);
-                    issue_qk(1, 0);
-                    umma_commit(&bars.k_free[0]);
-                }
-            }
-            for (int t = 0; t < T && ok && !*abort_flag; ++t) {
-                ok = mbar_wait(&bars.v_full[t & 1], (t >> 1) & 1, WAIT_LIMIT);
+            // two tiles of Q.K^T run ahead of the softmax (S is double-buffered per query tile)
+            for (int t = 0; t < 2 && t < T && ok; ++t) {
+                ok = wait_k(t);
                 if (!ok) break;
+                issue_qk(0, t);
+                issue_qk(1, t);
+                umma_commit(&bars.k_free[t % NK]);
+            }
+#ifdef HYQ_TC_TIMING
+            long long tacc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+            const long long tstart = clock64();
+#endif
+            for (int t = 0; t < T && ok && !*abort_flag; ++t) {
+                TSTAMP(m0_);
+                ok = mbar_wait(&bars.v_full[t % NV], (t / NV) & 1, WAIT_LIMIT);
+                if (!ok) break;
+                TSTAMP(m1_);
                 ok = issue_pv(0, t);
                 if (!ok) break;
-                if (t + 1 < T) {
-                    ok = wait_k(t + 1);
+                TSTAMP(m2_);
+                if (t + 2 < T) {
+                    ok = wait_k(t + 2);
                     if (!ok) break;
-                    tc_fence_after();
-                    issue_qk(0, t + 1);
                 }
+                TSTAMP(m3_);
+                if (t + 2 < T) issue_qk(0, t + 2);
+                TSTAMP(m4_);
                 ok = issue_pv(1, t);
                 if (!ok) break;
-                umma_commit(&bars.v_free[t & 1]);
-                if (t + 1 < T) {
-                    issue_qk(1, t + 1);
-                    umma_commit(&bars.k_free[(t + 1) & 1]);
+                TSTAMP(m5_);
+                umma_commit(&bars.v_free[t % NV]);
+                if (t + 2 < T) {
+                    issue_qk(1, t + 2);
+                    umma_commit(&bars.k_free[(t + 2) % NK]);
                 }
+                TSTAMP(m6_);
+                TACC(0, m0_, m1_); TACC(1, m1_, m2_); TACC(2, m2_, m3_); TACC(3, m3_, m4_); TACC(4, m4_, m5_); TACC(5, m5_, m6_);
             }
+#ifdef HYQ_TC_TIMING
+            if (p.timing && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) {
+                for (int e = 0; e < 6; ++e) p.timing[32 + e] = tacc[e];
+                p.timing[32 + 8] = T;
+                p.timing[32 + 9] = clock64() - tstart;
+            }
+#endif
             if (!ok) fail();
         }
     } else {
@@ -414,107 +475,95 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
         const bool row_live = i < L;
         const bool ragged = sq.i0 + BM > L;
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
-        const uint32_t ts = tmem + tm_s(q) + lane_addr, to = tmem + tm_o(q) + lane_addr;
+        const uint32_t to = tmem + tm_o(q) + lane_addr;
         const float q_scale = row_live ? __ldg(p.q_scales + (long)qhead * p.nb + i / HYQ_BLOCK_TOKENS) : 0.0f;
         const int cnt_r = (sq.nB > 0 && row_live && i - W >= 0) ? count_le(idx_row, p.k, i - W) : 0;
         const uint32_t* bits_row = p.vl_bits + (long)qhead * p.mask_words;
+        const float* ks_row = p.k_scales + (long)kvhead * p.nb;
         float m_used = -INFINITY, l_run = 0.0f;
         int n_act = 0;
         bool ok = true;
 
-        // scales and vertical-line bitmask words of a low-bit tile, fetched one tile ahead of their use
-        float nk0 = 0.0f, nk1 = 0.0f;
-        uint32_t nvl[4] = {0u, 0u, 0u, 0u};
+        // scale and vertical-line bitmask words of a low-bit tile, fetched one tile ahead of their use
+        float nks = 0.0f;
+        uint32_t nvl0 = 0u, nvl1 = 0u;
         auto prefetch_tile = [&](int t) {
             if (t >= nA) return;
-            nk0 = __ldg(p.k_scales + (long)kvhead * p.nb + min(2 * t, p.nb - 1));
-            nk1 = __ldg(p.k_scales + (long)kvhead * p.nb + min(2 * t + 1, p.nb - 1));
-#pragma unroll
-            for (int w = 0; w < 4; ++w) nvl[w] = (t * 4 + w < p.mask_words) ? __ldg(bits_row + t * 4 + w) : 0u;
+            nks = __ldg(ks_row + min(t, p.nb - 1));
+            nvl0 = (2 * t < p.mask_words) ? __ldg(bits_row + 2 * t) : 0u;
+            nvl1 = (2 * t + 1 < p.mask_words) ? __ldg(bits_row + 2 * t + 1) : 0u;
         };
         prefetch_tile(0);
 #ifdef HYQ_TC_TIMING
         long long tacc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+        const long long tstart = clock64();
 #endif
 
         for (int t = 0; t < T; ++t) {
-            const float k0 = nk0, k1 = nk1;
-            uint32_t vlw[4] = {nvl[0], nvl[1], nvl[2], nvl[3]};
+            const float ks = nks;
+            uint32_t vl0 = nvl0, vl1 = nvl1;
             prefetch_tile(t + 1);
             if (!active(q, t)) continue;
-            // ---- per-tile column bounds and scales
+            // ---- per-tile column bounds and scale
             int lo = 0, hi = -1;
             bool need_range;
-            float cs0, cs1;
+            float cs;
             const bool lowbit = t < nA;
             if (lowbit) {
                 const int j0 = t * BN;
                 hi = row_live ? min(i - W - j0, BN - 1) : -1;
                 need_range = (j0 + BN - 1 > sq.i0 - W) || ragged;
                 // a zero scale (all-zero tile) still has to let -inf pass through the multiply
-                cs0 = fmaxf(q_scale * k0 * p.scale_log2, 1e-37f);
-                cs1 = fmaxf(q_scale * k1 * p.scale_log2, 1e-37f);
+                cs = fmaxf(q_scale * ks * p.scale_log2, 1e-37f);
             } else if (t < nA + nB) {
                 const int c0 = (t - nA) * BN;
                 hi = min(cnt_r - c0 - 1, BN - 1);
                 need_range = true;
-                cs0 = cs1 = p.scale_log2;
-                vlw[0] = vlw[1] = vlw[2] = vlw[3] = 0u;
+                cs = p.scale_log2;
+                vl0 = vl1 = 0u;
             } else {
                 const int j0 = (tC0 + t - nA - nB) * BN;
                 lo = max(0, i - W + 1 - j0);
                 hi = row_live ? min(i - j0, BN - 1) : -1;
                 need_range = (j0 + BN - 1 > sq.i0) || (j0 <= sq.i1 - W) || ragged;
-                cs0 = cs1 = p.scale_log2;
-                vlw[0] = vlw[1] = vlw[2] = vlw[3] = 0u;
+                cs = p.scale_log2;
+                vl0 = vl1 = 0u;
             }
             const int lo_eff = (hi >= lo) ? lo : 4096;
             const unsigned span = (hi >= lo) ? (unsigned)(hi - lo) : 0u;
             const bool int_scores = lowbit && !LOWBIT_FP8;
+            const int buf = n_act & 1;
+            const uint32_t ts = tmem + tm_s(q, buf) + lane_addr;
 
             TSTAMP(c0_);
-            if (!mbar_wait(&bars.s_full[q], n_act & 1, WAIT_LIMIT)) { ok = false; break; }
+            if (!mbar_wait(&bars.s_full[q][buf], (n_act >> 1) & 1, WAIT_LIMIT)) { ok = false; break; }
             __syncwarp();
             tc_fence_after();
             TSTAMP(c1_);
 
-            const uint32_t knock = int_scores ? KNOCKOUT_S32 : KNOCKOUT_F32;
             // ---- boundary tiles: causal / window / validity limits of this row, applied in TMEM
-            if (need_range) mask_tile_in_tmem(ts, lo_eff, span, knock);
-            // ---- vertical-line keys inside a low-bit tile: their S columns become -inf
-            if ((vlw[0] | vlw[1] | vlw[2] | vlw[3]) != 0u) {
-#pragma unroll
-                for (int w = 0; w < 4; ++w) {
-                    uint32_t bits = vlw[w];
-                    while (bits) {
-                        const int c = __ffs(bits) - 1;
-                        bits &= bits - 1;
-                        tmem_st1(ts + w * 32 + c, knock);
-                    }
-                }
-                tmem_wait_st();
-            }
+            if (need_range) mask_tile_in_tmem(ts, lo_eff, span, int_scores ? KNOCKOUT_S32 : KNOCKOUT_F32);
             TSTAMP(c2_);
-            if (int_scores) ok = softmax_tile<true>(ts, to, cs0, cs1, n_act == 0, &bars.o_done[q], (n_act - 1) & 1, m_used, l_run);
-            else ok = softmax_tile<false>(ts, to, cs0, cs1, n_act == 0, &bars.o_done[q], (n_act - 1) & 1, m_used, l_run);
+            if (int_scores) ok = softmax_tile<true>(ts, to, cs, vl0, vl1, n_act == 0, &bars.o_done[q][(n_act - 1) & 1], ((n_act - 1) >> 1) & 1, m_used, l_run TPASS);
+            else ok = softmax_tile<false>(ts, to, cs, vl0, vl1, n_act == 0, &bars.o_done[q][(n_act - 1) & 1], ((n_act - 1) >> 1) & 1, m_used, l_run TPASS);
             if (!ok) break;
-            TSTAMP(c3_);
             tc_fence_before();
-            mbar_arrive(&bars.p_full[q]);
-            TSTAMP(c4_);
-            TACC(0, c0_, c1_); TACC(1, c1_, c2_); TACC(2, c2_, c3_); TACC(3, c3_, c4_);
-#ifdef HYQ_TC_TIMING
-            tacc[4] += 1;
-#endif
+            mbar_arrive(&bars.p_full[q][buf]);
+            TSTAMP(c3_);
+            TACC(0, c0_, c1_); TACC(1, c1_, c2_); TACC(7, c0_, c3_);
             ++n_act;
         }
-#ifdef HYQ_TC_TIMING
-        if (p.timing && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && (threadIdx.x & 127) == 0)
-            for (int e = 0; e < 5; ++e) p.timing[q * 8 + e] = tacc[e];
-#endif
 
+#ifdef HYQ_TC_TIMING
+        if (p.timing && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && (threadIdx.x & 127) == 0) {
+            for (int e = 0; e < 8; ++e) p.timing[q * 16 + e] = tacc[e];
+            p.timing[q * 16 + 8] = n_act;
+            p.timing[q * 16 + 9] = clock64() - tstart;
+        }
+#endif
         // ---- epilogue: O / l
-        if (ok && n_act > 0) ok = mbar_wait(&bars.o_done[q], (n_act - 1) & 1, WAIT_LIMIT);
+        // (the P.V before the last one finished earlier: MMAs complete in order)
+        if (ok && n_act > 0) ok = mbar_wait(&bars.o_done[q][(n_act - 1) & 1], ((n_act - 1) >> 1) & 1, WAIT_LIMIT);
         __syncwarp();
         if (ok && n_act > 0) {
             tc_fence_after();
@@ -563,9 +612,9 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
 
 // ---------------------------------------------------------------------------------------------
 #ifdef HYQ_TC_TIMING
-static __device__ long long g_timing[16];
-extern "C" int hyq_debug_read_timing(long long* host16) {
-    return cudaMemcpyFromSymbol(host16, g_timing, sizeof(long long) * 16) == cudaSuccess ? 0 : 5;
+static __device__ long long g_timing[48];
+extern "C" int hyq_debug_read_timing(long long* host32) {
+    return cudaMemcpyFromSymbol(host32, g_timing, sizeof(long long) * 48) == cudaSuccess ? 0 : 5;
 }
 #endif
 
@@ -596,13 +645,11 @@ int launch_attn_tc(const hyq_attn_args& a, float alpha, cudaStream_t st) {
     p.B = a.B; p.Hq = a.Hq; p.Hkv = a.Hkv; p.L = a.L; p.window = a.window; p.k = a.k;
     p.nb = (a.L + HYQ_BLOCK_TOKENS - 1) / HYQ_BLOCK_TOKENS;
     p.mask_words = w.mask_words;
-    p.lowbit_fp8 = int4 ? 1 : 0;
     p.out_fp32 = a.out_dtype == 1;
     p.scale_log2 = alpha * 1.4426950408889634f;
     p.q_scales = a.q_scales; p.k_scales = a.k_scales; p.vl_idx = a.vl_idx;
     p.vl_bits = reinterpret_cast<const uint32_t*>(base + w.vl_bits);
     p.out = a.out; p.lse = a.lse; p.status = a.status_word;
-    p.timing = nullptr;
 #ifdef HYQ_TC_TIMING
     cudaGetSymbolAddress(reinterpret_cast<void**>(&p.timing), g_timing);
 #endif
