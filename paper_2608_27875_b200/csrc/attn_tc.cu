@@ -13,8 +13,9 @@
 // was computed from and is the A operand of the P.V MMA (fp16 x fp16).  K/V tiles are loaded once
 // (4-stage rings) and used by both query tiles.
 //
-// Warp roles (320 threads): warps 0-3 and 4-7 are the softmax groups of query tile 0 and 1 (thread r
-// owns query row r = TMEM lane r), warp 8 lane 0 issues TMA loads, warp 9 lane 0 issues MMAs.
+// Warp roles (352 threads): warps 0-3 and 4-7 are the softmax groups of query tile 0 and 1 (thread r
+// owns query row r = TMEM lane r), warp 8 lane 0 issues TMA loads, warps 9 and 10 (lane 0) issue the
+// MMAs of query tile 0 and 1.
 // The running maximum is only raised when a tile exceeds it by more than 2^8 (the rescale of O is
 // then rare); integer scores become floats through a magic-number add folded into the exponent
 // FFMA.  Every mbarrier wait is bounded; when one expires the CTA records HYQ_ERR_TIMEOUT in the
@@ -29,7 +30,7 @@ using namespace sm100;
 
 constexpr int BM = 128, BN = 64, QT = 2;
 constexpr int NK = 4, NV = 4;                       // K and V ring depths
-constexpr int TC_THREADS = 320;
+constexpr int TC_THREADS = 352;
 constexpr long long WAIT_LIMIT = 4000000000LL;      // SM clocks (~2 s): far beyond any legitimate wait
 constexpr float RESCALE_THRESHOLD = 8.0f;           // log2 units
 
@@ -157,10 +158,10 @@ __device__ __forceinline__ float exp_chunk(const uint32_t (&raw)[BN], int col0, 
 }
 
 // one tile of the online softmax for one query row: S (TMEM) -> running (m, l) -> P (TMEM, fp16).
-// vl0 / vl1: bitmask of vertical-line keys among the 64 columns (they are skipped).
+// (columns that must not count were set to -inf in TMEM beforehand)
 // returns false when a bounded wait expired
 template <bool INT>
-__device__ __forceinline__ bool softmax_tile(uint32_t ts, uint32_t to, float cs, uint32_t vl0, uint32_t vl1, bool first,
+__device__ __forceinline__ bool softmax_tile(uint32_t ts, uint32_t to, float cs, bool first,
                                              uint64_t* o_done, uint32_t o_parity, float& m_used, float& l_run TARGS) {
     uint32_t raw[BN];
     TSTAMP(s0_);
@@ -171,15 +172,6 @@ __device__ __forceinline__ bool softmax_tile(uint32_t ts, uint32_t to, float cs,
         tmem_wait_ld();
     }
     TSTAMP(s1_);
-    constexpr uint32_t knock = INT ? KNOCKOUT_S32 : KNOCKOUT_F32;
-    if (vl0 != 0u) {                  // uniform over the warp
-#pragma unroll
-        for (int e = 0; e < 32; ++e) raw[e] = ((vl0 >> e) & 1u) ? knock : raw[e];
-    }
-    if (vl1 != 0u) {
-#pragma unroll
-        for (int e = 0; e < 32; ++e) raw[32 + e] = ((vl1 >> e) & 1u) ? knock : raw[32 + e];
-    }
     TSTAMP(s2_);
     const float f = row_max<INT>(raw);
     const float mt = (f == -INFINITY) ? -INFINITY : f * cs;
@@ -241,6 +233,94 @@ __device__ __forceinline__ void mask_tile_in_tmem(uint32_t ts, int lo_eff, unsig
     tmem_wait_st();
 }
 
+// the tile walk of one CTA: union of both query tiles' lists
+struct Walk {
+    int nA, nB, tC0, nC, T;
+};
+
+__device__ __forceinline__ bool tile_active(const QSched& s, const Walk& w, int t) {
+    if (!s.live) return false;
+    if (t < w.nA) return t < s.nA;
+    if (t < w.nA + w.nB) return t - w.nA < s.nB;
+    const int tile = w.tC0 + t - w.nA - w.nB;
+    return tile >= s.tC0 && tile <= s.tC1;
+}
+
+// advancing a shared-memory matrix descriptor by a byte offset only touches its 14-bit address field
+__device__ __forceinline__ uint64_t desc_advance(uint64_t desc, uint32_t bytes) { return desc + (uint64_t)(bytes >> 4); }
+
+// MMA issue for one query tile (one thread): S = Q.K^T two tiles ahead of the softmax, O += P.V behind it
+template <bool LOWBIT_FP8>
+__device__ __forceinline__ bool mma_issuer(int q, const QSched& sq, const Walk& w, TcBarriers& bars, unsigned char* smem,
+                                           uint32_t tmem, volatile int* abort_flag TARGS) {
+    const uint32_t idesc_lq = LOWBIT_FP8 ? make_idesc(ACC_F32, FMT_E4M3, FMT_E4M3, 0, 0, BM, BN)
+                                         : make_idesc(ACC_S32, FMT_S8, FMT_S8, 0, 0, BM, BN);
+    const uint32_t idesc_qk = make_idesc(ACC_F32, FMT_BF16, FMT_BF16, 0, 0, BM, BN);
+    const uint32_t idesc_pv = make_idesc(ACC_F32, FMT_F16, FMT_F16, 0, 1, BM, HYQ_D);
+    const uint64_t dq = make_smem_desc(smem_u32(smem + SQ_OFF + q * Q_TILE_BYTES), 0, 1024);
+    const uint64_t dqc = make_smem_desc(smem_u32(smem + SQC_OFF + q * QC_TILE_BYTES), 0, 1024);
+    const uint64_t dk0 = make_smem_desc(smem_u32(smem + SK_OFF), 0, 1024);
+    const uint64_t dv0 = make_smem_desc(smem_u32(smem + SV_OFF), V_STAGE_BYTES / 2, 1024);
+    const uint32_t ts0 = tmem + tm_s(q, 0), to = tmem + tm_o(q);
+    int n_qk = 0, n_pv = 0;                         // active tiles issued so far
+    if (!mbar_wait(&bars.q_full, 0, WAIT_LIMIT)) return false;
+
+    auto qk = [&](int t) -> bool {
+        if (!mbar_wait(&bars.k_full[t % NK], (t / NK) & 1, WAIT_LIMIT)) return false;
+        if (tile_active(sq, w, t)) {
+            tc_fence_after();
+            const uint64_t dk = desc_advance(dk0, (t % NK) * K_STAGE_BYTES);
+            const int buf = n_qk & 1;
+            const uint32_t d = ts0 + buf * BN;
+            if (t < w.nA) {
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) {
+                    if (LOWBIT_FP8) umma_ss_f8f6f4(d, desc_advance(dqc, kk * 32), desc_advance(dk, kk * 32), idesc_lq, kk > 0);
+                    else umma_ss_i8(d, desc_advance(dqc, kk * 32), desc_advance(dk, kk * 32), idesc_lq, kk > 0);
+                }
+            } else {
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk)
+                    umma_ss_f16(d, desc_advance(dq, (kk >> 2) * (Q_TILE_BYTES / 2) + (kk & 3) * 32),
+                                desc_advance(dk, (kk >> 2) * (K_STAGE_BYTES / 2) + (kk & 3) * 32), idesc_qk, kk > 0);
+            }
+            umma_commit(&bars.s_full[q][buf]);
+            ++n_qk;
+        }
+        umma_commit(&bars.k_free[t % NK]);          // one arrival per issuer; the ring slot is free after both
+        return true;
+    };
+    auto pv = [&](int t) -> bool {
+        if (!mbar_wait(&bars.v_full[t % NV], (t / NV) & 1, WAIT_LIMIT)) return false;
+        if (tile_active(sq, w, t)) {
+            const int buf = n_pv & 1;
+            if (!mbar_wait(&bars.p_full[q][buf], (n_pv >> 1) & 1, WAIT_LIMIT)) return false;
+            tc_fence_after();
+            const uint64_t dv = desc_advance(dv0, (t % NV) * V_STAGE_BYTES);
+            const uint32_t pa = ts0 + buf * BN;
+#pragma unroll
+            for (int kk = 0; kk < BN / 16; ++kk)
+                umma_ts_f16(to, pa + kk * 8, desc_advance(dv, kk * 2048), idesc_pv, (n_pv > 0 || kk > 0));
+            umma_commit(&bars.o_done[q][buf]);      // P.V number n of this query tile -> barrier n & 1
+            ++n_pv;
+        }
+        umma_commit(&bars.v_free[t % NV]);
+        return true;
+    };
+    // two tiles of Q.K^T run ahead of the softmax (S is double-buffered)
+    for (int t = 0; t < 2 && t < w.T; ++t)
+        if (!qk(t)) return false;
+    for (int t = 0; t < w.T && !*abort_flag; ++t) {
+        TSTAMP(m0_);
+        if (!pv(t)) return false;
+        TSTAMP(m1_);
+        if (t + 2 < w.T && !qk(t + 2)) return false;
+        TSTAMP(m2_);
+        TACC(0, m0_, m1_); TACC(1, m1_, m2_);
+    }
+    return true;
+}
+
 template <bool LOWBIT_FP8>       // true: low-bit codes are e4m3 bytes (kind::f8f6f4); false: int8 (kind::i8)
 __global__ void __launch_bounds__(TC_THREADS, 1)
 attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
@@ -261,16 +341,16 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
         mbar_init(&bars.q_full, 1);
         for (int s = 0; s < NK; ++s) {
             mbar_init(&bars.k_full[s], 1);
-            mbar_init(&bars.k_free[s], 1);
+            mbar_init(&bars.k_free[s], QT);
         }
         for (int s = 0; s < NV; ++s) {
             mbar_init(&bars.v_full[s], 1);
-            mbar_init(&bars.v_free[s], 1);
+            mbar_init(&bars.v_free[s], QT);
         }
         for (int q = 0; q < QT; ++q) {
             for (int bf = 0; bf < 2; ++bf) {
                 mbar_init(&bars.s_full[q][bf], 1);
-                mbar_init(&bars.p_full[q][bf], 128);
+                mbar_init(&bars.p_full[q][bf], 4);           // one arrival per softmax warp
                 mbar_init(&bars.o_done[q][bf], 1);
             }
         }
@@ -291,10 +371,8 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
     const uint32_t tmem = tmem_base_s;
 
     // per query tile: nA low-bit tiles, nB gathered vertical-line tiles, window tiles tC0..tC1
-    QSched qs[QT];
-#pragma unroll
-    for (int q = 0; q < QT; ++q) {
-        QSched& s = qs[q];
+    auto make_sched = [&](int q) {
+        QSched s;
         s.i0 = (pt * QT + q) * BM;
         s.live = s.i0 < L;
         s.i1 = min(s.i0 + BM - 1, L - 1);
@@ -302,20 +380,16 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
         s.nB = s.live ? (cnt_b_s[q] + BN - 1) / BN : 0;
         s.tC0 = max(0, s.i0 - W + 1) / BN;
         s.tC1 = (s.live && W > 0) ? s.i1 / BN : -1;
-    }
-    // the CTA walks the union of both lists (tile 1 holds the later rows, so its lists are the longer ones)
-    const int nA = max(qs[0].nA, qs[1].nA), nB = max(qs[0].nB, qs[1].nB);
-    const int tC0 = qs[0].tC0, tC1 = max(qs[0].tC1, qs[1].tC1);
-    const int nC = (W > 0) ? tC1 - tC0 + 1 : 0;
-    const int T = nA + nB + nC;
-    auto active = [&](int q, int t) -> bool {
-        const QSched& s = qs[q];
-        if (!s.live) return false;
-        if (t < nA) return t < s.nA;
-        if (t < nA + nB) return t - nA < s.nB;
-        const int tile = tC0 + t - nA - nB;
-        return tile >= s.tC0 && tile <= s.tC1;
+        return s;
     };
+    const QSched qs0 = make_sched(0), qs1 = make_sched(1);
+    // the CTA walks the union of both lists (tile 1 holds the later rows, so its lists are the longer ones)
+    Walk w;
+    w.nA = max(qs0.nA, qs1.nA);
+    w.nB = max(qs0.nB, qs1.nB);
+    w.tC0 = qs0.tC0;
+    w.nC = (W > 0) ? max(qs0.tC1, qs1.tC1) - w.tC0 + 1 : 0;
+    w.T = w.nA + w.nB + w.nC;
 
     volatile int* abort_flag = &abort_s;
     auto fail = [&]() {
@@ -330,22 +404,23 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
             prefetch_tmap(&maps.k);
             prefetch_tmap(&maps.kc);
             prefetch_tmap(&maps.vh16);
+            const int live[QT] = {qs0.live, qs1.live}, qi0[QT] = {qs0.i0, qs1.i0};
             uint32_t qbytes = 0;
             for (int q = 0; q < QT; ++q)
-                if (qs[q].live) qbytes += Q_TILE_BYTES + (nA > 0 ? QC_TILE_BYTES : 0);
+                if (live[q]) qbytes += Q_TILE_BYTES + (w.nA > 0 ? QC_TILE_BYTES : 0);
             mbar_arrive_expect_tx(&bars.q_full, qbytes);
             for (int q = 0; q < QT; ++q) {
-                if (!qs[q].live) continue;
-                tma_load_3d(smem + SQ_OFF + q * Q_TILE_BYTES, &maps.q, &bars.q_full, 0, qs[q].i0, qhead);
-                tma_load_3d(smem + SQ_OFF + q * Q_TILE_BYTES + Q_TILE_BYTES / 2, &maps.q, &bars.q_full, 64, qs[q].i0, qhead);
-                if (nA > 0) tma_load_3d(smem + SQC_OFF + q * QC_TILE_BYTES, &maps.qc, &bars.q_full, 0, qs[q].i0, qhead);
+                if (!live[q]) continue;
+                tma_load_3d(smem + SQ_OFF + q * Q_TILE_BYTES, &maps.q, &bars.q_full, 0, qi0[q], qhead);
+                tma_load_3d(smem + SQ_OFF + q * Q_TILE_BYTES + Q_TILE_BYTES / 2, &maps.q, &bars.q_full, 64, qi0[q], qhead);
+                if (w.nA > 0) tma_load_3d(smem + SQC_OFF + q * QC_TILE_BYTES, &maps.qc, &bars.q_full, 0, qi0[q], qhead);
             }
-            for (int t = 0; t < T && !*abort_flag; ++t) {
+            for (int t = 0; t < w.T && !*abort_flag; ++t) {
                 const int sk_i = t % NK, uk = t / NK, sv_i = t % NV, uv = t / NV;
                 unsigned char* sk = smem + SK_OFF + sk_i * K_STAGE_BYTES;
                 unsigned char* sv = smem + SV_OFF + sv_i * V_STAGE_BYTES;
-                const bool lowbit = t < nA, vl = !lowbit && t < nA + nB;
-                const int row = lowbit ? t * BN : (vl ? (t - nA) * BN : (tC0 + t - nA - nB) * BN);
+                const bool lowbit = t < w.nA, vl = !lowbit && t < w.nA + w.nB;
+                const int row = lowbit ? t * BN : (vl ? (t - w.nA) * BN : (w.tC0 + t - w.nA - w.nB) * BN);
                 const int hd = vl ? qhead : kvhead;
                 if (uk > 0 && !mbar_wait(&bars.k_free[sk_i], (uk - 1) & 1, WAIT_LIMIT)) { fail(); break; }
                 if (lowbit) {
@@ -366,116 +441,34 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                 }
             }
         }
-    } else if (warp == 9) {
-        // ------------------------------------------------------------------ MMA issuer
+    } else if (warp == 9 || warp == 10) {
+        // ------------------------------------------------------------------ MMA issuers (one per query tile)
         if (lane == 0) {
-            const uint32_t idesc_lq = LOWBIT_FP8 ? make_idesc(ACC_F32, FMT_E4M3, FMT_E4M3, 0, 0, BM, BN)
-                                                 : make_idesc(ACC_S32, FMT_S8, FMT_S8, 0, 0, BM, BN);
-            const uint32_t idesc_qk = make_idesc(ACC_F32, FMT_BF16, FMT_BF16, 0, 0, BM, BN);
-            const uint32_t idesc_pv = make_idesc(ACC_F32, FMT_F16, FMT_F16, 0, 1, BM, HYQ_D);
-            int n_qk[QT] = {0, 0}, n_pv[QT] = {0, 0};      // active tiles issued so far, per query tile
-            bool ok = mbar_wait(&bars.q_full, 0, WAIT_LIMIT);
-            auto wait_k = [&](int t) {
-                const bool r = mbar_wait(&bars.k_full[t % NK], (t / NK) & 1, WAIT_LIMIT);
-                tc_fence_after();
-                return r;
-            };
-            auto issue_qk = [&](int q, int t) {
-                if (!active(q, t)) return;
-                const uint32_t sk = smem_u32(smem + SK_OFF + (t % NK) * K_STAGE_BYTES);
-                const int buf = n_qk[q] & 1;
-                const uint32_t d = tmem + tm_s(q, buf);
-                if (t < nA) {
-                    const uint32_t sqc = smem_u32(smem + SQC_OFF + q * QC_TILE_BYTES);
-#pragma unroll
-                    for (int kk = 0; kk < 4; ++kk) {
-                        const uint64_t da = make_smem_desc(sqc + kk * 32, 0, 1024), db = make_smem_desc(sk + kk * 32, 0, 1024);
-                        if (LOWBIT_FP8) umma_ss_f8f6f4(d, da, db, idesc_lq, kk > 0);
-                        else umma_ss_i8(d, da, db, idesc_lq, kk > 0);
-                    }
-                } else {
-                    const uint32_t sq = smem_u32(smem + SQ_OFF + q * Q_TILE_BYTES);
-#pragma unroll
-                    for (int kk = 0; kk < 8; ++kk) {
-                        const uint32_t offq = (kk >> 2) * (Q_TILE_BYTES / 2) + (kk & 3) * 32;
-                        const uint32_t offk = (kk >> 2) * (K_STAGE_BYTES / 2) + (kk & 3) * 32;
-                        umma_ss_f16(d, make_smem_desc(sq + offq, 0, 1024), make_smem_desc(sk + offk, 0, 1024), idesc_qk, kk > 0);
-                    }
-                }
-                umma_commit(&bars.s_full[q][buf]);
-                ++n_qk[q];
-            };
-            auto issue_pv = [&](int q, int t) -> bool {
-                if (!active(q, t)) return true;
-                const int buf = n_pv[q] & 1;
-                if (!mbar_wait(&bars.p_full[q][buf], (n_pv[q] >> 1) & 1, WAIT_LIMIT)) return false;
-                tc_fence_after();
-                const uint32_t sv = smem_u32(smem + SV_OFF + (t % NV) * V_STAGE_BYTES);
-#pragma unroll
-                for (int kk = 0; kk < BN / 16; ++kk)
-                    umma_ts_f16(tmem + tm_o(q), tmem + tm_s(q, buf) + kk * 8,
-                                make_smem_desc(sv + kk * 2048, V_STAGE_BYTES / 2, 1024), idesc_pv, (n_pv[q] > 0 || kk > 0));
-                umma_commit(&bars.o_done[q][buf]);       // P.V number n of this query tile -> barrier n & 1
-                ++n_pv[q];
-                return true;
-            };
-            // two tiles of Q.K^T run ahead of the softmax (S is double-buffered per query tile)
-            for (int t = 0; t < 2 && t < T && ok; ++t) {
-                ok = wait_k(t);
-                if (!ok) break;
-                issue_qk(0, t);
-                issue_qk(1, t);
-                umma_commit(&bars.k_free[t % NK]);
-            }
 #ifdef HYQ_TC_TIMING
             long long tacc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
             const long long tstart = clock64();
 #endif
-            for (int t = 0; t < T && ok && !*abort_flag; ++t) {
-                TSTAMP(m0_);
-                ok = mbar_wait(&bars.v_full[t % NV], (t / NV) & 1, WAIT_LIMIT);
-                if (!ok) break;
-                TSTAMP(m1_);
-                ok = issue_pv(0, t);
-                if (!ok) break;
-                TSTAMP(m2_);
-                if (t + 2 < T) {
-                    ok = wait_k(t + 2);
-                    if (!ok) break;
-                }
-                TSTAMP(m3_);
-                if (t + 2 < T) issue_qk(0, t + 2);
-                TSTAMP(m4_);
-                ok = issue_pv(1, t);
-                if (!ok) break;
-                TSTAMP(m5_);
-                umma_commit(&bars.v_free[t % NV]);
-                if (t + 2 < T) {
-                    issue_qk(1, t + 2);
-                    umma_commit(&bars.k_free[(t + 2) % NK]);
-                }
-                TSTAMP(m6_);
-                TACC(0, m0_, m1_); TACC(1, m1_, m2_); TACC(2, m2_, m3_); TACC(3, m3_, m4_); TACC(4, m4_, m5_); TACC(5, m5_, m6_);
-            }
+            const int q = warp - 9;
+            const bool ok = mma_issuer<LOWBIT_FP8>(q, q ? qs1 : qs0, w, bars, smem, tmem, abort_flag TPASS);
+            if (!ok) fail();
 #ifdef HYQ_TC_TIMING
             if (p.timing && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) {
-                for (int e = 0; e < 6; ++e) p.timing[32 + e] = tacc[e];
-                p.timing[32 + 8] = T;
-                p.timing[32 + 9] = clock64() - tstart;
+                for (int e = 0; e < 2; ++e) p.timing[32 + q * 8 + e] = tacc[e];
+                p.timing[32 + q * 8 + 2] = w.T;
+                p.timing[32 + q * 8 + 3] = clock64() - tstart;
             }
 #endif
-            if (!ok) fail();
         }
-    } else {
+    } else if (warp < 8) {
         // ------------------------------------------------------------------ softmax groups
         const int q = warp >> 2;
-        const QSched sq = qs[q];
+        const QSched sq = q ? qs1 : qs0;
         const int r = threadIdx.x & 127;                // query row inside the tile = TMEM lane
         const int i = sq.i0 + r;
         const bool row_live = i < L;
         const bool ragged = sq.i0 + BM > L;
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
-        const uint32_t to = tmem + tm_o(q) + lane_addr;
+        const uint32_t to = tmem + tm_o(q) + lane_addr, ts0 = tmem + tm_s(q, 0) + lane_addr;
         const float q_scale = row_live ? __ldg(p.q_scales + (long)qhead * p.nb + i / HYQ_BLOCK_TOKENS) : 0.0f;
         const int cnt_r = (sq.nB > 0 && row_live && i - W >= 0) ? count_le(idx_row, p.k, i - W) : 0;
         const uint32_t* bits_row = p.vl_bits + (long)qhead * p.mask_words;
@@ -483,57 +476,85 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
         float m_used = -INFINITY, l_run = 0.0f;
         int n_act = 0;
         bool ok = true;
+        constexpr uint32_t knock_lq = LOWBIT_FP8 ? KNOCKOUT_F32 : KNOCKOUT_S32;
+
+        // own tile list: low-bit tiles [0, nA_own), vertical tiles, window tiles (positions in the CTA's walk)
+        const int a_end = sq.nA, b_beg = w.nA, b_end = w.nA + sq.nB;
+        const int c_beg = w.nA + w.nB + (sq.tC0 - w.tC0), c_end = (sq.tC1 >= sq.tC0) ? w.nA + w.nB + (sq.tC1 - w.tC0) + 1 : c_beg;
+        auto next_tile = [&](int t) -> int {            // first own tile at or after walk position t (or T)
+            if (!sq.live) return w.T;
+            if (t < a_end) return t;
+            if (t < b_beg) t = b_beg;
+            if (t < b_end) return t;
+            if (t < c_beg) t = c_beg;
+            return (t < c_end) ? t : w.T;
+        };
 
         // scale and vertical-line bitmask words of a low-bit tile, fetched one tile ahead of their use
         float nks = 0.0f;
         uint32_t nvl0 = 0u, nvl1 = 0u;
         auto prefetch_tile = [&](int t) {
-            if (t >= nA) return;
+            nks = 0.0f;
+            nvl0 = nvl1 = 0u;
+            if (t >= a_end) return;
             nks = __ldg(ks_row + min(t, p.nb - 1));
             nvl0 = (2 * t < p.mask_words) ? __ldg(bits_row + 2 * t) : 0u;
             nvl1 = (2 * t + 1 < p.mask_words) ? __ldg(bits_row + 2 * t + 1) : 0u;
         };
-        prefetch_tile(0);
+        // vertical-line keys of a low-bit tile: their S columns are set to -inf in TMEM (no wait here;
+        // the caller's next tcgen05.wait::st covers these stores)
+        auto knock_columns = [&](uint32_t ts, uint32_t v0, uint32_t v1) {
+            while (v0) {
+                const int c = __ffs(v0) - 1;
+                v0 &= v0 - 1;
+                tmem_st1(ts + c, knock_lq);
+            }
+            while (v1) {
+                const int c = __ffs(v1) - 1;
+                v1 &= v1 - 1;
+                tmem_st1(ts + 32 + c, knock_lq);
+            }
+        };
 #ifdef HYQ_TC_TIMING
         long long tacc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
         const long long tstart = clock64();
 #endif
-
-        for (int t = 0; t < T; ++t) {
+        int t = next_tile(0);
+        prefetch_tile(t);
+        bool knocked = false;                           // vertical columns of tile t already knocked out
+        while (t < w.T) {
             const float ks = nks;
-            uint32_t vl0 = nvl0, vl1 = nvl1;
-            prefetch_tile(t + 1);
-            if (!active(q, t)) continue;
+            const uint32_t vl0 = nvl0, vl1 = nvl1;
+            const int t_next = next_tile(t + 1);
+            prefetch_tile(t_next);
             // ---- per-tile column bounds and scale
             int lo = 0, hi = -1;
             bool need_range;
             float cs;
-            const bool lowbit = t < nA;
+            const bool lowbit = t < a_end;
             if (lowbit) {
                 const int j0 = t * BN;
                 hi = row_live ? min(i - W - j0, BN - 1) : -1;
                 need_range = (j0 + BN - 1 > sq.i0 - W) || ragged;
                 // a zero scale (all-zero tile) still has to let -inf pass through the multiply
                 cs = fmaxf(q_scale * ks * p.scale_log2, 1e-37f);
-            } else if (t < nA + nB) {
-                const int c0 = (t - nA) * BN;
+            } else if (t < b_end) {
+                const int c0 = (t - b_beg) * BN;
                 hi = min(cnt_r - c0 - 1, BN - 1);
                 need_range = true;
                 cs = p.scale_log2;
-                vl0 = vl1 = 0u;
             } else {
-                const int j0 = (tC0 + t - nA - nB) * BN;
+                const int j0 = (w.tC0 + t - w.nA - w.nB) * BN;
                 lo = max(0, i - W + 1 - j0);
                 hi = row_live ? min(i - j0, BN - 1) : -1;
                 need_range = (j0 + BN - 1 > sq.i0) || (j0 <= sq.i1 - W) || ragged;
                 cs = p.scale_log2;
-                vl0 = vl1 = 0u;
             }
             const int lo_eff = (hi >= lo) ? lo : 4096;
             const unsigned span = (hi >= lo) ? (unsigned)(hi - lo) : 0u;
             const bool int_scores = lowbit && !LOWBIT_FP8;
             const int buf = n_act & 1;
-            const uint32_t ts = tmem + tm_s(q, buf) + lane_addr;
+            const uint32_t ts = ts0 + buf * BN;
 
             TSTAMP(c0_);
             if (!mbar_wait(&bars.s_full[q][buf], (n_act >> 1) & 1, WAIT_LIMIT)) { ok = false; break; }
@@ -541,19 +562,35 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
             tc_fence_after();
             TSTAMP(c1_);
 
+            if (!knocked && (vl0 | vl1) != 0u) {
+                knock_columns(ts, vl0, vl1);
+                tmem_wait_st();
+            }
             // ---- boundary tiles: causal / window / validity limits of this row, applied in TMEM
             if (need_range) mask_tile_in_tmem(ts, lo_eff, span, int_scores ? KNOCKOUT_S32 : KNOCKOUT_F32);
             TSTAMP(c2_);
-            if (int_scores) ok = softmax_tile<true>(ts, to, cs, vl0, vl1, n_act == 0, &bars.o_done[q][(n_act - 1) & 1], ((n_act - 1) >> 1) & 1, m_used, l_run TPASS);
-            else ok = softmax_tile<false>(ts, to, cs, vl0, vl1, n_act == 0, &bars.o_done[q][(n_act - 1) & 1], ((n_act - 1) >> 1) & 1, m_used, l_run TPASS);
+            // if the next tile's scores have already landed, its vertical columns are knocked out now and
+            // the stores complete under this tile's exponentials
+            const int nbuf = buf ^ 1;
+            knocked = false;
+            if (t_next < a_end && (nvl0 | nvl1) != 0u) {         // uniform over the warp
+                knocked = __all_sync(0xffffffffu, mbar_try_wait(&bars.s_full[q][nbuf], ((n_act + 1) >> 1) & 1));
+                if (knocked) {
+                    tc_fence_after();
+                    knock_columns(ts0 + nbuf * BN, nvl0, nvl1);
+                }
+            }
+            if (int_scores) ok = softmax_tile<true>(ts, to, cs, n_act == 0, &bars.o_done[q][(n_act - 1) & 1], ((n_act - 1) >> 1) & 1, m_used, l_run TPASS);
+            else ok = softmax_tile<false>(ts, to, cs, n_act == 0, &bars.o_done[q][(n_act - 1) & 1], ((n_act - 1) >> 1) & 1, m_used, l_run TPASS);
             if (!ok) break;
             tc_fence_before();
-            mbar_arrive(&bars.p_full[q][buf]);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bars.p_full[q][buf]);
             TSTAMP(c3_);
             TACC(0, c0_, c1_); TACC(1, c1_, c2_); TACC(7, c0_, c3_);
             ++n_act;
+            t = t_next;
         }
-
 #ifdef HYQ_TC_TIMING
         if (p.timing && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && (threadIdx.x & 127) == 0) {
             for (int e = 0; e < 8; ++e) p.timing[q * 16 + e] = tacc[e];
@@ -584,14 +621,14 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                         uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.out) + ((long)qhead * L + i) * HYQ_D + c * 32);
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
-                            uint32_t w[4];
+                            uint32_t wd[4];
 #pragma unroll
                             for (int q2 = 0; q2 < 4; ++q2) {
                                 const __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(o[8 * e + 2 * q2]) * inv,
                                                                                 __uint_as_float(o[8 * e + 2 * q2 + 1]) * inv);
-                                w[q2] = *reinterpret_cast<const uint32_t*>(&b2);
+                                wd[q2] = *reinterpret_cast<const uint32_t*>(&b2);
                             }
-                            dst[e] = make_uint4(w[0], w[1], w[2], w[3]);
+                            dst[e] = make_uint4(wd[0], wd[1], wd[2], wd[3]);
                         }
                     }
                 }
