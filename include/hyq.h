@@ -87,6 +87,33 @@ int hyq_select_vertical(const void* q, const void* k_, int B, int Hq, int Hkv, i
                         size_t workspace_bytes, void* stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * hyq_select_vertical_static - hyq_select_vertical for callers that have no device memory to lend.
+ * (No counterpart in the paper: it computes exactly what hyq_select_vertical computes and exists
+ * only because of how its scratch memory is provided.)
+ *
+ *   Some callers cannot hand over a workspace: a plug-in running inside a serving process whose
+ *   memory pool already owns the whole GPU has nothing left to allocate from, and a latency-critical
+ *   loop cannot afford cudaMalloc, which synchronises the device.  For them the tail means and the fp64
+ *   scores are kept in a fixed array of HYQ_SELECT_STATIC_SCRATCH_BYTES that is part of the library
+ *   image: every GPU that loads the library carries those bytes until the process exits, used or not.
+ *   The call allocates nothing and frees nothing, neither itself nor through a library routine.
+ *
+ *   Arguments, results and errors are those of hyq_select_vertical without workspace / workspace_bytes,
+ *   plus: a problem whose scratch need (hyq_select_vertical_workspace) exceeds
+ *   HYQ_SELECT_STATIC_SCRATCH_BYTES returns HYQ_ERR_WORKSPACE and launches nothing.
+ *   (8 MiB covers B*Hq*(P + 128) <= 1 Mi scores, e.g. 32 query heads at L = 32768, window 1024.)
+ *
+ *   The first call on each device looks up the array's device address (one runtime query, made with
+ *   that device current, result cached); make that first call outside any stream capture.
+ *   All calls on a device share the one array and each call overwrites what the previous one left
+ *   (nothing in it has to start at zero): two calls whose kernels overlap on the GPU - different
+ *   streams, or different host threads - race on it.  Run them one after the other.
+ * ------------------------------------------------------------------------------------------- */
+#define HYQ_SELECT_STATIC_SCRATCH_BYTES (8u << 20)
+int hyq_select_vertical_static(const void* q, const void* k_, int B, int Hq, int Hkv, int Lq, int Lk, int D,
+                               int window, int n_tail, int k, int32_t* idx_out, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
  * hyq_quantize_blocks - Algorithm 2, Stage 2 (per-tile symmetric quantization).
  *
  *   One tile = block_tokens (64) consecutive tokens x all D channels of one (b, head), cut by

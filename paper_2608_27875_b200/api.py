@@ -17,7 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libhyq.so")
 HYQ_OK = 0
 IMPL_AUTO, IMPL_TCGEN05, IMPL_SIMT = 0, 1, 2
 EXPORTS = ("hyq_status_string", "hyq_version", "hyq_paper_k", "hyq_select_vertical_workspace",
-           "hyq_select_vertical", "hyq_quantize_blocks", "hyq_hybrid_attention_prefill_workspace",
+           "hyq_select_vertical", "hyq_select_vertical_static", "hyq_quantize_blocks", "hyq_hybrid_attention_prefill_workspace",
            "hyq_hybrid_attention_prefill")
 
 
@@ -58,6 +58,8 @@ def lib() -> ctypes.CDLL:
         L.hyq_select_vertical_workspace.argtypes = [ctypes.c_int] * 8 + [ctypes.POINTER(ctypes.c_size_t)]
         L.hyq_select_vertical.argtypes = ([ctypes.c_void_p] * 2 + [ctypes.c_int] * 9 +
                                           [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p])
+        L.hyq_select_vertical_static.argtypes = ([ctypes.c_void_p] * 2 + [ctypes.c_int] * 9 +
+                                                 [ctypes.c_void_p, ctypes.c_void_p])
         L.hyq_quantize_blocks.argtypes = ([ctypes.c_void_p] + [ctypes.c_int] * 6 +
                                           [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p])
         L.hyq_hybrid_attention_prefill_workspace.argtypes = [ctypes.POINTER(AttnArgs), ctypes.POINTER(ctypes.c_size_t)]
@@ -112,6 +114,26 @@ def hyq_select_vertical(q: torch.Tensor, k: torch.Tensor, window: int, k_sel: in
     _check(lib().hyq_select_vertical(q.data_ptr(), k.data_ptr(), B, Hq, Hkv, Lq, Lk, D, window, n_tail, k_eff,
                                      out.data_ptr(), workspace.data_ptr(), workspace.numel(), _stream()),
            "hyq_select_vertical")
+    return out
+
+
+SELECT_STATIC_SCRATCH_BYTES = 8 << 20
+
+
+def hyq_select_vertical_static(q: torch.Tensor, k: torch.Tensor, window: int, k_sel: int, n_tail: int = 0,
+                               out: torch.Tensor | None = None) -> torch.Tensor:
+    """Algorithm 1 with the library's built-in scratch array instead of a workspace: for callers that
+    cannot allocate device memory at call time.  Pass ``out`` to make the call allocation-free on the
+    Python side as well.  Calls on one device must not overlap; problems needing more than
+    ``SELECT_STATIC_SCRATCH_BYTES`` of scratch raise ``HyqError`` (workspace too small)."""
+    _dev(q, torch.bfloat16, "q"), _dev(k, torch.bfloat16, "k")
+    B, Hq, Lq, D = q.shape
+    _, Hkv, Lk, _ = k.shape
+    k_eff = k_sel if Lk - window > 0 else 0
+    if out is None:
+        out = torch.empty(B, Hq, k_eff, dtype=torch.int32, device=q.device)
+    _check(lib().hyq_select_vertical_static(q.data_ptr(), k.data_ptr(), B, Hq, Hkv, Lq, Lk, D, window, n_tail, k_eff,
+                                            out.data_ptr(), _stream()), "hyq_select_vertical_static")
     return out
 
 

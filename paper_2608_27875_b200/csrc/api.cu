@@ -72,6 +72,17 @@ int hyq_select_vertical(const void* q, const void* k_, int B, int Hq, int Hkv, i
     return launch_select(q, k_, B, Hq, Hkv, Lq, Lk, window, n_tail, k, idx_out, workspace, static_cast<cudaStream_t>(stream));
 }
 
+int hyq_select_vertical_static(const void* q, const void* k_, int B, int Hq, int Hkv, int Lq, int Lk, int D, int window,
+                               int n_tail, int k, int32_t* idx_out, void* stream) {
+    const int rc = check_select(q, k_, B, Hq, Hkv, Lq, Lk, D, window, n_tail, k);
+    if (rc != HYQ_OK) return rc;
+    const long P = (Lk - window > 0) ? (long)Lk - window : 0;
+    if (P == 0 || k == 0) return HYQ_OK;
+    if (!q || !k_ || !idx_out) return HYQ_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k_) || (reinterpret_cast<uintptr_t>(idx_out) & 3u)) return HYQ_ERR_ALIGNMENT;
+    return launch_select_static(q, k_, B, Hq, Hkv, Lq, Lk, window, n_tail, k, idx_out, static_cast<cudaStream_t>(stream));
+}
+
 int hyq_quantize_blocks(const void* x, int B, int H, int L, int D, int block_tokens, int format, void* codes_out,
                         float* scales_out, void* stream) {
     if (B <= 0 || H <= 0 || L <= 0) return HYQ_ERR_INVALID_ARG;

@@ -10,6 +10,8 @@
 //                      selected positions ascending; equal scores go to the lower position.
 // The fp64 chain is what makes the selected set reproducible bit for bit: ranking in lower
 // precision flips pairs whose scores differ by less than its rounding error.
+#include <mutex>
+
 #include "common.cuh"
 
 namespace hyq {
@@ -204,6 +206,41 @@ int launch_select(const void* q, const void* k, int B, int Hq, int Hkv, int Lq, 
 
     topk_kernel<<<B * Hq, TOPK_THREADS, 0, st>>>(scores, P, k_sel, idx_out);
     return launch_status();
+}
+
+// -------------------------------------------------------------------------------------------
+// Selection without caller-provided scratch: the tail means and the fp64 scores live in a fixed array
+// that is part of the library image on every device that loads it.
+static __device__ __align__(256) unsigned char g_select_scratch[HYQ_SELECT_STATIC_SCRATCH_BYTES];
+
+// Device address of g_select_scratch on the current device.  In host code the array's name is only
+// a handle for the runtime, never a pointer a kernel may use, so the address is looked up once per
+// device (with that device current) and cached.
+static int select_static_scratch(void** out) {
+    constexpr int MAX_DEVICES = 64;
+    static std::mutex mu;
+    static void* cached[MAX_DEVICES] = {};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return HYQ_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(mu);
+    if (cached[dev] == nullptr) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_select_scratch) != cudaSuccess || ptr == nullptr) return HYQ_ERR_CUDA;
+        cached[dev] = ptr;
+    }
+    *out = cached[dev];
+    return HYQ_OK;
+}
+
+int launch_select_static(const void* q, const void* k, int B, int Hq, int Hkv, int Lq, int Lk, int window, int n_tail,
+                         int k_sel, int32_t* idx_out, cudaStream_t st) {
+    if (select_workspace_bytes(B, Hq, Lk, window) > (size_t)HYQ_SELECT_STATIC_SCRATCH_BYTES) return HYQ_ERR_WORKSPACE;
+    void* scratch = nullptr;
+    const int rc = select_static_scratch(&scratch);
+    if (rc != HYQ_OK) return rc;
+    // every byte of scratch that the kernels read is written earlier in the same call, so nothing has to
+    // be cleared between calls
+    return launch_select(q, k, B, Hq, Hkv, Lq, Lk, window, n_tail, k_sel, idx_out, scratch, st);
 }
 
 }  // namespace hyq
