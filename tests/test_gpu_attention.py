@@ -99,3 +99,57 @@ def test_benchmark_configs_on_sampled_rows(name):
     idx = oracle.select_vertical(wl.bits(Q), wl.bits(K), w.window, w.k)
     rows = wl.sample_rows(w.L, w.window, n_random=24)
     _check(Q, K, V, w.fmts, idx, w.window, api.IMPL_TCGEN05, rows)
+
+
+def _run_whole_path(w):
+    """The launch configuration bench.py times: every head of the workload, whole path on the device."""
+    ensure_built()
+    Q, K, V = wl.make_inputs(w)
+    res = api.hybrid_prefill(Q.cuda(), K.cuda(), V.cuda(), w.window, w.k, w.fmts)
+    torch.cuda.synchronize()
+    return {n: t.cpu().numpy() for n, t in res.items()}
+
+
+@pytest.mark.parametrize("name,kv_heads,n_random", [("c1", [0, 7], 24), ("c2", [5], 16), ("c4", [2], 12), ("c3", [6], 4)])
+def test_full_size_workloads_in_the_benchmark_launch_configuration(name, kv_heads, n_random):
+    """Full benchmark sizes, all heads launched at once; the oracle recomputes whole (batch, KV head)
+    groups for selection and quantization (bit-exact) and sampled rows of the attention output."""
+    w = wl.CONFIGS[name]
+    got = _run_whole_path(w)
+    g = w.Hq // w.Hkv
+    b = w.B - 1
+    rows = wl.sample_rows(w.L, w.window, n_random=n_random, edge=2)
+    for kvh in kv_heads:
+        Qh, Kh, Vh = wl.make_inputs(w.scaled(B=b + 1), heads=[kvh])
+        Qh, Kh, Vh = Qh[b:b + 1], Kh[b:b + 1], Vh[b:b + 1]
+        qs_ = slice(kvh * g, (kvh + 1) * g)
+        ref_idx = oracle.select_vertical(wl.bits(Qh), wl.bits(Kh), w.window, w.k)
+        np.testing.assert_array_equal(got["idx"][b:b + 1, qs_], ref_idx)
+        qz = oracle_quant_all(Qh, Kh, Vh, w.fmts)
+        for (codes, scales), cn, sn, hs in zip(qz, ("q_codes", "k_codes", "v_codes"), ("q_scales", "k_scales", "v_scales"),
+                                               (qs_, slice(kvh, kvh + 1), slice(kvh, kvh + 1))):
+            np.testing.assert_array_equal(got[cn][b:b + 1, hs], codes)
+            np.testing.assert_array_equal(got[sn][b:b + 1, hs].view(np.uint32), scales.view(np.uint32))
+        ref = _ref(Qh, Kh, Vh, qz, w.fmts, ref_idx, w.window, rows)
+        out = got["out"][b:b + 1, qs_][:, :, rows]
+        assert np.isfinite(got["out"]).all()
+        max_abs, mean_rel = errors(out, ref)
+        assert max_abs <= MAX_ABS_TOL and mean_rel <= MEAN_REL_TOL, (name, kvh, max_abs, mean_rel)
+
+
+def test_tensor_core_and_cuda_core_kernels_agree_on_every_output_of_config1():
+    """Every row of every head at a benchmark size: two independent kernels, both within tolerance of the
+    definition on the sampled rows, must agree with each other everywhere."""
+    ensure_built()
+    w = wl.CONFIGS["c1"]
+    Q, K, V = (t.cuda() for t in wl.make_inputs(w))
+    idx = api.hyq_select_vertical(Q, K, w.window, w.k)
+    qz = [api.hyq_quantize_blocks(t, f) for t, f in zip((Q, K, V), w.fmts)]
+    (qc, qs), (kc, ks), (vc, vs) = qz
+    outs = [api.hyq_hybrid_attention_prefill(Q, K, V, qc, kc, vc, qs, ks, vs, w.fmts, idx, w.window, impl=impl)
+            for impl in (api.IMPL_TCGEN05, api.IMPL_SIMT)]
+    torch.cuda.synchronize()
+    diff = (outs[0] - outs[1]).abs()
+    assert torch.isfinite(outs[0]).all()
+    assert float(diff.max()) <= MAX_ABS_TOL
+    assert float(diff.sum() / outs[1].abs().sum()) <= MEAN_REL_TOL
