@@ -80,7 +80,7 @@ struct TcParams {
 
 struct TcBarriers {
     uint64_t q_full, k_full[MAX_STAGES], k_free[MAX_STAGES], v_full[MAX_STAGES], v_free[MAX_STAGES];
-    uint64_t s_full[QT][2], p_full[QT][2], o_done[QT][2];
+    uint64_t s_full[QT][2], p_full[QT][2], o_done[QT][2], xu_turn[QT];
 };
 
 // which key tiles a 128-row query tile visits in each pass
@@ -133,33 +133,13 @@ __device__ __forceinline__ float block_max(const uint32_t (&raw)[N], int c0) {
     }
 }
 
-// p = 2^(raw * c + bias) for 32 columns starting at `col0`, packed to fp16 pairs; returns their fp32 sum
-template <bool INT, int N>
-__device__ __forceinline__ float exp_chunk(const uint32_t (&raw)[N], int col0, float c, float bias, uint32_t (&pk)[16]) {
-    float s0 = 0.0f, s1 = 0.0f, s2 = 0.0f, s3 = 0.0f;
-#pragma unroll
-    for (int e = 0; e < 32; e += 4) {
-        float pv[4];
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const uint32_t rv = raw[col0 + e + u];
-            const float x = INT ? __uint_as_float(rv + INT_MAGIC) : __uint_as_float(rv);
-            pv[u] = ex2f(fmaf(x, c, bias));
-        }
-        s0 += pv[0]; s1 += pv[1]; s2 += pv[2]; s3 += pv[3];
-        const __half2 h01 = __floats2half2_rn(pv[0], pv[1]), h23 = __floats2half2_rn(pv[2], pv[3]);
-        pk[e >> 1] = *reinterpret_cast<const uint32_t*>(&h01);
-        pk[(e >> 1) + 1] = *reinterpret_cast<const uint32_t*>(&h23);
-    }
-    return (s0 + s1) + (s2 + s3);
-}
-
 // one tile of the online softmax for one query row: S (TMEM) -> running (m, l) -> P (TMEM, fp16).
 //   cs[b]   score scale of 64-column block b (includes log2 e)
 // (columns that must not count were set to -inf in TMEM beforehand)
 // returns false when a bounded wait expired
 template <bool INT, int TBN>
-__device__ __forceinline__ bool softmax_tile(uint32_t ts, uint32_t to, const float (&cs)[TBN / 64], bool first, uint64_t* o_done, uint32_t o_parity, float& m_used, float& l_run) {
+__device__ __forceinline__ bool softmax_tile(uint32_t ts, uint32_t to, const float (&cs)[TBN / 64], bool first, uint64_t* o_done, uint32_t o_parity, float& m_used, float& l_run,
+                                             uint64_t* turn_wait, uint32_t turn_parity, uint64_t* turn_pass) {
     uint32_t raw[TBN];
     {
         uint32_t (*rc)[32] = reinterpret_cast<uint32_t (*)[32]>(raw);
@@ -200,16 +180,40 @@ __device__ __forceinline__ bool softmax_tile(uint32_t ts, uint32_t to, const flo
         }
     }
     const float m_eff = (m_used == -INFINITY) ? 0.0f : m_used;
-    float rs = 0.0f;
+    // the exponentials of the two softmax groups take turns on the MUFU (see the caller)
+    if (turn_wait != nullptr && !mbar_wait(turn_wait, turn_parity, WAIT_LIMIT)) return false;
+    // all exponentials of the row first (in place, independent of each other), then sums, packs and stores
+#pragma unroll
+    for (int bl = 0; bl < TBN / 64; ++bl) {
+        const float sc = cs[bl];
+        const float bias = INT ? fmaf(-INT_MAGIC_F, sc, -m_eff) : -m_eff;
+#pragma unroll
+        for (int e = 0; e < 64; ++e) {
+            const uint32_t rv = raw[bl * 64 + e];
+            const float x = INT ? __uint_as_float(rv + INT_MAGIC) : __uint_as_float(rv);
+            raw[bl * 64 + e] = __float_as_uint(ex2f(fmaf(x, sc, bias)));
+        }
+    }
+    float acc[8] = {0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f};
 #pragma unroll
     for (int c = 0; c < TBN / 32; ++c) {
         uint32_t pk[16];
-        const float sc = cs[c / 2];
-        const float bias = INT ? fmaf(-INT_MAGIC_F, sc, -m_eff) : -m_eff;
-        rs += exp_chunk<INT>(raw, c * 32, sc, bias, pk);
+#pragma unroll
+        for (int e = 0; e < 32; e += 2) {
+            const float p0 = __uint_as_float(raw[c * 32 + e]), p1 = __uint_as_float(raw[c * 32 + e + 1]);
+            acc[e & 7] += p0;
+            acc[(e & 7) + 1] += p1;
+            const __half2 h2 = __floats2half2_rn(p0, p1);
+            pk[e >> 1] = *reinterpret_cast<const uint32_t*>(&h2);
+        }
         tmem_st16(ts + c * 16, pk);
     }
+    const float rs = ((acc[0] + acc[1]) + (acc[2] + acc[3])) + ((acc[4] + acc[5]) + (acc[6] + acc[7]));
     l_run += rs;
+    if (turn_pass != nullptr) {
+        __syncwarp();
+        if ((threadIdx.x & 31) == 0) mbar_arrive(turn_pass);
+    }
     tmem_wait_st();
     return true;
 }
@@ -234,23 +238,29 @@ struct Walk {
     int nA, nB, tC0, nC, T;
 };
 
-__device__ __forceinline__ bool tile_active(const QSched& s, const Walk& w, int t) {
-    if (!s.live) return false;
-    if (t < w.nA) return t < s.nA;
-    if (t < w.nA + w.nB) return t - w.nA < s.nB;
-    const int tile = w.tC0 + t - w.nA - w.nB;
-    return tile >= s.tC0 && tile <= s.tC1;
+// own tile ranges of one query tile inside the CTA's walk: [0, a_end) low-bit, [b_beg, b_end) vertical, [c_beg, c_end) window
+struct OwnTiles {
+    int a_end, b_beg, b_end, c_beg, c_end;
+    __device__ __forceinline__ bool has(int t) const { return t < a_end || (t >= b_beg && t < b_end) || (t >= c_beg && t < c_end); }
+};
+__device__ __forceinline__ OwnTiles own_tiles(const QSched& s, const Walk& w) {
+    OwnTiles o;
+    o.a_end = s.live ? s.nA : 0;
+    o.b_beg = w.nA;
+    o.b_end = s.live ? w.nA + s.nB : w.nA;
+    o.c_beg = w.nA + w.nB + (s.tC0 - w.tC0);
+    o.c_end = (s.live && s.tC1 >= s.tC0) ? w.nA + w.nB + (s.tC1 - w.tC0) + 1 : o.c_beg;
+    return o;
 }
 
-// advancing a shared-memory matrix descriptor by a byte offset only touches its 14-bit address field
-__device__ __forceinline__ uint64_t desc_advance(uint64_t desc, uint32_t bytes) { return desc + (uint64_t)(bytes >> 4); }
-
-// MMA issue for one query tile (one thread): S = Q.K^T runs NBUF tiles ahead of the softmax, O += P.V behind it
+// MMA issue for one query tile (one thread): S = Q.K^T runs NBUF tiles ahead of the softmax, O += P.V behind it.
+// The loop body is kept to waits, MMAs and commits: ring positions, parities and descriptors advance incrementally.
 template <bool LOWBIT_FP8, int TBN>
 __device__ __forceinline__ bool mma_issuer(int q, const QSched& sq, const Walk& w, TcBarriers& bars, unsigned char* smem,
                                            uint32_t tmem, volatile int* abort_flag) {
     using G = Geo<TBN>;
     constexpr int BN = TBN, NST = G::NST, NBUF = G::NBUF;
+    constexpr uint32_t STAGE16 = G::STAGE_BYTES >> 4;                  // descriptor address units per ring stage
     const uint32_t idesc_lq = LOWBIT_FP8 ? make_idesc(ACC_F32, FMT_E4M3, FMT_E4M3, 0, 0, BM, BN)
                                          : make_idesc(ACC_S32, FMT_S8, FMT_S8, 0, 0, BM, BN);
     const uint32_t idesc_qk = make_idesc(ACC_F32, FMT_BF16, FMT_BF16, 0, 0, BM, BN);
@@ -260,56 +270,62 @@ __device__ __forceinline__ bool mma_issuer(int q, const QSched& sq, const Walk& 
     const uint64_t dk0 = make_smem_desc(smem_u32(smem + SK_OFF), 0, 1024);
     const uint64_t dv0 = make_smem_desc(smem_u32(smem + SV_OFF), G::STAGE_BYTES / 2, 1024);
     const uint32_t ts0 = tmem + tm_s(q), to = tmem + tm_o(q);
-    int n_qk = 0, n_pv = 0;                         // active tiles issued so far
+    const OwnTiles own = own_tiles(sq, w);
+    const int nA = w.nA, T = w.T;
     if (!mbar_wait(&bars.q_full, 0, WAIT_LIMIT)) return false;
 
-    auto qk = [&](int t) -> bool {
-        if (!mbar_wait(&bars.k_full[t % NST], (t / NST) & 1, WAIT_LIMIT)) return false;
-        if (tile_active(sq, w, t)) {
+    // Q.K^T cursor
+    int tq = 0, kst = 0;
+    uint32_t kpar = 0, n_qk = 0;
+    auto qk = [&]() -> bool {
+        if (!mbar_wait(&bars.k_full[kst], kpar, WAIT_LIMIT)) return false;
+        if (own.has(tq)) {
             tc_fence_after();
-            const uint64_t dk = desc_advance(dk0, (t % NST) * G::STAGE_BYTES);
-            const int buf = n_qk % NBUF;
+            const uint64_t dk = dk0 + (uint64_t)(kst * STAGE16);
+            const uint32_t buf = n_qk % NBUF;
             const uint32_t d = ts0 + buf * BN;
-            if (t < w.nA) {
+            if (tq < nA) {
 #pragma unroll
                 for (int kk = 0; kk < 4; ++kk) {
-                    if (LOWBIT_FP8) umma_ss_f8f6f4(d, desc_advance(dqc, kk * 32), desc_advance(dk, kk * 32), idesc_lq, kk > 0);
-                    else umma_ss_i8(d, desc_advance(dqc, kk * 32), desc_advance(dk, kk * 32), idesc_lq, kk > 0);
+                    if (LOWBIT_FP8) umma_ss_f8f6f4(d, dqc + kk * 2, dk + kk * 2, idesc_lq, kk > 0);
+                    else umma_ss_i8(d, dqc + kk * 2, dk + kk * 2, idesc_lq, kk > 0);
                 }
             } else {
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk)
-                    umma_ss_f16(d, desc_advance(dq, (kk >> 2) * (Q_TILE_BYTES / 2) + (kk & 3) * 32),
-                                desc_advance(dk, (kk >> 2) * (G::STAGE_BYTES / 2) + (kk & 3) * 32), idesc_qk, kk > 0);
+                    umma_ss_f16(d, dq + ((kk >> 2) * (Q_TILE_BYTES / 32) + (kk & 3) * 2),
+                                dk + ((kk >> 2) * (G::STAGE_BYTES / 32) + (kk & 3) * 2), idesc_qk, kk > 0);
             }
             umma_commit(&bars.s_full[q][buf]);
             ++n_qk;
         }
-        umma_commit(&bars.k_free[t % NST]);         // one arrival per issuer; the ring slot is free after both
+        umma_commit(&bars.k_free[kst]);             // one arrival per issuer; the ring slot is free after both
+        ++tq;
+        if (++kst == NST) { kst = 0; kpar ^= 1u; }
         return true;
     };
-    auto pv = [&](int t) -> bool {
-        if (!mbar_wait(&bars.v_full[t % NST], (t / NST) & 1, WAIT_LIMIT)) return false;
-        if (tile_active(sq, w, t)) {
-            const int buf = n_pv % NBUF;
-            if (!mbar_wait(&bars.p_full[q][buf], (n_pv / NBUF) & 1, WAIT_LIMIT)) return false;
+    // P.V cursor
+    int vst = 0;
+    uint32_t vpar = 0, n_pv = 0;
+    for (int t = 0; t < NBUF && t < T; ++t)
+        if (!qk()) return false;
+    for (int t = 0; t < T; ++t) {
+        if (!mbar_wait(&bars.v_full[vst], vpar, WAIT_LIMIT)) return false;
+        if (own.has(t)) {
+            const uint32_t buf = n_pv % NBUF;
+            if (!mbar_wait(&bars.p_full[q][buf], (n_pv / NBUF) & 1u, WAIT_LIMIT)) return false;
             tc_fence_after();
-            const uint64_t dv = desc_advance(dv0, (t % NST) * G::STAGE_BYTES);
+            const uint64_t dv = dv0 + (uint64_t)(vst * STAGE16);
             const uint32_t pa = ts0 + buf * BN;
 #pragma unroll
-            for (int kk = 0; kk < BN / 16; ++kk)
-                umma_ts_f16(to, pa + kk * 8, desc_advance(dv, kk * 2048), idesc_pv, (n_pv > 0 || kk > 0));
-            umma_commit(&bars.o_done[q][n_pv & 1]);  // P.V number n of this query tile -> barrier n & 1
+            for (int kk = 0; kk < BN / 16; ++kk) umma_ts_f16(to, pa + kk * 8, dv + kk * 128, idesc_pv, (n_pv > 0 || kk > 0));
+            umma_commit(&bars.o_done[q][n_pv & 1u]);  // P.V number n of this query tile -> barrier n & 1
             ++n_pv;
         }
-        umma_commit(&bars.v_free[t % NST]);
-        return true;
-    };
-    for (int t = 0; t < NBUF && t < w.T; ++t)
-        if (!qk(t)) return false;
-    for (int t = 0; t < w.T && !*abort_flag; ++t) {
-        if (!pv(t)) return false;
-        if (t + NBUF < w.T && !qk(t + NBUF)) return false;
+        umma_commit(&bars.v_free[vst]);
+        if (++vst == NST) { vst = 0; vpar ^= 1u; }
+        if (tq < T && !qk()) return false;
+        if (*abort_flag) return true;
     }
     return true;
 }
@@ -347,6 +363,7 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                 mbar_init(&bars.p_full[q][bf], 4);           // one arrival per softmax warp
                 mbar_init(&bars.o_done[q][bf], 1);
             }
+            mbar_init(&bars.xu_turn[q], 4);
         }
         fence_mbar_init();
         abort_s = 0;
@@ -499,11 +516,12 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                 }
             }
         };
+        // tiles during which both groups are busy
+        const int n_own0 = qs0.live ? qs0.nA + qs0.nB + max(0, qs0.tC1 - qs0.tC0 + 1) : 0;
+        const int n_own1 = qs1.live ? qs1.nA + qs1.nB + max(0, qs1.tC1 - qs1.tC0 + 1) : 0;
+        const int n_pingpong = min(n_own0, n_own1);
         int t = next_tile(0);
         prefetch_tile(t);
-        // the two groups share the MUFU and issue ports: group 1 starts half a tile late (when group 0 has
-        // delivered its first P) so that one group's exponentials run under the other's waits
-        if (q == 1 && qs0.live && w.T > 0 && !mbar_wait(&bars.p_full[0][0], 0, WAIT_LIMIT)) ok = false;
         bool knocked = false;                           // vertical columns of tile t already knocked out in TMEM
         while (t < w.T && ok) {
             float ks[NSC];
@@ -574,10 +592,21 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                     }
                 }
             }
+            // ping-pong on the exponential phase while both groups still have tiles: group 0 may start tile n
+            // when group 1 has finished the exponentials of its tile n-1, group 1 when group 0 has finished tile n
+            uint64_t* tw = nullptr;
+            uint64_t* tp = nullptr;
+            uint32_t tpar = 0;
+            if (n_act < n_pingpong) {
+                tp = &bars.xu_turn[q ^ 1];
+                if (q == 1) { tw = &bars.xu_turn[1]; tpar = n_act & 1; }
+                else if (n_act > 0) { tw = &bars.xu_turn[0]; tpar = (n_act - 1) & 1; }
+                if (q == 1 && n_act + 1 >= n_pingpong) tp = nullptr;      // nobody waits for this last hand-over
+            }
             uint64_t* od = &bars.o_done[q][(n_act - 1) & 1];
             const uint32_t op = ((n_act - 1) >> 1) & 1;
-            if (int_scores) ok = softmax_tile<true, TBN>(ts, to, cs, n_act == 0, od, op, m_used, l_run);
-            else ok = softmax_tile<false, TBN>(ts, to, cs, n_act == 0, od, op, m_used, l_run);
+            if (int_scores) ok = softmax_tile<true, TBN>(ts, to, cs, n_act == 0, od, op, m_used, l_run, tw, tpar, tp);
+            else ok = softmax_tile<false, TBN>(ts, to, cs, n_act == 0, od, op, m_used, l_run, tw, tpar, tp);
             if (!ok) break;
             tc_fence_before();
             __syncwarp();
