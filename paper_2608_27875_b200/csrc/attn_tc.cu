@@ -16,8 +16,8 @@
 // Warp roles (352 threads): warps 0-3 and 4-7 are the softmax groups of query tile 0 and 1 (thread r
 // owns query row r = TMEM lane r), warp 8 lane 0 issues TMA loads, warps 9 and 10 (lane 0) issue the
 // MMAs of query tile 0 and 1.
-// The running maximum is only raised when a tile exceeds it by more than 2^8 (the rescale of O is
-// then rare); integer scores become floats through a magic-number add folded into the exponent
+// The exponentials are taken against a running reference maximum that is only raised when a tile
+// overshoots it by more than 2^8 (the rescale of O is then rare); integer scores become floats through a magic-number add folded into the exponent
 // FFMA.  Every mbarrier wait is bounded; when one expires the CTA records HYQ_ERR_TIMEOUT in the
 // status word and unwinds.
 #include <cuda_fp16.h>
@@ -32,7 +32,7 @@ constexpr int BM = 128, QT = 2;
 constexpr int RING_BYTES = 65536;                   // shared memory of the K ring and of the V ring
 constexpr int TC_THREADS = 352;
 constexpr long long WAIT_LIMIT = 4000000000LL;      // SM clocks (~2 s): far beyond any legitimate wait
-constexpr float RESCALE_THRESHOLD = 8.0f;           // log2 units
+constexpr float OVERSHOOT_LIMIT = 256.0f;           // a tile is redone when a probability exceeds 2^8 of the reference
 
 constexpr uint32_t Q_TILE_BYTES = BM * HYQ_D * 2, QC_TILE_BYTES = BM * HYQ_D;        // 32768, 16384
 constexpr uint32_t SQ_OFF = 0, SQC_OFF = QT * Q_TILE_BYTES, SK_OFF = SQC_OFF + QT * QC_TILE_BYTES;
@@ -80,7 +80,7 @@ struct TcParams {
 
 struct TcBarriers {
     uint64_t q_full, k_full[MAX_STAGES], k_free[MAX_STAGES], v_full[MAX_STAGES], v_free[MAX_STAGES];
-    uint64_t s_full[QT][2], p_full[QT][2], o_done[QT][2], xu_turn[QT];
+    uint64_t s_full[QT][2], p_full[QT][2], o_done[QT][2];
 };
 
 // which key tiles a 128-row query tile visits in each pass
@@ -133,13 +133,42 @@ __device__ __forceinline__ float block_max(const uint32_t (&raw)[N], int c0) {
     }
 }
 
+// exponentials of one row: pk = fp16 pairs of 2^(raw * cs + bias), returns their fp32 sum; pmax2 collects the
+// running maximum of the packed values (two lanes of a half2)
+template <bool INT, int TBN>
+__device__ __forceinline__ float exp_row(const uint32_t (&raw)[TBN], const float (&cs)[TBN / 64], float m_eff,
+                                         uint32_t (&pk)[TBN / 2], __half2& pmax2) {
+    float acc[8] = {0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+    for (int bl = 0; bl < TBN / 64; ++bl) {
+        const float sc = cs[bl];
+        const float bias = INT ? fmaf(-INT_MAGIC_F, sc, -m_eff) : -m_eff;
+#pragma unroll
+        for (int e = 0; e < 64; e += 2) {
+            const uint32_t r0 = raw[bl * 64 + e], r1 = raw[bl * 64 + e + 1];
+            const float p0 = ex2f(fmaf(INT ? __uint_as_float(r0 + INT_MAGIC) : __uint_as_float(r0), sc, bias));
+            const float p1 = ex2f(fmaf(INT ? __uint_as_float(r1 + INT_MAGIC) : __uint_as_float(r1), sc, bias));
+            acc[e & 7] += p0;
+            acc[(e & 7) + 1] += p1;
+            const __half2 h2 = __floats2half2_rn(p0, p1);
+            pmax2 = __hmax2(pmax2, h2);
+            pk[bl * 32 + (e >> 1)] = *reinterpret_cast<const uint32_t*>(&h2);
+        }
+    }
+    return ((acc[0] + acc[1]) + (acc[2] + acc[3])) + ((acc[4] + acc[5]) + (acc[6] + acc[7]));
+}
+
 // one tile of the online softmax for one query row: S (TMEM) -> running (m, l) -> P (TMEM, fp16).
 //   cs[b]   score scale of 64-column block b (includes log2 e)
 // (columns that must not count were set to -inf in TMEM beforehand)
+// Fast path: the exponentials are taken against the running reference maximum m_used without looking at
+// the tile's own maximum first; the tile is accepted when no probability exceeded OVERSHOOT_LIMIT.  Otherwise
+// (and while a row has no reference yet) the tile's maximum is computed, the reference is raised, O and l
+// are rescaled and the exponentials are redone.
 // returns false when a bounded wait expired
 template <bool INT, int TBN>
-__device__ __forceinline__ bool softmax_tile(uint32_t ts, uint32_t to, const float (&cs)[TBN / 64], bool first, uint64_t* o_done, uint32_t o_parity, float& m_used, float& l_run,
-                                             uint64_t* turn_wait, uint32_t turn_parity, uint64_t* turn_pass) {
+__device__ __forceinline__ bool softmax_tile(uint32_t ts, uint32_t to, const float (&cs)[TBN / 64], bool first, uint64_t* o_done,
+                                             uint32_t o_parity, float& m_used, float& l_run) {
     uint32_t raw[TBN];
     {
         uint32_t (*rc)[32] = reinterpret_cast<uint32_t (*)[32]>(raw);
@@ -147,72 +176,54 @@ __device__ __forceinline__ bool softmax_tile(uint32_t ts, uint32_t to, const flo
         for (int c = 0; c < TBN / 32; ++c) tmem_ld32(ts + c * 32, rc[c]);
         tmem_wait_ld();
     }
-    float mt = -INFINITY;
+    uint32_t pk[TBN / 2];
+    __half2 pmax2 = __floats2half2_rn(0.0f, 0.0f);
+    float rs = exp_row<INT, TBN>(raw, cs, (m_used == -INFINITY) ? 0.0f : m_used, pk, pmax2);
+    const float pmax = fmaxf(__low2float(pmax2), __high2float(pmax2));
+    // redo when this row has no reference yet, or a value overshot the reference by more than the threshold
+    // (NaN-safe: an overflow to inf fails the comparison too)
+    const bool redo = (m_used == -INFINITY) || !(pmax <= OVERSHOOT_LIMIT);
+    if (__any_sync(0xffffffffu, redo)) {
+        float mt = -INFINITY;
 #pragma unroll
-    for (int bl = 0; bl < TBN / 64; ++bl) {
-        const float f = block_max<INT>(raw, bl * 64);
-        mt = fmaxf(mt, (f == -INFINITY) ? -INFINITY : f * cs[bl]);
-    }
-
-    // raise the running maximum only when the tile exceeds it by the threshold
-    float alpha = 1.0f;
-    const bool raise = mt > m_used + RESCALE_THRESHOLD;          // also true for the first finite maximum
-    if (raise) {
-        alpha = ex2f(m_used - mt);                               // m_used = -inf -> 0
-        l_run *= alpha;
-        m_used = mt;
-    }
-    if (!first && __any_sync(0xffffffffu, raise)) {
-        // the previous P.V of this query tile must have landed before O is rescaled.  P.V number n
-        // signals barrier n & 1; the one before the previous is known to be complete (the S tile
-        // just read was issued after it), so the parity wait cannot alias.
-        if (!mbar_wait(o_done, o_parity, WAIT_LIMIT)) return false;
-        __syncwarp();
-        tc_fence_after();
+        for (int bl = 0; bl < TBN / 64; ++bl) {
+            const float f = block_max<INT>(raw, bl * 64);
+            mt = fmaxf(mt, (f == -INFINITY) ? -INFINITY : f * cs[bl]);
+        }
+        float alpha = 1.0f;
+        const bool raise = redo && mt > m_used;                  // rows that are fine keep their reference
+        if (raise) {
+            alpha = ex2f(m_used - mt);                           // m_used = -inf -> 0
+            l_run *= alpha;
+            m_used = mt;
+        }
+        if (!first && __any_sync(0xffffffffu, raise)) {
+            // the previous P.V of this query tile must have landed before O is rescaled.  P.V number n
+            // signals barrier n & 1; the one before the previous is known to be complete (the S tile
+            // just read was issued after it), so the parity wait cannot alias.
+            if (!mbar_wait(o_done, o_parity, WAIT_LIMIT)) return false;
+            __syncwarp();
+            tc_fence_after();
 #pragma unroll 1
-        for (int c = 0; c < 4; ++c) {
-            uint32_t o[32];
-            tmem_ld32(to + c * 32, o);
-            tmem_wait_ld();
+            for (int c = 0; c < 4; ++c) {
+                uint32_t o[32];
+                tmem_ld32(to + c * 32, o);
+                tmem_wait_ld();
 #pragma unroll
-            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-            tmem_st32(to + c * 32, o);
+                for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+                tmem_st32(to + c * 32, o);
+            }
+        }
+        if (raise) {
+            __half2 unused = __floats2half2_rn(0.0f, 0.0f);
+            rs = exp_row<INT, TBN>(raw, cs, m_used, pk, unused);
         }
     }
-    const float m_eff = (m_used == -INFINITY) ? 0.0f : m_used;
-    // the exponentials of the two softmax groups take turns on the MUFU (see the caller)
-    if (turn_wait != nullptr && !mbar_wait(turn_wait, turn_parity, WAIT_LIMIT)) return false;
-    // all exponentials of the row first (in place, independent of each other), then sums, packs and stores
-#pragma unroll
-    for (int bl = 0; bl < TBN / 64; ++bl) {
-        const float sc = cs[bl];
-        const float bias = INT ? fmaf(-INT_MAGIC_F, sc, -m_eff) : -m_eff;
-#pragma unroll
-        for (int e = 0; e < 64; ++e) {
-            const uint32_t rv = raw[bl * 64 + e];
-            const float x = INT ? __uint_as_float(rv + INT_MAGIC) : __uint_as_float(rv);
-            raw[bl * 64 + e] = __float_as_uint(ex2f(fmaf(x, sc, bias)));
-        }
-    }
-    float acc[8] = {0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f};
+    l_run += rs;
 #pragma unroll
     for (int c = 0; c < TBN / 32; ++c) {
-        uint32_t pk[16];
-#pragma unroll
-        for (int e = 0; e < 32; e += 2) {
-            const float p0 = __uint_as_float(raw[c * 32 + e]), p1 = __uint_as_float(raw[c * 32 + e + 1]);
-            acc[e & 7] += p0;
-            acc[(e & 7) + 1] += p1;
-            const __half2 h2 = __floats2half2_rn(p0, p1);
-            pk[e >> 1] = *reinterpret_cast<const uint32_t*>(&h2);
-        }
-        tmem_st16(ts + c * 16, pk);
-    }
-    const float rs = ((acc[0] + acc[1]) + (acc[2] + acc[3])) + ((acc[4] + acc[5]) + (acc[6] + acc[7]));
-    l_run += rs;
-    if (turn_pass != nullptr) {
-        __syncwarp();
-        if ((threadIdx.x & 31) == 0) mbar_arrive(turn_pass);
+        uint32_t (&pc)[16] = *reinterpret_cast<uint32_t (*)[16]>(&pk[c * 16]);
+        tmem_st16(ts + c * 16, pc);
     }
     tmem_wait_st();
     return true;
@@ -363,7 +374,6 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                 mbar_init(&bars.p_full[q][bf], 4);           // one arrival per softmax warp
                 mbar_init(&bars.o_done[q][bf], 1);
             }
-            mbar_init(&bars.xu_turn[q], 4);
         }
         fence_mbar_init();
         abort_s = 0;
@@ -516,10 +526,6 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                 }
             }
         };
-        // tiles during which both groups are busy
-        const int n_own0 = qs0.live ? qs0.nA + qs0.nB + max(0, qs0.tC1 - qs0.tC0 + 1) : 0;
-        const int n_own1 = qs1.live ? qs1.nA + qs1.nB + max(0, qs1.tC1 - qs1.tC0 + 1) : 0;
-        const int n_pingpong = min(n_own0, n_own1);
         int t = next_tile(0);
         prefetch_tile(t);
         bool knocked = false;                           // vertical columns of tile t already knocked out in TMEM
@@ -592,21 +598,10 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                     }
                 }
             }
-            // ping-pong on the exponential phase while both groups still have tiles: group 0 may start tile n
-            // when group 1 has finished the exponentials of its tile n-1, group 1 when group 0 has finished tile n
-            uint64_t* tw = nullptr;
-            uint64_t* tp = nullptr;
-            uint32_t tpar = 0;
-            if (n_act < n_pingpong) {
-                tp = &bars.xu_turn[q ^ 1];
-                if (q == 1) { tw = &bars.xu_turn[1]; tpar = n_act & 1; }
-                else if (n_act > 0) { tw = &bars.xu_turn[0]; tpar = (n_act - 1) & 1; }
-                if (q == 1 && n_act + 1 >= n_pingpong) tp = nullptr;      // nobody waits for this last hand-over
-            }
             uint64_t* od = &bars.o_done[q][(n_act - 1) & 1];
             const uint32_t op = ((n_act - 1) >> 1) & 1;
-            if (int_scores) ok = softmax_tile<true, TBN>(ts, to, cs, n_act == 0, od, op, m_used, l_run, tw, tpar, tp);
-            else ok = softmax_tile<false, TBN>(ts, to, cs, n_act == 0, od, op, m_used, l_run, tw, tpar, tp);
+            if (int_scores) ok = softmax_tile<true, TBN>(ts, to, cs, n_act == 0, od, op, m_used, l_run);
+            else ok = softmax_tile<false, TBN>(ts, to, cs, n_act == 0, od, op, m_used, l_run);
             if (!ok) break;
             tc_fence_before();
             __syncwarp();

@@ -153,3 +153,39 @@ def test_tensor_core_and_cuda_core_kernels_agree_on_every_output_of_config1():
     assert torch.isfinite(outs[0]).all()
     assert float(diff.max()) <= MAX_ABS_TOL
     assert float(diff.sum() / outs[1].abs().sum()) <= MEAN_REL_TOL
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("fmts", [INT8, INT4FP8])
+def test_row_maximum_that_keeps_rising_along_the_keys(impl, fmts):
+    """Scores that grow with the key position force the running maximum up tile after tile (every rescale
+    path of the online softmax), with late keys dominating early ones by many orders of magnitude."""
+    L, W, k = 900, 96, 10
+    g = torch.Generator().manual_seed(5)
+    u = torch.randn(128, generator=g)
+    u = u / u.norm()
+    ramp = torch.linspace(0.0, 1.0, L)[:, None]
+    Q = (0.3 * torch.randn(1, 2, L, 128, generator=g) + 6.0 * u).to(torch.bfloat16)
+    K = (0.3 * torch.randn(1, 2, L, 128, generator=g) + (40.0 * ramp) * u).to(torch.bfloat16)   # score ~ 21 * ramp (natural log units)
+    V = torch.randn(1, 2, L, 128, generator=g).to(torch.bfloat16)
+    idx = _rand_idx(1, 2, L - W, k, seed=3)
+    _check(Q, K, V, fmts, idx, W, impl)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_early_keys_dominate_and_all_zero_blocks(impl):
+    """The opposite order (the first keys carry almost all the mass, later tiles underflow) plus all-zero
+    K / V / Q blocks, whose scale is zero."""
+    L, W, k = 700, 64, 6
+    g = torch.Generator().manual_seed(9)
+    u = torch.randn(128, generator=g)
+    u = u / u.norm()
+    ramp = torch.linspace(1.0, 0.0, L)[:, None]
+    Q = (0.3 * torch.randn(1, 2, L, 128, generator=g) + 6.0 * u).to(torch.bfloat16)
+    K = (0.3 * torch.randn(1, 1, L, 128, generator=g) + (40.0 * ramp) * u).to(torch.bfloat16)
+    V = torch.randn(1, 1, L, 128, generator=g).to(torch.bfloat16)
+    K[0, 0, 128:192] = 0
+    V[0, 0, 256:320] = 0
+    Q[0, 1, 320:384] = 0
+    idx = _rand_idx(1, 2, L - W, k, seed=4)
+    _check(Q, K, V, INT8, idx, W, impl)
