@@ -341,6 +341,53 @@ __device__ __forceinline__ bool mma_issuer(int q, const QSched& sq, const Walk& 
     return true;
 }
 
+// TMA producer (one thread): the two query tiles once, then the K ring and the V ring along the CTA's walk
+template <int TBN>
+__device__ __forceinline__ bool tma_producer(const TcMaps& maps, const QSched& qs0, const QSched& qs1, const Walk& w, int qhead,
+                                             int kvhead, TcBarriers& bars, unsigned char* smem, volatile int* abort_flag) {
+    using G = Geo<TBN>;
+    constexpr int BN = TBN, NST = G::NST;
+    prefetch_tmap(&maps.q);
+    prefetch_tmap(&maps.k);
+    prefetch_tmap(&maps.kc);
+    prefetch_tmap(&maps.vh16);
+    const int live[QT] = {qs0.live, qs1.live}, qi0[QT] = {qs0.i0, qs1.i0};
+    uint32_t qbytes = 0;
+    for (int q = 0; q < QT; ++q)
+        if (live[q]) qbytes += Q_TILE_BYTES + (w.nA > 0 ? QC_TILE_BYTES : 0);
+    mbar_arrive_expect_tx(&bars.q_full, qbytes);
+    for (int q = 0; q < QT; ++q) {
+        if (!live[q]) continue;
+        tma_load_3d(smem + SQ_OFF + q * Q_TILE_BYTES, &maps.q, &bars.q_full, 0, qi0[q], qhead);
+        tma_load_3d(smem + SQ_OFF + q * Q_TILE_BYTES + Q_TILE_BYTES / 2, &maps.q, &bars.q_full, 64, qi0[q], qhead);
+        if (w.nA > 0) tma_load_3d(smem + SQC_OFF + q * QC_TILE_BYTES, &maps.qc, &bars.q_full, 0, qi0[q], qhead);
+    }
+    for (int t = 0; t < w.T && !*abort_flag; ++t) {
+        const int st = t % NST, use = t / NST;
+        unsigned char* sk = smem + SK_OFF + st * G::STAGE_BYTES;
+        unsigned char* sv = smem + SV_OFF + st * G::STAGE_BYTES;
+        const bool lowbit = t < w.nA, vl = !lowbit && t < w.nA + w.nB;
+        const int row = lowbit ? t * BN : (vl ? (t - w.nA) * BN : (w.tC0 + t - w.nA - w.nB) * BN);
+        const int hd = vl ? qhead : kvhead;
+        if (use > 0 && !mbar_wait(&bars.k_free[st], (use - 1) & 1, WAIT_LIMIT)) return false;
+        if (lowbit) {
+            mbar_arrive_expect_tx(&bars.k_full[st], G::KC_TILE_BYTES);
+            tma_load_3d(sk, &maps.kc, &bars.k_full[st], 0, row, hd);
+        } else {
+            const CUtensorMap* m = vl ? &maps.kvl : &maps.k;
+            mbar_arrive_expect_tx(&bars.k_full[st], G::STAGE_BYTES);
+            tma_load_3d(sk, m, &bars.k_full[st], 0, row, hd);
+            tma_load_3d(sk + G::STAGE_BYTES / 2, m, &bars.k_full[st], 64, row, hd);
+        }
+        if (use > 0 && !mbar_wait(&bars.v_free[st], (use - 1) & 1, WAIT_LIMIT)) return false;
+        const CUtensorMap* m = lowbit ? &maps.vh16 : (vl ? &maps.vvl : &maps.v16);
+        mbar_arrive_expect_tx(&bars.v_full[st], G::STAGE_BYTES);
+        tma_load_3d(sv, m, &bars.v_full[st], 0, row, hd);
+        tma_load_3d(sv + G::STAGE_BYTES / 2, m, &bars.v_full[st], 64, row, hd);
+    }
+    return true;
+}
+
 // TBN: keys per tile (64 or 128).  LOWBIT_FP8: low-bit codes are e4m3 bytes (kind::f8f6f4), else int8 (kind::i8)
 template <bool LOWBIT_FP8, int TBN>
 __global__ void __launch_bounds__(TC_THREADS, 1)
@@ -420,48 +467,7 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
 
     if (warp == 8) {
         // ------------------------------------------------------------------ TMA producer
-        if (lane == 0) {
-            prefetch_tmap(&maps.q);
-            prefetch_tmap(&maps.k);
-            prefetch_tmap(&maps.kc);
-            prefetch_tmap(&maps.vh16);
-            const int live[QT] = {qs0.live, qs1.live}, qi0[QT] = {qs0.i0, qs1.i0};
-            uint32_t qbytes = 0;
-            for (int q = 0; q < QT; ++q)
-                if (live[q]) qbytes += Q_TILE_BYTES + (w.nA > 0 ? QC_TILE_BYTES : 0);
-            mbar_arrive_expect_tx(&bars.q_full, qbytes);
-            for (int q = 0; q < QT; ++q) {
-                if (!live[q]) continue;
-                tma_load_3d(smem + SQ_OFF + q * Q_TILE_BYTES, &maps.q, &bars.q_full, 0, qi0[q], qhead);
-                tma_load_3d(smem + SQ_OFF + q * Q_TILE_BYTES + Q_TILE_BYTES / 2, &maps.q, &bars.q_full, 64, qi0[q], qhead);
-                if (w.nA > 0) tma_load_3d(smem + SQC_OFF + q * QC_TILE_BYTES, &maps.qc, &bars.q_full, 0, qi0[q], qhead);
-            }
-            for (int t = 0; t < w.T && !*abort_flag; ++t) {
-                const int st = t % NST, use = t / NST;
-                unsigned char* sk = smem + SK_OFF + st * G::STAGE_BYTES;
-                unsigned char* sv = smem + SV_OFF + st * G::STAGE_BYTES;
-                const bool lowbit = t < w.nA, vl = !lowbit && t < w.nA + w.nB;
-                const int row = lowbit ? t * BN : (vl ? (t - w.nA) * BN : (w.tC0 + t - w.nA - w.nB) * BN);
-                const int hd = vl ? qhead : kvhead;
-                if (use > 0 && !mbar_wait(&bars.k_free[st], (use - 1) & 1, WAIT_LIMIT)) { fail(); break; }
-                if (lowbit) {
-                    mbar_arrive_expect_tx(&bars.k_full[st], G::KC_TILE_BYTES);
-                    tma_load_3d(sk, &maps.kc, &bars.k_full[st], 0, row, hd);
-                } else {
-                    const CUtensorMap* m = vl ? &maps.kvl : &maps.k;
-                    mbar_arrive_expect_tx(&bars.k_full[st], G::STAGE_BYTES);
-                    tma_load_3d(sk, m, &bars.k_full[st], 0, row, hd);
-                    tma_load_3d(sk + G::STAGE_BYTES / 2, m, &bars.k_full[st], 64, row, hd);
-                }
-                if (use > 0 && !mbar_wait(&bars.v_free[st], (use - 1) & 1, WAIT_LIMIT)) { fail(); break; }
-                {
-                    const CUtensorMap* m = lowbit ? &maps.vh16 : (vl ? &maps.vvl : &maps.v16);
-                    mbar_arrive_expect_tx(&bars.v_full[st], G::STAGE_BYTES);
-                    tma_load_3d(sv, m, &bars.v_full[st], 0, row, hd);
-                    tma_load_3d(sv + G::STAGE_BYTES / 2, m, &bars.v_full[st], 64, row, hd);
-                }
-            }
-        }
+        if (lane == 0 && !tma_producer<TBN>(maps, qs0, qs1, w, qhead, kvhead, bars, smem, abort_flag)) fail();
     } else if (warp == 9 || warp == 10) {
         // ------------------------------------------------------------------ MMA issuers (one per query tile)
         if (lane == 0) {
@@ -658,8 +664,377 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
     }
 }
 
+// =============================================================================================
+// Variant with FOUR softmax groups (64-key tiles only): each query tile is served by two warpgroups
+// that take its key tiles alternately (group w owns S buffer w), so that every scheduler hosts four
+// softmax warps instead of two and TMEM / barrier round trips of one warp hide under the arithmetic
+// of the others.  Both groups of a query tile exponentiate against one shared per-row reference
+// maximum (shared memory); the decision whether tile n raises it is taken in tile order:
+//   group of tile n: scores -> row maximum -> wait for the decision of tile n-1 -> raise? (then: wait
+//   for P.V of tile n-1, rescale O, publish the new reference) -> signal "decision n" -> exponentials.
+// A group's partial row sum is kept relative to the reference it last saw and rescaled when it changes;
+// the two partial sums are exchanged through TMEM at the end.  Registers: 96 per thread (608 threads), so
+// a tile is read twice from TMEM in 32-column chunks (maximum pass, exponential pass).
+// =============================================================================================
+constexpr int TC4_THREADS = 608;                    // 16 softmax warps + TMA producer + 2 MMA issuers
+constexpr float RAISE_THRESHOLD = 8.0f;             // log2 units by which a tile must exceed the reference to raise it
+
+struct Tc4Barriers {
+    uint64_t dec[QT][2];        // decision of the tiles taken by group w of query tile q (4 arrivals: one per warp)
+    uint64_t fin[QT];           // both groups of query tile q have stored their partial sums (8 arrivals)
+};
+
+template <bool INT>
+__device__ __forceinline__ float chunk_max32(uint32_t ts, float m) {
+    uint32_t raw[32];
+    tmem_ld32(ts, raw);
+    tmem_wait_ld();
+    if (INT) {
+        int m0 = (int)raw[0], m1 = (int)raw[1], m2 = (int)raw[2], m3 = (int)raw[3];
+#pragma unroll
+        for (int e = 4; e < 32; e += 4) {
+            m0 = max(m0, (int)raw[e]);
+            m1 = max(m1, (int)raw[e + 1]);
+            m2 = max(m2, (int)raw[e + 2]);
+            m3 = max(m3, (int)raw[e + 3]);
+        }
+        const int mm = max(max(m0, m1), max(m2, m3));
+        return fmaxf(m, (mm < -(1 << 23)) ? -INFINITY : (float)mm);
+    } else {
+        float m0 = __uint_as_float(raw[0]), m1 = __uint_as_float(raw[1]), m2 = __uint_as_float(raw[2]), m3 = __uint_as_float(raw[3]);
+#pragma unroll
+        for (int e = 4; e < 32; e += 4) {
+            m0 = fmaxf(m0, __uint_as_float(raw[e]));
+            m1 = fmaxf(m1, __uint_as_float(raw[e + 1]));
+            m2 = fmaxf(m2, __uint_as_float(raw[e + 2]));
+            m3 = fmaxf(m3, __uint_as_float(raw[e + 3]));
+        }
+        return fmaxf(m, fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)));
+    }
+}
+
+// exponentials of 32 score columns at ts_in, stored as 16 columns of fp16 pairs at ts_out; returns their fp32 sum
+template <bool INT>
+__device__ __forceinline__ float chunk_exp32(uint32_t ts_in, uint32_t ts_out, float sc, float bias) {
+    uint32_t raw[32];
+    tmem_ld32(ts_in, raw);
+    tmem_wait_ld();
+    float a0 = 0.0f, a1 = 0.0f, a2 = 0.0f, a3 = 0.0f;
+    uint32_t pk[16];
+#pragma unroll
+    for (int e = 0; e < 32; e += 4) {
+        float pv[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const uint32_t rv = raw[e + u];
+            pv[u] = ex2f(fmaf(INT ? __uint_as_float(rv + INT_MAGIC) : __uint_as_float(rv), sc, bias));
+        }
+        a0 += pv[0]; a1 += pv[1]; a2 += pv[2]; a3 += pv[3];
+        const __half2 h01 = __floats2half2_rn(pv[0], pv[1]), h23 = __floats2half2_rn(pv[2], pv[3]);
+        pk[e >> 1] = *reinterpret_cast<const uint32_t*>(&h01);
+        pk[(e >> 1) + 1] = *reinterpret_cast<const uint32_t*>(&h23);
+    }
+    tmem_st16(ts_out, pk);
+    return (a0 + a1) + (a2 + a3);
+}
+
+template <bool LOWBIT_FP8>
+__global__ void __launch_bounds__(TC4_THREADS, 1)
+attn_tc4_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
+    constexpr int TBN = 64, BN = 64;
+    using G = Geo<TBN>;
+    constexpr int NST = G::NST;
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    __shared__ TcBarriers bars;
+    __shared__ Tc4Barriers bars4;
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int abort_s, cnt_b_s[QT];
+    __shared__ float m_ref_s[QT][BM];               // reference maximum of every query row (log2 units)
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int pt = gridDim.x - 1 - blockIdx.x;
+    const int h = blockIdx.y, b = blockIdx.z;
+    const int L = p.L, W = p.window, g = p.Hq / p.Hkv;
+    const int qhead = b * p.Hq + h, kvhead = b * p.Hkv + h / g;
+    const int32_t* idx_row = p.vl_idx + (long)qhead * p.k;
+
+    if (threadIdx.x == 0) {
+        mbar_init(&bars.q_full, 1);
+        for (int s = 0; s < NST; ++s) {
+            mbar_init(&bars.k_full[s], 1);
+            mbar_init(&bars.k_free[s], QT);
+            mbar_init(&bars.v_full[s], 1);
+            mbar_init(&bars.v_free[s], QT);
+        }
+        for (int q = 0; q < QT; ++q) {
+            for (int bf = 0; bf < 2; ++bf) {
+                mbar_init(&bars.s_full[q][bf], 1);
+                mbar_init(&bars.p_full[q][bf], 4);
+                mbar_init(&bars.o_done[q][bf], 1);
+                mbar_init(&bars4.dec[q][bf], 4);
+            }
+            mbar_init(&bars4.fin[q], 8);
+        }
+        fence_mbar_init();
+        abort_s = 0;
+    }
+    if (threadIdx.x < QT) {
+        const int i1 = min(pt * QT * BM + (int)threadIdx.x * BM + BM - 1, L - 1);
+        cnt_b_s[threadIdx.x] = (p.k > 0 && i1 - W >= 0) ? count_le(idx_row, p.k, i1 - W) : 0;
+    }
+    if (warp == 16) {
+        tmem_alloc(&tmem_base_s, TM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = tmem_base_s;
+
+    auto make_sched = [&](int q) {
+        QSched s;
+        s.i0 = (pt * QT + q) * BM;
+        s.live = s.i0 < L;
+        s.i1 = min(s.i0 + BM - 1, L - 1);
+        s.nA = (s.live && s.i1 - W >= 0) ? (s.i1 - W) / BN + 1 : 0;
+        s.nB = s.live ? (cnt_b_s[q] + BN - 1) / BN : 0;
+        s.tC0 = max(0, s.i0 - W + 1) / BN;
+        s.tC1 = (s.live && W > 0) ? s.i1 / BN : -1;
+        return s;
+    };
+    const QSched qs0 = make_sched(0), qs1 = make_sched(1);
+    Walk w;
+    w.nA = max(qs0.nA, qs1.nA);
+    w.nB = max(qs0.nB, qs1.nB);
+    w.tC0 = qs0.tC0;
+    w.nC = (W > 0) ? max(qs0.tC1, qs1.tC1) - w.tC0 + 1 : 0;
+    w.T = w.nA + w.nB + w.nC;
+
+    volatile int* abort_flag = &abort_s;
+    auto fail = [&]() {
+        *abort_flag = 1;
+        if (p.status) atomicExch(p.status, HYQ_ERR_TIMEOUT);
+    };
+
+    if (warp == 16) {
+        if (lane == 0 && !tma_producer<TBN>(maps, qs0, qs1, w, qhead, kvhead, bars, smem, abort_flag)) fail();
+    } else if (warp == 17 || warp == 18) {
+        if (lane == 0) {
+            const int q = warp - 17;
+            if (!mma_issuer<LOWBIT_FP8, TBN>(q, q ? qs1 : qs0, w, bars, smem, tmem, abort_flag)) fail();
+        }
+    } else if (warp < 16) {
+        // ------------------------------------------------------------------ softmax groups
+        const int q = warp >> 3, wsel = (warp >> 2) & 1;        // query tile, group within the query tile
+        const QSched sq = q ? qs1 : qs0;
+        if (sq.live) {
+            const int r = (warp & 3) * 32 + lane;               // query row inside the tile = TMEM lane
+            const int i = sq.i0 + r;
+            const bool row_live = i < L;
+            const bool ragged = sq.i0 + BM > L;
+            const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+            const uint32_t to = tmem + tm_o(q) + lane_addr;
+            const uint32_t ts = tmem + tm_s(q) + wsel * BN + lane_addr;           // this group's S buffer
+            const uint32_t ts_other = tmem + tm_s(q) + (wsel ^ 1) * BN + lane_addr;
+            const float q_scale = row_live ? __ldg(p.q_scales + (long)qhead * p.nb + i / HYQ_BLOCK_TOKENS) : 0.0f;
+            const int cnt_r = (sq.nB > 0 && row_live && i - W >= 0) ? count_le(idx_row, p.k, i - W) : 0;
+            const uint32_t* bits_row = p.vl_bits + (long)qhead * p.mask_words;
+            const float* ks_row = p.k_scales + (long)kvhead * p.nb;
+            constexpr uint32_t knock_lq = LOWBIT_FP8 ? KNOCKOUT_F32 : KNOCKOUT_S32;
+            const OwnTiles own = own_tiles(sq, w);
+            const int n_total = own.a_end + (own.b_end - own.b_beg) + (own.c_end - own.c_beg);
+            float m_l = -INFINITY, l_w = 0.0f;                  // partial row sum and the reference it is relative to
+            bool ok = true;
+
+            for (int n = wsel; n < n_total && ok; n += 2) {
+                // walk position of own tile number n
+                int t = n;
+                if (t >= own.a_end) {
+                    t = own.b_beg + (n - own.a_end);
+                    if (t >= own.b_end) t = own.c_beg + (n - own.a_end - (own.b_end - own.b_beg));
+                }
+                // ---- per-tile column bounds, scale, vertical-line words
+                int lo = 0, hi = -1;
+                bool need_range;
+                float cs;
+                uint32_t vl0 = 0u, vl1 = 0u;
+                const bool lowbit = t < own.a_end;
+                if (lowbit) {
+                    const int j0 = t * BN;
+                    hi = row_live ? min(i - W - j0, BN - 1) : -1;
+                    need_range = (j0 + BN - 1 > sq.i0 - W) || ragged;
+                    // a zero scale (all-zero tile) still has to let -inf pass through the multiply
+                    cs = fmaxf(q_scale * __ldg(ks_row + min(t, p.nb - 1)) * p.scale_log2, 1e-37f);
+                    vl0 = (2 * t < p.mask_words) ? __ldg(bits_row + 2 * t) : 0u;
+                    vl1 = (2 * t + 1 < p.mask_words) ? __ldg(bits_row + 2 * t + 1) : 0u;
+                } else if (t < own.b_end) {
+                    const int c0 = (t - own.b_beg) * BN;
+                    hi = min(cnt_r - c0 - 1, BN - 1);
+                    need_range = true;
+                    cs = p.scale_log2;
+                } else {
+                    const int j0 = (w.tC0 + t - w.nA - w.nB) * BN;
+                    lo = max(0, i - W + 1 - j0);
+                    hi = row_live ? min(i - j0, BN - 1) : -1;
+                    need_range = (j0 + BN - 1 > sq.i0) || (j0 <= sq.i1 - W) || ragged;
+                    cs = p.scale_log2;
+                }
+                const bool int_scores = lowbit && !LOWBIT_FP8;
+                const uint32_t use_par = (uint32_t)(n >> 1) & 1u;
+
+                if (!mbar_wait(&bars.s_full[q][wsel], use_par, WAIT_LIMIT)) { ok = false; break; }
+                __syncwarp();
+                tc_fence_after();
+                if (need_range) {
+                    const int lo_eff = (hi >= lo) ? lo : 4096;
+                    const unsigned span = (hi >= lo) ? (unsigned)(hi - lo) : 0u;
+                    mask_tile_in_tmem<TBN>(ts, lo_eff, span, int_scores ? KNOCKOUT_S32 : KNOCKOUT_F32);
+                }
+                if ((vl0 | vl1) != 0u) {                        // uniform over the warp
+                    while (vl0) { const int c = __ffs(vl0) - 1; vl0 &= vl0 - 1; tmem_st1(ts + c, knock_lq); }
+                    while (vl1) { const int c = __ffs(vl1) - 1; vl1 &= vl1 - 1; tmem_st1(ts + 32 + c, knock_lq); }
+                    tmem_wait_st();
+                }
+                // ---- pass 1: row maximum of the tile
+                float f = -INFINITY;
+                if (int_scores) { f = chunk_max32<true>(ts, f); f = chunk_max32<true>(ts + 32, f); }
+                else { f = chunk_max32<false>(ts, f); f = chunk_max32<false>(ts + 32, f); }
+                const float mt = (f == -INFINITY) ? -INFINITY : f * cs;
+
+                // ---- decision, in tile order: does this tile raise the row's reference maximum?
+                float m_cur = -INFINITY;
+                if (n > 0) {
+                    if (!mbar_wait(&bars4.dec[q][wsel ^ 1], (uint32_t)((n - 1) >> 1) & 1u, WAIT_LIMIT)) { ok = false; break; }
+                    m_cur = m_ref_s[q][r];
+                }
+                const bool raise = mt > m_cur + RAISE_THRESHOLD;   // also true for the first finite maximum
+                if (__any_sync(0xffffffffu, raise)) {
+                    if (n > 0) {
+                        // P.V of tile n-1 (the other group's) must have landed before O is rescaled
+                        if (!mbar_wait(&bars.o_done[q][(n - 1) & 1], (uint32_t)((n - 1) >> 1) & 1u, WAIT_LIMIT)) { ok = false; break; }
+                        __syncwarp();
+                        tc_fence_after();
+                        const float alpha = raise ? ex2f(m_cur - mt) : 1.0f;      // m_cur = -inf -> 0
+#pragma unroll 1
+                        for (int c = 0; c < 4; ++c) {
+                            uint32_t o[32];
+                            tmem_ld32(to + c * 32, o);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+                            tmem_st32(to + c * 32, o);
+                        }
+                        tmem_wait_st();
+                    }
+                    if (raise) {
+                        m_cur = mt;
+                        m_ref_s[q][r] = mt;
+                    }
+                }
+                if (n == 0 && !raise) m_ref_s[q][r] = -INFINITY;   // first tile fully masked for this row
+                if (m_cur != m_l) {                                  // the reference moved since this group's last tile
+                    l_w = (m_l == -INFINITY) ? 0.0f : l_w * ex2f(m_l - m_cur);
+                    m_l = m_cur;
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bars4.dec[q][wsel]);
+
+                // ---- pass 2: P = 2^(s - m) as fp16 over the first 32 columns of the buffer; row sum
+                const float m_eff = (m_cur == -INFINITY) ? 0.0f : m_cur;
+                const float bias = int_scores ? fmaf(-INT_MAGIC_F, cs, -m_eff) : -m_eff;
+                float rs;
+                if (int_scores) { rs = chunk_exp32<true>(ts, ts, cs, bias); rs += chunk_exp32<true>(ts + 32, ts + 16, cs, bias); }
+                else { rs = chunk_exp32<false>(ts, ts, cs, bias); rs += chunk_exp32<false>(ts + 32, ts + 16, cs, bias); }
+                l_w += rs;
+                tmem_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bars.p_full[q][wsel]);
+            }
+
+            // ---- epilogue: the last P.V, exchange of the partial sums through TMEM, O / l
+            // A parity wait is only unambiguous for the completion that directly follows one already known to
+            // be done: first the P.V of this group's own last tile (the one two before it is done, since its
+            // scores were issued after it), then, if the other group holds the very last tile, that one.
+            {
+                const int n_last = (n_total - 1) - (((n_total - 1) & 1) != wsel ? 1 : 0);     // own last tile, or < 0
+                if (ok && n_last >= 0) ok = mbar_wait(&bars.o_done[q][n_last & 1], (uint32_t)(n_last >> 1) & 1u, WAIT_LIMIT);
+                if (ok && n_total > 0 && n_last != n_total - 1)
+                    ok = mbar_wait(&bars.o_done[q][(n_total - 1) & 1], (uint32_t)((n_total - 1) >> 1) & 1u, WAIT_LIMIT);
+            }
+            __syncwarp();
+            if (ok) {
+                tc_fence_after();
+                tmem_st1(ts, __float_as_uint(l_w));
+                tmem_st1(ts + 1, __float_as_uint(m_l));
+                tmem_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bars4.fin[q]);
+                ok = mbar_wait(&bars4.fin[q], 0, WAIT_LIMIT);
+            }
+            __syncwarp();
+            if (ok) {
+                tc_fence_after();
+                const float l_o = __uint_as_float(tmem_ld1(ts_other));
+                const float m_o = __uint_as_float(tmem_ld1(ts_other + 1));
+                tmem_wait_ld();
+                const float m_f = fmaxf(m_l, m_o);
+                const float l_run = ((m_l == -INFINITY) ? 0.0f : l_w * ex2f(m_l - m_f)) + ((m_o == -INFINITY) ? 0.0f : l_o * ex2f(m_o - m_f));
+                const float inv = (l_run > 0.0f) ? 1.0f / l_run : 0.0f;
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {                  // this group writes channels [64 wsel, 64 wsel + 64)
+                    uint32_t o[32];
+                    const int ch = wsel * 64 + c * 32;
+                    tmem_ld32(to + ch, o);
+                    tmem_wait_ld();
+                    if (row_live) {
+                        if (p.out_fp32) {
+                            float4* dst = reinterpret_cast<float4*>(static_cast<float*>(p.out) + ((long)qhead * L + i) * HYQ_D + ch);
+#pragma unroll
+                            for (int e = 0; e < 8; ++e)
+                                dst[e] = make_float4(__uint_as_float(o[4 * e]) * inv, __uint_as_float(o[4 * e + 1]) * inv,
+                                                     __uint_as_float(o[4 * e + 2]) * inv, __uint_as_float(o[4 * e + 3]) * inv);
+                        } else {
+                            uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.out) + ((long)qhead * L + i) * HYQ_D + ch);
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                uint32_t wd[4];
+#pragma unroll
+                                for (int q2 = 0; q2 < 4; ++q2) {
+                                    const __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(o[8 * e + 2 * q2]) * inv,
+                                                                                    __uint_as_float(o[8 * e + 2 * q2 + 1]) * inv);
+                                    wd[q2] = *reinterpret_cast<const uint32_t*>(&b2);
+                                }
+                                dst[e] = make_uint4(wd[0], wd[1], wd[2], wd[3]);
+                            }
+                        }
+                    }
+                }
+                if (p.lse && row_live && wsel == 0) p.lse[(long)qhead * L + i] = (m_f + log2f(l_run)) * 0.6931471805599453f;
+            } else {
+                fail();
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 16) {
+        __syncwarp();
+        tmem_dealloc(tmem, TM_COLS);
+    }
+}
+
 // ---------------------------------------------------------------------------------------------
 size_t attn_tc_workspace_bytes(const hyq_attn_args& a) { return tc_workspace_layout(a).total; }
+
+#ifndef HYQ_FOUR_GROUPS
+#define HYQ_FOUR_GROUPS 1
+#endif
+constexpr bool FOUR_GROUPS = HYQ_FOUR_GROUPS != 0;
 
 template <int TBN>
 static int launch_attn_tc_impl(const hyq_attn_args& a, float alpha, cudaStream_t st) {
@@ -693,12 +1068,14 @@ static int launch_attn_tc_impl(const hyq_attn_args& a, float alpha, cudaStream_t
     p.vl_bits = reinterpret_cast<const uint32_t*>(base + w.vl_bits);
     p.out = a.out; p.lse = a.lse; p.status = a.status_word;
 
-    auto kern = int4 ? attn_tc_kernel<true, TBN> : attn_tc_kernel<false, TBN>;
+    const bool four = FOUR_GROUPS && TBN == 64;
+    auto kern = four ? (int4 ? attn_tc4_kernel<true> : attn_tc4_kernel<false>)
+                     : (int4 ? attn_tc_kernel<true, TBN> : attn_tc_kernel<false, TBN>);
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM_BYTES) != cudaSuccess)
         return HYQ_ERR_CUDA;
     const dim3 grid((a.L + QT * BM - 1) / (QT * BM), a.Hq, a.B);
     if (a.ev_kernel_start && cudaEventRecord(static_cast<cudaEvent_t>(a.ev_kernel_start), st) != cudaSuccess) return HYQ_ERR_CUDA;
-    kern<<<grid, TC_THREADS, TC_SMEM_BYTES, st>>>(maps, p);
+    kern<<<grid, four ? TC4_THREADS : TC_THREADS, TC_SMEM_BYTES, st>>>(maps, p);
     if (launch_status() != HYQ_OK) return HYQ_ERR_CUDA;
     if (a.ev_kernel_stop && cudaEventRecord(static_cast<cudaEvent_t>(a.ev_kernel_stop), st) != cudaSuccess) return HYQ_ERR_CUDA;
     return HYQ_OK;
