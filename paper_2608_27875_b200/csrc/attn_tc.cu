@@ -22,6 +22,8 @@
 // status word and unwinds.
 #include <cuda_fp16.h>
 
+#include <type_traits>
+
 #include "attn_common.cuh"
 #include "sm100.cuh"
 
@@ -61,6 +63,21 @@ constexpr float INT_MAGIC_F = 12582912.0f;
 constexpr uint32_t KNOCKOUT_F32 = 0xFF800000u;       // -inf
 constexpr uint32_t KNOCKOUT_S32 = KNOCKOUT_F32 - INT_MAGIC;   // becomes -inf after the magic add
 
+// Optional timeline trace for tuning (compiled in with -DHYQ_TRACE): SM clock stamps of one CTA's softmax warps
+// (slots 0-3: query tile, column half) and MMA issuers (slots 4, 5) for own tiles 100..163, read back by
+// hyq_debug_read_trace.
+#ifdef HYQ_TRACE
+__device__ long long g_trace[6 * 64 * 8];
+#define HYQ_TR(slot, n, e)                                                                                  \
+    do {                                                                                                    \
+        if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && (threadIdx.x & 31) == 0 && (n) >= 100 && \
+            (n) < 164)                                                                                      \
+            g_trace[((slot) * 64 + ((n) - 100)) * 8 + (e)] = clock64();                                     \
+    } while (0)
+#else
+#define HYQ_TR(slot, n, e) do { } while (0)
+#endif
+
 struct TcMaps {
     CUtensorMap q, k, qc, kc, v16, vh16, kvl, vvl;
 };
@@ -79,7 +96,7 @@ struct TcParams {
 };
 
 struct TcBarriers {
-    uint64_t q_full, k_full[MAX_STAGES], k_free[MAX_STAGES], v_full[MAX_STAGES], v_free[MAX_STAGES];
+    uint64_t q_full, kv_full[MAX_STAGES], kv_free[MAX_STAGES];   // ring stage = K tile and V tile of one walk position
     uint64_t s_full[QT][2], p_full[QT][2], o_done[QT][2];
 };
 
@@ -289,8 +306,9 @@ __device__ __forceinline__ bool mma_issuer(int q, const QSched& sq, const Walk& 
     int tq = 0, kst = 0;
     uint32_t kpar = 0, n_qk = 0;
     auto qk = [&]() -> bool {
-        if (!mbar_wait(&bars.k_full[kst], kpar, WAIT_LIMIT)) return false;
+        if (!mbar_wait(&bars.kv_full[kst], kpar, WAIT_LIMIT)) return false;
         if (own.has(tq)) {
+            HYQ_TR(4 + q, (int)n_qk, 0);
             tc_fence_after();
             const uint64_t dk = dk0 + (uint64_t)(kst * STAGE16);
             const uint32_t buf = n_qk % NBUF;
@@ -308,35 +326,41 @@ __device__ __forceinline__ bool mma_issuer(int q, const QSched& sq, const Walk& 
                                 dk + ((kk >> 2) * (G::STAGE_BYTES / 32) + (kk & 3) * 2), idesc_qk, kk > 0);
             }
             umma_commit(&bars.s_full[q][buf]);
+            HYQ_TR(4 + q, (int)n_qk, 1);
             ++n_qk;
         }
-        umma_commit(&bars.k_free[kst]);             // one arrival per issuer; the ring slot is free after both
         ++tq;
         if (++kst == NST) { kst = 0; kpar ^= 1u; }
         return true;
     };
     // P.V cursor
     int vst = 0;
-    uint32_t vpar = 0, n_pv = 0;
+    uint32_t n_pv = 0;
     for (int t = 0; t < NBUF && t < T; ++t)
         if (!qk()) return false;
     for (int t = 0; t < T; ++t) {
-        if (!mbar_wait(&bars.v_full[vst], vpar, WAIT_LIMIT)) return false;
+        // (the V tile of position t came in on the same barrier as its K tile, which Q.K^T waited for)
         if (own.has(t)) {
             const uint32_t buf = n_pv % NBUF;
+            HYQ_TR(4 + q, (int)n_pv, 4);
             if (!mbar_wait(&bars.p_full[q][buf], (n_pv / NBUF) & 1u, WAIT_LIMIT)) return false;
+            HYQ_TR(4 + q, (int)n_pv, 5);
             tc_fence_after();
             const uint64_t dv = dv0 + (uint64_t)(vst * STAGE16);
             const uint32_t pa = ts0 + buf * BN;
 #pragma unroll
             for (int kk = 0; kk < BN / 16; ++kk) umma_ts_f16(to, pa + kk * 8, dv + kk * 128, idesc_pv, (n_pv > 0 || kk > 0));
             umma_commit(&bars.o_done[q][n_pv & 1u]);  // P.V number n of this query tile -> barrier n & 1
+            HYQ_TR(4 + q, (int)n_pv, 6);
             ++n_pv;
+            umma_commit(&bars.kv_free[vst]);        // one arrival per issuer; the ring stage is free after both
+            HYQ_TR(4 + q, (int)n_pv - 1, 7);
+        } else {
+            mbar_arrive(&bars.kv_free[vst]);        // nothing of this query tile reads the stage
         }
-        umma_commit(&bars.v_free[vst]);
-        if (++vst == NST) { vst = 0; vpar ^= 1u; }
+        if (++vst == NST) vst = 0;
         if (tq < T && !qk()) return false;
-        if (*abort_flag) return true;
+        if ((t & 15) == 15 && *abort_flag) return true;
     }
     return true;
 }
@@ -369,21 +393,19 @@ __device__ __forceinline__ bool tma_producer(const TcMaps& maps, const QSched& q
         const bool lowbit = t < w.nA, vl = !lowbit && t < w.nA + w.nB;
         const int row = lowbit ? t * BN : (vl ? (t - w.nA) * BN : (w.tC0 + t - w.nA - w.nB) * BN);
         const int hd = vl ? qhead : kvhead;
-        if (use > 0 && !mbar_wait(&bars.k_free[st], (use - 1) & 1, WAIT_LIMIT)) return false;
+        if (use > 0 && !mbar_wait(&bars.kv_free[st], (use - 1) & 1, WAIT_LIMIT)) return false;
         if (lowbit) {
-            mbar_arrive_expect_tx(&bars.k_full[st], G::KC_TILE_BYTES);
-            tma_load_3d(sk, &maps.kc, &bars.k_full[st], 0, row, hd);
+            mbar_arrive_expect_tx(&bars.kv_full[st], G::KC_TILE_BYTES + G::STAGE_BYTES);
+            tma_load_3d(sk, &maps.kc, &bars.kv_full[st], 0, row, hd);
         } else {
             const CUtensorMap* m = vl ? &maps.kvl : &maps.k;
-            mbar_arrive_expect_tx(&bars.k_full[st], G::STAGE_BYTES);
-            tma_load_3d(sk, m, &bars.k_full[st], 0, row, hd);
-            tma_load_3d(sk + G::STAGE_BYTES / 2, m, &bars.k_full[st], 64, row, hd);
+            mbar_arrive_expect_tx(&bars.kv_full[st], 2 * G::STAGE_BYTES);
+            tma_load_3d(sk, m, &bars.kv_full[st], 0, row, hd);
+            tma_load_3d(sk + G::STAGE_BYTES / 2, m, &bars.kv_full[st], 64, row, hd);
         }
-        if (use > 0 && !mbar_wait(&bars.v_free[st], (use - 1) & 1, WAIT_LIMIT)) return false;
         const CUtensorMap* m = lowbit ? &maps.vh16 : (vl ? &maps.vvl : &maps.v16);
-        mbar_arrive_expect_tx(&bars.v_full[st], G::STAGE_BYTES);
-        tma_load_3d(sv, m, &bars.v_full[st], 0, row, hd);
-        tma_load_3d(sv + G::STAGE_BYTES / 2, m, &bars.v_full[st], 64, row, hd);
+        tma_load_3d(sv, m, &bars.kv_full[st], 0, row, hd);
+        tma_load_3d(sv + G::STAGE_BYTES / 2, m, &bars.kv_full[st], 64, row, hd);
     }
     return true;
 }
@@ -410,10 +432,8 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
     if (threadIdx.x == 0) {
         mbar_init(&bars.q_full, 1);
         for (int s = 0; s < NST; ++s) {
-            mbar_init(&bars.k_full[s], 1);
-            mbar_init(&bars.k_free[s], QT);
-            mbar_init(&bars.v_full[s], 1);
-            mbar_init(&bars.v_free[s], QT);
+            mbar_init(&bars.kv_full[s], 1);
+            mbar_init(&bars.kv_free[s], QT);
         }
         for (int q = 0; q < QT; ++q) {
             for (int bf = 0; bf < 2; ++bf) {
@@ -665,30 +685,37 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
 }
 
 // =============================================================================================
-// Variant with FOUR softmax groups (64-key tiles only): each query tile is served by two warpgroups
-// that take its key tiles alternately (group w owns S buffer w), so that every scheduler hosts four
-// softmax warps instead of two and TMEM / barrier round trips of one warp hide under the arithmetic
-// of the others.  Both groups of a query tile exponentiate against one shared per-row reference
-// maximum (shared memory); the decision whether tile n raises it is taken in tile order:
-//   group of tile n: scores -> row maximum -> wait for the decision of tile n-1 -> raise? (then: wait
-//   for P.V of tile n-1, rescale O, publish the new reference) -> signal "decision n" -> exponentials.
-// A group's partial row sum is kept relative to the reference it last saw and rescaled when it changes;
-// the two partial sums are exchanged through TMEM at the end.  Registers: 96 per thread (608 threads), so
-// a tile is read twice from TMEM in 32-column chunks (maximum pass, exponential pass).
+// Variant with TWO THREADS PER QUERY ROW (64-key tiles): each query tile is served by eight softmax
+// warps; thread (r, h) owns columns [32 h, 32 h + 32) of row r of every score tile.  Every scheduler
+// then hosts four softmax warps instead of two, and a thread holds 32 scores instead of 64 (no
+// register spills at 96 registers per thread).  TMEM layout, MMA issue and TMA production are those of
+// the kernel above (two S buffers per query tile, P over the S columns it came from).
+// The two threads of a row must exponentiate against the same reference maximum.  Per tile they take
+// the maximum of their own half, and the eight warps of the query tile vote (named barrier with OR
+// reduction) whether any row has to raise its reference.  In the common case nobody does and each
+// half proceeds on its own; otherwise every thread also reads the other half's scores from TMEM, so
+// both threads of a row arrive at the same new reference, rescale their half of O (64 channels
+// each) and their partial row sum.  The vote also orders "both halves have read S" before
+// "either half writes P over it".  The partial sums are added at the end (exchange through TMEM).
 // =============================================================================================
-constexpr int TC4_THREADS = 608;                    // 16 softmax warps + TMA producer + 2 MMA issuers
+constexpr int TCP_THREADS = 640;                    // TMA producer, 2 MMA issuers, 1 idle warp, 16 softmax warps
 constexpr float RAISE_THRESHOLD = 8.0f;             // log2 units by which a tile must exceed the reference to raise it
 
-struct Tc4Barriers {
-    uint64_t dec[QT][2];        // decision of the tiles taken by group w of query tile q (4 arrivals: one per warp)
-    uint64_t fin[QT];           // both groups of query tile q have stored their partial sums (8 arrivals)
-};
+// named barrier over `nthreads` threads with an OR reduction of `pred` (all threads of the participating warps call it)
+__device__ __forceinline__ bool bar_red_or(int id, int nthreads, bool pred) {
+    uint32_t out;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 p, %3, 0;\n\tbar.red.or.pred q, %1, %2, p;\n\tselp.u32 %0, 1, 0, q;\n\t}\n"
+        : "=r"(out) : "r"(id), "r"(nthreads), "r"((uint32_t)pred) : "memory");
+    return out != 0;
+}
+__device__ __forceinline__ void bar_sync_named(int id, int nthreads) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
 
+// row maximum of 32 raw scores held in registers (integers are compared as integers)
 template <bool INT>
-__device__ __forceinline__ float chunk_max32(uint32_t ts, float m) {
-    uint32_t raw[32];
-    tmem_ld32(ts, raw);
-    tmem_wait_ld();
+__device__ __forceinline__ float row_max32(const uint32_t (&raw)[32]) {
     if (INT) {
         int m0 = (int)raw[0], m1 = (int)raw[1], m2 = (int)raw[2], m3 = (int)raw[3];
 #pragma unroll
@@ -699,7 +726,7 @@ __device__ __forceinline__ float chunk_max32(uint32_t ts, float m) {
             m3 = max(m3, (int)raw[e + 3]);
         }
         const int mm = max(max(m0, m1), max(m2, m3));
-        return fmaxf(m, (mm < -(1 << 23)) ? -INFINITY : (float)mm);
+        return (mm < -(1 << 23)) ? -INFINITY : (float)mm;      // knocked-out entries sit far below any score
     } else {
         float m0 = __uint_as_float(raw[0]), m1 = __uint_as_float(raw[1]), m2 = __uint_as_float(raw[2]), m3 = __uint_as_float(raw[3]);
 #pragma unroll
@@ -709,18 +736,14 @@ __device__ __forceinline__ float chunk_max32(uint32_t ts, float m) {
             m2 = fmaxf(m2, __uint_as_float(raw[e + 2]));
             m3 = fmaxf(m3, __uint_as_float(raw[e + 3]));
         }
-        return fmaxf(m, fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)));
+        return fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
     }
 }
 
-// exponentials of 32 score columns at ts_in, stored as 16 columns of fp16 pairs at ts_out; returns their fp32 sum
+// exponentials of 32 raw scores: pk receives the fp16 pairs of 2^(raw * sc + bias); returns their fp32 sum
 template <bool INT>
-__device__ __forceinline__ float chunk_exp32(uint32_t ts_in, uint32_t ts_out, float sc, float bias) {
-    uint32_t raw[32];
-    tmem_ld32(ts_in, raw);
-    tmem_wait_ld();
+__device__ __forceinline__ float row_exp32(const uint32_t (&raw)[32], float sc, float bias, uint32_t (&pk)[16]) {
     float a0 = 0.0f, a1 = 0.0f, a2 = 0.0f, a3 = 0.0f;
-    uint32_t pk[16];
 #pragma unroll
     for (int e = 0; e < 32; e += 4) {
         float pv[4];
@@ -734,26 +757,29 @@ __device__ __forceinline__ float chunk_exp32(uint32_t ts_in, uint32_t ts_out, fl
         pk[e >> 1] = *reinterpret_cast<const uint32_t*>(&h01);
         pk[(e >> 1) + 1] = *reinterpret_cast<const uint32_t*>(&h23);
     }
-    tmem_st16(ts_out, pk);
     return (a0 + a1) + (a2 + a3);
 }
 
+// columns [c0, c0 + 32) of a boundary tile: entries outside [lo_eff, lo_eff + span] of this row become `knock`
+__device__ __forceinline__ void mask_cols32(uint32_t (&raw)[32], int c0, int lo_eff, unsigned span, uint32_t knock) {
+#pragma unroll
+    for (int e = 0; e < 32; ++e) raw[e] = ((unsigned)(c0 + e - lo_eff) <= span) ? raw[e] : knock;
+}
+
 template <bool LOWBIT_FP8>
-__global__ void __launch_bounds__(TC4_THREADS, 1)
-attn_tc4_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
+__global__ void __launch_bounds__(TCP_THREADS, 1)
+attn_tcp_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
     constexpr int TBN = 64, BN = 64;
     using G = Geo<TBN>;
     constexpr int NST = G::NST;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     __shared__ TcBarriers bars;
-    __shared__ Tc4Barriers bars4;
     __shared__ uint32_t tmem_base_s;
-    __shared__ int abort_s, cnt_b_s[QT];
-    __shared__ float m_ref_s[QT][BM];               // reference maximum of every query row (log2 units)
+    __shared__ int abort_s, cnt_b_s[QT], grp_abort_s[QT];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int pt = gridDim.x - 1 - blockIdx.x;
+    const int pt = gridDim.x - 1 - blockIdx.x;               // pair of query tiles; longest rows first
     const int h = blockIdx.y, b = blockIdx.z;
     const int L = p.L, W = p.window, g = p.Hq / p.Hkv;
     const int qhead = b * p.Hq + h, kvhead = b * p.Hkv + h / g;
@@ -762,19 +788,16 @@ attn_tc4_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
     if (threadIdx.x == 0) {
         mbar_init(&bars.q_full, 1);
         for (int s = 0; s < NST; ++s) {
-            mbar_init(&bars.k_full[s], 1);
-            mbar_init(&bars.k_free[s], QT);
-            mbar_init(&bars.v_full[s], 1);
-            mbar_init(&bars.v_free[s], QT);
+            mbar_init(&bars.kv_full[s], 1);
+            mbar_init(&bars.kv_free[s], QT);
         }
         for (int q = 0; q < QT; ++q) {
             for (int bf = 0; bf < 2; ++bf) {
                 mbar_init(&bars.s_full[q][bf], 1);
-                mbar_init(&bars.p_full[q][bf], 4);
+                mbar_init(&bars.p_full[q][bf], 8);           // one arrival per softmax warp of the query tile
                 mbar_init(&bars.o_done[q][bf], 1);
-                mbar_init(&bars4.dec[q][bf], 4);
             }
-            mbar_init(&bars4.fin[q], 8);
+            grp_abort_s[q] = 0;
         }
         fence_mbar_init();
         abort_s = 0;
@@ -783,7 +806,7 @@ attn_tc4_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
         const int i1 = min(pt * QT * BM + (int)threadIdx.x * BM + BM - 1, L - 1);
         cnt_b_s[threadIdx.x] = (p.k > 0 && i1 - W >= 0) ? count_le(idx_row, p.k, i1 - W) : 0;
     }
-    if (warp == 16) {
+    if (warp == 0) {
         tmem_alloc(&tmem_base_s, TM_COLS);
         tmem_relinquish();
     }
@@ -817,212 +840,246 @@ attn_tc4_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
         if (p.status) atomicExch(p.status, HYQ_ERR_TIMEOUT);
     };
 
-    if (warp == 16) {
+    // the single-thread roles sit in the lowest warps (the softmax warps 4..19 keep warp % 4 = TMEM lane quarter)
+    if (warp == 0) {
         if (lane == 0 && !tma_producer<TBN>(maps, qs0, qs1, w, qhead, kvhead, bars, smem, abort_flag)) fail();
-    } else if (warp == 17 || warp == 18) {
+    } else if (warp == 1 || warp == 2) {
         if (lane == 0) {
-            const int q = warp - 17;
+            const int q = warp - 1;
             if (!mma_issuer<LOWBIT_FP8, TBN>(q, q ? qs1 : qs0, w, bars, smem, tmem, abort_flag)) fail();
         }
-    } else if (warp < 16) {
-        // ------------------------------------------------------------------ softmax groups
-        const int q = warp >> 3, wsel = (warp >> 2) & 1;        // query tile, group within the query tile
+    } else if (warp >= 4) {
+        // ------------------------------------------------------------------ softmax warps
+        const int q = (warp - 4) >> 3, hsel = ((warp - 4) >> 2) & 1;    // query tile, column half
         const QSched sq = q ? qs1 : qs0;
-        if (sq.live) {
+        const int bar_id = 1 + q;                               // named barrier of this query tile's 256 softmax threads
+        const OwnTiles own = own_tiles(sq, w);
+        const int n_total = own.a_end + (own.b_end - own.b_beg) + (own.c_end - own.c_beg);
+        if (sq.live && n_total > 0) {
             const int r = (warp & 3) * 32 + lane;               // query row inside the tile = TMEM lane
             const int i = sq.i0 + r;
             const bool row_live = i < L;
             const bool ragged = sq.i0 + BM > L;
+            const int col0 = hsel * 32, col0_other = col0 ^ 32;
             const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
-            const uint32_t to = tmem + tm_o(q) + lane_addr;
-            const uint32_t ts = tmem + tm_s(q) + wsel * BN + lane_addr;           // this group's S buffer
-            const uint32_t ts_other = tmem + tm_s(q) + (wsel ^ 1) * BN + lane_addr;
+            const uint32_t to = tmem + tm_o(q) + lane_addr, ts0 = tmem + tm_s(q) + lane_addr;
             const float q_scale = row_live ? __ldg(p.q_scales + (long)qhead * p.nb + i / HYQ_BLOCK_TOKENS) : 0.0f;
             const int cnt_r = (sq.nB > 0 && row_live && i - W >= 0) ? count_le(idx_row, p.k, i - W) : 0;
-            const uint32_t* bits_row = p.vl_bits + (long)qhead * p.mask_words;
-            const float* ks_row = p.k_scales + (long)kvhead * p.nb;
             constexpr uint32_t knock_lq = LOWBIT_FP8 ? KNOCKOUT_F32 : KNOCKOUT_S32;
-            const OwnTiles own = own_tiles(sq, w);
-            const int n_total = own.a_end + (own.b_end - own.b_beg) + (own.c_end - own.c_beg);
-            float m_l = -INFINITY, l_w = 0.0f;                  // partial row sum and the reference it is relative to
-            bool ok = true;
+            float m_used = -INFINITY, l_h = 0.0f;               // reference maximum of the row; row sum of this half
+            bool dead = false;                                  // this warp ran into an expired wait
+            bool aborted = false;
 
-            for (int n = wsel; n < n_total && ok; n += 2) {
-                // walk position of own tile number n
-                int t = n;
-                if (t >= own.a_end) {
-                    t = own.b_beg + (n - own.a_end);
-                    if (t >= own.b_end) t = own.c_beg + (n - own.a_end - (own.b_end - own.b_beg));
+            // walk position of own tile number n
+            auto walk_pos = [&](int n) -> int {
+                if (n < own.a_end) return n;
+                const int tb = own.b_beg + (n - own.a_end);
+                return (tb < own.b_end) ? tb : own.c_beg + (n - own.a_end - (own.b_end - own.b_beg));
+            };
+            // K scale and this half's vertical-line bitmask word of a low-bit tile, fetched one tile ahead of their use
+            // (tile n of the low-bit pass sits at walk position n; its block and mask words exist for n < a_end)
+            const float* ks_ptr = p.k_scales + (long)kvhead * p.nb;
+            const uint32_t* vl_ptr = p.vl_bits + (long)qhead * p.mask_words + hsel;
+            float nks = 0.0f;
+            uint32_t nvl = 0u;
+            auto prefetch_tile = [&](int n) {
+                nks = 0.0f; nvl = 0u;
+                if (n >= own.a_end) return;
+                nks = __ldg(ks_ptr + n);
+                nvl = __ldg(vl_ptr + 2 * n);
+            };
+            prefetch_tile(0);
+            const float qs2 = q_scale * p.scale_log2;
+
+            // one tile of the online softmax for this thread's 32 columns.  Returns false when the query tile's
+            // softmax warps leave the loop together (an expired wait somewhere).
+            auto do_tile = [&](auto range_tag, int n, float cs, uint32_t vl, bool int_scores, int lo_eff, unsigned span) -> bool {
+                constexpr bool NEED_RANGE = decltype(range_tag)::value;
+                const uint32_t knock = int_scores ? KNOCKOUT_S32 : KNOCKOUT_F32;
+                const int buf = n & 1;
+                const uint32_t ts = ts0 + buf * BN;
+                uint32_t raw[32];
+                float mt = -INFINITY;
+                HYQ_TR(q * 2 + hsel, n, 0);
+                if (!dead && !__all_sync(0xffffffffu, mbar_wait(&bars.s_full[q][buf], (uint32_t)(n >> 1) & 1u, WAIT_LIMIT))) {
+                    dead = true;
+                    grp_abort_s[q] = 1;
                 }
-                // ---- per-tile column bounds, scale, vertical-line words
+                __syncwarp();
+                HYQ_TR(q * 2 + hsel, n, 1);
+                if (!dead) {
+                    tc_fence_after();
+                    // vertical-line keys of a low-bit tile: -inf into their S columns before the half is read
+                    if (vl != 0u) {                              // uniform over the warp
+                        while (vl) { const int c = __ffs(vl) - 1; vl &= vl - 1; tmem_st1(ts + col0 + c, knock_lq); }
+                        tmem_wait_st();
+                    }
+                    tmem_ld32(ts + col0, raw);
+                    tmem_wait_ld();
+                    if (NEED_RANGE) mask_cols32(raw, col0, lo_eff, span, knock);
+                    const float f = int_scores ? row_max32<true>(raw) : row_max32<false>(raw);
+                    mt = (f == -INFINITY) ? -INFINITY : f * cs;
+                }
+                // ---- vote: does any row of this query tile have to raise its reference maximum?
+                // (also: both halves have read their scores before either writes P over them)
+                tc_fence_before();
+                HYQ_TR(q * 2 + hsel, n, 3);
+                const bool any_raise = bar_red_or(bar_id, 256, dead || mt > m_used + RAISE_THRESHOLD);
+                HYQ_TR(q * 2 + hsel, n, 4);
+                if (any_raise) {
+                    if (*reinterpret_cast<volatile int*>(&grp_abort_s[q])) return false;
+                    tc_fence_after();
+                    // the other half's maximum, from its scores in TMEM (same knock-outs, same range mask)
+                    float mo;
+                    {
+                        uint32_t oth[32];
+                        tmem_ld32(ts + col0_other, oth);
+                        tmem_wait_ld();
+                        if (NEED_RANGE) mask_cols32(oth, col0_other, lo_eff, span, knock);
+                        const float fo = int_scores ? row_max32<true>(oth) : row_max32<false>(oth);
+                        mo = (fo == -INFINITY) ? -INFINITY : fo * cs;
+                    }
+                    tc_fence_before();
+                    bar_sync_named(bar_id, 256);                 // both halves are done reading before P is written
+                    const float m_new = fmaxf(mt, mo);
+                    const bool raise = m_new > m_used + RAISE_THRESHOLD;     // same verdict in both threads of the row
+                    const float alpha = raise ? ex2f(m_used - m_new) : 1.0f; // m_used = -inf -> 0
+                    if (n > 0 && __any_sync(0xffffffffu, raise)) {
+                        // P.V of tile n-1 must have landed before O is rescaled.  P.V number m signals barrier m & 1;
+                        // the one before the previous is complete (the scores just read were issued after it), so
+                        // the parity wait cannot alias.
+                        if (!__all_sync(0xffffffffu, mbar_wait(&bars.o_done[q][(n - 1) & 1], (uint32_t)((n - 1) >> 1) & 1u, WAIT_LIMIT))) {
+                            dead = true;
+                            grp_abort_s[q] = 1;
+                        } else {
+                            tc_fence_after();
+#pragma unroll 1
+                            for (int c = 0; c < 4; ++c) {       // this half rescales channels [64 hsel, 64 hsel + 64)
+                                uint32_t o[16];
+                                tmem_ld16(to + hsel * 64 + c * 16, o);
+                                tmem_wait_ld();
+#pragma unroll
+                                for (int e = 0; e < 16; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+                                tmem_st16(to + hsel * 64 + c * 16, o);
+                            }
+                            tmem_wait_st();
+                        }
+                    }
+                    if (raise) {
+                        l_h *= alpha;
+                        m_used = m_new;
+                    }
+                }
+                // ---- P = 2^(s - m) as fp16 pairs over the first 32 columns of the buffer; row sum of this half
+                if (!dead) {
+                    const float m_eff = (m_used == -INFINITY) ? 0.0f : m_used;
+                    const float bias = int_scores ? fmaf(-INT_MAGIC_F, cs, -m_eff) : -m_eff;
+                    uint32_t pk[16];
+                    l_h += int_scores ? row_exp32<true>(raw, cs, bias, pk) : row_exp32<false>(raw, cs, bias, pk);
+                    HYQ_TR(q * 2 + hsel, n, 5);
+                    tmem_st16(ts + hsel * 16, pk);
+                    tmem_wait_st();
+                    tc_fence_before();
+                    __syncwarp();
+                    HYQ_TR(q * 2 + hsel, n, 6);
+                    if (lane == 0) mbar_arrive(&bars.p_full[q][buf]);
+                    HYQ_TR(q * 2 + hsel, n, 7);
+                }
+                return true;
+            };
+
+            // ---- low-bit tiles that lie wholly below every row's window: no range mask, no bounds to compute
+            const int n_plain = ragged ? 0 : min(own.a_end, max(0, (sq.i0 - W + 1) / BN));
+            int n = 0;
+            for (; n < n_plain; ++n) {
+                HYQ_TR(q * 2 + hsel, n, 2);
+                // a zero scale (all-zero tile) still has to let -inf pass through the multiply
+                const float cs = fmaxf(qs2 * nks, 1e-37f);
+                const uint32_t vl = nvl;
+                prefetch_tile(n + 1);
+                if (!do_tile(std::false_type{}, n, cs, vl, !LOWBIT_FP8, 0, 0u)) { aborted = true; break; }
+            }
+            // ---- the remaining low-bit tiles, the vertical-line tiles and the window tiles
+            for (; n < n_total && !aborted; ++n) {
+                HYQ_TR(q * 2 + hsel, n, 2);
+                const int t = walk_pos(n);
+                const float ks = nks;
+                const uint32_t vl = nvl;
+                prefetch_tile(n + 1);
                 int lo = 0, hi = -1;
-                bool need_range;
                 float cs;
-                uint32_t vl0 = 0u, vl1 = 0u;
                 const bool lowbit = t < own.a_end;
                 if (lowbit) {
-                    const int j0 = t * BN;
-                    hi = row_live ? min(i - W - j0, BN - 1) : -1;
-                    need_range = (j0 + BN - 1 > sq.i0 - W) || ragged;
-                    // a zero scale (all-zero tile) still has to let -inf pass through the multiply
-                    cs = fmaxf(q_scale * __ldg(ks_row + min(t, p.nb - 1)) * p.scale_log2, 1e-37f);
-                    vl0 = (2 * t < p.mask_words) ? __ldg(bits_row + 2 * t) : 0u;
-                    vl1 = (2 * t + 1 < p.mask_words) ? __ldg(bits_row + 2 * t + 1) : 0u;
+                    hi = row_live ? min(i - W - t * BN, BN - 1) : -1;
+                    cs = fmaxf(qs2 * ks, 1e-37f);
                 } else if (t < own.b_end) {
-                    const int c0 = (t - own.b_beg) * BN;
-                    hi = min(cnt_r - c0 - 1, BN - 1);
-                    need_range = true;
+                    hi = min(cnt_r - (t - own.b_beg) * BN - 1, BN - 1);
                     cs = p.scale_log2;
                 } else {
                     const int j0 = (w.tC0 + t - w.nA - w.nB) * BN;
                     lo = max(0, i - W + 1 - j0);
                     hi = row_live ? min(i - j0, BN - 1) : -1;
-                    need_range = (j0 + BN - 1 > sq.i0) || (j0 <= sq.i1 - W) || ragged;
                     cs = p.scale_log2;
                 }
-                const bool int_scores = lowbit && !LOWBIT_FP8;
-                const uint32_t use_par = (uint32_t)(n >> 1) & 1u;
+                const int lo_eff = (hi >= lo) ? lo : 4096;
+                const unsigned span = (hi >= lo) ? (unsigned)(hi - lo) : 0u;
+                if (!do_tile(std::true_type{}, n, cs, vl, lowbit && !LOWBIT_FP8, lo_eff, span)) aborted = true;
+            }
 
-                if (!mbar_wait(&bars.s_full[q][wsel], use_par, WAIT_LIMIT)) { ok = false; break; }
-                __syncwarp();
+            // ---- epilogue: the last P.V (MMAs complete in order), sum of the two halves' row sums, O / l
+            bool ok = !aborted && !dead;
+            if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars.o_done[q][(n_total - 1) & 1], (uint32_t)((n_total - 1) >> 1) & 1u, WAIT_LIMIT));
+            if (!aborted) {                                     // uniform over the query tile's softmax warps
                 tc_fence_after();
-                if (need_range) {
-                    const int lo_eff = (hi >= lo) ? lo : 4096;
-                    const unsigned span = (hi >= lo) ? (unsigned)(hi - lo) : 0u;
-                    mask_tile_in_tmem<TBN>(ts, lo_eff, span, int_scores ? KNOCKOUT_S32 : KNOCKOUT_F32);
-                }
-                if ((vl0 | vl1) != 0u) {                        // uniform over the warp
-                    while (vl0) { const int c = __ffs(vl0) - 1; vl0 &= vl0 - 1; tmem_st1(ts + c, knock_lq); }
-                    while (vl1) { const int c = __ffs(vl1) - 1; vl1 &= vl1 - 1; tmem_st1(ts + 32 + c, knock_lq); }
-                    tmem_wait_st();
-                }
-                // ---- pass 1: row maximum of the tile
-                float f = -INFINITY;
-                if (int_scores) { f = chunk_max32<true>(ts, f); f = chunk_max32<true>(ts + 32, f); }
-                else { f = chunk_max32<false>(ts, f); f = chunk_max32<false>(ts + 32, f); }
-                const float mt = (f == -INFINITY) ? -INFINITY : f * cs;
-
-                // ---- decision, in tile order: does this tile raise the row's reference maximum?
-                float m_cur = -INFINITY;
-                if (n > 0) {
-                    if (!mbar_wait(&bars4.dec[q][wsel ^ 1], (uint32_t)((n - 1) >> 1) & 1u, WAIT_LIMIT)) { ok = false; break; }
-                    m_cur = m_ref_s[q][r];
-                }
-                const bool raise = mt > m_cur + RAISE_THRESHOLD;   // also true for the first finite maximum
-                if (__any_sync(0xffffffffu, raise)) {
-                    if (n > 0) {
-                        // P.V of tile n-1 (the other group's) must have landed before O is rescaled
-                        if (!mbar_wait(&bars.o_done[q][(n - 1) & 1], (uint32_t)((n - 1) >> 1) & 1u, WAIT_LIMIT)) { ok = false; break; }
-                        __syncwarp();
-                        tc_fence_after();
-                        const float alpha = raise ? ex2f(m_cur - mt) : 1.0f;      // m_cur = -inf -> 0
-#pragma unroll 1
-                        for (int c = 0; c < 4; ++c) {
-                            uint32_t o[32];
-                            tmem_ld32(to + c * 32, o);
-                            tmem_wait_ld();
-#pragma unroll
-                            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-                            tmem_st32(to + c * 32, o);
-                        }
-                        tmem_wait_st();
-                    }
-                    if (raise) {
-                        m_cur = mt;
-                        m_ref_s[q][r] = mt;
-                    }
-                }
-                if (n == 0 && !raise) m_ref_s[q][r] = -INFINITY;   // first tile fully masked for this row
-                if (m_cur != m_l) {                                  // the reference moved since this group's last tile
-                    l_w = (m_l == -INFINITY) ? 0.0f : l_w * ex2f(m_l - m_cur);
-                    m_l = m_cur;
-                }
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&bars4.dec[q][wsel]);
-
-                // ---- pass 2: P = 2^(s - m) as fp16 over the first 32 columns of the buffer; row sum
-                const float m_eff = (m_cur == -INFINITY) ? 0.0f : m_cur;
-                const float bias = int_scores ? fmaf(-INT_MAGIC_F, cs, -m_eff) : -m_eff;
-                float rs;
-                if (int_scores) { rs = chunk_exp32<true>(ts, ts, cs, bias); rs += chunk_exp32<true>(ts + 32, ts + 16, cs, bias); }
-                else { rs = chunk_exp32<false>(ts, ts, cs, bias); rs += chunk_exp32<false>(ts + 32, ts + 16, cs, bias); }
-                l_w += rs;
+                tmem_st1(ts0 + col0, __float_as_uint(l_h));     // column col0 of S buffer 0 (all MMAs are done)
                 tmem_wait_st();
                 tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&bars.p_full[q][wsel]);
-            }
-
-            // ---- epilogue: the last P.V, exchange of the partial sums through TMEM, O / l
-            // A parity wait is only unambiguous for the completion that directly follows one already known to
-            // be done: first the P.V of this group's own last tile (the one two before it is done, since its
-            // scores were issued after it), then, if the other group holds the very last tile, that one.
-            {
-                const int n_last = (n_total - 1) - (((n_total - 1) & 1) != wsel ? 1 : 0);     // own last tile, or < 0
-                if (ok && n_last >= 0) ok = mbar_wait(&bars.o_done[q][n_last & 1], (uint32_t)(n_last >> 1) & 1u, WAIT_LIMIT);
-                if (ok && n_total > 0 && n_last != n_total - 1)
-                    ok = mbar_wait(&bars.o_done[q][(n_total - 1) & 1], (uint32_t)((n_total - 1) >> 1) & 1u, WAIT_LIMIT);
-            }
-            __syncwarp();
-            if (ok) {
+                bar_sync_named(bar_id, 256);
                 tc_fence_after();
-                tmem_st1(ts, __float_as_uint(l_w));
-                tmem_st1(ts + 1, __float_as_uint(m_l));
-                tmem_wait_st();
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&bars4.fin[q]);
-                ok = mbar_wait(&bars4.fin[q], 0, WAIT_LIMIT);
-            }
-            __syncwarp();
-            if (ok) {
-                tc_fence_after();
-                const float l_o = __uint_as_float(tmem_ld1(ts_other));
-                const float m_o = __uint_as_float(tmem_ld1(ts_other + 1));
+                const float l_o = __uint_as_float(tmem_ld1(ts0 + col0_other));
                 tmem_wait_ld();
-                const float m_f = fmaxf(m_l, m_o);
-                const float l_run = ((m_l == -INFINITY) ? 0.0f : l_w * ex2f(m_l - m_f)) + ((m_o == -INFINITY) ? 0.0f : l_o * ex2f(m_o - m_f));
+                const float l_run = l_h + l_o;
                 const float inv = (l_run > 0.0f) ? 1.0f / l_run : 0.0f;
+                if (ok) {
 #pragma unroll
-                for (int c = 0; c < 2; ++c) {                  // this group writes channels [64 wsel, 64 wsel + 64)
-                    uint32_t o[32];
-                    const int ch = wsel * 64 + c * 32;
-                    tmem_ld32(to + ch, o);
-                    tmem_wait_ld();
-                    if (row_live) {
-                        if (p.out_fp32) {
-                            float4* dst = reinterpret_cast<float4*>(static_cast<float*>(p.out) + ((long)qhead * L + i) * HYQ_D + ch);
+                    for (int c = 0; c < 2; ++c) {              // this half writes channels [64 hsel, 64 hsel + 64)
+                        uint32_t o[32];
+                        const int ch = hsel * 64 + c * 32;
+                        tmem_ld32(to + ch, o);
+                        tmem_wait_ld();
+                        if (row_live) {
+                            if (p.out_fp32) {
+                                float4* dst = reinterpret_cast<float4*>(static_cast<float*>(p.out) + ((long)qhead * L + i) * HYQ_D + ch);
 #pragma unroll
-                            for (int e = 0; e < 8; ++e)
-                                dst[e] = make_float4(__uint_as_float(o[4 * e]) * inv, __uint_as_float(o[4 * e + 1]) * inv,
-                                                     __uint_as_float(o[4 * e + 2]) * inv, __uint_as_float(o[4 * e + 3]) * inv);
-                        } else {
-                            uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.out) + ((long)qhead * L + i) * HYQ_D + ch);
+                                for (int e = 0; e < 8; ++e)
+                                    dst[e] = make_float4(__uint_as_float(o[4 * e]) * inv, __uint_as_float(o[4 * e + 1]) * inv,
+                                                         __uint_as_float(o[4 * e + 2]) * inv, __uint_as_float(o[4 * e + 3]) * inv);
+                            } else {
+                                uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.out) + ((long)qhead * L + i) * HYQ_D + ch);
 #pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                uint32_t wd[4];
+                                for (int e = 0; e < 4; ++e) {
+                                    uint32_t wd[4];
 #pragma unroll
-                                for (int q2 = 0; q2 < 4; ++q2) {
-                                    const __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(o[8 * e + 2 * q2]) * inv,
-                                                                                    __uint_as_float(o[8 * e + 2 * q2 + 1]) * inv);
-                                    wd[q2] = *reinterpret_cast<const uint32_t*>(&b2);
+                                    for (int q2 = 0; q2 < 4; ++q2) {
+                                        const __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(o[8 * e + 2 * q2]) * inv,
+                                                                                        __uint_as_float(o[8 * e + 2 * q2 + 1]) * inv);
+                                        wd[q2] = *reinterpret_cast<const uint32_t*>(&b2);
+                                    }
+                                    dst[e] = make_uint4(wd[0], wd[1], wd[2], wd[3]);
                                 }
-                                dst[e] = make_uint4(wd[0], wd[1], wd[2], wd[3]);
                             }
                         }
                     }
+                    if (p.lse && row_live && hsel == 0) p.lse[(long)qhead * L + i] = (m_used + log2f(l_run)) * 0.6931471805599453f;
                 }
-                if (p.lse && row_live && wsel == 0) p.lse[(long)qhead * L + i] = (m_f + log2f(l_run)) * 0.6931471805599453f;
-            } else {
-                fail();
             }
+            if (!ok) fail();
         }
     }
 
     tc_fence_before();
     __syncthreads();
-    if (warp == 16) {
+    if (warp == 0) {
         __syncwarp();
         tmem_dealloc(tmem, TM_COLS);
     }
@@ -1031,10 +1088,11 @@ attn_tc4_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
 // ---------------------------------------------------------------------------------------------
 size_t attn_tc_workspace_bytes(const hyq_attn_args& a) { return tc_workspace_layout(a).total; }
 
-#ifndef HYQ_FOUR_GROUPS
-#define HYQ_FOUR_GROUPS 1
+// which kernel serves 64-key tiles: two threads per query row (default), or one thread per row
+#ifndef HYQ_PAIRED_ROWS
+#define HYQ_PAIRED_ROWS 1
 #endif
-constexpr bool FOUR_GROUPS = HYQ_FOUR_GROUPS != 0;
+constexpr bool PAIRED_ROWS = HYQ_PAIRED_ROWS != 0;
 
 template <int TBN>
 static int launch_attn_tc_impl(const hyq_attn_args& a, float alpha, cudaStream_t st) {
@@ -1068,14 +1126,14 @@ static int launch_attn_tc_impl(const hyq_attn_args& a, float alpha, cudaStream_t
     p.vl_bits = reinterpret_cast<const uint32_t*>(base + w.vl_bits);
     p.out = a.out; p.lse = a.lse; p.status = a.status_word;
 
-    const bool four = FOUR_GROUPS && TBN == 64;
-    auto kern = four ? (int4 ? attn_tc4_kernel<true> : attn_tc4_kernel<false>)
-                     : (int4 ? attn_tc_kernel<true, TBN> : attn_tc_kernel<false, TBN>);
+    const bool paired = PAIRED_ROWS && TBN == 64;
+    auto kern = paired ? (int4 ? attn_tcp_kernel<true> : attn_tcp_kernel<false>)
+                       : (int4 ? attn_tc_kernel<true, TBN> : attn_tc_kernel<false, TBN>);
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM_BYTES) != cudaSuccess)
         return HYQ_ERR_CUDA;
     const dim3 grid((a.L + QT * BM - 1) / (QT * BM), a.Hq, a.B);
     if (a.ev_kernel_start && cudaEventRecord(static_cast<cudaEvent_t>(a.ev_kernel_start), st) != cudaSuccess) return HYQ_ERR_CUDA;
-    kern<<<grid, four ? TC4_THREADS : TC_THREADS, TC_SMEM_BYTES, st>>>(maps, p);
+    kern<<<grid, paired ? TCP_THREADS : TC_THREADS, TC_SMEM_BYTES, st>>>(maps, p);
     if (launch_status() != HYQ_OK) return HYQ_ERR_CUDA;
     if (a.ev_kernel_stop && cudaEventRecord(static_cast<cudaEvent_t>(a.ev_kernel_stop), st) != cudaSuccess) return HYQ_ERR_CUDA;
     return HYQ_OK;
@@ -1086,3 +1144,9 @@ static int launch_attn_tc_impl(const hyq_attn_args& a, float alpha, cudaStream_t
 int launch_attn_tc(const hyq_attn_args& a, float alpha, cudaStream_t st) { return launch_attn_tc_impl<64>(a, alpha, st); }
 
 }  // namespace hyq
+
+#ifdef HYQ_TRACE
+extern "C" int hyq_debug_read_trace(long long* dst) {
+    return cudaMemcpyFromSymbol(dst, hyq::g_trace, sizeof(hyq::g_trace)) == cudaSuccess ? 0 : 1;
+}
+#endif
