@@ -305,8 +305,9 @@ __device__ __forceinline__ bool mma_issuer(int q, const QSched& sq, const Walk& 
     // Q.K^T cursor
     int tq = 0, kst = 0;
     uint32_t kpar = 0, n_qk = 0;
-    auto qk = [&]() -> bool {
-        if (!mbar_wait(&bars.kv_full[kst], kpar, WAIT_LIMIT)) return false;
+    // (k_ready: the stage of position tq is already known to have landed)
+    auto qk = [&](bool k_ready) -> bool {
+        if (!k_ready && !mbar_wait(&bars.kv_full[kst], kpar, WAIT_LIMIT)) return false;
         if (own.has(tq)) {
             HYQ_TR(4 + q, (int)n_qk, 0);
             tc_fence_after();
@@ -337,13 +338,17 @@ __device__ __forceinline__ bool mma_issuer(int q, const QSched& sq, const Walk& 
     int vst = 0;
     uint32_t n_pv = 0;
     for (int t = 0; t < NBUF && t < T; ++t)
-        if (!qk()) return false;
+        if (!qk(false)) return false;
     for (int t = 0; t < T; ++t) {
         // (the V tile of position t came in on the same barrier as its K tile, which Q.K^T waited for)
+        bool k_ready = false;
         if (own.has(t)) {
             const uint32_t buf = n_pv % NBUF;
             HYQ_TR(4 + q, (int)n_pv, 4);
-            if (!mbar_wait(&bars.p_full[q][buf], (n_pv / NBUF) & 1u, WAIT_LIMIT)) return false;
+            // P of this tile, and in the same round trip the ring stage of the Q.K^T that follows
+            const uint32_t done = mbar_test_wait2(&bars.p_full[q][buf], (n_pv / NBUF) & 1u, &bars.kv_full[kst], kpar);
+            k_ready = (done & 2u) != 0u && tq < T;
+            if (!(done & 1u) && !mbar_wait(&bars.p_full[q][buf], (n_pv / NBUF) & 1u, WAIT_LIMIT)) return false;
             HYQ_TR(4 + q, (int)n_pv, 5);
             tc_fence_after();
             const uint64_t dv = dv0 + (uint64_t)(vst * STAGE16);
@@ -359,7 +364,7 @@ __device__ __forceinline__ bool mma_issuer(int q, const QSched& sq, const Walk& 
             mbar_arrive(&bars.kv_free[vst]);        // nothing of this query tile reads the stage
         }
         if (++vst == NST) vst = 0;
-        if (tq < T && !qk()) return false;
+        if (tq < T && !qk(k_ready)) return false;
         if ((t & 15) == 15 && *abort_flag) return true;
     }
     return true;

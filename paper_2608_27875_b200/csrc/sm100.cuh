@@ -51,6 +51,19 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, long l
     return true;
 }
 
+// Tests two barriers back to back, so that the two shared-memory round trips overlap (a single-thread MMA issuer
+// pays one latency instead of two): bit 0 / bit 1 of the result = phase with parity0 / parity1 complete.
+__device__ __forceinline__ uint32_t mbar_test_wait2(uint64_t* bar0, uint32_t parity0, uint64_t* bar1, uint32_t parity1) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred P, Q;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 P, [%1], %2;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 Q, [%3], %4;\n\t"
+        "selp.u32 %0, 1, 0, P;\n\t@Q or.b32 %0, %0, 2;\n\t}\n"
+        : "=r"(done) : "r"(smem_u32(bar0)), "r"(parity0), "r"(smem_u32(bar1)), "r"(parity1) : "memory");
+    return done;
+}
+
 // ---- TMA --------------------------------------------------------------------------------------
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* m) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(m)) : "memory");
