@@ -719,6 +719,11 @@ __device__ __forceinline__ void bar_sync_named(int id, int nthreads) {
 }
 
 // row maximum of 32 raw scores held in registers (integers are compared as integers)
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
 template <bool INT>
 __device__ __forceinline__ float row_max32(const uint32_t (&raw)[32]) {
     if (INT) {
@@ -733,36 +738,76 @@ __device__ __forceinline__ float row_max32(const uint32_t (&raw)[32]) {
         const int mm = max(max(m0, m1), max(m2, m3));
         return (mm < -(1 << 23)) ? -INFINITY : (float)mm;      // knocked-out entries sit far below any score
     } else {
-        float m0 = __uint_as_float(raw[0]), m1 = __uint_as_float(raw[1]), m2 = __uint_as_float(raw[2]), m3 = __uint_as_float(raw[3]);
+        // three-input maximum: two columns per instruction
+        float m0 = fmax3(__uint_as_float(raw[0]), __uint_as_float(raw[1]), __uint_as_float(raw[2]));
+        float m1 = fmax3(__uint_as_float(raw[3]), __uint_as_float(raw[4]), __uint_as_float(raw[5]));
+        float m2 = fmaxf(__uint_as_float(raw[6]), __uint_as_float(raw[7]));
 #pragma unroll
-        for (int e = 4; e < 32; e += 4) {
-            m0 = fmaxf(m0, __uint_as_float(raw[e]));
-            m1 = fmaxf(m1, __uint_as_float(raw[e + 1]));
-            m2 = fmaxf(m2, __uint_as_float(raw[e + 2]));
-            m3 = fmaxf(m3, __uint_as_float(raw[e + 3]));
+        for (int e = 8; e < 32; e += 6) {
+            m0 = fmax3(m0, __uint_as_float(raw[e]), __uint_as_float(raw[e + 1]));
+            m1 = fmax3(m1, __uint_as_float(raw[e + 2]), __uint_as_float(raw[e + 3]));
+            m2 = fmax3(m2, __uint_as_float(raw[e + 4]), __uint_as_float(raw[e + 5]));
         }
-        return fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+        return fmax3(m0, m1, m2);
     }
 }
 
-// exponentials of 32 raw scores: pk receives the fp16 pairs of 2^(raw * sc + bias); returns their fp32 sum
+// packed fp32 pairs (one instruction for two lanes of arithmetic; sm_100 fma / add on .f32x2)
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+    uint64_t v;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(v) : "f"(lo), "f"(hi));
+    return v;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+
+// exponentials of 32 raw scores: pk receives the fp16 pairs of 2^(raw * sc + bias); returns their fp32 sum.
+// Float scores go through the packed fp32 pipe (scale-and-shift and the row sum on two columns per instruction);
+// integer scores first become floats by the magic-number add.
 template <bool INT>
 __device__ __forceinline__ float row_exp32(const uint32_t (&raw)[32], float sc, float bias, uint32_t (&pk)[16]) {
-    float a0 = 0.0f, a1 = 0.0f, a2 = 0.0f, a3 = 0.0f;
+    if (INT) {
+        float a0 = 0.0f, a1 = 0.0f, a2 = 0.0f, a3 = 0.0f;
 #pragma unroll
-    for (int e = 0; e < 32; e += 4) {
-        float pv[4];
+        for (int e = 0; e < 32; e += 4) {
+            float pv[4];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const uint32_t rv = raw[e + u];
-            pv[u] = ex2f(fmaf(INT ? __uint_as_float(rv + INT_MAGIC) : __uint_as_float(rv), sc, bias));
+            for (int u = 0; u < 4; ++u) pv[u] = ex2f(fmaf(__uint_as_float(raw[e + u] + INT_MAGIC), sc, bias));
+            a0 += pv[0]; a1 += pv[1]; a2 += pv[2]; a3 += pv[3];
+            const __half2 h01 = __floats2half2_rn(pv[0], pv[1]), h23 = __floats2half2_rn(pv[2], pv[3]);
+            pk[e >> 1] = *reinterpret_cast<const uint32_t*>(&h01);
+            pk[(e >> 1) + 1] = *reinterpret_cast<const uint32_t*>(&h23);
         }
-        a0 += pv[0]; a1 += pv[1]; a2 += pv[2]; a3 += pv[3];
-        const __half2 h01 = __floats2half2_rn(pv[0], pv[1]), h23 = __floats2half2_rn(pv[2], pv[3]);
-        pk[e >> 1] = *reinterpret_cast<const uint32_t*>(&h01);
-        pk[(e >> 1) + 1] = *reinterpret_cast<const uint32_t*>(&h23);
+        return (a0 + a1) + (a2 + a3);
+    } else {
+        const uint64_t sc2 = pack2(sc, sc), bias2 = pack2(bias, bias);
+        uint64_t acc0 = pack2(0.0f, 0.0f), acc1 = acc0;
+#pragma unroll
+        for (int e = 0; e < 32; e += 4) {
+            float x0, x1, x2, x3;
+            unpack2(fma2(pack2(__uint_as_float(raw[e]), __uint_as_float(raw[e + 1])), sc2, bias2), x0, x1);
+            unpack2(fma2(pack2(__uint_as_float(raw[e + 2]), __uint_as_float(raw[e + 3])), sc2, bias2), x2, x3);
+            const float p0 = ex2f(x0), p1 = ex2f(x1), p2 = ex2f(x2), p3 = ex2f(x3);
+            acc0 = add2(acc0, pack2(p0, p1));
+            acc1 = add2(acc1, pack2(p2, p3));
+            const __half2 h01 = __floats2half2_rn(p0, p1), h23 = __floats2half2_rn(p2, p3);
+            pk[e >> 1] = *reinterpret_cast<const uint32_t*>(&h01);
+            pk[(e >> 1) + 1] = *reinterpret_cast<const uint32_t*>(&h23);
+        }
+        float s0, s1, s2, s3;
+        unpack2(acc0, s0, s1);
+        unpack2(acc1, s2, s3);
+        return (s0 + s1) + (s2 + s3);
     }
-    return (a0 + a1) + (a2 + a3);
 }
 
 // columns [c0, c0 + 32) of a boundary tile: entries outside [lo_eff, lo_eff + span] of this row become `knock`
