@@ -398,7 +398,7 @@ __device__ __forceinline__ bool tma_producer(const TcMaps& maps, const QSched& q
         const bool lowbit = t < w.nA, vl = !lowbit && t < w.nA + w.nB;
         const int row = lowbit ? t * BN : (vl ? (t - w.nA) * BN : (w.tC0 + t - w.nA - w.nB) * BN);
         const int hd = vl ? qhead : kvhead;
-        if (use > 0 && !mbar_wait(&bars.kv_free[st], (use - 1) & 1, WAIT_LIMIT)) return false;
+        if (use > 0 && !mbar_wait_sleepy(&bars.kv_free[st], (use - 1) & 1, WAIT_LIMIT)) return false;
         if (lowbit) {
             mbar_arrive_expect_tx(&bars.kv_full[st], G::KC_TILE_BYTES + G::STAGE_BYTES);
             tma_load_3d(sk, &maps.kc, &bars.kv_full[st], 0, row, hd);
@@ -696,12 +696,13 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
 // register spills at 96 registers per thread).  TMEM layout, MMA issue and TMA production are those of
 // the kernel above (two S buffers per query tile, P over the S columns it came from).
 // The two threads of a row must exponentiate against the same reference maximum.  Per tile they take
-// the maximum of their own half, and the eight warps of the query tile vote (named barrier with OR
-// reduction) whether any row has to raise its reference.  In the common case nobody does and each
-// half proceeds on its own; otherwise every thread also reads the other half's scores from TMEM, so
-// both threads of a row arrive at the same new reference, rescale their half of O (64 channels
-// each) and their partial row sum.  The vote also orders "both halves have read S" before
-// "either half writes P over it".  The partial sums are added at the end (exchange through TMEM).
+// the maximum of their own half, and the two warps that share 32 query rows vote (named barrier of
+// 64 threads with OR reduction) whether any of these rows has to raise its reference.  In the common
+// case none does and each half proceeds on its own; otherwise every thread also reads the other
+// half's scores from TMEM, so both threads of a row arrive at the same new reference, rescale their
+// half of O (64 channels each) and their partial row sum.  The vote also orders "both halves have
+// read S" before "either half writes P over it".  The partial sums are added at the end (exchange
+// through TMEM).
 // =============================================================================================
 constexpr int TCP_THREADS = 640;                    // TMA producer, 2 MMA issuers, 1 idle warp, 16 softmax warps
 constexpr float RAISE_THRESHOLD = 8.0f;             // log2 units by which a tile must exceed the reference to raise it
@@ -718,38 +719,24 @@ __device__ __forceinline__ void bar_sync_named(int id, int nthreads) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
 }
 
-// row maximum of 32 raw scores held in registers (integers are compared as integers)
+// row maximum of 32 float scores held in registers
 __device__ __forceinline__ float fmax3(float a, float b, float c) {
     float d;
     asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
     return d;
 }
-template <bool INT>
 __device__ __forceinline__ float row_max32(const uint32_t (&raw)[32]) {
-    if (INT) {
-        int m0 = (int)raw[0], m1 = (int)raw[1], m2 = (int)raw[2], m3 = (int)raw[3];
+    // three-input maximum: two columns per instruction
+    float m0 = fmax3(__uint_as_float(raw[0]), __uint_as_float(raw[1]), __uint_as_float(raw[2]));
+    float m1 = fmax3(__uint_as_float(raw[3]), __uint_as_float(raw[4]), __uint_as_float(raw[5]));
+    float m2 = fmaxf(__uint_as_float(raw[6]), __uint_as_float(raw[7]));
 #pragma unroll
-        for (int e = 4; e < 32; e += 4) {
-            m0 = max(m0, (int)raw[e]);
-            m1 = max(m1, (int)raw[e + 1]);
-            m2 = max(m2, (int)raw[e + 2]);
-            m3 = max(m3, (int)raw[e + 3]);
-        }
-        const int mm = max(max(m0, m1), max(m2, m3));
-        return (mm < -(1 << 23)) ? -INFINITY : (float)mm;      // knocked-out entries sit far below any score
-    } else {
-        // three-input maximum: two columns per instruction
-        float m0 = fmax3(__uint_as_float(raw[0]), __uint_as_float(raw[1]), __uint_as_float(raw[2]));
-        float m1 = fmax3(__uint_as_float(raw[3]), __uint_as_float(raw[4]), __uint_as_float(raw[5]));
-        float m2 = fmaxf(__uint_as_float(raw[6]), __uint_as_float(raw[7]));
-#pragma unroll
-        for (int e = 8; e < 32; e += 6) {
-            m0 = fmax3(m0, __uint_as_float(raw[e]), __uint_as_float(raw[e + 1]));
-            m1 = fmax3(m1, __uint_as_float(raw[e + 2]), __uint_as_float(raw[e + 3]));
-            m2 = fmax3(m2, __uint_as_float(raw[e + 4]), __uint_as_float(raw[e + 5]));
-        }
-        return fmax3(m0, m1, m2);
+    for (int e = 8; e < 32; e += 6) {
+        m0 = fmax3(m0, __uint_as_float(raw[e]), __uint_as_float(raw[e + 1]));
+        m1 = fmax3(m1, __uint_as_float(raw[e + 2]), __uint_as_float(raw[e + 3]));
+        m2 = fmax3(m2, __uint_as_float(raw[e + 4]), __uint_as_float(raw[e + 5]));
     }
+    return fmax3(m0, m1, m2);
 }
 
 // packed fp32 pairs (one instruction for two lanes of arithmetic; sm_100 fma / add on .f32x2)
@@ -770,44 +757,27 @@ __device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
     return d;
 }
 
-// exponentials of 32 raw scores: pk receives the fp16 pairs of 2^(raw * sc + bias); returns their fp32 sum.
-// Float scores go through the packed fp32 pipe (scale-and-shift and the row sum on two columns per instruction);
-// integer scores first become floats by the magic-number add.
-template <bool INT>
+// exponentials of 32 float scores: pk receives the fp16 pairs of 2^(raw * sc + bias); returns their fp32 sum.
+// Scale-and-shift and the row sum go through the packed fp32 pipe (two columns per instruction).
 __device__ __forceinline__ float row_exp32(const uint32_t (&raw)[32], float sc, float bias, uint32_t (&pk)[16]) {
-    if (INT) {
-        float a0 = 0.0f, a1 = 0.0f, a2 = 0.0f, a3 = 0.0f;
+    const uint64_t sc2 = pack2(sc, sc), bias2 = pack2(bias, bias);
+    uint64_t acc0 = pack2(0.0f, 0.0f), acc1 = acc0;
 #pragma unroll
-        for (int e = 0; e < 32; e += 4) {
-            float pv[4];
-#pragma unroll
-            for (int u = 0; u < 4; ++u) pv[u] = ex2f(fmaf(__uint_as_float(raw[e + u] + INT_MAGIC), sc, bias));
-            a0 += pv[0]; a1 += pv[1]; a2 += pv[2]; a3 += pv[3];
-            const __half2 h01 = __floats2half2_rn(pv[0], pv[1]), h23 = __floats2half2_rn(pv[2], pv[3]);
-            pk[e >> 1] = *reinterpret_cast<const uint32_t*>(&h01);
-            pk[(e >> 1) + 1] = *reinterpret_cast<const uint32_t*>(&h23);
-        }
-        return (a0 + a1) + (a2 + a3);
-    } else {
-        const uint64_t sc2 = pack2(sc, sc), bias2 = pack2(bias, bias);
-        uint64_t acc0 = pack2(0.0f, 0.0f), acc1 = acc0;
-#pragma unroll
-        for (int e = 0; e < 32; e += 4) {
-            float x0, x1, x2, x3;
-            unpack2(fma2(pack2(__uint_as_float(raw[e]), __uint_as_float(raw[e + 1])), sc2, bias2), x0, x1);
-            unpack2(fma2(pack2(__uint_as_float(raw[e + 2]), __uint_as_float(raw[e + 3])), sc2, bias2), x2, x3);
-            const float p0 = ex2f(x0), p1 = ex2f(x1), p2 = ex2f(x2), p3 = ex2f(x3);
-            acc0 = add2(acc0, pack2(p0, p1));
-            acc1 = add2(acc1, pack2(p2, p3));
-            const __half2 h01 = __floats2half2_rn(p0, p1), h23 = __floats2half2_rn(p2, p3);
-            pk[e >> 1] = *reinterpret_cast<const uint32_t*>(&h01);
-            pk[(e >> 1) + 1] = *reinterpret_cast<const uint32_t*>(&h23);
-        }
-        float s0, s1, s2, s3;
-        unpack2(acc0, s0, s1);
-        unpack2(acc1, s2, s3);
-        return (s0 + s1) + (s2 + s3);
+    for (int e = 0; e < 32; e += 4) {
+        float x0, x1, x2, x3;
+        unpack2(fma2(pack2(__uint_as_float(raw[e]), __uint_as_float(raw[e + 1])), sc2, bias2), x0, x1);
+        unpack2(fma2(pack2(__uint_as_float(raw[e + 2]), __uint_as_float(raw[e + 3])), sc2, bias2), x2, x3);
+        const float p0 = ex2f(x0), p1 = ex2f(x1), p2 = ex2f(x2), p3 = ex2f(x3);
+        acc0 = add2(acc0, pack2(p0, p1));
+        acc1 = add2(acc1, pack2(p2, p3));
+        const __half2 h01 = __floats2half2_rn(p0, p1), h23 = __floats2half2_rn(p2, p3);
+        pk[e >> 1] = *reinterpret_cast<const uint32_t*>(&h01);
+        pk[(e >> 1) + 1] = *reinterpret_cast<const uint32_t*>(&h23);
     }
+    float s0, s1, s2, s3;
+    unpack2(acc0, s0, s1);
+    unpack2(acc1, s2, s3);
+    return (s0 + s1) + (s2 + s3);
 }
 
 // columns [c0, c0 + 32) of a boundary tile: entries outside [lo_eff, lo_eff + span] of this row become `knock`
@@ -826,7 +796,7 @@ attn_tcp_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     __shared__ TcBarriers bars;
     __shared__ uint32_t tmem_base_s;
-    __shared__ int abort_s, cnt_b_s[QT], grp_abort_s[QT];
+    __shared__ int abort_s, cnt_b_s[QT];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int pt = gridDim.x - 1 - blockIdx.x;               // pair of query tiles; longest rows first
@@ -847,7 +817,6 @@ attn_tcp_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                 mbar_init(&bars.p_full[q][bf], 8);           // one arrival per softmax warp of the query tile
                 mbar_init(&bars.o_done[q][bf], 1);
             }
-            grp_abort_s[q] = 0;
         }
         fence_mbar_init();
         abort_s = 0;
@@ -902,7 +871,8 @@ attn_tcp_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
         // ------------------------------------------------------------------ softmax warps
         const int q = (warp - 4) >> 3, hsel = ((warp - 4) >> 2) & 1;    // query tile, column half
         const QSched sq = q ? qs1 : qs0;
-        const int bar_id = 1 + q;                               // named barrier of this query tile's 256 softmax threads
+        // named barrier of the two warps that share this warp's 32 query rows (one per query tile and lane quarter)
+        const int bar_id = 1 + q * 4 + (warp & 3);
         const OwnTiles own = own_tiles(sq, w);
         const int n_total = own.a_end + (own.b_end - own.b_beg) + (own.c_end - own.c_beg);
         if (sq.live && n_total > 0) {
@@ -953,7 +923,6 @@ attn_tcp_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                 HYQ_TR(q * 2 + hsel, n, 0);
                 if (!dead && !__all_sync(0xffffffffu, mbar_wait(&bars.s_full[q][buf], (uint32_t)(n >> 1) & 1u, WAIT_LIMIT))) {
                     dead = true;
-                    grp_abort_s[q] = 1;
                 }
                 __syncwarp();
                 HYQ_TR(q * 2 + hsel, n, 1);
@@ -967,17 +936,23 @@ attn_tcp_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                     tmem_ld32(ts + col0, raw);
                     tmem_wait_ld();
                     if (NEED_RANGE) mask_cols32(raw, col0, lo_eff, span, knock);
-                    const float f = int_scores ? row_max32<true>(raw) : row_max32<false>(raw);
+                    // integer scores become the floats 2^23 + 2^22 + s by one integer add each (knocked-out entries
+                    // become -inf); the offset is taken out again by the bias of the exponent
+                    if (int_scores) {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) raw[e] += INT_MAGIC;
+                    }
+                    const float f = row_max32(raw) - (int_scores ? INT_MAGIC_F : 0.0f);
                     mt = (f == -INFINITY) ? -INFINITY : f * cs;
                 }
-                // ---- vote: does any row of this query tile have to raise its reference maximum?
+                // ---- vote of the two warps of these 32 rows: does any row have to raise its reference maximum?
                 // (also: both halves have read their scores before either writes P over them)
                 tc_fence_before();
                 HYQ_TR(q * 2 + hsel, n, 3);
-                const bool any_raise = bar_red_or(bar_id, 256, dead || mt > m_used + RAISE_THRESHOLD);
+                const bool any_raise = bar_red_or(bar_id, 64, dead || mt > m_used + RAISE_THRESHOLD);
                 HYQ_TR(q * 2 + hsel, n, 4);
                 if (any_raise) {
-                    if (*reinterpret_cast<volatile int*>(&grp_abort_s[q])) return false;
+                    if (bar_red_or(bar_id, 64, dead)) return false;         // one of the two warps ran into an expired wait
                     tc_fence_after();
                     // the other half's maximum, from its scores in TMEM (same knock-outs, same range mask)
                     float mo;
@@ -986,11 +961,15 @@ attn_tcp_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                         tmem_ld32(ts + col0_other, oth);
                         tmem_wait_ld();
                         if (NEED_RANGE) mask_cols32(oth, col0_other, lo_eff, span, knock);
-                        const float fo = int_scores ? row_max32<true>(oth) : row_max32<false>(oth);
+                        if (int_scores) {
+#pragma unroll
+                            for (int e = 0; e < 32; ++e) oth[e] += INT_MAGIC;
+                        }
+                        const float fo = row_max32(oth) - (int_scores ? INT_MAGIC_F : 0.0f);
                         mo = (fo == -INFINITY) ? -INFINITY : fo * cs;
                     }
                     tc_fence_before();
-                    bar_sync_named(bar_id, 256);                 // both halves are done reading before P is written
+                    bar_sync_named(bar_id, 64);                  // both halves are done reading before P is written
                     const float m_new = fmaxf(mt, mo);
                     const bool raise = m_new > m_used + RAISE_THRESHOLD;     // same verdict in both threads of the row
                     const float alpha = raise ? ex2f(m_used - m_new) : 1.0f; // m_used = -inf -> 0
@@ -1000,7 +979,6 @@ attn_tcp_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                         // the parity wait cannot alias.
                         if (!__all_sync(0xffffffffu, mbar_wait(&bars.o_done[q][(n - 1) & 1], (uint32_t)((n - 1) >> 1) & 1u, WAIT_LIMIT))) {
                             dead = true;
-                            grp_abort_s[q] = 1;
                         } else {
                             tc_fence_after();
 #pragma unroll 1
@@ -1025,7 +1003,7 @@ attn_tcp_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                     const float m_eff = (m_used == -INFINITY) ? 0.0f : m_used;
                     const float bias = int_scores ? fmaf(-INT_MAGIC_F, cs, -m_eff) : -m_eff;
                     uint32_t pk[16];
-                    l_h += int_scores ? row_exp32<true>(raw, cs, bias, pk) : row_exp32<false>(raw, cs, bias, pk);
+                    l_h += row_exp32(raw, cs, bias, pk);  // (integer scores were made floats above)
                     HYQ_TR(q * 2 + hsel, n, 5);
                     tmem_st16(ts + hsel * 16, pk);
                     tmem_wait_st();
@@ -1084,7 +1062,7 @@ attn_tcp_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                 tmem_st1(ts0 + col0, __float_as_uint(l_h));     // column col0 of S buffer 0 (all MMAs are done)
                 tmem_wait_st();
                 tc_fence_before();
-                bar_sync_named(bar_id, 256);
+                bar_sync_named(bar_id, 64);
                 tc_fence_after();
                 const float l_o = __uint_as_float(tmem_ld1(ts0 + col0_other));
                 tmem_wait_ld();

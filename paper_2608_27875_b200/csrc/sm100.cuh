@@ -51,6 +51,19 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, long l
     return true;
 }
 
+// Same contract as mbar_wait, but the thread sleeps between polls instead of spinning: a spinning single-thread warp
+// issues an instruction every few clocks and takes those issue slots (and MIO queue entries) away from the softmax
+// warps of its scheduler.  For threads that usually wait long and can afford to wake a few hundred clocks late.
+__device__ __forceinline__ bool mbar_wait_sleepy(uint64_t* bar, uint32_t parity, long long limit_cycles) {
+    if (mbar_test_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    do {
+        __nanosleep(64);
+        if (mbar_test_wait(bar, parity)) return true;
+    } while (clock64() - t0 <= limit_cycles);
+    return false;
+}
+
 // Tests two barriers back to back, so that the two shared-memory round trips overlap (a single-thread MMA issuer
 // pays one latency instead of two): bit 0 / bit 1 of the result = phase with parity0 / parity1 complete.
 __device__ __forceinline__ uint32_t mbar_test_wait2(uint64_t* bar0, uint32_t parity0, uint64_t* bar1, uint32_t parity1) {
