@@ -705,7 +705,7 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
 // through TMEM).
 // =============================================================================================
 constexpr int TCP_THREADS = 640;                    // TMA producer, 2 MMA issuers, 1 idle warp, 16 softmax warps
-constexpr float RAISE_THRESHOLD = 8.0f;             // log2 units by which a tile must exceed the reference to raise it
+constexpr float RAISE_THRESHOLD = 14.0f;            // log2 units by which a tile must exceed the reference to raise it (P stays below 2^14, inside fp16)
 
 // named barrier over `nthreads` threads with an OR reduction of `pred` (all threads of the participating warps call it)
 __device__ __forceinline__ bool bar_red_or(int id, int nthreads, bool pred) {
