@@ -10,16 +10,18 @@
 // All passes feed one running (m, l) per row and one fp32 O accumulator per query tile in TMEM.
 // S is double-buffered per query tile (4 x 64 TMEM columns), so Q.K^T of the next tile is done
 // before the softmax of the current one ends; P goes back to TMEM as fp16 over the S columns it
-// was computed from and is the A operand of the P.V MMA (fp16 x fp16).  K/V tiles are loaded once
-// (4-stage rings) and used by both query tiles.
+// was computed from and is the A operand of the P.V MMA (fp16 x fp16).  The K tile and the V tile of
+// a walk position share one stage of a 4-stage ring (one "full" and one "free" barrier per stage) and
+// are used by both query tiles.
 //
-// Warp roles (352 threads): warps 0-3 and 4-7 are the softmax groups of query tile 0 and 1 (thread r
-// owns query row r = TMEM lane r), warp 8 lane 0 issues TMA loads, warps 9 and 10 (lane 0) issue the
-// MMAs of query tile 0 and 1.
-// The exponentials are taken against a running reference maximum that is only raised when a tile
-// overshoots it by more than 2^8 (the rescale of O is then rare); integer scores become floats through a magic-number add folded into the exponent
-// FFMA.  Every mbarrier wait is bounded; when one expires the CTA records HYQ_ERR_TIMEOUT in the
-// status word and unwinds.
+// Warp roles (640 threads): warp 0 lane 0 issues the TMA loads, warps 1 and 2 (lane 0) issue the
+// MMAs of query tile 0 and 1, warp 3 idles, warps 4-19 are the softmax warps: eight per query tile,
+// two threads per query row (thread (r, h) owns columns [32 h, 32 h + 32) of row r = TMEM lane r of
+// every score tile), so that each of the four schedulers hosts four softmax warps and a thread holds
+// 32 scores.  The exponentials are taken against a per-row reference maximum that is only raised when
+// a tile exceeds it by more than 2^14 (the rescale of O is then rare); integer scores become floats
+// by a magic-number add.  Every mbarrier wait is bounded; when one expires the CTA records
+// HYQ_ERR_TIMEOUT in the status word and unwinds.
 #include <cuda_fp16.h>
 
 #include <type_traits>
@@ -32,9 +34,7 @@ using namespace sm100;
 
 constexpr int BM = 128, QT = 2;
 constexpr int RING_BYTES = 65536;                   // shared memory of the K ring and of the V ring
-constexpr int TC_THREADS = 352;
 constexpr long long WAIT_LIMIT = 4000000000LL;      // SM clocks (~2 s): far beyond any legitimate wait
-constexpr float OVERSHOOT_LIMIT = 256.0f;           // a tile is redone when a probability exceeds 2^8 of the reference
 
 constexpr uint32_t Q_TILE_BYTES = BM * HYQ_D * 2, QC_TILE_BYTES = BM * HYQ_D;        // 32768, 16384
 constexpr uint32_t SQ_OFF = 0, SQC_OFF = QT * Q_TILE_BYTES, SK_OFF = SQC_OFF + QT * QC_TILE_BYTES;
@@ -42,7 +42,7 @@ constexpr uint32_t SV_OFF = SK_OFF + RING_BYTES;
 constexpr uint32_t TILE_SMEM = SV_OFF + RING_BYTES;                 // 229376
 constexpr int MAX_STAGES = 4;
 
-// per tile width: 64 keys -> 4-stage rings and two S buffers per query tile; 128 keys -> 2 stages, one buffer
+// geometry that follows from the keys per tile (64: 4-stage ring, two S buffers per query tile)
 template <int TBN> struct Geo {
     static constexpr int BN = TBN;
     static constexpr int NBUF = 128 / TBN;                              // S buffers per query tile (128 TMEM columns)
@@ -119,146 +119,6 @@ __device__ __forceinline__ int count_le(const int32_t* __restrict__ idx, int k, 
         if (__ldg(idx + mid) <= v) lo = mid + 1; else hi = mid;
     }
     return lo;
-}
-
-// ---- softmax building blocks: one thread = one query row, its BN scores held in registers ---------
-// row maximum of the raw scores of one 64-column quantization block (integers are compared as integers)
-template <bool INT, int N>
-__device__ __forceinline__ float block_max(const uint32_t (&raw)[N], int c0) {
-    if (INT) {
-        int m0 = (int)raw[c0], m1 = (int)raw[c0 + 1], m2 = (int)raw[c0 + 2], m3 = (int)raw[c0 + 3];
-#pragma unroll
-        for (int e = 4; e < 64; e += 4) {
-            m0 = max(m0, (int)raw[c0 + e]);
-            m1 = max(m1, (int)raw[c0 + e + 1]);
-            m2 = max(m2, (int)raw[c0 + e + 2]);
-            m3 = max(m3, (int)raw[c0 + e + 3]);
-        }
-        const int m = max(max(m0, m1), max(m2, m3));
-        return (m < -(1 << 23)) ? -INFINITY : (float)m;      // knocked-out entries sit far below any score
-    } else {
-        float m0 = __uint_as_float(raw[c0]), m1 = __uint_as_float(raw[c0 + 1]), m2 = __uint_as_float(raw[c0 + 2]),
-              m3 = __uint_as_float(raw[c0 + 3]);
-#pragma unroll
-        for (int e = 4; e < 64; e += 4) {
-            m0 = fmaxf(m0, __uint_as_float(raw[c0 + e]));
-            m1 = fmaxf(m1, __uint_as_float(raw[c0 + e + 1]));
-            m2 = fmaxf(m2, __uint_as_float(raw[c0 + e + 2]));
-            m3 = fmaxf(m3, __uint_as_float(raw[c0 + e + 3]));
-        }
-        return fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
-    }
-}
-
-// exponentials of one row: pk = fp16 pairs of 2^(raw * cs + bias), returns their fp32 sum; pmax2 collects the
-// running maximum of the packed values (two lanes of a half2)
-template <bool INT, int TBN>
-__device__ __forceinline__ float exp_row(const uint32_t (&raw)[TBN], const float (&cs)[TBN / 64], float m_eff,
-                                         uint32_t (&pk)[TBN / 2], __half2& pmax2) {
-    float acc[8] = {0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f};
-#pragma unroll
-    for (int bl = 0; bl < TBN / 64; ++bl) {
-        const float sc = cs[bl];
-        const float bias = INT ? fmaf(-INT_MAGIC_F, sc, -m_eff) : -m_eff;
-#pragma unroll
-        for (int e = 0; e < 64; e += 2) {
-            const uint32_t r0 = raw[bl * 64 + e], r1 = raw[bl * 64 + e + 1];
-            const float p0 = ex2f(fmaf(INT ? __uint_as_float(r0 + INT_MAGIC) : __uint_as_float(r0), sc, bias));
-            const float p1 = ex2f(fmaf(INT ? __uint_as_float(r1 + INT_MAGIC) : __uint_as_float(r1), sc, bias));
-            acc[e & 7] += p0;
-            acc[(e & 7) + 1] += p1;
-            const __half2 h2 = __floats2half2_rn(p0, p1);
-            pmax2 = __hmax2(pmax2, h2);
-            pk[bl * 32 + (e >> 1)] = *reinterpret_cast<const uint32_t*>(&h2);
-        }
-    }
-    return ((acc[0] + acc[1]) + (acc[2] + acc[3])) + ((acc[4] + acc[5]) + (acc[6] + acc[7]));
-}
-
-// one tile of the online softmax for one query row: S (TMEM) -> running (m, l) -> P (TMEM, fp16).
-//   cs[b]   score scale of 64-column block b (includes log2 e)
-// (columns that must not count were set to -inf in TMEM beforehand)
-// Fast path: the exponentials are taken against the running reference maximum m_used without looking at
-// the tile's own maximum first; the tile is accepted when no probability exceeded OVERSHOOT_LIMIT.  Otherwise
-// (and while a row has no reference yet) the tile's maximum is computed, the reference is raised, O and l
-// are rescaled and the exponentials are redone.
-// returns false when a bounded wait expired
-template <bool INT, int TBN>
-__device__ __forceinline__ bool softmax_tile(uint32_t ts, uint32_t to, const float (&cs)[TBN / 64], bool first, uint64_t* o_done,
-                                             uint32_t o_parity, float& m_used, float& l_run) {
-    uint32_t raw[TBN];
-    {
-        uint32_t (*rc)[32] = reinterpret_cast<uint32_t (*)[32]>(raw);
-#pragma unroll
-        for (int c = 0; c < TBN / 32; ++c) tmem_ld32(ts + c * 32, rc[c]);
-        tmem_wait_ld();
-    }
-    uint32_t pk[TBN / 2];
-    __half2 pmax2 = __floats2half2_rn(0.0f, 0.0f);
-    float rs = exp_row<INT, TBN>(raw, cs, (m_used == -INFINITY) ? 0.0f : m_used, pk, pmax2);
-    const float pmax = fmaxf(__low2float(pmax2), __high2float(pmax2));
-    // redo when this row has no reference yet, or a value overshot the reference by more than the threshold
-    // (NaN-safe: an overflow to inf fails the comparison too)
-    const bool redo = (m_used == -INFINITY) || !(pmax <= OVERSHOOT_LIMIT);
-    if (__any_sync(0xffffffffu, redo)) {
-        float mt = -INFINITY;
-#pragma unroll
-        for (int bl = 0; bl < TBN / 64; ++bl) {
-            const float f = block_max<INT>(raw, bl * 64);
-            mt = fmaxf(mt, (f == -INFINITY) ? -INFINITY : f * cs[bl]);
-        }
-        float alpha = 1.0f;
-        const bool raise = redo && mt > m_used;                  // rows that are fine keep their reference
-        if (raise) {
-            alpha = ex2f(m_used - mt);                           // m_used = -inf -> 0
-            l_run *= alpha;
-            m_used = mt;
-        }
-        if (!first && __any_sync(0xffffffffu, raise)) {
-            // the previous P.V of this query tile must have landed before O is rescaled.  P.V number n
-            // signals barrier n & 1; the one before the previous is known to be complete (the S tile
-            // just read was issued after it), so the parity wait cannot alias.
-            if (!mbar_wait(o_done, o_parity, WAIT_LIMIT)) return false;
-            __syncwarp();
-            tc_fence_after();
-#pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
-                uint32_t o[32];
-                tmem_ld32(to + c * 32, o);
-                tmem_wait_ld();
-#pragma unroll
-                for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-                tmem_st32(to + c * 32, o);
-            }
-        }
-        if (raise) {
-            __half2 unused = __floats2half2_rn(0.0f, 0.0f);
-            rs = exp_row<INT, TBN>(raw, cs, m_used, pk, unused);
-        }
-    }
-    l_run += rs;
-#pragma unroll
-    for (int c = 0; c < TBN / 32; ++c) {
-        uint32_t (&pc)[16] = *reinterpret_cast<uint32_t (*)[16]>(&pk[c * 16]);
-        tmem_st16(ts + c * 16, pc);
-    }
-    tmem_wait_st();
-    return true;
-}
-
-// boundary tiles: columns outside [lo_eff, lo_eff + span] of this row are set to -inf in TMEM
-template <int TBN>
-__device__ __forceinline__ void mask_tile_in_tmem(uint32_t ts, int lo_eff, unsigned span, uint32_t knock) {
-#pragma unroll 1
-    for (int c = 0; c < TBN / 32; ++c) {
-        uint32_t raw[32];
-        tmem_ld32(ts + c * 32, raw);
-        tmem_wait_ld();
-#pragma unroll
-        for (int e = 0; e < 32; ++e) raw[e] = ((unsigned)(c * 32 + e - lo_eff) <= span) ? raw[e] : knock;
-        tmem_st32(ts + c * 32, raw);
-    }
-    tmem_wait_st();
 }
 
 // the tile walk of one CTA: union of both query tiles' lists
@@ -415,296 +275,15 @@ __device__ __forceinline__ bool tma_producer(const TcMaps& maps, const QSched& q
     return true;
 }
 
-// TBN: keys per tile (64 or 128).  LOWBIT_FP8: low-bit codes are e4m3 bytes (kind::f8f6f4), else int8 (kind::i8)
-template <bool LOWBIT_FP8, int TBN>
-__global__ void __launch_bounds__(TC_THREADS, 1)
-attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
-    using G = Geo<TBN>;
-    constexpr int BN = TBN, NST = G::NST, NBUF = G::NBUF, NSC = G::NSC, NVW = G::NVW;
-    extern __shared__ unsigned char smem_raw[];
-    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    __shared__ TcBarriers bars;
-    __shared__ uint32_t tmem_base_s;
-    __shared__ int abort_s, cnt_b_s[QT];
-
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int pt = gridDim.x - 1 - blockIdx.x;               // pair of query tiles; longest rows first
-    const int h = blockIdx.y, b = blockIdx.z;
-    const int L = p.L, W = p.window, g = p.Hq / p.Hkv;
-    const int qhead = b * p.Hq + h, kvhead = b * p.Hkv + h / g;
-    const int32_t* idx_row = p.vl_idx + (long)qhead * p.k;
-
-    if (threadIdx.x == 0) {
-        mbar_init(&bars.q_full, 1);
-        for (int s = 0; s < NST; ++s) {
-            mbar_init(&bars.kv_full[s], 1);
-            mbar_init(&bars.kv_free[s], QT);
-        }
-        for (int q = 0; q < QT; ++q) {
-            for (int bf = 0; bf < 2; ++bf) {
-                mbar_init(&bars.s_full[q][bf], 1);
-                mbar_init(&bars.p_full[q][bf], 4);           // one arrival per softmax warp
-                mbar_init(&bars.o_done[q][bf], 1);
-            }
-        }
-        fence_mbar_init();
-        abort_s = 0;
-    }
-    if (threadIdx.x < QT) {
-        const int i1 = min(pt * QT * BM + (int)threadIdx.x * BM + BM - 1, L - 1);
-        cnt_b_s[threadIdx.x] = (p.k > 0 && i1 - W >= 0) ? count_le(idx_row, p.k, i1 - W) : 0;
-    }
-    if (warp == 8) {
-        tmem_alloc(&tmem_base_s, TM_COLS);
-        tmem_relinquish();
-    }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem = tmem_base_s;
-
-    // per query tile: nA low-bit tiles, nB gathered vertical-line tiles, window tiles tC0..tC1
-    auto make_sched = [&](int q) {
-        QSched s;
-        s.i0 = (pt * QT + q) * BM;
-        s.live = s.i0 < L;
-        s.i1 = min(s.i0 + BM - 1, L - 1);
-        s.nA = (s.live && s.i1 - W >= 0) ? (s.i1 - W) / BN + 1 : 0;
-        s.nB = s.live ? (cnt_b_s[q] + BN - 1) / BN : 0;
-        s.tC0 = max(0, s.i0 - W + 1) / BN;
-        s.tC1 = (s.live && W > 0) ? s.i1 / BN : -1;
-        return s;
-    };
-    const QSched qs0 = make_sched(0), qs1 = make_sched(1);
-    // the CTA walks the union of both lists (tile 1 holds the later rows, so its lists are the longer ones)
-    Walk w;
-    w.nA = max(qs0.nA, qs1.nA);
-    w.nB = max(qs0.nB, qs1.nB);
-    w.tC0 = qs0.tC0;
-    w.nC = (W > 0) ? max(qs0.tC1, qs1.tC1) - w.tC0 + 1 : 0;
-    w.T = w.nA + w.nB + w.nC;
-
-    volatile int* abort_flag = &abort_s;
-    auto fail = [&]() {
-        *abort_flag = 1;
-        if (p.status) atomicExch(p.status, HYQ_ERR_TIMEOUT);
-    };
-
-    if (warp == 8) {
-        // ------------------------------------------------------------------ TMA producer
-        if (lane == 0 && !tma_producer<TBN>(maps, qs0, qs1, w, qhead, kvhead, bars, smem, abort_flag)) fail();
-    } else if (warp == 9 || warp == 10) {
-        // ------------------------------------------------------------------ MMA issuers (one per query tile)
-        if (lane == 0) {
-            const int q = warp - 9;
-            if (!mma_issuer<LOWBIT_FP8, TBN>(q, q ? qs1 : qs0, w, bars, smem, tmem, abort_flag)) fail();
-        }
-    } else if (warp < 8) {
-        // ------------------------------------------------------------------ softmax groups
-        const int q = warp >> 2;
-        const QSched sq = q ? qs1 : qs0;
-        const int r = threadIdx.x & 127;                // query row inside the tile = TMEM lane
-        const int i = sq.i0 + r;
-        const bool row_live = i < L;
-        const bool ragged = sq.i0 + BM > L;
-        const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
-        const uint32_t to = tmem + tm_o(q) + lane_addr, ts0 = tmem + tm_s(q) + lane_addr;
-        const float q_scale = row_live ? __ldg(p.q_scales + (long)qhead * p.nb + i / HYQ_BLOCK_TOKENS) : 0.0f;
-        const int cnt_r = (sq.nB > 0 && row_live && i - W >= 0) ? count_le(idx_row, p.k, i - W) : 0;
-        const uint32_t* bits_row = p.vl_bits + (long)qhead * p.mask_words;
-        const float* ks_row = p.k_scales + (long)kvhead * p.nb;
-        float m_used = -INFINITY, l_run = 0.0f;
-        int n_act = 0;
-        bool ok = true;
-        constexpr uint32_t knock_lq = LOWBIT_FP8 ? KNOCKOUT_F32 : KNOCKOUT_S32;
-
-        // own tile list: low-bit tiles [0, nA_own), vertical tiles, window tiles (positions in the CTA's walk)
-        const int a_end = sq.nA, b_beg = w.nA, b_end = w.nA + sq.nB;
-        const int c_beg = w.nA + w.nB + (sq.tC0 - w.tC0), c_end = (sq.tC1 >= sq.tC0) ? w.nA + w.nB + (sq.tC1 - w.tC0) + 1 : c_beg;
-        auto next_tile = [&](int t) -> int {            // first own tile at or after walk position t (or T)
-            if (!sq.live) return w.T;
-            if (t < a_end) return t;
-            if (t < b_beg) t = b_beg;
-            if (t < b_end) return t;
-            if (t < c_beg) t = c_beg;
-            return (t < c_end) ? t : w.T;
-        };
-
-        // scales and vertical-line bitmask words of a low-bit tile, fetched one tile ahead of their use
-        float nks[NSC];
-        uint32_t nvl[NVW];
-        auto prefetch_tile = [&](int t) {
-#pragma unroll
-            for (int e = 0; e < NSC; ++e) nks[e] = 0.0f;
-#pragma unroll
-            for (int e = 0; e < NVW; ++e) nvl[e] = 0u;
-            if (t >= a_end) return;
-#pragma unroll
-            for (int e = 0; e < NSC; ++e) nks[e] = __ldg(ks_row + min(t * NSC + e, p.nb - 1));
-#pragma unroll
-            for (int e = 0; e < NVW; ++e) nvl[e] = (t * NVW + e < p.mask_words) ? __ldg(bits_row + t * NVW + e) : 0u;
-        };
-        // vertical-line keys of a low-bit tile: their S columns are set to -inf in TMEM (no wait here;
-        // the caller's next tcgen05.wait::st covers these stores)
-        auto knock_columns = [&](uint32_t ts, const uint32_t (&v)[NVW]) {
-#pragma unroll
-            for (int e = 0; e < NVW; ++e) {
-                uint32_t bits = v[e];
-                while (bits) {
-                    const int c = __ffs(bits) - 1;
-                    bits &= bits - 1;
-                    tmem_st1(ts + e * 32 + c, knock_lq);
-                }
-            }
-        };
-        int t = next_tile(0);
-        prefetch_tile(t);
-        bool knocked = false;                           // vertical columns of tile t already knocked out in TMEM
-        while (t < w.T && ok) {
-            float ks[NSC];
-            uint32_t vlw[NVW];
-            uint32_t any_vl = 0u;
-#pragma unroll
-            for (int e = 0; e < NSC; ++e) ks[e] = nks[e];
-#pragma unroll
-            for (int e = 0; e < NVW; ++e) { vlw[e] = nvl[e]; any_vl |= nvl[e]; }
-            const int t_next = next_tile(t + 1);
-            prefetch_tile(t_next);
-            // ---- per-tile column bounds and scales
-            int lo = 0, hi = -1;
-            bool need_range;
-            float cs[NSC];
-            const bool lowbit = t < a_end;
-            if (lowbit) {
-                const int j0 = t * BN;
-                hi = row_live ? min(i - W - j0, BN - 1) : -1;
-                need_range = (j0 + BN - 1 > sq.i0 - W) || ragged;
-                // a zero scale (all-zero tile) still has to let -inf pass through the multiply
-#pragma unroll
-                for (int e = 0; e < NSC; ++e) cs[e] = fmaxf(q_scale * ks[e] * p.scale_log2, 1e-37f);
-            } else if (t < b_end) {
-                const int c0 = (t - b_beg) * BN;
-                hi = min(cnt_r - c0 - 1, BN - 1);
-                need_range = true;
-#pragma unroll
-                for (int e = 0; e < NSC; ++e) cs[e] = p.scale_log2;
-            } else {
-                const int j0 = (w.tC0 + t - w.nA - w.nB) * BN;
-                lo = max(0, i - W + 1 - j0);
-                hi = row_live ? min(i - j0, BN - 1) : -1;
-                need_range = (j0 + BN - 1 > sq.i0) || (j0 <= sq.i1 - W) || ragged;
-#pragma unroll
-                for (int e = 0; e < NSC; ++e) cs[e] = p.scale_log2;
-            }
-            const int lo_eff = (hi >= lo) ? lo : 4096;
-            const unsigned span = (hi >= lo) ? (unsigned)(hi - lo) : 0u;
-            const bool int_scores = lowbit && !LOWBIT_FP8;
-            const int buf = n_act % NBUF;
-            const uint32_t ts = ts0 + buf * BN;
-
-            if (!mbar_wait(&bars.s_full[q][buf], (n_act / NBUF) & 1, WAIT_LIMIT)) { ok = false; break; }
-            __syncwarp();
-            tc_fence_after();
-
-            // ---- boundary tiles: causal / window / validity limits of this row, applied in TMEM
-            if (need_range) mask_tile_in_tmem<TBN>(ts, lo_eff, span, int_scores ? KNOCKOUT_S32 : KNOCKOUT_F32);
-            // ---- vertical-line keys of a low-bit tile: -inf into their S columns.  With two S buffers the next
-            // tile is done ahead of time when its scores have already landed (the stores then complete under
-            // this tile's exponentials)
-            if (any_vl != 0u && !knocked) {
-                knock_columns(ts, vlw);
-                tmem_wait_st();
-            }
-            knocked = false;
-            if (NBUF == 2) {
-                uint32_t nany = 0u;
-#pragma unroll
-                for (int e = 0; e < NVW; ++e) nany |= nvl[e];
-                if (t_next < a_end && nany != 0u) {               // uniform over the warp
-                    const int nbuf = (n_act + 1) % NBUF;
-                    knocked = __all_sync(0xffffffffu, mbar_test_wait(&bars.s_full[q][nbuf], ((n_act + 1) / NBUF) & 1));
-                    if (knocked) {
-                        tc_fence_after();
-                        knock_columns(ts0 + nbuf * BN, nvl);
-                    }
-                }
-            }
-            uint64_t* od = &bars.o_done[q][(n_act - 1) & 1];
-            const uint32_t op = ((n_act - 1) >> 1) & 1;
-            if (int_scores) ok = softmax_tile<true, TBN>(ts, to, cs, n_act == 0, od, op, m_used, l_run);
-            else ok = softmax_tile<false, TBN>(ts, to, cs, n_act == 0, od, op, m_used, l_run);
-            if (!ok) break;
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&bars.p_full[q][buf]);
-            ++n_act;
-            t = t_next;
-        }
-        // ---- epilogue: O / l
-        // (the P.V before the last one finished earlier: MMAs complete in order)
-        if (ok && n_act > 0) ok = mbar_wait(&bars.o_done[q][(n_act - 1) & 1], ((n_act - 1) >> 1) & 1, WAIT_LIMIT);
-        __syncwarp();
-        if (ok && n_act > 0) {
-            tc_fence_after();
-            const float inv = (l_run > 0.0f) ? 1.0f / l_run : 0.0f;
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint32_t o[32];
-                tmem_ld32(to + c * 32, o);
-                tmem_wait_ld();
-                if (row_live) {
-                    if (p.out_fp32) {
-                        float4* dst = reinterpret_cast<float4*>(static_cast<float*>(p.out) + ((long)qhead * L + i) * HYQ_D + c * 32);
-#pragma unroll
-                        for (int e = 0; e < 8; ++e)
-                            dst[e] = make_float4(__uint_as_float(o[4 * e]) * inv, __uint_as_float(o[4 * e + 1]) * inv,
-                                                 __uint_as_float(o[4 * e + 2]) * inv, __uint_as_float(o[4 * e + 3]) * inv);
-                    } else {
-                        uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.out) + ((long)qhead * L + i) * HYQ_D + c * 32);
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            uint32_t wd[4];
-#pragma unroll
-                            for (int q2 = 0; q2 < 4; ++q2) {
-                                const __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(o[8 * e + 2 * q2]) * inv,
-                                                                                __uint_as_float(o[8 * e + 2 * q2 + 1]) * inv);
-                                wd[q2] = *reinterpret_cast<const uint32_t*>(&b2);
-                            }
-                            dst[e] = make_uint4(wd[0], wd[1], wd[2], wd[3]);
-                        }
-                    }
-                }
-            }
-            if (p.lse && row_live) p.lse[(long)qhead * L + i] = (m_used + log2f(l_run)) * 0.6931471805599453f;
-        } else if (!ok) {
-            fail();
-        }
-    }
-
-    tc_fence_before();
-    __syncthreads();
-    if (warp == 8) {
-        __syncwarp();
-        tmem_dealloc(tmem, TM_COLS);
-    }
-}
-
-// =============================================================================================
-// Variant with TWO THREADS PER QUERY ROW (64-key tiles): each query tile is served by eight softmax
-// warps; thread (r, h) owns columns [32 h, 32 h + 32) of row r of every score tile.  Every scheduler
-// then hosts four softmax warps instead of two, and a thread holds 32 scores instead of 64 (no
-// register spills at 96 registers per thread).  TMEM layout, MMA issue and TMA production are those of
-// the kernel above (two S buffers per query tile, P over the S columns it came from).
-// The two threads of a row must exponentiate against the same reference maximum.  Per tile they take
-// the maximum of their own half, and the two warps that share 32 query rows vote (named barrier of
-// 64 threads with OR reduction) whether any of these rows has to raise its reference.  In the common
-// case none does and each half proceeds on its own; otherwise every thread also reads the other
-// half's scores from TMEM, so both threads of a row arrive at the same new reference, rescale their
-// half of O (64 channels each) and their partial row sum.  The vote also orders "both halves have
-// read S" before "either half writes P over it".  The partial sums are added at the end (exchange
-// through TMEM).
-// =============================================================================================
-constexpr int TCP_THREADS = 640;                    // TMA producer, 2 MMA issuers, 1 idle warp, 16 softmax warps
+// ---- softmax warps: two threads per query row ----------------------------------------------------
+// The two threads of a row must exponentiate against the same reference maximum.  Per tile they take the maximum
+// of their own 32 columns, and the two warps that share 32 query rows vote (named barrier of 64 threads with OR
+// reduction) whether any of these rows has to raise its reference.  In the common case none does and each half
+// proceeds on its own; otherwise every thread also reads the other half's scores from TMEM, so both threads of a
+// row arrive at the same new reference, rescale their half of O (64 channels each) and their partial row sum.
+// The vote also orders "both halves have read S" before "either half writes P over it".  The partial sums are
+// added at the end (exchange through TMEM).
+constexpr int TC_THREADS = 640;                     // TMA producer, 2 MMA issuers, 1 idle warp, 16 softmax warps
 constexpr float RAISE_THRESHOLD = 14.0f;            // log2 units by which a tile must exceed the reference to raise it (P stays below 2^14, inside fp16)
 
 // named barrier over `nthreads` threads with an OR reduction of `pred` (all threads of the participating warps call it)
@@ -787,8 +366,8 @@ __device__ __forceinline__ void mask_cols32(uint32_t (&raw)[32], int c0, int lo_
 }
 
 template <bool LOWBIT_FP8>
-__global__ void __launch_bounds__(TCP_THREADS, 1)
-attn_tcp_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
+__global__ void __launch_bounds__(TC_THREADS, 1)
+attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
     constexpr int TBN = 64, BN = 64;
     using G = Geo<TBN>;
     constexpr int NST = G::NST;
@@ -1116,14 +695,8 @@ attn_tcp_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
 // ---------------------------------------------------------------------------------------------
 size_t attn_tc_workspace_bytes(const hyq_attn_args& a) { return tc_workspace_layout(a).total; }
 
-// which kernel serves 64-key tiles: two threads per query row (default), or one thread per row
-#ifndef HYQ_PAIRED_ROWS
-#define HYQ_PAIRED_ROWS 1
-#endif
-constexpr bool PAIRED_ROWS = HYQ_PAIRED_ROWS != 0;
-
-template <int TBN>
-static int launch_attn_tc_impl(const hyq_attn_args& a, float alpha, cudaStream_t st) {
+int launch_attn_tc(const hyq_attn_args& a, float alpha, cudaStream_t st) {
+    constexpr int TBN = 64;                                             // keys per tile
     const TcWorkspace w = tc_workspace_layout(a);
     const int rc = launch_tc_prepass(a, w, st);
     if (rc != HYQ_OK) return rc;
@@ -1154,22 +727,16 @@ static int launch_attn_tc_impl(const hyq_attn_args& a, float alpha, cudaStream_t
     p.vl_bits = reinterpret_cast<const uint32_t*>(base + w.vl_bits);
     p.out = a.out; p.lse = a.lse; p.status = a.status_word;
 
-    const bool paired = PAIRED_ROWS && TBN == 64;
-    auto kern = paired ? (int4 ? attn_tcp_kernel<true> : attn_tcp_kernel<false>)
-                       : (int4 ? attn_tc_kernel<true, TBN> : attn_tc_kernel<false, TBN>);
+    auto kern = int4 ? attn_tc_kernel<true> : attn_tc_kernel<false>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM_BYTES) != cudaSuccess)
         return HYQ_ERR_CUDA;
     const dim3 grid((a.L + QT * BM - 1) / (QT * BM), a.Hq, a.B);
     if (a.ev_kernel_start && cudaEventRecord(static_cast<cudaEvent_t>(a.ev_kernel_start), st) != cudaSuccess) return HYQ_ERR_CUDA;
-    kern<<<grid, paired ? TCP_THREADS : TC_THREADS, TC_SMEM_BYTES, st>>>(maps, p);
+    kern<<<grid, TC_THREADS, TC_SMEM_BYTES, st>>>(maps, p);
     if (launch_status() != HYQ_OK) return HYQ_ERR_CUDA;
     if (a.ev_kernel_stop && cudaEventRecord(static_cast<cudaEvent_t>(a.ev_kernel_stop), st) != cudaSuccess) return HYQ_ERR_CUDA;
     return HYQ_OK;
 }
-
-// 64-key tiles (two S buffers per query tile) measured faster than 128-key tiles (one buffer) on every
-// benchmark configuration; the kernel template keeps both geometries.
-int launch_attn_tc(const hyq_attn_args& a, float alpha, cudaStream_t st) { return launch_attn_tc_impl<64>(a, alpha, st); }
 
 }  // namespace hyq
 
