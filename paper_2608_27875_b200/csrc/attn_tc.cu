@@ -463,7 +463,6 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
             const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
             const uint32_t to = tmem + tm_o(q) + lane_addr, ts0 = tmem + tm_s(q) + lane_addr;
             const float q_scale = row_live ? __ldg(p.q_scales + (long)qhead * p.nb + i / HYQ_BLOCK_TOKENS) : 0.0f;
-            const int cnt_r = (sq.nB > 0 && row_live && i - W >= 0) ? count_le(idx_row, p.k, i - W) : 0;
             constexpr uint32_t knock_lq = LOWBIT_FP8 ? KNOCKOUT_F32 : KNOCKOUT_S32;
             float m_used = -INFINITY, l_h = 0.0f;               // reference maximum of the row; row sum of this half
             bool dead = false;                                  // this warp ran into an expired wait
@@ -607,6 +606,8 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                 if (!do_tile(std::false_type{}, n, cs, vl, !LOWBIT_FP8, 0, 0u)) { aborted = true; break; }
             }
             // ---- the remaining low-bit tiles, the vertical-line tiles and the window tiles
+            // (number of vertical-line keys this row may use: only needed from here on)
+            const int cnt_r = (!aborted && sq.nB > 0 && row_live && i - W >= 0) ? count_le(idx_row, p.k, i - W) : 0;
             for (; n < n_total && !aborted; ++n) {
                 HYQ_TR(q * 2 + hsel, n, 2);
                 const int t = walk_pos(n);
