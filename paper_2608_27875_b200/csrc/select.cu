@@ -102,33 +102,21 @@ __device__ __forceinline__ unsigned long long order_key(double s) {
     return (u >> 63) ? ~u : (u | 0x8000000000000000ull);
 }
 
-// exclusive prefix of a 0/1 flag over the CTA, plus the CTA total
-__device__ __forceinline__ int block_exclusive_scan(bool flag, int* warp_tot, int& total) {
-    const unsigned ball = __ballot_sync(0xffffffffu, flag);
-    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-    const int in_warp = __popc(ball & ((1u << lane) - 1u));
-    __syncthreads();                                  // warp_tot is reused by consecutive scans
-    if (lane == 0) warp_tot[wid] = __popc(ball);
-    __syncthreads();
-    int before = 0, tot = 0;
-#pragma unroll
-    for (int w = 0; w < TOPK_THREADS / 32; ++w) {
-        const int c = warp_tot[w];
-        before += (w < wid) ? c : 0;
-        tot += c;
-    }
-    total = tot;
-    return before + in_warp;
-}
-
+// One CTA per (b, query head); every warp owns a contiguous segment of the row (coalesced reads, no CTA-wide
+// synchronisation inside a scan of the row).
 __global__ void __launch_bounds__(TOPK_THREADS)
 topk_kernel(const double* __restrict__ scores, int P, int k, int32_t* __restrict__ idx_out) {
+    constexpr int NW = TOPK_THREADS / 32;
+    __shared__ int whist[NW][256];                     // one digit histogram per warp (no contention across warps)
     __shared__ int hist[256];
-    __shared__ int warp_tot[TOPK_THREADS / 32];
+    __shared__ int warp_gt[NW], warp_eq[NW];
     __shared__ unsigned long long sh_prefix;
     __shared__ int sh_krem;
     const double* row = scores + (long)blockIdx.x * P;
     int32_t* out = idx_out + (long)blockIdx.x * k;
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    const int per = (P + NW - 1) / NW;
+    const int seg0 = min(P, wid * per), seg1 = min(P, seg0 + per);
 
     // radix select: after the loop `prefix` is the key of the k-th largest score and k_rem how
     // many positions holding exactly that key are still to be taken
@@ -136,45 +124,77 @@ topk_kernel(const double* __restrict__ scores, int P, int k, int32_t* __restrict
     int k_rem = k;
     for (int pass = 0; pass < 8; ++pass) {
         const int shift = 56 - 8 * pass;
-        for (int e = threadIdx.x; e < 256; e += TOPK_THREADS) hist[e] = 0;
-        __syncthreads();
-        for (int p = threadIdx.x; p < P; p += TOPK_THREADS) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) whist[wid][lane + 32 * e] = 0;
+        __syncwarp();
+        for (int p = seg0 + lane; p < seg1; p += 32) {
             const unsigned long long key = order_key(row[p]);
             if (pass == 0 || (key >> (shift + 8)) == (prefix >> (shift + 8)))
-                atomicAdd(&hist[(int)((key >> shift) & 0xFF)], 1);
+                atomicAdd(&whist[wid][(int)((key >> shift) & 0xFF)], 1);
         }
         __syncthreads();
-        if (threadIdx.x == 0) {
-            int cum = 0, d = 255;
-            for (; d > 0; --d) {
-                if (cum + hist[d] >= k_rem) break;
-                cum += hist[d];
+        if (threadIdx.x < 256) {
+            int tot = 0;
+#pragma unroll 8
+            for (int w = 0; w < NW; ++w) tot += whist[w][threadIdx.x];
+            hist[threadIdx.x] = tot;
+        }
+        __syncthreads();
+        // the digit d whose bin holds the k_rem-th largest candidate: the largest d with
+        // count(bins above d) < k_rem <= count(bins d and above); lane l of warp 0 looks at bins 255-8l .. 248-8l
+        if (wid == 0) {
+            const int hi = 255 - 8 * lane;
+            int mine = 0;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) mine += hist[hi - j];
+            int incl = mine;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int v = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += v;
             }
-            sh_prefix = prefix | ((unsigned long long)d << shift);
-            sh_krem = k_rem - cum;
+            int above = incl - mine;                   // candidates in bins above this lane's eight
+            if (above < k_rem && k_rem <= incl) {      // exactly one lane (the candidates number at least k_rem)
+                int d = hi;
+                for (; d > hi - 7; --d) {
+                    if (above + hist[d] >= k_rem) break;
+                    above += hist[d];
+                }
+                sh_prefix = prefix | ((unsigned long long)d << shift);
+                sh_krem = k_rem - above;
+            }
         }
         __syncthreads();
         prefix = sh_prefix;
         k_rem = sh_krem;
-        __syncthreads();
     }
 
-    // ordered compaction: positions ascending; among keys equal to the threshold the first k_rem
-    int taken = 0, eq_seen = 0;
-    for (int base = 0; base < P; base += TOPK_THREADS) {
-        const int p = base + threadIdx.x;
-        unsigned long long key = 0ull;
-        const bool live = p < P;
-        if (live) key = order_key(row[p]);
-        const bool eq = live && key == prefix;
-        int eq_tot, sel_tot;
-        const int eq_rank = eq_seen + block_exclusive_scan(eq, warp_tot, eq_tot);
-        const bool sel = live && (key > prefix || (eq && eq_rank < k_rem));
-        const int pos = taken + block_exclusive_scan(sel, warp_tot, sel_tot);
-        if (sel && pos < k) out[pos] = p;
-        eq_seen += eq_tot;
-        taken += sel_tot;
-        if (taken >= k) break;
+    // ordered compaction: positions ascending; among keys equal to the threshold the first k_rem.
+    // Scan 1 counts, per warp segment, the keys above and equal to the threshold; scan 2 writes: the output
+    // slot of a selected position = (keys above the threshold before it) + min(keys equal before it, k_rem).
+    int n_gt = 0, n_eq = 0;
+    for (int base = seg0; base < seg1; base += 32) {
+        const int p = base + lane;
+        const unsigned long long key = (p < seg1) ? order_key(row[p]) : 0ull;
+        n_gt += __popc(__ballot_sync(0xffffffffu, p < seg1 && key > prefix));
+        n_eq += __popc(__ballot_sync(0xffffffffu, p < seg1 && key == prefix));
+    }
+    if (lane == 0) { warp_gt[wid] = n_gt; warp_eq[wid] = n_eq; }
+    __syncthreads();
+    int gt_run = 0, eq_run = 0;
+    for (int w = 0; w < wid; ++w) { gt_run += warp_gt[w]; eq_run += warp_eq[w]; }
+    const unsigned lt_mask = (1u << lane) - 1u;
+    for (int base = seg0; base < seg1; base += 32) {
+        const int p = base + lane;
+        const bool live = p < seg1;
+        const unsigned long long key = live ? order_key(row[p]) : 0ull;
+        const bool gt = live && key > prefix, eq = live && key == prefix;
+        const unsigned b_gt = __ballot_sync(0xffffffffu, gt), b_eq = __ballot_sync(0xffffffffu, eq);
+        const int eq_rank = eq_run + __popc(b_eq & lt_mask);
+        const int pos = gt_run + __popc(b_gt & lt_mask) + min(eq_rank, k_rem);
+        if ((gt || (eq && eq_rank < k_rem)) && pos < k) out[pos] = p;
+        gt_run += __popc(b_gt);
+        eq_run += __popc(b_eq);
     }
 }
 
