@@ -155,6 +155,53 @@ def test_tensor_core_and_cuda_core_kernels_agree_on_every_output_of_config1():
     assert float(diff.sum() / outs[1].abs().sum()) <= MEAN_REL_TOL
 
 
+def _two_kernels(Q, K, V, fmts, W, k):
+    Qd, Kd, Vd = Q.cuda(), K.cuda(), V.cuda()
+    if k == 0:
+        idx = None
+    elif W == 0:        # no observation window to select from: any ascending index set serves
+        idx = torch.from_numpy(_rand_idx(Q.shape[0], Q.shape[1], Q.shape[2], k, seed=k)).cuda()
+    else:
+        idx = api.hyq_select_vertical(Qd, Kd, W, k)
+    (qc, qs), (kc, ks), (vc, vs) = [api.hyq_quantize_blocks(t, f) for t, f in zip((Qd, Kd, Vd), fmts)]
+    outs = [api.hyq_hybrid_attention_prefill(Qd, Kd, Vd, qc, kc, vc, qs, ks, vs, fmts, idx, W, impl=impl)
+            for impl in (api.IMPL_TCGEN05, api.IMPL_SIMT, api.IMPL_TCGEN05)]
+    torch.cuda.synchronize()
+    return outs
+
+
+@pytest.mark.parametrize("seed", range(32))
+def test_random_shapes_tensor_core_matches_cuda_core_and_repeats_bit_for_bit(seed):
+    """Seeded random shapes (ragged lengths, windows off the tile grid, GQA groups, both format sets, flat
+    and steeply rising score profiles): the tensor-core kernel and the plain CUDA-core kernel are
+    independent implementations of the same definition and must agree on every output; two runs of the
+    tensor-core kernel on the same inputs must be identical bit for bit (no dependence on timing)."""
+    ensure_built()
+    rng = np.random.default_rng(1000 + seed)
+    g = torch.Generator().manual_seed(2000 + seed)
+    long_rows = seed >= 24                        # a few cases with dozens of key tiles per query tile
+    B = 1 if long_rows else int(rng.integers(1, 3))
+    Hkv = 1 if long_rows else int(rng.integers(1, 3))
+    Hq = Hkv * int(rng.choice([1, 2, 4]))
+    L = int(rng.integers(2000, 6000)) if long_rows else int(rng.integers(1, 1400))
+    W = int(rng.choice([0, 1, 17, 64, 100, 128, 300, 1024]))
+    k = int(rng.integers(0, max(1, min(L - W, 64)))) if L - W > 0 else 0
+    fmts = INT8 if seed % 2 == 0 else INT4FP8
+    u = torch.randn(128, generator=g)
+    u = u / u.norm()
+    slope = float(rng.choice([0.0, 0.0, 20.0, -20.0, 60.0]))
+    ramp = torch.linspace(0.0, 1.0, L)[:, None]
+    Q = (0.3 * torch.randn(B, Hq, L, 128, generator=g) + 6.0 * u).to(torch.bfloat16)
+    K = (0.3 * torch.randn(B, Hkv, L, 128, generator=g) + (slope * ramp) * u).to(torch.bfloat16)
+    V = torch.randn(B, Hkv, L, 128, generator=g).to(torch.bfloat16)
+    tc, simt, tc_again = _two_kernels(Q, K, V, fmts, W, k)
+    assert torch.isfinite(tc).all()
+    assert torch.equal(tc, tc_again)
+    diff = (tc - simt).abs()
+    assert float(diff.max()) <= MAX_ABS_TOL, (B, Hq, Hkv, L, W, k, slope, float(diff.max()))
+    assert float(diff.sum() / simt.abs().sum().clamp_min(1e-30)) <= MEAN_REL_TOL, (B, Hq, Hkv, L, W, k, slope)
+
+
 @pytest.mark.parametrize("impl", IMPLS)
 @pytest.mark.parametrize("fmts", [INT8, INT4FP8])
 def test_row_maximum_that_keeps_rising_along_the_keys(impl, fmts):
