@@ -36,7 +36,7 @@ def build(force: bool = False) -> str:
 
 class _AttnIn(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int) for n in
-                ("B", "Hq", "Hkv", "L", "D", "W", "k", "block_tokens", "q_fmt", "k_fmt", "v_fmt")] + [
+                ("B", "Hq", "Hkv", "L", "Lq", "D", "W", "k", "block_tokens", "q_fmt", "k_fmt", "v_fmt")] + [
         ("alpha", ctypes.c_double)] + [(n, ctypes.c_void_p) for n in
                                        ("q", "k_", "v", "q_codes", "k_codes", "v_codes",
                                         "q_scales", "k_scales", "v_scales", "vl_idx")]
@@ -121,21 +121,22 @@ def select_vertical(q_bits, k_bits, window: int, k: int, n_tail: int = 0, return
 
 def _attn_in(q_bits, k_bits, v_bits, qc, kc, vc, qs, ks, vs, fmts, vl_idx, window, block_tokens, alpha):
     q, kk, v = _u16(q_bits, 4), _u16(k_bits, 4), _u16(v_bits, 4)
-    B, Hq, L, D = q.shape
-    Hkv = kk.shape[1]
-    assert kk.shape == (B, Hkv, L, D) and v.shape == kk.shape
+    B, Hq, Lq, D = q.shape                      # Lq query rows, end-aligned with the L keys (Lq == L: whole prefill)
+    Hkv, L = kk.shape[1], kk.shape[2]
+    assert kk.shape == (B, Hkv, L, D) and v.shape == kk.shape and 0 < Lq <= L
     qc, kc, vc = (np.ascontiguousarray(c, dtype=np.uint8) for c in (qc, kc, vc))
     qs, ks, vs = (np.ascontiguousarray(s, dtype=np.float32) for s in (qs, ks, vs))
     nb = (L + block_tokens - 1) // block_tokens
-    assert qc.shape == (B, Hq, L, code_row_bytes(fmts[0], D)), qc.shape
+    nbq = (Lq + block_tokens - 1) // block_tokens
+    assert qc.shape == (B, Hq, Lq, code_row_bytes(fmts[0], D)), qc.shape
     assert kc.shape == (B, Hkv, L, code_row_bytes(fmts[1], D)), kc.shape
     assert vc.shape == (B, Hkv, L, code_row_bytes(fmts[2], D)), vc.shape
-    assert qs.shape == (B, Hq, nb) and ks.shape == (B, Hkv, nb) and vs.shape == (B, Hkv, nb)
+    assert qs.shape == (B, Hq, nbq) and ks.shape == (B, Hkv, nb) and vs.shape == (B, Hkv, nb)
     if vl_idx is None:
         vl_idx = np.zeros((B, Hq, 0), dtype=np.int32)
     vl = np.ascontiguousarray(vl_idx, dtype=np.int32)
     assert vl.shape[:2] == (B, Hq)
-    a = _AttnIn(B=B, Hq=Hq, Hkv=Hkv, L=L, D=D, W=window, k=vl.shape[2], block_tokens=block_tokens,
+    a = _AttnIn(B=B, Hq=Hq, Hkv=Hkv, L=L, Lq=Lq, D=D, W=window, k=vl.shape[2], block_tokens=block_tokens,
                 q_fmt=fmts[0], k_fmt=fmts[1], v_fmt=fmts[2],
                 alpha=(1.0 / np.sqrt(D)) if alpha is None else float(alpha),
                 q=q.ctypes.data, k_=kk.ctypes.data, v=v.ctypes.data,
@@ -143,14 +144,16 @@ def _attn_in(q_bits, k_bits, v_bits, qc, kc, vc, qs, ks, vs, fmts, vl_idx, windo
                 q_scales=qs.ctypes.data, k_scales=ks.ctypes.data, v_scales=vs.ctypes.data,
                 vl_idx=vl.ctypes.data)
     keep = (q, kk, v, qc, kc, vc, qs, ks, vs, vl)
-    return a, keep, (B, Hq, L, D)
+    return a, keep, (B, Hq, Lq, D)
 
 
 def attention_rows(q_bits, k_bits, v_bits, q_codes, k_codes, v_codes, q_scales, k_scales, v_scales,
                    fmts, vl_idx, window: int, rows=None, block_tokens: int = 64, alpha=None,
                    return_lse: bool = False, return_fp_pairs: bool = False):
     """Eq. 6-7 by definition (two-pass fp64 softmax over every key j <= i).
-    rows: query positions to compute (default all).  Returns fp64 [B,Hq,n_rows,D]."""
+    q holds Lq <= L query rows, end-aligned with the L keys (the query block of Algorithm 2; row r sits at
+    position L - Lq + r); Lq == L is the whole prefill.
+    rows: rows of the query block to compute (default all).  Returns fp64 [B,Hq,n_rows,D]."""
     a, keep, (B, Hq, L, D) = _attn_in(q_bits, k_bits, v_bits, q_codes, k_codes, v_codes, q_scales,
                                       k_scales, v_scales, fmts, vl_idx, window, block_tokens, alpha)
     rows = np.arange(L, dtype=np.int32) if rows is None else np.ascontiguousarray(rows, dtype=np.int32)

@@ -205,8 +205,11 @@ int oracle_select(const uint16_t* q, const uint16_t* k_, int B, int Hq, int Hkv,
 /* out is [B,Hq,n_rows,D] fp64, lse (optional) is [B,Hq,n_rows].              */
 /* fp_pairs (optional) returns the number of FP pairs met.                    */
 /* ------------------------------------------------------------------------- */
+/* L: number of keys (L_K).  Lq: number of query rows (the query block of Algorithm 2), end-aligned with
+   the keys: query row i sits at position L - Lq + i.  Lq = L is the whole prefill.  q, q_codes and q_scales
+   hold Lq rows (quantization blocks counted from the first row of the block). */
 typedef struct {
-    int B, Hq, Hkv, L, D, W, k, block_tokens;
+    int B, Hq, Hkv, L, Lq, D, W, k, block_tokens;
     int q_fmt, k_fmt, v_fmt;
     double alpha;
     const uint16_t *q, *k_, *v;
@@ -246,13 +249,13 @@ static double* widen_head(const uint16_t* x, int L, int D) {
 typedef struct { double *qf, *qh, *kf, *kh, *vf, *vh; } head_views_t;
 
 static int load_head(const attn_in_t* a, int b, int h, head_views_t* hv) {
-    const int g = a->Hq / a->Hkv, kvh = h / g, L = a->L, D = a->D, bt = a->block_tokens;
-    const int nb = (L + bt - 1) / bt;
+    const int g = a->Hq / a->Hkv, kvh = h / g, L = a->L, Lq = a->Lq, D = a->D, bt = a->block_tokens;
+    const int nb = (L + bt - 1) / bt, nbq = (Lq + bt - 1) / bt;
     const long qo = ((long)b * a->Hq + h), ko = ((long)b * a->Hkv + kvh);
-    hv->qf = widen_head(a->q + qo * L * D, L, D);
+    hv->qf = widen_head(a->q + qo * Lq * D, Lq, D);
     hv->kf = widen_head(a->k_ + ko * L * D, L, D);
     hv->vf = widen_head(a->v + ko * L * D, L, D);
-    hv->qh = dequant_head(a->q_codes + qo * L * code_row_bytes(a->q_fmt, D), a->q_scales + qo * nb, a->q_fmt, L, D, bt);
+    hv->qh = dequant_head(a->q_codes + qo * Lq * code_row_bytes(a->q_fmt, D), a->q_scales + qo * nbq, a->q_fmt, Lq, D, bt);
     hv->kh = dequant_head(a->k_codes + ko * L * code_row_bytes(a->k_fmt, D), a->k_scales + ko * nb, a->k_fmt, L, D, bt);
     hv->vh = dequant_head(a->v_codes + ko * L * code_row_bytes(a->v_fmt, D), a->v_scales + ko * nb, a->v_fmt, L, D, bt);
     return (hv->qf && hv->kf && hv->vf && hv->qh && hv->kh && hv->vh) ? 0 : 2;
@@ -273,8 +276,8 @@ static double pair_score(const attn_in_t* a, const head_views_t* hv, int i, int 
 
 int oracle_attention_rows(const attn_in_t* a, const int32_t* rows, int n_rows, double* out,
                           double* lse, long long* fp_pairs) {
-    if (a->Hkv <= 0 || a->Hq % a->Hkv) return 1;
-    const int D = a->D, L = a->L;
+    if (a->Hkv <= 0 || a->Hq % a->Hkv || a->Lq <= 0 || a->Lq > a->L) return 1;
+    const int D = a->D, L = a->L, off = a->L - a->Lq;   /* query row r sits at position off + r */
     long long fp_total = 0;
     int err = 0;
     for (int bh = 0; bh < a->B * a->Hq && !err; ++bh) {
@@ -285,9 +288,9 @@ int oracle_attention_rows(const attn_in_t* a, const int32_t* rows, int n_rows, d
         mark_vl(a, b, h, is_vl);
 #pragma omp parallel for schedule(dynamic) reduction(+ : fp_total)
         for (int r = 0; r < n_rows; ++r) {
-            const int i = rows[r];
+            const int qi = rows[r], i = qi + off;      /* row of the query block, its position among the keys */
             double* o = out + ((long)bh * n_rows + r) * D;
-            if (i < 0 || i >= L) { err = 1; continue; }
+            if (qi < 0 || qi >= a->Lq) { err = 1; continue; }
             double* s = (double*)malloc(sizeof(double) * (i + 1));
             uint8_t* fp = (uint8_t*)malloc((size_t)(i + 1));
             if (!s || !fp) { err = 2; free(s); free(fp); continue; }
@@ -295,7 +298,7 @@ int oracle_attention_rows(const attn_in_t* a, const int32_t* rows, int n_rows, d
             for (int j = 0; j <= i; ++j) {
                 fp[j] = (uint8_t)(is_vl[j] || (i - j < a->W));
                 fp_total += fp[j];
-                s[j] = pair_score(a, &hv, i, j, fp[j]);
+                s[j] = pair_score(a, &hv, qi, j, fp[j]);
                 if (s[j] > m) m = s[j];
             }
             double denom = 0.0;
@@ -344,8 +347,8 @@ static void flash_os(const double* s, const double* const* vals, int n, int D, d
 
 int oracle_attention_segmented_rows(const attn_in_t* a, const int32_t* rows, int n_rows, int tile_n,
                                     double* out) {
-    if (a->Hkv <= 0 || a->Hq % a->Hkv || tile_n <= 0) return 1;
-    const int D = a->D, L = a->L;
+    if (a->Hkv <= 0 || a->Hq % a->Hkv || tile_n <= 0 || a->Lq <= 0 || a->Lq > a->L) return 1;
+    const int D = a->D, L = a->L, off = a->L - a->Lq;
     for (int bh = 0; bh < a->B * a->Hq; ++bh) {
         const int b = bh / a->Hq, h = bh % a->Hq;
         uint8_t* is_vl = (uint8_t*)malloc((size_t)L);
@@ -354,7 +357,7 @@ int oracle_attention_segmented_rows(const attn_in_t* a, const int32_t* rows, int
         mark_vl(a, b, h, is_vl);
 #pragma omp parallel for schedule(dynamic)
         for (int r = 0; r < n_rows; ++r) {
-            const int i = rows[r];
+            const int qi = rows[r], i = qi + off;
             double* o = out + ((long)bh * n_rows + r) * D;
             double m = -INFINITY, l = 0.0;
             double* acc = (double*)calloc((size_t)D, sizeof(double));
@@ -371,7 +374,7 @@ int oracle_attention_segmented_rows(const attn_in_t* a, const int32_t* rows, int
                     const int n = (n_mem - t0 < tile_n) ? n_mem - t0 : tile_n;
                     for (int c = 0; c < n; ++c) {
                         const int j = members[t0 + c];
-                        s[c] = pair_score(a, &hv, i, j, seg != 0);
+                        s[c] = pair_score(a, &hv, qi, j, seg != 0);
                         vals[c] = ((seg != 0) ? hv.vf : hv.vh) + (long)j * D;
                     }
                     flash_os(s, vals, n, D, &m, &l, acc);

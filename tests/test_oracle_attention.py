@@ -183,3 +183,69 @@ def test_hybrid_reduces_error_as_the_paper_reports():
     qz8 = _quant(Q, K, V, (INT8,) * 3)
     e8 = np.abs(_call(Q, K, V, qz8, (INT8,) * 3, None, 0) - exact).mean()
     assert e8 < 0.25 * err["uniform"]
+
+
+# ---- query block shorter than the keys (Algorithm 2: a query block against the full K, V; end-aligned) ----------
+@pytest.mark.parametrize("fmts", [(INT8, INT8, INT8), (INT4, INT4, FP8)])
+def test_block_aligned_query_block_reproduces_the_tail_rows_of_the_whole_prefill(fmts):
+    """When the query block starts on a quantization-block boundary its codes and scales are slices of the
+    whole prefill's, every (row, key) pair is classified and scored alike, and the rows must come out
+    identical to the last rows of the whole prefill, bit for bit."""
+    L, W, kk, bt, D = 200, 24, 7, 8, 16
+    q, k, v = _qkv(B=2, Hq=4, Hkv=2, L=L, D=D, seed=3)
+    qz = _quant(q, k, v, fmts, bt)
+    idx = _rand_idx(2, 4, L, W, kk, seed=5)
+    full = _call(q, k, v, qz, fmts, idx, W, bt=bt)
+    for Lq in (bt, 5 * bt, L):                   # offsets L - Lq = 192, 160, 0: multiples of the block size
+        off = L - Lq
+        (qc, qs), kz, vz = qz
+        qz_blk = ((qc[:, :, off:], qs[:, :, off // bt:]), kz, vz)
+        got = _call(q[:, :, off:], k, v, qz_blk, fmts, idx, W, bt=bt)
+        assert got.shape == (2, 4, Lq, D)
+        assert np.array_equal(got, full[:, :, off:])
+
+
+def test_single_query_row_with_a_covering_window_is_the_textbook_softmax():
+    """L_Q = 1 and W >= L_K: every pair is full precision, the row is the last position."""
+    L, D = 37, 16
+    q, k, v = _qkv(B=1, Hq=2, Hkv=1, L=L, D=D, seed=8)
+    q1 = q[:, :, -1:]
+    fm = (INT8, INT8, INT8)
+    qz = [oracle.quantize(wl.bits(q1), INT8, 64), oracle.quantize(wl.bits(k), INT8, 64), oracle.quantize(wl.bits(v), INT8, 64)]
+    got, lse = _call(q1, k, v, qz, fm, None, L, return_lse=True)
+    s = torch.einsum("bhqd,bkd->bhqk", q1.double(), k[:, 0].double()) / math.sqrt(D)
+    ref = torch.einsum("bhqk,bkd->bhqd", torch.softmax(s, -1), v[:, 0].double())
+    assert np.abs(got - ref.numpy()).max() < 1e-12
+    assert np.abs(lse - torch.logsumexp(s, -1).numpy()).max() < 1e-12
+
+
+@pytest.mark.parametrize("Lq", [1, 13, 70])
+def test_query_block_off_the_block_grid_segmented_walk_and_pair_count(Lq):
+    """A query block that does not start on a quantization-block boundary carries its own Q blocks.  The
+    literal three-segment walk must agree with the single softmax, and the number of full-precision pairs
+    has a closed form: row r sits at position p = L - Lq + r and has min(p + 1, W) window keys plus the
+    vertical keys at positions <= p - W."""
+    L, W, kk, bt, D = 150, 20, 9, 16, 16
+    fmts = (INT8, INT8, INT8)
+    q, k, v = _qkv(B=1, Hq=2, Hkv=2, L=L, D=D, seed=11)
+    qb = q[:, :, L - Lq:]
+    qz = _quant(qb, k, v, fmts, bt)
+    idx = _rand_idx(1, 2, L, W, kk, seed=2)
+    got, n_fp = _call(qb, k, v, qz, fmts, idx, W, bt=bt, return_fp_pairs=True)
+    (qc, qs), (kc, ks), (vc, vs) = qz
+    seg = oracle.attention_segmented_rows(wl.bits(qb), wl.bits(k), wl.bits(v), qc, kc, vc, qs, ks, vs, fmts, idx, W,
+                                          None, 8, bt)
+    assert np.abs(got - seg).max() < 1e-12
+    expect = 0
+    for h in range(2):
+        for r in range(Lq):
+            p = L - Lq + r
+            expect += min(p + 1, W) + int((idx[0, h] <= p - W).sum())
+    assert n_fp == expect
+
+
+def test_query_block_longer_than_the_keys_is_rejected():
+    q, k, v = _qkv(B=1, Hq=1, Hkv=1, L=20, D=16, seed=1)
+    qz = _quant(q, k[:, :, :10], v[:, :, :10], (INT8, INT8, INT8), 64)
+    with pytest.raises((ValueError, AssertionError)):
+        _call(q, k[:, :, :10], v[:, :, :10], qz, (INT8, INT8, INT8), None, 4)
