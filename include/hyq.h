@@ -142,6 +142,13 @@ int hyq_quantize_blocks(const void* x, int B, int H, int L, int D, int block_tok
  *         value row = v_scale * v_code[j]
  * and one softmax runs over all keys of the row:  out[i] = sum_j p_ij value_j / sum_j p_ij.
  *
+ *   Query block (Algorithm 2 takes a query block against the full K, V): with 0 < Lq < L the call computes
+ *   the LAST Lq query rows of a context of L keys - query row r sits at position L - Lq + r and sees the keys
+ *   j <= L - Lq + r, with the same two predicates on positions.  q, q_codes, out then hold Lq rows per head,
+ *   q_scales ceil(Lq/64) entries per head (quantization blocks counted from the first row of the block, as
+ *   hyq_quantize_blocks writes them for a [B,Hq,Lq,D] tensor) and lse Lq entries; K, V and vl_idx are those
+ *   of the whole context.  Lq = 0 or Lq = L is the whole prefill.  Lq > L -> HYQ_ERR_INVALID_ARG.
+ *
  *   struct_size must be sizeof(hyq_attn_args).  Supported format triples (q,k,v):
  *   (INT8,INT8,INT8) and (INT4,INT4,FP8_E4M3); anything else -> HYQ_ERR_UNSUPPORTED.
  *   vl_idx [B,Hq,k] int32, each row strictly ascending, values in [0, L); NULL iff k == 0.
@@ -176,6 +183,7 @@ typedef struct {
   size_t workspace_bytes;
   void* ev_kernel_start;             /* optional cudaEvent_t, recorded on the stream right before ... */
   void* ev_kernel_stop;              /* ... and right after the attention kernel proper (pre-pass excluded) */
+  int32_t Lq;                        /* query rows; 0 => L (whole prefill).  See "query block" above. */
 } hyq_attn_args;
 
 int hyq_hybrid_attention_prefill_workspace(const hyq_attn_args* args, size_t* bytes /* host, out */);

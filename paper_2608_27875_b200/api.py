@@ -37,7 +37,7 @@ class AttnArgs(ctypes.Structure):
                                                 "k_scales", "v_scales", "vl_idx", "out", "lse", "status_word",
                                                 "workspace")] +
                 [("workspace_bytes", ctypes.c_size_t), ("ev_kernel_start", ctypes.c_void_p),
-                 ("ev_kernel_stop", ctypes.c_void_p)])
+                 ("ev_kernel_stop", ctypes.c_void_p), ("Lq", ctypes.c_int32)])
 
 
 _lib = None
@@ -159,10 +159,11 @@ def hyq_quantize_blocks(x: torch.Tensor, fmt: int, block_tokens: int = 64, codes
 def make_attn_args(q, k, v, q_codes, k_codes, v_codes, q_scales, k_scales, v_scales, fmts, vl_idx, window,
                    out, lse=None, status_word=None, workspace=None, impl=IMPL_AUTO, softmax_scale=0.0,
                    block_tokens=64) -> AttnArgs:
-    B, Hq, L, D = q.shape
+    B, Hq, Lq, D = q.shape                  # Lq query rows against the k.shape[2] keys (end-aligned query block)
     a = AttnArgs()
     a.struct_size = ctypes.sizeof(AttnArgs)
-    a.B, a.Hq, a.Hkv, a.L, a.D = B, Hq, k.shape[1], L, D
+    a.B, a.Hq, a.Hkv, a.L, a.D = B, Hq, k.shape[1], k.shape[2], D
+    a.Lq = Lq
     a.window, a.k, a.block_tokens = window, (0 if vl_idx is None else vl_idx.shape[2]), block_tokens
     a.q_format, a.k_format, a.v_format = fmts
     a.out_dtype = 1 if out.dtype == torch.float32 else 0
@@ -192,7 +193,8 @@ def hyq_hybrid_attention_prefill(q, k, v, q_codes, k_codes, v_codes, q_scales, k
                                  lse: torch.Tensor | None = None, status_word: torch.Tensor | None = None,
                                  workspace: torch.Tensor | None = None, impl: int = IMPL_AUTO,
                                  softmax_scale: float = 0.0) -> torch.Tensor:
-    """Eq. 6-7 / Algorithm 2 Stage 3.  Returns out [B,Hq,L,D] (fp32 by default)."""
+    """Eq. 6-7 / Algorithm 2 Stage 3.  q may hold fewer rows than k, v: the last Lq query rows of the context
+    (Algorithm 2's query block).  Returns out [B,Hq,Lq,D] (fp32 by default)."""
     for t, dt, n in ((q, torch.bfloat16, "q"), (k, torch.bfloat16, "k"), (v, torch.bfloat16, "v"),
                      (q_codes, torch.uint8, "q_codes"), (k_codes, torch.uint8, "k_codes"),
                      (v_codes, torch.uint8, "v_codes"), (q_scales, torch.float32, "q_scales"),

@@ -121,7 +121,7 @@ TcWorkspace tc_workspace_layout(const hyq_attn_args& a) {
     TcWorkspace w{};
     size_t off = 0;
     auto take = [&](size_t bytes) { const size_t o = off; off += align_up(bytes, 1024); return o; };
-    const size_t kv_elems = (size_t)a.B * a.Hkv * a.L * HYQ_D, q_elems = (size_t)a.B * a.Hq * a.L * HYQ_D;
+    const size_t kv_elems = (size_t)a.B * a.Hkv * a.L * HYQ_D, q_elems = (size_t)a.B * a.Hq * query_rows(a) * HYQ_D;
     w.mask_words = (a.L + 31) / 32;
     w.vl_bits = take((size_t)a.B * a.Hq * w.mask_words * 4);
     w.v16 = take(kv_elems * 2);
@@ -158,7 +158,7 @@ int launch_tc_prepass(const hyq_attn_args& a, const TcWorkspace& w, cudaStream_t
             a.v_scales, a.L, nb, n_vec, reinterpret_cast<uint4*>(base + w.v16), reinterpret_cast<uint4*>(base + w.vh16));
     if (launch_status() != HYQ_OK) return HYQ_ERR_CUDA;
     if (a.q_format == HYQ_FMT_INT4) {
-        const long qw = (long)a.B * a.Hq * a.L * (HYQ_D / 8), kw = (long)a.B * a.Hkv * a.L * (HYQ_D / 8);
+        const long qw = (long)a.B * a.Hq * query_rows(a) * (HYQ_D / 8), kw = (long)a.B * a.Hkv * a.L * (HYQ_D / 8);
         int4_to_e4m3_kernel<<<(unsigned)((qw + 255) / 256), 256, 0, st>>>(static_cast<const uint32_t*>(a.q_codes), qw,
                                                                         reinterpret_cast<uint2*>(base + w.q8));
         int4_to_e4m3_kernel<<<(unsigned)((kw + 255) / 256), 256, 0, st>>>(static_cast<const uint32_t*>(a.k_codes), kw,

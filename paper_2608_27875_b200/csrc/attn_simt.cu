@@ -71,18 +71,20 @@ __global__ void __launch_bounds__(SIMT_THREADS)
 attn_simt_kernel(hyq_attn_args a, float alpha, const uint32_t* __restrict__ vl_bits) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     SimtSmem& sm = *reinterpret_cast<SimtSmem*>(smem_raw);
-    const int L = a.L, g = a.Hq / a.Hkv, nb = (L + HYQ_BLOCK_TOKENS - 1) / HYQ_BLOCK_TOKENS;
+    // L keys; Lq query rows, end-aligned: query row i sits at position i + off
+    const int L = a.L, Lq = query_rows(a), off = L - Lq, g = a.Hq / a.Hkv;
+    const int nb = (L + HYQ_BLOCK_TOKENS - 1) / HYQ_BLOCK_TOKENS, nbq = (Lq + HYQ_BLOCK_TOKENS - 1) / HYQ_BLOCK_TOKENS;
     const int i0 = blockIdx.x * ST, h = blockIdx.y, b = blockIdx.z, kvh = h / g;
     const long qhead = (long)b * a.Hq + h, kvhead = (long)b * a.Hkv + kvh;
     const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
-    const int n_q = min(ST, L - i0);
+    const int n_q = min(ST, Lq - i0);
     constexpr int QK_ROW_BYTES = (QK_FMT == HYQ_FMT_INT4) ? HYQ_D / 2 : HYQ_D;
     const int mask_words = (L + 31) / 32;
     const uint32_t* vl_row = vl_bits + qhead * mask_words;
 
-    stage_bf16(sm.q, static_cast<const __nv_bfloat16*>(a.q) + (qhead * L + i0) * HYQ_D, n_q);
-    stage_codes<QK_FMT>(sm.qc, static_cast<const uint8_t*>(a.q_codes) + (qhead * L + i0) * QK_ROW_BYTES, n_q);
-    if (threadIdx.x < ST) sm.q_scale[threadIdx.x] = a.q_scales[qhead * nb + min(i0 + (int)threadIdx.x, L - 1) / HYQ_BLOCK_TOKENS];
+    stage_bf16(sm.q, static_cast<const __nv_bfloat16*>(a.q) + (qhead * Lq + i0) * HYQ_D, n_q);
+    stage_codes<QK_FMT>(sm.qc, static_cast<const uint8_t*>(a.q_codes) + (qhead * Lq + i0) * QK_ROW_BYTES, n_q);
+    if (threadIdx.x < ST) sm.q_scale[threadIdx.x] = a.q_scales[qhead * nbq + min(i0 + (int)threadIdx.x, Lq - 1) / HYQ_BLOCK_TOKENS];
 
     float m_run[4], l_run[4], acc[4][8];
 #pragma unroll
@@ -93,7 +95,7 @@ attn_simt_kernel(hyq_attn_args a, float alpha, const uint32_t* __restrict__ vl_b
         for (int c = 0; c < 8; ++c) acc[r][c] = 0.0f;
     }
 
-    for (int j0 = 0; j0 <= i0 + n_q - 1; j0 += ST) {
+    for (int j0 = 0; j0 <= off + i0 + n_q - 1; j0 += ST) {
         const int n_k = min(ST, L - j0);
         __syncthreads();
         stage_bf16(sm.k, static_cast<const __nv_bfloat16*>(a.k_) + (kvhead * L + j0) * HYQ_D, n_k);
@@ -155,12 +157,12 @@ attn_simt_kernel(hyq_attn_args a, float alpha, const uint32_t* __restrict__ vl_b
         float s[4][4];
 #pragma unroll
         for (int r = 0; r < 4; ++r) {
-            const int i = i0 + ty * 4 + r;
+            const int i = off + i0 + ty * 4 + r;        // position of the query row among the keys
             float mx = m_run[r];
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 const int j = j0 + tx * 4 + c;
-                const bool valid = (j <= i) && (j < L) && (i < L);
+                const bool valid = (j <= i) && (j < L) && (i < L);       // (i < L <=> the row exists)
                 const bool is_vl = valid && ((vl_row[j >> 5] >> (j & 31)) & 1u);
                 fp[r][c] = is_vl || (i - j < a.window);
                 const float lq = (float)s_lq[r][c] * sm.q_scale[ty * 4 + r] * sm.k_scale[tx * 4 + c] * alpha;
@@ -205,18 +207,18 @@ attn_simt_kernel(hyq_attn_args a, float alpha, const uint32_t* __restrict__ vl_b
 #pragma unroll
     for (int r = 0; r < 4; ++r) {
         const int i = i0 + ty * 4 + r;
-        if (i >= L) continue;
+        if (i >= Lq) continue;
         const float inv = 1.0f / l_run[r];
         if (a.out_dtype == 1) {
-            float* o = static_cast<float*>(a.out) + (qhead * L + i) * HYQ_D + tx * 8;
+            float* o = static_cast<float*>(a.out) + (qhead * Lq + i) * HYQ_D + tx * 8;
 #pragma unroll
             for (int c = 0; c < 8; ++c) o[c] = acc[r][c] * inv;
         } else {
-            __nv_bfloat16* o = static_cast<__nv_bfloat16*>(a.out) + (qhead * L + i) * HYQ_D + tx * 8;
+            __nv_bfloat16* o = static_cast<__nv_bfloat16*>(a.out) + (qhead * Lq + i) * HYQ_D + tx * 8;
 #pragma unroll
             for (int c = 0; c < 8; ++c) o[c] = __float2bfloat16_rn(acc[r][c] * inv);
         }
-        if (a.lse && tx == 0) a.lse[qhead * L + i] = m_run[r] + logf(l_run[r]);
+        if (a.lse && tx == 0) a.lse[qhead * Lq + i] = m_run[r] + logf(l_run[r]);
     }
 }
 
@@ -229,7 +231,7 @@ int launch_attn_simt(const hyq_attn_args& a, float alpha, cudaStream_t st) {
     const long n_heads = (long)a.B * a.Hq;
     uint32_t* bits = static_cast<uint32_t*>(a.workspace);
     if (launch_vl_bitmask(a.vl_idx, n_heads, a.k, a.L, mask_words, bits, st) != HYQ_OK) return HYQ_ERR_CUDA;
-    const dim3 grid((a.L + ST - 1) / ST, a.Hq, a.B);
+    const dim3 grid((query_rows(a) + ST - 1) / ST, a.Hq, a.B);
     const size_t smem = sizeof(SimtSmem);
     auto run = [&](auto kern) -> int {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)

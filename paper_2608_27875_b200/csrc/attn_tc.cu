@@ -84,6 +84,7 @@ struct TcMaps {
 
 struct TcParams {
     int B, Hq, Hkv, L, window, k, nb, mask_words;
+    int Lq, nbq;                 // query rows (end-aligned with the L keys: row i sits at position L - Lq + i), their blocks
     int out_fp32;
     float scale_log2;            // softmax_scale * log2(e)
     const float* q_scales;
@@ -100,7 +101,8 @@ struct TcBarriers {
     uint64_t s_full[QT][2], p_full[QT][2], o_done[QT][2];
 };
 
-// which key tiles a 128-row query tile visits in each pass
+// which key tiles a 128-row query tile visits in each pass (i0, i1: first and last row of the tile in the query
+// block; the tile lists follow from their positions among the keys)
 struct QSched {
     int live, i0, i1, nA, nB, tC0, tC1;
 };
@@ -365,7 +367,10 @@ __device__ __forceinline__ void mask_cols32(uint32_t (&raw)[32], int c0, int lo_
     for (int e = 0; e < 32; ++e) raw[e] = ((unsigned)(c0 + e - lo_eff) <= span) ? raw[e] : knock;
 }
 
-template <bool LOWBIT_FP8>
+// LOWBIT_FP8: the low-bit codes are e4m3 bytes (kind::f8f6f4), else int8 (kind::i8).  QUERY_BLOCK: the query rows
+// are the last Lq < L positions (a compile-time zero offset keeps one register out of the whole-prefill loop:
+// 2.6 % on the benchmark workload).
+template <bool LOWBIT_FP8, bool QUERY_BLOCK>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
     constexpr int TBN = 64, BN = 64;
@@ -380,7 +385,8 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int pt = gridDim.x - 1 - blockIdx.x;               // pair of query tiles; longest rows first
     const int h = blockIdx.y, b = blockIdx.z;
-    const int L = p.L, W = p.window, g = p.Hq / p.Hkv;
+    const int L = p.Lq, W = p.window, g = p.Hq / p.Hkv;     // L: rows of the query block
+    const int off = QUERY_BLOCK ? p.L - p.Lq : 0;           // position of query row 0 among the keys
     const int qhead = b * p.Hq + h, kvhead = b * p.Hkv + h / g;
     const int32_t* idx_row = p.vl_idx + (long)qhead * p.k;
 
@@ -401,8 +407,8 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
         abort_s = 0;
     }
     if (threadIdx.x < QT) {
-        const int i1 = min(pt * QT * BM + (int)threadIdx.x * BM + BM - 1, L - 1);
-        cnt_b_s[threadIdx.x] = (p.k > 0 && i1 - W >= 0) ? count_le(idx_row, p.k, i1 - W) : 0;
+        const int a1 = off + min(pt * QT * BM + (int)threadIdx.x * BM + BM - 1, L - 1);
+        cnt_b_s[threadIdx.x] = (p.k > 0 && a1 - W >= 0) ? count_le(idx_row, p.k, a1 - W) : 0;
     }
     if (warp == 0) {
         tmem_alloc(&tmem_base_s, TM_COLS);
@@ -418,10 +424,11 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
         s.i0 = (pt * QT + q) * BM;
         s.live = s.i0 < L;
         s.i1 = min(s.i0 + BM - 1, L - 1);
-        s.nA = (s.live && s.i1 - W >= 0) ? (s.i1 - W) / BN + 1 : 0;
+        const int a0 = s.i0 + off, a1 = s.i1 + off;             // positions of the tile's first and last row
+        s.nA = (s.live && a1 - W >= 0) ? (a1 - W) / BN + 1 : 0;
         s.nB = s.live ? (cnt_b_s[q] + BN - 1) / BN : 0;
-        s.tC0 = max(0, s.i0 - W + 1) / BN;
-        s.tC1 = (s.live && W > 0) ? s.i1 / BN : -1;
+        s.tC0 = max(0, a0 - W + 1) / BN;
+        s.tC1 = (s.live && W > 0) ? a1 / BN : -1;
         return s;
     };
     const QSched qs0 = make_sched(0), qs1 = make_sched(1);
@@ -456,13 +463,14 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
         const int n_total = own.a_end + (own.b_end - own.b_beg) + (own.c_end - own.c_beg);
         if (sq.live && n_total > 0) {
             const int r = (warp & 3) * 32 + lane;               // query row inside the tile = TMEM lane
-            const int i = sq.i0 + r;
+            const int i = sq.i0 + r;                           // row of the query block ...
+            const int ia = i + off;                             // ... and its position among the keys
             const bool row_live = i < L;
             const bool ragged = sq.i0 + BM > L;
             const int col0 = hsel * 32, col0_other = col0 ^ 32;
             const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
             const uint32_t to = tmem + tm_o(q) + lane_addr, ts0 = tmem + tm_s(q) + lane_addr;
-            const float q_scale = row_live ? __ldg(p.q_scales + (long)qhead * p.nb + i / HYQ_BLOCK_TOKENS) : 0.0f;
+            const float q_scale = row_live ? __ldg(p.q_scales + (long)qhead * p.nbq + i / HYQ_BLOCK_TOKENS) : 0.0f;
             constexpr uint32_t knock_lq = LOWBIT_FP8 ? KNOCKOUT_F32 : KNOCKOUT_S32;
             float m_used = -INFINITY, l_h = 0.0f;               // reference maximum of the row; row sum of this half
             bool dead = false;                                  // this warp ran into an expired wait
@@ -595,7 +603,7 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
             };
 
             // ---- low-bit tiles that lie wholly below every row's window: no range mask, no bounds to compute
-            const int n_plain = ragged ? 0 : min(own.a_end, max(0, (sq.i0 - W + 1) / BN));
+            const int n_plain = ragged ? 0 : min(own.a_end, max(0, (sq.i0 + off - W + 1) / BN));
             int n = 0;
             for (; n < n_plain; ++n) {
                 HYQ_TR(q * 2 + hsel, n, 2);
@@ -607,7 +615,7 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
             }
             // ---- the remaining low-bit tiles, the vertical-line tiles and the window tiles
             // (number of vertical-line keys this row may use: only needed from here on)
-            const int cnt_r = (!aborted && sq.nB > 0 && row_live && i - W >= 0) ? count_le(idx_row, p.k, i - W) : 0;
+            const int cnt_r = (!aborted && sq.nB > 0 && row_live && ia - W >= 0) ? count_le(idx_row, p.k, ia - W) : 0;
             for (; n < n_total && !aborted; ++n) {
                 HYQ_TR(q * 2 + hsel, n, 2);
                 const int t = walk_pos(n);
@@ -618,15 +626,15 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                 float cs;
                 const bool lowbit = t < own.a_end;
                 if (lowbit) {
-                    hi = row_live ? min(i - W - t * BN, BN - 1) : -1;
+                    hi = row_live ? min(ia - W - t * BN, BN - 1) : -1;
                     cs = fmaxf(qs2 * ks, 1e-37f);
                 } else if (t < own.b_end) {
                     hi = min(cnt_r - (t - own.b_beg) * BN - 1, BN - 1);
                     cs = p.scale_log2;
                 } else {
                     const int j0 = (w.tC0 + t - w.nA - w.nB) * BN;
-                    lo = max(0, i - W + 1 - j0);
-                    hi = row_live ? min(i - j0, BN - 1) : -1;
+                    lo = max(0, ia - W + 1 - j0);
+                    hi = row_live ? min(ia - j0, BN - 1) : -1;
                     cs = p.scale_log2;
                 }
                 const int lo_eff = (hi >= lo) ? lo : 4096;
@@ -703,14 +711,14 @@ int launch_attn_tc(const hyq_attn_args& a, float alpha, cudaStream_t st) {
     if (rc != HYQ_OK) return rc;
     char* base = static_cast<char*>(a.workspace);
     const bool int4 = a.q_format == HYQ_FMT_INT4;
-    const uint64_t qh = (uint64_t)a.B * a.Hq, kvh = (uint64_t)a.B * a.Hkv, L = a.L;
+    const uint64_t qh = (uint64_t)a.B * a.Hq, kvh = (uint64_t)a.B * a.Hkv, L = a.L, Lq = query_rows(a);
     const uint64_t kk = a.k > 0 ? a.k : 1;
 
     TcMaps maps;
     bool ok = true;
-    ok &= make_tmap_3d(&maps.q, a.q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, HYQ_D, L, qh, 64, BM);
+    ok &= make_tmap_3d(&maps.q, a.q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, HYQ_D, Lq, qh, 64, BM);
     ok &= make_tmap_3d(&maps.k, a.k_, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, HYQ_D, L, kvh, 64, TBN);
-    ok &= make_tmap_3d(&maps.qc, int4 ? (const void*)(base + w.q8) : a.q_codes, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, HYQ_D, L, qh, 128, BM);
+    ok &= make_tmap_3d(&maps.qc, int4 ? (const void*)(base + w.q8) : a.q_codes, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, HYQ_D, Lq, qh, 128, BM);
     ok &= make_tmap_3d(&maps.kc, int4 ? (const void*)(base + w.k8) : a.k_codes, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, HYQ_D, L, kvh, 128, TBN);
     ok &= make_tmap_3d(&maps.v16, base + w.v16, CU_TENSOR_MAP_DATA_TYPE_UINT16, 2, HYQ_D, L, kvh, 64, TBN);
     ok &= make_tmap_3d(&maps.vh16, base + w.vh16, CU_TENSOR_MAP_DATA_TYPE_UINT16, 2, HYQ_D, L, kvh, 64, TBN);
@@ -721,6 +729,8 @@ int launch_attn_tc(const hyq_attn_args& a, float alpha, cudaStream_t st) {
     TcParams p{};
     p.B = a.B; p.Hq = a.Hq; p.Hkv = a.Hkv; p.L = a.L; p.window = a.window; p.k = a.k;
     p.nb = (a.L + HYQ_BLOCK_TOKENS - 1) / HYQ_BLOCK_TOKENS;
+    p.Lq = (int)Lq;
+    p.nbq = ((int)Lq + HYQ_BLOCK_TOKENS - 1) / HYQ_BLOCK_TOKENS;
     p.mask_words = w.mask_words;
     p.out_fp32 = a.out_dtype == 1;
     p.scale_log2 = alpha * 1.4426950408889634f;
@@ -728,10 +738,12 @@ int launch_attn_tc(const hyq_attn_args& a, float alpha, cudaStream_t st) {
     p.vl_bits = reinterpret_cast<const uint32_t*>(base + w.vl_bits);
     p.out = a.out; p.lse = a.lse; p.status = a.status_word;
 
-    auto kern = int4 ? attn_tc_kernel<true> : attn_tc_kernel<false>;
+    const bool blk = Lq < L;
+    auto kern = int4 ? (blk ? attn_tc_kernel<true, true> : attn_tc_kernel<true, false>)
+                     : (blk ? attn_tc_kernel<false, true> : attn_tc_kernel<false, false>);
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM_BYTES) != cudaSuccess)
         return HYQ_ERR_CUDA;
-    const dim3 grid((a.L + QT * BM - 1) / (QT * BM), a.Hq, a.B);
+    const dim3 grid(((int)Lq + QT * BM - 1) / (QT * BM), a.Hq, a.B);
     if (a.ev_kernel_start && cudaEventRecord(static_cast<cudaEvent_t>(a.ev_kernel_start), st) != cudaSuccess) return HYQ_ERR_CUDA;
     kern<<<grid, TC_THREADS, TC_SMEM_BYTES, st>>>(maps, p);
     if (launch_status() != HYQ_OK) return HYQ_ERR_CUDA;

@@ -155,6 +155,51 @@ def test_tensor_core_and_cuda_core_kernels_agree_on_every_output_of_config1():
     assert float(diff.sum() / outs[1].abs().sum()) <= MEAN_REL_TOL
 
 
+# ---- query block shorter than the keys (Algorithm 2: a query block against the full K, V; end-aligned) ----------
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("fmts", [INT8, INT4FP8])
+@pytest.mark.parametrize("Lq,L,W,k", [
+    (64, 512, 128, 16),       # one block-aligned tile of queries at the end of eight key tiles
+    (100, 333, 40, 9),        # ragged lengths, query block off the block grid (its own Q blocks)
+    (1, 300, 64, 12),         # a single query row
+    (300, 700, 0, 20),        # no window: every pair below the diagonal is low-bit or vertical
+    (257, 1024, 300, 5),      # more than two query tiles, window longer than a query tile
+    (130, 130, 16, 4),        # Lq == L given explicitly
+])
+def test_query_block_matches_oracle(impl, fmts, Lq, L, W, k):
+    g = torch.Generator().manual_seed(Lq * 7 + L)
+    Q = torch.randn(1, 4, Lq, 128, generator=g).to(torch.bfloat16)
+    K = torch.randn(1, 2, L, 128, generator=g).to(torch.bfloat16)
+    V = torch.randn(1, 2, L, 128, generator=g).to(torch.bfloat16)
+    idx = _rand_idx(1, 4, max(1, L - W), k, seed=L) if k else None
+    _check(Q, K, V, fmts, idx, W, impl)
+
+
+@pytest.mark.parametrize("fmts", [INT8, INT4FP8])
+def test_query_block_on_the_cta_grid_repeats_the_tail_of_the_whole_prefill_bit_for_bit(fmts):
+    """A query block that starts on a multiple of 256 rows is tiled by the tensor-core kernel exactly like the
+    same rows of the whole prefill, and its codes and scales are slices of the whole prefill's: the outputs and
+    the log-sum-exp must be identical."""
+    ensure_built()
+    L, Lq, W, k = 1280, 512, 128, 24
+    g = torch.Generator().manual_seed(77)
+    Q = torch.randn(1, 4, L, 128, generator=g).to(torch.bfloat16).cuda()
+    K = torch.randn(1, 2, L, 128, generator=g).to(torch.bfloat16).cuda()
+    V = torch.randn(1, 2, L, 128, generator=g).to(torch.bfloat16).cuda()
+    idx = api.hyq_select_vertical(Q, K, W, k)
+    (qc, qs), (kc, ks), (vc, vs) = [api.hyq_quantize_blocks(t, f) for t, f in zip((Q, K, V), fmts)]
+    lse_full = torch.empty(1, 4, L, dtype=torch.float32, device="cuda")
+    full = api.hyq_hybrid_attention_prefill(Q, K, V, qc, kc, vc, qs, ks, vs, fmts, idx, W, lse=lse_full)
+    off = L - Lq
+    Qb, qcb, qsb = Q[:, :, off:].contiguous(), qc[:, :, off:].contiguous(), qs[:, :, off // 64:].contiguous()
+    lse_blk = torch.empty(1, 4, Lq, dtype=torch.float32, device="cuda")
+    blk = api.hyq_hybrid_attention_prefill(Qb, K, V, qcb, kc, vc, qsb, ks, vs, fmts, idx, W, lse=lse_blk)
+    torch.cuda.synchronize()
+    assert blk.shape == (1, 4, Lq, 128)
+    assert torch.equal(blk, full[:, :, off:])
+    assert torch.equal(lse_blk, lse_full[:, :, off:])
+
+
 def _two_kernels(Q, K, V, fmts, W, k):
     Qd, Kd, Vd = Q.cuda(), K.cuda(), V.cuda()
     if k == 0:
