@@ -13,7 +13,8 @@
  *     Q is [B, Hq, L, D]; K and V are [B, Hkv, L, D]; bf16 unless stated.
  *     Hq % Hkv == 0; query head h reads kv head h / (Hq / Hkv) (Algorithm 1's
  *     reshape Hq -> Hkv x g).  D must be 128.  L >= 1 is arbitrary (ragged tails
- *     are handled); Lq == Lk == L.
+ *     are handled).  The attention call also takes a query block of Lq < L rows
+ *     (see there); everywhere else the queries number L.
  *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Calls
  *     enqueue work and return; they never synchronise.
  *   - The caller owns every buffer, including `workspace`; the library allocates
