@@ -36,7 +36,8 @@ def build(force: bool = False) -> str:
 
 class _AttnIn(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int) for n in
-                ("B", "Hq", "Hkv", "L", "Lq", "D", "W", "k", "block_tokens", "q_fmt", "k_fmt", "v_fmt")] + [
+                ("B", "Hq", "Hkv", "L", "Lq", "fixed_window", "D", "W", "k", "block_tokens", "q_fmt", "k_fmt",
+                 "v_fmt")] + [
         ("alpha", ctypes.c_double)] + [(n, ctypes.c_void_p) for n in
                                        ("q", "k_", "v", "q_codes", "k_codes", "v_codes",
                                         "q_scales", "k_scales", "v_scales", "vl_idx")]
@@ -119,7 +120,8 @@ def select_vertical(q_bits, k_bits, window: int, k: int, n_tail: int = 0, return
     return (idx, scores) if return_scores else idx
 
 
-def _attn_in(q_bits, k_bits, v_bits, qc, kc, vc, qs, ks, vs, fmts, vl_idx, window, block_tokens, alpha):
+def _attn_in(q_bits, k_bits, v_bits, qc, kc, vc, qs, ks, vs, fmts, vl_idx, window, block_tokens, alpha,
+             fixed_window=False):
     q, kk, v = _u16(q_bits, 4), _u16(k_bits, 4), _u16(v_bits, 4)
     B, Hq, Lq, D = q.shape                      # Lq query rows, end-aligned with the L keys (Lq == L: whole prefill)
     Hkv, L = kk.shape[1], kk.shape[2]
@@ -136,7 +138,7 @@ def _attn_in(q_bits, k_bits, v_bits, qc, kc, vc, qs, ks, vs, fmts, vl_idx, windo
         vl_idx = np.zeros((B, Hq, 0), dtype=np.int32)
     vl = np.ascontiguousarray(vl_idx, dtype=np.int32)
     assert vl.shape[:2] == (B, Hq)
-    a = _AttnIn(B=B, Hq=Hq, Hkv=Hkv, L=L, Lq=Lq, D=D, W=window, k=vl.shape[2], block_tokens=block_tokens,
+    a = _AttnIn(B=B, Hq=Hq, Hkv=Hkv, L=L, Lq=Lq, fixed_window=int(bool(fixed_window)), D=D, W=window, k=vl.shape[2], block_tokens=block_tokens,
                 q_fmt=fmts[0], k_fmt=fmts[1], v_fmt=fmts[2],
                 alpha=(1.0 / np.sqrt(D)) if alpha is None else float(alpha),
                 q=q.ctypes.data, k_=kk.ctypes.data, v=v.ctypes.data,
@@ -149,13 +151,15 @@ def _attn_in(q_bits, k_bits, v_bits, qc, kc, vc, qs, ks, vs, fmts, vl_idx, windo
 
 def attention_rows(q_bits, k_bits, v_bits, q_codes, k_codes, v_codes, q_scales, k_scales, v_scales,
                    fmts, vl_idx, window: int, rows=None, block_tokens: int = 64, alpha=None,
-                   return_lse: bool = False, return_fp_pairs: bool = False):
+                   return_lse: bool = False, return_fp_pairs: bool = False, fixed_window: bool = False):
     """Eq. 6-7 by definition (two-pass fp64 softmax over every key j <= i).
     q holds Lq <= L query rows, end-aligned with the L keys (the query block of Algorithm 2; row r sits at
     position L - Lq + r); Lq == L is the whole prefill.
+    fixed_window: the window keys are the last `window` keys for every row (Algorithm 2's K_Win taken literally)
+    instead of each row's own last `window` positions.
     rows: rows of the query block to compute (default all).  Returns fp64 [B,Hq,n_rows,D]."""
     a, keep, (B, Hq, L, D) = _attn_in(q_bits, k_bits, v_bits, q_codes, k_codes, v_codes, q_scales,
-                                      k_scales, v_scales, fmts, vl_idx, window, block_tokens, alpha)
+                                      k_scales, v_scales, fmts, vl_idx, window, block_tokens, alpha, fixed_window)
     rows = np.arange(L, dtype=np.int32) if rows is None else np.ascontiguousarray(rows, dtype=np.int32)
     out = np.zeros((B, Hq, len(rows), D), dtype=np.float64)
     lse = np.zeros((B, Hq, len(rows)), dtype=np.float64)
@@ -174,11 +178,11 @@ def attention_rows(q_bits, k_bits, v_bits, q_codes, k_codes, v_codes, q_scales, 
 
 def attention_segmented_rows(q_bits, k_bits, v_bits, q_codes, k_codes, v_codes, q_scales, k_scales,
                              v_scales, fmts, vl_idx, window: int, rows=None, tile_n: int = 64,
-                             block_tokens: int = 64, alpha=None):
+                             block_tokens: int = 64, alpha=None, fixed_window: bool = False):
     """Algorithm 2 Stage 3 taken literally (segments A, B, C with the running
     (m, l, acc) update).  Returns fp64 [B,Hq,n_rows,D]."""
     a, keep, (B, Hq, L, D) = _attn_in(q_bits, k_bits, v_bits, q_codes, k_codes, v_codes, q_scales,
-                                      k_scales, v_scales, fmts, vl_idx, window, block_tokens, alpha)
+                                      k_scales, v_scales, fmts, vl_idx, window, block_tokens, alpha, fixed_window)
     rows = np.arange(L, dtype=np.int32) if rows is None else np.ascontiguousarray(rows, dtype=np.int32)
     out = np.zeros((B, Hq, len(rows), D), dtype=np.float64)
     rc = _load().oracle_attention_segmented_rows(ctypes.byref(a), _ptr(rows), len(rows), tile_n, _ptr(out))

@@ -207,9 +207,11 @@ int oracle_select(const uint16_t* q, const uint16_t* k_, int B, int Hq, int Hkv,
 /* ------------------------------------------------------------------------- */
 /* L: number of keys (L_K).  Lq: number of query rows (the query block of Algorithm 2), end-aligned with
    the keys: query row i sits at position L - Lq + i.  Lq = L is the whole prefill.  q, q_codes and q_scales
-   hold Lq rows (quantization blocks counted from the first row of the block). */
+   hold Lq rows (quantization blocks counted from the first row of the block).
+   fixed_window: 0 = per-row sliding window (key j is a window key of the row at position i iff i - j < W);
+   1 = Algorithm 2's K_Win taken literally: the last W keys, [L - W, L), for every row of the block. */
 typedef struct {
-    int B, Hq, Hkv, L, Lq, D, W, k, block_tokens;
+    int B, Hq, Hkv, L, Lq, fixed_window, D, W, k, block_tokens;
     int q_fmt, k_fmt, v_fmt;
     double alpha;
     const uint16_t *q, *k_, *v;
@@ -264,6 +266,11 @@ static void free_head(head_views_t* hv) {
     free(hv->qf); free(hv->qh); free(hv->kf); free(hv->kh); free(hv->vf); free(hv->vh);
 }
 
+/* is key j a window key of the query row at position i? */
+static int in_window(const attn_in_t* a, int i, int j) {
+    return a->fixed_window ? (j >= a->L - a->W) : (i - j < a->W);
+}
+
 /* alpha * <q_i, k_j> in the pair's class */
 static double pair_score(const attn_in_t* a, const head_views_t* hv, int i, int j, int fp) {
     const int D = a->D;
@@ -296,7 +303,7 @@ int oracle_attention_rows(const attn_in_t* a, const int32_t* rows, int n_rows, d
             if (!s || !fp) { err = 2; free(s); free(fp); continue; }
             double m = -INFINITY;
             for (int j = 0; j <= i; ++j) {
-                fp[j] = (uint8_t)(is_vl[j] || (i - j < a->W));
+                fp[j] = (uint8_t)(is_vl[j] || in_window(a, i, j));
                 fp_total += fp[j];
                 s[j] = pair_score(a, &hv, qi, j, fp[j]);
                 if (s[j] > m) m = s[j];
@@ -367,7 +374,7 @@ int oracle_attention_segmented_rows(const attn_in_t* a, const int32_t* rows, int
             for (int seg = 0; seg < 3; ++seg) {
                 int n_mem = 0;                      /* keys of this segment, in position order */
                 for (int j = 0; j <= i; ++j) {
-                    const int cls = (i - j < a->W) ? 2 : (is_vl[j] ? 1 : 0);
+                    const int cls = in_window(a, i, j) ? 2 : (is_vl[j] ? 1 : 0);
                     if (cls == seg) members[n_mem++] = j;
                 }
                 for (int t0 = 0; t0 < n_mem; t0 += tile_n) {

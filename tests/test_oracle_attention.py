@@ -249,3 +249,48 @@ def test_query_block_longer_than_the_keys_is_rejected():
     qz = _quant(q, k[:, :, :10], v[:, :, :10], (INT8, INT8, INT8), 64)
     with pytest.raises((ValueError, AssertionError)):
         _call(q, k[:, :, :10], v[:, :, :10], qz, (INT8, INT8, INT8), None, 4)
+
+
+# ---- Algorithm 2's window taken literally: the last W keys for every row of the query block ------------------
+def test_fixed_tail_window_agrees_with_the_sliding_window_on_the_last_row_only():
+    """For the last row both window forms name the same keys, [L - W, L); for earlier rows the fixed window
+    holds fewer causal keys, so the classes differ and (with quantization error) so do the outputs."""
+    L, W, kk, bt = 120, 30, 6, 16
+    fmts = (INT8, INT8, INT8)
+    q, k, v = _qkv(B=1, Hq=2, Hkv=1, L=L, D=16, seed=21)
+    qz = _quant(q, k, v, fmts, bt)
+    idx = _rand_idx(1, 2, L, W, kk, seed=9)
+    slide = _call(q, k, v, qz, fmts, idx, W, bt=bt)
+    fixed = _call(q, k, v, qz, fmts, idx, W, bt=bt, fixed_window=True)
+    assert np.array_equal(slide[:, :, -1], fixed[:, :, -1])
+    assert not np.array_equal(slide[:, :, L // 2], fixed[:, :, L // 2])
+
+
+@pytest.mark.parametrize("Lq", [1, 25, 64, 150])
+def test_fixed_tail_window_pair_count_segments_and_full_precision_limit(Lq):
+    """Row at position p has max(0, p - (L - W) + 1) window keys and the vertical keys at positions <= p
+    (all of them lie below L - W); the literal three-segment walk agrees with the single softmax; and with
+    W >= L the fixed window covers every key, i.e. exact causal attention."""
+    L, W, kk, bt, D = 150, 40, 8, 16, 16
+    fmts = (INT4, INT4, FP8)
+    q, k, v = _qkv(B=1, Hq=2, Hkv=2, L=L, D=D, seed=31)
+    qb = q[:, :, L - Lq:]
+    qz = _quant(qb, k, v, fmts, bt)
+    idx = _rand_idx(1, 2, L, W, kk, seed=4)
+    got, n_fp = _call(qb, k, v, qz, fmts, idx, W, bt=bt, return_fp_pairs=True, fixed_window=True)
+    (qc, qs), (kc, ks), (vc, vs) = qz
+    seg = oracle.attention_segmented_rows(wl.bits(qb), wl.bits(k), wl.bits(v), qc, kc, vc, qs, ks, vs, fmts, idx, W,
+                                          None, 8, bt, fixed_window=True)
+    assert np.abs(got - seg).max() < 1e-12
+    expect = 0
+    for h in range(2):
+        for r in range(Lq):
+            p = L - Lq + r
+            expect += max(0, p - (L - W) + 1) + int((idx[0, h] <= p).sum())
+    assert n_fp == expect
+    exact = _call(qb, k, v, qz, fmts, None, L, bt=bt, fixed_window=True)
+    s = torch.einsum("bhqd,bhkd->bhqk", qb.double(), k.double()) / math.sqrt(D)
+    pos = torch.arange(L - Lq, L)[:, None]
+    s = s.masked_fill(torch.arange(L)[None, :] > pos, float("-inf"))
+    ref = torch.einsum("bhqk,bhkd->bhqd", torch.softmax(s, -1), v.double())
+    assert np.abs(exact - ref.numpy()).max() < 1e-12
