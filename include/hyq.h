@@ -150,6 +150,11 @@ int hyq_quantize_blocks(const void* x, int B, int H, int L, int D, int block_tok
  *   hyq_quantize_blocks writes them for a [B,Hq,Lq,D] tensor) and lse Lq entries; K, V and vl_idx are those
  *   of the whole context.  Lq = 0 or Lq = L is the whole prefill.  Lq > L -> HYQ_ERR_INVALID_ARG.
  *
+ *   Window form: HYQ_WINDOW_SLIDING - key j is a window key of the row at position i iff i - j < window (every
+ *   row has its own last `window` positions; the form the whole prefill needs).  HYQ_WINDOW_FIXED_TAIL -
+ *   Algorithm 2's K_Win taken literally: the window keys are the last `window` keys [L - window, L) for every
+ *   row of the block (rows before L - window then have no window keys).  Both forms agree on the last row.
+ *
  *   struct_size must be sizeof(hyq_attn_args).  Supported format triples (q,k,v):
  *   (INT8,INT8,INT8) and (INT4,INT4,FP8_E4M3); anything else -> HYQ_ERR_UNSUPPORTED.
  *   vl_idx [B,Hq,k] int32, each row strictly ascending, values in [0, L); NULL iff k == 0.
@@ -159,6 +164,8 @@ int hyq_quantize_blocks(const void* x, int B, int H, int L, int D, int block_tok
  *   bounded waits expires (the output is then undefined); untouched otherwise.
  *   ev_kernel_start / ev_kernel_stop: optional caller-created CUDA events for profiling (NULL to skip).
  * ------------------------------------------------------------------------------------------- */
+enum { HYQ_WINDOW_SLIDING = 0, HYQ_WINDOW_FIXED_TAIL = 1 };
+
 typedef struct {
   uint32_t struct_size;
   int32_t B, Hq, Hkv, L, D;
@@ -185,6 +192,7 @@ typedef struct {
   void* ev_kernel_start;             /* optional cudaEvent_t, recorded on the stream right before ... */
   void* ev_kernel_stop;              /* ... and right after the attention kernel proper (pre-pass excluded) */
   int32_t Lq;                        /* query rows; 0 => L (whole prefill).  See "query block" above. */
+  int32_t window_mode;               /* HYQ_WINDOW_SLIDING (0, default) or HYQ_WINDOW_FIXED_TAIL (1) */
 } hyq_attn_args;
 
 int hyq_hybrid_attention_prefill_workspace(const hyq_attn_args* args, size_t* bytes /* host, out */);

@@ -16,6 +16,7 @@ LIB_PATH = os.path.join(_HERE, "libhyq.so")
 
 HYQ_OK = 0
 IMPL_AUTO, IMPL_TCGEN05, IMPL_SIMT = 0, 1, 2
+WINDOW_SLIDING, WINDOW_FIXED_TAIL = 0, 1
 EXPORTS = ("hyq_status_string", "hyq_version", "hyq_paper_k", "hyq_select_vertical_workspace",
            "hyq_select_vertical", "hyq_select_vertical_static", "hyq_quantize_blocks", "hyq_hybrid_attention_prefill_workspace",
            "hyq_hybrid_attention_prefill")
@@ -37,7 +38,7 @@ class AttnArgs(ctypes.Structure):
                                                 "k_scales", "v_scales", "vl_idx", "out", "lse", "status_word",
                                                 "workspace")] +
                 [("workspace_bytes", ctypes.c_size_t), ("ev_kernel_start", ctypes.c_void_p),
-                 ("ev_kernel_stop", ctypes.c_void_p), ("Lq", ctypes.c_int32)])
+                 ("ev_kernel_stop", ctypes.c_void_p), ("Lq", ctypes.c_int32), ("window_mode", ctypes.c_int32)])
 
 
 _lib = None
@@ -158,12 +159,13 @@ def hyq_quantize_blocks(x: torch.Tensor, fmt: int, block_tokens: int = 64, codes
 
 def make_attn_args(q, k, v, q_codes, k_codes, v_codes, q_scales, k_scales, v_scales, fmts, vl_idx, window,
                    out, lse=None, status_word=None, workspace=None, impl=IMPL_AUTO, softmax_scale=0.0,
-                   block_tokens=64) -> AttnArgs:
+                   block_tokens=64, window_mode=WINDOW_SLIDING) -> AttnArgs:
     B, Hq, Lq, D = q.shape                  # Lq query rows against the k.shape[2] keys (end-aligned query block)
     a = AttnArgs()
     a.struct_size = ctypes.sizeof(AttnArgs)
     a.B, a.Hq, a.Hkv, a.L, a.D = B, Hq, k.shape[1], k.shape[2], D
     a.Lq = Lq
+    a.window_mode = window_mode
     a.window, a.k, a.block_tokens = window, (0 if vl_idx is None else vl_idx.shape[2]), block_tokens
     a.q_format, a.k_format, a.v_format = fmts
     a.out_dtype = 1 if out.dtype == torch.float32 else 0
@@ -192,7 +194,7 @@ def hyq_hybrid_attention_prefill(q, k, v, q_codes, k_codes, v_codes, q_scales, k
                                  vl_idx, window: int, out: torch.Tensor | None = None, out_dtype=torch.float32,
                                  lse: torch.Tensor | None = None, status_word: torch.Tensor | None = None,
                                  workspace: torch.Tensor | None = None, impl: int = IMPL_AUTO,
-                                 softmax_scale: float = 0.0) -> torch.Tensor:
+                                 softmax_scale: float = 0.0, window_mode: int = WINDOW_SLIDING) -> torch.Tensor:
     """Eq. 6-7 / Algorithm 2 Stage 3.  q may hold fewer rows than k, v: the last Lq query rows of the context
     (Algorithm 2's query block).  Returns out [B,Hq,Lq,D] (fp32 by default)."""
     for t, dt, n in ((q, torch.bfloat16, "q"), (k, torch.bfloat16, "k"), (v, torch.bfloat16, "v"),
@@ -205,7 +207,7 @@ def hyq_hybrid_attention_prefill(q, k, v, q_codes, k_codes, v_codes, q_scales, k
     if out is None:
         out = torch.empty(q.shape, dtype=out_dtype, device=q.device)
     args = make_attn_args(q, k, v, q_codes, k_codes, v_codes, q_scales, k_scales, v_scales, fmts, vl_idx, window,
-                          out, lse, status_word, workspace, impl, softmax_scale)
+                          out, lse, status_word, workspace, impl, softmax_scale, window_mode=window_mode)
     if workspace is None:
         need = hyq_hybrid_attention_prefill_workspace(args)
         workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=q.device)

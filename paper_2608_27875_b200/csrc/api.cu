@@ -97,6 +97,7 @@ static int check_attn(const hyq_attn_args* a, bool need_pointers) {
     if (!a || a->struct_size != sizeof(hyq_attn_args)) return HYQ_ERR_INVALID_ARG;
     if (a->B <= 0 || a->Hq <= 0 || a->Hkv <= 0 || a->L <= 0 || a->window < 0 || a->k < 0) return HYQ_ERR_INVALID_ARG;
     if (a->Hq % a->Hkv || a->k > a->L || a->Lq < 0 || a->Lq > a->L) return HYQ_ERR_INVALID_ARG;
+    if (a->window_mode != HYQ_WINDOW_SLIDING && a->window_mode != HYQ_WINDOW_FIXED_TAIL) return HYQ_ERR_INVALID_ARG;
     if (a->out_dtype != 0 && a->out_dtype != 1) return HYQ_ERR_INVALID_ARG;
     if (a->impl < HYQ_IMPL_AUTO || a->impl > HYQ_IMPL_SIMT) return HYQ_ERR_INVALID_ARG;
     if (a->D != HYQ_D || a->block_tokens != HYQ_BLOCK_TOKENS) return HYQ_ERR_UNSUPPORTED;

@@ -164,7 +164,7 @@ attn_simt_kernel(hyq_attn_args a, float alpha, const uint32_t* __restrict__ vl_b
                 const int j = j0 + tx * 4 + c;
                 const bool valid = (j <= i) && (j < L) && (i < L);       // (i < L <=> the row exists)
                 const bool is_vl = valid && ((vl_row[j >> 5] >> (j & 31)) & 1u);
-                fp[r][c] = is_vl || (i - j < a.window);
+                fp[r][c] = is_vl || (a.window_mode == HYQ_WINDOW_FIXED_TAIL ? (j >= L - a.window) : (i - j < a.window));
                 const float lq = (float)s_lq[r][c] * sm.q_scale[ty * 4 + r] * sm.k_scale[tx * 4 + c] * alpha;
                 s[r][c] = valid ? (fp[r][c] ? s_fp[r][c] * alpha : lq) : -INFINITY;
                 mx = fmaxf(mx, s[r][c]);

@@ -85,6 +85,7 @@ struct TcMaps {
 struct TcParams {
     int B, Hq, Hkv, L, window, k, nb, mask_words;
     int Lq, nbq;                 // query rows (end-aligned with the L keys: row i sits at position L - Lq + i), their blocks
+    int fixed_tail;              // window form: the last `window` keys for every row instead of each row's own
     int out_fp32;
     float scale_log2;            // softmax_scale * log2(e)
     const float* q_scales;
@@ -387,6 +388,12 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
     const int h = blockIdx.y, b = blockIdx.z;
     const int L = p.Lq, W = p.window, g = p.Hq / p.Hkv;     // L: rows of the query block
     const int off = QUERY_BLOCK ? p.L - p.Lq : 0;           // position of query row 0 among the keys
+    // Last low-bit-eligible key position of the row at position x: x - W with the per-row sliding window,
+    // min(x, L_K - W - 1) with the fixed tail window (both as min(x, lim) - wsub).  Its window keys start right
+    // after it, and the vertical keys it may use are those at or below it.
+    const int q_lim = (QUERY_BLOCK && p.fixed_tail) ? p.L - W - 1 : 0x7fffffff;
+    const int q_sub = (QUERY_BLOCK && p.fixed_tail) ? 0 : W;
+    auto qhi = [&](int x) -> int { return QUERY_BLOCK ? min(x, q_lim) - q_sub : x - W; };
     const int qhead = b * p.Hq + h, kvhead = b * p.Hkv + h / g;
     const int32_t* idx_row = p.vl_idx + (long)qhead * p.k;
 
@@ -408,7 +415,7 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
     }
     if (threadIdx.x < QT) {
         const int a1 = off + min(pt * QT * BM + (int)threadIdx.x * BM + BM - 1, L - 1);
-        cnt_b_s[threadIdx.x] = (p.k > 0 && a1 - W >= 0) ? count_le(idx_row, p.k, a1 - W) : 0;
+        cnt_b_s[threadIdx.x] = (p.k > 0 && qhi(a1) >= 0) ? count_le(idx_row, p.k, qhi(a1)) : 0;
     }
     if (warp == 0) {
         tmem_alloc(&tmem_base_s, TM_COLS);
@@ -425,9 +432,9 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
         s.live = s.i0 < L;
         s.i1 = min(s.i0 + BM - 1, L - 1);
         const int a0 = s.i0 + off, a1 = s.i1 + off;             // positions of the tile's first and last row
-        s.nA = (s.live && a1 - W >= 0) ? (a1 - W) / BN + 1 : 0;
+        s.nA = (s.live && qhi(a1) >= 0) ? qhi(a1) / BN + 1 : 0;
         s.nB = s.live ? (cnt_b_s[q] + BN - 1) / BN : 0;
-        s.tC0 = max(0, a0 - W + 1) / BN;
+        s.tC0 = max(0, qhi(a0) + 1) / BN;
         s.tC1 = (s.live && W > 0) ? a1 / BN : -1;
         return s;
     };
@@ -603,7 +610,7 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
             };
 
             // ---- low-bit tiles that lie wholly below every row's window: no range mask, no bounds to compute
-            const int n_plain = ragged ? 0 : min(own.a_end, max(0, (sq.i0 + off - W + 1) / BN));
+            const int n_plain = ragged ? 0 : min(own.a_end, max(0, (qhi(sq.i0 + off) + 1) / BN));
             int n = 0;
             for (; n < n_plain; ++n) {
                 HYQ_TR(q * 2 + hsel, n, 2);
@@ -615,7 +622,7 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
             }
             // ---- the remaining low-bit tiles, the vertical-line tiles and the window tiles
             // (number of vertical-line keys this row may use: only needed from here on)
-            const int cnt_r = (!aborted && sq.nB > 0 && row_live && ia - W >= 0) ? count_le(idx_row, p.k, ia - W) : 0;
+            const int cnt_r = (!aborted && sq.nB > 0 && row_live && qhi(ia) >= 0) ? count_le(idx_row, p.k, qhi(ia)) : 0;
             for (; n < n_total && !aborted; ++n) {
                 HYQ_TR(q * 2 + hsel, n, 2);
                 const int t = walk_pos(n);
@@ -626,14 +633,14 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                 float cs;
                 const bool lowbit = t < own.a_end;
                 if (lowbit) {
-                    hi = row_live ? min(ia - W - t * BN, BN - 1) : -1;
+                    hi = row_live ? min(qhi(ia) - t * BN, BN - 1) : -1;
                     cs = fmaxf(qs2 * ks, 1e-37f);
                 } else if (t < own.b_end) {
                     hi = min(cnt_r - (t - own.b_beg) * BN - 1, BN - 1);
                     cs = p.scale_log2;
                 } else {
                     const int j0 = (w.tC0 + t - w.nA - w.nB) * BN;
-                    lo = max(0, ia - W + 1 - j0);
+                    lo = max(0, qhi(ia) + 1 - j0);
                     hi = row_live ? min(ia - j0, BN - 1) : -1;
                     cs = p.scale_log2;
                 }
@@ -730,6 +737,7 @@ int launch_attn_tc(const hyq_attn_args& a, float alpha, cudaStream_t st) {
     p.B = a.B; p.Hq = a.Hq; p.Hkv = a.Hkv; p.L = a.L; p.window = a.window; p.k = a.k;
     p.nb = (a.L + HYQ_BLOCK_TOKENS - 1) / HYQ_BLOCK_TOKENS;
     p.Lq = (int)Lq;
+    p.fixed_tail = a.window_mode == HYQ_WINDOW_FIXED_TAIL;
     p.nbq = ((int)Lq + HYQ_BLOCK_TOKENS - 1) / HYQ_BLOCK_TOKENS;
     p.mask_words = w.mask_words;
     p.out_fp32 = a.out_dtype == 1;
@@ -738,7 +746,7 @@ int launch_attn_tc(const hyq_attn_args& a, float alpha, cudaStream_t st) {
     p.vl_bits = reinterpret_cast<const uint32_t*>(base + w.vl_bits);
     p.out = a.out; p.lse = a.lse; p.status = a.status_word;
 
-    const bool blk = Lq < L;
+    const bool blk = Lq < L || p.fixed_tail;      // the general instantiation (the other one is the whole prefill)
     auto kern = int4 ? (blk ? attn_tc_kernel<true, true> : attn_tc_kernel<true, false>)
                      : (blk ? attn_tc_kernel<false, true> : attn_tc_kernel<false, false>);
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM_BYTES) != cudaSuccess)

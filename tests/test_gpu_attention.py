@@ -175,6 +175,34 @@ def test_query_block_matches_oracle(impl, fmts, Lq, L, W, k):
     _check(Q, K, V, fmts, idx, W, impl)
 
 
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("fmts", [INT8, INT4FP8])
+@pytest.mark.parametrize("Lq,L,W,k", [
+    (64, 512, 128, 16),       # the block lies inside the fixed window
+    (100, 333, 40, 9),        # rows before L - W have no window keys at all
+    (1, 300, 64, 12),
+    (600, 600, 100, 20),      # the whole prefill with the fixed tail window
+    (257, 1024, 300, 5),
+    (90, 400, 0, 7),          # no window
+])
+def test_fixed_tail_window_matches_oracle(impl, fmts, Lq, L, W, k):
+    """Algorithm 2's K_Win taken literally: the last W keys are the window of every row of the query block."""
+    ensure_built()
+    g = torch.Generator().manual_seed(Lq * 11 + L)
+    Q = torch.randn(1, 4, Lq, 128, generator=g).to(torch.bfloat16)
+    K = torch.randn(1, 2, L, 128, generator=g).to(torch.bfloat16)
+    V = torch.randn(1, 2, L, 128, generator=g).to(torch.bfloat16)
+    idx = _rand_idx(1, 4, max(1, L - W), k, seed=L) if k else None
+    qz = oracle_quant_all(Q, K, V, fmts)
+    got = gpu_attention(Q, K, V, qz, fmts, idx, W, impl, window_mode=api.WINDOW_FIXED_TAIL).numpy()
+    (qc, qs), (kc, ks), (vc, vs) = qz
+    ref = oracle.attention_rows(wl.bits(Q), wl.bits(K), wl.bits(V), qc, kc, vc, qs, ks, vs, fmts, idx, W,
+                                fixed_window=True)
+    assert np.isfinite(got).all()
+    max_abs, mean_rel = errors(got, ref)
+    assert max_abs <= MAX_ABS_TOL and mean_rel <= MEAN_REL_TOL, (max_abs, mean_rel)
+
+
 @pytest.mark.parametrize("fmts", [INT8, INT4FP8])
 def test_query_block_on_the_cta_grid_repeats_the_tail_of_the_whole_prefill_bit_for_bit(fmts):
     """A query block that starts on a multiple of 256 rows is tiled by the tensor-core kernel exactly like the
@@ -245,6 +273,35 @@ def test_random_shapes_tensor_core_matches_cuda_core_and_repeats_bit_for_bit(see
     diff = (tc - simt).abs()
     assert float(diff.max()) <= MAX_ABS_TOL, (B, Hq, Hkv, L, W, k, slope, float(diff.max()))
     assert float(diff.sum() / simt.abs().sum().clamp_min(1e-30)) <= MEAN_REL_TOL, (B, Hq, Hkv, L, W, k, slope)
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_random_query_blocks_and_window_forms_both_kernels_agree(seed):
+    """Seeded random query blocks (any length up to the keys, on and off the tile grid) under both window
+    forms: the tensor-core and the CUDA-core kernel must agree everywhere."""
+    ensure_built()
+    rng = np.random.default_rng(5000 + seed)
+    g = torch.Generator().manual_seed(6000 + seed)
+    L = int(rng.integers(2, 1500))
+    Lq = int(rng.integers(1, L + 1))
+    W = int(rng.choice([0, 1, 50, 64, 200, 700]))
+    k = int(rng.integers(0, max(1, min(L - W, 48)))) if L - W > 0 else 0
+    mode = int(rng.integers(0, 2))
+    fmts = INT8 if seed % 2 == 0 else INT4FP8
+    Hkv = int(rng.integers(1, 3))
+    Hq = Hkv * int(rng.choice([1, 2]))
+    Q = torch.randn(1, Hq, Lq, 128, generator=g).to(torch.bfloat16).cuda()
+    K = torch.randn(1, Hkv, L, 128, generator=g).to(torch.bfloat16).cuda()
+    V = torch.randn(1, Hkv, L, 128, generator=g).to(torch.bfloat16).cuda()
+    idx = torch.from_numpy(_rand_idx(1, Hq, L - W, k, seed=seed)).cuda() if k else None
+    (qc, qs), (kc, ks), (vc, vs) = [api.hyq_quantize_blocks(t, f) for t, f in zip((Q, K, V), fmts)]
+    tc, simt = [api.hyq_hybrid_attention_prefill(Q, K, V, qc, kc, vc, qs, ks, vs, fmts, idx, W, impl=impl,
+                                                 window_mode=mode) for impl in (api.IMPL_TCGEN05, api.IMPL_SIMT)]
+    torch.cuda.synchronize()
+    assert tc.shape == (1, Hq, Lq, 128) and torch.isfinite(tc).all()
+    diff = (tc - simt).abs()
+    assert float(diff.max()) <= MAX_ABS_TOL, (L, Lq, W, k, mode, float(diff.max()))
+    assert float(diff.sum() / simt.abs().sum().clamp_min(1e-30)) <= MEAN_REL_TOL, (L, Lq, W, k, mode)
 
 
 @pytest.mark.parametrize("impl", IMPLS)
