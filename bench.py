@@ -30,6 +30,9 @@ if ROOT not in sys.path:
 from paper_2608_27875_b200 import workloads as wl  # noqa: E402
 
 METRIC = "hybrid prefill attention effective TFLOPS"
+# the arithmetic types the path computes in, per low-bit format of Q and K
+DTYPE_NOTE = {wl.FMT_INT4: "int4 x int4 -> f32 scores (e4m3 MMA), fp16 P.V, bf16 full-precision tiles",
+              wl.FMT_INT8: "int8 x int8 -> s32 scores, fp16 P.V, bf16 full-precision tiles"}
 NOMINAL = {"bf16_tflops": 2250.0, "lowbit_tflops": 4500.0, "hbm_gbs": 8000.0}
 FALLBACK = {"bf16_tflops": 1590.0, "hbm_gbs": 6650.0}
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu
@@ -277,6 +280,90 @@ class PipelinedHostPath:
         return max(int(p_.status.item()) for p_ in self.slots)
 
 
+def run_query_block(args, w: wl.Workload):
+    """`--lq N`: the same path for a query block of the last N rows against the full K, V (Algorithm 2's query
+    block; chunked prefill): select on the block's tail queries, quantize the block and K, V, fused attention with
+    Lq = N.  One JSON line with the metric on the block's causal pairs; device-resident inputs; one GPU."""
+    import ctypes
+    from paper_2608_27875_b200 import api, build
+    build.build()
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    L, Lq, D, W = w.L, args.lq, w.D, w.window
+    assert 0 < Lq <= L
+    Q, K, V = (t.to(dev) for t in wl.make_inputs(w))
+    Qb = Q[:, :, L - Lq:].contiguous()
+    mode = api.WINDOW_FIXED_TAIL if args.fixed_tail else api.WINDOW_SLIDING
+    nbq, nb = -(-Lq // 64), -(-L // 64)
+    e = lambda *sh, dt=torch.uint8: torch.empty(*sh, dtype=dt, device=dev)   # noqa: E731
+    idx = e(w.B, w.Hq, w.k, dt=torch.int32)
+    sel_ws = e(max(16, api.hyq_select_vertical_workspace(w.B, w.Hq, w.Hkv, Lq, L, D, W, w.k)))
+    qc, kc, vc = (e(w.B, h, n, api.code_row_bytes(f, D)) for h, n, f in zip((w.Hq, w.Hkv, w.Hkv), (Lq, L, L), w.fmts))
+    qs, ks, vs = e(w.B, w.Hq, nbq, dt=torch.float32), e(w.B, w.Hkv, nb, dt=torch.float32), e(w.B, w.Hkv, nb, dt=torch.float32)
+    out = e(w.B, w.Hq, Lq, D, dt=torch.float32)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    a = api.make_attn_args(Qb, K, V, qc, kc, vc, qs, ks, vs, w.fmts, idx, W, out, status_word=status, window_mode=mode)
+    ws = e(max(16, api.hyq_hybrid_attention_prefill_workspace(a)))
+    a.workspace, a.workspace_bytes = ws.data_ptr(), ws.numel()
+    kev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    for ev in kev:
+        ev.record()
+    a.ev_kernel_start, a.ev_kernel_stop = (ev.cuda_event for ev in kev)
+
+    def step():
+        api.hyq_select_vertical(Qb, K, W, w.k, workspace=sel_ws, out=idx)
+        api.hyq_quantize_blocks(Qb, w.q_fmt, codes=qc, scales=qs)
+        api.hyq_quantize_blocks(K, w.k_fmt, codes=kc, scales=ks)
+        api.hyq_quantize_blocks(V, w.v_fmt, codes=vc, scales=vs)
+        rc = api.lib().hyq_hybrid_attention_prefill(ctypes.byref(a), torch.cuda.current_stream().cuda_stream)
+        assert rc == 0, rc
+
+    for _ in range(max(3, args.warmup)):
+        step()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(0)
+    sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for _ in range(args.steps):
+        step()
+    ev1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    assert int(status.item()) == 0, "attention kernel reported a device-side error"
+    ms = ev0.elapsed_time(ev1) / args.steps
+    k_ms = kev[0].elapsed_time(kev[1])
+    off = L - Lq
+    pairs = w.B * w.Hq * (L * (L + 1) - off * (off + 1)) // 2
+    pos = torch.arange(off, L, device=dev)
+    if args.fixed_tail:
+        n_win = int(torch.clamp(pos - (L - W) + 1, min=0).sum()) * w.B * w.Hq
+        lim = torch.clamp(pos, max=L - W - 1)
+    else:
+        n_win = int(torch.clamp(pos + 1, max=W).sum()) * w.B * w.Hq
+        lim = pos - W
+    n_vl = int((idx.long().unsqueeze(-1) <= lim.view(1, 1, 1, -1)).sum()) if w.k else 0
+    n_fp = n_win + n_vl
+    peaks = measured_peaks()
+    flops = 4 * D * pairs
+    t_meas = 4 * D * (n_fp / (peaks["bf16_tflops"] * 1e12) + (pairs - n_fp) / (2 * peaks["bf16_tflops"] * 1e12))
+    t_nom = 4 * D * (n_fp / (NOMINAL["bf16_tflops"] * 1e12) + (pairs - n_fp) / (NOMINAL["lowbit_tflops"] * 1e12))
+    print(json.dumps({
+        "metric": METRIC, "value": flops / (ms * 1e-3) / 1e12, "unit": "TFLOPS", "n_gpus": 1, "steps": args.steps,
+        "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": DTYPE_NOTE.get(w.q_fmt, "mixed"), "data": "synthetic",
+        "config": {"workload": f"{w.name}, query block of the last {Lq} rows of {L}", "B": w.B, "Hq": w.Hq, "Hkv": w.Hkv,
+                   "L": L, "Lq": Lq, "D": D, "window": W, "window_form": "fixed tail" if args.fixed_tail else "sliding",
+                   "k": w.k, "formats": list(w.fmts), "step": "select + quantize Q block, K, V + fused attention",
+                   "l2": "K, V and their codes exceed L2" if 4 * w.B * w.Hkv * L * D > 126e6 else "inputs fit L2"},
+        "roofline": {"bound": "tensor", "kernel": "attn_tc_kernel", "achieved": flops / (k_ms * 1e-3) / 1e12,
+                     "peak": flops / t_meas / 1e12, "unit": "TFLOP/s", "frac": t_meas * 1e3 / k_ms, "traffic": None,
+                     "kernel_ms": k_ms, "frac_nominal": t_nom * 1e3 / k_ms, "fp_pair_share": n_fp / pairs,
+                     "peak_source": peaks["source"]},
+        "gpu_launches": (3 + 3 + (3 if w.k > 0 else 1) + (2 if w.q_fmt == wl.FMT_INT4 else 0) + 1) * args.steps,
+        "clocks": clocks}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -286,6 +373,8 @@ def main():
     ap.add_argument("--impl", default="hyq", choices=["hyq", "reference"])
     ap.add_argument("--seq", type=int, default=0, help="override the sequence length (profiling on a smaller case)")
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of oracle time for cpu_baseline")
+    ap.add_argument("--lq", type=int, default=0, help="measure a query block of the last LQ rows against the full K, V")
+    ap.add_argument("--fixed-tail", action="store_true", help="with --lq: Algorithm 2's fixed tail window")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "hyq" else args.warmup
     w = wl.CONFIGS[args.config]
@@ -293,6 +382,9 @@ def main():
         w = w.scaled(L=args.seq, k=max(1, w.k * args.seq // w.L), n_plant=max(1, w.n_plant * args.seq // w.L))
     if args.impl == "reference":
         run_reference(args, w)
+        return
+    if args.lq:
+        run_query_block(args, w)
         return
 
     import ctypes
@@ -414,8 +506,7 @@ def main():
     line = {
         "metric": METRIC, "value": value, "unit": "TFLOPS", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "int4 x int4 -> f32 scores (e4m3 MMA), fp16 P.V, bf16 full-precision tiles" if w.q_fmt == wl.FMT_INT4
-                 else "int8 x int8 -> s32 scores, fp16 P.V, bf16 full-precision tiles",
+        "dtype": DTYPE_NOTE[wl.FMT_INT4 if w.q_fmt == wl.FMT_INT4 else wl.FMT_INT8],
         "data": "synthetic",
         "config": {"workload": w.name, "B": w.B * world, "Hq": w.Hq, "Hkv": w.Hkv, "L": w.L, "D": w.D, "window": w.window,
                    "k": w.k, "formats": list(w.fmts), "l2": "inputs larger than L2 (Q+K+V bf16 = %.0f MB per step)" % (h2d / 1e6),
