@@ -32,7 +32,10 @@ from paper_2608_27875_b200 import workloads as wl  # noqa: E402
 METRIC = "hybrid prefill attention effective TFLOPS"
 # the arithmetic types the path computes in, per low-bit format of Q and K
 DTYPE_NOTE = {wl.FMT_INT4: "int4 x int4 -> f32 scores (e4m3 MMA), fp16 P.V, bf16 full-precision tiles",
-              wl.FMT_INT8: "int8 x int8 -> s32 scores, fp16 P.V, bf16 full-precision tiles"}
+              wl.FMT_INT8: "int8 x int8 -> s32 scores, fp16 P.V, bf16 full-precision tiles",
+              wl.FMT_FP8_E4M3: "e4m3 x e4m3 -> f32 scores, fp16 P.V, bf16 full-precision tiles"}
+FORMAT_SETS = {"int8": (wl.FMT_INT8,) * 3, "fp8": (wl.FMT_FP8_E4M3,) * 3,
+               "int4": (wl.FMT_INT4, wl.FMT_INT4, wl.FMT_FP8_E4M3)}
 NOMINAL = {"bf16_tflops": 2250.0, "lowbit_tflops": 4500.0, "hbm_gbs": 8000.0}
 FALLBACK = {"bf16_tflops": 1590.0, "hbm_gbs": 6650.0}
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu
@@ -375,11 +378,16 @@ def main():
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of oracle time for cpu_baseline")
     ap.add_argument("--lq", type=int, default=0, help="measure a query block of the last LQ rows against the full K, V")
     ap.add_argument("--fixed-tail", action="store_true", help="with --lq: Algorithm 2's fixed tail window")
+    ap.add_argument("--formats", default="", choices=["", *sorted(FORMAT_SETS)],
+                    help="override the workload's (Q, K, V) low-bit formats (default: as the workload defines them)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "hyq" else args.warmup
     w = wl.CONFIGS[args.config]
     if args.seq:
         w = w.scaled(L=args.seq, k=max(1, w.k * args.seq // w.L), n_plant=max(1, w.n_plant * args.seq // w.L))
+    if args.formats:
+        fq, fk, fv = FORMAT_SETS[args.formats]
+        w = w.scaled(q_fmt=fq, k_fmt=fk, v_fmt=fv)
     if args.impl == "reference":
         run_reference(args, w)
         return
@@ -506,7 +514,7 @@ def main():
     line = {
         "metric": METRIC, "value": value, "unit": "TFLOPS", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": DTYPE_NOTE[wl.FMT_INT4 if w.q_fmt == wl.FMT_INT4 else wl.FMT_INT8],
+        "dtype": DTYPE_NOTE[w.q_fmt],
         "data": "synthetic",
         "config": {"workload": w.name, "B": w.B * world, "Hq": w.Hq, "Hkv": w.Hkv, "L": w.L, "D": w.D, "window": w.window,
                    "k": w.k, "formats": list(w.fmts), "l2": "inputs larger than L2 (Q+K+V bf16 = %.0f MB per step)" % (h2d / 1e6),

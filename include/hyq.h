@@ -156,7 +156,8 @@ int hyq_quantize_blocks(const void* x, int B, int H, int L, int D, int block_tok
  *   row of the block (rows before L - window then have no window keys).  Both forms agree on the last row.
  *
  *   struct_size must be sizeof(hyq_attn_args).  Supported format triples (q,k,v):
- *   (INT8,INT8,INT8) and (INT4,INT4,FP8_E4M3); anything else -> HYQ_ERR_UNSUPPORTED.
+ *   (INT8,INT8,INT8), (FP8_E4M3,FP8_E4M3,FP8_E4M3) - the paper's two bit widths, c_B = 127 and 448 - and
+ *   (INT4,INT4,FP8_E4M3); anything else -> HYQ_ERR_UNSUPPORTED.
  *   vl_idx [B,Hq,k] int32, each row strictly ascending, values in [0, L); NULL iff k == 0.
  *   out [B,Hq,L,D]: fp32 (out_dtype 1) or bf16 (out_dtype 0, RNE of the fp32 result).
  *   lse: optional [B,Hq,L] fp32 natural-log-sum-exp of the scaled scores (NULL to skip).

@@ -103,7 +103,8 @@ static int check_attn(const hyq_attn_args* a, bool need_pointers) {
     if (a->D != HYQ_D || a->block_tokens != HYQ_BLOCK_TOKENS) return HYQ_ERR_UNSUPPORTED;
     const bool int8 = a->q_format == HYQ_FMT_INT8 && a->k_format == HYQ_FMT_INT8 && a->v_format == HYQ_FMT_INT8;
     const bool int4 = a->q_format == HYQ_FMT_INT4 && a->k_format == HYQ_FMT_INT4 && a->v_format == HYQ_FMT_FP8_E4M3;
-    if (!int8 && !int4) return HYQ_ERR_UNSUPPORTED;
+    const bool fp8 = a->q_format == HYQ_FMT_FP8_E4M3 && a->k_format == HYQ_FMT_FP8_E4M3 && a->v_format == HYQ_FMT_FP8_E4M3;
+    if (!int8 && !int4 && !fp8) return HYQ_ERR_UNSUPPORTED;
     if (!need_pointers) return HYQ_OK;
     const void* ptrs[] = {a->q, a->k_, a->v, a->q_codes, a->k_codes, a->v_codes, a->q_scales, a->k_scales, a->v_scales, a->out};
     for (const void* p : ptrs)

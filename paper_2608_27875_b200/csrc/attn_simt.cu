@@ -32,6 +32,11 @@ struct SimtSmem {
     float k_scale[ST];
 };
 
+__device__ __forceinline__ float e4m3_to_float(uint8_t code) {
+    const __half_raw hr = __nv_cvt_fp8_to_halfraw(code, __NV_E4M3);
+    return __half2float(__half(hr));
+}
+
 // 8 signed 4-bit codes (one 32-bit word) -> two words of int8 codes
 __device__ __forceinline__ void unpack_int4x8(uint32_t w, uint32_t& lo, uint32_t& hi) {
     uint32_t o[2] = {0u, 0u};
@@ -44,7 +49,7 @@ __device__ __forceinline__ void unpack_int4x8(uint32_t w, uint32_t& lo, uint32_t
     hi = o[1];
 }
 
-// stage `rows` code rows (int8 or packed int4) as int8 words; rows beyond n_rows are zero
+// stage `rows` code rows (int8, e4m3 bytes, or packed int4 widened to int8) as byte words; rows beyond n_rows are zero
 template <int FMT>
 __device__ __forceinline__ void stage_codes(uint32_t* dst, const uint8_t* src, int n_rows) {
     constexpr int ROW_WORDS = (FMT == HYQ_FMT_INT4) ? HYQ_D / 8 : HYQ_D / 4;
@@ -108,12 +113,7 @@ attn_simt_kernel(hyq_attn_args a, float alpha, const uint32_t* __restrict__ vl_b
                 vf = __bfloat162float(static_cast<const __nv_bfloat16*>(a.v)[(kvhead * L + j0 + r) * HYQ_D + c]);
                 const uint8_t code = static_cast<const uint8_t*>(a.v_codes)[(kvhead * L + j0 + r) * HYQ_D + c];
                 const float sv = a.v_scales[kvhead * nb + (j0 + r) / HYQ_BLOCK_TOKENS];
-                if (V_FMT == HYQ_FMT_INT8) {
-                    vq = (float)(int8_t)code * sv;
-                } else {
-                    const __half_raw hr = __nv_cvt_fp8_to_halfraw(code, __NV_E4M3);
-                    vq = __half2float(__half(hr)) * sv;
-                }
+                vq = ((V_FMT == HYQ_FMT_INT8) ? (float)(int8_t)code : e4m3_to_float(code)) * sv;
             }
             sm.v[r * V_STRIDE + c] = vf;
             sm.vh[r * V_STRIDE + c] = vq;
@@ -139,6 +139,11 @@ attn_simt_kernel(hyq_attn_args a, float alpha, const uint32_t* __restrict__ vl_b
 #pragma unroll
                 for (int c = 0; c < 4; ++c) s_fp[r][c] = fmaf(qh[r], kh[c], fmaf(ql[r], kl[c], s_fp[r][c]));
         }
+        float s_lqf[4][4];                               // e4m3 codes: the code products are summed as floats
+#pragma unroll
+        for (int r = 0; r < 4; ++r)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) s_lqf[r][c] = 0.0f;
         for (int w = 0; w < HYQ_D / 4; ++w) {
             int qv[4], kv[4];
 #pragma unroll
@@ -146,10 +151,27 @@ attn_simt_kernel(hyq_attn_args a, float alpha, const uint32_t* __restrict__ vl_b
                 qv[r] = (int)sm.qc[(ty * 4 + r) * C_STRIDE + w];
                 kv[r] = (int)sm.kc[(tx * 4 + r) * C_STRIDE + w];
             }
+            if (QK_FMT == HYQ_FMT_FP8_E4M3) {
+                float qf[4][4], kf[4][4];
 #pragma unroll
-            for (int r = 0; r < 4; ++r)
+                for (int r = 0; r < 4; ++r)
 #pragma unroll
-                for (int c = 0; c < 4; ++c) s_lq[r][c] = __dp4a(qv[r], kv[c], s_lq[r][c]);
+                    for (int e = 0; e < 4; ++e) {
+                        qf[r][e] = e4m3_to_float((uint8_t)((uint32_t)qv[r] >> (8 * e)));
+                        kf[r][e] = e4m3_to_float((uint8_t)((uint32_t)kv[r] >> (8 * e)));
+                    }
+#pragma unroll
+                for (int r = 0; r < 4; ++r)
+#pragma unroll
+                    for (int c = 0; c < 4; ++c)
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) s_lqf[r][c] = fmaf(qf[r][e], kf[c][e], s_lqf[r][c]);
+            } else {
+#pragma unroll
+                for (int r = 0; r < 4; ++r)
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) s_lq[r][c] = __dp4a(qv[r], kv[c], s_lq[r][c]);
+            }
         }
 
         // class selection, masks, online softmax
@@ -165,7 +187,8 @@ attn_simt_kernel(hyq_attn_args a, float alpha, const uint32_t* __restrict__ vl_b
                 const bool valid = (j <= i) && (j < L) && (i < L);       // (i < L <=> the row exists)
                 const bool is_vl = valid && ((vl_row[j >> 5] >> (j & 31)) & 1u);
                 fp[r][c] = is_vl || (a.window_mode == HYQ_WINDOW_FIXED_TAIL ? (j >= L - a.window) : (i - j < a.window));
-                const float lq = (float)s_lq[r][c] * sm.q_scale[ty * 4 + r] * sm.k_scale[tx * 4 + c] * alpha;
+                const float code_dot = (QK_FMT == HYQ_FMT_FP8_E4M3) ? s_lqf[r][c] : (float)s_lq[r][c];
+                const float lq = code_dot * sm.q_scale[ty * 4 + r] * sm.k_scale[tx * 4 + c] * alpha;
                 s[r][c] = valid ? (fp[r][c] ? s_fp[r][c] * alpha : lq) : -INFINITY;
                 mx = fmaxf(mx, s[r][c]);
             }
@@ -241,6 +264,7 @@ int launch_attn_simt(const hyq_attn_args& a, float alpha, cudaStream_t st) {
     };
     if (a.q_format == HYQ_FMT_INT8 && a.v_format == HYQ_FMT_INT8) return run(attn_simt_kernel<HYQ_FMT_INT8, HYQ_FMT_INT8>);
     if (a.q_format == HYQ_FMT_INT4 && a.v_format == HYQ_FMT_FP8_E4M3) return run(attn_simt_kernel<HYQ_FMT_INT4, HYQ_FMT_FP8_E4M3>);
+    if (a.q_format == HYQ_FMT_FP8_E4M3 && a.v_format == HYQ_FMT_FP8_E4M3) return run(attn_simt_kernel<HYQ_FMT_FP8_E4M3, HYQ_FMT_FP8_E4M3>);
     return HYQ_ERR_UNSUPPORTED;
 }
 

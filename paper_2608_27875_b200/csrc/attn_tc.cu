@@ -747,8 +747,10 @@ int launch_attn_tc(const hyq_attn_args& a, float alpha, cudaStream_t st) {
     p.out = a.out; p.lse = a.lse; p.status = a.status_word;
 
     const bool blk = Lq < L || p.fixed_tail;      // the general instantiation (the other one is the whole prefill)
-    auto kern = int4 ? (blk ? attn_tc_kernel<true, true> : attn_tc_kernel<true, false>)
-                     : (blk ? attn_tc_kernel<false, true> : attn_tc_kernel<false, false>);
+    // e4m3 bytes on the low-bit side: FP8 codes as they are, or INT4 codes widened by the pre-pass
+    const bool lowbit_fp8 = a.q_format != HYQ_FMT_INT8;
+    auto kern = lowbit_fp8 ? (blk ? attn_tc_kernel<true, true> : attn_tc_kernel<true, false>)
+                           : (blk ? attn_tc_kernel<false, true> : attn_tc_kernel<false, false>);
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM_BYTES) != cudaSuccess)
         return HYQ_ERR_CUDA;
     const dim3 grid(((int)Lq + QT * BM - 1) / (QT * BM), a.Hq, a.B);

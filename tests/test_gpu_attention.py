@@ -12,6 +12,7 @@ from paper_2608_27875_b200 import api, workloads as wl
 pytestmark = pytest.mark.gpu
 INT8 = (wl.FMT_INT8,) * 3
 INT4FP8 = (wl.FMT_INT4, wl.FMT_INT4, wl.FMT_FP8_E4M3)
+FP8ALL = (wl.FMT_FP8_E4M3,) * 3
 IMPLS = [pytest.param(api.IMPL_SIMT, id="simt"), pytest.param(api.IMPL_TCGEN05, id="umma")]
 
 
@@ -40,7 +41,7 @@ def _check(Q, K, V, fmts, idx, window, impl, rows=None):
 
 
 @pytest.mark.parametrize("impl", IMPLS)
-@pytest.mark.parametrize("fmts", [INT8, INT4FP8])
+@pytest.mark.parametrize("fmts", [INT8, INT4FP8, FP8ALL])
 @pytest.mark.parametrize("B,Hq,Hkv,L,W,k", [
     (1, 2, 2, 512, 128, 16),      # several tiles
     (2, 4, 2, 333, 40, 9),        # ragged tail, window not a tile multiple
@@ -259,7 +260,7 @@ def test_random_shapes_tensor_core_matches_cuda_core_and_repeats_bit_for_bit(see
     L = int(rng.integers(2000, 6000)) if long_rows else int(rng.integers(1, 1400))
     W = int(rng.choice([0, 1, 17, 64, 100, 128, 300, 1024]))
     k = int(rng.integers(0, max(1, min(L - W, 64)))) if L - W > 0 else 0
-    fmts = INT8 if seed % 2 == 0 else INT4FP8
+    fmts = (INT8, INT4FP8, FP8ALL)[seed % 3]
     u = torch.randn(128, generator=g)
     u = u / u.norm()
     slope = float(rng.choice([0.0, 0.0, 20.0, -20.0, 60.0]))
@@ -287,7 +288,7 @@ def test_random_query_blocks_and_window_forms_both_kernels_agree(seed):
     W = int(rng.choice([0, 1, 50, 64, 200, 700]))
     k = int(rng.integers(0, max(1, min(L - W, 48)))) if L - W > 0 else 0
     mode = int(rng.integers(0, 2))
-    fmts = INT8 if seed % 2 == 0 else INT4FP8
+    fmts = (INT8, INT4FP8, FP8ALL)[seed % 3]
     Hkv = int(rng.integers(1, 3))
     Hq = Hkv * int(rng.choice([1, 2]))
     Q = torch.randn(1, Hq, Lq, 128, generator=g).to(torch.bfloat16).cuda()

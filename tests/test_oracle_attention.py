@@ -108,6 +108,7 @@ def _brute(q, k, v, qh, kh, vh, idx, W, alpha):
 
 
 @pytest.mark.parametrize("fmts,W,kk", [((INT8, INT8, INT8), 5, 4), ((INT4, INT4, FP8), 8, 3),
+                                       ((FP8, FP8, FP8), 6, 5),
                                        ((INT8, INT8, INT8), 0, 6), ((INT8, INT8, INT8), 1, 0)])
 def test_against_brute_force(fmts, W, kk):
     bt = 8
