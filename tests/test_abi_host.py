@@ -96,8 +96,11 @@ def test_attention_argument_checks(lib):
     assert call(_args(Hkv=3)) == 1
     assert call(_args(D=64)) == 2
     assert call(_args(block_tokens=32)) == 2
-    assert call(_args(q_format=1, k_format=1, v_format=1)) == 2       # FP8 Q/K not built
+    assert call(_args(q_format=1, k_format=0, v_format=1)) == 2       # Q and K formats must match
     assert call(_args(q_format=2, k_format=2, v_format=0)) == 2       # INT4 with INT8 V not built
+    assert call(_args(Lq=-1)) == 1
+    assert call(_args(Lq=10 ** 6)) == 1                               # query block longer than the keys
+    assert call(_args(window_mode=2)) == 1
     assert call(_args(out=None)) == 1
     assert call(_args(vl_idx=None)) == 1                              # k > 0 needs indices
     assert call(_args(q=0x10008)) == 4
