@@ -86,7 +86,7 @@ __device__ __forceinline__ uint32_t mbar_test_wait2(uint64_t* bar0, uint32_t par
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* m) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(m)) : "memory");
 }
-// 3-D tiled load global -> shared, completion on an mbarrier (no multicast)
+// 3-D tiled load global -> shared of this CTA only, completion on an mbarrier
 __device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* m, uint64_t* bar, int x, int y, int z) {
     asm volatile(
         "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
