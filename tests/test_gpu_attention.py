@@ -138,6 +138,26 @@ def test_full_size_workloads_in_the_benchmark_launch_configuration(name, kv_head
         assert max_abs <= MAX_ABS_TOL and mean_rel <= MEAN_REL_TOL, (name, kvh, max_abs, mean_rel)
 
 
+@pytest.mark.parametrize("name,Lq,mode", [("c1", 2048, 0), ("c2", 4096, 0), ("c2", 4096, 1)])
+def test_benchmark_size_query_block_on_sampled_rows(name, Lq, mode):
+    """The configuration `bench.py --lq` times: the last Lq rows of a benchmark-size context (one KV head's
+    query heads), both window forms, checked against the oracle on sampled rows of the block."""
+    ensure_built()
+    w = wl.CONFIGS[name]
+    Q, K, V = wl.make_inputs(w, heads=[w.Hkv - 1])
+    Qb = Q[:, :, w.L - Lq:].contiguous()
+    idx = oracle.select_vertical(wl.bits(Qb), wl.bits(K), w.window, w.k)
+    rows = np.unique(np.concatenate([[0, 1, 63, 64, 255, 256, Lq - 2, Lq - 1],
+                                     np.random.default_rng(7).integers(0, Lq, 12)])).astype(np.int32)
+    qz = oracle_quant_all(Qb, K, V, w.fmts)
+    got = gpu_attention(Qb, K, V, qz, w.fmts, idx, w.window, api.IMPL_TCGEN05, window_mode=mode).numpy()[:, :, rows]
+    (qc, qs), (kc, ks), (vc, vs) = qz
+    ref = oracle.attention_rows(wl.bits(Qb), wl.bits(K), wl.bits(V), qc, kc, vc, qs, ks, vs, w.fmts, idx, w.window,
+                                rows, fixed_window=bool(mode))
+    max_abs, mean_rel = errors(got, ref)
+    assert max_abs <= MAX_ABS_TOL and mean_rel <= MEAN_REL_TOL, (name, Lq, mode, max_abs, mean_rel)
+
+
 def test_tensor_core_and_cuda_core_kernels_agree_on_every_output_of_config1():
     """Every row of every head at a benchmark size: two independent kernels, both within tolerance of the
     definition on the sampled rows, must agree with each other everywhere."""
