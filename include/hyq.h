@@ -149,6 +149,9 @@ int hyq_quantize_blocks(const void* x, int B, int H, int L, int D, int block_tok
  *   q_scales ceil(Lq/64) entries per head (quantization blocks counted from the first row of the block, as
  *   hyq_quantize_blocks writes them for a [B,Hq,Lq,D] tensor) and lse Lq entries; K, V and vl_idx are those
  *   of the whole context.  Lq = 0 or Lq = L is the whole prefill.  Lq > L -> HYQ_ERR_INVALID_ARG.
+ *   (For short blocks the tensor-core path splits the keys over several CTAs per query tile and merges the
+ *   partial results; the workspace query accounts for their buffers.  Results do not depend on the split up to
+ *   fp32 rounding.)
  *
  *   Window form: HYQ_WINDOW_SLIDING - key j is a window key of the row at position i iff i - j < window (every
  *   row has its own last `window` positions; the form the whole prefill needs).  HYQ_WINDOW_FIXED_TAIL -

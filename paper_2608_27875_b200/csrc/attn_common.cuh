@@ -16,9 +16,17 @@ struct TcWorkspace {
     size_t vvl;         // fp16 [B*Hq][k][D]            gathered vertical-line V rows
     size_t q8;          // u8   [B*Hq][Lq][D]           INT4 only: Q codes as e4m3 bytes
     size_t k8;          // u8   [B*Hkv][L][D]           INT4 only: K codes as e4m3 bytes
+    size_t part_o;      // f32  [splits][B*Hq][Lq][D]   split keys only: partial accumulators ...
+    size_t part_ml;     // f32  [splits][B*Hq][Lq][2]   ... and (reference maximum, row sum) per row
     size_t total;
     int mask_words;
+    int splits;         // CTAs per pair of query tiles (1: the keys are not split)
 };
+
+// Short query blocks leave most SMs without a CTA (one CTA per 256 query rows and head): the walk over the keys is
+// then split over several CTAs.  Returns how many (1..8), so that the grid reaches about two CTAs per SM while
+// every slice keeps a useful number of key tiles.
+int tc_key_splits(const hyq_attn_args& a);
 
 TcWorkspace tc_workspace_layout(const hyq_attn_args& a);
 int launch_tc_prepass(const hyq_attn_args& a, const TcWorkspace& w, cudaStream_t st);

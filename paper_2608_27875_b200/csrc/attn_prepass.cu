@@ -117,6 +117,19 @@ int launch_vl_bitmask(const int32_t* idx, long n_heads, int k, int L, int mask_w
 }
 
 // ---------------------------------------------------------------------------------------------
+int tc_key_splits(const hyq_attn_args& a) {
+    const int Lq = query_rows(a);
+    if (Lq >= a.L) return 1;                                     // the whole prefill fills the GPU by itself
+    const long ctas = (long)((Lq + 255) / 256) * a.Hq * a.B;
+    const long target = 2 * 148;                                 // about two CTAs per SM
+    if (ctas >= target / 2) return 1;
+    const int key_tiles = (a.L + 63) / 64;                       // upper bound of a CTA's walk
+    long s = (target + ctas - 1) / ctas;
+    s = s < 8 ? s : 8;
+    while (s > 1 && key_tiles / s < 16) --s;                     // at least 16 key tiles per slice
+    return (int)s;
+}
+
 TcWorkspace tc_workspace_layout(const hyq_attn_args& a) {
     TcWorkspace w{};
     size_t off = 0;
@@ -131,6 +144,10 @@ TcWorkspace tc_workspace_layout(const hyq_attn_args& a) {
     const bool int4 = a.q_format == HYQ_FMT_INT4;
     w.q8 = int4 ? take(q_elems) : 0;
     w.k8 = int4 ? take(kv_elems) : 0;
+    w.splits = tc_key_splits(a);
+    const size_t rows = (size_t)a.B * a.Hq * query_rows(a);
+    w.part_o = w.splits > 1 ? take((size_t)w.splits * rows * HYQ_D * 4) : 0;
+    w.part_ml = w.splits > 1 ? take((size_t)w.splits * rows * 2 * 4) : 0;
     w.total = off;
     return w;
 }

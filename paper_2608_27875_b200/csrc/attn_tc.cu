@@ -86,6 +86,9 @@ struct TcParams {
     int B, Hq, Hkv, L, window, k, nb, mask_words;
     int Lq, nbq;                 // query rows (end-aligned with the L keys: row i sits at position L - Lq + i), their blocks
     int fixed_tail;              // window form: the last `window` keys for every row instead of each row's own
+    int splits;                  // CTAs per pair of query tiles, each on a slice of the walk (short query blocks)
+    float* part_o;               // splits > 1: unnormalised partial outputs [splits][B*Hq][Lq][D] ...
+    float* part_ml;              // ... and (reference maximum in log2 units, row sum) [splits][B*Hq][Lq][2]
     int out_fp32;
     float scale_log2;            // softmax_scale * log2(e)
     const float* q_scales;
@@ -127,6 +130,7 @@ __device__ __forceinline__ int count_le(const int32_t* __restrict__ idx, int k, 
 // the tile walk of one CTA: union of both query tiles' lists
 struct Walk {
     int nA, nB, tC0, nC, T;
+    int t0, t1;                 // the positions [t0, t1) this CTA works on (all of [0, T) unless the keys are split)
 };
 
 // own tile ranges of one query tile inside the CTA's walk: [0, a_end) low-bit, [b_beg, b_end) vertical, [c_beg, c_end) window
@@ -134,6 +138,10 @@ struct OwnTiles {
     int a_end, b_beg, b_end, c_beg, c_end;
     __device__ __forceinline__ bool has(int t) const { return t < a_end || (t >= b_beg && t < b_end) || (t >= c_beg && t < c_end); }
 };
+// number of own tiles at walk positions below t
+__device__ __forceinline__ int own_before(const OwnTiles& o, int t) {
+    return min(t, o.a_end) + min(max(t - o.b_beg, 0), o.b_end - o.b_beg) + min(max(t - o.c_beg, 0), o.c_end - o.c_beg);
+}
 __device__ __forceinline__ OwnTiles own_tiles(const QSched& s, const Walk& w) {
     OwnTiles o;
     o.a_end = s.live ? s.nA : 0;
@@ -162,12 +170,13 @@ __device__ __forceinline__ bool mma_issuer(int q, const QSched& sq, const Walk& 
     const uint64_t dv0 = make_smem_desc(smem_u32(smem + SV_OFF), G::STAGE_BYTES / 2, 1024);
     const uint32_t ts0 = tmem + tm_s(q), to = tmem + tm_o(q);
     const OwnTiles own = own_tiles(sq, w);
-    const int nA = w.nA, T = w.T;
+    const int nA = w.nA;
     if (!mbar_wait(&bars.q_full, 0, WAIT_LIMIT)) return false;
 
     // Q.K^T cursor
-    int tq = 0, kst = 0;
+    int tq = w.t0, kst = 0;
     uint32_t kpar = 0, n_qk = 0;
+    const int T1 = w.t1;
     // (k_ready: the stage of position tq is already known to have landed)
     auto qk = [&](bool k_ready) -> bool {
         if (!k_ready && !mbar_wait(&bars.kv_full[kst], kpar, WAIT_LIMIT)) return false;
@@ -200,9 +209,9 @@ __device__ __forceinline__ bool mma_issuer(int q, const QSched& sq, const Walk& 
     // P.V cursor
     int vst = 0;
     uint32_t n_pv = 0;
-    for (int t = 0; t < NBUF && t < T; ++t)
+    for (int t = 0; t < NBUF && tq < T1; ++t)
         if (!qk(false)) return false;
-    for (int t = 0; t < T; ++t) {
+    for (int t = w.t0; t < T1; ++t) {
         // (the V tile of position t came in on the same barrier as its K tile, which Q.K^T waited for)
         bool k_ready = false;
         if (own.has(t)) {
@@ -210,7 +219,7 @@ __device__ __forceinline__ bool mma_issuer(int q, const QSched& sq, const Walk& 
             HYQ_TR(4 + q, (int)n_pv, 4);
             // P of this tile, and in the same round trip the ring stage of the Q.K^T that follows
             const uint32_t done = mbar_test_wait2(&bars.p_full[q][buf], (n_pv / NBUF) & 1u, &bars.kv_full[kst], kpar);
-            k_ready = (done & 2u) != 0u && tq < T;
+            k_ready = (done & 2u) != 0u && tq < T1;
             if (!(done & 1u) && !mbar_wait(&bars.p_full[q][buf], (n_pv / NBUF) & 1u, WAIT_LIMIT)) return false;
             HYQ_TR(4 + q, (int)n_pv, 5);
             tc_fence_after();
@@ -227,7 +236,7 @@ __device__ __forceinline__ bool mma_issuer(int q, const QSched& sq, const Walk& 
             mbar_arrive(&bars.kv_free[vst]);        // nothing of this query tile reads the stage
         }
         if (++vst == NST) vst = 0;
-        if (tq < T && !qk(k_ready)) return false;
+        if (tq < T1 && !qk(k_ready)) return false;
         if ((t & 15) == 15 && *abort_flag) return true;
     }
     return true;
@@ -254,8 +263,8 @@ __device__ __forceinline__ bool tma_producer(const TcMaps& maps, const QSched& q
         tma_load_3d(smem + SQ_OFF + q * Q_TILE_BYTES + Q_TILE_BYTES / 2, &maps.q, &bars.q_full, 64, qi0[q], qhead);
         if (w.nA > 0) tma_load_3d(smem + SQC_OFF + q * QC_TILE_BYTES, &maps.qc, &bars.q_full, 0, qi0[q], qhead);
     }
-    for (int t = 0; t < w.T && !*abort_flag; ++t) {
-        const int st = t % NST, use = t / NST;
+    for (int t = w.t0; t < w.t1 && !*abort_flag; ++t) {
+        const int st = (t - w.t0) % NST, use = (t - w.t0) / NST;
         unsigned char* sk = smem + SK_OFF + st * G::STAGE_BYTES;
         unsigned char* sv = smem + SV_OFF + st * G::STAGE_BYTES;
         const bool lowbit = t < w.nA, vl = !lowbit && t < w.nA + w.nB;
@@ -371,7 +380,9 @@ __device__ __forceinline__ void mask_cols32(uint32_t (&raw)[32], int c0, int lo_
 // LOWBIT_FP8: the low-bit codes are e4m3 bytes (kind::f8f6f4), else int8 (kind::i8).  QUERY_BLOCK: the query rows
 // are the last Lq < L positions (a compile-time zero offset keeps one register out of the whole-prefill loop:
 // 2.6 % on the benchmark workload).
-template <bool LOWBIT_FP8, bool QUERY_BLOCK>
+// SPLIT (short query blocks only): several CTAs share a pair of query tiles, each on a contiguous slice of the
+// walk; they leave unnormalised partial results that attn_merge_kernel combines by their reference maxima.
+template <bool LOWBIT_FP8, bool QUERY_BLOCK, bool SPLIT = false>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
     constexpr int TBN = 64, BN = 64;
@@ -384,7 +395,9 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
     __shared__ int abort_s, cnt_b_s[QT];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int pt = gridDim.x - 1 - blockIdx.x;               // pair of query tiles; longest rows first
+    const int pt_lin = gridDim.x - 1 - blockIdx.x;           // pair of query tiles (and slice); longest rows first
+    const int pt = SPLIT ? pt_lin / p.splits : pt_lin;
+    const int split = SPLIT ? pt_lin % p.splits : 0;
     const int h = blockIdx.y, b = blockIdx.z;
     const int L = p.Lq, W = p.window, g = p.Hq / p.Hkv;     // L: rows of the query block
     const int off = QUERY_BLOCK ? p.L - p.Lq : 0;           // position of query row 0 among the keys
@@ -445,6 +458,8 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
     w.tC0 = qs0.tC0;
     w.nC = (W > 0) ? max(qs0.tC1, qs1.tC1) - w.tC0 + 1 : 0;
     w.T = w.nA + w.nB + w.nC;
+    w.t0 = SPLIT ? (int)((long)w.T * split / p.splits) : 0;
+    w.t1 = SPLIT ? (int)((long)w.T * (split + 1) / p.splits) : w.T;
 
     volatile int* abort_flag = &abort_s;
     auto fail = [&]() {
@@ -467,8 +482,16 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
         // named barrier of the two warps that share this warp's 32 query rows (one per query tile and lane quarter)
         const int bar_id = 1 + q * 4 + (warp & 3);
         const OwnTiles own = own_tiles(sq, w);
-        const int n_total = own.a_end + (own.b_end - own.b_beg) + (own.c_end - own.c_beg);
-        if (sq.live && n_total > 0) {
+        // own tiles of this CTA: numbers [n0, n_total) in the query tile's own list (all of it unless the keys are split)
+        const int n0 = SPLIT ? own_before(own, w.t0) : 0;
+        const int n_total = SPLIT ? own_before(own, w.t1) : own.a_end + (own.b_end - own.b_beg) + (own.c_end - own.c_beg);
+        if (SPLIT && sq.live && n_total <= n0) {
+            // nothing of this query tile lies in the slice: an empty partial result
+            const int i = sq.i0 + (warp & 3) * 32 + lane;
+            if ((((warp - 4) >> 2) & 1) == 0 && i < L)
+                reinterpret_cast<float2*>(p.part_ml)[((long)split * gridDim.y * gridDim.z + qhead) * L + i] = make_float2(-INFINITY, 0.0f);
+        }
+        if (sq.live && n_total > n0) {
             const int r = (warp & 3) * 32 + lane;               // query row inside the tile = TMEM lane
             const int i = sq.i0 + r;                           // row of the query block ...
             const int ia = i + off;                             // ... and its position among the keys
@@ -501,7 +524,7 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                 nks = __ldg(ks_ptr + n);
                 nvl = __ldg(vl_ptr + 2 * n);
             };
-            prefetch_tile(0);
+            prefetch_tile(n0);
             const float qs2 = q_scale * p.scale_log2;
 
             // one tile of the online softmax for this thread's 32 columns.  Returns false when the query tile's
@@ -509,12 +532,13 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
             auto do_tile = [&](auto range_tag, int n, float cs, uint32_t vl, bool int_scores, int lo_eff, unsigned span) -> bool {
                 constexpr bool NEED_RANGE = decltype(range_tag)::value;
                 const uint32_t knock = int_scores ? KNOCKOUT_S32 : KNOCKOUT_F32;
-                const int buf = n & 1;
+                const int nl = n - n0;                          // tile number within this CTA's slice
+                const int buf = nl & 1;
                 const uint32_t ts = ts0 + buf * BN;
                 uint32_t raw[32];
                 float mt = -INFINITY;
                 HYQ_TR(q * 2 + hsel, n, 0);
-                if (!dead && !__all_sync(0xffffffffu, mbar_wait(&bars.s_full[q][buf], (uint32_t)(n >> 1) & 1u, WAIT_LIMIT))) {
+                if (!dead && !__all_sync(0xffffffffu, mbar_wait(&bars.s_full[q][buf], (uint32_t)(nl >> 1) & 1u, WAIT_LIMIT))) {
                     dead = true;
                 }
                 __syncwarp();
@@ -566,11 +590,11 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                     const float m_new = fmaxf(mt, mo);
                     const bool raise = m_new > m_used + RAISE_THRESHOLD;     // same verdict in both threads of the row
                     const float alpha = raise ? ex2f(m_used - m_new) : 1.0f; // m_used = -inf -> 0
-                    if (n > 0 && __any_sync(0xffffffffu, raise)) {
+                    if (nl > 0 && __any_sync(0xffffffffu, raise)) {
                         // P.V of tile n-1 must have landed before O is rescaled.  P.V number m signals barrier m & 1;
                         // the one before the previous is complete (the scores just read were issued after it), so
                         // the parity wait cannot alias.
-                        if (!__all_sync(0xffffffffu, mbar_wait(&bars.o_done[q][(n - 1) & 1], (uint32_t)((n - 1) >> 1) & 1u, WAIT_LIMIT))) {
+                        if (!__all_sync(0xffffffffu, mbar_wait(&bars.o_done[q][(nl - 1) & 1], (uint32_t)((nl - 1) >> 1) & 1u, WAIT_LIMIT))) {
                             dead = true;
                         } else {
                             tc_fence_after();
@@ -611,8 +635,8 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
 
             // ---- low-bit tiles that lie wholly below every row's window: no range mask, no bounds to compute
             const int n_plain = ragged ? 0 : min(own.a_end, max(0, (qhi(sq.i0 + off) + 1) / BN));
-            int n = 0;
-            for (; n < n_plain; ++n) {
+            int n = n0;
+            for (; n < min(n_plain, n_total); ++n) {
                 HYQ_TR(q * 2 + hsel, n, 2);
                 // a zero scale (all-zero tile) still has to let -inf pass through the multiply
                 const float cs = fmaxf(qs2 * nks, 1e-37f);
@@ -651,7 +675,7 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
 
             // ---- epilogue: the last P.V (MMAs complete in order), sum of the two halves' row sums, O / l
             bool ok = !aborted && !dead;
-            if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars.o_done[q][(n_total - 1) & 1], (uint32_t)((n_total - 1) >> 1) & 1u, WAIT_LIMIT));
+            if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars.o_done[q][(n_total - n0 - 1) & 1], (uint32_t)((n_total - n0 - 1) >> 1) & 1u, WAIT_LIMIT));
             if (!aborted) {                                     // uniform over the query tile's softmax warps
                 tc_fence_after();
                 tmem_st1(ts0 + col0, __float_as_uint(l_h));     // column col0 of S buffer 0 (all MMAs are done)
@@ -663,7 +687,25 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                 tmem_wait_ld();
                 const float l_run = l_h + l_o;
                 const float inv = (l_run > 0.0f) ? 1.0f / l_run : 0.0f;
-                if (ok) {
+                if (SPLIT) {
+                    // partial result of this slice: O as accumulated (relative to m_used), the pair (m_used, l)
+                    const long prow = ((long)split * gridDim.y * gridDim.z + qhead) * L + i;
+                    if (ok) {
+#pragma unroll
+                        for (int c = 0; c < 2; ++c) {
+                            uint32_t o[32];
+                            const int ch = hsel * 64 + c * 32;
+                            tmem_ld32(to + ch, o);
+                            tmem_wait_ld();
+                            if (row_live) {
+                                uint4* dst = reinterpret_cast<uint4*>(p.part_o + prow * HYQ_D + ch);
+#pragma unroll
+                                for (int e = 0; e < 8; ++e) dst[e] = make_uint4(o[4 * e], o[4 * e + 1], o[4 * e + 2], o[4 * e + 3]);
+                            }
+                        }
+                        if (row_live && hsel == 0) reinterpret_cast<float2*>(p.part_ml)[prow] = make_float2(m_used, l_run);
+                    }
+                } else if (ok) {
 #pragma unroll
                     for (int c = 0; c < 2; ++c) {              // this half writes channels [64 hsel, 64 hsel + 64)
                         uint32_t o[32];
@@ -708,6 +750,40 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
     }
 }
 
+// Combines the partial results of the key slices of a short query block: every slice s left, per row, its
+// accumulator O_s relative to its own reference maximum m_s (log2 units) and its row sum l_s; the row's result is
+// sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s with M = max_s m_s.  One thread per row and four channels.
+__global__ void __launch_bounds__(256)
+attn_merge_kernel(const float* __restrict__ part_o, const float* __restrict__ part_ml, int splits, long n_rows, void* out,
+                  int out_fp32, float* lse) {
+    const long e = (long)blockIdx.x * blockDim.x + threadIdx.x;
+    const long row = e / (HYQ_D / 4);
+    const int c4 = (int)(e % (HYQ_D / 4));
+    if (row >= n_rows) return;
+    float m = -INFINITY;
+    for (int s = 0; s < splits; ++s) m = fmaxf(m, __ldg(part_ml + ((long)s * n_rows + row) * 2));
+    float4 acc = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+    float l = 0.0f;
+    for (int s = 0; s < splits; ++s) {
+        const float2 ml = __ldg(reinterpret_cast<const float2*>(part_ml) + (long)s * n_rows + row);
+        if (!(ml.y > 0.0f)) continue;                           // empty slice: its accumulator was not written
+        const float wgt = exp2f(ml.x - m);
+        const float4 o = __ldg(reinterpret_cast<const float4*>(part_o + ((long)s * n_rows + row) * HYQ_D) + c4);
+        acc.x = fmaf(wgt, o.x, acc.x); acc.y = fmaf(wgt, o.y, acc.y); acc.z = fmaf(wgt, o.z, acc.z); acc.w = fmaf(wgt, o.w, acc.w);
+        l = fmaf(wgt, ml.y, l);
+    }
+    const float inv = (l > 0.0f) ? 1.0f / l : 0.0f;
+    acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
+    if (out_fp32) {
+        reinterpret_cast<float4*>(static_cast<float*>(out) + row * HYQ_D)[c4] = acc;
+    } else {
+        const __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
+        reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(out) + row * HYQ_D)[c4] =
+            make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
+    }
+    if (lse && c4 == 0) lse[row] = (m + log2f(l)) * 0.6931471805599453f;
+}
+
 // ---------------------------------------------------------------------------------------------
 size_t attn_tc_workspace_bytes(const hyq_attn_args& a) { return tc_workspace_layout(a).total; }
 
@@ -738,6 +814,9 @@ int launch_attn_tc(const hyq_attn_args& a, float alpha, cudaStream_t st) {
     p.nb = (a.L + HYQ_BLOCK_TOKENS - 1) / HYQ_BLOCK_TOKENS;
     p.Lq = (int)Lq;
     p.fixed_tail = a.window_mode == HYQ_WINDOW_FIXED_TAIL;
+    p.splits = w.splits;
+    p.part_o = reinterpret_cast<float*>(base + w.part_o);
+    p.part_ml = reinterpret_cast<float*>(base + w.part_ml);
     p.nbq = ((int)Lq + HYQ_BLOCK_TOKENS - 1) / HYQ_BLOCK_TOKENS;
     p.mask_words = w.mask_words;
     p.out_fp32 = a.out_dtype == 1;
@@ -749,14 +828,21 @@ int launch_attn_tc(const hyq_attn_args& a, float alpha, cudaStream_t st) {
     const bool blk = Lq < L || p.fixed_tail;      // the general instantiation (the other one is the whole prefill)
     // e4m3 bytes on the low-bit side: FP8 codes as they are, or INT4 codes widened by the pre-pass
     const bool lowbit_fp8 = a.q_format != HYQ_FMT_INT8;
-    auto kern = lowbit_fp8 ? (blk ? attn_tc_kernel<true, true> : attn_tc_kernel<true, false>)
+    const bool split = w.splits > 1;               // (only ever chosen for short query blocks)
+    auto kern = split ? (lowbit_fp8 ? attn_tc_kernel<true, true, true> : attn_tc_kernel<false, true, true>)
+              : lowbit_fp8 ? (blk ? attn_tc_kernel<true, true> : attn_tc_kernel<true, false>)
                            : (blk ? attn_tc_kernel<false, true> : attn_tc_kernel<false, false>);
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM_BYTES) != cudaSuccess)
         return HYQ_ERR_CUDA;
-    const dim3 grid(((int)Lq + QT * BM - 1) / (QT * BM), a.Hq, a.B);
+    const dim3 grid((((int)Lq + QT * BM - 1) / (QT * BM)) * w.splits, a.Hq, a.B);
     if (a.ev_kernel_start && cudaEventRecord(static_cast<cudaEvent_t>(a.ev_kernel_start), st) != cudaSuccess) return HYQ_ERR_CUDA;
     kern<<<grid, TC_THREADS, TC_SMEM_BYTES, st>>>(maps, p);
     if (launch_status() != HYQ_OK) return HYQ_ERR_CUDA;
+    if (split) {
+        const long n_rows = (long)a.B * a.Hq * (long)Lq, n_thr = n_rows * (HYQ_D / 4);
+        attn_merge_kernel<<<(unsigned)((n_thr + 255) / 256), 256, 0, st>>>(p.part_o, p.part_ml, w.splits, n_rows, a.out, p.out_fp32, a.lse);
+        if (launch_status() != HYQ_OK) return HYQ_ERR_CUDA;
+    }
     if (a.ev_kernel_stop && cudaEventRecord(static_cast<cudaEvent_t>(a.ev_kernel_stop), st) != cudaSuccess) return HYQ_ERR_CUDA;
     return HYQ_OK;
 }

@@ -158,6 +158,41 @@ def test_benchmark_size_query_block_on_sampled_rows(name, Lq, mode):
     assert max_abs <= MAX_ABS_TOL and mean_rel <= MEAN_REL_TOL, (name, Lq, mode, max_abs, mean_rel)
 
 
+@pytest.mark.parametrize("fmts", [INT8, INT4FP8, FP8ALL])
+@pytest.mark.parametrize("Lq,L,W,k,mode", [(1, 4096, 256, 40, 0), (100, 5000, 128, 64, 0), (256, 8192, 512, 80, 1),
+                                           (300, 6000, 0, 30, 0), (512, 16384, 1024, 100, 0)])
+def test_short_query_blocks_with_the_keys_split_over_ctas(fmts, Lq, L, W, k, mode):
+    """Short query blocks against long contexts: the tensor-core path splits the keys over several CTAs per
+    query tile and merges their partial results.  Outputs and the log-sum-exp must agree with the CUDA-core
+    kernel (which never splits) everywhere, and with the oracle on sampled rows; the bf16 output must be the
+    rounding of the fp32 one."""
+    ensure_built()
+    g = torch.Generator().manual_seed(Lq + L)
+    Q = torch.randn(1, 2, Lq, 128, generator=g).to(torch.bfloat16).cuda()
+    K = torch.randn(1, 1, L, 128, generator=g).to(torch.bfloat16).cuda()
+    V = torch.randn(1, 1, L, 128, generator=g).to(torch.bfloat16).cuda()
+    idx = torch.from_numpy(_rand_idx(1, 2, L - W, k, seed=L)).cuda()
+    (qc, qs), (kc, ks), (vc, vs) = [api.hyq_quantize_blocks(t, f) for t, f in zip((Q, K, V), fmts)]
+    lse = [torch.empty(1, 2, Lq, dtype=torch.float32, device="cuda") for _ in range(2)]
+    tc, simt = [api.hyq_hybrid_attention_prefill(Q, K, V, qc, kc, vc, qs, ks, vs, fmts, idx, W, impl=impl, lse=l_,
+                                                 window_mode=mode)
+                for impl, l_ in zip((api.IMPL_TCGEN05, api.IMPL_SIMT), lse)]
+    tc16 = api.hyq_hybrid_attention_prefill(Q, K, V, qc, kc, vc, qs, ks, vs, fmts, idx, W, impl=api.IMPL_TCGEN05,
+                                            out_dtype=torch.bfloat16, window_mode=mode)
+    torch.cuda.synchronize()
+    assert torch.isfinite(tc).all()
+    diff = (tc - simt).abs()
+    assert float(diff.max()) <= MAX_ABS_TOL and float(diff.sum() / simt.abs().sum()) <= MEAN_REL_TOL
+    assert float((lse[0] - lse[1]).abs().max()) <= 2e-3
+    assert torch.equal(tc16, tc.to(torch.bfloat16))
+    rows = np.unique(np.concatenate([[0, Lq - 1], np.random.default_rng(3).integers(0, Lq, 4)])).astype(np.int32)
+    t = lambda x: x.cpu().numpy()   # noqa: E731
+    ref = oracle.attention_rows(wl.bits(Q.cpu()), wl.bits(K.cpu()), wl.bits(V.cpu()), t(qc), t(kc), t(vc), t(qs), t(ks), t(vs),
+                                fmts, t(idx), W, rows, fixed_window=bool(mode))
+    max_abs, mean_rel = errors(t(tc)[:, :, rows], ref)
+    assert max_abs <= MAX_ABS_TOL and mean_rel <= MEAN_REL_TOL, (max_abs, mean_rel)
+
+
 def test_tensor_core_and_cuda_core_kernels_agree_on_every_output_of_config1():
     """Every row of every head at a benchmark size: two independent kernels, both within tolerance of the
     definition on the sampled rows, must agree with each other everywhere."""
