@@ -40,7 +40,7 @@ NOMINAL = {"bf16_tflops": 2250.0, "lowbit_tflops": 4500.0, "hbm_gbs": 8000.0}
 FALLBACK = {"bf16_tflops": 1590.0, "hbm_gbs": 6650.0}
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu
 # capture summarised under profiles/ (bytes per launch of the benchmark workload; None = no capture yet)
-NCU_TRAFFIC_BYTES = {"c2": 693101824 + 516921600}
+NCU_TRAFFIC_BYTES = {"c2": 695749888 + 515654400}
 
 
 def measured_peaks():
