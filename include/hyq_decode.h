@@ -1,0 +1,115 @@
+/*
+ * hyq_decode.h - C ABI of the decode side of the B200 (sm_100a) HyQuant library:
+ *
+ *   hyq_freeze                    Algorithm 4 (prefill -> decode hybrid KV-cache organisation)
+ *   hyq_hybrid_attention_decode   Algorithm 3 / Section 3.3 (one new token against the hybrid cache,
+ *                                 low-bit rows dequantized inside the attention kernel)
+ *
+ * The common rules of hyq.h hold (device pointers, contiguous row-major arrays, caller-owned buffers,
+ * calls enqueue on `stream` and return, arguments checked on the host before anything is launched,
+ * D = 128, Hq % Hkv == 0 with g = Hq / Hkv <= 8 query heads per KV head).
+ *
+ * The hybrid cache of one layer (Algorithm 4's four buffers), per (batch b, KV head h):
+ *
+ *   window       k_win, v_win  [B,Hkv,W',D] bf16   the last W' = min(window, N) prefill rows
+ *   vertical     k_vl, v_vl    [B,Hkv,k,D]  bf16   rows vl_idx[b,h,:] of the prefill cache, in that order
+ *   staging      k_s, v_s      [B,Hkv,staging_capacity,D] bf16, of which the first n_staging rows are
+ *                              valid; the caller appends new tokens' rows there (plain copies) and
+ *                              counts them in n_staging.  Folding staged rows into the other buffers
+ *                              is not described by the paper and not part of this library.
+ *   quantized    the other nQ = N - W' - k prefix rows, COMPACTED in ascending position order and cut
+ *                into groups of `group` (64) consecutive compacted rows x all D channels; each group is
+ *                quantized exactly as hyq_quantize_blocks quantizes a tile (INT4, c_B = 7, fp32 scale
+ *                per group; the last group may be ragged).  Per head the row count is padded to
+ *                nQp = 64 * ceil(nQ / 64); padding rows hold unspecified codes and are never used.
+ *       kq_codes  [B,Hkv,nQp,D/2] bytes: row-major, channel 2m in the low nibble and 2m+1 in the high
+ *                 nibble of byte m, two's complement (hyq_quantize_blocks' INT4 layout).
+ *       vq_codes  [B,Hkv,nQp/16,1024] bytes, FRAGMENT-MAJOR: the codes of 16 consecutive compacted rows
+ *                 form one 1024-byte tile laid out as 32 lanes x 8 little-endian 32-bit words; nibble n
+ *                 (bits 4n..4n+3) of word x of lane l = 4r + j holds
+ *                     channel 64*(x >> 2) + 8*r + 2*(x & 3) + (n & 1)
+ *                     of row  2*j + (n >> 2) + 8*((n >> 1) & 1)          of the tile,
+ *                 i.e. each lane of a warp reads 32 contiguous bytes and owns, without any shuffle, the
+ *                 operand registers of the warp-level matrix instruction that accumulates P.V.
+ *       kq_scales, vq_scales  [B,Hkv,nQp/64] fp32.
+ *
+ * (Quant(.; G) over compacted rows, and one vertical set per KV head given by the caller, are this
+ * library's readings: Algorithm 4 does not say how groups are cut after rows are removed, and Algorithm 1
+ * yields one set per query head.)
+ */
+#ifndef HYQ_DECODE_H_
+#define HYQ_DECODE_H_
+
+#include "hyq.h"
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct {
+  uint32_t struct_size;
+  int32_t B, Hq, Hkv, D;
+  int32_t N;                    /* prefill rows frozen */
+  int32_t window;               /* W; the window buffers hold min(W, N) rows */
+  int32_t k;                    /* vertical rows per KV head, 0 <= k <= N - min(W, N) */
+  int32_t group;                /* G: must be 64 */
+  int32_t format;               /* K and V code format: must be HYQ_FMT_INT4 (K4V4) */
+  int32_t staging_capacity;     /* W_s: rows allocated per head in k_s / v_s (may be 0) */
+  int32_t n_staging;            /* valid staging rows, 0 <= n_staging <= staging_capacity */
+  void* kq_codes;
+  void* vq_codes;
+  float* kq_scales;
+  float* vq_scales;
+  void* k_vl;
+  void* v_vl;
+  void* k_win;
+  void* v_win;
+  void* k_s;
+  void* v_s;
+} hyq_kv_cache;
+
+typedef struct {
+  int64_t quantized_rows;        /* nQ */
+  int64_t padded_rows;           /* nQp */
+  size_t kq_codes_bytes, vq_codes_bytes;     /* whole batch, each */
+  size_t scales_bytes;                       /* each of kq_scales, vq_scales */
+  size_t vertical_bytes, window_bytes, staging_bytes;   /* each of the K and V buffers */
+} hyq_kv_cache_sizes;
+
+/* Host-only: buffer sizes for a cache description (pointers ignored).  Errors as hyq_freeze. */
+int hyq_kv_cache_query_sizes(const hyq_kv_cache* cache, hyq_kv_cache_sizes* sizes /* host, out */);
+
+/* ---------------------------------------------------------------------------------------------
+ * hyq_freeze - Algorithm 4.  Reads the prefill cache k_, v [B,Hkv,N,D] bf16 and vl_idx [B,Hkv,k]
+ * int32 (each row strictly ascending, values in [0, N - min(W,N)); NULL iff k == 0), writes the window,
+ * vertical and quantized buffers of `cache` (layouts above).  The staging buffers are not touched
+ * (an empty staging buffer is n_staging = 0).  The prefill cache may be freed once the enqueued
+ * work has completed.  Errors: INVALID_ARG (null pointer, sizes out of range, struct_size),
+ * UNSUPPORTED (D != 128, group != 64, format != INT4, g > 8), ALIGNMENT (any buffer not 16-byte aligned).
+ * ------------------------------------------------------------------------------------------- */
+int hyq_freeze(const void* k_, const void* v, const int32_t* vl_idx, const hyq_kv_cache* cache, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * hyq_hybrid_attention_decode - Algorithm 3 / Section 3.3 for one token per sequence:
+ *     s_j   = softmax_scale * <q[b,h], key_j>      over every cached row j of KV head h / g, where
+ *             key_j / value_j = scale(group) * code for quantized rows, the bf16 row otherwise
+ *     out[b,h] = sum_j softmax(s)_j value_j
+ *   The four segments are read once; the rows are cut into `splits` slices that independent CTAs reduce
+ *   with an online softmax, and a second kernel merges the slices (the split/ReduceSoftmax of Algorithm 3,
+ *   applied to all four segments instead of the quantized one only: one softmax either way).
+ *
+ *   q [B,Hq,D] bf16 (device).  out [B,Hq,D]: bf16 (out_dtype 0) or fp32 (1).  lse: optional [B,Hq] fp32,
+ *   natural-log-sum-exp of the scaled scores (NULL to skip).  softmax_scale 0 => 1/sqrt(D).
+ *   splits: S >= 1, or 0 for a choice that fills the GPU.  workspace: hyq_hybrid_attention_decode_workspace
+ *   bytes (the slices' partial results).  The cache must hold at least one row in total.
+ *   Errors: as hyq_freeze, plus WORKSPACE.
+ * ------------------------------------------------------------------------------------------- */
+int hyq_hybrid_attention_decode_workspace(const hyq_kv_cache* cache, int splits, size_t* bytes /* host, out */);
+int hyq_hybrid_attention_decode(const void* q, const hyq_kv_cache* cache, float softmax_scale, int splits,
+                                int out_dtype, void* out, float* lse, void* workspace, size_t workspace_bytes,
+                                void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HYQ_DECODE_H_ */

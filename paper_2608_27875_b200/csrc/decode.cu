@@ -1,0 +1,364 @@
+// Hybrid-precision KV-cache attention for one new token (Algorithm 3 / Section 3.3).
+//
+// The op is a stream over the cache: every cached row is read once, 128 B per INT4 row (K + V) and 512 B per
+// bf16 row, against 2 * g * 128 multiply-adds per row and tensor - HBM-bound once the arithmetic is cheap
+// enough.  With g = 4 query heads per KV head, CUDA-core FMAs plus the nibble unpacking would need more
+// issue slots than the memory system leaves time for, and a tcgen05 path would have to write the
+// dequantized tile to shared memory first (4x the bytes that came from HBM, more than the shared-memory
+// bandwidth that 1/148th of 7 TB/s allows).  So the codes are dequantized in registers, straight into the
+// operand layout of the warp-level matrix instruction (mma.sync m16n8k16, fp32 accumulate), with the long
+// side of the instruction on the keys (Q.K^T) or the channels (P.V) and the 8-wide side on the g heads:
+//
+//   S^T[16 keys x 8 heads]   = Khat[16 x 128] . q^T            8 k-steps; A from the codes, B from q (fp16)
+//   O^T[128 ch  x 8 heads]  += Vhat^T[128 x 16] . P^T[16 x 8]  8 m-tiles; A from the codes, B = P^T
+//
+// The contraction index of the first product and the row index of the second may be permuted freely, so
+// each lane takes whatever channels arrive in its own 16-byte loads; P^T's operand layout is the transpose
+// of S^T's accumulator layout, which `movmatrix` provides for 8x8 b16 blocks.  V's codes are stored by
+// Freeze in exactly the operand order (see hyq_decode.h), K's stay row-major.  INT4 -> fp16 is one LOP3
+// (nibble ^ 8 | 0x6400 = 1032 + code) and one packed subtract for two codes.
+// The bf16 segments (vertical rows, staging, window) go through the same two products with bf16 operands;
+// there V^T's key pairs are formed from two rows' words with byte permutes.
+//
+// Grid: (splits, B * Hkv).  A CTA owns a contiguous slice of the head's 16-row tiles (all four segments
+// form one tile list); its 4 warps take tiles round-robin, each with its own online-softmax state, which
+// are merged through shared memory; the slices' (m, l, acc) go to the workspace and decode_merge_kernel
+// applies ReduceSoftmax.  Softmax is lazy: a tile only raises the running reference maximum when one of its
+// scores exceeds it by more than 2^DEC_RAISE (warp vote), so the usual tile costs four compares, four ex2
+// and no shuffle.
+#include <cuda_fp16.h>
+
+#include "decode_common.cuh"
+
+namespace hyq {
+
+constexpr int DEC_THREADS = 128;
+constexpr int DEC_WARPS = DEC_THREADS / 32;
+constexpr float DEC_RAISE = 8.0f;          // log2 units; P <= 2^8 stays far inside fp16 / bf16 range
+
+struct DecParams {
+    int g, splits;
+    long nQ, nQp;
+    int k, W, n_s, Ws;
+    float scale_log2;
+    const uint8_t* kq; const uint8_t* vq; const float* ks; const float* vs;
+    const uint4 *k_vl, *v_vl, *k_s, *v_s, *k_win, *v_win;
+    const uint4* q;
+    float* part_acc;     // [unit][split][8 heads][128 channels]  unnormalised
+    float* part_ml;      // [unit][split][8 heads][2]             reference maximum (log2 units), row sum
+};
+
+__device__ __forceinline__ void mma_f16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                        uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                         uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+// 8x8 b16 transpose across the warp: lane 4r+j gives (row r, cols 2j, 2j+1), receives the same of the transpose
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
+    uint32_t d;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+    return d;
+}
+// two INT4 codes (two's complement nibbles at bits 0-3 and 16-19 of w) -> packed fp16 values
+__device__ __forceinline__ uint32_t dq4(uint32_t w) {
+    uint32_t h;
+    asm("lop3.b32 %0, %1, 0x000F000F, 0x64086408, 0x6A;" : "=r"(h) : "r"(w));      // (w & mask) ^ magic = 1032 + code
+    asm("sub.rn.f16x2 %0, %1, %2;" : "=r"(h) : "r"(h), "r"(0x64086408u));
+    return h;
+}
+__device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
+    uint32_t d;
+    asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    return d;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    uint32_t d;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    return d;
+}
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ uint32_t word_of(const uint4& v, int i) {
+    return i == 0 ? v.x : i == 1 ? v.y : i == 2 ? v.z : v.w;
+}
+// channel of accumulator row (m-tile x, lane row r, e = 0: row r, 1: row r + 8); also V's code layout
+__device__ __forceinline__ int acc_channel(int x, int r, int e) { return 64 * (x >> 2) + 8 * r + 2 * (x & 3) + e; }
+
+struct SoftmaxState {
+    float m0, m1, l0, l1;      // heads 2j and 2j+1 of this lane: reference maximum (log2 units), partial row sum
+};
+
+// One tile's scores (keys r and r+8, heads 2j and 2j+1; log2 units, masked = -inf) -> weights p[4].
+// Raises the reference maxima and rescales the accumulators only when some score is far above them.
+__device__ __forceinline__ void softmax_tile(SoftmaxState& st, float (&acc)[8][4], const float (&s)[4], float (&p)[4]) {
+    const bool far = fmaxf(s[0], s[2]) > st.m0 + DEC_RAISE || fmaxf(s[1], s[3]) > st.m1 + DEC_RAISE;
+    if (__any_sync(0xffffffffu, far)) {
+        float t0 = fmaxf(s[0], s[2]), t1 = fmaxf(s[1], s[3]);
+#pragma unroll
+        for (int o = 4; o < 32; o <<= 1) {
+            t0 = fmaxf(t0, __shfl_xor_sync(0xffffffffu, t0, o));
+            t1 = fmaxf(t1, __shfl_xor_sync(0xffffffffu, t1, o));
+        }
+        const float n0 = fmaxf(st.m0, t0), n1 = fmaxf(st.m1, t1);
+        const float c0 = n0 == -INFINITY ? 1.0f : ex2(st.m0 - n0), c1 = n1 == -INFINITY ? 1.0f : ex2(st.m1 - n1);
+        st.m0 = n0; st.m1 = n1;
+        st.l0 *= c0; st.l1 *= c1;
+#pragma unroll
+        for (int x = 0; x < 8; ++x) { acc[x][0] *= c0; acc[x][2] *= c0; acc[x][1] *= c1; acc[x][3] *= c1; }
+    }
+    p[0] = ex2(s[0] - st.m0); p[2] = ex2(s[2] - st.m0);
+    p[1] = ex2(s[1] - st.m1); p[3] = ex2(s[3] - st.m1);
+    st.l0 += p[0] + p[2];
+    st.l1 += p[1] + p[3];
+}
+
+__global__ void __launch_bounds__(DEC_THREADS, 4)
+decode_kernel(const DecParams p) {
+    const int split = blockIdx.x;
+    const long unit = blockIdx.y;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, r = lane >> 2, j = lane & 3;
+
+    __shared__ __align__(16) uint16_t qs[DEC_MAX_GROUP][HYQ_D];      // bf16 bits, heads >= g zero
+    __shared__ float red_ml[DEC_WARPS][DEC_MAX_GROUP][2];
+    __shared__ float red_acc[DEC_WARPS][DEC_MAX_GROUP][HYQ_D];
+
+    {   // q of the g heads of this KV head: thread t loads 8 channels of head t >> 4
+        const int h = threadIdx.x >> 4, c8 = threadIdx.x & 15;
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (h < p.g) v = __ldg(p.q + (unit * p.g + h) * 16 + c8);
+        *reinterpret_cast<uint4*>(&qs[h][c8 * 8]) = v;
+    }
+    __syncthreads();
+
+    const long Tq = (p.nQ + 15) / 16;
+    const int Tvl = (p.k + 15) / 16, Ts = (p.n_s + 15) / 16, Tw = (p.W + 15) / 16;
+    const long T = Tq + Tvl + Ts + Tw;
+    const long lo = T * split / p.splits, hi = T * (split + 1) / p.splits;
+
+    SoftmaxState st = {-INFINITY, -INFINITY, 0.0f, 0.0f};
+    float acc[8][4];
+#pragma unroll
+    for (int x = 0; x < 8; ++x) acc[x][0] = acc[x][1] = acc[x][2] = acc[x][3] = 0.0f;
+
+    // ---------------- quantized prefix ----------------
+    const long q_hi = hi < Tq ? hi : Tq;
+    if (lo + warp < q_hi) {
+        uint32_t qf[16];                                   // q^T operand, fp16: k-step c -> qf[2c], qf[2c+1]
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            const int base = 32 * j + 8 * (c >> 1) + 2 * (c & 1);
+            const uint16_t* qr = qs[r];
+            auto f16 = [&](int ch) { return __float2half_rn(__uint_as_float((uint32_t)qr[ch] << 16)); };
+            const __half2 h0 = __halves2half2(f16(base), f16(base + 4));
+            const __half2 h1 = __halves2half2(f16(base + 1), f16(base + 5));
+            qf[2 * c] = *reinterpret_cast<const uint32_t*>(&h0);
+            qf[2 * c + 1] = *reinterpret_cast<const uint32_t*>(&h1);
+        }
+        const uint4* kq = reinterpret_cast<const uint4*>(p.kq + unit * p.nQp * 64);
+        const uint4* vq = reinterpret_cast<const uint4*>(p.vq + unit * (p.nQp / 16) * DEC_VTILE_BYTES);
+        const float* ks = p.ks + unit * (p.nQp / 64);
+        const float* vs = p.vs + unit * (p.nQp / 64);
+
+        long t = lo + warp;
+        uint4 ka = __ldg(kq + (t * 16 + r) * 4 + j), kb = __ldg(kq + (t * 16 + r + 8) * 4 + j);
+        uint4 va = __ldg(vq + t * 64 + lane * 2), vb = __ldg(vq + t * 64 + lane * 2 + 1);
+        float fk = __ldg(ks + (t >> 2)), fv = __ldg(vs + (t >> 2));
+        for (; t < q_hi; t += DEC_WARPS) {
+            const long tn = t + DEC_WARPS < q_hi ? t + DEC_WARPS : t;      // prefetch (the last one re-reads itself)
+            const uint4 nka = __ldg(kq + (tn * 16 + r) * 4 + j), nkb = __ldg(kq + (tn * 16 + r + 8) * 4 + j);
+            const uint4 nva = __ldg(vq + tn * 64 + lane * 2), nvb = __ldg(vq + tn * 64 + lane * 2 + 1);
+            const float nfk = __ldg(ks + (tn >> 2)), nfv = __ldg(vs + (tn >> 2));
+
+            float c4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                const uint32_t wa = word_of(ka, c >> 1) >> (8 * (c & 1)), wb = word_of(kb, c >> 1) >> (8 * (c & 1));
+                mma_f16(c4, dq4(wa), dq4(wb), dq4(wa >> 4), dq4(wb >> 4), qf[2 * c], qf[2 * c + 1]);
+            }
+            const float f = fk * p.scale_log2;
+            const long row = t * 16 + r;
+            float s[4], pw[4];
+            s[0] = row < p.nQ ? c4[0] * f : -INFINITY;     s[1] = row < p.nQ ? c4[1] * f : -INFINITY;
+            s[2] = row + 8 < p.nQ ? c4[2] * f : -INFINITY; s[3] = row + 8 < p.nQ ? c4[3] * f : -INFINITY;
+            softmax_tile(st, acc, s, pw);
+            const uint32_t b0 = movmatrix_trans(pack_f16(pw[0] * fv, pw[1] * fv));
+            const uint32_t b1 = movmatrix_trans(pack_f16(pw[2] * fv, pw[3] * fv));
+#pragma unroll
+            for (int x = 0; x < 8; ++x) {
+                const uint32_t w = word_of(x < 4 ? va : vb, x & 3);
+                mma_f16(acc[x], dq4(w), dq4(w >> 4), dq4(w >> 8), dq4(w >> 12), b0, b1);
+            }
+            ka = nka; kb = nkb; va = nva; vb = nvb; fk = nfk; fv = nfv;
+        }
+    }
+
+    // ---------------- bf16 segments: vertical rows, staging, window ----------------
+    long f_lo = lo > Tq ? lo : Tq;
+    // keep the round-robin phase of the tile list so that the warps stay balanced across the boundary
+    long t = f_lo + ((warp - (f_lo - lo)) % DEC_WARPS + DEC_WARPS) % DEC_WARPS;
+    if (t < hi) {
+        uint32_t qb[16];                                   // q^T operand, bf16
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            const int base = 32 * (c >> 1) + 8 * j + 4 * (c & 1);
+            qb[2 * c] = *reinterpret_cast<const uint32_t*>(&qs[r][base]);
+            qb[2 * c + 1] = *reinterpret_cast<const uint32_t*>(&qs[r][base + 2]);
+        }
+        for (; t < hi; t += DEC_WARPS) {
+            long u = t - Tq;
+            const uint4 *kseg, *vseg;
+            int n;
+            if (u < Tvl) { kseg = p.k_vl + unit * p.k * 16; vseg = p.v_vl + unit * p.k * 16; n = p.k; }
+            else if ((u -= Tvl) < Ts) { kseg = p.k_s + unit * p.Ws * 16; vseg = p.v_s + unit * p.Ws * 16; n = p.n_s; }
+            else { u -= Ts; kseg = p.k_win + unit * p.W * 16; vseg = p.v_win + unit * p.W * 16; n = p.W; }
+            const int row0 = (int)u * 16;
+            const int ra = min(row0 + r, n - 1), rb = min(row0 + r + 8, n - 1);
+            uint4 ka[4], kb[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { ka[i] = __ldg(kseg + (long)ra * 16 + 4 * i + j); kb[i] = __ldg(kseg + (long)rb * 16 + 4 * i + j); }
+            uint4 vv[4][2];
+#pragma unroll
+            for (int sIdx = 0; sIdx < 4; ++sIdx) {
+                const int key = min(row0 + 2 * j + (sIdx & 1) + 8 * (sIdx >> 1), n - 1);
+                vv[sIdx][0] = __ldg(vseg + (long)key * 16 + r);
+                vv[sIdx][1] = __ldg(vseg + (long)key * 16 + 8 + r);
+            }
+            float c4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                const int wd = 2 * (c & 1);
+                mma_bf16(c4, word_of(ka[c >> 1], wd), word_of(kb[c >> 1], wd), word_of(ka[c >> 1], wd + 1),
+                         word_of(kb[c >> 1], wd + 1), qb[2 * c], qb[2 * c + 1]);
+            }
+            float s[4], pw[4];
+            s[0] = row0 + r < n ? c4[0] * p.scale_log2 : -INFINITY;     s[1] = row0 + r < n ? c4[1] * p.scale_log2 : -INFINITY;
+            s[2] = row0 + r + 8 < n ? c4[2] * p.scale_log2 : -INFINITY; s[3] = row0 + r + 8 < n ? c4[3] * p.scale_log2 : -INFINITY;
+            softmax_tile(st, acc, s, pw);
+            const uint32_t b0 = movmatrix_trans(pack_bf16(pw[0], pw[1]));
+            const uint32_t b1 = movmatrix_trans(pack_bf16(pw[2], pw[3]));
+#pragma unroll
+            for (int x = 0; x < 8; ++x) {
+                const uint32_t w0 = word_of(vv[0][x >> 2], x & 3), w1 = word_of(vv[1][x >> 2], x & 3);
+                const uint32_t w2 = word_of(vv[2][x >> 2], x & 3), w3 = word_of(vv[3][x >> 2], x & 3);
+                mma_bf16(acc[x], __byte_perm(w0, w1, 0x5410), __byte_perm(w0, w1, 0x7632), __byte_perm(w2, w3, 0x5410),
+                         __byte_perm(w2, w3, 0x7632), b0, b1);
+            }
+        }
+    }
+
+    // ---------------- merge the warps' states, write the slice's partial result ----------------
+#pragma unroll
+    for (int o = 4; o < 32; o <<= 1) {
+        st.l0 += __shfl_xor_sync(0xffffffffu, st.l0, o);
+        st.l1 += __shfl_xor_sync(0xffffffffu, st.l1, o);
+    }
+    if (r == 0) {
+        red_ml[warp][2 * j][0] = st.m0; red_ml[warp][2 * j][1] = st.l0;
+        red_ml[warp][2 * j + 1][0] = st.m1; red_ml[warp][2 * j + 1][1] = st.l1;
+    }
+#pragma unroll
+    for (int x = 0; x < 8; ++x) {
+        red_acc[warp][2 * j][acc_channel(x, r, 0)] = acc[x][0];
+        red_acc[warp][2 * j + 1][acc_channel(x, r, 0)] = acc[x][1];
+        red_acc[warp][2 * j][acc_channel(x, r, 1)] = acc[x][2];
+        red_acc[warp][2 * j + 1][acc_channel(x, r, 1)] = acc[x][3];
+    }
+    __syncthreads();
+    const long slot = unit * p.splits + split;
+    for (int h = 0; h < p.g; ++h) {
+        float M = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < DEC_WARPS; ++w) M = fmaxf(M, red_ml[w][h][0]);
+        float L = 0.0f, A = 0.0f;
+#pragma unroll
+        for (int w = 0; w < DEC_WARPS; ++w) {
+            const float mw = red_ml[w][h][0];
+            const float wt = mw == -INFINITY ? 0.0f : ex2(mw - M);
+            L += red_ml[w][h][1] * wt;
+            A += red_acc[w][h][threadIdx.x] * wt;
+        }
+        p.part_acc[(slot * DEC_MAX_GROUP + h) * HYQ_D + threadIdx.x] = A;
+        if (threadIdx.x == 0) {
+            p.part_ml[(slot * DEC_MAX_GROUP + h) * 2] = M;
+            p.part_ml[(slot * DEC_MAX_GROUP + h) * 2 + 1] = L;
+        }
+    }
+}
+
+// ReduceSoftmax of Algorithm 3 over the slices; one CTA per (b, kv head), one thread per channel.
+__global__ void __launch_bounds__(HYQ_D)
+decode_merge_kernel(const float* __restrict__ part_acc, const float* __restrict__ part_ml, int g, int splits,
+                    int out_fp32, void* __restrict__ out, float* __restrict__ lse) {
+    const long unit = blockIdx.x;
+    for (int h = 0; h < g; ++h) {
+        float M = -INFINITY;
+        for (int s = 0; s < splits; ++s) M = fmaxf(M, __ldg(part_ml + ((unit * splits + s) * DEC_MAX_GROUP + h) * 2));
+        float L = 0.0f, A = 0.0f;
+        for (int s = 0; s < splits; ++s) {
+            const long slot = (unit * splits + s) * DEC_MAX_GROUP + h;
+            const float ms = __ldg(part_ml + slot * 2);
+            const float wt = ms == -INFINITY ? 0.0f : ex2(ms - M);
+            L += __ldg(part_ml + slot * 2 + 1) * wt;
+            A += __ldg(part_acc + slot * HYQ_D + threadIdx.x) * wt;
+        }
+        const float o = A / L;
+        const long oi = (unit * g + h) * HYQ_D + threadIdx.x;
+        if (out_fp32) static_cast<float*>(out)[oi] = o;
+        else static_cast<__nv_bfloat16*>(out)[oi] = __float2bfloat16_rn(o);
+        if (lse && threadIdx.x == 0) lse[unit * g + h] = (M + log2f(L)) * 0.6931471805599453f;
+    }
+}
+
+static long decode_tiles(const hyq_kv_cache& c) {
+    const CacheGeo g = cache_geo(c);
+    return (g.nQ + 15) / 16 + (c.k + 15) / 16 + (c.n_staging + 15) / 16 + (g.W + 15) / 16;
+}
+
+int decode_auto_splits(const hyq_kv_cache& c) {
+    const long units = (long)c.B * c.Hkv;
+    const long T = decode_tiles(c);
+    long s = (148L * 4 + units - 1) / units;            // about four CTAs per SM
+    const long cap = T / 8 > 1 ? T / 8 : 1;             // at least two tiles per warp
+    if (s > cap) s = cap;
+    if (s > 64) s = 64;
+    return (int)(s < 1 ? 1 : s);
+}
+
+size_t decode_workspace_bytes(const hyq_kv_cache& c, int splits) {
+    const size_t slots = (size_t)c.B * c.Hkv * splits * DEC_MAX_GROUP;
+    return align_up(slots * HYQ_D * sizeof(float), 16) + align_up(slots * 2 * sizeof(float), 16);
+}
+
+int launch_decode(const void* q, const hyq_kv_cache& c, float alpha, int splits, int out_dtype, void* out, float* lse,
+                  void* workspace, cudaStream_t st) {
+    const CacheGeo geo = cache_geo(c);
+    const long units = (long)c.B * c.Hkv;
+    DecParams p;
+    p.g = c.Hq / c.Hkv; p.splits = splits;
+    p.nQ = geo.nQ; p.nQp = geo.nQp; p.k = c.k; p.W = geo.W; p.n_s = c.n_staging; p.Ws = c.staging_capacity;
+    p.scale_log2 = alpha * 1.4426950408889634f;
+    p.kq = static_cast<const uint8_t*>(c.kq_codes); p.vq = static_cast<const uint8_t*>(c.vq_codes);
+    p.ks = c.kq_scales; p.vs = c.vq_scales;
+    p.k_vl = static_cast<const uint4*>(c.k_vl); p.v_vl = static_cast<const uint4*>(c.v_vl);
+    p.k_s = static_cast<const uint4*>(c.k_s); p.v_s = static_cast<const uint4*>(c.v_s);
+    p.k_win = static_cast<const uint4*>(c.k_win); p.v_win = static_cast<const uint4*>(c.v_win);
+    p.q = static_cast<const uint4*>(q);
+    const size_t slots = (size_t)units * splits * DEC_MAX_GROUP;
+    p.part_acc = static_cast<float*>(workspace);
+    p.part_ml = reinterpret_cast<float*>(static_cast<char*>(workspace) + align_up(slots * HYQ_D * sizeof(float), 16));
+    decode_kernel<<<dim3((unsigned)splits, (unsigned)units), DEC_THREADS, 0, st>>>(p);
+    decode_merge_kernel<<<(unsigned)units, HYQ_D, 0, st>>>(p.part_acc, p.part_ml, p.g, splits, out_dtype, out, lse);
+    return launch_status();
+}
+
+}  // namespace hyq

@@ -1,0 +1,40 @@
+// Geometry of the hybrid KV cache shared by the Freeze and decode kernels (layout only).
+#pragma once
+#include "common.cuh"
+#include "../../include/hyq_decode.h"
+
+namespace hyq {
+
+constexpr int DEC_TILE_KEYS = 16;          // rows per matrix-instruction tile
+constexpr int DEC_VTILE_BYTES = 1024;      // 16 rows x 128 channels x 4 bits
+constexpr int DEC_MAX_GROUP = 8;           // query heads per KV head (the n = 8 side of m16n8k16)
+
+struct CacheGeo {
+    int W;              // rows in the window buffers: min(window, N)
+    long nQ, nQp;       // quantized rows per head: valid, padded to whole groups of 64
+};
+
+static inline CacheGeo cache_geo(const hyq_kv_cache& c) {
+    CacheGeo g;
+    g.W = c.window < c.N ? c.window : c.N;
+    g.nQ = (long)c.N - g.W - c.k;
+    g.nQp = (g.nQ + 63) / 64 * 64;
+    return g;
+}
+
+// Byte of a V tile that holds channels (d, d + 1), d even, of row `key` (0..15) of the tile: lane l = 4r + j
+// owns 32 bytes; word x, nibble n of that lane is channel 64*(x>>2) + 8r + 2*(x&3) + (n&1) of row
+// 2j + (n>>2) + 8*((n>>1)&1).
+__host__ __device__ __forceinline__ int vq_byte_offset(int key, int d) {
+    const int j = (key & 7) >> 1, n = ((key >> 3) << 1) | ((key & 1) << 2);
+    const int r = (d >> 3) & 7, x = ((d >> 6) << 2) | ((d >> 1) & 3);
+    return (4 * r + j) * 32 + x * 4 + (n >> 1);
+}
+
+int launch_freeze(const void* k_, const void* v, const int32_t* vl_idx, const hyq_kv_cache& c, cudaStream_t st);
+int decode_auto_splits(const hyq_kv_cache& c);
+size_t decode_workspace_bytes(const hyq_kv_cache& c, int splits);
+int launch_decode(const void* q, const hyq_kv_cache& c, float alpha, int splits, int out_dtype, void* out, float* lse,
+                  void* workspace, cudaStream_t st);
+
+}  // namespace hyq

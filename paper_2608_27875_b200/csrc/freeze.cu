@@ -1,0 +1,146 @@
+// Freeze (Algorithm 4): builds the hybrid KV cache of the decode stage from the prefill cache.
+//
+// Two kernels, both HBM-bound and read-once / write-once:
+//   gather_rows_kernel     copies the vertical rows (by index) and the window rows (a slice) as bf16;
+//   freeze_quantize_kernel one CTA per group of 64 COMPACTED rows of one (b, kv head) and one tensor
+//                          (K or V): finds the source rows (the complement of the ascending vertical
+//                          set, by binary search), quantizes the 64 x 128 group to INT4 with the
+//                          arithmetic of the per-tile quantizer (fp32, one rounding per operation), and
+//                          writes K row-major and V in the fragment-major tile layout the decode kernel
+//                          loads straight into matrix-instruction operand registers.
+#include "common.cuh"
+#include "decode_common.cuh"
+
+namespace hyq {
+
+constexpr int FRZ_THREADS = 128;
+
+// Source position of compacted row p: p + j with j the number of vertical indices below it,
+// i.e. the smallest j with idx[j] - j > p (idx ascending, so idx[j] - j never decreases).
+__device__ __forceinline__ int source_row(const int32_t* __restrict__ idx, int k, int p) {
+    int lo = 0, hi = k;
+    while (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        if (__ldg(idx + mid) - mid > p) hi = mid; else lo = mid + 1;
+    }
+    return p + lo;
+}
+
+__global__ void __launch_bounds__(FRZ_THREADS)
+gather_rows_kernel(const uint4* __restrict__ k_, const uint4* __restrict__ v, const int32_t* __restrict__ idx,
+                   int N, int W, int k_vl, uint4* __restrict__ k_vl_out, uint4* __restrict__ v_vl_out,
+                   uint4* __restrict__ k_win, uint4* __restrict__ v_win) {
+    const long head = blockIdx.y;
+    const int o = blockIdx.x * 8 + (threadIdx.x >> 4);
+    const int c = threadIdx.x & 15;                       // 16 x 16 bytes = one 256-byte row
+    if (o >= k_vl + W) return;
+    const int P = N - W;
+    const bool vl = o < k_vl;
+    const int src = vl ? __ldg(idx + head * k_vl + o) : P + (o - k_vl);
+    const long s = (head * N + src) * 16 + c;
+    const long d = vl ? (head * k_vl + o) * 16 + c : (head * W + (o - k_vl)) * 16 + c;
+    (vl ? k_vl_out : k_win)[d] = __ldg(k_ + s);
+    (vl ? v_vl_out : v_win)[d] = __ldg(v + s);
+}
+
+__global__ void __launch_bounds__(FRZ_THREADS)
+freeze_quantize_kernel(const uint4* __restrict__ k_, const uint4* __restrict__ v, const int32_t* __restrict__ idx,
+                       int N, int k_vl, int nQ, int nQp, uint8_t* __restrict__ kq, uint8_t* __restrict__ vq,
+                       float* __restrict__ ks, float* __restrict__ vs) {
+    const int grp = blockIdx.x;
+    const long head = blockIdx.y;
+    const bool is_v = blockIdx.z == 1;
+    const uint4* x = (is_v ? v : k_) + head * N * 16;
+    const int32_t* hidx = idx + head * k_vl;
+
+    __shared__ int src[64];
+    __shared__ float warp_max[FRZ_THREADS / 32];
+    __shared__ __align__(16) uint8_t vtile[4 * DEC_VTILE_BYTES];
+    if (threadIdx.x < 64) {
+        const int p = grp * 64 + threadIdx.x;
+        src[threadIdx.x] = p < nQ ? source_row(hidx, k_vl, p) : -1;
+    }
+    __syncthreads();
+
+    uint4 r[4][2];
+    float amax = 0.0f;
+#pragma unroll
+    for (int gi = 0; gi < 4; ++gi) {
+        const int u = threadIdx.x + gi * FRZ_THREADS;     // 16-channel unit: row u >> 3, channels 16 * (u & 7)
+        const int s = src[u >> 3];
+        if (s >= 0) {
+            r[gi][0] = __ldg(x + (long)s * 16 + (u & 7) * 2);
+            r[gi][1] = __ldg(x + (long)s * 16 + (u & 7) * 2 + 1);
+        } else {
+            r[gi][0] = make_uint4(0, 0, 0, 0);
+            r[gi][1] = make_uint4(0, 0, 0, 0);
+        }
+        const uint32_t* w = reinterpret_cast<const uint32_t*>(&r[gi][0]);
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            amax = fmaxf(amax, fabsf(bf16_lo(w[c])));
+            amax = fmaxf(amax, fabsf(bf16_hi(w[c])));
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+    if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = amax;
+    __syncthreads();
+    amax = fmaxf(fmaxf(warp_max[0], warp_max[1]), fmaxf(warp_max[2], warp_max[3]));
+
+    const bool dead = !(amax >= 0x1p-100f);
+    const float inv = dead ? 0.0f : __fdiv_rn(7.0f, amax);
+    if (threadIdx.x == 0) (is_v ? vs : ks)[head * (nQp / 64) + grp] = dead ? 0.0f : __fdiv_rn(amax, 7.0f);
+
+#pragma unroll
+    for (int gi = 0; gi < 4; ++gi) {
+        const int u = threadIdx.x + gi * FRZ_THREADS;
+        const int row = u >> 3, ch0 = (u & 7) * 16;
+        const uint32_t* w = reinterpret_cast<const uint32_t*>(&r[gi][0]);
+        uint8_t b[8];
+#pragma unroll
+        for (int m = 0; m < 8; ++m) {
+            const int q0 = max(-7, min(7, __float2int_rn(__fmul_rn(bf16_lo(w[m]), inv))));
+            const int q1 = max(-7, min(7, __float2int_rn(__fmul_rn(bf16_hi(w[m]), inv))));
+            b[m] = (uint8_t)((q0 & 0xF) | ((q1 & 0xF) << 4));
+        }
+        if (!is_v) {
+            uint32_t o0 = b[0] | (b[1] << 8) | (b[2] << 16) | ((uint32_t)b[3] << 24);
+            uint32_t o1 = b[4] | (b[5] << 8) | (b[6] << 16) | ((uint32_t)b[7] << 24);
+            *reinterpret_cast<uint2*>(kq + ((head * nQp + grp * 64 + row) * 64 + ch0 / 2)) = make_uint2(o0, o1);
+        } else {
+            const int tile = row >> 4, key = row & 15;
+#pragma unroll
+            for (int m = 0; m < 8; ++m) vtile[tile * DEC_VTILE_BYTES + vq_byte_offset(key, ch0 + 2 * m)] = b[m];
+        }
+    }
+    if (is_v) {
+        __syncthreads();
+        uint4* dst = reinterpret_cast<uint4*>(vq + (head * (nQp / 16) + grp * 4) * (long)DEC_VTILE_BYTES);
+        const uint4* s4 = reinterpret_cast<const uint4*>(vtile);
+        dst[threadIdx.x] = s4[threadIdx.x];
+        dst[threadIdx.x + FRZ_THREADS] = s4[threadIdx.x + FRZ_THREADS];
+    }
+}
+
+int launch_freeze(const void* k_, const void* v, const int32_t* vl_idx, const hyq_kv_cache& c, cudaStream_t st) {
+    const CacheGeo g = cache_geo(c);
+    const long heads = (long)c.B * c.Hkv;
+    const uint4* k4 = static_cast<const uint4*>(k_);
+    const uint4* v4 = static_cast<const uint4*>(v);
+    if (c.k + g.W > 0) {
+        const dim3 grid((unsigned)((c.k + g.W + 7) / 8), (unsigned)heads);
+        gather_rows_kernel<<<grid, FRZ_THREADS, 0, st>>>(k4, v4, vl_idx, c.N, g.W, c.k, static_cast<uint4*>(c.k_vl),
+                                                         static_cast<uint4*>(c.v_vl), static_cast<uint4*>(c.k_win),
+                                                         static_cast<uint4*>(c.v_win));
+    }
+    if (g.nQ > 0) {
+        const dim3 grid((unsigned)(g.nQp / 64), (unsigned)heads, 2);
+        freeze_quantize_kernel<<<grid, FRZ_THREADS, 0, st>>>(k4, v4, vl_idx, c.N, c.k, (int)g.nQ, (int)g.nQp,
+                                                             static_cast<uint8_t*>(c.kq_codes),
+                                                             static_cast<uint8_t*>(c.vq_codes), c.kq_scales, c.vq_scales);
+    }
+    return launch_status();
+}
+
+}  // namespace hyq

@@ -6,7 +6,7 @@ import re
 
 import pytest
 
-from paper_2608_27875_b200 import api, build
+from paper_2608_27875_b200 import api, build, decode_api
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
@@ -18,11 +18,13 @@ def lib():
 
 
 def test_every_declared_symbol_is_exported(lib):
-    header = open(os.path.join(ROOT, "include", "hyq.h")).read()
-    declared = set(re.findall(r"\b(hyq_[a-z_0-9]+)\s*\(", header))
-    assert declared == set(api.EXPORTS)
-    for name in declared:
-        assert hasattr(lib, name), name
+    for header_name, exports in (("hyq.h", api.EXPORTS), ("hyq_decode.h", decode_api.EXPORTS)):
+        header = open(os.path.join(ROOT, "include", header_name)).read()
+        header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)                 # declarations only, not prose
+        declared = set(re.findall(r"\b(hyq_[a-z_0-9]+)\s*\(", header))
+        assert declared == set(exports), header_name
+        for name in declared:
+            assert hasattr(lib, name), name
 
 
 def test_status_strings_and_version(lib):
@@ -113,3 +115,35 @@ def test_binding_fails_loudly_without_the_library(monkeypatch, tmp_path):
     monkeypatch.setattr(api, "LIB_PATH", str(tmp_path / "missing.so"))
     with pytest.raises(RuntimeError, match="missing"):
         api.lib()
+
+
+def test_decode_side_argument_checks(lib):
+    """Cache descriptions are checked on the host before anything is launched (no GPU needed: every call
+    below must fail in the checks, or is a host-only size query)."""
+    L = decode_api._lib()
+    sizes = decode_api.KvCacheSizes()
+    d = decode_api.make_desc(B=2, Hq=32, Hkv=8, N=1000, window=100, k=37)
+    assert L.hyq_kv_cache_query_sizes(ctypes.byref(d), ctypes.byref(sizes)) == 0
+    assert sizes.quantized_rows == 863 and sizes.padded_rows == 896
+    assert sizes.kq_codes_bytes == sizes.vq_codes_bytes == 16 * 896 * 64 and sizes.scales_bytes == 16 * 14 * 4
+    assert sizes.vertical_bytes == 16 * 37 * 256 and sizes.window_bytes == 16 * 100 * 256
+    assert sizes.staging_bytes == 16 * 128 * 256
+    n = ctypes.c_size_t(0)
+    assert L.hyq_hybrid_attention_decode_workspace(ctypes.byref(d), 5, ctypes.byref(n)) == 0
+    assert n.value == 16 * 5 * 8 * (128 + 2) * 4
+    assert L.hyq_hybrid_attention_decode_workspace(ctypes.byref(d), 0, ctypes.byref(n)) == 0 and n.value > 0
+    w_all = decode_api.make_desc(B=1, Hq=4, Hkv=4, N=50, window=80, k=0)          # window longer than the cache
+    assert L.hyq_kv_cache_query_sizes(ctypes.byref(w_all), ctypes.byref(sizes)) == 0
+    assert sizes.quantized_rows == 0 and sizes.window_bytes == 4 * 50 * 256
+    bad = [dict(k=901), dict(Hq=30), dict(D=64), dict(group=32), dict(fmt=api.FMT_INT8), dict(Hq=128),
+           dict(n_staging=129), dict(N=0)]
+    expect = [1, 1, 2, 2, 2, 2, 1, 1]
+    for kw, code in zip(bad, expect):
+        args = dict(B=2, Hq=32, Hkv=8, N=1000, window=100, k=37)
+        args.update(kw)
+        assert L.hyq_kv_cache_query_sizes(ctypes.byref(decode_api.make_desc(**args)), ctypes.byref(sizes)) == code, kw
+    d.struct_size = 8
+    assert L.hyq_kv_cache_query_sizes(ctypes.byref(d), ctypes.byref(sizes)) == 1
+    d.struct_size = ctypes.sizeof(decode_api.KvCacheDesc)
+    assert L.hyq_freeze(None, None, None, ctypes.byref(d), None) == 1            # null buffers
+    assert L.hyq_hybrid_attention_decode(None, ctypes.byref(d), 0.0, 0, 0, None, None, None, 0, None) == 1

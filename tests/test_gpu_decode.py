@@ -1,0 +1,164 @@
+"""GPU parity of the decode side against the oracle: Freeze (Algorithm 4) bit-exact, the hybrid KV-cache
+attention of one token (Algorithm 3) within the attention tolerances."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from oracle import decode as od
+from paper_2608_27875_b200 import decode_api as dapi, workloads as wl
+from gpu_util import MAX_ABS_TOL, MEAN_REL_TOL, ensure_built, errors, rand_bf16
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    ensure_built()
+
+
+def _idx(B, H, P, kk, seed):
+    rng = np.random.default_rng(seed)
+    return np.stack([np.stack([np.sort(rng.choice(P, kk, replace=False)) for _ in range(H)])
+                     for _ in range(B)]).astype(np.int32)
+
+
+def _v_tiles_to_rows(vq: np.ndarray) -> np.ndarray:
+    """Undoes the fragment-major V layout as the header documents it, written out nibble by nibble:
+    [.., tiles, 1024] bytes -> [.., tiles*16, 64] bytes in the row-major INT4 layout."""
+    lead = vq.shape[:-2]
+    tiles = vq.shape[-2]
+    words = vq.reshape(lead + (tiles, 32, 8, 4)).astype(np.uint32)
+    words = words[..., 0] | (words[..., 1] << 8) | (words[..., 2] << 16) | (words[..., 3] << 24)   # [.., tiles, lane, x]
+    rows = np.zeros(lead + (tiles, 16, 128), dtype=np.uint8)
+    for lane in range(32):
+        r, j = lane >> 2, lane & 3
+        for x in range(8):
+            for n in range(8):
+                ch = 64 * (x >> 2) + 8 * r + 2 * (x & 3) + (n & 1)
+                key = 2 * j + (n >> 2) + 8 * ((n >> 1) & 1)
+                rows[..., key, ch] = (words[..., lane, x] >> (4 * n)) & 0xF
+    packed = rows[..., 0::2] | (rows[..., 1::2] << 4)
+    return packed.reshape(lead + (tiles * 16, 64))
+
+
+def _freeze_both(K, V, idx, W, Hq, staging_capacity=128):
+    ref = od.freeze(wl.bits(K), wl.bits(V), idx, W, staging_capacity=staging_capacity)
+    idx_t = None if idx is None or idx.shape[2] == 0 else torch.from_numpy(idx).cuda()
+    cache = dapi.hyq_freeze(K.cuda(), V.cuda(), idx_t, W, Hq, staging_capacity)
+    torch.cuda.synchronize()
+    return ref, cache
+
+
+def _stage(ref, cache, n_s, seed):
+    B, H, D = ref["B"], ref["Hkv"], ref["D"]
+    for i in range(n_s):
+        kn, vn = rand_bf16((B, H, D), seed + 2 * i), rand_bf16((B, H, D), seed + 2 * i + 1)
+        od.append_staging(ref, wl.bits(kn), wl.bits(vn))
+        cache.append(kn.cuda(), vn.cuda())
+
+
+def _assert_cache_equal(ref, cache):
+    nQ, kk, W = ref["nQ"], ref["k"], ref["window"]
+    b = {n: t.cpu().numpy() if t.dtype != torch.bfloat16 else wl.bits(t.cpu()) for n, t in cache.buffers.items()}
+    assert int(cache.sizes.quantized_rows) == nQ
+    if nQ:
+        ng = -(-nQ // 64)
+        assert np.array_equal(b["kq_codes"][:, :, :nQ], ref["kq_codes"])
+        assert np.array_equal(_v_tiles_to_rows(b["vq_codes"])[:, :, :nQ], ref["vq_codes"])
+        assert np.array_equal(b["kq_scales"][:, :, :ng].view(np.uint32), ref["kq_scales"].view(np.uint32))
+        assert np.array_equal(b["vq_scales"][:, :, :ng].view(np.uint32), ref["vq_scales"].view(np.uint32))
+    if kk:
+        assert np.array_equal(b["k_vl"][:, :, :kk], ref["k_vl"]) and np.array_equal(b["v_vl"][:, :, :kk], ref["v_vl"])
+    if W:
+        assert np.array_equal(b["k_win"][:, :, :W], ref["k_win"]) and np.array_equal(b["v_win"][:, :, :W], ref["v_win"])
+
+
+FREEZE_SHAPES = [  # B, Hkv, N, W, k
+    (1, 2, 300, 40, 9), (2, 3, 1000, 128, 37), (1, 1, 64, 0, 0), (1, 2, 129, 1, 64), (1, 2, 50, 80, 0),
+    (1, 2, 200, 20, 180), (2, 8, 4096, 512, 82), (1, 1, 65, 0, 1),
+]
+
+
+@pytest.mark.parametrize("B,Hkv,N,W,kk", FREEZE_SHAPES)
+def test_freeze_is_bit_exact(B, Hkv, N, W, kk):
+    K, V = rand_bf16((B, Hkv, N, 128), 1, 1.5), rand_bf16((B, Hkv, N, 128), 2)
+    K[:, :, : N // 3] *= 0.01                               # groups with very different scales
+    idx = _idx(B, Hkv, N - min(W, N), kk, 3) if kk else None
+    ref, cache = _freeze_both(K, V, idx, W, Hq=Hkv)
+    _assert_cache_equal(ref, cache)
+
+
+def test_freeze_of_an_all_zero_group_and_clustered_vertical_rows():
+    B, Hkv, N, W = 1, 2, 700, 60
+    K, V = rand_bf16((B, Hkv, N, 128), 4), rand_bf16((B, Hkv, N, 128), 5)
+    K[:, :, 100:300] = 0
+    idx = np.tile(np.concatenate([np.arange(0, 40), np.arange(320, 330), np.arange(630, 640)]).astype(np.int32), (B, Hkv, 1))
+    ref, cache = _freeze_both(K, V, idx, W, Hq=Hkv)
+    assert (ref["kq_scales"] == 0).any()
+    _assert_cache_equal(ref, cache)
+
+
+DECODE_SHAPES = [  # B, Hq, Hkv, N, W, k, n_s, splits
+    (1, 4, 1, 300, 40, 9, 0, 1), (1, 4, 1, 300, 40, 9, 3, 0), (2, 8, 2, 1000, 128, 37, 5, 3), (1, 2, 2, 64, 0, 0, 1, 1),
+    (1, 8, 1, 129, 1, 64, 0, 2), (1, 6, 2, 50, 80, 0, 0, 0), (1, 4, 2, 200, 20, 180, 17, 4), (1, 16, 2, 2000, 100, 50, 128, 0),
+    (1, 5, 1, 777, 33, 21, 2, 7), (1, 4, 1, 40, 8, 3, 0, 50), (2, 32, 8, 4096, 512, 82, 16, 0), (1, 1, 1, 17, 16, 0, 0, 1),
+]
+
+
+@pytest.mark.parametrize("B,Hq,Hkv,N,W,kk,n_s,splits", DECODE_SHAPES)
+def test_decode_attention_matches_oracle(B, Hq, Hkv, N, W, kk, n_s, splits):
+    K, V = rand_bf16((B, Hkv, N, 128), 11, 1.3), rand_bf16((B, Hkv, N, 128), 12)
+    q = rand_bf16((B, Hq, 128), 13, 1.5)
+    idx = _idx(B, Hkv, N - min(W, N), kk, 14) if kk else None
+    ref, cache = _freeze_both(K, V, idx, W, Hq)
+    _stage(ref, cache, n_s, 100)
+    want, lse_want = od.decode_attention(wl.bits(q), ref)
+    lse = torch.empty(B, Hq, dtype=torch.float32, device="cuda")
+    got = dapi.hyq_hybrid_attention_decode(q.cuda(), cache, splits=splits, out_dtype=torch.float32, lse=lse)
+    torch.cuda.synchronize()
+    mx, rel = errors(got.cpu().numpy(), want)
+    assert mx <= MAX_ABS_TOL and rel <= MEAN_REL_TOL, (mx, rel)
+    assert np.abs(lse.cpu().numpy() - lse_want).max() <= 2e-3
+    got16 = dapi.hyq_hybrid_attention_decode(q.cuda(), cache, splits=splits, out_dtype=torch.bfloat16)
+    assert torch.equal(got16.cpu(), got.cpu().to(torch.bfloat16))
+
+
+def test_decode_with_peaked_scores_and_late_maxima():
+    """A planted key that dominates (scores far above the rest) sits late in the quantized prefix, another
+    in the window: the lazy reference maximum has to be raised mid-stream in several warps and slices."""
+    B, Hq, Hkv, N, W, kk = 1, 8, 2, 3000, 64, 30
+    K, V = rand_bf16((B, Hkv, N, 128), 21), rand_bf16((B, Hkv, N, 128), 22)
+    q = rand_bf16((B, Hq, 128), 23)
+    u = torch.nn.functional.normalize(torch.randn(128, generator=torch.Generator().manual_seed(24)), dim=0)
+    qf = q.float() + 6.0 * u
+    q = qf.to(torch.bfloat16)
+    for pos, amp in ((2500, 8.0), (N - 5, 10.0), (17, 5.0)):
+        K[:, :, pos] = (K[:, :, pos].float() + amp * u).to(torch.bfloat16)
+    idx = _idx(B, Hkv, N - W, kk, 25)
+    ref, cache = _freeze_both(K, V, idx, W, Hq)
+    want, _ = od.decode_attention(wl.bits(q), ref)
+    for splits in (1, 5, 0):
+        got = dapi.hyq_hybrid_attention_decode(q.cuda(), cache, splits=splits, out_dtype=torch.float32)
+        mx, rel = errors(got.cpu().numpy(), want)
+        assert mx <= MAX_ABS_TOL and rel <= MEAN_REL_TOL, (splits, mx, rel)
+
+
+def test_decode_at_benchmark_size_and_repeatable():
+    """The benchmark's cache shape (32 / 8 heads, 32768 frozen rows, 2 % vertical, window 1024, a full staging
+    buffer) at batch 2, every head against the oracle; two runs are bit-identical."""
+    B, Hq, Hkv, N, W = 2, 32, 8, 32768, 1024
+    kk = oracle_k = int(np.ceil((N - W) * 0.02))
+    K, V = rand_bf16((B, Hkv, N, 128), 31), rand_bf16((B, Hkv, N, 128), 32)
+    q = rand_bf16((B, Hq, 128), 33)
+    idx = _idx(B, Hkv, N - W, kk, 34)
+    ref, cache = _freeze_both(K, V, idx, W, Hq)
+    _assert_cache_equal(ref, cache)
+    _stage(ref, cache, 128, 300)
+    want, _ = od.decode_attention(wl.bits(q), ref)
+    got = dapi.hyq_hybrid_attention_decode(q.cuda(), cache, out_dtype=torch.float32)
+    again = dapi.hyq_hybrid_attention_decode(q.cuda(), cache, out_dtype=torch.float32)
+    mx, rel = errors(got.cpu().numpy(), want)
+    assert mx <= MAX_ABS_TOL and rel <= MEAN_REL_TOL, (mx, rel)
+    assert torch.equal(got, again)
+    assert oracle_k == cache.desc.k
