@@ -367,6 +367,105 @@ def run_query_block(args, w: wl.Workload):
         "clocks": clocks}))
 
 
+def run_decode(args, w: wl.Workload):
+    """`--decode`: the decode side on the same cache shape.  Freeze (Algorithm 4) builds the hybrid K4V4 cache
+    of `--batch` sequences from a synthetic prefill cache (vertical sets from Algorithm 1 on the first query head
+    of every KV group), the staging buffer is filled, and the timed step is one hyq_hybrid_attention_decode call
+    (Algorithm 3: slice kernel + merge kernel) for one new token per sequence, over cache replicas used
+    round-robin so that no call finds its cache in L2.  One JSON line; one GPU."""
+    from paper_2608_27875_b200 import api, build, decode_api as dapi
+    build.build()
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    w = w.scaled(B=args.batch)
+    g = w.Hq // w.Hkv
+    Q, K, V = wl.make_inputs(w)
+    K, V = K.to(dev), V.to(dev)
+    q_tail = Q[:, ::g].contiguous().to(dev)                 # Algorithm 1 with H = H_KV heads
+    idx = api.hyq_select_vertical(q_tail, K, w.window, w.k)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    cache = dapi.hyq_freeze(K, V, idx, w.window, w.Hq, staging_capacity=args.staging)
+    torch.cuda.synchronize()
+    e0.record()
+    dapi.hyq_freeze(K, V, idx, w.window, w.Hq, staging_capacity=args.staging, cache=cache)
+    e1.record()
+    torch.cuda.synchronize()
+    freeze_ms = e0.elapsed_time(e1)
+    gen = torch.Generator(device=dev).manual_seed(w.seed + 5)
+    new_rows = [(torch.randn(w.B, w.Hkv, w.D, device=dev, generator=gen).to(torch.bfloat16),
+                 torch.randn(w.B, w.Hkv, w.D, device=dev, generator=gen).to(torch.bfloat16)) for _ in range(args.staging)]
+    # Replicas of the cache at different addresses, used round-robin: a call never finds its cache in L2
+    # (more than three L2 sizes of other replicas are read in between) and no flush kernel dirties L2
+    # right before a timed call.
+    by = cache.bytes_read_per_token()
+    n_rep = 1 + int(np.ceil(3 * 126e6 / by))
+    caches = [cache] + [dapi.hyq_freeze(K, V, idx, w.window, w.Hq, staging_capacity=args.staging) for _ in range(n_rep - 1)]
+    for c in caches:
+        for kn, vn in new_rows:
+            c.append(kn, vn)
+    q = Q[:, :, -1].contiguous().to(dev)
+    out = torch.empty(w.B, w.Hq, w.D, dtype=torch.bfloat16, device=dev)
+    ws = torch.empty(max(16, dapi.hyq_hybrid_attention_decode_workspace(cache, args.splits)), dtype=torch.uint8, device=dev)
+    call = lambda i: dapi.hyq_hybrid_attention_decode(q, caches[i % n_rep], splits=args.splits, out=out, workspace=ws)   # noqa: E731
+    for i in range(max(3, args.warmup)):
+        call(i)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(0)
+    sampler.start()
+    e0.record()
+    for i in range(args.steps):
+        call(i)
+    e1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1) / args.steps
+    # end to end: the token's query from pinned host memory, the output back to the host, every step
+    q_host, out_host = q.cpu().pin_memory(), torch.empty(out.shape, dtype=out.dtype).pin_memory()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for i in range(args.steps):
+        q.copy_(q_host, non_blocking=True)
+        call(i)
+        out_host.copy_(out, non_blocking=True)
+        torch.cuda.synchronize()
+    e2e_ms = (time.perf_counter() - t0) / args.steps * 1e3
+    cache = caches[(args.steps - 1) % n_rep]
+    by = cache.bytes_read_per_token()
+    peaks = measured_peaks()
+    rows = w.L + args.staging
+    # CPU baseline: the oracle on one sequence's cache (Freeze + one token), all heads
+    import oracle
+    from oracle import decode as od
+    kb, vb = wl.bits(K[:1].cpu()), wl.bits(V[:1].cpu())
+    ref = od.freeze(kb, vb, idx[:1].cpu().numpy(), w.window, staging_capacity=args.staging)
+    for kn, vn in new_rows:
+        od.append_staging(ref, wl.bits(kn[:1].cpu()), wl.bits(vn[:1].cpu()))
+    t0 = time.perf_counter()
+    want, _ = od.decode_attention(wl.bits(q[:1].cpu()), ref)
+    cpu_s = time.perf_counter() - t0
+    err = np.abs(out[:1].float().cpu().numpy() - want)
+    print(json.dumps({
+        "metric": "hybrid decode attention latency per token step", "value": ms * 1e3, "unit": "us", "n_gpus": 1,
+        "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": False,
+        "scaling": "weak", "vs_baseline": None,
+        "dtype": "int4 codes -> fp16 in registers, fp16 / bf16 mma.sync with f32 accumulation", "data": "synthetic",
+        "config": {"workload": f"{w.name} cache shape, decode of one token per sequence", "B": w.B, "Hq": w.Hq,
+                   "Hkv": w.Hkv, "N": w.L, "D": w.D, "window": w.window, "k": w.k, "staging_rows": args.staging,
+                   "format": "K4V4, group 64", "splits": args.splits, "cached_rows_per_head": rows,
+                   "l2": f"{n_rep} cache replicas used round-robin ({by * (n_rep - 1) / 1e6:.0f} MB read between reuses)",
+                   "freeze_ms": freeze_ms},
+        "roofline": {"bound": "hbm", "kernel": "decode_kernel + decode_merge_kernel (one call)",
+                     "achieved": by / (ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": by / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES.get("decode"),
+                     "bytes_per_call": by, "peak_source": peaks["source"]},
+        "cpu_baseline": {"value": cpu_s * 1e6 * w.B, "unit": "us", "cores": oracle.num_threads(), "kind": "oracle",
+                         "sample": "oracle attention of one sequence (all heads) timed, scaled by the batch size"},
+        "e2e": {"value": e2e_ms * 1e3, "unit": "us", "h2d_bytes_per_step": q_host.numel() * 2,
+                "d2h_bytes_per_step": out_host.numel() * 2},
+        "check": {"max_abs_err_vs_oracle_seq0": float(err.max())},
+        "gpu_launches": 2 * args.steps, "clocks": clocks}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -378,6 +477,10 @@ def main():
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of oracle time for cpu_baseline")
     ap.add_argument("--lq", type=int, default=0, help="measure a query block of the last LQ rows against the full K, V")
     ap.add_argument("--fixed-tail", action="store_true", help="with --lq: Algorithm 2's fixed tail window")
+    ap.add_argument("--decode", action="store_true", help="measure the decode side (Freeze + one-token attention)")
+    ap.add_argument("--batch", type=int, default=8, help="with --decode: sequences in the batch")
+    ap.add_argument("--staging", type=int, default=128, help="with --decode: staged rows (W_s, all filled)")
+    ap.add_argument("--splits", type=int, default=0, help="with --decode: slices per KV head (0 = library's choice)")
     ap.add_argument("--formats", default="", choices=["", *sorted(FORMAT_SETS)],
                     help="override the workload's (Q, K, V) low-bit formats (default: as the workload defines them)")
     args = ap.parse_args()
@@ -393,6 +496,9 @@ def main():
         return
     if args.lq:
         run_query_block(args, w)
+        return
+    if args.decode:
+        run_decode(args, w)
         return
 
     import ctypes

@@ -100,7 +100,7 @@ int hyq_freeze(const void* k_, const void* v, const int32_t* vl_idx, const hyq_k
  *
  *   q [B,Hq,D] bf16 (device).  out [B,Hq,D]: bf16 (out_dtype 0) or fp32 (1).  lse: optional [B,Hq] fp32,
  *   natural-log-sum-exp of the scaled scores (NULL to skip).  softmax_scale 0 => 1/sqrt(D).
- *   splits: S >= 1, or 0 for a choice that fills the GPU.  workspace: hyq_hybrid_attention_decode_workspace
+ *   splits: 1 <= S <= 1024, or 0 for a choice that fills the GPU.  workspace: hyq_hybrid_attention_decode_workspace
  *   bytes (the slices' partial results).  The cache must hold at least one row in total.
  *   Errors: as hyq_freeze, plus WORKSPACE.
  * ------------------------------------------------------------------------------------------- */

@@ -54,7 +54,7 @@ int hyq_freeze(const void* k_, const void* v, const int32_t* vl_idx, const hyq_k
 }
 
 int hyq_hybrid_attention_decode_workspace(const hyq_kv_cache* cache, int splits, size_t* bytes) {
-    if (!bytes || splits < 0) return HYQ_ERR_INVALID_ARG;
+    if (!bytes || splits < 0 || splits > 1024) return HYQ_ERR_INVALID_ARG;
     const int rc = check_cache(cache, false);
     if (rc != HYQ_OK) return rc;
     *bytes = decode_workspace_bytes(*cache, splits > 0 ? splits : decode_auto_splits(*cache));
@@ -65,7 +65,7 @@ int hyq_hybrid_attention_decode(const void* q, const hyq_kv_cache* cache, float 
                                 void* out, float* lse, void* workspace, size_t workspace_bytes, void* stream) {
     const int rc = check_cache(cache, true);
     if (rc != HYQ_OK) return rc;
-    if (!q || !out || !workspace || splits < 0 || splits > 65535) return HYQ_ERR_INVALID_ARG;
+    if (!q || !out || !workspace || splits < 0 || splits > 1024) return HYQ_ERR_INVALID_ARG;
     if (out_dtype != 0 && out_dtype != 1) return HYQ_ERR_INVALID_ARG;
     if (!aligned16(q) || !aligned16(out) || !aligned16(workspace)) return HYQ_ERR_ALIGNMENT;
     const int s = splits > 0 ? splits : decode_auto_splits(*cache);

@@ -16,7 +16,7 @@
 // each lane takes whatever channels arrive in its own 16-byte loads; P^T's operand layout is the transpose
 // of S^T's accumulator layout, which `movmatrix` provides for 8x8 b16 blocks.  V's codes are stored by
 // Freeze in exactly the operand order (see hyq_decode.h), K's stay row-major.  INT4 -> fp16 is one LOP3
-// (nibble ^ 8 | 0x6400 = 1032 + code) and one packed subtract for two codes.
+// (nibble ^ 8 | 0x6400 = 1032 + code) and one packed subtract or fma for two codes.
 // The bf16 segments (vertical rows, staging, window) go through the same two products with bf16 operands;
 // there V^T's key pairs are formed from two rows' words with byte permutes.
 //
@@ -34,6 +34,10 @@ namespace hyq {
 
 constexpr int DEC_THREADS = 128;
 constexpr int DEC_WARPS = DEC_THREADS / 32;
+#ifndef DEC_CTAS_PER_SM
+#define DEC_CTAS_PER_SM 4                   // resident CTAs per SM the register budget is set for
+#endif
+constexpr int DEC_FP_COST = 4;              // bytes of a bf16 tile over bytes of an INT4 tile
 constexpr float DEC_RAISE = 8.0f;          // log2 units; P <= 2^8 stays far inside fp16 / bf16 range
 
 struct DecParams {
@@ -66,11 +70,20 @@ __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
     asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
     return d;
 }
-// two INT4 codes (two's complement nibbles at bits 0-3 and 16-19 of w) -> packed fp16 values
-__device__ __forceinline__ uint32_t dq4(uint32_t w) {
+// Two INT4 codes (two's complement nibbles) -> packed fp16 values, without unpacking shifts where possible:
+// dq4_lo takes the nibbles at bits 0-3 / 16-19: (w & 0x000F000F) ^ 0x64086408 is fp16 1032 + code, minus 1032;
+// dq4_hi takes the nibbles at bits 4-7 / 20-23: (w & 0x00F000F0) ^ 0x64806480 is fp16 16 * (72 + code), so one
+// packed fma (x / 16 - 72) finishes it.  Both are exact.
+__device__ __forceinline__ uint32_t dq4_lo(uint32_t w) {
     uint32_t h;
-    asm("lop3.b32 %0, %1, 0x000F000F, 0x64086408, 0x6A;" : "=r"(h) : "r"(w));      // (w & mask) ^ magic = 1032 + code
+    asm("lop3.b32 %0, %1, 0x000F000F, 0x64086408, 0x6A;" : "=r"(h) : "r"(w));
     asm("sub.rn.f16x2 %0, %1, %2;" : "=r"(h) : "r"(h), "r"(0x64086408u));
+    return h;
+}
+__device__ __forceinline__ uint32_t dq4_hi(uint32_t w) {
+    uint32_t h;
+    asm("lop3.b32 %0, %1, 0x00F000F0, 0x64806480, 0x6A;" : "=r"(h) : "r"(w));
+    asm("fma.rn.f16x2 %0, %1, %2, %3;" : "=r"(h) : "r"(h), "r"(0x2C002C00u), "r"(0xD480D480u));
     return h;
 }
 __device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
@@ -122,7 +135,7 @@ __device__ __forceinline__ void softmax_tile(SoftmaxState& st, float (&acc)[8][4
     st.l1 += p[1] + p[3];
 }
 
-__global__ void __launch_bounds__(DEC_THREADS, 4)
+__global__ void __launch_bounds__(DEC_THREADS, DEC_CTAS_PER_SM)
 decode_kernel(const DecParams p) {
     const int split = blockIdx.x;
     const long unit = blockIdx.y;
@@ -142,8 +155,12 @@ decode_kernel(const DecParams p) {
 
     const long Tq = (p.nQ + 15) / 16;
     const int Tvl = (p.k + 15) / 16, Ts = (p.n_s + 15) / 16, Tw = (p.W + 15) / 16;
-    const long T = Tq + Tvl + Ts + Tw;
-    const long lo = T * split / p.splits, hi = T * (split + 1) / p.splits;
+    // The slices are equal in BYTES, not tiles: a bf16 tile moves four times what an INT4 tile moves.
+    const long Tf = Tvl + Ts + Tw, cost = Tq + DEC_FP_COST * Tf;
+    const long ca = cost * split / p.splits, cb = cost * (split + 1) / p.splits;
+    const long q_lo = ca < Tq ? ca : Tq, q_hi = cb < Tq ? cb : Tq;
+    const long f_lo = Tq + (ca > Tq ? (ca - Tq + DEC_FP_COST - 1) / DEC_FP_COST : 0);
+    const long f_hi = Tq + (cb > Tq ? (cb - Tq + DEC_FP_COST - 1) / DEC_FP_COST : 0);
 
     SoftmaxState st = {-INFINITY, -INFINITY, 0.0f, 0.0f};
     float acc[8][4];
@@ -151,8 +168,7 @@ decode_kernel(const DecParams p) {
     for (int x = 0; x < 8; ++x) acc[x][0] = acc[x][1] = acc[x][2] = acc[x][3] = 0.0f;
 
     // ---------------- quantized prefix ----------------
-    const long q_hi = hi < Tq ? hi : Tq;
-    if (lo + warp < q_hi) {
+    if (q_lo + warp < q_hi) {
         uint32_t qf[16];                                   // q^T operand, fp16: k-step c -> qf[2c], qf[2c+1]
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
@@ -169,7 +185,7 @@ decode_kernel(const DecParams p) {
         const float* ks = p.ks + unit * (p.nQp / 64);
         const float* vs = p.vs + unit * (p.nQp / 64);
 
-        long t = lo + warp;
+        long t = q_lo + warp;
         uint4 ka = __ldg(kq + (t * 16 + r) * 4 + j), kb = __ldg(kq + (t * 16 + r + 8) * 4 + j);
         uint4 va = __ldg(vq + t * 64 + lane * 2), vb = __ldg(vq + t * 64 + lane * 2 + 1);
         float fk = __ldg(ks + (t >> 2)), fv = __ldg(vs + (t >> 2));
@@ -183,30 +199,32 @@ decode_kernel(const DecParams p) {
 #pragma unroll
             for (int c = 0; c < 8; ++c) {
                 const uint32_t wa = word_of(ka, c >> 1) >> (8 * (c & 1)), wb = word_of(kb, c >> 1) >> (8 * (c & 1));
-                mma_f16(c4, dq4(wa), dq4(wb), dq4(wa >> 4), dq4(wb >> 4), qf[2 * c], qf[2 * c + 1]);
+                mma_f16(c4, dq4_lo(wa), dq4_lo(wb), dq4_hi(wa), dq4_hi(wb), qf[2 * c], qf[2 * c + 1]);
             }
             const float f = fk * p.scale_log2;
             const long row = t * 16 + r;
             float s[4], pw[4];
-            s[0] = row < p.nQ ? c4[0] * f : -INFINITY;     s[1] = row < p.nQ ? c4[1] * f : -INFINITY;
-            s[2] = row + 8 < p.nQ ? c4[2] * f : -INFINITY; s[3] = row + 8 < p.nQ ? c4[3] * f : -INFINITY;
+            s[0] = c4[0] * f; s[1] = c4[1] * f; s[2] = c4[2] * f; s[3] = c4[3] * f;
+            if (t * 16 + 16 > p.nQ) {                       // ragged last tile of the prefix (warp-uniform)
+                if (row >= p.nQ) s[0] = s[1] = -INFINITY;
+                if (row + 8 >= p.nQ) s[2] = s[3] = -INFINITY;
+            }
             softmax_tile(st, acc, s, pw);
             const uint32_t b0 = movmatrix_trans(pack_f16(pw[0] * fv, pw[1] * fv));
             const uint32_t b1 = movmatrix_trans(pack_f16(pw[2] * fv, pw[3] * fv));
 #pragma unroll
             for (int x = 0; x < 8; ++x) {
                 const uint32_t w = word_of(x < 4 ? va : vb, x & 3);
-                mma_f16(acc[x], dq4(w), dq4(w >> 4), dq4(w >> 8), dq4(w >> 12), b0, b1);
+                mma_f16(acc[x], dq4_lo(w), dq4_hi(w), dq4_lo(w >> 8), dq4_hi(w >> 8), b0, b1);
             }
             ka = nka; kb = nkb; va = nva; vb = nvb; fk = nfk; fv = nfv;
         }
     }
 
     // ---------------- bf16 segments: vertical rows, staging, window ----------------
-    long f_lo = lo > Tq ? lo : Tq;
     // keep the round-robin phase of the tile list so that the warps stay balanced across the boundary
-    long t = f_lo + ((warp - (f_lo - lo)) % DEC_WARPS + DEC_WARPS) % DEC_WARPS;
-    if (t < hi) {
+    long t = f_lo + ((warp - (q_hi - q_lo)) % DEC_WARPS + DEC_WARPS) % DEC_WARPS;
+    if (t < f_hi) {
         uint32_t qb[16];                                   // q^T operand, bf16
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
@@ -214,7 +232,7 @@ decode_kernel(const DecParams p) {
             qb[2 * c] = *reinterpret_cast<const uint32_t*>(&qs[r][base]);
             qb[2 * c + 1] = *reinterpret_cast<const uint32_t*>(&qs[r][base + 2]);
         }
-        for (; t < hi; t += DEC_WARPS) {
+        for (; t < f_hi; t += DEC_WARPS) {
             long u = t - Tq;
             const uint4 *kseg, *vseg;
             int n;
@@ -226,19 +244,19 @@ decode_kernel(const DecParams p) {
             uint4 ka[4], kb[4];
 #pragma unroll
             for (int i = 0; i < 4; ++i) { ka[i] = __ldg(kseg + (long)ra * 16 + 4 * i + j); kb[i] = __ldg(kseg + (long)rb * 16 + 4 * i + j); }
-            uint4 vv[4][2];
-#pragma unroll
-            for (int sIdx = 0; sIdx < 4; ++sIdx) {
-                const int key = min(row0 + 2 * j + (sIdx & 1) + 8 * (sIdx >> 1), n - 1);
-                vv[sIdx][0] = __ldg(vseg + (long)key * 16 + r);
-                vv[sIdx][1] = __ldg(vseg + (long)key * 16 + 8 + r);
-            }
             float c4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
 #pragma unroll
             for (int c = 0; c < 8; ++c) {
                 const int wd = 2 * (c & 1);
                 mma_bf16(c4, word_of(ka[c >> 1], wd), word_of(kb[c >> 1], wd), word_of(ka[c >> 1], wd + 1),
                          word_of(kb[c >> 1], wd + 1), qb[2 * c], qb[2 * c + 1]);
+            }
+            uint4 vv[4][2];
+#pragma unroll
+            for (int sIdx = 0; sIdx < 4; ++sIdx) {
+                const int key = min(row0 + 2 * j + (sIdx & 1) + 8 * (sIdx >> 1), n - 1);
+                vv[sIdx][0] = __ldg(vseg + (long)key * 16 + r);
+                vv[sIdx][1] = __ldg(vseg + (long)key * 16 + 8 + r);
             }
             float s[4], pw[4];
             s[0] = row0 + r < n ? c4[0] * p.scale_log2 : -INFINITY;     s[1] = row0 + r < n ? c4[1] * p.scale_log2 : -INFINITY;
@@ -295,28 +313,47 @@ decode_kernel(const DecParams p) {
     }
 }
 
-// ReduceSoftmax of Algorithm 3 over the slices; one CTA per (b, kv head), one thread per channel.
+// ReduceSoftmax of Algorithm 3 over the slices; one CTA per (b, kv head, query head), one thread per channel.
+// The slices' (m, l) pairs are staged in shared memory first so that the channel loop is a run of
+// independent loads (the kernel is pure latency otherwise: it moves a few hundred KB).
+constexpr int DEC_MAX_SPLITS = 1024;
 __global__ void __launch_bounds__(HYQ_D)
 decode_merge_kernel(const float* __restrict__ part_acc, const float* __restrict__ part_ml, int g, int splits,
                     int out_fp32, void* __restrict__ out, float* __restrict__ lse) {
     const long unit = blockIdx.x;
-    for (int h = 0; h < g; ++h) {
-        float M = -INFINITY;
-        for (int s = 0; s < splits; ++s) M = fmaxf(M, __ldg(part_ml + ((unit * splits + s) * DEC_MAX_GROUP + h) * 2));
-        float L = 0.0f, A = 0.0f;
-        for (int s = 0; s < splits; ++s) {
-            const long slot = (unit * splits + s) * DEC_MAX_GROUP + h;
-            const float ms = __ldg(part_ml + slot * 2);
-            const float wt = ms == -INFINITY ? 0.0f : ex2(ms - M);
-            L += __ldg(part_ml + slot * 2 + 1) * wt;
-            A += __ldg(part_acc + slot * HYQ_D + threadIdx.x) * wt;
-        }
-        const float o = A / L;
-        const long oi = (unit * g + h) * HYQ_D + threadIdx.x;
-        if (out_fp32) static_cast<float*>(out)[oi] = o;
-        else static_cast<__nv_bfloat16*>(out)[oi] = __float2bfloat16_rn(o);
-        if (lse && threadIdx.x == 0) lse[unit * g + h] = (M + log2f(L)) * 0.6931471805599453f;
+    const int h = blockIdx.y;
+    __shared__ float wt[DEC_MAX_SPLITS];
+    __shared__ float red[2][HYQ_D / 32];
+    const long slot0 = unit * splits * DEC_MAX_GROUP + h;          // slice s sits at slot0 + s * DEC_MAX_GROUP
+    float M = -INFINITY;
+    for (int s = threadIdx.x; s < splits; s += HYQ_D) {
+        wt[s] = __ldg(part_ml + (slot0 + (long)s * DEC_MAX_GROUP) * 2);
+        M = fmaxf(M, wt[s]);
     }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+    if ((threadIdx.x & 31) == 0) red[0][threadIdx.x >> 5] = M;
+    __syncthreads();
+    M = fmaxf(fmaxf(red[0][0], red[0][1]), fmaxf(red[0][2], red[0][3]));
+    float L = 0.0f;
+    for (int s = threadIdx.x; s < splits; s += HYQ_D) {
+        const float w = wt[s] == -INFINITY ? 0.0f : ex2(wt[s] - M);
+        L += __ldg(part_ml + (slot0 + (long)s * DEC_MAX_GROUP) * 2 + 1) * w;
+        wt[s] = w;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) L += __shfl_xor_sync(0xffffffffu, L, o);
+    if ((threadIdx.x & 31) == 0) red[1][threadIdx.x >> 5] = L;
+    __syncthreads();
+    L = (red[1][0] + red[1][1]) + (red[1][2] + red[1][3]);
+    float A = 0.0f;
+#pragma unroll 8
+    for (int s = 0; s < splits; ++s) A += __ldg(part_acc + (slot0 + (long)s * DEC_MAX_GROUP) * HYQ_D + threadIdx.x) * wt[s];
+    const float o = A / L;
+    const long oi = (unit * g + h) * HYQ_D + threadIdx.x;
+    if (out_fp32) static_cast<float*>(out)[oi] = o;
+    else static_cast<__nv_bfloat16*>(out)[oi] = __float2bfloat16_rn(o);
+    if (lse && threadIdx.x == 0) lse[unit * g + h] = (M + log2f(L)) * 0.6931471805599453f;
 }
 
 static long decode_tiles(const hyq_kv_cache& c) {
@@ -327,10 +364,10 @@ static long decode_tiles(const hyq_kv_cache& c) {
 int decode_auto_splits(const hyq_kv_cache& c) {
     const long units = (long)c.B * c.Hkv;
     const long T = decode_tiles(c);
-    long s = (148L * 4 + units - 1) / units;            // about four CTAs per SM
-    const long cap = T / 8 > 1 ? T / 8 : 1;             // at least two tiles per warp
+    long s = 148L * DEC_CTAS_PER_SM / units;            // one full wave of resident CTAs, never a second partial one
+    const long cap = T / 8 > 1 ? T / 8 : 1;             // at least two tiles per warp on average
     if (s > cap) s = cap;
-    if (s > 64) s = 64;
+    if (s > 64) s = 64;                                 // DEC_MAX_SPLITS bounds explicit requests
     return (int)(s < 1 ? 1 : s);
 }
 
@@ -357,7 +394,7 @@ int launch_decode(const void* q, const hyq_kv_cache& c, float alpha, int splits,
     p.part_acc = static_cast<float*>(workspace);
     p.part_ml = reinterpret_cast<float*>(static_cast<char*>(workspace) + align_up(slots * HYQ_D * sizeof(float), 16));
     decode_kernel<<<dim3((unsigned)splits, (unsigned)units), DEC_THREADS, 0, st>>>(p);
-    decode_merge_kernel<<<(unsigned)units, HYQ_D, 0, st>>>(p.part_acc, p.part_ml, p.g, splits, out_dtype, out, lse);
+    decode_merge_kernel<<<dim3((unsigned)units, (unsigned)p.g), HYQ_D, 0, st>>>(p.part_acc, p.part_ml, p.g, splits, out_dtype, out, lse);
     return launch_status();
 }
 
