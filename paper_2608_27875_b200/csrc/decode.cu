@@ -111,28 +111,74 @@ struct SoftmaxState {
     float m0, m1, l0, l1;      // heads 2j and 2j+1 of this lane: reference maximum (log2 units), partial row sum
 };
 
-// One tile's scores (keys r and r+8, heads 2j and 2j+1; log2 units, masked = -inf) -> weights p[4].
-// Raises the reference maxima and rescales the accumulators only when some score is far above them.
-__device__ __forceinline__ void softmax_tile(SoftmaxState& st, float (&acc)[8][4], const float (&s)[4], float (&p)[4]) {
-    const bool far = fmaxf(s[0], s[2]) > st.m0 + DEC_RAISE || fmaxf(s[1], s[3]) > st.m1 + DEC_RAISE;
+// One tile's raw scores c4 (keys r and r+8, heads 2j and 2j+1) times f (log2 units) -> weights p[4].
+// MASKED: rows flagged invalid (past the end of a segment) get weight zero.  The reference maxima are raised,
+// and the accumulators rescaled, only when some score is more than 2^DEC_RAISE above them (warp vote).
+template <bool MASKED>
+__device__ __forceinline__ void softmax_tile(SoftmaxState& st, float (&acc)[8][4], const float (&c4)[4], float f,
+                                             bool valid_a, bool valid_b, float (&p)[4]) {
+    float d0 = fmaf(c4[0], f, -st.m0), d2 = fmaf(c4[2], f, -st.m0);
+    float d1 = fmaf(c4[1], f, -st.m1), d3 = fmaf(c4[3], f, -st.m1);
+    if (MASKED) {
+        if (!valid_a) d0 = d1 = -INFINITY;
+        if (!valid_b) d2 = d3 = -INFINITY;
+    }
+    const bool far = fmaxf(d0, d2) > DEC_RAISE || fmaxf(d1, d3) > DEC_RAISE;
     if (__any_sync(0xffffffffu, far)) {
-        float t0 = fmaxf(s[0], s[2]), t1 = fmaxf(s[1], s[3]);
+        float s0 = c4[0] * f, s1 = c4[1] * f, s2 = c4[2] * f, s3 = c4[3] * f;
+        if (MASKED) {
+            if (!valid_a) s0 = s1 = -INFINITY;
+            if (!valid_b) s2 = s3 = -INFINITY;
+        }
+        float t0 = fmaxf(s0, s2), t1 = fmaxf(s1, s3);
 #pragma unroll
         for (int o = 4; o < 32; o <<= 1) {
             t0 = fmaxf(t0, __shfl_xor_sync(0xffffffffu, t0, o));
             t1 = fmaxf(t1, __shfl_xor_sync(0xffffffffu, t1, o));
         }
-        const float n0 = fmaxf(st.m0, t0), n1 = fmaxf(st.m1, t1);
-        const float c0 = n0 == -INFINITY ? 1.0f : ex2(st.m0 - n0), c1 = n1 == -INFINITY ? 1.0f : ex2(st.m1 - n1);
+        const float n0 = fmaxf(st.m0, t0), n1 = fmaxf(st.m1, t1);      // finite: every tile has a valid row
+        const float c0 = ex2(st.m0 - n0), c1 = ex2(st.m1 - n1);        // 0 on the first tile (m = -inf)
         st.m0 = n0; st.m1 = n1;
         st.l0 *= c0; st.l1 *= c1;
 #pragma unroll
         for (int x = 0; x < 8; ++x) { acc[x][0] *= c0; acc[x][2] *= c0; acc[x][1] *= c1; acc[x][3] *= c1; }
+        d0 = s0 - n0; d2 = s2 - n0; d1 = s1 - n1; d3 = s3 - n1;
     }
-    p[0] = ex2(s[0] - st.m0); p[2] = ex2(s[2] - st.m0);
-    p[1] = ex2(s[1] - st.m1); p[3] = ex2(s[3] - st.m1);
+    p[0] = ex2(d0); p[1] = ex2(d1); p[2] = ex2(d2); p[3] = ex2(d3);
     st.l0 += p[0] + p[2];
     st.l1 += p[1] + p[3];
+}
+
+// One 16-row tile of the quantized prefix as it sits in registers: K rows r and r+8 (this lane's 16 bytes each),
+// the lane's 32 bytes of the V tile, and the group's two scales.
+struct QTile {
+    uint4 ka, kb, va, vb;
+    float fk, fv;
+};
+__device__ __forceinline__ void load_qtile(QTile& d, const uint4* pk, const uint4* pv, const float* pks, const float* pvs) {
+    d.ka = __ldg(pk); d.kb = __ldg(pk + 32);
+    d.va = __ldg(pv); d.vb = __ldg(pv + 1);
+    d.fk = __ldg(pks); d.fv = __ldg(pvs);
+}
+
+template <bool RAGGED>
+__device__ __forceinline__ void quant_tile(const QTile& d, const uint32_t (&qf)[16], float scale_log2, int rows_valid, int r,
+                                           SoftmaxState& st, float (&acc)[8][4]) {
+    float c4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+        const uint32_t wa = word_of(d.ka, c >> 1) >> (8 * (c & 1)), wb = word_of(d.kb, c >> 1) >> (8 * (c & 1));
+        mma_f16(c4, dq4_lo(wa), dq4_lo(wb), dq4_hi(wa), dq4_hi(wb), qf[2 * c], qf[2 * c + 1]);
+    }
+    float pw[4];
+    softmax_tile<RAGGED>(st, acc, c4, d.fk * scale_log2, r < rows_valid, r + 8 < rows_valid, pw);
+    const uint32_t b0 = movmatrix_trans(pack_f16(pw[0] * d.fv, pw[1] * d.fv));
+    const uint32_t b1 = movmatrix_trans(pack_f16(pw[2] * d.fv, pw[3] * d.fv));
+#pragma unroll
+    for (int x = 0; x < 8; ++x) {
+        const uint32_t w = word_of(x < 4 ? d.va : d.vb, x & 3);
+        mma_f16(acc[x], dq4_lo(w), dq4_hi(w), dq4_lo(w >> 8), dq4_hi(w >> 8), b0, b1);
+    }
 }
 
 __global__ void __launch_bounds__(DEC_THREADS, DEC_CTAS_PER_SM)
@@ -180,45 +226,33 @@ decode_kernel(const DecParams p) {
             qf[2 * c] = *reinterpret_cast<const uint32_t*>(&h0);
             qf[2 * c + 1] = *reinterpret_cast<const uint32_t*>(&h1);
         }
-        const uint4* kq = reinterpret_cast<const uint4*>(p.kq + unit * p.nQp * 64);
-        const uint4* vq = reinterpret_cast<const uint4*>(p.vq + unit * (p.nQp / 16) * DEC_VTILE_BYTES);
-        const float* ks = p.ks + unit * (p.nQp / 64);
-        const float* vs = p.vs + unit * (p.nQp / 64);
-
-        long t = q_lo + warp;
-        uint4 ka = __ldg(kq + (t * 16 + r) * 4 + j), kb = __ldg(kq + (t * 16 + r + 8) * 4 + j);
-        uint4 va = __ldg(vq + t * 64 + lane * 2), vb = __ldg(vq + t * 64 + lane * 2 + 1);
-        float fk = __ldg(ks + (t >> 2)), fv = __ldg(vs + (t >> 2));
-        for (; t < q_hi; t += DEC_WARPS) {
-            const long tn = t + DEC_WARPS < q_hi ? t + DEC_WARPS : t;      // prefetch (the last one re-reads itself)
-            const uint4 nka = __ldg(kq + (tn * 16 + r) * 4 + j), nkb = __ldg(kq + (tn * 16 + r + 8) * 4 + j);
-            const uint4 nva = __ldg(vq + tn * 64 + lane * 2), nvb = __ldg(vq + tn * 64 + lane * 2 + 1);
-            const float nfk = __ldg(ks + (tn >> 2)), nfv = __ldg(vs + (tn >> 2));
-
-            float c4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-#pragma unroll
-            for (int c = 0; c < 8; ++c) {
-                const uint32_t wa = word_of(ka, c >> 1) >> (8 * (c & 1)), wb = word_of(kb, c >> 1) >> (8 * (c & 1));
-                mma_f16(c4, dq4_lo(wa), dq4_lo(wb), dq4_hi(wa), dq4_hi(wb), qf[2 * c], qf[2 * c + 1]);
-            }
-            const float f = fk * p.scale_log2;
-            const long row = t * 16 + r;
-            float s[4], pw[4];
-            s[0] = c4[0] * f; s[1] = c4[1] * f; s[2] = c4[2] * f; s[3] = c4[3] * f;
-            if (t * 16 + 16 > p.nQ) {                       // ragged last tile of the prefix (warp-uniform)
-                if (row >= p.nQ) s[0] = s[1] = -INFINITY;
-                if (row + 8 >= p.nQ) s[2] = s[3] = -INFINITY;
-            }
-            softmax_tile(st, acc, s, pw);
-            const uint32_t b0 = movmatrix_trans(pack_f16(pw[0] * fv, pw[1] * fv));
-            const uint32_t b1 = movmatrix_trans(pack_f16(pw[2] * fv, pw[3] * fv));
-#pragma unroll
-            for (int x = 0; x < 8; ++x) {
-                const uint32_t w = word_of(x < 4 ? va : vb, x & 3);
-                mma_f16(acc[x], dq4_lo(w), dq4_hi(w), dq4_lo(w >> 8), dq4_hi(w >> 8), b0, b1);
-            }
-            ka = nka; kb = nkb; va = nva; vb = nvb; fk = nfk; fv = nfv;
+        // this warp's tiles: t0, t0 + 4, ...; pointers advance by constants, two register sets alternate so
+        // that the next tile's loads are in flight while the current one is processed
+        const long t0 = q_lo + warp;
+        const int n_my = (int)((q_hi - t0 + DEC_WARPS - 1) / DEC_WARPS);
+        const bool has_ragged = (p.nQ & 15) && t0 + (long)(n_my - 1) * DEC_WARPS == Tq - 1;
+        const int n_loop = n_my - (has_ragged ? 1 : 0);
+        const uint4* pk = reinterpret_cast<const uint4*>(p.kq + unit * p.nQp * 64) + (t0 * 16 + r) * 4 + j;
+        const uint4* pv = reinterpret_cast<const uint4*>(p.vq + unit * (p.nQp / 16) * DEC_VTILE_BYTES) + t0 * 64 + lane * 2;
+        const float* pks = p.ks + unit * (p.nQp / 64) + (t0 >> 2);
+        const float* pvs = p.vs + unit * (p.nQp / 64) + (t0 >> 2);
+        auto advance = [&]() { pk += DEC_WARPS * 64; pv += DEC_WARPS * 64; ++pks; ++pvs; };
+        QTile A, B;
+        load_qtile(A, pk, pv, pks, pvs);
+        B = A;
+        advance();
+        int i = 0;
+        for (;;) {
+            if (i + 1 < n_my) { load_qtile(B, pk, pv, pks, pvs); advance(); }
+            if (i >= n_loop) break;
+            quant_tile<false>(A, qf, p.scale_log2, 16, r, st, acc);
+            ++i;
+            if (i + 1 < n_my) { load_qtile(A, pk, pv, pks, pvs); advance(); }
+            if (i >= n_loop) break;
+            quant_tile<false>(B, qf, p.scale_log2, 16, r, st, acc);
+            ++i;
         }
+        if (has_ragged) quant_tile<true>((n_loop & 1) ? B : A, qf, p.scale_log2, (int)(p.nQ & 15), r, st, acc);
     }
 
     // ---------------- bf16 segments: vertical rows, staging, window ----------------
@@ -258,10 +292,9 @@ decode_kernel(const DecParams p) {
                 vv[sIdx][0] = __ldg(vseg + (long)key * 16 + r);
                 vv[sIdx][1] = __ldg(vseg + (long)key * 16 + 8 + r);
             }
-            float s[4], pw[4];
-            s[0] = row0 + r < n ? c4[0] * p.scale_log2 : -INFINITY;     s[1] = row0 + r < n ? c4[1] * p.scale_log2 : -INFINITY;
-            s[2] = row0 + r + 8 < n ? c4[2] * p.scale_log2 : -INFINITY; s[3] = row0 + r + 8 < n ? c4[3] * p.scale_log2 : -INFINITY;
-            softmax_tile(st, acc, s, pw);
+            float pw[4];
+            if (row0 + 16 > n) softmax_tile<true>(st, acc, c4, p.scale_log2, row0 + r < n, row0 + r + 8 < n, pw);
+            else softmax_tile<false>(st, acc, c4, p.scale_log2, true, true, pw);
             const uint32_t b0 = movmatrix_trans(pack_bf16(pw[0], pw[1]));
             const uint32_t b1 = movmatrix_trans(pack_bf16(pw[2], pw[3]));
 #pragma unroll
