@@ -25,12 +25,14 @@
  *       kq_codes  [B,Hkv,nQp,D/2] bytes: row-major, channel 2m in the low nibble and 2m+1 in the high
  *                 nibble of byte m, two's complement (hyq_quantize_blocks' INT4 layout).
  *       vq_codes  [B,Hkv,nQp/16,1024] bytes, FRAGMENT-MAJOR: the codes of 16 consecutive compacted rows
- *                 form one 1024-byte tile laid out as 32 lanes x 8 little-endian 32-bit words; nibble n
- *                 (bits 4n..4n+3) of word x of lane l = 4r + j holds
+ *                 form one 1024-byte tile of 32 lanes x 8 little-endian 32-bit words, word x of lane l at
+ *                 byte 512*(x >> 2) + 16*l + 4*(x & 3); nibble n (bits 4n..4n+3) of word x of lane
+ *                 l = 4r + j holds
  *                     channel 64*(x >> 2) + 8*r + 2*(x & 3) + (n & 1)
  *                     of row  2*j + (n >> 2) + 8*((n >> 1) & 1)          of the tile,
- *                 i.e. each lane of a warp reads 32 contiguous bytes and owns, without any shuffle, the
- *                 operand registers of the warp-level matrix instruction that accumulates P.V.
+ *                 i.e. each lane of a warp reads two 16-byte pieces (the warp: two contiguous 512-byte
+ *                 runs) and owns, without any shuffle, the operand registers of the warp-level matrix
+ *                 instruction that accumulates P.V.
  *       kq_scales, vq_scales  [B,Hkv,nQp/64] fp32.
  *
  * (Quant(.; G) over compacted rows, and one vertical set per KV head given by the caller, are this

@@ -37,6 +37,8 @@ constexpr int DEC_WARPS = DEC_THREADS / 32;
 #ifndef DEC_CTAS_PER_SM
 #define DEC_CTAS_PER_SM 4                   // resident CTAs per SM the register budget is set for
 #endif
+constexpr int DEC_STAGES = 3;               // tiles in flight per warp (cp.async ring)
+constexpr int DEC_STAGE_BYTES = 2048;       // 1 KB K codes + 1 KB V codes
 constexpr int DEC_FP_COST = 4;              // bytes of a bf16 tile over bytes of an INT4 tile
 constexpr float DEC_RAISE = 8.0f;          // log2 units; P <= 2^8 stays far inside fp16 / bf16 range
 
@@ -101,6 +103,18 @@ __device__ __forceinline__ float ex2(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+// Ampere-style asynchronous 16-byte copy global -> shared (no register staging, completion by groups)
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
 __device__ __forceinline__ uint32_t word_of(const uint4& v, int i) {
     return i == 0 ? v.x : i == 1 ? v.y : i == 2 ? v.z : v.w;
 }
@@ -150,16 +164,11 @@ __device__ __forceinline__ void softmax_tile(SoftmaxState& st, float (&acc)[8][4
 }
 
 // One 16-row tile of the quantized prefix as it sits in registers: K rows r and r+8 (this lane's 16 bytes each),
-// the lane's 32 bytes of the V tile, and the group's two scales.
+// the lane's 2 x 16 bytes of the V tile, and the group's two scales.
 struct QTile {
     uint4 ka, kb, va, vb;
     float fk, fv;
 };
-__device__ __forceinline__ void load_qtile(QTile& d, const uint4* pk, const uint4* pv, const float* pks, const float* pvs) {
-    d.ka = __ldg(pk); d.kb = __ldg(pk + 32);
-    d.va = __ldg(pv); d.vb = __ldg(pv + 1);
-    d.fk = __ldg(pks); d.fv = __ldg(pvs);
-}
 
 template <bool RAGGED>
 __device__ __forceinline__ void quant_tile(const QTile& d, const uint32_t (&qf)[16], float scale_log2, int rows_valid, int r,
@@ -189,7 +198,12 @@ decode_kernel(const DecParams p) {
 
     __shared__ __align__(16) uint16_t qs[DEC_MAX_GROUP][HYQ_D];      // bf16 bits, heads >= g zero
     __shared__ float red_ml[DEC_WARPS][DEC_MAX_GROUP][2];
-    __shared__ float red_acc[DEC_WARPS][DEC_MAX_GROUP][HYQ_D];
+    // per warp: a ring of DEC_STAGES tiles (1 KB of K codes + 1 KB of V codes each) filled by cp.async; every lane
+    // reads back exactly the bytes it copied, so the ring needs no barrier.  Reused (after a CTA barrier) for the
+    // warps' accumulators when the CTA merges them.
+    extern __shared__ __align__(16) uint8_t ring_mem[];
+    float (*red_acc)[DEC_MAX_GROUP][HYQ_D] = reinterpret_cast<float (*)[DEC_MAX_GROUP][HYQ_D]>(ring_mem);
+    static_assert(DEC_STAGES * DEC_STAGE_BYTES >= DEC_MAX_GROUP * HYQ_D * 4, "rings too small for the merge");
 
     {   // q of the g heads of this KV head: thread t loads 8 channels of head t >> 4
         const int h = threadIdx.x >> 4, c8 = threadIdx.x & 15;
@@ -226,34 +240,43 @@ decode_kernel(const DecParams p) {
             qf[2 * c] = *reinterpret_cast<const uint32_t*>(&h0);
             qf[2 * c + 1] = *reinterpret_cast<const uint32_t*>(&h1);
         }
-        // this warp's tiles: t0, t0 + 4, ...; pointers advance by constants, two register sets alternate so
-        // that the next tile's loads are in flight while the current one is processed
+        // this warp's tiles: t0, t0 + 4, ...  Tile i is copied into ring stage i % DEC_STAGES DEC_STAGES tiles ahead
+        // of its use; one commit group per tile (empty past the end) keeps the group arithmetic uniform.
         const long t0 = q_lo + warp;
         const int n_my = (int)((q_hi - t0 + DEC_WARPS - 1) / DEC_WARPS);
         const bool has_ragged = (p.nQ & 15) && t0 + (long)(n_my - 1) * DEC_WARPS == Tq - 1;
-        const int n_loop = n_my - (has_ragged ? 1 : 0);
-        const uint4* pk = reinterpret_cast<const uint4*>(p.kq + unit * p.nQp * 64) + (t0 * 16 + r) * 4 + j;
-        const uint4* pv = reinterpret_cast<const uint4*>(p.vq + unit * (p.nQp / 16) * DEC_VTILE_BYTES) + t0 * 64 + lane * 2;
+        const uint8_t* gk = p.kq + unit * p.nQp * 64 + t0 * 1024 + lane * 16;
+        const uint8_t* gv = p.vq + unit * (p.nQp / 16) * DEC_VTILE_BYTES + t0 * 1024 + lane * 16;
         const float* pks = p.ks + unit * (p.nQp / 64) + (t0 >> 2);
         const float* pvs = p.vs + unit * (p.nQp / 64) + (t0 >> 2);
-        auto advance = [&]() { pk += DEC_WARPS * 64; pv += DEC_WARPS * 64; ++pks; ++pvs; };
-        QTile A, B;
-        load_qtile(A, pk, pv, pks, pvs);
-        B = A;
-        advance();
-        int i = 0;
-        for (;;) {
-            if (i + 1 < n_my) { load_qtile(B, pk, pv, pks, pvs); advance(); }
-            if (i >= n_loop) break;
-            quant_tile<false>(A, qf, p.scale_log2, 16, r, st, acc);
-            ++i;
-            if (i + 1 < n_my) { load_qtile(A, pk, pv, pks, pvs); advance(); }
-            if (i >= n_loop) break;
-            quant_tile<false>(B, qf, p.scale_log2, 16, r, st, acc);
-            ++i;
+        const uint32_t ring = (uint32_t)__cvta_generic_to_shared(ring_mem) + warp * (DEC_STAGES * DEC_STAGE_BYTES) + lane * 16;
+        auto issue = [&](uint32_t stage_addr) {
+            cp_async16(stage_addr, gk); cp_async16(stage_addr + 512, gk + 512);
+            cp_async16(stage_addr + 1024, gv); cp_async16(stage_addr + 1536, gv + 512);
+            gk += DEC_WARPS * 1024; gv += DEC_WARPS * 1024;
+        };
+#pragma unroll
+        for (int s = 0; s < DEC_STAGES; ++s) {
+            if (s < n_my) issue(ring + s * DEC_STAGE_BYTES);
+            cp_async_commit();
         }
-        if (has_ragged) quant_tile<true>((n_loop & 1) ? B : A, qf, p.scale_log2, (int)(p.nQ & 15), r, st, acc);
+        float fk = __ldg(pks), fv = __ldg(pvs);
+        uint32_t stage_addr = ring;
+        for (int i = 0; i < n_my; ++i) {
+            cp_async_wait<DEC_STAGES - 1>();                // tile i has landed
+            QTile A;
+            A.ka = lds128(stage_addr); A.kb = lds128(stage_addr + 512);
+            A.va = lds128(stage_addr + 1024); A.vb = lds128(stage_addr + 1536);
+            A.fk = fk; A.fv = fv;
+            if (i + DEC_STAGES < n_my) issue(stage_addr);   // refill the stage just emptied (own bytes only)
+            cp_async_commit();
+            if (i + 1 < n_my) { fk = __ldg(pks + i + 1); fv = __ldg(pvs + i + 1); }
+            stage_addr = (i % DEC_STAGES == DEC_STAGES - 1) ? ring : stage_addr + DEC_STAGE_BYTES;
+            if (has_ragged && i == n_my - 1) quant_tile<true>(A, qf, p.scale_log2, (int)(p.nQ & 15), r, st, acc);
+            else quant_tile<false>(A, qf, p.scale_log2, 16, r, st, acc);
+        }
     }
+    cp_async_wait<0>();
 
     // ---------------- bf16 segments: vertical rows, staging, window ----------------
     // keep the round-robin phase of the tile list so that the warps stay balanced across the boundary
@@ -308,6 +331,7 @@ decode_kernel(const DecParams p) {
     }
 
     // ---------------- merge the warps' states, write the slice's partial result ----------------
+    __syncthreads();                                       // every warp is done with its ring
 #pragma unroll
     for (int o = 4; o < 32; o <<= 1) {
         st.l0 += __shfl_xor_sync(0xffffffffu, st.l0, o);
@@ -426,7 +450,14 @@ int launch_decode(const void* q, const hyq_kv_cache& c, float alpha, int splits,
     const size_t slots = (size_t)units * splits * DEC_MAX_GROUP;
     p.part_acc = static_cast<float*>(workspace);
     p.part_ml = reinterpret_cast<float*>(static_cast<char*>(workspace) + align_up(slots * HYQ_D * sizeof(float), 16));
-    decode_kernel<<<dim3((unsigned)splits, (unsigned)units), DEC_THREADS, 0, st>>>(p);
+    constexpr int ring_bytes = DEC_WARPS * DEC_STAGES * DEC_STAGE_BYTES;
+    static bool attr_set = false;          // same value every time: a benign race between host threads
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ring_bytes) != cudaSuccess)
+            return HYQ_ERR_CUDA;
+        attr_set = true;
+    }
+    decode_kernel<<<dim3((unsigned)splits, (unsigned)units), DEC_THREADS, ring_bytes, st>>>(p);
     decode_merge_kernel<<<dim3((unsigned)units, (unsigned)p.g), HYQ_D, 0, st>>>(p.part_acc, p.part_ml, p.g, splits, out_dtype, out, lse);
     return launch_status();
 }

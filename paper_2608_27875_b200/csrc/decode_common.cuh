@@ -23,12 +23,12 @@ static inline CacheGeo cache_geo(const hyq_kv_cache& c) {
 }
 
 // Byte of a V tile that holds channels (d, d + 1), d even, of row `key` (0..15) of the tile: lane l = 4r + j
-// owns 32 bytes; word x, nibble n of that lane is channel 64*(x>>2) + 8r + 2*(x&3) + (n&1) of row
-// 2j + (n>>2) + 8*((n>>1)&1).
+// owns words x = 0..3 at bytes [16l, 16l + 16) and words x = 4..7 at bytes [512 + 16l, 512 + 16l + 16); nibble n of
+// word x of that lane is channel 64*(x>>2) + 8r + 2*(x&3) + (n&1) of row 2j + (n>>2) + 8*((n>>1)&1).
 __host__ __device__ __forceinline__ int vq_byte_offset(int key, int d) {
     const int j = (key & 7) >> 1, n = ((key >> 3) << 1) | ((key & 1) << 2);
     const int r = (d >> 3) & 7, x = ((d >> 6) << 2) | ((d >> 1) & 3);
-    return (4 * r + j) * 32 + x * 4 + (n >> 1);
+    return (x >> 2) * 512 + (4 * r + j) * 16 + (x & 3) * 4 + (n >> 1);
 }
 
 int launch_freeze(const void* k_, const void* v, const int32_t* vl_idx, const hyq_kv_cache& c, cudaStream_t st);

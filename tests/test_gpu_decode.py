@@ -28,8 +28,9 @@ def _v_tiles_to_rows(vq: np.ndarray) -> np.ndarray:
     [.., tiles, 1024] bytes -> [.., tiles*16, 64] bytes in the row-major INT4 layout."""
     lead = vq.shape[:-2]
     tiles = vq.shape[-2]
-    words = vq.reshape(lead + (tiles, 32, 8, 4)).astype(np.uint32)
-    words = words[..., 0] | (words[..., 1] << 8) | (words[..., 2] << 16) | (words[..., 3] << 24)   # [.., tiles, lane, x]
+    by = vq.reshape(lead + (tiles, 2, 32, 4, 4)).astype(np.uint32)                  # [.., tile, x >> 2, lane, x & 3, byte]
+    words = by[..., 0] | (by[..., 1] << 8) | (by[..., 2] << 16) | (by[..., 3] << 24)
+    words = np.moveaxis(words, -3, -2).reshape(lead + (tiles, 32, 8))               # [.., tile, lane, x]
     rows = np.zeros(lead + (tiles, 16, 128), dtype=np.uint8)
     for lane in range(32):
         r, j = lane >> 2, lane & 3
