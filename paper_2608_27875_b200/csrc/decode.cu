@@ -37,7 +37,10 @@ constexpr int DEC_WARPS = DEC_THREADS / 32;
 #ifndef DEC_CTAS_PER_SM
 #define DEC_CTAS_PER_SM 4                   // resident CTAs per SM the register budget is set for
 #endif
-constexpr int DEC_STAGES = 3;               // tiles in flight per warp (cp.async ring)
+#ifndef DEC_STAGES_N
+#define DEC_STAGES_N 3
+#endif
+constexpr int DEC_STAGES = DEC_STAGES_N;    // tiles in flight per warp (cp.async ring)
 constexpr int DEC_STAGE_BYTES = 2048;       // 1 KB K codes + 1 KB V codes
 constexpr int DEC_FP_COST = 4;              // bytes of a bf16 tile over bytes of an INT4 tile
 constexpr float DEC_RAISE = 8.0f;          // log2 units; P <= 2^8 stays far inside fp16 / bf16 range
@@ -88,6 +91,34 @@ __device__ __forceinline__ uint32_t dq4_hi(uint32_t w) {
     asm("fma.rn.f16x2 %0, %1, %2, %3;" : "=r"(h) : "r"(h), "r"(0x2C002C00u), "r"(0xD480D480u));
     return h;
 }
+// K side only: the codes enter the matrix instruction as fp16 SUBNORMALS with no arithmetic at all - the nibble
+// (xor 8, i.e. code + 8) placed in mantissa bits 0-3 is (code + 8) * 2^-24, placed in bits 4-7 it is
+// (code + 8) * 2^-20.  The factor 16 of the second form is taken out of q's operand for those channels, the
+// common 2^-24 goes into the score scale, and the +8 becomes 8 * sum_d q_d per head, subtracted from the score
+// (a cancellation of a few units against a dot product of eight k-steps: harmless in fp32).  The products
+// fp16 x fp16 are exact in the instruction's fp32 accumulation.
+#ifndef DEC_K_SUBNORMAL
+#define DEC_K_SUBNORMAL 1
+#endif
+__device__ __forceinline__ uint32_t kq4_lo(uint32_t w) {
+#if DEC_K_SUBNORMAL
+    uint32_t h;
+    asm("lop3.b32 %0, %1, 0x000F000F, 0x00080008, 0x6A;" : "=r"(h) : "r"(w));
+    return h;
+#else
+    return dq4_lo(w);
+#endif
+}
+__device__ __forceinline__ uint32_t kq4_hi(uint32_t w) {
+#if DEC_K_SUBNORMAL
+    uint32_t h;
+    asm("lop3.b32 %0, %1, 0x00F000F0, 0x00800080, 0x6A;" : "=r"(h) : "r"(w));
+    return h;
+#else
+    return dq4_hi(w);
+#endif
+}
+constexpr float DEC_K_UNIT = DEC_K_SUBNORMAL ? 16777216.0f : 1.0f;      // 2^24: undoes the subnormal placement
 __device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
     uint32_t d;
     asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
@@ -128,18 +159,21 @@ struct SoftmaxState {
 // One tile's raw scores c4 (keys r and r+8, heads 2j and 2j+1) times f (log2 units) -> weights p[4].
 // MASKED: rows flagged invalid (past the end of a segment) get weight zero.  The reference maxima are raised,
 // and the accumulators rescaled, only when some score is more than 2^DEC_RAISE above them (warp vote).
+// b0, b1: per-head constants subtracted from the raw scores before scaling (zero unless the K operand carries
+// an offset).
 template <bool MASKED>
 __device__ __forceinline__ void softmax_tile(SoftmaxState& st, float (&acc)[8][4], const float (&c4)[4], float f,
-                                             bool valid_a, bool valid_b, float (&p)[4]) {
-    float d0 = fmaf(c4[0], f, -st.m0), d2 = fmaf(c4[2], f, -st.m0);
-    float d1 = fmaf(c4[1], f, -st.m1), d3 = fmaf(c4[3], f, -st.m1);
+                                             float b0, float b1, bool valid_a, bool valid_b, float (&p)[4]) {
+    const float mm0 = fmaf(b0, f, st.m0), mm1 = fmaf(b1, f, st.m1);
+    float d0 = fmaf(c4[0], f, -mm0), d2 = fmaf(c4[2], f, -mm0);
+    float d1 = fmaf(c4[1], f, -mm1), d3 = fmaf(c4[3], f, -mm1);
     if (MASKED) {
         if (!valid_a) d0 = d1 = -INFINITY;
         if (!valid_b) d2 = d3 = -INFINITY;
     }
     const bool far = fmaxf(d0, d2) > DEC_RAISE || fmaxf(d1, d3) > DEC_RAISE;
     if (__any_sync(0xffffffffu, far)) {
-        float s0 = c4[0] * f, s1 = c4[1] * f, s2 = c4[2] * f, s3 = c4[3] * f;
+        float s0 = (c4[0] - b0) * f, s1 = (c4[1] - b1) * f, s2 = (c4[2] - b0) * f, s3 = (c4[3] - b1) * f;
         if (MASKED) {
             if (!valid_a) s0 = s1 = -INFINITY;
             if (!valid_b) s2 = s3 = -INFINITY;
@@ -171,16 +205,16 @@ struct QTile {
 };
 
 template <bool RAGGED>
-__device__ __forceinline__ void quant_tile(const QTile& d, const uint32_t (&qf)[16], float scale_log2, int rows_valid, int r,
-                                           SoftmaxState& st, float (&acc)[8][4]) {
+__device__ __forceinline__ void quant_tile(const QTile& d, const uint32_t (&qf)[16], float scale_log2, float bias0, float bias1,
+                                           int rows_valid, int r, SoftmaxState& st, float (&acc)[8][4]) {
     float c4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
 #pragma unroll
     for (int c = 0; c < 8; ++c) {
         const uint32_t wa = word_of(d.ka, c >> 1) >> (8 * (c & 1)), wb = word_of(d.kb, c >> 1) >> (8 * (c & 1));
-        mma_f16(c4, dq4_lo(wa), dq4_lo(wb), dq4_hi(wa), dq4_hi(wb), qf[2 * c], qf[2 * c + 1]);
+        mma_f16(c4, kq4_lo(wa), kq4_lo(wb), kq4_hi(wa), kq4_hi(wb), qf[2 * c], qf[2 * c + 1]);
     }
     float pw[4];
-    softmax_tile<RAGGED>(st, acc, c4, d.fk * scale_log2, r < rows_valid, r + 8 < rows_valid, pw);
+    softmax_tile<RAGGED>(st, acc, c4, d.fk * scale_log2, bias0, bias1, r < rows_valid, r + 8 < rows_valid, pw);
     const uint32_t b0 = movmatrix_trans(pack_f16(pw[0] * d.fv, pw[1] * d.fv));
     const uint32_t b1 = movmatrix_trans(pack_f16(pw[2] * d.fv, pw[3] * d.fv));
 #pragma unroll
@@ -198,6 +232,7 @@ decode_kernel(const DecParams p) {
 
     __shared__ __align__(16) uint16_t qs[DEC_MAX_GROUP][HYQ_D];      // bf16 bits, heads >= g zero
     __shared__ float red_ml[DEC_WARPS][DEC_MAX_GROUP][2];
+    __shared__ float q_sum[DEC_MAX_GROUP];                            // sum over channels of q as the K product sees it
     // per warp: a ring of DEC_STAGES tiles (1 KB of K codes + 1 KB of V codes each) filled by cp.async; every lane
     // reads back exactly the bytes it copied, so the ring needs no barrier.  Reused (after a CTA barrier) for the
     // warps' accumulators when the CTA merges them.
@@ -210,6 +245,17 @@ decode_kernel(const DecParams p) {
         uint4 v = make_uint4(0, 0, 0, 0);
         if (h < p.g) v = __ldg(p.q + (unit * p.g + h) * 16 + c8);
         *reinterpret_cast<uint4*>(&qs[h][c8 * 8]) = v;
+        // Odd channels sit in the high nibbles: their q enters the product as fp16(q / 16), times 16 here.
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+        float sum = 0.0f;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            sum += __half2float(__float2half_rn(bf16_lo(w[i])));
+            sum += 16.0f * __half2float(__float2half_rn(bf16_hi(w[i]) * 0.0625f));
+        }
+#pragma unroll
+        for (int o = 1; o < 16; o <<= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+        if (c8 == 0) q_sum[h] = sum;
     }
     __syncthreads();
 
@@ -236,7 +282,12 @@ decode_kernel(const DecParams p) {
             const uint16_t* qr = qs[r];
             auto f16 = [&](int ch) { return __float2half_rn(__uint_as_float((uint32_t)qr[ch] << 16)); };
             const __half2 h0 = __halves2half2(f16(base), f16(base + 4));
+#if DEC_K_SUBNORMAL
+            auto f16s = [&](int ch) { return __float2half_rn(__uint_as_float((uint32_t)qr[ch] << 16) * 0.0625f); };
+            const __half2 h1 = __halves2half2(f16s(base + 1), f16s(base + 5));
+#else
             const __half2 h1 = __halves2half2(f16(base + 1), f16(base + 5));
+#endif
             qf[2 * c] = *reinterpret_cast<const uint32_t*>(&h0);
             qf[2 * c + 1] = *reinterpret_cast<const uint32_t*>(&h1);
         }
@@ -262,6 +313,9 @@ decode_kernel(const DecParams p) {
         }
         float fk = __ldg(pks), fv = __ldg(pvs);
         uint32_t stage_addr = ring;
+        const float kscale = p.scale_log2 * DEC_K_UNIT;
+        const float b0 = DEC_K_SUBNORMAL ? q_sum[2 * j] * (8.0f / DEC_K_UNIT) : 0.0f;
+        const float b1 = DEC_K_SUBNORMAL ? q_sum[2 * j + 1] * (8.0f / DEC_K_UNIT) : 0.0f;
         for (int i = 0; i < n_my; ++i) {
             cp_async_wait<DEC_STAGES - 1>();                // tile i has landed
             QTile A;
@@ -272,8 +326,8 @@ decode_kernel(const DecParams p) {
             cp_async_commit();
             if (i + 1 < n_my) { fk = __ldg(pks + i + 1); fv = __ldg(pvs + i + 1); }
             stage_addr = (i % DEC_STAGES == DEC_STAGES - 1) ? ring : stage_addr + DEC_STAGE_BYTES;
-            if (has_ragged && i == n_my - 1) quant_tile<true>(A, qf, p.scale_log2, (int)(p.nQ & 15), r, st, acc);
-            else quant_tile<false>(A, qf, p.scale_log2, 16, r, st, acc);
+            if (has_ragged && i == n_my - 1) quant_tile<true>(A, qf, kscale, b0, b1, (int)(p.nQ & 15), r, st, acc);
+            else quant_tile<false>(A, qf, kscale, b0, b1, 16, r, st, acc);
         }
     }
     cp_async_wait<0>();
@@ -316,8 +370,8 @@ decode_kernel(const DecParams p) {
                 vv[sIdx][1] = __ldg(vseg + (long)key * 16 + 8 + r);
             }
             float pw[4];
-            if (row0 + 16 > n) softmax_tile<true>(st, acc, c4, p.scale_log2, row0 + r < n, row0 + r + 8 < n, pw);
-            else softmax_tile<false>(st, acc, c4, p.scale_log2, true, true, pw);
+            if (row0 + 16 > n) softmax_tile<true>(st, acc, c4, p.scale_log2, 0.0f, 0.0f, row0 + r < n, row0 + r + 8 < n, pw);
+            else softmax_tile<false>(st, acc, c4, p.scale_log2, 0.0f, 0.0f, true, true, pw);
             const uint32_t b0 = movmatrix_trans(pack_bf16(pw[0], pw[1]));
             const uint32_t b1 = movmatrix_trans(pack_bf16(pw[2], pw[3]));
 #pragma unroll
