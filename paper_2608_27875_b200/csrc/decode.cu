@@ -20,8 +20,8 @@
 // The bf16 segments (vertical rows, staging, window) go through the same two products with bf16 operands;
 // there V^T's key pairs are formed from two rows' words with byte permutes.
 //
-// Grid: (splits, B * Hkv).  A CTA owns a contiguous slice of the head's 16-row tiles (all four segments
-// form one tile list); its 4 warps take tiles round-robin, each with its own online-softmax state, which
+// Grid: (splits, B * Hkv).  A CTA owns a contiguous slice of the head's INT4 tiles and one of its bf16 tiles
+// (the three bf16 segments form one tile list); its 4 warps take tiles round-robin, each with its own online-softmax state, which
 // are merged through shared memory; the slices' (m, l, acc) go to the workspace and decode_merge_kernel
 // applies ReduceSoftmax.  Softmax is lazy: a tile only raises the running reference maximum when one of its
 // scores exceeds it by more than 2^DEC_RAISE (warp vote), so the usual tile costs four compares, four ex2
@@ -42,7 +42,6 @@ constexpr int DEC_WARPS = DEC_THREADS / 32;
 #endif
 constexpr int DEC_STAGES = DEC_STAGES_N;    // tiles in flight per warp (cp.async ring)
 constexpr int DEC_STAGE_BYTES = 2048;       // 1 KB K codes + 1 KB V codes
-constexpr int DEC_FP_COST = 4;              // bytes of a bf16 tile over bytes of an INT4 tile
 constexpr float DEC_RAISE = 8.0f;          // log2 units; P <= 2^8 stays far inside fp16 / bf16 range
 
 struct DecParams {
@@ -261,12 +260,11 @@ decode_kernel(const DecParams p) {
 
     const long Tq = (p.nQ + 15) / 16;
     const int Tvl = (p.k + 15) / 16, Ts = (p.n_s + 15) / 16, Tw = (p.W + 15) / 16;
-    // The slices are equal in BYTES, not tiles: a bf16 tile moves four times what an INT4 tile moves.
-    const long Tf = Tvl + Ts + Tw, cost = Tq + DEC_FP_COST * Tf;
-    const long ca = cost * split / p.splits, cb = cost * (split + 1) / p.splits;
-    const long q_lo = ca < Tq ? ca : Tq, q_hi = cb < Tq ? cb : Tq;
-    const long f_lo = Tq + (ca > Tq ? (ca - Tq + DEC_FP_COST - 1) / DEC_FP_COST : 0);
-    const long f_hi = Tq + (cb > Tq ? (cb - Tq + DEC_FP_COST - 1) / DEC_FP_COST : 0);
+    // Every slice takes the same share of the INT4 tiles AND of the bf16 tiles (a bf16 tile moves four times the
+    // bytes and goes through a different loop), so all CTAs of a head carry the same mix of work.
+    const long Tf = Tvl + Ts + Tw;
+    const long q_lo = Tq * split / p.splits, q_hi = Tq * (split + 1) / p.splits;
+    const long f_lo = Tq + Tf * split / p.splits, f_hi = Tq + Tf * (split + 1) / p.splits;
 
     SoftmaxState st = {-INFINITY, -INFINITY, 0.0f, 0.0f};
     float acc[8][4];
@@ -333,7 +331,7 @@ decode_kernel(const DecParams p) {
     cp_async_wait<0>();
 
     // ---------------- bf16 segments: vertical rows, staging, window ----------------
-    // keep the round-robin phase of the tile list so that the warps stay balanced across the boundary
+    // continue the round-robin where the INT4 tiles left off so that the warps stay balanced
     long t = f_lo + ((warp - (q_hi - q_lo)) % DEC_WARPS + DEC_WARPS) % DEC_WARPS;
     if (t < f_hi) {
         uint32_t qb[16];                                   // q^T operand, bf16
