@@ -41,6 +41,9 @@ FALLBACK = {"bf16_tflops": 1590.0, "hbm_gbs": 6650.0}
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu
 # capture summarised under profiles/ (bytes per launch of the benchmark workload; None = no capture yet)
 NCU_TRAFFIC_BYTES = {"c2": 695749888 + 515654400}
+# decode_kernel on the c2 cache shape, captured at batch 4 (157.152 MB read + 4.299 MB written); traffic grows in
+# proportion to the batch, so the bench scales it by B / 4
+NCU_DECODE_TRAFFIC_BYTES_B4 = 157152000 + 4299008
 
 
 def measured_peaks():
@@ -456,7 +459,7 @@ def run_decode(args, w: wl.Workload):
                    "freeze_ms": freeze_ms},
         "roofline": {"bound": "hbm", "kernel": "decode_kernel + decode_merge_kernel (one call)",
                      "achieved": by / (ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                     "frac": by / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES.get("decode"),
+                     "frac": by / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "traffic": (NCU_DECODE_TRAFFIC_BYTES_B4 * w.B // 4 if (w.name, w.L, args.staging) == ("c2", 32768, 128) else None),
                      "bytes_per_call": by, "peak_source": peaks["source"]},
         "cpu_baseline": {"value": cpu_s * 1e6 * w.B, "unit": "us", "cores": oracle.num_threads(), "kind": "oracle",
                          "sample": "oracle attention of one sequence (all heads) timed, scaled by the batch size"},
