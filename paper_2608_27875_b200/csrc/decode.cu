@@ -37,8 +37,11 @@ constexpr int DEC_WARPS = DEC_THREADS / 32;
 #ifndef DEC_CTAS_PER_SM
 #define DEC_CTAS_PER_SM 4                   // resident CTAs per SM the register budget is set for
 #endif
+#ifndef DEC_PAIR
+#define DEC_PAIR 1                           // INT4 tiles are processed two at a time
+#endif
 #ifndef DEC_STAGES_N
-#define DEC_STAGES_N 3
+#define DEC_STAGES_N 4
 #endif
 constexpr int DEC_STAGES = DEC_STAGES_N;    // tiles in flight per warp (cp.async ring)
 constexpr int DEC_STAGE_BYTES = 2048;       // 1 KB K codes + 1 KB V codes
@@ -223,6 +226,40 @@ __device__ __forceinline__ void quant_tile(const QTile& d, const uint32_t (&qf)[
     }
 }
 
+// Two full tiles at once: both Q.K^T chains are issued back to back and the second tile's softmax runs while the
+// first tile's P.V instructions are in flight - more independent work per warp, which is what a kernel with
+// few warps per SM lacks.  P.V of the first tile precedes the second softmax because that softmax may rescale
+// the accumulators.
+__device__ __forceinline__ void quant_tile_pair(const QTile& d0, const QTile& d1, const uint32_t (&qf)[16], float scale_log2,
+                                                float bias0, float bias1, SoftmaxState& st, float (&acc)[8][4]) {
+    float ca[4] = {0.0f, 0.0f, 0.0f, 0.0f}, cb[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+        const int sh = 8 * (c & 1);
+        const uint32_t wa = word_of(d0.ka, c >> 1) >> sh, wb = word_of(d0.kb, c >> 1) >> sh;
+        mma_f16(ca, kq4_lo(wa), kq4_lo(wb), kq4_hi(wa), kq4_hi(wb), qf[2 * c], qf[2 * c + 1]);
+        const uint32_t xa = word_of(d1.ka, c >> 1) >> sh, xb = word_of(d1.kb, c >> 1) >> sh;
+        mma_f16(cb, kq4_lo(xa), kq4_lo(xb), kq4_hi(xa), kq4_hi(xb), qf[2 * c], qf[2 * c + 1]);
+    }
+    float pw[4];
+    softmax_tile<false>(st, acc, ca, d0.fk * scale_log2, bias0, bias1, true, true, pw);
+    uint32_t b0 = movmatrix_trans(pack_f16(pw[0] * d0.fv, pw[1] * d0.fv));
+    uint32_t b1 = movmatrix_trans(pack_f16(pw[2] * d0.fv, pw[3] * d0.fv));
+#pragma unroll
+    for (int x = 0; x < 8; ++x) {
+        const uint32_t w = word_of(x < 4 ? d0.va : d0.vb, x & 3);
+        mma_f16(acc[x], dq4_lo(w), dq4_hi(w), dq4_lo(w >> 8), dq4_hi(w >> 8), b0, b1);
+    }
+    softmax_tile<false>(st, acc, cb, d1.fk * scale_log2, bias0, bias1, true, true, pw);
+    b0 = movmatrix_trans(pack_f16(pw[0] * d1.fv, pw[1] * d1.fv));
+    b1 = movmatrix_trans(pack_f16(pw[2] * d1.fv, pw[3] * d1.fv));
+#pragma unroll
+    for (int x = 0; x < 8; ++x) {
+        const uint32_t w = word_of(x < 4 ? d1.va : d1.vb, x & 3);
+        mma_f16(acc[x], dq4_lo(w), dq4_hi(w), dq4_lo(w >> 8), dq4_hi(w >> 8), b0, b1);
+    }
+}
+
 __global__ void __launch_bounds__(DEC_THREADS, DEC_CTAS_PER_SM)
 decode_kernel(const DecParams p) {
     const int split = blockIdx.x;
@@ -309,22 +346,34 @@ decode_kernel(const DecParams p) {
             if (s < n_my) issue(ring + s * DEC_STAGE_BYTES);
             cp_async_commit();
         }
-        float fk = __ldg(pks), fv = __ldg(pvs);
         uint32_t stage_addr = ring;
         const float kscale = p.scale_log2 * DEC_K_UNIT;
         const float b0 = DEC_K_SUBNORMAL ? q_sum[2 * j] * (8.0f / DEC_K_UNIT) : 0.0f;
         const float b1 = DEC_K_SUBNORMAL ? q_sum[2 * j + 1] * (8.0f / DEC_K_UNIT) : 0.0f;
-        for (int i = 0; i < n_my; ++i) {
+        const int n_full = n_my - (has_ragged ? 1 : 0);
+        auto fetch = [&](QTile& d, int i) {                 // ring stage of tile i -> registers, then refill it
+            d.ka = lds128(stage_addr); d.kb = lds128(stage_addr + 512);
+            d.va = lds128(stage_addr + 1024); d.vb = lds128(stage_addr + 1536);
+            d.fk = __ldg(pks + i); d.fv = __ldg(pvs + i);
+            if (i + DEC_STAGES < n_my) issue(stage_addr);   // own bytes only: no barrier
+            cp_async_commit();
+            stage_addr = (i % DEC_STAGES == DEC_STAGES - 1) ? ring : stage_addr + DEC_STAGE_BYTES;
+        };
+        int i = 0;
+#if DEC_PAIR
+        for (; i + 2 <= n_full; i += 2) {
+            cp_async_wait<DEC_STAGES - 2>();                // tiles i and i + 1 have landed
+            QTile A, B;
+            fetch(A, i);
+            fetch(B, i + 1);
+            quant_tile_pair(A, B, qf, kscale, b0, b1, st, acc);
+        }
+#endif
+        for (; i < n_my; ++i) {
             cp_async_wait<DEC_STAGES - 1>();                // tile i has landed
             QTile A;
-            A.ka = lds128(stage_addr); A.kb = lds128(stage_addr + 512);
-            A.va = lds128(stage_addr + 1024); A.vb = lds128(stage_addr + 1536);
-            A.fk = fk; A.fv = fv;
-            if (i + DEC_STAGES < n_my) issue(stage_addr);   // refill the stage just emptied (own bytes only)
-            cp_async_commit();
-            if (i + 1 < n_my) { fk = __ldg(pks + i + 1); fv = __ldg(pvs + i + 1); }
-            stage_addr = (i % DEC_STAGES == DEC_STAGES - 1) ? ring : stage_addr + DEC_STAGE_BYTES;
-            if (has_ragged && i == n_my - 1) quant_tile<true>(A, qf, kscale, b0, b1, (int)(p.nQ & 15), r, st, acc);
+            fetch(A, i);
+            if (i >= n_full) quant_tile<true>(A, qf, kscale, b0, b1, (int)(p.nQ & 15), r, st, acc);
             else quant_tile<false>(A, qf, kscale, b0, b1, 16, r, st, acc);
         }
     }
