@@ -120,6 +120,35 @@ def select_vertical(q_bits, k_bits, window: int, k: int, n_tail: int = 0, return
     return (idx, scores) if return_scores else idx
 
 
+def exp_det(x) -> np.ndarray:
+    """The oracle's operation-by-operation exp for x <= 0 (Eq. 4 scores decide an index set)."""
+    x = np.ascontiguousarray(x, dtype=np.float64)
+    out = np.zeros(x.shape, dtype=np.float64)
+    _load().oracle_exp_det(_ptr(x), ctypes.c_long(x.size), _ptr(out))
+    return out
+
+
+def select_vertical_mass(q_bits, k_bits, window: int, k: int, n_queries: int = 0, alpha: float | None = None,
+                         return_scores: bool = False):
+    """Eq. 4-5: column mass of the softmax rows of the last n_queries queries, top-k over the non-window
+    prefix.  Returns int32 [B,Hq,k] ascending (and optionally the fp64 scores [B,Hq,P])."""
+    q = _u16(q_bits, 4)
+    kk = _u16(k_bits, 4)
+    B, Hq, Lq, D = q.shape
+    Bk, Hkv, Lk, Dk = kk.shape
+    assert B == Bk and D == Dk
+    P = max(0, Lk - window)
+    kk_eff = 0 if P == 0 else k
+    idx = np.zeros((B, Hq, kk_eff), dtype=np.int32)
+    scores = np.zeros((B, Hq, P), dtype=np.float64) if return_scores else None
+    a = 1.0 / np.sqrt(np.float64(D)) if alpha is None else float(alpha)
+    rc = _load().oracle_select_mass(_ptr(q), _ptr(kk), B, Hq, Hkv, Lq, Lk, D, window, n_queries, kk_eff,
+                                    ctypes.c_double(a), _ptr(idx), _ptr(scores) if return_scores else None)
+    if rc:
+        raise ValueError(f"oracle_select_mass failed ({rc})")
+    return (idx, scores) if return_scores else idx
+
+
 def _attn_in(q_bits, k_bits, v_bits, qc, kc, vc, qs, ks, vs, fmts, vl_idx, window, block_tokens, alpha,
              fixed_window=False):
     q, kk, v = _u16(q_bits, 4), _u16(k_bits, 4), _u16(v_bits, 4)

@@ -193,6 +193,124 @@ int oracle_select(const uint16_t* q, const uint16_t* k_, int B, int Hq, int Hkv,
 }
 
 /* ------------------------------------------------------------------------- */
+/* Eq. 4-5: vertical-line score as accumulated column mass.                    */
+/*   a_{t,j} = softmax over the keys j <= pos(t) of alpha * <q_t, k_j>         */
+/*   S(p)    = sum over the query set T of a_{t,p},   p in the prefix [0, P)    */
+/*   I       = TopK(S, k), ties towards the lower position, ascending          */
+/* T is the last n_queries query rows (0: min(W, Lq), Algorithm 1's tail); the   */
+/* query block is end-aligned with the keys: row i sits at position            */
+/* Lk - Lq + i.  n_queries <= W, so every prefix key is visible to every t.    */
+/*                                                                             */
+/* Because the scores decide an index set that the GPU must reproduce exactly, */
+/* the arithmetic is fixed operation by operation (all fp64, round to nearest):*/
+/*   s       = (fma chain over channels 0..D-1 from 0) * alpha                 */
+/*   exp     = exp_det below (range reduction by ln2 in two parts, degree-13   */
+/*             Taylor polynomial by Horner fma, exact scaling by 2^n)          */
+/*   row sum = per chunk of 64 consecutive keys (aligned at multiples of 64):  */
+/*             m_c = max, z_c = balanced pairwise tree over exp(s - m_c) with  */
+/*             masked keys contributing 0; then m = max_c m_c and              */
+/*             Z = sum_c z_c * exp(m_c - m), added in ascending chunk order    */
+/*   S(p)    = sum over t ascending of exp(s - m_t) / Z_t                      */
+/* ------------------------------------------------------------------------- */
+static double exp_det(double x) {
+    if (!(x >= -690.0)) return 0.0;                 /* also -inf; the caller never passes x > 0 by much */
+    const double n = rint(x * 1.4426950408889634);
+    double r = fma(n, -6.93147180369123816490e-01, x);
+    r = fma(n, -1.90821492927058770002e-10, r);
+    double p = 1.0 / 6227020800.0;                  /* 1/13! */
+    p = fma(p, r, 1.0 / 479001600.0);
+    p = fma(p, r, 1.0 / 39916800.0);
+    p = fma(p, r, 1.0 / 3628800.0);
+    p = fma(p, r, 1.0 / 362880.0);
+    p = fma(p, r, 1.0 / 40320.0);
+    p = fma(p, r, 1.0 / 5040.0);
+    p = fma(p, r, 1.0 / 720.0);
+    p = fma(p, r, 1.0 / 120.0);
+    p = fma(p, r, 1.0 / 24.0);
+    p = fma(p, r, 1.0 / 6.0);
+    p = fma(p, r, 0.5);
+    p = fma(p, r, 1.0);
+    p = fma(p, r, 1.0);
+    union { uint64_t u; double d; } two_n;
+    two_n.u = (uint64_t)((int64_t)n + 1023) << 52;  /* n >= -996: a normal number */
+    return p * two_n.d;
+}
+
+void oracle_exp_det(const double* x, long n, double* out) {
+    for (long i = 0; i < n; ++i) out[i] = exp_det(x[i]);
+}
+
+static double tree_sum64(double* e) {               /* balanced pairwise tree: (0,1),(2,3).. then pairs of pairs */
+    for (int step = 1; step < 64; step <<= 1)
+        for (int i = 0; i < 64; i += 2 * step) e[i] = e[i] + e[i + step];
+    return e[0];
+}
+
+int oracle_select_mass(const uint16_t* q, const uint16_t* k_, int B, int Hq, int Hkv, int Lq, int Lk, int D, int W,
+                       int n_queries, int k, double alpha, int32_t* idx_out, double* scores_out) {
+    if (Hkv <= 0 || Hq % Hkv) return 1;
+    const int g = Hq / Hkv;
+    const int P = (Lk - W > 0) ? Lk - W : 0;
+    if (P == 0 || k == 0) return 0;
+    if (k > P || k < 0 || Lq > Lk) return 1;
+    const int nT = n_queries ? n_queries : (W < Lq ? W : Lq);
+    if (nT <= 0 || nT > Lq || nT > W) return 1;
+    const int n_chunks = (Lk + 63) / 64;
+    int err = 0;
+#pragma omp parallel for schedule(dynamic)
+    for (int bh = 0; bh < B * Hq; ++bh) {
+        const int b = bh / Hq, h = bh % Hq, kvh = h / g;
+        const uint16_t* kh = k_ + ((long)b * Hkv + kvh) * Lk * D;
+        double* S = (double*)calloc((size_t)P, sizeof(double));
+        double* srow = (double*)malloc(sizeof(double) * (size_t)Lk);
+        double* mc = (double*)malloc(sizeof(double) * (size_t)n_chunks);
+        double* zc = (double*)malloc(sizeof(double) * (size_t)n_chunks);
+        scored_t* sc = (scored_t*)malloc(sizeof(scored_t) * (size_t)P);
+        if (!S || !srow || !mc || !zc || !sc) { err = 2; free(S); free(srow); free(mc); free(zc); free(sc); continue; }
+        for (int i = Lq - nT; i < Lq; ++i) {        /* t ascending */
+            const int pos = Lk - Lq + i;
+            const uint16_t* qr = q + (((long)b * Hq + h) * Lq + i) * D;
+            for (int j = 0; j <= pos; ++j) {
+                double acc = 0.0;
+                for (int d = 0; d < D; ++d)
+                    acc = fma((double)bf16_to_f32(qr[d]), (double)bf16_to_f32(kh[(long)j * D + d]), acc);
+                srow[j] = acc * alpha;
+            }
+            const int nc = pos / 64 + 1;
+            double m = -INFINITY;
+            for (int c = 0; c < nc; ++c) {
+                double e[64], cm = -INFINITY;
+                for (int u = 0; u < 64; ++u) {
+                    const int j = 64 * c + u;
+                    if (j <= pos && srow[j] > cm) cm = srow[j];
+                }
+                for (int u = 0; u < 64; ++u) {
+                    const int j = 64 * c + u;
+                    e[u] = j <= pos ? exp_det(srow[j] - cm) : 0.0;
+                }
+                mc[c] = cm;
+                zc[c] = tree_sum64(e);
+                if (cm > m) m = cm;
+            }
+            double Z = 0.0;
+            for (int c = 0; c < nc; ++c) Z = Z + zc[c] * exp_det(mc[c] - m);
+            for (int p = 0; p < P; ++p) S[p] = S[p] + exp_det(srow[p] - m) / Z;
+        }
+        for (int p = 0; p < P; ++p) {
+            sc[p].s = S[p];
+            sc[p].p = p;
+            if (scores_out) scores_out[(long)bh * P + p] = S[p];
+        }
+        qsort(sc, P, sizeof(scored_t), cmp_scored);
+        int32_t* out = idx_out + (long)bh * k;
+        for (int c = 0; c < k; ++c) out[c] = sc[c].p;
+        qsort(out, k, sizeof(int32_t), cmp_int);
+        free(S); free(srow); free(mc); free(zc); free(sc);
+    }
+    return err;
+}
+
+/* ------------------------------------------------------------------------- */
 /* Eq. 6-7: hybrid-precision causal attention, by its definition.             */
 /* For query row i of head h and every key j <= i:                            */
 /*   the pair is full precision (FP) when j is a vertical-line key of (b,h)   */
