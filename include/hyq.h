@@ -5,6 +5,7 @@
  * (Algorithm 2: Stage 1 -> Stage 2 -> Stage 3):
  *
  *   hyq_select_vertical            Algorithm 1 (vertical token identification)
+ *   hyq_select_vertical_mass       Eq. 4-5 (the same selection from accumulated softmax column mass)
  *   hyq_quantize_blocks            Algorithm 2, Stage 2 (per-tile quantization)
  *   hyq_hybrid_attention_prefill   Eq. 6-7 / Algorithm 2, Stage 3 (fused hybrid softmax attention)
  *
@@ -113,6 +114,30 @@ int hyq_select_vertical(const void* q, const void* k_, int B, int Hq, int Hkv, i
 #define HYQ_SELECT_STATIC_SCRATCH_BYTES (8u << 20)
 int hyq_select_vertical_static(const void* q, const void* k_, int B, int Hq, int Hkv, int Lq, int Lk, int D,
                                int window, int n_tail, int k, int32_t* idx_out, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * hyq_select_vertical_mass - Eq. 4-5: the vertical-line score as accumulated column mass.
+ *
+ *   T    = the last n_queries query rows (n_queries == 0: min(window, Lq), Algorithm 1's tail); the query
+ *          block is end-aligned with the keys: row i sits at position Lk - Lq + i.  n_queries <= window, so
+ *          that every candidate key is visible to every query of T.
+ *   a_tj = softmax over the keys j <= pos(t) of softmax_scale * <Q[t], K[j]>            (bf16 originals)
+ *   S[p] = sum over t in T of a_tp,    p in the non-window prefix [0, P),  P = max(0, Lk - window)
+ *   idx_out[b, h, :] = positions of the k largest S, ties towards the lower position, ASCENDING.
+ *
+ *   All arithmetic is fp64 with a fixed order of operations (fma chain over channels, a polynomial exp,
+ *   row sums as 64-key chunk trees combined in ascending order, queries added in ascending order), so the
+ *   selected set is reproducible bit for bit.  Cost: two passes of n_queries * Lk * D fp64 fma per head -
+ *   meant for a handful of tail queries (tens), not for the whole window.
+ *
+ *   Arguments, outputs and errors as hyq_select_vertical, plus: n_queries > min(window, Lq) or Lq > Lk ->
+ *   INVALID_ARG.  softmax_scale 0 => 1/sqrt(D).  workspace: hyq_select_vertical_mass_workspace bytes.
+ * ------------------------------------------------------------------------------------------- */
+int hyq_select_vertical_mass_workspace(int B, int Hq, int Hkv, int Lq, int Lk, int D, int window, int n_queries,
+                                       int k, size_t* bytes /* host, out */);
+int hyq_select_vertical_mass(const void* q, const void* k_, int B, int Hq, int Hkv, int Lq, int Lk, int D,
+                             int window, int n_queries, int k, float softmax_scale, int32_t* idx_out,
+                             void* workspace, size_t workspace_bytes, void* stream);
 
 /* ---------------------------------------------------------------------------------------------
  * hyq_quantize_blocks - Algorithm 2, Stage 2 (per-tile symmetric quantization).

@@ -18,7 +18,8 @@ HYQ_OK = 0
 IMPL_AUTO, IMPL_TCGEN05, IMPL_SIMT = 0, 1, 2
 WINDOW_SLIDING, WINDOW_FIXED_TAIL = 0, 1
 EXPORTS = ("hyq_status_string", "hyq_version", "hyq_paper_k", "hyq_select_vertical_workspace",
-           "hyq_select_vertical", "hyq_select_vertical_static", "hyq_quantize_blocks", "hyq_hybrid_attention_prefill_workspace",
+           "hyq_select_vertical", "hyq_select_vertical_static", "hyq_select_vertical_mass_workspace",
+           "hyq_select_vertical_mass", "hyq_quantize_blocks", "hyq_hybrid_attention_prefill_workspace",
            "hyq_hybrid_attention_prefill")
 
 
@@ -61,6 +62,9 @@ def lib() -> ctypes.CDLL:
                                           [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p])
         L.hyq_select_vertical_static.argtypes = ([ctypes.c_void_p] * 2 + [ctypes.c_int] * 9 +
                                                  [ctypes.c_void_p, ctypes.c_void_p])
+        L.hyq_select_vertical_mass_workspace.argtypes = [ctypes.c_int] * 9 + [ctypes.POINTER(ctypes.c_size_t)]
+        L.hyq_select_vertical_mass.argtypes = ([ctypes.c_void_p] * 2 + [ctypes.c_int] * 9 + [ctypes.c_float] +
+                                               [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p])
         L.hyq_quantize_blocks.argtypes = ([ctypes.c_void_p] + [ctypes.c_int] * 6 +
                                           [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p])
         L.hyq_hybrid_attention_prefill_workspace.argtypes = [ctypes.POINTER(AttnArgs), ctypes.POINTER(ctypes.c_size_t)]
@@ -115,6 +119,28 @@ def hyq_select_vertical(q: torch.Tensor, k: torch.Tensor, window: int, k_sel: in
     _check(lib().hyq_select_vertical(q.data_ptr(), k.data_ptr(), B, Hq, Hkv, Lq, Lk, D, window, n_tail, k_eff,
                                      out.data_ptr(), workspace.data_ptr(), workspace.numel(), _stream()),
            "hyq_select_vertical")
+    return out
+
+
+def hyq_select_vertical_mass(q: torch.Tensor, k: torch.Tensor, window: int, k_sel: int, n_queries: int = 0,
+                             softmax_scale: float = 0.0, workspace: torch.Tensor | None = None,
+                             out: torch.Tensor | None = None) -> torch.Tensor:
+    """Eq. 4-5: top-k of the softmax column mass of the last ``n_queries`` queries.  q [B,Hq,Lq,D],
+    k [B,Hkv,Lk,D] bf16 CUDA -> int32 [B,Hq,k_sel] ascending."""
+    _dev(q, torch.bfloat16, "q"), _dev(k, torch.bfloat16, "k")
+    B, Hq, Lq, D = q.shape
+    _, Hkv, Lk, _ = k.shape
+    k_eff = k_sel if Lk - window > 0 else 0
+    if out is None:
+        out = torch.empty(B, Hq, k_eff, dtype=torch.int32, device=q.device)
+    n = ctypes.c_size_t(0)
+    _check(lib().hyq_select_vertical_mass_workspace(B, Hq, Hkv, Lq, Lk, D, window, n_queries, k_eff, ctypes.byref(n)),
+           "hyq_select_vertical_mass_workspace")
+    if workspace is None:
+        workspace = torch.empty(max(int(n.value), 16), dtype=torch.uint8, device=q.device)
+    _check(lib().hyq_select_vertical_mass(q.data_ptr(), k.data_ptr(), B, Hq, Hkv, Lq, Lk, D, window, n_queries, k_eff,
+                                          softmax_scale, out.data_ptr(), workspace.data_ptr(), workspace.numel(),
+                                          _stream()), "hyq_select_vertical_mass")
     return out
 
 

@@ -83,6 +83,45 @@ int hyq_select_vertical_static(const void* q, const void* k_, int B, int Hq, int
     return launch_select_static(q, k_, B, Hq, Hkv, Lq, Lk, window, n_tail, k, idx_out, static_cast<cudaStream_t>(stream));
 }
 
+static int check_select_mass(int B, int Hq, int Hkv, int Lq, int Lk, int D, int window, int n_queries, int k, int* n_eff) {
+    if (n_queries < 0) return HYQ_ERR_INVALID_ARG;
+    const int rc = check_select(nullptr, nullptr, B, Hq, Hkv, Lq, Lk, D, window, n_queries, k);
+    if (rc != HYQ_OK) return rc;
+    const int tail = window < Lq ? window : Lq;
+    *n_eff = n_queries ? n_queries : tail;
+    const long P = (Lk - window > 0) ? (long)Lk - window : 0;
+    if (P == 0 || k == 0) return HYQ_OK;
+    if (Lq > Lk || *n_eff > tail || *n_eff <= 0) return HYQ_ERR_INVALID_ARG;
+    return HYQ_OK;
+}
+
+int hyq_select_vertical_mass_workspace(int B, int Hq, int Hkv, int Lq, int Lk, int D, int window, int n_queries, int k,
+                                       size_t* bytes) {
+    if (!bytes) return HYQ_ERR_INVALID_ARG;
+    int nT = 0;
+    const int rc = check_select_mass(B, Hq, Hkv, Lq, Lk, D, window, n_queries, k, &nT);
+    if (rc != HYQ_OK) return rc;
+    *bytes = select_mass_workspace_bytes(B, Hq, Lk, window, nT);
+    return HYQ_OK;
+}
+
+int hyq_select_vertical_mass(const void* q, const void* k_, int B, int Hq, int Hkv, int Lq, int Lk, int D, int window,
+                             int n_queries, int k, float softmax_scale, int32_t* idx_out, void* workspace,
+                             size_t workspace_bytes, void* stream) {
+    int nT = 0;
+    const int rc = check_select_mass(B, Hq, Hkv, Lq, Lk, D, window, n_queries, k, &nT);
+    if (rc != HYQ_OK) return rc;
+    const long P = (Lk - window > 0) ? (long)Lk - window : 0;
+    if (P == 0 || k == 0) return HYQ_OK;
+    if (!q || !k_ || !idx_out || !workspace) return HYQ_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k_) || !aligned16(workspace) || (reinterpret_cast<uintptr_t>(idx_out) & 3u))
+        return HYQ_ERR_ALIGNMENT;
+    if (workspace_bytes < select_mass_workspace_bytes(B, Hq, Lk, window, nT)) return HYQ_ERR_WORKSPACE;
+    const double alpha = softmax_scale != 0.0f ? (double)softmax_scale : 1.0 / std::sqrt((double)D);
+    return launch_select_mass(q, k_, B, Hq, Hkv, Lq, Lk, window, nT, k, alpha, idx_out, workspace,
+                              static_cast<cudaStream_t>(stream));
+}
+
 int hyq_quantize_blocks(const void* x, int B, int H, int L, int D, int block_tokens, int format, void* codes_out,
                         float* scales_out, void* stream) {
     if (B <= 0 || H <= 0 || L <= 0) return HYQ_ERR_INVALID_ARG;

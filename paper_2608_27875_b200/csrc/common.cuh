@@ -27,6 +27,10 @@ int launch_quantize(const void* x, long n_heads, int L, int format, void* codes,
 int launch_select(const void* q, const void* k, int B, int Hq, int Hkv, int Lq, int Lk, int window, int n_tail,
                   int k_sel, int32_t* idx_out, void* ws, cudaStream_t st);
 size_t select_workspace_bytes(int B, int Hq, int Lk, int window);
+int launch_topk(const double* scores, long rows, int P, int k_sel, int32_t* idx_out, cudaStream_t st);
+size_t select_mass_workspace_bytes(int B, int Hq, int Lk, int window, int n_queries);
+int launch_select_mass(const void* q, const void* k, int B, int Hq, int Hkv, int Lq, int Lk, int window, int n_queries,
+                       int k_sel, double alpha, int32_t* idx_out, void* ws, cudaStream_t st);
 int launch_select_static(const void* q, const void* k, int B, int Hq, int Hkv, int Lq, int Lk, int window, int n_tail,
                          int k_sel, int32_t* idx_out, cudaStream_t st);
 

@@ -228,6 +228,12 @@ int launch_select(const void* q, const void* k, int B, int Hq, int Hkv, int Lq, 
     return launch_status();
 }
 
+// top-k of `rows` score rows of length P (shared with the column-mass selector)
+int launch_topk(const double* scores, long rows, int P, int k_sel, int32_t* idx_out, cudaStream_t st) {
+    topk_kernel<<<(unsigned)rows, TOPK_THREADS, 0, st>>>(scores, P, k_sel, idx_out);
+    return launch_status();
+}
+
 // -------------------------------------------------------------------------------------------
 // Selection without caller-provided scratch: the tail means and the fp64 scores live in a fixed array
 // that is part of the library image on every device that loads it.
