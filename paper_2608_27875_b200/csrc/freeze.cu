@@ -14,6 +14,7 @@
 namespace hyq {
 
 constexpr int FRZ_THREADS = 128;
+constexpr int FRZ_WIN = 128;         // vertical indices staged per group for the source-row search
 
 // Source position of compacted row p: p + j with j the number of vertical indices below it,
 // i.e. the smallest j with idx[j] - j > p (idx ascending, so idx[j] - j never decreases).
@@ -54,11 +55,43 @@ freeze_quantize_kernel(const uint4* __restrict__ k_, const uint4* __restrict__ v
     const int32_t* hidx = idx + head * k_vl;
 
     __shared__ int src[64];
+    __shared__ int win[FRZ_WIN], j0_sh;
     __shared__ float warp_max[FRZ_THREADS / 32];
     __shared__ __align__(16) uint8_t vtile[4 * DEC_VTILE_BYTES];
+    // Source rows of the group's 64 compacted rows in three dependent memory round trips instead of ten:
+    // warp 0 finds j0 = the number of vertical rows before the group's first row by a 32-way search, a window of
+    // the index list starting there goes to shared memory, and each row finishes its own search in that window
+    // (a row whose answer lies beyond the window - long runs of vertical rows - falls back to the global search).
+    const int p0 = grp * 64;
+    if (threadIdx.x < 32) {
+        int lo = 0, hi = k_vl;                              // smallest j in [lo, hi] with idx[j] - j > p0
+        while (lo < hi) {
+            const int step = (hi - lo + 31) >> 5;
+            const int pos = lo + (int)threadIdx.x * step;
+            const bool below = pos < hi && __ldg(hidx + pos) - pos <= p0;      // predicate still false at pos
+            const int f = __popc(__ballot_sync(0xffffffffu, below));            // falses form a prefix of the lanes
+            const int new_lo = f ? lo + (f - 1) * step + 1 : lo;
+            const int new_hi = f == 0 ? lo : (f < 32 && lo + f * step < hi ? lo + f * step : hi);
+            lo = new_lo; hi = new_hi;
+        }
+        if (threadIdx.x == 0) j0_sh = lo;
+    }
+    __syncthreads();
+    const int j0 = j0_sh;
+    if (threadIdx.x < FRZ_WIN) win[threadIdx.x] = j0 + (int)threadIdx.x < k_vl ? __ldg(hidx + j0 + threadIdx.x) : 0x7fffffff;
+    __syncthreads();
     if (threadIdx.x < 64) {
-        const int p = grp * 64 + threadIdx.x;
-        src[threadIdx.x] = p < nQ ? source_row(hidx, k_vl, p) : -1;
+        const int p = p0 + threadIdx.x;
+        int s = -1;
+        if (p < nQ) {
+            int lo = 0, hi = FRZ_WIN;                       // smallest w with win[w] - (j0 + w) > p
+            while (lo < hi) {
+                const int mid = (lo + hi) >> 1;
+                if (win[mid] == 0x7fffffff || win[mid] - (j0 + mid) > p) hi = mid; else lo = mid + 1;
+            }
+            s = lo < FRZ_WIN ? p + j0 + lo : source_row(hidx, k_vl, p);
+        }
+        src[threadIdx.x] = s;
     }
     __syncthreads();
 

@@ -94,7 +94,8 @@ def test_freeze_of_an_all_zero_group_and_clustered_vertical_rows():
     B, Hkv, N, W = 1, 2, 700, 60
     K, V = rand_bf16((B, Hkv, N, 128), 4), rand_bf16((B, Hkv, N, 128), 5)
     K[:, :, 100:300] = 0
-    idx = np.tile(np.concatenate([np.arange(0, 40), np.arange(320, 330), np.arange(630, 640)]).astype(np.int32), (B, Hkv, 1))
+    idx = np.tile(np.concatenate([np.arange(0, 40), np.arange(320, 330), np.arange(400, 600),     # a run longer than the
+                                  np.arange(630, 640)]).astype(np.int32), (B, Hkv, 1))            # kernel's index window
     ref, cache = _freeze_both(K, V, idx, W, Hq=Hkv)
     assert (ref["kq_scales"] == 0).any()
     _assert_cache_equal(ref, cache)
