@@ -35,6 +35,8 @@
  *                 instruction that accumulates P.V.
  *       kq_scales, vq_scales  [B,Hkv,nQp/64] fp32.
  *
+ * With capacities set (cap_* fields) the row counts after [B,Hkv, in the shapes above are the capacities.
+ *
  * (Quant(.; G) over compacted rows, and one vertical set per KV head given by the caller, are this
  * library's readings: Algorithm 4 does not say how groups are cut after rows are removed, and Algorithm 1
  * yields one set per query head.)
@@ -68,6 +70,11 @@ typedef struct {
   void* v_win;
   void* k_s;
   void* v_s;
+  /* Row capacities per (b, KV head) of the quantized, vertical and window buffers, i.e. the strides between
+   * heads: 0 = tight (nQp, k, W' as derived from N, window, k).  Larger capacities let sequences of different
+   * lengths share one batch allocation (see hyq_hybrid_attention_decode_ragged); cap_quantized_rows must be a
+   * multiple of 64 and each capacity at least the tight value. */
+  int32_t cap_quantized_rows, cap_vertical, cap_window;
 } hyq_kv_cache;
 
 typedef struct {
@@ -110,6 +117,20 @@ int hyq_hybrid_attention_decode_workspace(const hyq_kv_cache* cache, int splits,
 int hyq_hybrid_attention_decode(const void* q, const hyq_kv_cache* cache, float softmax_scale, int splits,
                                 int out_dtype, void* out, float* lse, void* workspace, size_t workspace_bytes,
                                 void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * hyq_hybrid_attention_decode_ragged - the same attention for a batch of sequences of DIFFERENT lengths
+ * (the serving case: every sequence has its own prefix length, vertical count and staging fill).
+ *   `cache` describes the allocation: B sequences, strides given by the capacities (tight values if 0), and
+ *   N / window / k / n_staging are upper bounds only.  lengths [B][4] int32 (device): for sequence b the valid
+ *   rows {quantized, vertical, window, staging}, each at most the corresponding capacity, at least one row in
+ *   total.  Sequence b's buffers are what hyq_freeze writes when called with B = 1, that sequence's own
+ *   N / window / k, the batch's capacities, and the buffer pointers advanced to sequence b.
+ *   Everything else as hyq_hybrid_attention_decode (same kernels; the slices of a head are cut from its own rows).
+ * ------------------------------------------------------------------------------------------- */
+int hyq_hybrid_attention_decode_ragged(const void* q, const hyq_kv_cache* cache, const int32_t* lengths,
+                                       float softmax_scale, int splits, int out_dtype, void* out, float* lse,
+                                       void* workspace, size_t workspace_bytes, void* stream);
 
 #ifdef __cplusplus
 }

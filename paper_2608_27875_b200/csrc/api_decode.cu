@@ -15,6 +15,10 @@ static int check_cache(const hyq_kv_cache* c, bool need_pointers) {
     if (c->D != HYQ_D || c->group != 64 || c->format != HYQ_FMT_INT4 || c->Hq / c->Hkv > DEC_MAX_GROUP)
         return HYQ_ERR_UNSUPPORTED;
     if ((long)c->B * c->Hkv > 65535) return HYQ_ERR_UNSUPPORTED;
+    if (c->cap_quantized_rows < 0 || c->cap_vertical < 0 || c->cap_window < 0) return HYQ_ERR_INVALID_ARG;
+    if ((c->cap_quantized_rows && (c->cap_quantized_rows % 64 || c->cap_quantized_rows < g.nQp)) ||
+        (c->cap_vertical && c->cap_vertical < c->k) || (c->cap_window && c->cap_window < g.W))
+        return HYQ_ERR_INVALID_ARG;
     if (!need_pointers) return HYQ_OK;
     if (g.nQ > 0 && (!c->kq_codes || !c->vq_codes || !c->kq_scales || !c->vq_scales)) return HYQ_ERR_INVALID_ARG;
     if (c->k > 0 && (!c->k_vl || !c->v_vl)) return HYQ_ERR_INVALID_ARG;
@@ -36,11 +40,11 @@ int hyq_kv_cache_query_sizes(const hyq_kv_cache* cache, hyq_kv_cache_sizes* size
     const size_t heads = (size_t)cache->B * cache->Hkv;
     sizes->quantized_rows = g.nQ;
     sizes->padded_rows = g.nQp;
-    sizes->kq_codes_bytes = heads * g.nQp * (HYQ_D / 2);
-    sizes->vq_codes_bytes = heads * g.nQp * (HYQ_D / 2);
-    sizes->scales_bytes = heads * (g.nQp / 64) * sizeof(float);
-    sizes->vertical_bytes = heads * cache->k * HYQ_D * 2;
-    sizes->window_bytes = heads * g.W * HYQ_D * 2;
+    sizes->kq_codes_bytes = heads * g.sQ * (HYQ_D / 2);
+    sizes->vq_codes_bytes = heads * g.sQ * (HYQ_D / 2);
+    sizes->scales_bytes = heads * (g.sQ / 64) * sizeof(float);
+    sizes->vertical_bytes = heads * g.sK * HYQ_D * 2;
+    sizes->window_bytes = heads * g.sW * HYQ_D * 2;
     sizes->staging_bytes = heads * cache->staging_capacity * HYQ_D * 2;
     return HYQ_OK;
 }
@@ -71,7 +75,21 @@ int hyq_hybrid_attention_decode(const void* q, const hyq_kv_cache* cache, float 
     const int s = splits > 0 ? splits : decode_auto_splits(*cache);
     if (workspace_bytes < decode_workspace_bytes(*cache, s)) return HYQ_ERR_WORKSPACE;
     const float alpha = softmax_scale != 0.0f ? softmax_scale : 1.0f / std::sqrt((float)cache->D);
-    return launch_decode(q, *cache, alpha, s, out_dtype, out, lse, workspace, static_cast<cudaStream_t>(stream));
+    return launch_decode(q, *cache, nullptr, alpha, s, out_dtype, out, lse, workspace, static_cast<cudaStream_t>(stream));
+}
+
+int hyq_hybrid_attention_decode_ragged(const void* q, const hyq_kv_cache* cache, const int32_t* lengths, float softmax_scale,
+                                       int splits, int out_dtype, void* out, float* lse, void* workspace,
+                                       size_t workspace_bytes, void* stream) {
+    const int rc = check_cache(cache, true);
+    if (rc != HYQ_OK) return rc;
+    if (!q || !out || !workspace || !lengths || splits < 0 || splits > 1024) return HYQ_ERR_INVALID_ARG;
+    if (out_dtype != 0 && out_dtype != 1) return HYQ_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(out) || !aligned16(workspace) || !aligned16(lengths)) return HYQ_ERR_ALIGNMENT;
+    const int s = splits > 0 ? splits : decode_auto_splits(*cache);
+    if (workspace_bytes < decode_workspace_bytes(*cache, s)) return HYQ_ERR_WORKSPACE;
+    const float alpha = softmax_scale != 0.0f ? softmax_scale : 1.0f / std::sqrt((float)cache->D);
+    return launch_decode(q, *cache, lengths, alpha, s, out_dtype, out, lse, workspace, static_cast<cudaStream_t>(stream));
 }
 
 }  // extern "C"

@@ -48,9 +48,11 @@ constexpr int DEC_STAGE_BYTES = 2048;       // 1 KB K codes + 1 KB V codes
 constexpr float DEC_RAISE = 8.0f;          // log2 units; P <= 2^8 stays far inside fp16 / bf16 range
 
 struct DecParams {
-    int g, splits;
-    long nQ, nQp;
-    int k, W, n_s, Ws;
+    int g, splits, Hkv;
+    long nQ, sQ;         // quantized rows per head (valid), rows between heads
+    int k, W, n_s;       // valid rows of the vertical, window and staging buffers ...
+    int sK, sW, Ws;      // ... and rows between heads
+    const int4* lens;    // optional per-sequence {quantized, vertical, window, staging} valid rows (ragged batch)
     float scale_log2;
     const uint8_t* kq; const uint8_t* vq; const float* ks; const float* vs;
     const uint4 *k_vl, *v_vl, *k_s, *v_s, *k_win, *v_win;
@@ -295,8 +297,14 @@ decode_kernel(const DecParams p) {
     }
     __syncthreads();
 
-    const long Tq = (p.nQ + 15) / 16;
-    const int Tvl = (p.k + 15) / 16, Ts = (p.n_s + 15) / 16, Tw = (p.W + 15) / 16;
+    long nQ = p.nQ;
+    int n_vl = p.k, n_win = p.W, n_stg = p.n_s;
+    if (p.lens) {                                           // ragged batch: this sequence's own row counts
+        const int4 l = __ldg(p.lens + unit / p.Hkv);
+        nQ = l.x; n_vl = l.y; n_win = l.z; n_stg = l.w;
+    }
+    const long Tq = (nQ + 15) / 16;
+    const int Tvl = (n_vl + 15) / 16, Ts = (n_stg + 15) / 16, Tw = (n_win + 15) / 16;
     // Every slice takes the same share of the INT4 tiles AND of the bf16 tiles (a bf16 tile moves four times the
     // bytes and goes through a different loop), so all CTAs of a head carry the same mix of work.
     const long Tf = Tvl + Ts + Tw;
@@ -330,11 +338,11 @@ decode_kernel(const DecParams p) {
         // of its use; one commit group per tile (empty past the end) keeps the group arithmetic uniform.
         const long t0 = q_lo + warp;
         const int n_my = (int)((q_hi - t0 + DEC_WARPS - 1) / DEC_WARPS);
-        const bool has_ragged = (p.nQ & 15) && t0 + (long)(n_my - 1) * DEC_WARPS == Tq - 1;
-        const uint8_t* gk = p.kq + unit * p.nQp * 64 + t0 * 1024 + lane * 16;
-        const uint8_t* gv = p.vq + unit * (p.nQp / 16) * DEC_VTILE_BYTES + t0 * 1024 + lane * 16;
-        const float* pks = p.ks + unit * (p.nQp / 64) + (t0 >> 2);
-        const float* pvs = p.vs + unit * (p.nQp / 64) + (t0 >> 2);
+        const bool has_ragged = (nQ & 15) && t0 + (long)(n_my - 1) * DEC_WARPS == Tq - 1;
+        const uint8_t* gk = p.kq + unit * p.sQ * 64 + t0 * 1024 + lane * 16;
+        const uint8_t* gv = p.vq + unit * (p.sQ / 16) * DEC_VTILE_BYTES + t0 * 1024 + lane * 16;
+        const float* pks = p.ks + unit * (p.sQ / 64) + (t0 >> 2);
+        const float* pvs = p.vs + unit * (p.sQ / 64) + (t0 >> 2);
         const uint32_t ring = (uint32_t)__cvta_generic_to_shared(ring_mem) + warp * (DEC_STAGES * DEC_STAGE_BYTES) + lane * 16;
         auto issue = [&](uint32_t stage_addr) {
             cp_async16(stage_addr, gk); cp_async16(stage_addr + 512, gk + 512);
@@ -373,7 +381,7 @@ decode_kernel(const DecParams p) {
             cp_async_wait<DEC_STAGES - 1>();                // tile i has landed
             QTile A;
             fetch(A, i);
-            if (i >= n_full) quant_tile<true>(A, qf, kscale, b0, b1, (int)(p.nQ & 15), r, st, acc);
+            if (i >= n_full) quant_tile<true>(A, qf, kscale, b0, b1, (int)(nQ & 15), r, st, acc);
             else quant_tile<false>(A, qf, kscale, b0, b1, 16, r, st, acc);
         }
     }
@@ -394,9 +402,9 @@ decode_kernel(const DecParams p) {
             long u = t - Tq;
             const uint4 *kseg, *vseg;
             int n;
-            if (u < Tvl) { kseg = p.k_vl + unit * p.k * 16; vseg = p.v_vl + unit * p.k * 16; n = p.k; }
-            else if ((u -= Tvl) < Ts) { kseg = p.k_s + unit * p.Ws * 16; vseg = p.v_s + unit * p.Ws * 16; n = p.n_s; }
-            else { u -= Ts; kseg = p.k_win + unit * p.W * 16; vseg = p.v_win + unit * p.W * 16; n = p.W; }
+            if (u < Tvl) { kseg = p.k_vl + unit * p.sK * 16; vseg = p.v_vl + unit * p.sK * 16; n = n_vl; }
+            else if ((u -= Tvl) < Ts) { kseg = p.k_s + unit * p.Ws * 16; vseg = p.v_s + unit * p.Ws * 16; n = n_stg; }
+            else { u -= Ts; kseg = p.k_win + unit * p.sW * 16; vseg = p.v_win + unit * p.sW * 16; n = n_win; }
             const int row0 = (int)u * 16;
             const int ra = min(row0 + r, n - 1), rb = min(row0 + r + 8, n - 1);
             uint4 ka[4], kb[4];
@@ -507,7 +515,7 @@ decode_merge_kernel(const float* __restrict__ part_acc, const float* __restrict_
     float A = 0.0f;
 #pragma unroll 8
     for (int s = 0; s < splits; ++s) A += __ldg(part_acc + (slot0 + (long)s * DEC_MAX_GROUP) * HYQ_D + threadIdx.x) * wt[s];
-    const float o = A / L;
+    const float o = L > 0.0f ? A / L : 0.0f;               // a sequence with no cached row at all: zeros
     const long oi = (unit * g + h) * HYQ_D + threadIdx.x;
     if (out_fp32) static_cast<float*>(out)[oi] = o;
     else static_cast<__nv_bfloat16*>(out)[oi] = __float2bfloat16_rn(o);
@@ -534,13 +542,15 @@ size_t decode_workspace_bytes(const hyq_kv_cache& c, int splits) {
     return align_up(slots * HYQ_D * sizeof(float), 16) + align_up(slots * 2 * sizeof(float), 16);
 }
 
-int launch_decode(const void* q, const hyq_kv_cache& c, float alpha, int splits, int out_dtype, void* out, float* lse,
-                  void* workspace, cudaStream_t st) {
+int launch_decode(const void* q, const hyq_kv_cache& c, const int32_t* lengths, float alpha, int splits, int out_dtype,
+                  void* out, float* lse, void* workspace, cudaStream_t st) {
     const CacheGeo geo = cache_geo(c);
     const long units = (long)c.B * c.Hkv;
     DecParams p;
     p.g = c.Hq / c.Hkv; p.splits = splits;
-    p.nQ = geo.nQ; p.nQp = geo.nQp; p.k = c.k; p.W = geo.W; p.n_s = c.n_staging; p.Ws = c.staging_capacity;
+    p.Hkv = c.Hkv; p.lens = reinterpret_cast<const int4*>(lengths);
+    p.nQ = geo.nQ; p.sQ = geo.sQ; p.k = c.k; p.W = geo.W; p.n_s = c.n_staging;
+    p.sK = (int)geo.sK; p.sW = (int)geo.sW; p.Ws = c.staging_capacity;
     p.scale_log2 = alpha * 1.4426950408889634f;
     p.kq = static_cast<const uint8_t*>(c.kq_codes); p.vq = static_cast<const uint8_t*>(c.vq_codes);
     p.ks = c.kq_scales; p.vs = c.vq_scales;

@@ -12,6 +12,7 @@ constexpr int DEC_MAX_GROUP = 8;           // query heads per KV head (the n = 8
 struct CacheGeo {
     int W;              // rows in the window buffers: min(window, N)
     long nQ, nQp;       // quantized rows per head: valid, padded to whole groups of 64
+    long sQ, sK, sW;    // rows between consecutive heads in the quantized, vertical and window buffers
 };
 
 static inline CacheGeo cache_geo(const hyq_kv_cache& c) {
@@ -19,6 +20,9 @@ static inline CacheGeo cache_geo(const hyq_kv_cache& c) {
     g.W = c.window < c.N ? c.window : c.N;
     g.nQ = (long)c.N - g.W - c.k;
     g.nQp = (g.nQ + 63) / 64 * 64;
+    g.sQ = c.cap_quantized_rows ? c.cap_quantized_rows : g.nQp;
+    g.sK = c.cap_vertical ? c.cap_vertical : c.k;
+    g.sW = c.cap_window ? c.cap_window : g.W;
     return g;
 }
 
@@ -34,7 +38,7 @@ __host__ __device__ __forceinline__ int vq_byte_offset(int key, int d) {
 int launch_freeze(const void* k_, const void* v, const int32_t* vl_idx, const hyq_kv_cache& c, cudaStream_t st);
 int decode_auto_splits(const hyq_kv_cache& c);
 size_t decode_workspace_bytes(const hyq_kv_cache& c, int splits);
-int launch_decode(const void* q, const hyq_kv_cache& c, float alpha, int splits, int out_dtype, void* out, float* lse,
-                  void* workspace, cudaStream_t st);
+int launch_decode(const void* q, const hyq_kv_cache& c, const int32_t* lengths, float alpha, int splits, int out_dtype,
+                  void* out, float* lse, void* workspace, cudaStream_t st);
 
 }  // namespace hyq

@@ -29,7 +29,7 @@ __device__ __forceinline__ int source_row(const int32_t* __restrict__ idx, int k
 
 __global__ void __launch_bounds__(FRZ_THREADS)
 gather_rows_kernel(const uint4* __restrict__ k_, const uint4* __restrict__ v, const int32_t* __restrict__ idx,
-                   int N, int W, int k_vl, uint4* __restrict__ k_vl_out, uint4* __restrict__ v_vl_out,
+                   int N, int W, int k_vl, long sK, long sW, uint4* __restrict__ k_vl_out, uint4* __restrict__ v_vl_out,
                    uint4* __restrict__ k_win, uint4* __restrict__ v_win) {
     const long head = blockIdx.y;
     const int o = blockIdx.x * 8 + (threadIdx.x >> 4);
@@ -39,14 +39,14 @@ gather_rows_kernel(const uint4* __restrict__ k_, const uint4* __restrict__ v, co
     const bool vl = o < k_vl;
     const int src = vl ? __ldg(idx + head * k_vl + o) : P + (o - k_vl);
     const long s = (head * N + src) * 16 + c;
-    const long d = vl ? (head * k_vl + o) * 16 + c : (head * W + (o - k_vl)) * 16 + c;
+    const long d = vl ? (head * sK + o) * 16 + c : (head * sW + (o - k_vl)) * 16 + c;
     (vl ? k_vl_out : k_win)[d] = __ldg(k_ + s);
     (vl ? v_vl_out : v_win)[d] = __ldg(v + s);
 }
 
 __global__ void __launch_bounds__(FRZ_THREADS)
 freeze_quantize_kernel(const uint4* __restrict__ k_, const uint4* __restrict__ v, const int32_t* __restrict__ idx,
-                       int N, int k_vl, int nQ, int nQp, uint8_t* __restrict__ kq, uint8_t* __restrict__ vq,
+                       int N, int k_vl, int nQ, long nQp, uint8_t* __restrict__ kq, uint8_t* __restrict__ vq,
                        float* __restrict__ ks, float* __restrict__ vs) {
     const int grp = blockIdx.x;
     const long head = blockIdx.y;
@@ -163,13 +163,13 @@ int launch_freeze(const void* k_, const void* v, const int32_t* vl_idx, const hy
     const uint4* v4 = static_cast<const uint4*>(v);
     if (c.k + g.W > 0) {
         const dim3 grid((unsigned)((c.k + g.W + 7) / 8), (unsigned)heads);
-        gather_rows_kernel<<<grid, FRZ_THREADS, 0, st>>>(k4, v4, vl_idx, c.N, g.W, c.k, static_cast<uint4*>(c.k_vl),
+        gather_rows_kernel<<<grid, FRZ_THREADS, 0, st>>>(k4, v4, vl_idx, c.N, g.W, c.k, g.sK, g.sW, static_cast<uint4*>(c.k_vl),
                                                          static_cast<uint4*>(c.v_vl), static_cast<uint4*>(c.k_win),
                                                          static_cast<uint4*>(c.v_win));
     }
     if (g.nQ > 0) {
         const dim3 grid((unsigned)(g.nQp / 64), (unsigned)heads, 2);
-        freeze_quantize_kernel<<<grid, FRZ_THREADS, 0, st>>>(k4, v4, vl_idx, c.N, c.k, (int)g.nQ, (int)g.nQp,
+        freeze_quantize_kernel<<<grid, FRZ_THREADS, 0, st>>>(k4, v4, vl_idx, c.N, c.k, (int)g.nQ, g.sQ,
                                                              static_cast<uint8_t*>(c.kq_codes),
                                                              static_cast<uint8_t*>(c.vq_codes), c.kq_scales, c.vq_scales);
     }

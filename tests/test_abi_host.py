@@ -142,6 +142,14 @@ def test_decode_side_argument_checks(lib):
         args = dict(B=2, Hq=32, Hkv=8, N=1000, window=100, k=37)
         args.update(kw)
         assert L.hyq_kv_cache_query_sizes(ctypes.byref(decode_api.make_desc(**args)), ctypes.byref(sizes)) == code, kw
+    caps = decode_api.make_desc(B=2, Hq=32, Hkv=8, N=1000, window=100, k=37, cap_quantized_rows=1024, cap_vertical=64, cap_window=128)
+    assert L.hyq_kv_cache_query_sizes(ctypes.byref(caps), ctypes.byref(sizes)) == 0
+    assert sizes.kq_codes_bytes == 16 * 1024 * 64 and sizes.vertical_bytes == 16 * 64 * 256 and sizes.window_bytes == 16 * 128 * 256
+    for kw in (dict(cap_quantized_rows=1000), dict(cap_quantized_rows=832), dict(cap_vertical=36), dict(cap_window=99)):
+        args = dict(B=2, Hq=32, Hkv=8, N=1000, window=100, k=37)
+        args.update(kw)
+        assert L.hyq_kv_cache_query_sizes(ctypes.byref(decode_api.make_desc(**args)), ctypes.byref(sizes)) == 1, kw
+    assert L.hyq_hybrid_attention_decode_ragged(None, ctypes.byref(d), None, 0.0, 0, 0, None, None, None, 0, None) == 1
     d.struct_size = 8
     assert L.hyq_kv_cache_query_sizes(ctypes.byref(d), ctypes.byref(sizes)) == 1
     d.struct_size = ctypes.sizeof(decode_api.KvCacheDesc)

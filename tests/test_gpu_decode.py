@@ -164,3 +164,37 @@ def test_decode_at_benchmark_size_and_repeatable():
     assert mx <= MAX_ABS_TOL and rel <= MEAN_REL_TOL, (mx, rel)
     assert torch.equal(got, again)
     assert oracle_k == cache.desc.k
+
+
+def test_ragged_batch_matches_the_oracle_sequence_by_sequence():
+    """Sequences of different lengths, vertical counts and staging fills in one allocation (capacity strides) and
+    one launch: every sequence against its own oracle cache; a sequence shorter than the window has no prefix."""
+    Hq, Hkv, W = 8, 2, 64
+    seqs = [(1000, 37, 5), (333, 0, 0), (40, 0, 3), (2000, 100, 128), (129, 1, 1)]          # N, k, staged rows
+    rc = dapi.RaggedKvCache(len(seqs), Hq, Hkv, max_N=2000, window=W, max_k=100)
+    refs, qs = [], []
+    for b, (N, kk, n_s) in enumerate(seqs):
+        K, V = rand_bf16((1, Hkv, N, 128), 40 + b, 1.3), rand_bf16((1, Hkv, N, 128), 50 + b)
+        idx = _idx(1, Hkv, N - min(W, N), kk, 60 + b) if kk else None
+        ref = od.freeze(wl.bits(K), wl.bits(V), idx, W)
+        rc.freeze_sequence(b, K.cuda(), V.cuda(), None if idx is None else torch.from_numpy(idx).cuda())
+        for i in range(n_s):
+            kn, vn = rand_bf16((1, Hkv, 128), 700 + 10 * b + i), rand_bf16((1, Hkv, 128), 900 + 10 * b + i)
+            od.append_staging(ref, wl.bits(kn), wl.bits(vn))
+            rc.append(b, kn[0].cuda(), vn[0].cuda())
+        refs.append(ref)
+        qs.append(rand_bf16((1, Hq, 128), 80 + b, 1.5))
+    q = torch.cat(qs)
+    assert rc.lengths_host.tolist() == [[r["nQ"], r["k"], r["window"], r["n_s"]] for r in refs]
+    for splits in (0, 1, 7):
+        got = dapi.hyq_hybrid_attention_decode_ragged(q.cuda(), rc, splits=splits, out_dtype=torch.float32)
+        torch.cuda.synchronize()
+        for b, ref in enumerate(refs):
+            want, _ = od.decode_attention(wl.bits(qs[b]), ref)
+            mx, rel = errors(got[b:b + 1].cpu().numpy(), want)
+            assert mx <= MAX_ABS_TOL and rel <= MEAN_REL_TOL, (splits, b, mx, rel)
+    # the frozen codes of a sequence inside the batch allocation are those of a stand-alone Freeze
+    b = 3
+    nq = refs[b]["nQ"]
+    assert np.array_equal(rc.batch.buffers["kq_codes"][b, :, :nq].cpu().numpy(), refs[b]["kq_codes"][0])
+    assert np.array_equal(_v_tiles_to_rows(rc.batch.buffers["vq_codes"][b].cpu().numpy())[:, :nq], refs[b]["vq_codes"][0])
