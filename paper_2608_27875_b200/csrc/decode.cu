@@ -267,6 +267,9 @@ decode_kernel(const DecParams p) {
     const int split = blockIdx.x;
     const long unit = blockIdx.y;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, r = lane >> 2, j = lane & 3;
+    // the merge kernel may be made resident while this grid runs (programmatic dependent launch): it waits for
+    // this grid's completion before it reads anything, so only its launch latency is taken off the path
+    asm volatile("griddepcontrol.launch_dependents;");
 
     __shared__ __align__(16) uint16_t qs[DEC_MAX_GROUP][HYQ_D];      // bf16 bits, heads >= g zero
     __shared__ float red_ml[DEC_WARPS][DEC_MAX_GROUP][2];
@@ -488,6 +491,7 @@ decode_merge_kernel(const float* __restrict__ part_acc, const float* __restrict_
                     int out_fp32, void* __restrict__ out, float* __restrict__ lse) {
     const long unit = blockIdx.x;
     const int h = blockIdx.y;
+    asm volatile("griddepcontrol.wait;" ::: "memory");       // the slice kernel has completed and its results are visible
     __shared__ float wt[DEC_MAX_SPLITS];
     __shared__ float red[2][HYQ_D / 32];
     const long slot0 = unit * splits * DEC_MAX_GROUP + h;          // slice s sits at slot0 + s * DEC_MAX_GROUP
@@ -569,7 +573,18 @@ int launch_decode(const void* q, const hyq_kv_cache& c, const int32_t* lengths, 
         attr_set = true;
     }
     decode_kernel<<<dim3((unsigned)splits, (unsigned)units), DEC_THREADS, ring_bytes, st>>>(p);
-    decode_merge_kernel<<<dim3((unsigned)units, (unsigned)p.g), HYQ_D, 0, st>>>(p.part_acc, p.part_ml, p.g, splits, out_dtype, out, lse);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)units, (unsigned)p.g);
+    cfg.blockDim = dim3(HYQ_D);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const float* pa = p.part_acc;
+    const float* pm = p.part_ml;
+    if (cudaLaunchKernelEx(&cfg, decode_merge_kernel, pa, pm, p.g, splits, out_dtype, out, lse) != cudaSuccess) return HYQ_ERR_CUDA;
     return launch_status();
 }
 
