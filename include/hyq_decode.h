@@ -18,10 +18,10 @@
  *                              counts them in n_staging.  Folding staged rows into the other buffers
  *                              is not described by the paper and not part of this library.
  *   quantized    the other nQ = N - W' - k prefix rows, COMPACTED in ascending position order and cut
- *                into groups of `group` (64) consecutive compacted rows x all D channels; each group is
+ *                into groups of `group` (G = 32, 64 or 128) consecutive compacted rows x all D channels; each group is
  *                quantized exactly as hyq_quantize_blocks quantizes a tile (INT4, c_B = 7, fp32 scale
  *                per group; the last group may be ragged).  Per head the row count is padded to
- *                nQp = 64 * ceil(nQ / 64); padding rows hold unspecified codes and are never used.
+ *                nQp = G * ceil(nQ / G); padding rows hold unspecified codes and are never used.
  *       kq_codes  [B,Hkv,nQp,D/2] bytes: row-major, channel 2m in the low nibble and 2m+1 in the high
  *                 nibble of byte m, two's complement (hyq_quantize_blocks' INT4 layout).
  *       vq_codes  [B,Hkv,nQp/16,1024] bytes, FRAGMENT-MAJOR: the codes of 16 consecutive compacted rows
@@ -33,7 +33,7 @@
  *                 i.e. each lane of a warp reads two 16-byte pieces (the warp: two contiguous 512-byte
  *                 runs) and owns, without any shuffle, the operand registers of the warp-level matrix
  *                 instruction that accumulates P.V.
- *       kq_scales, vq_scales  [B,Hkv,nQp/64] fp32.
+ *       kq_scales, vq_scales  [B,Hkv,nQp/G] fp32.
  *
  * With capacities set (cap_* fields) the row counts after [B,Hkv, in the shapes above are the capacities.
  *
@@ -56,7 +56,7 @@ typedef struct {
   int32_t N;                    /* prefill rows frozen */
   int32_t window;               /* W; the window buffers hold min(W, N) rows */
   int32_t k;                    /* vertical rows per KV head, 0 <= k <= N - min(W, N) */
-  int32_t group;                /* G: must be 64 */
+  int32_t group;                /* G: 32, 64 or 128 rows per scale group */
   int32_t format;               /* K and V code format: must be HYQ_FMT_INT4 (K4V4) */
   int32_t staging_capacity;     /* W_s: rows allocated per head in k_s / v_s (may be 0) */
   int32_t n_staging;            /* valid staging rows, 0 <= n_staging <= staging_capacity */
@@ -73,7 +73,7 @@ typedef struct {
   /* Row capacities per (b, KV head) of the quantized, vertical and window buffers, i.e. the strides between
    * heads: 0 = tight (nQp, k, W' as derived from N, window, k).  Larger capacities let sequences of different
    * lengths share one batch allocation (see hyq_hybrid_attention_decode_ragged); cap_quantized_rows must be a
-   * multiple of 64 and each capacity at least the tight value. */
+   * multiple of G and each capacity at least the tight value. */
   int32_t cap_quantized_rows, cap_vertical, cap_window;
 } hyq_kv_cache;
 
@@ -94,7 +94,7 @@ int hyq_kv_cache_query_sizes(const hyq_kv_cache* cache, hyq_kv_cache_sizes* size
  * vertical and quantized buffers of `cache` (layouts above).  The staging buffers are not touched
  * (an empty staging buffer is n_staging = 0).  The prefill cache may be freed once the enqueued
  * work has completed.  Errors: INVALID_ARG (null pointer, sizes out of range, struct_size),
- * UNSUPPORTED (D != 128, group != 64, format != INT4, g > 8), ALIGNMENT (any buffer not 16-byte aligned).
+ * UNSUPPORTED (D != 128, group not 32 / 64 / 128, format != INT4, g > 8), ALIGNMENT (any buffer not 16-byte aligned).
  * ------------------------------------------------------------------------------------------- */
 int hyq_freeze(const void* k_, const void* v, const int32_t* vl_idx, const hyq_kv_cache* cache, void* stream);
 

@@ -10,13 +10,14 @@ static int check_cache(const hyq_kv_cache* c, bool need_pointers) {
     if (c->B <= 0 || c->Hq <= 0 || c->Hkv <= 0 || c->N <= 0 || c->window < 0 || c->k < 0) return HYQ_ERR_INVALID_ARG;
     if (c->Hq % c->Hkv) return HYQ_ERR_INVALID_ARG;
     if (c->staging_capacity < 0 || c->n_staging < 0 || c->n_staging > c->staging_capacity) return HYQ_ERR_INVALID_ARG;
+    if (c->D != HYQ_D || (c->group != 32 && c->group != 64 && c->group != 128) || c->format != HYQ_FMT_INT4 ||
+        c->Hq / c->Hkv > DEC_MAX_GROUP)
+        return HYQ_ERR_UNSUPPORTED;
     const CacheGeo g = cache_geo(*c);
     if (c->k > c->N - g.W) return HYQ_ERR_INVALID_ARG;
-    if (c->D != HYQ_D || c->group != 64 || c->format != HYQ_FMT_INT4 || c->Hq / c->Hkv > DEC_MAX_GROUP)
-        return HYQ_ERR_UNSUPPORTED;
     if ((long)c->B * c->Hkv > 65535) return HYQ_ERR_UNSUPPORTED;
     if (c->cap_quantized_rows < 0 || c->cap_vertical < 0 || c->cap_window < 0) return HYQ_ERR_INVALID_ARG;
-    if ((c->cap_quantized_rows && (c->cap_quantized_rows % 64 || c->cap_quantized_rows < g.nQp)) ||
+    if ((c->cap_quantized_rows && (c->cap_quantized_rows % c->group || c->cap_quantized_rows < g.nQp)) ||
         (c->cap_vertical && c->cap_vertical < c->k) || (c->cap_window && c->cap_window < g.W))
         return HYQ_ERR_INVALID_ARG;
     if (!need_pointers) return HYQ_OK;
@@ -42,7 +43,7 @@ int hyq_kv_cache_query_sizes(const hyq_kv_cache* cache, hyq_kv_cache_sizes* size
     sizes->padded_rows = g.nQp;
     sizes->kq_codes_bytes = heads * g.sQ * (HYQ_D / 2);
     sizes->vq_codes_bytes = heads * g.sQ * (HYQ_D / 2);
-    sizes->scales_bytes = heads * (g.sQ / 64) * sizeof(float);
+    sizes->scales_bytes = heads * (g.sQ / cache->group) * sizeof(float);
     sizes->vertical_bytes = heads * g.sK * HYQ_D * 2;
     sizes->window_bytes = heads * g.sW * HYQ_D * 2;
     sizes->staging_bytes = heads * cache->staging_capacity * HYQ_D * 2;

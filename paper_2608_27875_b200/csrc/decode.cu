@@ -49,6 +49,7 @@ constexpr float DEC_RAISE = 8.0f;          // log2 units; P <= 2^8 stays far ins
 
 struct DecParams {
     int g, splits, Hkv;
+    int gshift;          // log2(rows per scale group / 16): 16-row tile t belongs to group t >> gshift
     long nQ, sQ;         // quantized rows per head (valid), rows between heads
     int k, W, n_s;       // valid rows of the vertical, window and staging buffers ...
     int sK, sW, Ws;      // ... and rows between heads
@@ -344,8 +345,9 @@ decode_kernel(const DecParams p) {
         const bool has_ragged = (nQ & 15) && t0 + (long)(n_my - 1) * DEC_WARPS == Tq - 1;
         const uint8_t* gk = p.kq + unit * p.sQ * 64 + t0 * 1024 + lane * 16;
         const uint8_t* gv = p.vq + unit * (p.sQ / 16) * DEC_VTILE_BYTES + t0 * 1024 + lane * 16;
-        const float* pks = p.ks + unit * (p.sQ / 64) + (t0 >> 2);
-        const float* pvs = p.vs + unit * (p.sQ / 64) + (t0 >> 2);
+        const int gshift = p.gshift;
+        const float* pks = p.ks + unit * (p.sQ >> (p.gshift + 4));
+        const float* pvs = p.vs + unit * (p.sQ >> (p.gshift + 4));
         const uint32_t ring = (uint32_t)__cvta_generic_to_shared(ring_mem) + warp * (DEC_STAGES * DEC_STAGE_BYTES) + lane * 16;
         auto issue = [&](uint32_t stage_addr) {
             cp_async16(stage_addr, gk); cp_async16(stage_addr + 512, gk + 512);
@@ -365,7 +367,8 @@ decode_kernel(const DecParams p) {
         auto fetch = [&](QTile& d, int i) {                 // ring stage of tile i -> registers, then refill it
             d.ka = lds128(stage_addr); d.kb = lds128(stage_addr + 512);
             d.va = lds128(stage_addr + 1024); d.vb = lds128(stage_addr + 1536);
-            d.fk = __ldg(pks + i); d.fv = __ldg(pvs + i);
+            const int grp = ((int)t0 + i * DEC_WARPS) >> gshift;
+            d.fk = __ldg(pks + grp); d.fv = __ldg(pvs + grp);
             if (i + DEC_STAGES < n_my) issue(stage_addr);   // own bytes only: no barrier
             cp_async_commit();
             stage_addr = (i % DEC_STAGES == DEC_STAGES - 1) ? ring : stage_addr + DEC_STAGE_BYTES;
@@ -552,6 +555,7 @@ int launch_decode(const void* q, const hyq_kv_cache& c, const int32_t* lengths, 
     const long units = (long)c.B * c.Hkv;
     DecParams p;
     p.g = c.Hq / c.Hkv; p.splits = splits;
+    p.gshift = c.group == 32 ? 1 : c.group == 64 ? 2 : 3;
     p.Hkv = c.Hkv; p.lens = reinterpret_cast<const int4*>(lengths);
     p.nQ = geo.nQ; p.sQ = geo.sQ; p.k = c.k; p.W = geo.W; p.n_s = c.n_staging;
     p.sK = (int)geo.sK; p.sW = (int)geo.sW; p.Ws = c.staging_capacity;

@@ -11,7 +11,7 @@ constexpr int DEC_MAX_GROUP = 8;           // query heads per KV head (the n = 8
 
 struct CacheGeo {
     int W;              // rows in the window buffers: min(window, N)
-    long nQ, nQp;       // quantized rows per head: valid, padded to whole groups of 64
+    long nQ, nQp;       // quantized rows per head: valid, padded to whole groups of G rows
     long sQ, sK, sW;    // rows between consecutive heads in the quantized, vertical and window buffers
 };
 
@@ -19,7 +19,8 @@ static inline CacheGeo cache_geo(const hyq_kv_cache& c) {
     CacheGeo g;
     g.W = c.window < c.N ? c.window : c.N;
     g.nQ = (long)c.N - g.W - c.k;
-    g.nQp = (g.nQ + 63) / 64 * 64;
+    const long G = c.group > 0 ? c.group : 64;
+    g.nQp = (g.nQ + G - 1) / G * G;
     g.sQ = c.cap_quantized_rows ? c.cap_quantized_rows : g.nQp;
     g.sK = c.cap_vertical ? c.cap_vertical : c.k;
     g.sW = c.cap_window ? c.cap_window : g.W;

@@ -2,9 +2,9 @@
 //
 // Two kernels, both HBM-bound and read-once / write-once:
 //   gather_rows_kernel     copies the vertical rows (by index) and the window rows (a slice) as bf16;
-//   freeze_quantize_kernel one CTA per group of 64 COMPACTED rows of one (b, kv head) and one tensor
+//   freeze_quantize_kernel one CTA per group of G (32, 64 or 128) COMPACTED rows of one (b, kv head) and one tensor
 //                          (K or V): finds the source rows (the complement of the ascending vertical
-//                          set, by binary search), quantizes the 64 x 128 group to INT4 with the
+//                          set, by binary search), quantizes the G x 128 group to INT4 with the
 //                          arithmetic of the per-tile quantizer (fp32, one rounding per operation), and
 //                          writes K row-major and V in the fragment-major tile layout the decode kernel
 //                          loads straight into matrix-instruction operand registers.
@@ -13,7 +13,7 @@
 
 namespace hyq {
 
-constexpr int FRZ_THREADS = 128;
+constexpr int FRZ_THREADS = 128;     // gather kernel; the quantizer runs 2 * G threads (64 elements per thread)
 constexpr int FRZ_WIN = 128;         // vertical indices staged per group for the source-row search
 
 // Source position of compacted row p: p + j with j the number of vertical indices below it,
@@ -44,7 +44,8 @@ gather_rows_kernel(const uint4* __restrict__ k_, const uint4* __restrict__ v, co
     (vl ? v_vl_out : v_win)[d] = __ldg(v + s);
 }
 
-__global__ void __launch_bounds__(FRZ_THREADS)
+template <int G>
+__global__ void __launch_bounds__(2 * G)
 freeze_quantize_kernel(const uint4* __restrict__ k_, const uint4* __restrict__ v, const int32_t* __restrict__ idx,
                        int N, int k_vl, int nQ, long nQp, uint8_t* __restrict__ kq, uint8_t* __restrict__ vq,
                        float* __restrict__ ks, float* __restrict__ vs) {
@@ -54,15 +55,16 @@ freeze_quantize_kernel(const uint4* __restrict__ k_, const uint4* __restrict__ v
     const uint4* x = (is_v ? v : k_) + head * N * 16;
     const int32_t* hidx = idx + head * k_vl;
 
-    __shared__ int src[64];
+    constexpr int NT = 2 * G;                                  // threads of this CTA
+    __shared__ int src[G];
     __shared__ int win[FRZ_WIN], j0_sh;
-    __shared__ float warp_max[FRZ_THREADS / 32];
-    __shared__ __align__(16) uint8_t vtile[4 * DEC_VTILE_BYTES];
-    // Source rows of the group's 64 compacted rows in three dependent memory round trips instead of ten:
+    __shared__ float warp_max[NT / 32];
+    __shared__ __align__(16) uint8_t vtile[(G / 16) * DEC_VTILE_BYTES];
+    // Source rows of the group's G compacted rows in three dependent memory round trips instead of ten:
     // warp 0 finds j0 = the number of vertical rows before the group's first row by a 32-way search, a window of
     // the index list starting there goes to shared memory, and each row finishes its own search in that window
     // (a row whose answer lies beyond the window - long runs of vertical rows - falls back to the global search).
-    const int p0 = grp * 64;
+    const int p0 = grp * G;
     if (threadIdx.x < 32) {
         int lo = 0, hi = k_vl;                              // smallest j in [lo, hi] with idx[j] - j > p0
         while (lo < hi) {
@@ -78,9 +80,9 @@ freeze_quantize_kernel(const uint4* __restrict__ k_, const uint4* __restrict__ v
     }
     __syncthreads();
     const int j0 = j0_sh;
-    if (threadIdx.x < FRZ_WIN) win[threadIdx.x] = j0 + (int)threadIdx.x < k_vl ? __ldg(hidx + j0 + threadIdx.x) : 0x7fffffff;
+    for (int i = threadIdx.x; i < FRZ_WIN; i += NT) win[i] = j0 + i < k_vl ? __ldg(hidx + j0 + i) : 0x7fffffff;
     __syncthreads();
-    if (threadIdx.x < 64) {
+    if (threadIdx.x < G) {
         const int p = p0 + threadIdx.x;
         int s = -1;
         if (p < nQ) {
@@ -99,7 +101,7 @@ freeze_quantize_kernel(const uint4* __restrict__ k_, const uint4* __restrict__ v
     float amax = 0.0f;
 #pragma unroll
     for (int gi = 0; gi < 4; ++gi) {
-        const int u = threadIdx.x + gi * FRZ_THREADS;     // 16-channel unit: row u >> 3, channels 16 * (u & 7)
+        const int u = threadIdx.x + gi * NT;              // 16-channel unit: row u >> 3, channels 16 * (u & 7)
         const int s = src[u >> 3];
         if (s >= 0) {
             r[gi][0] = __ldg(x + (long)s * 16 + (u & 7) * 2);
@@ -119,15 +121,17 @@ freeze_quantize_kernel(const uint4* __restrict__ k_, const uint4* __restrict__ v
     for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
     if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = amax;
     __syncthreads();
-    amax = fmaxf(fmaxf(warp_max[0], warp_max[1]), fmaxf(warp_max[2], warp_max[3]));
+    amax = warp_max[0];
+#pragma unroll
+    for (int w = 1; w < NT / 32; ++w) amax = fmaxf(amax, warp_max[w]);
 
     const bool dead = !(amax >= 0x1p-100f);
     const float inv = dead ? 0.0f : __fdiv_rn(7.0f, amax);
-    if (threadIdx.x == 0) (is_v ? vs : ks)[head * (nQp / 64) + grp] = dead ? 0.0f : __fdiv_rn(amax, 7.0f);
+    if (threadIdx.x == 0) (is_v ? vs : ks)[head * (nQp / G) + grp] = dead ? 0.0f : __fdiv_rn(amax, 7.0f);
 
 #pragma unroll
     for (int gi = 0; gi < 4; ++gi) {
-        const int u = threadIdx.x + gi * FRZ_THREADS;
+        const int u = threadIdx.x + gi * NT;
         const int row = u >> 3, ch0 = (u & 7) * 16;
         const uint32_t* w = reinterpret_cast<const uint32_t*>(&r[gi][0]);
         uint8_t b[8];
@@ -140,7 +144,7 @@ freeze_quantize_kernel(const uint4* __restrict__ k_, const uint4* __restrict__ v
         if (!is_v) {
             uint32_t o0 = b[0] | (b[1] << 8) | (b[2] << 16) | ((uint32_t)b[3] << 24);
             uint32_t o1 = b[4] | (b[5] << 8) | (b[6] << 16) | ((uint32_t)b[7] << 24);
-            *reinterpret_cast<uint2*>(kq + ((head * nQp + grp * 64 + row) * 64 + ch0 / 2)) = make_uint2(o0, o1);
+            *reinterpret_cast<uint2*>(kq + ((head * nQp + grp * G + row) * 64 + ch0 / 2)) = make_uint2(o0, o1);
         } else {
             const int tile = row >> 4, key = row & 15;
 #pragma unroll
@@ -149,10 +153,10 @@ freeze_quantize_kernel(const uint4* __restrict__ k_, const uint4* __restrict__ v
     }
     if (is_v) {
         __syncthreads();
-        uint4* dst = reinterpret_cast<uint4*>(vq + (head * (nQp / 16) + grp * 4) * (long)DEC_VTILE_BYTES);
+        uint4* dst = reinterpret_cast<uint4*>(vq + (head * (nQp / 16) + grp * (G / 16)) * (long)DEC_VTILE_BYTES);
         const uint4* s4 = reinterpret_cast<const uint4*>(vtile);
         dst[threadIdx.x] = s4[threadIdx.x];
-        dst[threadIdx.x + FRZ_THREADS] = s4[threadIdx.x + FRZ_THREADS];
+        dst[threadIdx.x + NT] = s4[threadIdx.x + NT];
     }
 }
 
@@ -168,10 +172,15 @@ int launch_freeze(const void* k_, const void* v, const int32_t* vl_idx, const hy
                                                          static_cast<uint4*>(c.v_win));
     }
     if (g.nQ > 0) {
-        const dim3 grid((unsigned)(g.nQp / 64), (unsigned)heads, 2);
-        freeze_quantize_kernel<<<grid, FRZ_THREADS, 0, st>>>(k4, v4, vl_idx, c.N, c.k, (int)g.nQ, g.sQ,
-                                                             static_cast<uint8_t*>(c.kq_codes),
-                                                             static_cast<uint8_t*>(c.vq_codes), c.kq_scales, c.vq_scales);
+        const dim3 grid((unsigned)(g.nQp / c.group), (unsigned)heads, 2);
+        auto* kq = static_cast<uint8_t*>(c.kq_codes);
+        auto* vq = static_cast<uint8_t*>(c.vq_codes);
+        if (c.group == 32)
+            freeze_quantize_kernel<32><<<grid, 64, 0, st>>>(k4, v4, vl_idx, c.N, c.k, (int)g.nQ, g.sQ, kq, vq, c.kq_scales, c.vq_scales);
+        else if (c.group == 64)
+            freeze_quantize_kernel<64><<<grid, 128, 0, st>>>(k4, v4, vl_idx, c.N, c.k, (int)g.nQ, g.sQ, kq, vq, c.kq_scales, c.vq_scales);
+        else
+            freeze_quantize_kernel<128><<<grid, 256, 0, st>>>(k4, v4, vl_idx, c.N, c.k, (int)g.nQ, g.sQ, kq, vq, c.kq_scales, c.vq_scales);
     }
     return launch_status();
 }

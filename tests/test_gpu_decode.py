@@ -43,10 +43,10 @@ def _v_tiles_to_rows(vq: np.ndarray) -> np.ndarray:
     return packed.reshape(lead + (tiles * 16, 64))
 
 
-def _freeze_both(K, V, idx, W, Hq, staging_capacity=128):
-    ref = od.freeze(wl.bits(K), wl.bits(V), idx, W, staging_capacity=staging_capacity)
+def _freeze_both(K, V, idx, W, Hq, staging_capacity=128, group=64):
+    ref = od.freeze(wl.bits(K), wl.bits(V), idx, W, group=group, staging_capacity=staging_capacity)
     idx_t = None if idx is None or idx.shape[2] == 0 else torch.from_numpy(idx).cuda()
-    cache = dapi.hyq_freeze(K.cuda(), V.cuda(), idx_t, W, Hq, staging_capacity)
+    cache = dapi.hyq_freeze(K.cuda(), V.cuda(), idx_t, W, Hq, staging_capacity, group=group)
     torch.cuda.synchronize()
     return ref, cache
 
@@ -64,7 +64,7 @@ def _assert_cache_equal(ref, cache):
     b = {n: t.cpu().numpy() if t.dtype != torch.bfloat16 else wl.bits(t.cpu()) for n, t in cache.buffers.items()}
     assert int(cache.sizes.quantized_rows) == nQ
     if nQ:
-        ng = -(-nQ // 64)
+        ng = -(-nQ // ref["group"])
         assert np.array_equal(b["kq_codes"][:, :, :nQ], ref["kq_codes"])
         assert np.array_equal(_v_tiles_to_rows(b["vq_codes"])[:, :, :nQ], ref["vq_codes"])
         assert np.array_equal(b["kq_scales"][:, :, :ng].view(np.uint32), ref["kq_scales"].view(np.uint32))
@@ -124,6 +124,25 @@ def test_decode_attention_matches_oracle(B, Hq, Hkv, N, W, kk, n_s, splits):
     assert np.abs(lse.cpu().numpy() - lse_want).max() <= 2e-3
     got16 = dapi.hyq_hybrid_attention_decode(q.cuda(), cache, splits=splits, out_dtype=torch.bfloat16)
     assert torch.equal(got16.cpu(), got.cpu().to(torch.bfloat16))
+
+
+@pytest.mark.parametrize("group", [32, 128])
+@pytest.mark.parametrize("B,Hq,Hkv,N,W,kk,n_s", [(1, 4, 1, 300, 40, 9, 3), (2, 8, 2, 1000, 128, 37, 0), (1, 8, 2, 2117, 100, 50, 17),
+                                                 (1, 2, 2, 64, 0, 0, 1)])
+def test_other_group_sizes(group, B, Hq, Hkv, N, W, kk, n_s):
+    """Algorithm 4's group size G = 32 and 128: cache bit-exact, attention within tolerance."""
+    K, V = rand_bf16((B, Hkv, N, 128), 71, 1.3), rand_bf16((B, Hkv, N, 128), 72)
+    K[:, :, : N // 2] *= 0.05
+    q = rand_bf16((B, Hq, 128), 73, 1.5)
+    idx = _idx(B, Hkv, N - min(W, N), kk, 74) if kk else None
+    ref, cache = _freeze_both(K, V, idx, W, Hq, group=group)
+    _assert_cache_equal(ref, cache)
+    _stage(ref, cache, n_s, 500)
+    want, _ = od.decode_attention(wl.bits(q), ref)
+    for splits in (0, 3):
+        got = dapi.hyq_hybrid_attention_decode(q.cuda(), cache, splits=splits, out_dtype=torch.float32)
+        mx, rel = errors(got.cpu().numpy(), want)
+        assert mx <= MAX_ABS_TOL and rel <= MEAN_REL_TOL, (splits, mx, rel)
 
 
 def test_decode_with_peaked_scores_and_late_maxima():
