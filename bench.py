@@ -382,12 +382,13 @@ def run_decode(args, w: wl.Workload):
     torch.cuda.set_device(dev)
     w = w.scaled(B=args.batch)
     g = w.Hq // w.Hkv
+    kv_fmt = wl.FMT_INT8 if args.kv_format == "int8" else wl.FMT_INT4
     Q, K, V = wl.make_inputs(w)
     K, V = K.to(dev), V.to(dev)
     q_tail = Q[:, ::g].contiguous().to(dev)                 # Algorithm 1 with H = H_KV heads
     idx = api.hyq_select_vertical(q_tail, K, w.window, w.k)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    cache = dapi.hyq_freeze(K, V, idx, w.window, w.Hq, staging_capacity=args.staging)
+    cache = dapi.hyq_freeze(K, V, idx, w.window, w.Hq, staging_capacity=args.staging, fmt=kv_fmt)
     torch.cuda.synchronize()
     e0.record()
     dapi.hyq_freeze(K, V, idx, w.window, w.Hq, staging_capacity=args.staging, cache=cache)
@@ -402,7 +403,8 @@ def run_decode(args, w: wl.Workload):
     # right before a timed call.
     by = cache.bytes_read_per_token()
     n_rep = 1 + int(np.ceil(3 * 126e6 / by))
-    caches = [cache] + [dapi.hyq_freeze(K, V, idx, w.window, w.Hq, staging_capacity=args.staging) for _ in range(n_rep - 1)]
+    caches = [cache] + [dapi.hyq_freeze(K, V, idx, w.window, w.Hq, staging_capacity=args.staging, fmt=kv_fmt)
+                        for _ in range(n_rep - 1)]
     for c in caches:
         for kn, vn in new_rows:
             c.append(kn, vn)
@@ -440,7 +442,7 @@ def run_decode(args, w: wl.Workload):
     import oracle
     from oracle import decode as od
     kb, vb = wl.bits(K[:1].cpu()), wl.bits(V[:1].cpu())
-    ref = od.freeze(kb, vb, idx[:1].cpu().numpy(), w.window, staging_capacity=args.staging)
+    ref = od.freeze(kb, vb, idx[:1].cpu().numpy(), w.window, fmts=(kv_fmt, kv_fmt), staging_capacity=args.staging)
     for kn, vn in new_rows:
         od.append_staging(ref, wl.bits(kn[:1].cpu()), wl.bits(vn[:1].cpu()))
     t0 = time.perf_counter()
@@ -451,15 +453,15 @@ def run_decode(args, w: wl.Workload):
         "metric": "hybrid decode attention latency per token step", "value": ms * 1e3, "unit": "us", "n_gpus": 1,
         "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": False,
         "scaling": "weak", "vs_baseline": None,
-        "dtype": "int4 codes -> fp16 in registers, fp16 / bf16 mma.sync with f32 accumulation", "data": "synthetic",
+        "dtype": f"{args.kv_format} codes -> fp16 in registers, fp16 / bf16 mma.sync with f32 accumulation", "data": "synthetic",
         "config": {"workload": f"{w.name} cache shape, decode of one token per sequence", "B": w.B, "Hq": w.Hq,
                    "Hkv": w.Hkv, "N": w.L, "D": w.D, "window": w.window, "k": w.k, "staging_rows": args.staging,
-                   "format": "K4V4, group 64", "splits": args.splits, "cached_rows_per_head": rows,
+                   "format": ("K8V8" if kv_fmt == wl.FMT_INT8 else "K4V4") + ", group 64", "splits": args.splits, "cached_rows_per_head": rows,
                    "l2": f"{n_rep} cache replicas used round-robin ({by * (n_rep - 1) / 1e6:.0f} MB read between reuses)",
                    "freeze_ms": freeze_ms},
         "roofline": {"bound": "hbm", "kernel": "decode_kernel + decode_merge_kernel (one call)",
                      "achieved": by / (ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                     "frac": by / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "traffic": (NCU_DECODE_TRAFFIC_BYTES_B4 * w.B // 4 if (w.name, w.L, args.staging) == ("c2", 32768, 128) else None),
+                     "frac": by / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "traffic": (NCU_DECODE_TRAFFIC_BYTES_B4 * w.B // 4 if (w.name, w.L, args.staging, args.kv_format) == ("c2", 32768, 128, "int4") else None),
                      "bytes_per_call": by, "peak_source": peaks["source"]},
         "cpu_baseline": {"value": cpu_s * 1e6 * w.B, "unit": "us", "cores": oracle.num_threads(), "kind": "oracle",
                          "sample": "oracle attention of one sequence (all heads) timed, scaled by the batch size"},
@@ -484,6 +486,7 @@ def main():
     ap.add_argument("--batch", type=int, default=8, help="with --decode: sequences in the batch")
     ap.add_argument("--staging", type=int, default=128, help="with --decode: staged rows (W_s, all filled)")
     ap.add_argument("--splits", type=int, default=0, help="with --decode: slices per KV head (0 = library's choice)")
+    ap.add_argument("--kv-format", default="int4", choices=["int4", "int8"], help="with --decode: cache code format (K4V4 / K8V8)")
     ap.add_argument("--formats", default="", choices=["", *sorted(FORMAT_SETS)],
                     help="override the workload's (Q, K, V) low-bit formats (default: as the workload defines them)")
     args = ap.parse_args()

@@ -263,6 +263,44 @@ __device__ __forceinline__ void quant_tile_pair(const QTile& d0, const QTile& d1
     }
 }
 
+// ---- INT8 cache (K8V8) ----------------------------------------------------------------------------------------
+// A 16-row tile is 2 KB of K codes (row-major, 128 B per row) and 2 KB of V codes (operand order, see
+// vq8_byte_offset).  K bytes enter Q.K^T as fp16 subnormals: byte ^ 0x80 = code + 128 in mantissa bits 0-7, upper byte
+// zero, is (code + 128) * 2^-24; a byte permute builds two of them per register and the +128 becomes a per-head score
+// constant.  V bytes are made exact: (byte ^ 0x80) under the constant byte 0x64 is fp16 1024 + code + 128, minus 1152.
+struct QTile8 {
+    uint4 k[4];          // row r: bytes [16j, +16) in k[0] and [64 + 16j, +16) in k[1]; row r + 8 in k[2], k[3]
+    uint4 v[4];          // this lane's 16 bytes of each of the V tile's four 512-byte runs
+    float fk, fv;
+};
+
+template <bool RAGGED>
+__device__ __forceinline__ void quant_tile8(const QTile8& d, const uint32_t (&qf)[16], float scale_log2, float bias0, float bias1,
+                                            int rows_valid, int r, SoftmaxState& st, float (&acc)[8][4]) {
+    float c4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+        const uint32_t wa = word_of(d.k[c >> 2], c & 3) ^ 0x80808080u, wb = word_of(d.k[2 + (c >> 2)], c & 3) ^ 0x80808080u;
+        mma_f16(c4, __byte_perm(wa, 0u, 0x4140), __byte_perm(wb, 0u, 0x4140), __byte_perm(wa, 0u, 0x4342),
+                __byte_perm(wb, 0u, 0x4342), qf[2 * c], qf[2 * c + 1]);
+    }
+    float pw[4];
+    softmax_tile<RAGGED>(st, acc, c4, d.fk * scale_log2, bias0, bias1, r < rows_valid, r + 8 < rows_valid, pw);
+    const uint32_t b0 = movmatrix_trans(pack_f16(pw[0] * d.fv, pw[1] * d.fv));
+    const uint32_t b1 = movmatrix_trans(pack_f16(pw[2] * d.fv, pw[3] * d.fv));
+    auto exact = [](uint32_t w, uint32_t sel) {           // two bytes of w -> packed fp16 code values
+        uint32_t h = __byte_perm(w, 0x64646464u, sel);
+        asm("sub.rn.f16x2 %0, %1, %2;" : "=r"(h) : "r"(h), "r"(0x64806480u));
+        return h;
+    };
+#pragma unroll
+    for (int x = 0; x < 8; ++x) {
+        const uint32_t w0 = word_of(d.v[x >> 1], 2 * (x & 1)) ^ 0x80808080u, w1 = word_of(d.v[x >> 1], 2 * (x & 1) + 1) ^ 0x80808080u;
+        mma_f16(acc[x], exact(w0, 0x4140), exact(w0, 0x4342), exact(w1, 0x4140), exact(w1, 0x4342), b0, b1);
+    }
+}
+
+template <bool FMT8>
 __global__ void __launch_bounds__(DEC_THREADS, DEC_CTAS_PER_SM)
 decode_kernel(const DecParams p) {
     const int split = blockIdx.x;
@@ -293,7 +331,8 @@ decode_kernel(const DecParams p) {
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             sum += __half2float(__float2half_rn(bf16_lo(w[i])));
-            sum += 16.0f * __half2float(__float2half_rn(bf16_hi(w[i]) * 0.0625f));
+            sum += FMT8 ? __half2float(__float2half_rn(bf16_hi(w[i])))
+                        : 16.0f * __half2float(__float2half_rn(bf16_hi(w[i]) * 0.0625f));
         }
 #pragma unroll
         for (int o = 1; o < 16; o <<= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
@@ -321,7 +360,7 @@ decode_kernel(const DecParams p) {
     for (int x = 0; x < 8; ++x) acc[x][0] = acc[x][1] = acc[x][2] = acc[x][3] = 0.0f;
 
     // ---------------- quantized prefix ----------------
-    if (q_lo + warp < q_hi) {
+    if (!FMT8 && q_lo + warp < q_hi) {
         uint32_t qf[16];                                   // q^T operand, fp16: k-step c -> qf[2c], qf[2c+1]
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
@@ -389,6 +428,56 @@ decode_kernel(const DecParams p) {
             fetch(A, i);
             if (i >= n_full) quant_tile<true>(A, qf, kscale, b0, b1, (int)(nQ & 15), r, st, acc);
             else quant_tile<false>(A, qf, kscale, b0, b1, 16, r, st, acc);
+        }
+    }
+    if (FMT8 && q_lo + warp < q_hi) {
+        uint32_t qf[16];                                   // k-step c: channels 64 (c >> 2) + 16 j + 4 (c & 3) + {0,1} and + {2,3}
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            const int base = 64 * (c >> 2) + 16 * j + 4 * (c & 3);
+            const uint16_t* qr = qs[r];
+            auto f16 = [&](int ch) { return __float2half_rn(__uint_as_float((uint32_t)qr[ch] << 16)); };
+            const __half2 h0 = __halves2half2(f16(base), f16(base + 1)), h1 = __halves2half2(f16(base + 2), f16(base + 3));
+            qf[2 * c] = *reinterpret_cast<const uint32_t*>(&h0);
+            qf[2 * c + 1] = *reinterpret_cast<const uint32_t*>(&h1);
+        }
+        constexpr int ST8 = 2, ST8_BYTES = DEC_STAGES * DEC_STAGE_BYTES / ST8;      // the same ring as two 4 KB stages
+        static_assert(ST8_BYTES == 4096, "an INT8 tile is 2 KB of K and 2 KB of V");
+        const long t0 = q_lo + warp;
+        const int n_my = (int)((q_hi - t0 + DEC_WARPS - 1) / DEC_WARPS);
+        const bool has_ragged = (nQ & 15) && t0 + (long)(n_my - 1) * DEC_WARPS == Tq - 1;
+        const uint8_t* gk = p.kq + unit * p.sQ * 128 + t0 * 2048 + r * 128 + j * 16;       // bytes [16j, +16) and [64 + 16j, +16) of row r
+        const uint8_t* gv = p.vq + unit * (p.sQ / 16) * 2048 + t0 * 2048 + lane * 16;
+        const int gshift = p.gshift;
+        const float* pks = p.ks + unit * (p.sQ >> (p.gshift + 4));
+        const float* pvs = p.vs + unit * (p.sQ >> (p.gshift + 4));
+        const uint32_t ring = (uint32_t)__cvta_generic_to_shared(ring_mem) + warp * (DEC_STAGES * DEC_STAGE_BYTES) + lane * 16;
+        auto issue = [&](uint32_t sa) {
+            cp_async16(sa, gk); cp_async16(sa + 512, gk + 64);
+            cp_async16(sa + 1024, gk + 1024); cp_async16(sa + 1536, gk + 1088);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) cp_async16(sa + 2048 + i * 512, gv + i * 512);
+            gk += DEC_WARPS * 2048; gv += DEC_WARPS * 2048;
+        };
+#pragma unroll
+        for (int s = 0; s < ST8; ++s) {
+            if (s < n_my) issue(ring + s * ST8_BYTES);
+            cp_async_commit();
+        }
+        const float kscale = p.scale_log2 * 16777216.0f;
+        const float b0 = q_sum[2 * j] * (128.0f / 16777216.0f), b1 = q_sum[2 * j + 1] * (128.0f / 16777216.0f);
+        for (int i = 0; i < n_my; ++i) {
+            cp_async_wait<ST8 - 1>();                       // tile i has landed
+            const uint32_t sa = ring + (i & 1) * ST8_BYTES;
+            QTile8 A;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) { A.k[u] = lds128(sa + u * 512); A.v[u] = lds128(sa + 2048 + u * 512); }
+            const int grp = ((int)t0 + i * DEC_WARPS) >> gshift;
+            A.fk = __ldg(pks + grp); A.fv = __ldg(pvs + grp);
+            if (i + ST8 < n_my) issue(sa);                  // own bytes only: no barrier
+            cp_async_commit();
+            if (has_ragged && i == n_my - 1) quant_tile8<true>(A, qf, kscale, b0, b1, (int)(nQ & 15), r, st, acc);
+            else quant_tile8<false>(A, qf, kscale, b0, b1, 16, r, st, acc);
         }
     }
     cp_async_wait<0>();
@@ -572,11 +661,13 @@ int launch_decode(const void* q, const hyq_kv_cache& c, const int32_t* lengths, 
     constexpr int ring_bytes = DEC_WARPS * DEC_STAGES * DEC_STAGE_BYTES;
     static bool attr_set = false;          // same value every time: a benign race between host threads
     if (!attr_set) {
-        if (cudaFuncSetAttribute(decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ring_bytes) != cudaSuccess)
+        if (cudaFuncSetAttribute(decode_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, ring_bytes) != cudaSuccess ||
+            cudaFuncSetAttribute(decode_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ring_bytes) != cudaSuccess)
             return HYQ_ERR_CUDA;
         attr_set = true;
     }
-    decode_kernel<<<dim3((unsigned)splits, (unsigned)units), DEC_THREADS, ring_bytes, st>>>(p);
+    if (c.format == HYQ_FMT_INT8) decode_kernel<true><<<dim3((unsigned)splits, (unsigned)units), DEC_THREADS, ring_bytes, st>>>(p);
+    else decode_kernel<false><<<dim3((unsigned)splits, (unsigned)units), DEC_THREADS, ring_bytes, st>>>(p);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)units, (unsigned)p.g);
     cfg.blockDim = dim3(HYQ_D);

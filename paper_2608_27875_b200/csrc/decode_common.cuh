@@ -36,6 +36,16 @@ __host__ __device__ __forceinline__ int vq_byte_offset(int key, int d) {
     return (x >> 2) * 512 + (4 * r + j) * 16 + (x & 3) * 4 + (n >> 1);
 }
 
+// Same for an INT8 V tile (2048 bytes): byte of channel d of row `key`.  Lane l = 4r + j owns bytes [16l, 16l + 16) of
+// each of the tile's four 512-byte runs, 16 words in all; word 2x + (key >> 3) holds, in byte order, (channel e = 0,
+// key bit 0 = 0), (e = 0, 1), (e = 1, 0), (e = 1, 1) of accumulator row pair x - so a byte permute picks the two
+// key-adjacent codes of an operand register.
+__host__ __device__ __forceinline__ int vq8_byte_offset(int key, int d) {
+    const int j = (key & 7) >> 1, r = (d >> 3) & 7, x = ((d >> 6) << 2) | ((d >> 1) & 3);
+    const int w = 2 * x + (key >> 3);
+    return (w >> 2) * 512 + (4 * r + j) * 16 + (w & 3) * 4 + (d & 1) * 2 + (key & 1);
+}
+
 int launch_freeze(const void* k_, const void* v, const int32_t* vl_idx, const hyq_kv_cache& c, cudaStream_t st);
 int decode_auto_splits(const hyq_kv_cache& c);
 size_t decode_workspace_bytes(const hyq_kv_cache& c, int splits);

@@ -44,7 +44,7 @@ gather_rows_kernel(const uint4* __restrict__ k_, const uint4* __restrict__ v, co
     (vl ? v_vl_out : v_win)[d] = __ldg(v + s);
 }
 
-template <int G>
+template <int G, bool FMT8>
 __global__ void __launch_bounds__(2 * G)
 freeze_quantize_kernel(const uint4* __restrict__ k_, const uint4* __restrict__ v, const int32_t* __restrict__ idx,
                        int N, int k_vl, int nQ, long nQp, uint8_t* __restrict__ kq, uint8_t* __restrict__ vq,
@@ -59,7 +59,10 @@ freeze_quantize_kernel(const uint4* __restrict__ k_, const uint4* __restrict__ v
     __shared__ int src[G];
     __shared__ int win[FRZ_WIN], j0_sh;
     __shared__ float warp_max[NT / 32];
-    __shared__ __align__(16) uint8_t vtile[(G / 16) * DEC_VTILE_BYTES];
+    constexpr int ROW_BYTES = FMT8 ? HYQ_D : HYQ_D / 2;        // code bytes per row
+    constexpr int TILE_BYTES = 16 * ROW_BYTES;                 // one 16-row V tile
+    constexpr float CB = FMT8 ? 127.0f : 7.0f;
+    __shared__ __align__(16) uint8_t vtile[(G / 16) * TILE_BYTES];
     // Source rows of the group's G compacted rows in three dependent memory round trips instead of ten:
     // warp 0 finds j0 = the number of vertical rows before the group's first row by a 32-way search, a window of
     // the index list starting there goes to shared memory, and each row finishes its own search in that window
@@ -126,37 +129,57 @@ freeze_quantize_kernel(const uint4* __restrict__ k_, const uint4* __restrict__ v
     for (int w = 1; w < NT / 32; ++w) amax = fmaxf(amax, warp_max[w]);
 
     const bool dead = !(amax >= 0x1p-100f);
-    const float inv = dead ? 0.0f : __fdiv_rn(7.0f, amax);
-    if (threadIdx.x == 0) (is_v ? vs : ks)[head * (nQp / G) + grp] = dead ? 0.0f : __fdiv_rn(amax, 7.0f);
+    const float inv = dead ? 0.0f : __fdiv_rn(CB, amax);
+    if (threadIdx.x == 0) (is_v ? vs : ks)[head * (nQp / G) + grp] = dead ? 0.0f : __fdiv_rn(amax, CB);
 
 #pragma unroll
     for (int gi = 0; gi < 4; ++gi) {
         const int u = threadIdx.x + gi * NT;
         const int row = u >> 3, ch0 = (u & 7) * 16;
         const uint32_t* w = reinterpret_cast<const uint32_t*>(&r[gi][0]);
-        uint8_t b[8];
+        if (FMT8) {
+            uint8_t b[16];
 #pragma unroll
-        for (int m = 0; m < 8; ++m) {
-            const int q0 = max(-7, min(7, __float2int_rn(__fmul_rn(bf16_lo(w[m]), inv))));
-            const int q1 = max(-7, min(7, __float2int_rn(__fmul_rn(bf16_hi(w[m]), inv))));
-            b[m] = (uint8_t)((q0 & 0xF) | ((q1 & 0xF) << 4));
-        }
-        if (!is_v) {
-            uint32_t o0 = b[0] | (b[1] << 8) | (b[2] << 16) | ((uint32_t)b[3] << 24);
-            uint32_t o1 = b[4] | (b[5] << 8) | (b[6] << 16) | ((uint32_t)b[7] << 24);
-            *reinterpret_cast<uint2*>(kq + ((head * nQp + grp * G + row) * 64 + ch0 / 2)) = make_uint2(o0, o1);
+            for (int m = 0; m < 8; ++m) {
+                b[2 * m] = (uint8_t)max(-127, min(127, __float2int_rn(__fmul_rn(bf16_lo(w[m]), inv))));
+                b[2 * m + 1] = (uint8_t)max(-127, min(127, __float2int_rn(__fmul_rn(bf16_hi(w[m]), inv))));
+            }
+            if (!is_v) {
+                uint32_t o[4];
+#pragma unroll
+                for (int c4 = 0; c4 < 4; ++c4)
+                    o[c4] = b[4 * c4] | (b[4 * c4 + 1] << 8) | (b[4 * c4 + 2] << 16) | ((uint32_t)b[4 * c4 + 3] << 24);
+                *reinterpret_cast<uint4*>(kq + ((head * nQp + grp * G + row) * ROW_BYTES + ch0)) = make_uint4(o[0], o[1], o[2], o[3]);
+            } else {
+                const int tile = row >> 4, key = row & 15;
+#pragma unroll
+                for (int m = 0; m < 16; ++m) vtile[tile * TILE_BYTES + vq8_byte_offset(key, ch0 + m)] = b[m];
+            }
         } else {
-            const int tile = row >> 4, key = row & 15;
+            uint8_t b[8];
 #pragma unroll
-            for (int m = 0; m < 8; ++m) vtile[tile * DEC_VTILE_BYTES + vq_byte_offset(key, ch0 + 2 * m)] = b[m];
+            for (int m = 0; m < 8; ++m) {
+                const int q0 = max(-7, min(7, __float2int_rn(__fmul_rn(bf16_lo(w[m]), inv))));
+                const int q1 = max(-7, min(7, __float2int_rn(__fmul_rn(bf16_hi(w[m]), inv))));
+                b[m] = (uint8_t)((q0 & 0xF) | ((q1 & 0xF) << 4));
+            }
+            if (!is_v) {
+                uint32_t o0 = b[0] | (b[1] << 8) | (b[2] << 16) | ((uint32_t)b[3] << 24);
+                uint32_t o1 = b[4] | (b[5] << 8) | (b[6] << 16) | ((uint32_t)b[7] << 24);
+                *reinterpret_cast<uint2*>(kq + ((head * nQp + grp * G + row) * ROW_BYTES + ch0 / 2)) = make_uint2(o0, o1);
+            } else {
+                const int tile = row >> 4, key = row & 15;
+#pragma unroll
+                for (int m = 0; m < 8; ++m) vtile[tile * TILE_BYTES + vq_byte_offset(key, ch0 + 2 * m)] = b[m];
+            }
         }
     }
     if (is_v) {
         __syncthreads();
-        uint4* dst = reinterpret_cast<uint4*>(vq + (head * (nQp / 16) + grp * (G / 16)) * (long)DEC_VTILE_BYTES);
+        uint4* dst = reinterpret_cast<uint4*>(vq + (head * (nQp / 16) + grp * (G / 16)) * (long)TILE_BYTES);
         const uint4* s4 = reinterpret_cast<const uint4*>(vtile);
-        dst[threadIdx.x] = s4[threadIdx.x];
-        dst[threadIdx.x + NT] = s4[threadIdx.x + NT];
+#pragma unroll
+        for (int i = 0; i < (G / 16) * TILE_BYTES / 16 / NT; ++i) dst[threadIdx.x + i * NT] = s4[threadIdx.x + i * NT];
     }
 }
 
@@ -175,12 +198,12 @@ int launch_freeze(const void* k_, const void* v, const int32_t* vl_idx, const hy
         const dim3 grid((unsigned)(g.nQp / c.group), (unsigned)heads, 2);
         auto* kq = static_cast<uint8_t*>(c.kq_codes);
         auto* vq = static_cast<uint8_t*>(c.vq_codes);
-        if (c.group == 32)
-            freeze_quantize_kernel<32><<<grid, 64, 0, st>>>(k4, v4, vl_idx, c.N, c.k, (int)g.nQ, g.sQ, kq, vq, c.kq_scales, c.vq_scales);
-        else if (c.group == 64)
-            freeze_quantize_kernel<64><<<grid, 128, 0, st>>>(k4, v4, vl_idx, c.N, c.k, (int)g.nQ, g.sQ, kq, vq, c.kq_scales, c.vq_scales);
-        else
-            freeze_quantize_kernel<128><<<grid, 256, 0, st>>>(k4, v4, vl_idx, c.N, c.k, (int)g.nQ, g.sQ, kq, vq, c.kq_scales, c.vq_scales);
+#define HYQ_FRZ(G_, F8_) freeze_quantize_kernel<G_, F8_><<<grid, 2 * G_, 0, st>>>(k4, v4, vl_idx, c.N, c.k, (int)g.nQ, g.sQ, kq, vq, c.kq_scales, c.vq_scales)
+        const bool f8 = c.format == HYQ_FMT_INT8;
+        if (c.group == 32) { if (f8) HYQ_FRZ(32, true); else HYQ_FRZ(32, false); }
+        else if (c.group == 64) { if (f8) HYQ_FRZ(64, true); else HYQ_FRZ(64, false); }
+        else { if (f8) HYQ_FRZ(128, true); else HYQ_FRZ(128, false); }
+#undef HYQ_FRZ
     }
     return launch_status();
 }

@@ -9,7 +9,7 @@ from dataclasses import dataclass, field
 import torch
 
 from . import api
-from .workloads import FMT_INT4
+from .workloads import FMT_INT4, FMT_INT8
 
 EXPORTS = ("hyq_kv_cache_query_sizes", "hyq_freeze", "hyq_hybrid_attention_decode_workspace",
            "hyq_hybrid_attention_decode", "hyq_hybrid_attention_decode_ragged")
@@ -95,7 +95,8 @@ class HybridKvCache:
         heads = d.B * d.Hkv
         nq = int(s.quantized_rows)
         w = min(d.window, d.N)
-        return heads * (nq * d.D + 2 * (-(-nq // d.group)) * 4 + (d.k + w + d.n_staging) * d.D * 4)
+        code_bytes = 2 * d.D if d.format == FMT_INT8 else d.D    # K + V codes of one row
+        return heads * (nq * code_bytes + 2 * (-(-nq // d.group)) * 4 + (d.k + w + d.n_staging) * d.D * 4)
 
 
 def alloc_cache(desc: KvCacheDesc, device="cuda") -> HybridKvCache:
@@ -106,7 +107,8 @@ def alloc_cache(desc: KvCacheDesc, device="cuda") -> HybridKvCache:
     kcap = desc.cap_vertical or desc.k
     u8 = lambda *shape: torch.empty(*shape, dtype=torch.uint8, device=device)          # noqa: E731
     bf = lambda *shape: torch.empty(*shape, dtype=torch.bfloat16, device=device)       # noqa: E731
-    buf = dict(kq_codes=u8(B, H, max(nqp, 1), D // 2), vq_codes=u8(B, H, max(nqp // 16, 1), 1024),
+    rb = D if desc.format == FMT_INT8 else D // 2               # code bytes per row
+    buf = dict(kq_codes=u8(B, H, max(nqp, 1), rb), vq_codes=u8(B, H, max(nqp // 16, 1), 16 * rb),
                kq_scales=torch.empty(B, H, max(nqp // desc.group, 1), dtype=torch.float32, device=device),
                vq_scales=torch.empty(B, H, max(nqp // desc.group, 1), dtype=torch.float32, device=device),
                k_vl=bf(B, H, max(kcap, 1), D), v_vl=bf(B, H, max(kcap, 1), D),
@@ -118,13 +120,14 @@ def alloc_cache(desc: KvCacheDesc, device="cuda") -> HybridKvCache:
 
 
 def hyq_freeze(k: torch.Tensor, v: torch.Tensor, vl_idx: torch.Tensor | None, window: int, Hq: int,
-               staging_capacity: int = 128, cache: HybridKvCache | None = None, group: int = 64) -> HybridKvCache:
+               staging_capacity: int = 128, cache: HybridKvCache | None = None, group: int = 64,
+               fmt: int = FMT_INT4) -> HybridKvCache:
     """Algorithm 4.  k, v [B,Hkv,N,D] bf16 CUDA; vl_idx int32 [B,Hkv,k] ascending (None: no vertical rows)."""
     api._dev(k, torch.bfloat16, "k"), api._dev(v, torch.bfloat16, "v")
     B, Hkv, N, D = k.shape
     kk = 0 if vl_idx is None else int(vl_idx.shape[2])
     if cache is None:
-        cache = alloc_cache(make_desc(B, Hq, Hkv, N, window, kk, staging_capacity, D=D, group=group), k.device)
+        cache = alloc_cache(make_desc(B, Hq, Hkv, N, window, kk, staging_capacity, D=D, group=group, fmt=fmt), k.device)
     if kk:
         api._dev(vl_idx, torch.int32, "vl_idx")
     api._check(_lib().hyq_freeze(k.data_ptr(), v.data_ptr(), vl_idx.data_ptr() if kk else None,

@@ -43,10 +43,22 @@ def _v_tiles_to_rows(vq: np.ndarray) -> np.ndarray:
     return packed.reshape(lead + (tiles * 16, 64))
 
 
-def _freeze_both(K, V, idx, W, Hq, staging_capacity=128, group=64):
-    ref = od.freeze(wl.bits(K), wl.bits(V), idx, W, group=group, staging_capacity=staging_capacity)
+def _v8_tiles_to_rows(vq: np.ndarray) -> np.ndarray:
+    """Undoes the INT8 fragment-major V layout as the header documents it: [.., tiles, 2048] -> [.., tiles*16, 128]."""
+    lead, tiles = vq.shape[:-2], vq.shape[-2]
+    rows = np.zeros(lead + (tiles, 16, 128), dtype=np.uint8)
+    for key in range(16):
+        for d in range(128):
+            j, r, x = (key & 7) >> 1, (d >> 3) & 7, ((d >> 6) << 2) | ((d >> 1) & 3)
+            w = 2 * x + (key >> 3)
+            rows[..., key, d] = vq[..., (w >> 2) * 512 + (4 * r + j) * 16 + (w & 3) * 4 + (d & 1) * 2 + (key & 1)]
+    return rows.reshape(lead + (tiles * 16, 128))
+
+
+def _freeze_both(K, V, idx, W, Hq, staging_capacity=128, group=64, fmt=oracle.FMT_INT4):
+    ref = od.freeze(wl.bits(K), wl.bits(V), idx, W, group=group, fmts=(fmt, fmt), staging_capacity=staging_capacity)
     idx_t = None if idx is None or idx.shape[2] == 0 else torch.from_numpy(idx).cuda()
-    cache = dapi.hyq_freeze(K.cuda(), V.cuda(), idx_t, W, Hq, staging_capacity, group=group)
+    cache = dapi.hyq_freeze(K.cuda(), V.cuda(), idx_t, W, Hq, staging_capacity, group=group, fmt=fmt)
     torch.cuda.synchronize()
     return ref, cache
 
@@ -66,7 +78,8 @@ def _assert_cache_equal(ref, cache):
     if nQ:
         ng = -(-nQ // ref["group"])
         assert np.array_equal(b["kq_codes"][:, :, :nQ], ref["kq_codes"])
-        assert np.array_equal(_v_tiles_to_rows(b["vq_codes"])[:, :, :nQ], ref["vq_codes"])
+        unpermute = _v8_tiles_to_rows if ref["fmts"][1] == oracle.FMT_INT8 else _v_tiles_to_rows
+        assert np.array_equal(unpermute(b["vq_codes"])[:, :, :nQ], ref["vq_codes"])
         assert np.array_equal(b["kq_scales"][:, :, :ng].view(np.uint32), ref["kq_scales"].view(np.uint32))
         assert np.array_equal(b["vq_scales"][:, :, :ng].view(np.uint32), ref["vq_scales"].view(np.uint32))
     if kk:
@@ -143,6 +156,26 @@ def test_other_group_sizes(group, B, Hq, Hkv, N, W, kk, n_s):
         got = dapi.hyq_hybrid_attention_decode(q.cuda(), cache, splits=splits, out_dtype=torch.float32)
         mx, rel = errors(got.cpu().numpy(), want)
         assert mx <= MAX_ABS_TOL and rel <= MEAN_REL_TOL, (splits, mx, rel)
+
+
+@pytest.mark.parametrize("group", [32, 64, 128])
+@pytest.mark.parametrize("B,Hq,Hkv,N,W,kk,n_s,splits", [(1, 4, 1, 300, 40, 9, 3, 0), (2, 8, 2, 1000, 128, 37, 0, 3), (1, 16, 2, 2117, 100, 50, 17, 0),
+                                                        (1, 2, 2, 64, 0, 0, 1, 1), (1, 5, 1, 777, 33, 21, 2, 7), (1, 4, 2, 200, 20, 180, 5, 2)])
+def test_int8_cache(group, B, Hq, Hkv, N, W, kk, n_s, splits):
+    """K8V8: codes, scales and layouts bit-exact; attention within tolerance (and closer to exact attention than K4V4)."""
+    K, V = rand_bf16((B, Hkv, N, 128), 81, 1.3), rand_bf16((B, Hkv, N, 128), 82)
+    K[:, :, : N // 2] *= 0.05
+    q = rand_bf16((B, Hq, 128), 83, 1.5)
+    idx = _idx(B, Hkv, N - min(W, N), kk, 84) if kk else None
+    ref, cache = _freeze_both(K, V, idx, W, Hq, group=group, fmt=oracle.FMT_INT8)
+    _assert_cache_equal(ref, cache)
+    _stage(ref, cache, n_s, 600)
+    want, lse_want = od.decode_attention(wl.bits(q), ref)
+    lse = torch.empty(B, Hq, dtype=torch.float32, device="cuda")
+    got = dapi.hyq_hybrid_attention_decode(q.cuda(), cache, splits=splits, out_dtype=torch.float32, lse=lse)
+    mx, rel = errors(got.cpu().numpy(), want)
+    assert mx <= MAX_ABS_TOL and rel <= MEAN_REL_TOL, (mx, rel)
+    assert np.abs(lse.cpu().numpy() - lse_want).max() <= 2e-3
 
 
 def test_decode_with_peaked_scores_and_late_maxima():
