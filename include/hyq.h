@@ -41,7 +41,7 @@ extern "C" {
 enum {
   HYQ_OK = 0,
   HYQ_ERR_INVALID_ARG = 1,   /* null pointer, non-positive size, k > P, Hq % Hkv != 0 ... */
-  HYQ_ERR_UNSUPPORTED = 2,   /* D != 128, block_tokens != 64, format combination not built */
+  HYQ_ERR_UNSUPPORTED = 2,   /* D != 128, block_tokens not 32 / 64 / 128, format combination not built */
   HYQ_ERR_WORKSPACE = 3,     /* workspace_bytes smaller than the matching *_workspace query */
   HYQ_ERR_ALIGNMENT = 4,     /* a pointer is not 16-byte aligned */
   HYQ_ERR_CUDA = 5,          /* a CUDA runtime / driver call failed (launch, tensor map) */
@@ -142,7 +142,7 @@ int hyq_select_vertical_mass(const void* q, const void* k_, int B, int Hq, int H
 /* ---------------------------------------------------------------------------------------------
  * hyq_quantize_blocks - Algorithm 2, Stage 2 (per-tile symmetric quantization).
  *
- *   One tile = block_tokens (64) consecutive tokens x all D channels of one (b, head), cut by
+ *   One tile = block_tokens (32, 64 or 128; the workloads use 64) consecutive tokens x all D channels of one (b, head), cut by
  *   original position; the last tile of a head may be ragged.
  *     absmax = max |x| over the tile
  *     scale  = absmax / c          c = 127 (INT8), 448 (FP8 e4m3), 7 (INT4)
@@ -198,7 +198,7 @@ enum { HYQ_WINDOW_SLIDING = 0, HYQ_WINDOW_FIXED_TAIL = 1 };
 typedef struct {
   uint32_t struct_size;
   int32_t B, Hq, Hkv, L, D;
-  int32_t window, k, block_tokens;
+  int32_t window, k, block_tokens;   /* block_tokens: 32, 64 or 128, as given to hyq_quantize_blocks for Q, K and V */
   int32_t q_format, k_format, v_format;
   int32_t out_dtype;                 /* 0 = bf16, 1 = fp32 */
   int32_t impl;                      /* HYQ_IMPL_* */

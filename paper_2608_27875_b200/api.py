@@ -220,7 +220,8 @@ def hyq_hybrid_attention_prefill(q, k, v, q_codes, k_codes, v_codes, q_scales, k
                                  vl_idx, window: int, out: torch.Tensor | None = None, out_dtype=torch.float32,
                                  lse: torch.Tensor | None = None, status_word: torch.Tensor | None = None,
                                  workspace: torch.Tensor | None = None, impl: int = IMPL_AUTO,
-                                 softmax_scale: float = 0.0, window_mode: int = WINDOW_SLIDING) -> torch.Tensor:
+                                 softmax_scale: float = 0.0, window_mode: int = WINDOW_SLIDING,
+                                 block_tokens: int = 64) -> torch.Tensor:
     """Eq. 6-7 / Algorithm 2 Stage 3.  q may hold fewer rows than k, v: the last Lq query rows of the context
     (Algorithm 2's query block).  Returns out [B,Hq,Lq,D] (fp32 by default)."""
     for t, dt, n in ((q, torch.bfloat16, "q"), (k, torch.bfloat16, "k"), (v, torch.bfloat16, "v"),
@@ -233,7 +234,8 @@ def hyq_hybrid_attention_prefill(q, k, v, q_codes, k_codes, v_codes, q_scales, k
     if out is None:
         out = torch.empty(q.shape, dtype=out_dtype, device=q.device)
     args = make_attn_args(q, k, v, q_codes, k_codes, v_codes, q_scales, k_scales, v_scales, fmts, vl_idx, window,
-                          out, lse, status_word, workspace, impl, softmax_scale, window_mode=window_mode)
+                          out, lse, status_word, workspace, impl, softmax_scale, block_tokens=block_tokens,
+                          window_mode=window_mode)
     if workspace is None:
         need = hyq_hybrid_attention_prefill_workspace(args)
         workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=q.device)

@@ -9,6 +9,7 @@ from __future__ import annotations
 
 import glob
 import os
+import re
 import subprocess
 import sys
 from concurrent.futures import ThreadPoolExecutor
@@ -44,7 +45,10 @@ def build(force: bool = False, verbose: bool = False) -> str:
     for src in sources():
         obj = os.path.join(OBJ, os.path.basename(src)[:-3] + ".o")
         objs.append(obj)
-        if force or not os.path.exists(obj) or os.path.getmtime(obj) < max(os.path.getmtime(src), hdr_time):
+        # a source that includes another .cu (the kernels compiled a second time) depends on it
+        dep_time = max([os.path.getmtime(src), hdr_time] +
+                       [os.path.getmtime(os.path.join(CSRC, inc)) for inc in re.findall(r'#include "([^"]+\.cu)"', open(src).read())])
+        if force or not os.path.exists(obj) or os.path.getmtime(obj) < dep_time:
             jobs.append([_nvcc()] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-c", "-o", obj, src])
     if jobs:
         with ThreadPoolExecutor(max_workers=min(8, len(jobs))) as ex:

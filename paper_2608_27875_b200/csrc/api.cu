@@ -8,6 +8,9 @@ size_t attn_simt_workspace_bytes(const hyq_attn_args& a);
 int launch_attn_simt(const hyq_attn_args& a, float alpha, cudaStream_t st);
 size_t attn_tc_workspace_bytes(const hyq_attn_args& a);
 int launch_attn_tc(const hyq_attn_args& a, float alpha, cudaStream_t st);
+namespace tcbt {
+int launch_attn_tc(const hyq_attn_args& a, float alpha, cudaStream_t st);     // 32- and 128-token quantization blocks
+}
 }  // namespace hyq
 
 using namespace hyq;
@@ -126,10 +129,10 @@ int hyq_quantize_blocks(const void* x, int B, int H, int L, int D, int block_tok
                         float* scales_out, void* stream) {
     if (B <= 0 || H <= 0 || L <= 0) return HYQ_ERR_INVALID_ARG;
     if (!x || !codes_out || !scales_out) return HYQ_ERR_INVALID_ARG;
-    if (D != HYQ_D || block_tokens != HYQ_BLOCK_TOKENS) return HYQ_ERR_UNSUPPORTED;
+    if (D != HYQ_D || !block_tokens_ok(block_tokens)) return HYQ_ERR_UNSUPPORTED;
     if (format != HYQ_FMT_INT8 && format != HYQ_FMT_FP8_E4M3 && format != HYQ_FMT_INT4) return HYQ_ERR_UNSUPPORTED;
     if (!aligned16(x) || !aligned16(codes_out) || (reinterpret_cast<uintptr_t>(scales_out) & 3u)) return HYQ_ERR_ALIGNMENT;
-    return launch_quantize(x, (long)B * H, L, format, codes_out, scales_out, static_cast<cudaStream_t>(stream));
+    return launch_quantize(x, (long)B * H, L, block_tokens, format, codes_out, scales_out, static_cast<cudaStream_t>(stream));
 }
 
 static int check_attn(const hyq_attn_args* a, bool need_pointers) {
@@ -139,7 +142,7 @@ static int check_attn(const hyq_attn_args* a, bool need_pointers) {
     if (a->window_mode != HYQ_WINDOW_SLIDING && a->window_mode != HYQ_WINDOW_FIXED_TAIL) return HYQ_ERR_INVALID_ARG;
     if (a->out_dtype != 0 && a->out_dtype != 1) return HYQ_ERR_INVALID_ARG;
     if (a->impl < HYQ_IMPL_AUTO || a->impl > HYQ_IMPL_SIMT) return HYQ_ERR_INVALID_ARG;
-    if (a->D != HYQ_D || a->block_tokens != HYQ_BLOCK_TOKENS) return HYQ_ERR_UNSUPPORTED;
+    if (a->D != HYQ_D || !block_tokens_ok(a->block_tokens)) return HYQ_ERR_UNSUPPORTED;
     const bool int8 = a->q_format == HYQ_FMT_INT8 && a->k_format == HYQ_FMT_INT8 && a->v_format == HYQ_FMT_INT8;
     const bool int4 = a->q_format == HYQ_FMT_INT4 && a->k_format == HYQ_FMT_INT4 && a->v_format == HYQ_FMT_FP8_E4M3;
     const bool fp8 = a->q_format == HYQ_FMT_FP8_E4M3 && a->k_format == HYQ_FMT_FP8_E4M3 && a->v_format == HYQ_FMT_FP8_E4M3;
@@ -172,7 +175,8 @@ int hyq_hybrid_attention_prefill(const hyq_attn_args* args, void* stream) {
     if (need > 0 && (!args->workspace || args->workspace_bytes < need)) return HYQ_ERR_WORKSPACE;
     const float alpha = args->softmax_scale != 0.0f ? args->softmax_scale : 1.0f / sqrtf((float)args->D);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    return use_simt(args) ? launch_attn_simt(*args, alpha, st) : launch_attn_tc(*args, alpha, st);
+    if (use_simt(args)) return launch_attn_simt(*args, alpha, st);
+    return args->block_tokens == HYQ_BLOCK_TOKENS ? launch_attn_tc(*args, alpha, st) : tcbt::launch_attn_tc(*args, alpha, st);
 }
 
 }  // extern "C"

@@ -50,14 +50,14 @@ __global__ void gather_vl_kernel(const __nv_bfloat16* __restrict__ kmat, const _
 // V (bf16) -> fp16 and V^ = code * scale -> fp16; one thread per 8 channels
 template <int V_FMT>
 __global__ void v_to_fp16_kernel(const uint4* __restrict__ v, const uint2* __restrict__ v_codes,
-                                 const float* __restrict__ v_scales, int L, int nb, long n_vec,
+                                 const float* __restrict__ v_scales, int L, int nb, int block_tokens, long n_vec,
                                  uint4* __restrict__ v16, uint4* __restrict__ vh16) {
     const long e = (long)blockIdx.x * blockDim.x + threadIdx.x;
     if (e >= n_vec) return;
     const long row = e / (HYQ_D / 8);                // global token row over all (b, kv head)
     const long head = row / L;
     const int tok = (int)(row - head * L);
-    const float sc = v_scales[head * nb + tok / HYQ_BLOCK_TOKENS];
+    const float sc = v_scales[head * nb + tok / block_tokens];
     const uint4 w = __ldg(v + e);
     const uint32_t ws[4] = {w.x, w.y, w.z, w.w};
     uint32_t o[4], oh[4];
@@ -164,15 +164,15 @@ int launch_tc_prepass(const hyq_attn_args& a, const TcWorkspace& w, cudaStream_t
             a.k, n, reinterpret_cast<__nv_bfloat16*>(base + w.kvl), reinterpret_cast<__half*>(base + w.vvl));
         if (launch_status() != HYQ_OK) return HYQ_ERR_CUDA;
     }
-    const int nb = (a.L + HYQ_BLOCK_TOKENS - 1) / HYQ_BLOCK_TOKENS;
+    const int nb = (a.L + a.block_tokens - 1) / a.block_tokens;
     const long n_vec = (long)a.B * a.Hkv * a.L * (HYQ_D / 8);
     const unsigned vgrid = (unsigned)((n_vec + 255) / 256);
     if (a.v_format == HYQ_FMT_INT8)
         v_to_fp16_kernel<HYQ_FMT_INT8><<<vgrid, 256, 0, st>>>(static_cast<const uint4*>(a.v), static_cast<const uint2*>(a.v_codes),
-            a.v_scales, a.L, nb, n_vec, reinterpret_cast<uint4*>(base + w.v16), reinterpret_cast<uint4*>(base + w.vh16));
+            a.v_scales, a.L, nb, a.block_tokens, n_vec, reinterpret_cast<uint4*>(base + w.v16), reinterpret_cast<uint4*>(base + w.vh16));
     else
         v_to_fp16_kernel<HYQ_FMT_FP8_E4M3><<<vgrid, 256, 0, st>>>(static_cast<const uint4*>(a.v), static_cast<const uint2*>(a.v_codes),
-            a.v_scales, a.L, nb, n_vec, reinterpret_cast<uint4*>(base + w.v16), reinterpret_cast<uint4*>(base + w.vh16));
+            a.v_scales, a.L, nb, a.block_tokens, n_vec, reinterpret_cast<uint4*>(base + w.v16), reinterpret_cast<uint4*>(base + w.vh16));
     if (launch_status() != HYQ_OK) return HYQ_ERR_CUDA;
     if (a.q_format == HYQ_FMT_INT4) {
         const long qw = (long)a.B * a.Hq * query_rows(a) * (HYQ_D / 8), kw = (long)a.B * a.Hkv * a.L * (HYQ_D / 8);

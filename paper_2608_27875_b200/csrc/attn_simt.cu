@@ -78,7 +78,8 @@ attn_simt_kernel(hyq_attn_args a, float alpha, const uint32_t* __restrict__ vl_b
     SimtSmem& sm = *reinterpret_cast<SimtSmem*>(smem_raw);
     // L keys; Lq query rows, end-aligned: query row i sits at position i + off
     const int L = a.L, Lq = query_rows(a), off = L - Lq, g = a.Hq / a.Hkv;
-    const int nb = (L + HYQ_BLOCK_TOKENS - 1) / HYQ_BLOCK_TOKENS, nbq = (Lq + HYQ_BLOCK_TOKENS - 1) / HYQ_BLOCK_TOKENS;
+    const int bt = a.block_tokens;                       // tokens per quantization block (32, 64 or 128)
+    const int nb = (L + bt - 1) / bt, nbq = (Lq + bt - 1) / bt;
     const int i0 = blockIdx.x * ST, h = blockIdx.y, b = blockIdx.z, kvh = h / g;
     const long qhead = (long)b * a.Hq + h, kvhead = (long)b * a.Hkv + kvh;
     const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
@@ -89,7 +90,7 @@ attn_simt_kernel(hyq_attn_args a, float alpha, const uint32_t* __restrict__ vl_b
 
     stage_bf16(sm.q, static_cast<const __nv_bfloat16*>(a.q) + (qhead * Lq + i0) * HYQ_D, n_q);
     stage_codes<QK_FMT>(sm.qc, static_cast<const uint8_t*>(a.q_codes) + (qhead * Lq + i0) * QK_ROW_BYTES, n_q);
-    if (threadIdx.x < ST) sm.q_scale[threadIdx.x] = a.q_scales[qhead * nbq + min(i0 + (int)threadIdx.x, Lq - 1) / HYQ_BLOCK_TOKENS];
+    if (threadIdx.x < ST) sm.q_scale[threadIdx.x] = a.q_scales[qhead * nbq + min(i0 + (int)threadIdx.x, Lq - 1) / bt];
 
     float m_run[4], l_run[4], acc[4][8];
 #pragma unroll
@@ -105,14 +106,14 @@ attn_simt_kernel(hyq_attn_args a, float alpha, const uint32_t* __restrict__ vl_b
         __syncthreads();
         stage_bf16(sm.k, static_cast<const __nv_bfloat16*>(a.k_) + (kvhead * L + j0) * HYQ_D, n_k);
         stage_codes<QK_FMT>(sm.kc, static_cast<const uint8_t*>(a.k_codes) + (kvhead * L + j0) * QK_ROW_BYTES, n_k);
-        if (threadIdx.x < ST) sm.k_scale[threadIdx.x] = a.k_scales[kvhead * nb + min(j0 + (int)threadIdx.x, L - 1) / HYQ_BLOCK_TOKENS];
+        if (threadIdx.x < ST) sm.k_scale[threadIdx.x] = a.k_scales[kvhead * nb + min(j0 + (int)threadIdx.x, L - 1) / bt];
         for (int e = threadIdx.x; e < ST * HYQ_D; e += SIMT_THREADS) {
             const int r = e / HYQ_D, c = e % HYQ_D;
             float vf = 0.0f, vq = 0.0f;
             if (r < n_k) {
                 vf = __bfloat162float(static_cast<const __nv_bfloat16*>(a.v)[(kvhead * L + j0 + r) * HYQ_D + c]);
                 const uint8_t code = static_cast<const uint8_t*>(a.v_codes)[(kvhead * L + j0 + r) * HYQ_D + c];
-                const float sv = a.v_scales[kvhead * nb + (j0 + r) / HYQ_BLOCK_TOKENS];
+                const float sv = a.v_scales[kvhead * nb + (j0 + r) / bt];
                 vq = ((V_FMT == HYQ_FMT_INT8) ? (float)(int8_t)code : e4m3_to_float(code)) * sv;
             }
             sm.v[r * V_STRIDE + c] = vf;

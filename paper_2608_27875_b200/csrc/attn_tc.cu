@@ -29,7 +29,19 @@
 #include "attn_common.cuh"
 #include "sm100.cuh"
 
+// This file is compiled twice: as it stands (64-token quantization blocks, the size every workload uses) and,
+// through attn_tc_bt.cu with HYQ_TC_VARIANT_BT = 1, a second time into namespace hyq::tcbt with the block size a
+// run-time parameter (32 or 128 tokens).  The kernel's loop is sensitive to every live register - compiling the
+// parameter in, even behind a compile-time-false branch, cost the 64-token path 5 % - so the default translation
+// unit is kept token for token what it was.
+#ifndef HYQ_TC_VARIANT_BT
+#define HYQ_TC_VARIANT_BT 0
+#endif
+
 namespace hyq {
+#if HYQ_TC_VARIANT_BT
+namespace tcbt {
+#endif
 using namespace sm100;
 
 constexpr int BM = 128, QT = 2;
@@ -66,7 +78,7 @@ constexpr uint32_t KNOCKOUT_S32 = KNOCKOUT_F32 - INT_MAGIC;   // becomes -inf af
 // Optional timeline trace for tuning (compiled in with -DHYQ_TRACE): SM clock stamps of one CTA's softmax warps
 // (slots 0-3: query tile, column half) and MMA issuers (slots 4, 5) for own tiles 100..163, read back by
 // hyq_debug_read_trace.
-#ifdef HYQ_TRACE
+#if defined(HYQ_TRACE) && !HYQ_TC_VARIANT_BT
 __device__ long long g_trace[6 * 64 * 8];
 #define HYQ_TR(slot, n, e)                                                                                  \
     do {                                                                                                    \
@@ -84,6 +96,9 @@ struct TcMaps {
 
 struct TcParams {
     int B, Hq, Hkv, L, window, k, nb, mask_words;
+#if HYQ_TC_VARIANT_BT
+    int bt_shift;                // log2(tokens per quantization block): 5 or 7
+#endif
     int Lq, nbq;                 // query rows (end-aligned with the L keys: row i sits at position L - Lq + i), their blocks
     int fixed_tail;              // window form: the last `window` keys for every row instead of each row's own
     int splits;                  // CTAs per pair of query tiles, each on a slice of the walk (short query blocks)
@@ -500,7 +515,12 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
             const int col0 = hsel * 32, col0_other = col0 ^ 32;
             const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
             const uint32_t to = tmem + tm_o(q) + lane_addr, ts0 = tmem + tm_s(q) + lane_addr;
+#if HYQ_TC_VARIANT_BT
+            const int bsh = p.bt_shift;
+            const float q_scale = row_live ? __ldg(p.q_scales + (long)qhead * p.nbq + (i >> bsh)) : 0.0f;
+#else
             const float q_scale = row_live ? __ldg(p.q_scales + (long)qhead * p.nbq + i / HYQ_BLOCK_TOKENS) : 0.0f;
+#endif
             constexpr uint32_t knock_lq = LOWBIT_FP8 ? KNOCKOUT_F32 : KNOCKOUT_S32;
             float m_used = -INFINITY, l_h = 0.0f;               // reference maximum of the row; row sum of this half
             bool dead = false;                                  // this warp ran into an expired wait
@@ -514,14 +534,23 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
             };
             // K scale and this half's vertical-line bitmask word of a low-bit tile, fetched one tile ahead of their use
             // (tile n of the low-bit pass sits at walk position n; its block and mask words exist for n < a_end)
+#if HYQ_TC_VARIANT_BT
+            // a 64-key tile n lies in block n / 2 (128-token blocks) or in blocks 2n and 2n + 1, one per column half (32)
+            const float* ks_ptr = p.k_scales + (long)kvhead * p.nb + (bsh == 5 ? hsel : 0);
+#else
             const float* ks_ptr = p.k_scales + (long)kvhead * p.nb;
+#endif
             const uint32_t* vl_ptr = p.vl_bits + (long)qhead * p.mask_words + hsel;
             float nks = 0.0f;
             uint32_t nvl = 0u;
             auto prefetch_tile = [&](int n) {
                 nks = 0.0f; nvl = 0u;
                 if (n >= own.a_end) return;
+#if HYQ_TC_VARIANT_BT
+                nks = __ldg(ks_ptr + ((n << 6) >> bsh));
+#else
                 nks = __ldg(ks_ptr + n);
+#endif
                 nvl = __ldg(vl_ptr + 2 * n);
             };
             prefetch_tile(n0);
@@ -583,7 +612,14 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                             for (int e = 0; e < 32; ++e) oth[e] += INT_MAGIC;
                         }
                         const float fo = row_max32(oth) - (int_scores ? INT_MAGIC_F : 0.0f);
+#if HYQ_TC_VARIANT_BT
+                        // 32-token blocks: the other column half of a low-bit tile has its own K scale
+                        float cs_other = cs;
+                        if (bsh == 5 && n < own.a_end) cs_other = fmaxf(qs2 * __ldg(ks_ptr + 2 * n + 1 - 2 * hsel), 1e-37f);
+                        mo = (fo == -INFINITY) ? -INFINITY : fo * cs_other;
+#else
                         mo = (fo == -INFINITY) ? -INFINITY : fo * cs;
+#endif
                     }
                     tc_fence_before();
                     bar_sync_named(bar_id, 64);                  // both halves are done reading before P is written
@@ -811,13 +847,22 @@ int launch_attn_tc(const hyq_attn_args& a, float alpha, cudaStream_t st) {
 
     TcParams p{};
     p.B = a.B; p.Hq = a.Hq; p.Hkv = a.Hkv; p.L = a.L; p.window = a.window; p.k = a.k;
+#if HYQ_TC_VARIANT_BT
+    p.nb = (a.L + a.block_tokens - 1) / a.block_tokens;
+    p.bt_shift = a.block_tokens == 32 ? 5 : 7;
+#else
     p.nb = (a.L + HYQ_BLOCK_TOKENS - 1) / HYQ_BLOCK_TOKENS;
+#endif
     p.Lq = (int)Lq;
     p.fixed_tail = a.window_mode == HYQ_WINDOW_FIXED_TAIL;
     p.splits = w.splits;
     p.part_o = reinterpret_cast<float*>(base + w.part_o);
     p.part_ml = reinterpret_cast<float*>(base + w.part_ml);
+#if HYQ_TC_VARIANT_BT
+    p.nbq = ((int)Lq + a.block_tokens - 1) / a.block_tokens;
+#else
     p.nbq = ((int)Lq + HYQ_BLOCK_TOKENS - 1) / HYQ_BLOCK_TOKENS;
+#endif
     p.mask_words = w.mask_words;
     p.out_fp32 = a.out_dtype == 1;
     p.scale_log2 = alpha * 1.4426950408889634f;
@@ -847,9 +892,12 @@ int launch_attn_tc(const hyq_attn_args& a, float alpha, cudaStream_t st) {
     return HYQ_OK;
 }
 
+#if HYQ_TC_VARIANT_BT
+}  // namespace tcbt
+#endif
 }  // namespace hyq
 
-#ifdef HYQ_TRACE
+#if defined(HYQ_TRACE) && !HYQ_TC_VARIANT_BT
 extern "C" int hyq_debug_read_trace(long long* dst) {
     return cudaMemcpyFromSymbol(dst, hyq::g_trace, sizeof(hyq::g_trace)) == cudaSuccess ? 0 : 1;
 }

@@ -23,7 +23,8 @@ __host__ __device__ constexpr size_t align_up(size_t x, size_t a) { return (x + 
 static inline int launch_status() { return cudaGetLastError() == cudaSuccess ? HYQ_OK : HYQ_ERR_CUDA; }
 
 // internal launchers (defined in the kernel files)
-int launch_quantize(const void* x, long n_heads, int L, int format, void* codes, float* scales, cudaStream_t st);
+int launch_quantize(const void* x, long n_heads, int L, int block_tokens, int format, void* codes, float* scales, cudaStream_t st);
+static inline bool block_tokens_ok(int bt) { return bt == 32 || bt == 64 || bt == 128; }
 int launch_select(const void* q, const void* k, int B, int Hq, int Hkv, int Lq, int Lk, int window, int n_tail,
                   int k_sel, int32_t* idx_out, void* ws, cudaStream_t st);
 size_t select_workspace_bytes(int B, int Hq, int Lk, int window);

@@ -1,7 +1,7 @@
 // Per-tile symmetric quantization (Algorithm 2, Stage 2).
 //
-// One CTA of 128 threads owns one tile of 64 tokens x 128 channels: 16 KB of bf16 that is
-// contiguous in memory.  Each thread keeps its 64 elements in registers (4 groups of 16
+// One CTA of 2 * BT threads owns one tile of BT (32, 64 or 128) tokens x 128 channels: contiguous bf16
+// (16 KB for the default 64 tokens).  Each thread keeps its 64 elements in registers (4 groups of 16
 // consecutive channels, 32-byte loads), the tile absmax is a warp-shuffle reduction plus one
 // shared-memory step across the 4 warps, and the codes leave as 16-byte (8-bit formats) or
 // 8-byte (INT4) vector stores.  The tile is read once and written once: HBM-bound.
@@ -14,18 +14,18 @@
 
 namespace hyq {
 
-constexpr int QUANT_THREADS = 128;
 constexpr int QUANT_GROUPS = 4;                       // groups of 16 elements per thread
 
-template <int FMT>
-__global__ void __launch_bounds__(QUANT_THREADS)
+template <int FMT, int BT>
+__global__ void __launch_bounds__(2 * BT)
 quantize_tiles_kernel(const uint4* __restrict__ x, int L, int nb, uint8_t* __restrict__ codes,
                       float* __restrict__ scales) {
+    constexpr int QUANT_THREADS = 2 * BT;
     const long tile = blockIdx.x;                     // (b*H + h) * nb + n
     const long head = tile / nb;
     const int n = (int)(tile - head * nb);
-    const int t0 = n * HYQ_BLOCK_TOKENS;
-    const int tokens = min(HYQ_BLOCK_TOKENS, L - t0);
+    const int t0 = n * BT;
+    const int tokens = min(BT, L - t0);
     const int n_elems = tokens * HYQ_D;
     const long elem0 = (head * L + t0) * (long)HYQ_D;
     const uint4* src = x + elem0 / 8;
@@ -54,7 +54,9 @@ quantize_tiles_kernel(const uint4* __restrict__ x, int L, int nb, uint8_t* __res
     __shared__ float warp_max[QUANT_THREADS / 32];
     if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = amax;
     __syncthreads();
-    amax = fmaxf(fmaxf(warp_max[0], warp_max[1]), fmaxf(warp_max[2], warp_max[3]));
+    amax = warp_max[0];
+#pragma unroll
+    for (int w = 1; w < QUANT_THREADS / 32; ++w) amax = fmaxf(amax, warp_max[w]);
 
     constexpr float c = (FMT == HYQ_FMT_INT8) ? 127.0f : (FMT == HYQ_FMT_FP8_E4M3) ? 448.0f : 7.0f;
     const bool dead = !(amax >= 0x1p-100f);
@@ -103,21 +105,31 @@ quantize_tiles_kernel(const uint4* __restrict__ x, int L, int nb, uint8_t* __res
     }
 }
 
-int launch_quantize(const void* x, long n_heads, int L, int format, void* codes, float* scales, cudaStream_t st) {
-    const int nb = (L + HYQ_BLOCK_TOKENS - 1) / HYQ_BLOCK_TOKENS;
-    const long tiles = n_heads * nb;
-    if (tiles <= 0) return HYQ_OK;
-    if (tiles > 0x7fffffffL) return HYQ_ERR_INVALID_ARG;
-    const dim3 grid((unsigned)tiles), block(QUANT_THREADS);
-    const uint4* xs = static_cast<const uint4*>(x);
-    uint8_t* cs = static_cast<uint8_t*>(codes);
+template <int BT>
+static int launch_quantize_bt(const uint4* xs, long tiles, int L, int nb, int format, uint8_t* cs, float* scales, cudaStream_t st) {
+    const dim3 grid((unsigned)tiles), block(2 * BT);
     switch (format) {
-        case HYQ_FMT_INT8: quantize_tiles_kernel<HYQ_FMT_INT8><<<grid, block, 0, st>>>(xs, L, nb, cs, scales); break;
-        case HYQ_FMT_FP8_E4M3: quantize_tiles_kernel<HYQ_FMT_FP8_E4M3><<<grid, block, 0, st>>>(xs, L, nb, cs, scales); break;
-        case HYQ_FMT_INT4: quantize_tiles_kernel<HYQ_FMT_INT4><<<grid, block, 0, st>>>(xs, L, nb, cs, scales); break;
+        case HYQ_FMT_INT8: quantize_tiles_kernel<HYQ_FMT_INT8, BT><<<grid, block, 0, st>>>(xs, L, nb, cs, scales); break;
+        case HYQ_FMT_FP8_E4M3: quantize_tiles_kernel<HYQ_FMT_FP8_E4M3, BT><<<grid, block, 0, st>>>(xs, L, nb, cs, scales); break;
+        case HYQ_FMT_INT4: quantize_tiles_kernel<HYQ_FMT_INT4, BT><<<grid, block, 0, st>>>(xs, L, nb, cs, scales); break;
         default: return HYQ_ERR_UNSUPPORTED;
     }
     return launch_status();
+}
+
+int launch_quantize(const void* x, long n_heads, int L, int block_tokens, int format, void* codes, float* scales, cudaStream_t st) {
+    const int nb = (L + block_tokens - 1) / block_tokens;
+    const long tiles = n_heads * nb;
+    if (tiles <= 0) return HYQ_OK;
+    if (tiles > 0x7fffffffL) return HYQ_ERR_INVALID_ARG;
+    const uint4* xs = static_cast<const uint4*>(x);
+    uint8_t* cs = static_cast<uint8_t*>(codes);
+    switch (block_tokens) {
+        case 32: return launch_quantize_bt<32>(xs, tiles, L, nb, format, cs, scales, st);
+        case 64: return launch_quantize_bt<64>(xs, tiles, L, nb, format, cs, scales, st);
+        case 128: return launch_quantize_bt<128>(xs, tiles, L, nb, format, cs, scales, st);
+        default: return HYQ_ERR_UNSUPPORTED;
+    }
 }
 
 }  // namespace hyq

@@ -26,11 +26,11 @@ def errors(got: np.ndarray, ref: np.ndarray):
     return float(d.max()), float(d.sum() / np.abs(ref).sum())
 
 
-def oracle_quant_all(Q, K, V, fmts):
-    return [oracle.quantize(wl.bits(t), f, 64) for t, f in zip((Q, K, V), fmts)]
+def oracle_quant_all(Q, K, V, fmts, block_tokens=64):
+    return [oracle.quantize(wl.bits(t), f, block_tokens) for t, f in zip((Q, K, V), fmts)]
 
 
-def gpu_attention(Q, K, V, qz, fmts, idx, window, impl, out_dtype=torch.float32, lse=False, window_mode=0):
+def gpu_attention(Q, K, V, qz, fmts, idx, window, impl, out_dtype=torch.float32, lse=False, window_mode=0, block_tokens=64):
     """Runs the library's attention on the oracle's codes/scales/indices (so that this step is
     compared on identical inputs)."""
     dev = "cuda"
@@ -41,7 +41,7 @@ def gpu_attention(Q, K, V, qz, fmts, idx, window, impl, out_dtype=torch.float32,
     status = torch.zeros(1, dtype=torch.int32, device=dev)
     out = api.hyq_hybrid_attention_prefill(Q.to(dev), K.to(dev), V.to(dev), t(qc), t(kc), t(vc), t(qs), t(ks), t(vs),
                                            fmts, idx_t, window, impl=impl, out_dtype=out_dtype, lse=lse_t,
-                                           status_word=status, window_mode=window_mode)
+                                           status_word=status, window_mode=window_mode, block_tokens=block_tokens)
     torch.cuda.synchronize()
     assert int(status.item()) == 0, "kernel reported a device-side error"
     return (out.cpu(), lse_t.cpu()) if lse else out.cpu()

@@ -69,7 +69,7 @@ def test_select_argument_checks(lib):
 def test_quantize_argument_checks(lib):
     assert lib.hyq_quantize_blocks(None, 1, 1, 64, 128, 64, 0, None, None, None) == 1
     assert lib.hyq_quantize_blocks(0x1000, 1, 1, 64, 64, 64, 0, 0x2000, 0x3000, None) == 2      # D
-    assert lib.hyq_quantize_blocks(0x1000, 1, 1, 64, 128, 32, 0, 0x2000, 0x3000, None) == 2     # block size
+    assert lib.hyq_quantize_blocks(0x1000, 1, 1, 64, 128, 48, 0, 0x2000, 0x3000, None) == 2     # block size (32, 64, 128 only)
     assert lib.hyq_quantize_blocks(0x1000, 1, 1, 64, 128, 64, 7, 0x2000, 0x3000, None) == 2     # format
     assert lib.hyq_quantize_blocks(0x1004, 1, 1, 64, 128, 64, 0, 0x2000, 0x3000, None) == 4
     assert lib.hyq_quantize_blocks(0x1000, 0, 1, 64, 128, 64, 0, 0x2000, 0x3000, None) == 1
@@ -97,7 +97,7 @@ def test_attention_argument_checks(lib):
     assert call(_args(struct_size=8)) == 1
     assert call(_args(Hkv=3)) == 1
     assert call(_args(D=64)) == 2
-    assert call(_args(block_tokens=32)) == 2
+    assert call(_args(block_tokens=48)) == 2
     assert call(_args(q_format=1, k_format=0, v_format=1)) == 2       # Q and K formats must match
     assert call(_args(q_format=2, k_format=2, v_format=0)) == 2       # INT4 with INT8 V not built
     assert call(_args(Lq=-1)) == 1

@@ -60,6 +60,24 @@ def test_small_shapes_match_oracle(impl, fmts, B, Hq, Hkv, L, W, k):
 
 
 @pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("bt", [32, 128])
+@pytest.mark.parametrize("fmts", [INT8, INT4FP8, FP8ALL])
+@pytest.mark.parametrize("B,Hq,Hkv,L,W,k", [(1, 2, 2, 512, 128, 16), (2, 4, 2, 333, 40, 9), (1, 2, 2, 200, 0, 12), (1, 4, 1, 1000, 64, 30)])
+def test_other_quantization_block_sizes(impl, bt, fmts, B, Hq, Hkv, L, W, k):
+    """32- and 128-token quantization blocks (scales per half tile / per two tiles); K rows of very different
+    magnitude so that neighbouring blocks have very different scales."""
+    Q, K, V = (rand_bf16((B, h, L, 128), seed=L + n + bt) for n, h in enumerate((Hq, Hkv, Hkv)))
+    K = (K.float() * (1.0 + 3.0 * ((torch.arange(L) // 32) % 3).view(1, 1, L, 1))).to(torch.bfloat16)
+    idx = _rand_idx(B, Hq, max(0, L - W), k, seed=L)
+    ensure_built()
+    qz = oracle_quant_all(Q, K, V, fmts, bt)
+    got = gpu_attention(Q, K, V, qz, fmts, idx, W, impl, block_tokens=bt).numpy()
+    ref = _ref(Q, K, V, qz, fmts, idx, W, None, block_tokens=bt)
+    max_abs, mean_rel = errors(got, ref)
+    assert np.isfinite(got).all() and max_abs <= MAX_ABS_TOL and mean_rel <= MEAN_REL_TOL, (max_abs, mean_rel)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
 def test_vertical_keys_inside_the_window_and_beyond_the_diagonal(impl):
     """Index sets are free to name keys that a given row sees through its window or not at all."""
     L, W = 300, 50

@@ -11,11 +11,11 @@ pytestmark = pytest.mark.gpu
 FMTS = [wl.FMT_INT8, wl.FMT_FP8_E4M3, wl.FMT_INT4]
 
 
-def _check(x, fmt):
+def _check(x, fmt, bt=64):
     ensure_built()
-    codes, scales = api.hyq_quantize_blocks(x.cuda(), fmt)
+    codes, scales = api.hyq_quantize_blocks(x.cuda(), fmt, bt)
     torch.cuda.synchronize()
-    ref_codes, ref_scales = oracle.quantize(wl.bits(x), fmt, 64)
+    ref_codes, ref_scales = oracle.quantize(wl.bits(x), fmt, bt)
     np.testing.assert_array_equal(scales.cpu().numpy().view(np.uint32), ref_scales.view(np.uint32))
     np.testing.assert_array_equal(codes.cpu().numpy(), ref_codes)
 
@@ -24,6 +24,13 @@ def _check(x, fmt):
 @pytest.mark.parametrize("shape", [(1, 2, 2048, 128), (2, 3, 1000, 128), (1, 1, 1, 128), (1, 5, 63, 128), (1, 2, 65, 128)])
 def test_matches_oracle(fmt, shape):
     _check(rand_bf16(shape, seed=sum(shape) + fmt), fmt)
+
+
+@pytest.mark.parametrize("bt", [32, 128])
+@pytest.mark.parametrize("fmt", FMTS)
+@pytest.mark.parametrize("shape", [(1, 2, 2048, 128), (2, 3, 1000, 128), (1, 1, 1, 128), (1, 5, 127, 128), (1, 2, 129, 128)])
+def test_other_block_sizes_match_oracle(fmt, shape, bt):
+    _check(rand_bf16(shape, seed=sum(shape) + fmt + bt), fmt, bt)
 
 
 @pytest.mark.parametrize("fmt", FMTS)
