@@ -78,3 +78,56 @@ def test_two_ranks_reproduce_the_unsharded_result():
     np.testing.assert_array_equal(ret["idx"], ref["idx"])
     np.testing.assert_allclose(ret["out"], ref["out"], rtol=0, atol=1e-13)
     assert ret["t_max"] == 11.0                            # max over ranks of (10, 11)
+
+
+# ---- the decode side shards by the same (batch, KV head) units ------------------------------------------------
+def _decode_inputs():
+    g = torch.Generator().manual_seed(91)
+    B, Hq, Hkv, N, D = 2, 6, 3, 150, 16
+    k = torch.randn(B, Hkv, N, D, generator=g).to(torch.bfloat16)
+    v = torch.randn(B, Hkv, N, D, generator=g).to(torch.bfloat16)
+    q = torch.randn(B, Hq, D, generator=g).to(torch.bfloat16)
+    rng = np.random.default_rng(92)
+    idx = np.stack([np.stack([np.sort(rng.choice(N - 20, 7, replace=False)) for _ in range(Hkv)]) for _ in range(B)]).astype(np.int32)
+    return q, k, v, idx
+
+
+def _decode_worker(rank, world, port, ret):
+    from oracle import decode as od
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        q, k, v, idx = _decode_inputs()
+        g = q.shape[1] // k.shape[1]
+        mine = {}
+        for b, kvh in sharding.shard_units(k.shape[0], k.shape[1], world, rank):
+            # Freeze and one token on this unit's tensors alone
+            cache = od.freeze(wl.bits(k[b:b + 1, kvh:kvh + 1]), wl.bits(v[b:b + 1, kvh:kvh + 1]), idx[b:b + 1, kvh:kvh + 1], 20, group=16)
+            out, _ = od.decode_attention(wl.bits(q[b:b + 1, kvh * g:(kvh + 1) * g]), cache)
+            mine[(b, kvh)] = out[0]
+        gathered = [None] * world
+        dist.all_gather_object(gathered, mine)
+        if rank == 0:
+            full = {}
+            for part in gathered:
+                assert not (set(part) & set(full))
+                full.update(part)
+            out = np.zeros((q.shape[0], q.shape[1], q.shape[2]))
+            for (b, kvh), o_ in full.items():
+                out[b, kvh * g:(kvh + 1) * g] = o_
+            ret["out"], ret["n_units"] = out, len(full)
+    finally:
+        dist.destroy_process_group()
+
+
+def test_two_ranks_reproduce_the_unsharded_decode_step():
+    from oracle import decode as od
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    ret = mp.Manager().dict()
+    mp.spawn(_decode_worker, args=(2, port, ret), nprocs=2, join=True)
+    q, k, v, idx = _decode_inputs()
+    ref, _ = od.decode_attention(wl.bits(q), od.freeze(wl.bits(k), wl.bits(v), idx, 20, group=16))
+    assert ret["n_units"] == k.shape[0] * k.shape[1]
+    np.testing.assert_allclose(ret["out"], ref, rtol=0, atol=1e-13)
