@@ -7,7 +7,8 @@
  *
  * The common rules of hyq.h hold (device pointers, contiguous row-major arrays, caller-owned buffers,
  * calls enqueue on `stream` and return, arguments checked on the host before anything is launched,
- * D = 128, Hq % Hkv == 0 with g = Hq / Hkv <= 8 query heads per KV head).
+ * D = 128, Hq % Hkv == 0 with g = Hq / Hkv <= 64 query heads per KV head; more than 8 are served 8 at a time by
+ * separate CTAs that read the same cache rows).
  *
  * The hybrid cache of one layer (Algorithm 4's four buffers), per (batch b, KV head h):
  *
@@ -100,7 +101,7 @@ int hyq_kv_cache_query_sizes(const hyq_kv_cache* cache, hyq_kv_cache_sizes* size
  * vertical and quantized buffers of `cache` (layouts above).  The staging buffers are not touched
  * (an empty staging buffer is n_staging = 0).  The prefill cache may be freed once the enqueued
  * work has completed.  Errors: INVALID_ARG (null pointer, sizes out of range, struct_size),
- * UNSUPPORTED (D != 128, group not 32 / 64 / 128, format not INT4 / INT8, g > 8), ALIGNMENT (any buffer not 16-byte aligned).
+ * UNSUPPORTED (D != 128, group not 32 / 64 / 128, format not INT4 / INT8, g > 64), ALIGNMENT (any buffer not 16-byte aligned).
  * ------------------------------------------------------------------------------------------- */
 int hyq_freeze(const void* k_, const void* v, const int32_t* vl_idx, const hyq_kv_cache* cache, void* stream);
 

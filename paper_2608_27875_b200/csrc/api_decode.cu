@@ -12,11 +12,11 @@ static int check_cache(const hyq_kv_cache* c, bool need_pointers) {
     if (c->staging_capacity < 0 || c->n_staging < 0 || c->n_staging > c->staging_capacity) return HYQ_ERR_INVALID_ARG;
     if (c->D != HYQ_D || (c->group != 32 && c->group != 64 && c->group != 128) ||
         (c->format != HYQ_FMT_INT4 && c->format != HYQ_FMT_INT8) ||
-        c->Hq / c->Hkv > DEC_MAX_GROUP)
+        c->Hq / c->Hkv > 8 * DEC_MAX_GROUP)
         return HYQ_ERR_UNSUPPORTED;
     const CacheGeo g = cache_geo(*c);
     if (c->k > c->N - g.W) return HYQ_ERR_INVALID_ARG;
-    if ((long)c->B * c->Hkv > 65535) return HYQ_ERR_UNSUPPORTED;
+    if ((long)c->B * c->Hkv * ((c->Hq / c->Hkv + DEC_MAX_GROUP - 1) / DEC_MAX_GROUP) > 65535) return HYQ_ERR_UNSUPPORTED;
     if (c->cap_quantized_rows < 0 || c->cap_vertical < 0 || c->cap_window < 0) return HYQ_ERR_INVALID_ARG;
     if ((c->cap_quantized_rows && (c->cap_quantized_rows % c->group || c->cap_quantized_rows < g.nQp)) ||
         (c->cap_vertical && c->cap_vertical < c->k) || (c->cap_window && c->cap_window < g.W))

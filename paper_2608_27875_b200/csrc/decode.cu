@@ -49,6 +49,7 @@ constexpr float DEC_RAISE = 8.0f;          // log2 units; P <= 2^8 stays far ins
 
 struct DecParams {
     int g, splits, Hkv;
+    int hgroups;         // ceil(g / 8): a KV head with more than 8 query heads is served by several CTAs per slice
     int gshift;          // log2(rows per scale group / 16): 16-row tile t belongs to group t >> gshift
     long nQ, sQ;         // quantized rows per head (valid), rows between heads
     int k, W, n_s;       // valid rows of the vertical, window and staging buffers ...
@@ -304,7 +305,9 @@ template <bool FMT8>
 __global__ void __launch_bounds__(DEC_THREADS, DEC_CTAS_PER_SM)
 decode_kernel(const DecParams p) {
     const int split = blockIdx.x;
-    const long unit = blockIdx.y;
+    // blockIdx.y = (b * Hkv + kv head) * hgroups + head group: up to 8 of the KV head's g query heads per CTA
+    const long unit = blockIdx.y / p.hgroups;
+    const int h_base = (int)(blockIdx.y % p.hgroups) * DEC_MAX_GROUP, g_here = min(DEC_MAX_GROUP, p.g - h_base);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, r = lane >> 2, j = lane & 3;
     // the merge kernel may be made resident while this grid runs (programmatic dependent launch): it waits for
     // this grid's completion before it reads anything, so only its launch latency is taken off the path
@@ -323,7 +326,7 @@ decode_kernel(const DecParams p) {
     {   // q of the g heads of this KV head: thread t loads 8 channels of head t >> 4
         const int h = threadIdx.x >> 4, c8 = threadIdx.x & 15;
         uint4 v = make_uint4(0, 0, 0, 0);
-        if (h < p.g) v = __ldg(p.q + (unit * p.g + h) * 16 + c8);
+        if (h < g_here) v = __ldg(p.q + (unit * p.g + h_base + h) * 16 + c8);
         *reinterpret_cast<uint4*>(&qs[h][c8 * 8]) = v;
         // Odd channels sit in the high nibbles: their q enters the product as fp16(q / 16), times 16 here.
         const uint32_t w[4] = {v.x, v.y, v.z, v.w};
@@ -553,8 +556,8 @@ decode_kernel(const DecParams p) {
         red_acc[warp][2 * j + 1][acc_channel(x, r, 1)] = acc[x][3];
     }
     __syncthreads();
-    const long slot = unit * p.splits + split;
-    for (int h = 0; h < p.g; ++h) {
+    const long slot = (long)blockIdx.y * p.splits + split;
+    for (int h = 0; h < g_here; ++h) {
         float M = -INFINITY;
 #pragma unroll
         for (int w = 0; w < DEC_WARPS; ++w) M = fmaxf(M, red_ml[w][h][0]);
@@ -579,10 +582,12 @@ decode_kernel(const DecParams p) {
 // independent loads (the kernel is pure latency otherwise: it moves a few hundred KB).
 constexpr int DEC_MAX_SPLITS = 1024;
 __global__ void __launch_bounds__(HYQ_D)
-decode_merge_kernel(const float* __restrict__ part_acc, const float* __restrict__ part_ml, int g, int splits,
+decode_merge_kernel(const float* __restrict__ part_acc, const float* __restrict__ part_ml, int g, int hgroups, int splits,
                     int out_fp32, void* __restrict__ out, float* __restrict__ lse) {
-    const long unit = blockIdx.x;
-    const int h = blockIdx.y;
+    const long unit = blockIdx.x;                                  // (b * Hkv + kv head) * hgroups + head group
+    const int h = blockIdx.y;                                      // head within the group
+    const int h_base = (int)(unit % hgroups) * DEC_MAX_GROUP;
+    if (h_base + h >= g) return;
     asm volatile("griddepcontrol.wait;" ::: "memory");       // the slice kernel has completed and its results are visible
     __shared__ float wt[DEC_MAX_SPLITS];
     __shared__ float red[2][HYQ_D / 32];
@@ -612,10 +617,11 @@ decode_merge_kernel(const float* __restrict__ part_acc, const float* __restrict_
 #pragma unroll 8
     for (int s = 0; s < splits; ++s) A += __ldg(part_acc + (slot0 + (long)s * DEC_MAX_GROUP) * HYQ_D + threadIdx.x) * wt[s];
     const float o = L > 0.0f ? A / L : 0.0f;               // a sequence with no cached row at all: zeros
-    const long oi = (unit * g + h) * HYQ_D + threadIdx.x;
+    const long head = (unit / hgroups) * g + h_base + h;
+    const long oi = head * HYQ_D + threadIdx.x;
     if (out_fp32) static_cast<float*>(out)[oi] = o;
     else static_cast<__nv_bfloat16*>(out)[oi] = __float2bfloat16_rn(o);
-    if (lse && threadIdx.x == 0) lse[unit * g + h] = (M + log2f(L)) * 0.6931471805599453f;
+    if (lse && threadIdx.x == 0) lse[head] = (M + log2f(L)) * 0.6931471805599453f;
 }
 
 static long decode_tiles(const hyq_kv_cache& c) {
@@ -624,7 +630,7 @@ static long decode_tiles(const hyq_kv_cache& c) {
 }
 
 int decode_auto_splits(const hyq_kv_cache& c) {
-    const long units = (long)c.B * c.Hkv;
+    const long units = (long)c.B * c.Hkv * ((c.Hq / c.Hkv + DEC_MAX_GROUP - 1) / DEC_MAX_GROUP);
     const long T = decode_tiles(c);
     long s = 148L * DEC_CTAS_PER_SM / units;            // one full wave of resident CTAs, never a second partial one
     const long cap = T / 8 > 1 ? T / 8 : 1;             // at least two tiles per warp on average
@@ -634,16 +640,17 @@ int decode_auto_splits(const hyq_kv_cache& c) {
 }
 
 size_t decode_workspace_bytes(const hyq_kv_cache& c, int splits) {
-    const size_t slots = (size_t)c.B * c.Hkv * splits * DEC_MAX_GROUP;
+    const size_t slots = (size_t)c.B * c.Hkv * ((c.Hq / c.Hkv + DEC_MAX_GROUP - 1) / DEC_MAX_GROUP) * splits * DEC_MAX_GROUP;
     return align_up(slots * HYQ_D * sizeof(float), 16) + align_up(slots * 2 * sizeof(float), 16);
 }
 
 int launch_decode(const void* q, const hyq_kv_cache& c, const int32_t* lengths, float alpha, int splits, int out_dtype,
                   void* out, float* lse, void* workspace, cudaStream_t st) {
     const CacheGeo geo = cache_geo(c);
-    const long units = (long)c.B * c.Hkv;
     DecParams p;
     p.g = c.Hq / c.Hkv; p.splits = splits;
+    p.hgroups = (p.g + DEC_MAX_GROUP - 1) / DEC_MAX_GROUP;
+    const long units = (long)c.B * c.Hkv * p.hgroups;         // CTA rows of the grid: (b, kv head, head group)
     p.gshift = c.group == 32 ? 1 : c.group == 64 ? 2 : 3;
     p.Hkv = c.Hkv; p.lens = reinterpret_cast<const int4*>(lengths);
     p.nQ = geo.nQ; p.sQ = geo.sQ; p.k = c.k; p.W = geo.W; p.n_s = c.n_staging;
@@ -669,7 +676,7 @@ int launch_decode(const void* q, const hyq_kv_cache& c, const int32_t* lengths, 
     if (c.format == HYQ_FMT_INT8) decode_kernel<true><<<dim3((unsigned)splits, (unsigned)units), DEC_THREADS, ring_bytes, st>>>(p);
     else decode_kernel<false><<<dim3((unsigned)splits, (unsigned)units), DEC_THREADS, ring_bytes, st>>>(p);
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)units, (unsigned)p.g);
+    cfg.gridDim = dim3((unsigned)units, (unsigned)(p.g < DEC_MAX_GROUP ? p.g : DEC_MAX_GROUP));
     cfg.blockDim = dim3(HYQ_D);
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
@@ -679,7 +686,7 @@ int launch_decode(const void* q, const hyq_kv_cache& c, const int32_t* lengths, 
     cfg.numAttrs = 1;
     const float* pa = p.part_acc;
     const float* pm = p.part_ml;
-    if (cudaLaunchKernelEx(&cfg, decode_merge_kernel, pa, pm, p.g, splits, out_dtype, out, lse) != cudaSuccess) return HYQ_ERR_CUDA;
+    if (cudaLaunchKernelEx(&cfg, decode_merge_kernel, pa, pm, p.g, p.hgroups, splits, out_dtype, out, lse) != cudaSuccess) return HYQ_ERR_CUDA;
     return launch_status();
 }
 

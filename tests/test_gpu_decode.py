@@ -178,6 +178,24 @@ def test_int8_cache(group, B, Hq, Hkv, N, W, kk, n_s, splits):
     assert np.abs(lse.cpu().numpy() - lse_want).max() <= 2e-3
 
 
+@pytest.mark.parametrize("fmt", [oracle.FMT_INT4, oracle.FMT_INT8])
+@pytest.mark.parametrize("B,Hq,Hkv,N,W,kk,n_s,splits", [(1, 32, 2, 1500, 64, 30, 5, 0), (2, 12, 1, 700, 32, 11, 0, 3), (1, 18, 2, 333, 40, 9, 2, 1),
+                                                        (1, 64, 1, 400, 16, 5, 1, 2)])
+def test_more_than_eight_query_heads_per_kv_head(fmt, B, Hq, Hkv, N, W, kk, n_s, splits):
+    """g = 16 (two KV heads for 32 query heads), 12, 9 and 64: eight heads per CTA, several CTAs per slice."""
+    K, V = rand_bf16((B, Hkv, N, 128), 91, 1.3), rand_bf16((B, Hkv, N, 128), 92)
+    q = rand_bf16((B, Hq, 128), 93, 1.5)
+    idx = _idx(B, Hkv, N - W, kk, 94)
+    ref, cache = _freeze_both(K, V, idx, W, Hq, fmt=fmt)
+    _stage(ref, cache, n_s, 800)
+    want, lse_want = od.decode_attention(wl.bits(q), ref)
+    lse = torch.empty(B, Hq, dtype=torch.float32, device="cuda")
+    got = dapi.hyq_hybrid_attention_decode(q.cuda(), cache, splits=splits, out_dtype=torch.float32, lse=lse)
+    mx, rel = errors(got.cpu().numpy(), want)
+    assert mx <= MAX_ABS_TOL and rel <= MEAN_REL_TOL, (mx, rel)
+    assert np.abs(lse.cpu().numpy() - lse_want).max() <= 2e-3
+
+
 def test_decode_with_peaked_scores_and_late_maxima():
     """A planted key that dominates (scores far above the rest) sits late in the quantized prefix, another
     in the window: the lazy reference maximum has to be raised mid-stream in several warps and slices."""
