@@ -525,14 +525,21 @@ decode_kernel(const DecParams p) {
             float pw[4];
             if (row0 + 16 > n) softmax_tile<true>(st, acc, c4, p.scale_log2, 0.0f, 0.0f, row0 + r < n, row0 + r + 8 < n, pw);
             else softmax_tile<false>(st, acc, c4, p.scale_log2, 0.0f, 0.0f, true, true, pw);
-            const uint32_t b0 = movmatrix_trans(pack_bf16(pw[0], pw[1]));
-            const uint32_t b1 = movmatrix_trans(pack_bf16(pw[2], pw[3]));
+            // The weights go into the bf16 product as a sum of two bf16 numbers (p = hi + lo, 16 significant bits):
+            // with one bf16 the 2^-9 rounding of a dominant full-precision key would show in the output.
+            const uint32_t h01 = pack_bf16(pw[0], pw[1]), h23 = pack_bf16(pw[2], pw[3]);
+            const uint32_t l01 = pack_bf16(pw[0] - bf16_lo(h01), pw[1] - bf16_hi(h01));
+            const uint32_t l23 = pack_bf16(pw[2] - bf16_lo(h23), pw[3] - bf16_hi(h23));
+            const uint32_t b0 = movmatrix_trans(h01), b1 = movmatrix_trans(h23);
+            const uint32_t b0l = movmatrix_trans(l01), b1l = movmatrix_trans(l23);
 #pragma unroll
             for (int x = 0; x < 8; ++x) {
                 const uint32_t w0 = word_of(vv[0][x >> 2], x & 3), w1 = word_of(vv[1][x >> 2], x & 3);
                 const uint32_t w2 = word_of(vv[2][x >> 2], x & 3), w3 = word_of(vv[3][x >> 2], x & 3);
-                mma_bf16(acc[x], __byte_perm(w0, w1, 0x5410), __byte_perm(w0, w1, 0x7632), __byte_perm(w2, w3, 0x5410),
-                         __byte_perm(w2, w3, 0x7632), b0, b1);
+                const uint32_t a0 = __byte_perm(w0, w1, 0x5410), a1 = __byte_perm(w0, w1, 0x7632);
+                const uint32_t a2 = __byte_perm(w2, w3, 0x5410), a3 = __byte_perm(w2, w3, 0x7632);
+                mma_bf16(acc[x], a0, a1, a2, a3, b0, b1);
+                mma_bf16(acc[x], a0, a1, a2, a3, b0l, b1l);
             }
         }
     }

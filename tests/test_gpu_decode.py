@@ -216,6 +216,25 @@ def test_decode_with_peaked_scores_and_late_maxima():
         assert mx <= MAX_ABS_TOL and rel <= MEAN_REL_TOL, (splits, mx, rel)
 
 
+def test_a_dominant_full_precision_key_keeps_its_precision():
+    """One window key takes almost all of the weight: the output is that key's value row, so any rounding of the
+    weights in the full-precision product shows directly.  (A single bf16 weight would leave 1e-3 here.)"""
+    B, Hq, Hkv, N, W = 1, 4, 2, 700, 64
+    K, V = rand_bf16((B, Hkv, N, 128), 101, 0.3), rand_bf16((B, Hkv, N, 128), 102, 2.0)
+    q = rand_bf16((B, Hq, 128), 103)
+    u = torch.nn.functional.normalize(torch.randn(128, generator=torch.Generator().manual_seed(104)), dim=0)
+    q = (q.float() + 8.0 * u).to(torch.bfloat16)
+    for pos, amp in ((N - 7, 6.0), (N - 30, 5.5)):                      # two window keys of comparable, dominant weight
+        K[:, :, pos] = (K[:, :, pos].float() + amp * u).to(torch.bfloat16)
+    idx = _idx(B, Hkv, N - W, 20, 105)
+    for fmt in (oracle.FMT_INT4, oracle.FMT_INT8):
+        ref, cache = _freeze_both(K, V, idx, W, Hq, fmt=fmt)
+        want, _ = od.decode_attention(wl.bits(q), ref)
+        got = dapi.hyq_hybrid_attention_decode(q.cuda(), cache, out_dtype=torch.float32)
+        mx, rel = errors(got.cpu().numpy(), want)
+        assert rel <= 4e-4, (fmt, mx, rel)
+
+
 def test_decode_at_benchmark_size_and_repeatable():
     """The benchmark's cache shape (32 / 8 heads, 32768 frozen rows, 2 % vertical, window 1024, a full staging
     buffer) at batch 2, every head against the oracle; two runs are bit-identical."""
