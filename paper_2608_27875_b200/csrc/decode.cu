@@ -673,12 +673,16 @@ int launch_decode(const void* q, const hyq_kv_cache& c, const int32_t* lengths, 
     p.part_acc = static_cast<float*>(workspace);
     p.part_ml = reinterpret_cast<float*>(static_cast<char*>(workspace) + align_up(slots * HYQ_D * sizeof(float), 16));
     constexpr int ring_bytes = DEC_WARPS * DEC_STAGES * DEC_STAGE_BYTES;
-    static bool attr_set = false;          // same value every time: a benign race between host threads
-    if (!attr_set) {
+    // the opt-in to more than 48 KB of dynamic shared memory is per device: once per device and process
+    // (same value every time, so a race between host threads is benign)
+    static bool attr_set[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return HYQ_ERR_CUDA;
+    if (!attr_set[dev]) {
         if (cudaFuncSetAttribute(decode_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, ring_bytes) != cudaSuccess ||
             cudaFuncSetAttribute(decode_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ring_bytes) != cudaSuccess)
             return HYQ_ERR_CUDA;
-        attr_set = true;
+        attr_set[dev] = true;
     }
     if (c.format == HYQ_FMT_INT8) decode_kernel<true><<<dim3((unsigned)splits, (unsigned)units), DEC_THREADS, ring_bytes, st>>>(p);
     else decode_kernel<false><<<dim3((unsigned)splits, (unsigned)units), DEC_THREADS, ring_bytes, st>>>(p);

@@ -229,12 +229,15 @@ int launch_select_mass(const void* q, const void* k, int B, int Hq, int Hkv, int
     const auto* kb = static_cast<const __nv_bfloat16*>(k);
 
     constexpr int smem = MASS_QTILE * HYQ_D * (int)sizeof(double);     // 64 KB
-    static bool attr_set = false;                                       // same values every time: a benign race
-    if (!attr_set) {
+    // (per device and process; same values every time, so a race between host threads is benign)
+    static bool attr_set[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return HYQ_ERR_CUDA;
+    if (!attr_set[dev]) {
         if (cudaFuncSetAttribute(mass_chunk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
             cudaFuncSetAttribute(mass_column_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
             return HYQ_ERR_CUDA;
-        attr_set = true;
+        attr_set[dev] = true;
     }
     mass_chunk_kernel<<<dim3((n_chunks + MASS_CHUNKS - 1) / MASS_CHUNKS, Hkv, B), MASS_THREADS, smem, st>>>(qb, kb, Hq, Hkv, Lq, Lk, nT, n_chunks, alpha, chunk_m, chunk_z);
     if (launch_status() != HYQ_OK) return HYQ_ERR_CUDA;
