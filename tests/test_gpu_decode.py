@@ -235,6 +235,26 @@ def test_a_dominant_full_precision_key_keeps_its_precision():
         assert rel <= 4e-4, (fmt, mx, rel)
 
 
+def test_decode_calls_can_be_captured_in_a_cuda_graph():
+    """The call enqueues two kernels (the second as a programmatic dependent) and nothing else: it can be recorded in a
+    CUDA graph and replayed, with the result of the eager call."""
+    B, Hq, Hkv, N, W, kk = 2, 8, 2, 3000, 128, 40
+    K, V = rand_bf16((B, Hkv, N, 128), 111), rand_bf16((B, Hkv, N, 128), 112)
+    q = rand_bf16((B, Hq, 128), 113).cuda()
+    _, cache = _freeze_both(K, V, _idx(B, Hkv, N - W, kk, 114), W, Hq)
+    out = torch.empty(B, Hq, 128, dtype=torch.float32, device="cuda")
+    ws = torch.empty(dapi.hyq_hybrid_attention_decode_workspace(cache) + 16, dtype=torch.uint8, device="cuda")
+    eager = dapi.hyq_hybrid_attention_decode(q, cache, out_dtype=torch.float32).clone()      # also the first, uncaptured call
+    graph, stream = torch.cuda.CUDAGraph(), torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        with torch.cuda.graph(graph, stream=stream):
+            dapi.hyq_hybrid_attention_decode(q, cache, out=out, workspace=ws)
+    out.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(out, eager)
+
+
 def test_decode_at_benchmark_size_and_repeatable():
     """The benchmark's cache shape (32 / 8 heads, 32768 frozen rows, 2 % vertical, window 1024, a full staging
     buffer) at batch 2, every head against the oracle; two runs are bit-identical."""
