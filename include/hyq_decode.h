@@ -101,7 +101,7 @@ int hyq_kv_cache_query_sizes(const hyq_kv_cache* cache, hyq_kv_cache_sizes* size
  * vertical and quantized buffers of `cache` (layouts above).  The staging buffers are not touched
  * (an empty staging buffer is n_staging = 0).  The prefill cache may be freed once the enqueued
  * work has completed.  Errors: INVALID_ARG (null pointer, sizes out of range, struct_size),
- * UNSUPPORTED (D != 128, group not 32 / 64 / 128, format not INT4 / INT8, g > 64), ALIGNMENT (any buffer not 16-byte aligned).
+ * UNSUPPORTED (D != 128, group not 32 / 64 / 128, format not INT4 / INT8, g > 64), ALIGNMENT (a code or bf16 buffer not 16-byte aligned, a scale array not 4-byte aligned).
  * ------------------------------------------------------------------------------------------- */
 int hyq_freeze(const void* k_, const void* v, const int32_t* vl_idx, const hyq_kv_cache* cache, void* stream);
 

@@ -26,9 +26,11 @@ static int check_cache(const hyq_kv_cache* c, bool need_pointers) {
     if (c->k > 0 && (!c->k_vl || !c->v_vl)) return HYQ_ERR_INVALID_ARG;
     if (g.W > 0 && (!c->k_win || !c->v_win)) return HYQ_ERR_INVALID_ARG;
     if (c->n_staging > 0 && (!c->k_s || !c->v_s)) return HYQ_ERR_INVALID_ARG;
-    const void* al[] = {c->kq_codes, c->vq_codes, c->kq_scales, c->vq_scales, c->k_vl, c->v_vl, c->k_win, c->v_win, c->k_s, c->v_s};
+    const void* al[] = {c->kq_codes, c->vq_codes, c->k_vl, c->v_vl, c->k_win, c->v_win, c->k_s, c->v_s};
     for (const void* p : al)
         if (!aligned16(p)) return HYQ_ERR_ALIGNMENT;
+    // the scales are read one float at a time (a sequence's slice of a batch allocation need not be 16-byte aligned)
+    if ((reinterpret_cast<uintptr_t>(c->kq_scales) | reinterpret_cast<uintptr_t>(c->vq_scales)) & 3u) return HYQ_ERR_ALIGNMENT;
     return HYQ_OK;
 }
 

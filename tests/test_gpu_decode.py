@@ -216,6 +216,26 @@ def test_decode_with_peaked_scores_and_late_maxima():
         assert mx <= MAX_ABS_TOL and rel <= MEAN_REL_TOL, (splits, mx, rel)
 
 
+def test_ragged_batch_whose_scale_slices_are_not_16_byte_aligned():
+    """Short sequences: a sequence's slice of the batch's scale arrays starts at a multiple of 8 bytes only."""
+    Hq, Hkv, W = 2, 1, 8
+    seqs = [(100, 3), (70, 0), (90, 5)]
+    rc = dapi.RaggedKvCache(len(seqs), Hq, Hkv, max_N=100, window=W, max_k=5)
+    assert rc.batch.buffers["kq_scales"][1].data_ptr() % 16 == 8
+    q = rand_bf16((len(seqs), Hq, 128), 120)
+    refs = []
+    for b, (N, kk) in enumerate(seqs):
+        K, V = rand_bf16((1, Hkv, N, 128), 121 + b), rand_bf16((1, Hkv, N, 128), 131 + b)
+        idx = _idx(1, Hkv, N - W, kk, 141 + b) if kk else None
+        refs.append(od.freeze(wl.bits(K), wl.bits(V), idx, W))
+        rc.freeze_sequence(b, K.cuda(), V.cuda(), None if idx is None else torch.from_numpy(idx).cuda())
+    got = dapi.hyq_hybrid_attention_decode_ragged(q.cuda(), rc, out_dtype=torch.float32)
+    for b, ref in enumerate(refs):
+        want, _ = od.decode_attention(wl.bits(q[b:b + 1]), ref)
+        mx, rel = errors(got[b:b + 1].cpu().numpy(), want)
+        assert mx <= MAX_ABS_TOL and rel <= MEAN_REL_TOL, (b, mx, rel)
+
+
 def test_a_dominant_full_precision_key_keeps_its_precision():
     """One window key takes almost all of the weight: the output is that key's value row, so any rounding of the
     weights in the full-precision product shows directly.  (A single bf16 weight would leave 1e-3 here.)"""
