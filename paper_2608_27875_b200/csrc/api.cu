@@ -30,7 +30,7 @@ const char* hyq_status_string(int status) {
     }
 }
 
-int hyq_version(void) { return 1; }
+int hyq_version(void) { return 2; }   // 2: decode side, column-mass selector, block sizes
 
 int hyq_paper_k(int Lk, int window, double ratio) {
     const long P = (Lk - window > 0) ? (long)Lk - window : 0;
