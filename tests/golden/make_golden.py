@@ -1,4 +1,4 @@
-"""Writes tests/golden/oracle_small_case.json from the CPU oracle alone.
+"""Writes tests/golden/oracle_small_case.json and tests/golden/oracle_decode_case.json from the CPU oracle alone.
 
 The paper prints no worked numeric example for the prefill path, so this
 fixture is a regression anchor, not an external pin: it freezes what the pinned
@@ -39,8 +39,36 @@ def compute():
     }
 
 
+def compute_decode():
+    """The decode side on the same tensors: Eq. 4-5 selection from 8 tail queries (first query head of every KV group),
+    Freeze (Algorithm 4, K4V4, groups of 64), two staged rows, one token (Algorithm 3)."""
+    from oracle import decode as od
+    w = wl.CONFIGS["c0"].scaled(**CASE)
+    Q, K, V = wl.make_inputs(w)
+    g = CASE["Hq"] // CASE["Hkv"]
+    idx_mass, scores = oracle.select_vertical_mass(wl.bits(Q), wl.bits(K), w.window, w.k, 8, return_scores=True)
+    idx_kv = np.ascontiguousarray(idx_mass[:, ::g])
+    cache = od.freeze(wl.bits(K), wl.bits(V), idx_kv, w.window)
+    for i in (3, 17):
+        od.append_staging(cache, wl.bits(K)[:, :, i], wl.bits(V)[:, :, i + 1])
+    out, lse = od.decode_attention(wl.bits(Q[:, :, -1].contiguous()), cache)
+    seg, _ = od.decode_attention_segmented(wl.bits(Q[:, :, -1].contiguous()), cache, splits=3, tile=16)
+    assert np.allclose(seg, out, rtol=1e-11, atol=1e-13)
+    return {
+        "case": CASE, "n_queries": 8, "formats": "K4V4, groups of 64 compacted rows, staging rows 3 and 17/18",
+        "mass_idx": idx_mass.tolist(),
+        "mass_scores_head2_first6": [float.hex(float(x)) for x in scores[0, 2, :6]],
+        "quantized_positions_head1_first12": cache["iq"][0, 1, :12].tolist(),
+        "kq_scales_bits": cache["kq_scales"].view(np.uint32).tolist(),
+        "vq_codes_row9_head0": cache["vq_codes"][0, 0, 9].tolist(),
+        "lse": [float.hex(float(x)) for x in lse[0]],
+        "out_first8": [[float.hex(float(x)) for x in out[0, h, :8]] for h in range(CASE["Hq"])],
+    }
+
+
 if __name__ == "__main__":
-    path = os.path.join(os.path.dirname(os.path.abspath(__file__)), "oracle_small_case.json")
-    with open(path, "w") as f:
-        json.dump(compute(), f, indent=1)
-    print("wrote", path)
+    here = os.path.dirname(os.path.abspath(__file__))
+    for name, fn in (("oracle_small_case.json", compute), ("oracle_decode_case.json", compute_decode)):
+        with open(os.path.join(here, name), "w") as f:
+            json.dump(fn(), f, indent=1)
+        print("wrote", os.path.join(here, name))
