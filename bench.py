@@ -382,7 +382,7 @@ def run_decode(args, w: wl.Workload):
     torch.cuda.set_device(dev)
     w = w.scaled(B=args.batch)
     g = w.Hq // w.Hkv
-    kv_fmt = wl.FMT_INT8 if args.kv_format == "int8" else wl.FMT_INT4
+    kv_fmt = {"int4": wl.FMT_INT4, "int8": wl.FMT_INT8, "fp8": wl.FMT_FP8_E4M3}[args.kv_format]
     Q, K, V = wl.make_inputs(w)
     K, V = K.to(dev), V.to(dev)
     q_tail = Q[:, ::g].contiguous().to(dev)                 # Algorithm 1 with H = H_KV heads
@@ -456,7 +456,7 @@ def run_decode(args, w: wl.Workload):
         "dtype": f"{args.kv_format} codes -> fp16 in registers, fp16 / bf16 mma.sync with f32 accumulation", "data": "synthetic",
         "config": {"workload": f"{w.name} cache shape, decode of one token per sequence", "B": w.B, "Hq": w.Hq,
                    "Hkv": w.Hkv, "N": w.L, "D": w.D, "window": w.window, "k": w.k, "staging_rows": args.staging,
-                   "format": ("K8V8" if kv_fmt == wl.FMT_INT8 else "K4V4") + ", group 64", "splits": args.splits, "cached_rows_per_head": rows,
+                   "format": {"int4": "K4V4", "int8": "K8V8 (INT8)", "fp8": "K8V8 (FP8 e4m3)"}[args.kv_format] + ", group 64", "splits": args.splits, "cached_rows_per_head": rows,
                    "l2": f"{n_rep} cache replicas used round-robin ({by * (n_rep - 1) / 1e6:.0f} MB read between reuses)",
                    "freeze_ms": freeze_ms},
         "roofline": {"bound": "hbm", "kernel": "decode_kernel + decode_merge_kernel (one call)",
@@ -486,7 +486,7 @@ def main():
     ap.add_argument("--batch", type=int, default=8, help="with --decode: sequences in the batch")
     ap.add_argument("--staging", type=int, default=128, help="with --decode: staged rows (W_s, all filled)")
     ap.add_argument("--splits", type=int, default=0, help="with --decode: slices per KV head (0 = library's choice)")
-    ap.add_argument("--kv-format", default="int4", choices=["int4", "int8"], help="with --decode: cache code format (K4V4 / K8V8)")
+    ap.add_argument("--kv-format", default="int4", choices=["int4", "int8", "fp8"], help="with --decode: cache code format (K4V4 / K8V8 / FP8 e4m3)")
     ap.add_argument("--formats", default="", choices=["", *sorted(FORMAT_SETS)],
                     help="override the workload's (Q, K, V) low-bit formats (default: as the workload defines them)")
     args = ap.parse_args()

@@ -20,7 +20,7 @@
  *                              is not described by the paper and not part of this library.
  *   quantized    the other nQ = N - W' - k prefix rows, COMPACTED in ascending position order and cut
  *                into groups of `group` (G = 32, 64 or 128) consecutive compacted rows x all D channels; each group is
- *                quantized exactly as hyq_quantize_blocks quantizes a tile (INT4, c_B = 7, or INT8, c_B = 127;
+ *                quantized exactly as hyq_quantize_blocks quantizes a tile (INT4, c_B = 7; INT8, c_B = 127; FP8 e4m3, c_B = 448;
  *                fp32 scale per group; the last group may be ragged).  Per head the row count is padded to
  *                nQp = G * ceil(nQ / G); padding rows hold unspecified codes and are never used.
  *       kq_codes  [B,Hkv,nQp,D/2] bytes: row-major, channel 2m in the low nibble and 2m+1 in the high
@@ -34,7 +34,7 @@
  *                 i.e. each lane of a warp reads two 16-byte pieces (the warp: two contiguous 512-byte
  *                 runs) and owns, without any shuffle, the operand registers of the warp-level matrix
  *                 instruction that accumulates P.V.
- *       INT8 caches: kq_codes [B,Hkv,nQp,D] bytes row-major (two's complement); vq_codes [B,Hkv,nQp/16,2048]
+ *       INT8 and FP8 caches: kq_codes [B,Hkv,nQp,D] bytes row-major (two's complement / e4m3); vq_codes [B,Hkv,nQp/16,2048]
  *                 bytes, fragment-major again: the tile is four 512-byte runs, lane l = 4r + j owns bytes
  *                 [16l, 16l + 16) of each, i.e. 16 words; word w = 2x + (row >> 3) sits at byte
  *                 512*(w >> 2) + 16*l + 4*(w & 3), and its four bytes hold, in order, the codes of
@@ -64,7 +64,7 @@ typedef struct {
   int32_t window;               /* W; the window buffers hold min(W, N) rows */
   int32_t k;                    /* vertical rows per KV head, 0 <= k <= N - min(W, N) */
   int32_t group;                /* G: 32, 64 or 128 rows per scale group */
-  int32_t format;               /* K and V code format: HYQ_FMT_INT4 (K4V4) or HYQ_FMT_INT8 (K8V8) */
+  int32_t format;               /* K and V code format: HYQ_FMT_INT4 (K4V4), HYQ_FMT_INT8 or HYQ_FMT_FP8_E4M3 (K8V8) */
   int32_t staging_capacity;     /* W_s: rows allocated per head in k_s / v_s (may be 0) */
   int32_t n_staging;            /* valid staging rows, 0 <= n_staging <= staging_capacity */
   void* kq_codes;
@@ -101,7 +101,7 @@ int hyq_kv_cache_query_sizes(const hyq_kv_cache* cache, hyq_kv_cache_sizes* size
  * vertical and quantized buffers of `cache` (layouts above).  The staging buffers are not touched
  * (an empty staging buffer is n_staging = 0).  The prefill cache may be freed once the enqueued
  * work has completed.  Errors: INVALID_ARG (null pointer, sizes out of range, struct_size),
- * UNSUPPORTED (D != 128, group not 32 / 64 / 128, format not INT4 / INT8, g > 64), ALIGNMENT (a code or bf16 buffer not 16-byte aligned, a scale array not 4-byte aligned).
+ * UNSUPPORTED (D != 128, group not 32 / 64 / 128, format not INT4 / INT8 / FP8_E4M3, g > 64), ALIGNMENT (a code or bf16 buffer not 16-byte aligned, a scale array not 4-byte aligned).
  * ------------------------------------------------------------------------------------------- */
 int hyq_freeze(const void* k_, const void* v, const int32_t* vl_idx, const hyq_kv_cache* cache, void* stream);
 

@@ -11,7 +11,7 @@ static int check_cache(const hyq_kv_cache* c, bool need_pointers) {
     if (c->Hq % c->Hkv) return HYQ_ERR_INVALID_ARG;
     if (c->staging_capacity < 0 || c->n_staging < 0 || c->n_staging > c->staging_capacity) return HYQ_ERR_INVALID_ARG;
     if (c->D != HYQ_D || (c->group != 32 && c->group != 64 && c->group != 128) ||
-        (c->format != HYQ_FMT_INT4 && c->format != HYQ_FMT_INT8) ||
+        (c->format != HYQ_FMT_INT4 && c->format != HYQ_FMT_INT8 && c->format != HYQ_FMT_FP8_E4M3) ||
         c->Hq / c->Hkv > 8 * DEC_MAX_GROUP)
         return HYQ_ERR_UNSUPPORTED;
     const CacheGeo g = cache_geo(*c);
@@ -44,7 +44,7 @@ int hyq_kv_cache_query_sizes(const hyq_kv_cache* cache, hyq_kv_cache_sizes* size
     const size_t heads = (size_t)cache->B * cache->Hkv;
     sizes->quantized_rows = g.nQ;
     sizes->padded_rows = g.nQp;
-    const size_t row_bytes = cache->format == HYQ_FMT_INT8 ? HYQ_D : HYQ_D / 2;
+    const size_t row_bytes = cache->format == HYQ_FMT_INT4 ? HYQ_D / 2 : HYQ_D;
     sizes->kq_codes_bytes = heads * g.sQ * row_bytes;
     sizes->vq_codes_bytes = heads * g.sQ * row_bytes;
     sizes->scales_bytes = heads * (g.sQ / cache->group) * sizeof(float);

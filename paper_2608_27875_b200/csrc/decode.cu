@@ -275,15 +275,32 @@ struct QTile8 {
     float fk, fv;
 };
 
-template <bool RAGGED>
+// FP8 e4m3 bytes: (byte & 0x7F) << 7 under the sign bit is the fp16 number with the same exponent and mantissa fields,
+// i.e. the code's value times 2^-8 (exponent bias 15 against 7), subnormals included.  K leaves the 2^-8 to the score
+// scale, V multiplies it back (exact: |code| <= 448).
+__device__ __forceinline__ uint32_t e4m3_pair(uint32_t w, uint32_t sel) {     // sel: 0x1404 bytes 0,1; 0x3424 bytes 2,3
+    const uint32_t x = __byte_perm(w, 0u, sel);                               // each byte in the high byte of its half
+    const uint32_t mag = (x >> 1) & 0x3F803F80u;
+    uint32_t h;
+    asm("lop3.b32 %0, %1, 0x80008000, %2, 0xEA;" : "=r"(h) : "r"(x), "r"(mag));      // (x & sign bits) | mag
+    return h;
+}
+
+template <bool RAGGED, bool FP8 = false>
 __device__ __forceinline__ void quant_tile8(const QTile8& d, const uint32_t (&qf)[16], float scale_log2, float bias0, float bias1,
                                             int rows_valid, int r, SoftmaxState& st, float (&acc)[8][4]) {
     float c4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
 #pragma unroll
     for (int c = 0; c < 8; ++c) {
-        const uint32_t wa = word_of(d.k[c >> 2], c & 3) ^ 0x80808080u, wb = word_of(d.k[2 + (c >> 2)], c & 3) ^ 0x80808080u;
-        mma_f16(c4, __byte_perm(wa, 0u, 0x4140), __byte_perm(wb, 0u, 0x4140), __byte_perm(wa, 0u, 0x4342),
-                __byte_perm(wb, 0u, 0x4342), qf[2 * c], qf[2 * c + 1]);
+        if (FP8) {
+            const uint32_t wa = word_of(d.k[c >> 2], c & 3), wb = word_of(d.k[2 + (c >> 2)], c & 3);
+            mma_f16(c4, e4m3_pair(wa, 0x1404), e4m3_pair(wb, 0x1404), e4m3_pair(wa, 0x3424), e4m3_pair(wb, 0x3424),
+                    qf[2 * c], qf[2 * c + 1]);
+        } else {
+            const uint32_t wa = word_of(d.k[c >> 2], c & 3) ^ 0x80808080u, wb = word_of(d.k[2 + (c >> 2)], c & 3) ^ 0x80808080u;
+            mma_f16(c4, __byte_perm(wa, 0u, 0x4140), __byte_perm(wb, 0u, 0x4140), __byte_perm(wa, 0u, 0x4342),
+                    __byte_perm(wb, 0u, 0x4342), qf[2 * c], qf[2 * c + 1]);
+        }
     }
     float pw[4];
     softmax_tile<RAGGED>(st, acc, c4, d.fk * scale_log2, bias0, bias1, r < rows_valid, r + 8 < rows_valid, pw);
@@ -294,16 +311,28 @@ __device__ __forceinline__ void quant_tile8(const QTile8& d, const uint32_t (&qf
         asm("sub.rn.f16x2 %0, %1, %2;" : "=r"(h) : "r"(h), "r"(0x64806480u));
         return h;
     };
+    auto value8 = [](uint32_t w, uint32_t sel) {          // two e4m3 bytes of w -> packed fp16 values
+        uint32_t h = e4m3_pair(w, sel);
+        asm("mul.rn.f16x2 %0, %1, %2;" : "=r"(h) : "r"(h), "r"(0x5C005C00u));         // times 256
+        return h;
+    };
 #pragma unroll
     for (int x = 0; x < 8; ++x) {
+        if (FP8) {
+            const uint32_t w0 = word_of(d.v[x >> 1], 2 * (x & 1)), w1 = word_of(d.v[x >> 1], 2 * (x & 1) + 1);
+            mma_f16(acc[x], value8(w0, 0x1404), value8(w0, 0x3424), value8(w1, 0x1404), value8(w1, 0x3424), b0, b1);
+            continue;
+        }
         const uint32_t w0 = word_of(d.v[x >> 1], 2 * (x & 1)) ^ 0x80808080u, w1 = word_of(d.v[x >> 1], 2 * (x & 1) + 1) ^ 0x80808080u;
         mma_f16(acc[x], exact(w0, 0x4140), exact(w0, 0x4342), exact(w1, 0x4140), exact(w1, 0x4342), b0, b1);
     }
 }
 
-template <bool FMT8>
+template <int KVF>      // cache code format: HYQ_FMT_INT4, HYQ_FMT_INT8 or HYQ_FMT_FP8_E4M3
 __global__ void __launch_bounds__(DEC_THREADS, DEC_CTAS_PER_SM)
 decode_kernel(const DecParams p) {
+    constexpr bool FMT8 = KVF != HYQ_FMT_INT4;             // byte-wide codes
+    constexpr bool FP8 = KVF == HYQ_FMT_FP8_E4M3;
     const int split = blockIdx.x;
     // blockIdx.y = (b * Hkv + kv head) * hgroups + head group: up to 8 of the KV head's g query heads per CTA
     const long unit = blockIdx.y / p.hgroups;
@@ -467,8 +496,9 @@ decode_kernel(const DecParams p) {
             if (s < n_my) issue(ring + s * ST8_BYTES);
             cp_async_commit();
         }
-        const float kscale = p.scale_log2 * 16777216.0f;
-        const float b0 = q_sum[2 * j] * (128.0f / 16777216.0f), b1 = q_sum[2 * j + 1] * (128.0f / 16777216.0f);
+        // INT8: subnormal operand (2^-24) and the +128 offset; FP8: the 2^-8 of the exponent-bias trick, no offset
+        const float kscale = p.scale_log2 * (FP8 ? 256.0f : 16777216.0f);
+        const float b0 = FP8 ? 0.0f : q_sum[2 * j] * (128.0f / 16777216.0f), b1 = FP8 ? 0.0f : q_sum[2 * j + 1] * (128.0f / 16777216.0f);
         for (int i = 0; i < n_my; ++i) {
             cp_async_wait<ST8 - 1>();                       // tile i has landed
             const uint32_t sa = ring + (i & 1) * ST8_BYTES;
@@ -479,8 +509,8 @@ decode_kernel(const DecParams p) {
             A.fk = __ldg(pks + grp); A.fv = __ldg(pvs + grp);
             if (i + ST8 < n_my) issue(sa);                  // own bytes only: no barrier
             cp_async_commit();
-            if (has_ragged && i == n_my - 1) quant_tile8<true>(A, qf, kscale, b0, b1, (int)(nQ & 15), r, st, acc);
-            else quant_tile8<false>(A, qf, kscale, b0, b1, 16, r, st, acc);
+            if (has_ragged && i == n_my - 1) quant_tile8<true, FP8>(A, qf, kscale, b0, b1, (int)(nQ & 15), r, st, acc);
+            else quant_tile8<false, FP8>(A, qf, kscale, b0, b1, 16, r, st, acc);
         }
     }
     cp_async_wait<0>();
@@ -685,13 +715,16 @@ int launch_decode(const void* q, const hyq_kv_cache& c, const int32_t* lengths, 
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return HYQ_ERR_CUDA;
     if (!attr_set[dev]) {
-        if (cudaFuncSetAttribute(decode_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, ring_bytes) != cudaSuccess ||
-            cudaFuncSetAttribute(decode_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ring_bytes) != cudaSuccess)
+        if (cudaFuncSetAttribute(decode_kernel<HYQ_FMT_INT4>, cudaFuncAttributeMaxDynamicSharedMemorySize, ring_bytes) != cudaSuccess ||
+            cudaFuncSetAttribute(decode_kernel<HYQ_FMT_INT8>, cudaFuncAttributeMaxDynamicSharedMemorySize, ring_bytes) != cudaSuccess ||
+            cudaFuncSetAttribute(decode_kernel<HYQ_FMT_FP8_E4M3>, cudaFuncAttributeMaxDynamicSharedMemorySize, ring_bytes) != cudaSuccess)
             return HYQ_ERR_CUDA;
         attr_set[dev] = true;
     }
-    if (c.format == HYQ_FMT_INT8) decode_kernel<true><<<dim3((unsigned)splits, (unsigned)units), DEC_THREADS, ring_bytes, st>>>(p);
-    else decode_kernel<false><<<dim3((unsigned)splits, (unsigned)units), DEC_THREADS, ring_bytes, st>>>(p);
+    const dim3 grid((unsigned)splits, (unsigned)units);
+    if (c.format == HYQ_FMT_INT8) decode_kernel<HYQ_FMT_INT8><<<grid, DEC_THREADS, ring_bytes, st>>>(p);
+    else if (c.format == HYQ_FMT_FP8_E4M3) decode_kernel<HYQ_FMT_FP8_E4M3><<<grid, DEC_THREADS, ring_bytes, st>>>(p);
+    else decode_kernel<HYQ_FMT_INT4><<<grid, DEC_THREADS, ring_bytes, st>>>(p);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)units, (unsigned)(p.g < DEC_MAX_GROUP ? p.g : DEC_MAX_GROUP));
     cfg.blockDim = dim3(HYQ_D);

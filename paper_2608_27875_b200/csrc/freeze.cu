@@ -8,6 +8,8 @@
 //                          arithmetic of the per-tile quantizer (fp32, one rounding per operation), and
 //                          writes K row-major and V in the fragment-major tile layout the decode kernel
 //                          loads straight into matrix-instruction operand registers.
+#include <cuda_fp8.h>
+
 #include "common.cuh"
 #include "decode_common.cuh"
 
@@ -44,7 +46,7 @@ gather_rows_kernel(const uint4* __restrict__ k_, const uint4* __restrict__ v, co
     (vl ? v_vl_out : v_win)[d] = __ldg(v + s);
 }
 
-template <int G, bool FMT8>
+template <int G, int FMT>
 __global__ void __launch_bounds__(2 * G)
 freeze_quantize_kernel(const uint4* __restrict__ k_, const uint4* __restrict__ v, const int32_t* __restrict__ idx,
                        int N, int k_vl, int nQ, long nQp, uint8_t* __restrict__ kq, uint8_t* __restrict__ vq,
@@ -59,9 +61,10 @@ freeze_quantize_kernel(const uint4* __restrict__ k_, const uint4* __restrict__ v
     __shared__ int src[G];
     __shared__ int win[FRZ_WIN], j0_sh;
     __shared__ float warp_max[NT / 32];
+    constexpr bool FMT8 = FMT != HYQ_FMT_INT4;                 // byte-wide codes (INT8 or FP8 e4m3)
     constexpr int ROW_BYTES = FMT8 ? HYQ_D : HYQ_D / 2;        // code bytes per row
     constexpr int TILE_BYTES = 16 * ROW_BYTES;                 // one 16-row V tile
-    constexpr float CB = FMT8 ? 127.0f : 7.0f;
+    constexpr float CB = FMT == HYQ_FMT_INT8 ? 127.0f : FMT == HYQ_FMT_FP8_E4M3 ? 448.0f : 7.0f;
     __shared__ __align__(16) uint8_t vtile[(G / 16) * TILE_BYTES];
     // Source rows of the group's G compacted rows in three dependent memory round trips instead of ten:
     // warp 0 finds j0 = the number of vertical rows before the group's first row by a 32-way search, a window of
@@ -141,8 +144,15 @@ freeze_quantize_kernel(const uint4* __restrict__ k_, const uint4* __restrict__ v
             uint8_t b[16];
 #pragma unroll
             for (int m = 0; m < 8; ++m) {
-                b[2 * m] = (uint8_t)max(-127, min(127, __float2int_rn(__fmul_rn(bf16_lo(w[m]), inv))));
-                b[2 * m + 1] = (uint8_t)max(-127, min(127, __float2int_rn(__fmul_rn(bf16_hi(w[m]), inv))));
+                const float y0 = __fmul_rn(bf16_lo(w[m]), inv), y1 = __fmul_rn(bf16_hi(w[m]), inv);
+                if (FMT == HYQ_FMT_FP8_E4M3) {
+                    const uint32_t two = dead ? 0u : __nv_cvt_float2_to_fp8x2(make_float2(y0, y1), __NV_SATFINITE, __NV_E4M3);   // no -0 in a zero group
+                    b[2 * m] = (uint8_t)(two & 0xFF);
+                    b[2 * m + 1] = (uint8_t)(two >> 8);
+                } else {
+                    b[2 * m] = (uint8_t)max(-127, min(127, __float2int_rn(y0)));
+                    b[2 * m + 1] = (uint8_t)max(-127, min(127, __float2int_rn(y1)));
+                }
             }
             if (!is_v) {
                 uint32_t o[4];
@@ -199,10 +209,11 @@ int launch_freeze(const void* k_, const void* v, const int32_t* vl_idx, const hy
         auto* kq = static_cast<uint8_t*>(c.kq_codes);
         auto* vq = static_cast<uint8_t*>(c.vq_codes);
 #define HYQ_FRZ(G_, F8_) freeze_quantize_kernel<G_, F8_><<<grid, 2 * G_, 0, st>>>(k4, v4, vl_idx, c.N, c.k, (int)g.nQ, g.sQ, kq, vq, c.kq_scales, c.vq_scales)
-        const bool f8 = c.format == HYQ_FMT_INT8;
-        if (c.group == 32) { if (f8) HYQ_FRZ(32, true); else HYQ_FRZ(32, false); }
-        else if (c.group == 64) { if (f8) HYQ_FRZ(64, true); else HYQ_FRZ(64, false); }
-        else { if (f8) HYQ_FRZ(128, true); else HYQ_FRZ(128, false); }
+#define HYQ_FRZ_F(G_) do { if (c.format == HYQ_FMT_INT8) HYQ_FRZ(G_, HYQ_FMT_INT8); else if (c.format == HYQ_FMT_FP8_E4M3) HYQ_FRZ(G_, HYQ_FMT_FP8_E4M3); else HYQ_FRZ(G_, HYQ_FMT_INT4); } while (0)
+        if (c.group == 32) HYQ_FRZ_F(32);
+        else if (c.group == 64) HYQ_FRZ_F(64);
+        else HYQ_FRZ_F(128);
+#undef HYQ_FRZ_F
 #undef HYQ_FRZ
     }
     return launch_status();

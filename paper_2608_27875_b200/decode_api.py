@@ -95,7 +95,7 @@ class HybridKvCache:
         heads = d.B * d.Hkv
         nq = int(s.quantized_rows)
         w = min(d.window, d.N)
-        code_bytes = 2 * d.D if d.format == FMT_INT8 else d.D    # K + V codes of one row
+        code_bytes = d.D if d.format == FMT_INT4 else 2 * d.D    # K + V codes of one row
         return heads * (nq * code_bytes + 2 * (-(-nq // d.group)) * 4 + (d.k + w + d.n_staging) * d.D * 4)
 
 
@@ -107,7 +107,7 @@ def alloc_cache(desc: KvCacheDesc, device="cuda") -> HybridKvCache:
     kcap = desc.cap_vertical or desc.k
     u8 = lambda *shape: torch.empty(*shape, dtype=torch.uint8, device=device)          # noqa: E731
     bf = lambda *shape: torch.empty(*shape, dtype=torch.bfloat16, device=device)       # noqa: E731
-    rb = D if desc.format == FMT_INT8 else D // 2               # code bytes per row
+    rb = D // 2 if desc.format == FMT_INT4 else D               # code bytes per row
     buf = dict(kq_codes=u8(B, H, max(nqp, 1), rb), vq_codes=u8(B, H, max(nqp // 16, 1), 16 * rb),
                kq_scales=torch.empty(B, H, max(nqp // desc.group, 1), dtype=torch.float32, device=device),
                vq_scales=torch.empty(B, H, max(nqp // desc.group, 1), dtype=torch.float32, device=device),

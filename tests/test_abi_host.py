@@ -135,7 +135,7 @@ def test_decode_side_argument_checks(lib):
     w_all = decode_api.make_desc(B=1, Hq=4, Hkv=4, N=50, window=80, k=0)          # window longer than the cache
     assert L.hyq_kv_cache_query_sizes(ctypes.byref(w_all), ctypes.byref(sizes)) == 0
     assert sizes.quantized_rows == 0 and sizes.window_bytes == 4 * 50 * 256
-    bad = [dict(k=901), dict(Hq=30), dict(D=64), dict(group=48), dict(fmt=api.FMT_FP8_E4M3), dict(Hq=1024),
+    bad = [dict(k=901), dict(Hq=30), dict(D=64), dict(group=48), dict(fmt=7), dict(Hq=1024),
            dict(n_staging=129), dict(N=0)]
     expect = [1, 1, 2, 2, 2, 2, 1, 1]
     for kw, code in zip(bad, expect):

@@ -78,7 +78,7 @@ def _assert_cache_equal(ref, cache):
     if nQ:
         ng = -(-nQ // ref["group"])
         assert np.array_equal(b["kq_codes"][:, :, :nQ], ref["kq_codes"])
-        unpermute = _v8_tiles_to_rows if ref["fmts"][1] == oracle.FMT_INT8 else _v_tiles_to_rows
+        unpermute = _v_tiles_to_rows if ref["fmts"][1] == oracle.FMT_INT4 else _v8_tiles_to_rows
         assert np.array_equal(unpermute(b["vq_codes"])[:, :, :nQ], ref["vq_codes"])
         assert np.array_equal(b["kq_scales"][:, :, :ng].view(np.uint32), ref["kq_scales"].view(np.uint32))
         assert np.array_equal(b["vq_scales"][:, :, :ng].view(np.uint32), ref["vq_scales"].view(np.uint32))
@@ -158,16 +158,17 @@ def test_other_group_sizes(group, B, Hq, Hkv, N, W, kk, n_s):
         assert mx <= MAX_ABS_TOL and rel <= MEAN_REL_TOL, (splits, mx, rel)
 
 
+@pytest.mark.parametrize("fmt", [oracle.FMT_INT8, oracle.FMT_FP8_E4M3])
 @pytest.mark.parametrize("group", [32, 64, 128])
 @pytest.mark.parametrize("B,Hq,Hkv,N,W,kk,n_s,splits", [(1, 4, 1, 300, 40, 9, 3, 0), (2, 8, 2, 1000, 128, 37, 0, 3), (1, 16, 2, 2117, 100, 50, 17, 0),
                                                         (1, 2, 2, 64, 0, 0, 1, 1), (1, 5, 1, 777, 33, 21, 2, 7), (1, 4, 2, 200, 20, 180, 5, 2)])
-def test_int8_cache(group, B, Hq, Hkv, N, W, kk, n_s, splits):
-    """K8V8: codes, scales and layouts bit-exact; attention within tolerance (and closer to exact attention than K4V4)."""
+def test_byte_wide_caches(fmt, group, B, Hq, Hkv, N, W, kk, n_s, splits):
+    """K8V8 with INT8 or FP8 e4m3 codes: codes, scales and layouts bit-exact; attention within tolerance."""
     K, V = rand_bf16((B, Hkv, N, 128), 81, 1.3), rand_bf16((B, Hkv, N, 128), 82)
     K[:, :, : N // 2] *= 0.05
     q = rand_bf16((B, Hq, 128), 83, 1.5)
     idx = _idx(B, Hkv, N - min(W, N), kk, 84) if kk else None
-    ref, cache = _freeze_both(K, V, idx, W, Hq, group=group, fmt=oracle.FMT_INT8)
+    ref, cache = _freeze_both(K, V, idx, W, Hq, group=group, fmt=fmt)
     _assert_cache_equal(ref, cache)
     _stage(ref, cache, n_s, 600)
     want, lse_want = od.decode_attention(wl.bits(q), ref)
@@ -178,7 +179,7 @@ def test_int8_cache(group, B, Hq, Hkv, N, W, kk, n_s, splits):
     assert np.abs(lse.cpu().numpy() - lse_want).max() <= 2e-3
 
 
-@pytest.mark.parametrize("fmt", [oracle.FMT_INT4, oracle.FMT_INT8])
+@pytest.mark.parametrize("fmt", [oracle.FMT_INT4, oracle.FMT_INT8, oracle.FMT_FP8_E4M3])
 @pytest.mark.parametrize("B,Hq,Hkv,N,W,kk,n_s,splits", [(1, 32, 2, 1500, 64, 30, 5, 0), (2, 12, 1, 700, 32, 11, 0, 3), (1, 18, 2, 333, 40, 9, 2, 1),
                                                         (1, 64, 1, 400, 16, 5, 1, 2)])
 def test_more_than_eight_query_heads_per_kv_head(fmt, B, Hq, Hkv, N, W, kk, n_s, splits):
@@ -247,7 +248,7 @@ def test_a_dominant_full_precision_key_keeps_its_precision():
     for pos, amp in ((N - 7, 6.0), (N - 30, 5.5)):                      # two window keys of comparable, dominant weight
         K[:, :, pos] = (K[:, :, pos].float() + amp * u).to(torch.bfloat16)
     idx = _idx(B, Hkv, N - W, 20, 105)
-    for fmt in (oracle.FMT_INT4, oracle.FMT_INT8):
+    for fmt in (oracle.FMT_INT4, oracle.FMT_INT8, oracle.FMT_FP8_E4M3):
         ref, cache = _freeze_both(K, V, idx, W, Hq, fmt=fmt)
         want, _ = od.decode_attention(wl.bits(q), ref)
         got = dapi.hyq_hybrid_attention_decode(q.cuda(), cache, out_dtype=torch.float32)
