@@ -106,6 +106,15 @@ int hyq_kv_cache_query_sizes(const hyq_kv_cache* cache, hyq_kv_cache_sizes* size
 int hyq_freeze(const void* k_, const void* v, const int32_t* vl_idx, const hyq_kv_cache* cache, void* stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * hyq_kv_cache_append - places one new token's key and value rows in the staging buffer (Algorithm 4's
+ * "newly generated tokens are first placed in a small staging buffer"): k_new, v_new [B,Hkv,D] bf16 (device)
+ * are copied to row cache->n_staging of k_s / v_s.  The description is not modified: the caller counts the row
+ * (n_staging + 1) in the description it passes to the next attention call.  n_staging == staging_capacity ->
+ * HYQ_ERR_INVALID_ARG (buffer full).  Other errors as hyq_freeze.
+ * ------------------------------------------------------------------------------------------- */
+int hyq_kv_cache_append(const void* k_new, const void* v_new, const hyq_kv_cache* cache, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
  * hyq_hybrid_attention_decode - Algorithm 3 / Section 3.3 for one token per sequence:
  *     s_j   = softmax_scale * <q[b,h], key_j>      over every cached row j of KV head h / g, where
  *             key_j / value_j = scale(group) * code for quantized rows, the bf16 row otherwise

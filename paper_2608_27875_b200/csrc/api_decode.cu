@@ -62,6 +62,14 @@ int hyq_freeze(const void* k_, const void* v, const int32_t* vl_idx, const hyq_k
     return launch_freeze(k_, v, vl_idx, *cache, static_cast<cudaStream_t>(stream));
 }
 
+int hyq_kv_cache_append(const void* k_new, const void* v_new, const hyq_kv_cache* cache, void* stream) {
+    const int rc = check_cache(cache, false);
+    if (rc != HYQ_OK) return rc;
+    if (!k_new || !v_new || !cache->k_s || !cache->v_s || cache->n_staging >= cache->staging_capacity) return HYQ_ERR_INVALID_ARG;
+    if (!aligned16(k_new) || !aligned16(v_new) || !aligned16(cache->k_s) || !aligned16(cache->v_s)) return HYQ_ERR_ALIGNMENT;
+    return launch_cache_append(k_new, v_new, *cache, static_cast<cudaStream_t>(stream));
+}
+
 int hyq_hybrid_attention_decode_workspace(const hyq_kv_cache* cache, int splits, size_t* bytes) {
     if (!bytes || splits < 0 || splits > 1024) return HYQ_ERR_INVALID_ARG;
     const int rc = check_cache(cache, false);

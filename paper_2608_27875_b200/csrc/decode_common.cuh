@@ -47,6 +47,7 @@ __host__ __device__ __forceinline__ int vq8_byte_offset(int key, int d) {
 }
 
 int launch_freeze(const void* k_, const void* v, const int32_t* vl_idx, const hyq_kv_cache& c, cudaStream_t st);
+int launch_cache_append(const void* k_new, const void* v_new, const hyq_kv_cache& c, cudaStream_t st);
 int decode_auto_splits(const hyq_kv_cache& c);
 size_t decode_workspace_bytes(const hyq_kv_cache& c, int splits);
 int launch_decode(const void* q, const hyq_kv_cache& c, const int32_t* lengths, float alpha, int splits, int out_dtype,

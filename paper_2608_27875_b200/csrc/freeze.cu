@@ -193,6 +193,26 @@ freeze_quantize_kernel(const uint4* __restrict__ k_, const uint4* __restrict__ v
     }
 }
 
+// one new token per sequence: rows [B*Hkv][128] bf16 -> row `row` of every head's staging buffer
+__global__ void __launch_bounds__(FRZ_THREADS)
+append_rows_kernel(const uint4* __restrict__ k_new, const uint4* __restrict__ v_new, long heads, int row, int Ws,
+                   uint4* __restrict__ k_s, uint4* __restrict__ v_s) {
+    const long e = (long)blockIdx.x * FRZ_THREADS + threadIdx.x;     // 16 x 16 bytes per head row
+    if (e >= heads * 16) return;
+    const long head = e >> 4, c = e & 15;
+    const long d = (head * Ws + row) * 16 + c;
+    k_s[d] = __ldg(k_new + e);
+    v_s[d] = __ldg(v_new + e);
+}
+
+int launch_cache_append(const void* k_new, const void* v_new, const hyq_kv_cache& c, cudaStream_t st) {
+    const long heads = (long)c.B * c.Hkv;
+    append_rows_kernel<<<(unsigned)((heads * 16 + FRZ_THREADS - 1) / FRZ_THREADS), FRZ_THREADS, 0, st>>>(
+        static_cast<const uint4*>(k_new), static_cast<const uint4*>(v_new), heads, c.n_staging, c.staging_capacity,
+        static_cast<uint4*>(c.k_s), static_cast<uint4*>(c.v_s));
+    return launch_status();
+}
+
 int launch_freeze(const void* k_, const void* v, const int32_t* vl_idx, const hyq_kv_cache& c, cudaStream_t st) {
     const CacheGeo g = cache_geo(c);
     const long heads = (long)c.B * c.Hkv;

@@ -11,7 +11,7 @@ import torch
 from . import api
 from .workloads import FMT_INT4, FMT_INT8
 
-EXPORTS = ("hyq_kv_cache_query_sizes", "hyq_freeze", "hyq_hybrid_attention_decode_workspace",
+EXPORTS = ("hyq_kv_cache_query_sizes", "hyq_freeze", "hyq_kv_cache_append", "hyq_hybrid_attention_decode_workspace",
            "hyq_hybrid_attention_decode", "hyq_hybrid_attention_decode_ragged")
 
 
@@ -41,6 +41,7 @@ def _lib():
     if not _bound:
         L.hyq_kv_cache_query_sizes.argtypes = [ctypes.POINTER(KvCacheDesc), ctypes.POINTER(KvCacheSizes)]
         L.hyq_freeze.argtypes = [ctypes.c_void_p] * 3 + [ctypes.POINTER(KvCacheDesc), ctypes.c_void_p]
+        L.hyq_kv_cache_append.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(KvCacheDesc), ctypes.c_void_p]
         L.hyq_hybrid_attention_decode_workspace.argtypes = [ctypes.POINTER(KvCacheDesc), ctypes.c_int,
                                                             ctypes.POINTER(ctypes.c_size_t)]
         L.hyq_hybrid_attention_decode.argtypes = [ctypes.c_void_p, ctypes.POINTER(KvCacheDesc), ctypes.c_float,
@@ -81,13 +82,11 @@ class HybridKvCache:
         return int(self.desc.n_staging)
 
     def append(self, k_new: torch.Tensor, v_new: torch.Tensor) -> None:
-        """Copies one token's rows ([B,Hkv,D] bf16) into the staging buffer (plain device copies)."""
-        n = self.n_staging
-        if n >= self.desc.staging_capacity:
-            raise ValueError("staging buffer full")
-        self.buffers["k_s"][:, :, n].copy_(k_new)
-        self.buffers["v_s"][:, :, n].copy_(v_new)
-        self.desc.n_staging = n + 1
+        """Places one token's rows ([B,Hkv,D] bf16, contiguous) in the staging buffer (hyq_kv_cache_append)."""
+        api._dev(k_new, torch.bfloat16, "k_new"), api._dev(v_new, torch.bfloat16, "v_new")
+        api._check(_lib().hyq_kv_cache_append(k_new.data_ptr(), v_new.data_ptr(), ctypes.byref(self.desc), api._stream()),
+                   "hyq_kv_cache_append")
+        self.desc.n_staging = self.n_staging + 1
 
     def bytes_read_per_token(self) -> int:
         """Bytes of cache one attention call reads: codes, scales and the valid bf16 rows."""
@@ -195,10 +194,13 @@ class RaggedKvCache:
     def append(self, b: int, k_new: torch.Tensor, v_new: torch.Tensor) -> None:
         """One token's rows ([Hkv,D] bf16) of sequence b into its staging buffer."""
         n = int(self.lengths_host[b, 3])
-        if n >= self.batch.desc.staging_capacity:
-            raise ValueError("staging buffer full")
-        self.batch.buffers["k_s"][b, :, n].copy_(k_new)
-        self.batch.buffers["v_s"][b, :, n].copy_(v_new)
+        api._dev(k_new, torch.bfloat16, "k_new"), api._dev(v_new, torch.bfloat16, "v_new")
+        one = KvCacheDesc()
+        ctypes.memmove(ctypes.byref(one), ctypes.byref(self.batch.desc), ctypes.sizeof(KvCacheDesc))
+        one.B, one.n_staging = 1, n                      # sequence b's staging buffers as a batch of one
+        one.k_s, one.v_s = self.batch.buffers["k_s"][b].data_ptr(), self.batch.buffers["v_s"][b].data_ptr()
+        api._check(_lib().hyq_kv_cache_append(k_new.data_ptr(), v_new.data_ptr(), ctypes.byref(one), api._stream()),
+                   "hyq_kv_cache_append")
         self.lengths_host[b, 3] = n + 1
         self.lengths.copy_(self.lengths_host)
 

@@ -154,4 +154,10 @@ def test_decode_side_argument_checks(lib):
     assert L.hyq_kv_cache_query_sizes(ctypes.byref(d), ctypes.byref(sizes)) == 1
     d.struct_size = ctypes.sizeof(decode_api.KvCacheDesc)
     assert L.hyq_freeze(None, None, None, ctypes.byref(d), None) == 1            # null buffers
+    assert L.hyq_kv_cache_append(None, None, ctypes.byref(d), None) == 1
+    full = decode_api.make_desc(B=2, Hq=32, Hkv=8, N=1000, window=100, k=37)
+    full.k_s, full.v_s, full.n_staging = 0x10000, 0x20000, full.staging_capacity
+    assert L.hyq_kv_cache_append(0x30000, 0x40000, ctypes.byref(full), None) == 1          # staging buffer full
+    full.n_staging = 3
+    assert L.hyq_kv_cache_append(0x30008, 0x40000, ctypes.byref(full), None) == 4          # misaligned rows
     assert L.hyq_hybrid_attention_decode(None, ctypes.byref(d), 0.0, 0, 0, None, None, None, 0, None) == 1

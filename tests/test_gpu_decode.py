@@ -114,6 +114,23 @@ def test_freeze_of_an_all_zero_group_and_clustered_vertical_rows():
     _assert_cache_equal(ref, cache)
 
 
+def test_staging_rows_land_where_the_oracle_puts_them_and_a_full_buffer_is_refused():
+    B, Hkv, N, W, cap = 3, 5, 200, 30, 6
+    K, V = rand_bf16((B, Hkv, N, 128), 6), rand_bf16((B, Hkv, N, 128), 7)
+    ref, cache = _freeze_both(K, V, _idx(B, Hkv, N - W, 4, 8), W, Hq=Hkv, staging_capacity=cap)
+    cache.buffers["k_s"].fill_(-3.0), cache.buffers["v_s"].fill_(-3.0)          # untouched rows keep this marker
+    marker = int(wl.bits(torch.tensor([-3.0], dtype=torch.bfloat16))[0])
+    for n in range(1, cap + 1):
+        _stage(ref, cache, 1, 10 * n)
+        for name in ("k_s", "v_s"):
+            got = wl.bits(cache.buffers[name].cpu())
+            assert np.array_equal(got[:, :, :n], ref[name][:, :, :n]) and (got[:, :, n:] == marker).all()
+    assert cache.n_staging == cap
+    with pytest.raises(dapi.api.HyqError):
+        cache.append(rand_bf16((B, Hkv, 128), 1).cuda(), rand_bf16((B, Hkv, 128), 2).cuda())
+    assert cache.n_staging == cap
+
+
 DECODE_SHAPES = [  # B, Hq, Hkv, N, W, k, n_s, splits
     (1, 4, 1, 300, 40, 9, 0, 1), (1, 4, 1, 300, 40, 9, 3, 0), (2, 8, 2, 1000, 128, 37, 5, 3), (1, 2, 2, 64, 0, 0, 1, 1),
     (1, 8, 1, 129, 1, 64, 0, 2), (1, 6, 2, 50, 80, 0, 0, 0), (1, 4, 2, 200, 20, 180, 17, 4), (1, 16, 2, 2000, 100, 50, 128, 0),
