@@ -15,9 +15,9 @@
  *   window       k_win, v_win  [B,Hkv,W',D] bf16   the last W' = min(window, N) prefill rows
  *   vertical     k_vl, v_vl    [B,Hkv,k,D]  bf16   rows vl_idx[b,h,:] of the prefill cache, in that order
  *   staging      k_s, v_s      [B,Hkv,staging_capacity,D] bf16, of which the first n_staging rows are
- *                              valid; the caller appends new tokens' rows there (plain copies) and
- *                              counts them in n_staging.  Folding staged rows into the other buffers
- *                              is not described by the paper and not part of this library.
+ *                              valid; hyq_kv_cache_append writes a new token's rows to row n_staging and
+ *                              the caller counts them in n_staging.  Folding staged rows into the other
+ *                              buffers is not described by the paper and not part of this library.
  *   quantized    the other nQ = N - W' - k prefix rows, COMPACTED in ascending position order and cut
  *                into groups of `group` (G = 32, 64 or 128) consecutive compacted rows x all D channels; each group is
  *                quantized exactly as hyq_quantize_blocks quantizes a tile (INT4, c_B = 7; INT8, c_B = 127; FP8 e4m3, c_B = 448;
