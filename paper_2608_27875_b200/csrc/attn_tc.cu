@@ -37,6 +37,11 @@
 #ifndef HYQ_TC_VARIANT_BT
 #define HYQ_TC_VARIANT_BT 0
 #endif
+// One softmax thread per query row (four warps per query tile, 64 columns per thread, no pairwise vote) in the default
+// translation unit; the run-time block-size variant keeps two threads per row (its column halves have separate K scales).
+#ifndef HYQ_OTPR
+#define HYQ_OTPR (!HYQ_TC_VARIANT_BT)
+#endif
 
 namespace hyq {
 #if HYQ_TC_VARIANT_BT
@@ -226,7 +231,45 @@ __device__ __forceinline__ bool mma_issuer(int q, const QSched& sq, const Walk& 
     uint32_t n_pv = 0;
     for (int t = 0; t < NBUF && tq < T1; ++t)
         if (!qk(false)) return false;
+    // Steady state of the low-bit pass, four walk positions per trip: this thread's pace is set by the dependent
+    // instructions it executes per tile, so ring stages, S buffers, barrier addresses and descriptors are compile-time
+    // offsets here and the parities change once per trip.  Taken only where the cursors are in phase (V stage 0,
+    // K stage 2, even tile counts) and all eight tiles involved are low-bit tiles of this query tile.
+    constexpr bool FAST = (NST == 4 && NBUF == 2);
+    const uint32_t a_bars = smem_u32(&bars);
+    const int fast_end = min(own.a_end, T1) - 5;
     for (int t = w.t0; t < T1; ++t) {
+        if (FAST && t < fast_end && vst == 0 && kst == 2 && n_pv > 0 && ((n_pv | n_qk) & 1u) == 0 && tq == t + 2) {
+            const uint32_t pp = (n_pv >> 1) & 1u;
+            bool ok = true;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int ks = (2 + i) & 3, bf = i & 1;
+                const uint32_t a_p = a_bars + (uint32_t)offsetof(TcBarriers, p_full) + (q * 2 + bf) * 8;
+                const uint32_t a_kf = a_bars + (uint32_t)offsetof(TcBarriers, kv_full) + ks * 8;
+                const uint32_t ppi = i < 2 ? pp : pp ^ 1u, kpi = i < 2 ? kpar : kpar ^ 1u;
+                const uint32_t done = mbar_test_wait2_a(a_p, ppi, a_kf, kpi);
+                if (!(done & 1u) && !mbar_wait_a(a_p, ppi, WAIT_LIMIT)) { ok = false; break; }
+                tc_fence_after();
+#pragma unroll
+                for (int kk = 0; kk < BN / 16; ++kk)
+                    umma_ts_f16(to, ts0 + bf * BN + kk * 8, dv0 + (uint64_t)(i * STAGE16 + kk * 128), idesc_pv, 1u);
+                umma_commit_a(a_bars + (uint32_t)offsetof(TcBarriers, o_done) + (q * 2 + bf) * 8);
+                umma_commit_a(a_bars + (uint32_t)offsetof(TcBarriers, kv_free) + i * 8);
+                if (!(done & 2u) && !mbar_wait_a(a_kf, kpi, WAIT_LIMIT)) { ok = false; break; }
+                tc_fence_after();
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) {
+                    if (LOWBIT_FP8) umma_ss_f8f6f4(ts0 + bf * BN, dqc + kk * 2, dk0 + (uint64_t)(ks * STAGE16 + kk * 2), idesc_lq, kk > 0);
+                    else umma_ss_i8(ts0 + bf * BN, dqc + kk * 2, dk0 + (uint64_t)(ks * STAGE16 + kk * 2), idesc_lq, kk > 0);
+                }
+                umma_commit_a(a_bars + (uint32_t)offsetof(TcBarriers, s_full) + (q * 2 + bf) * 8);
+            }
+            if (!ok) return false;
+            n_pv += 4; n_qk += 4; tq += 4; kpar ^= 1u; t += 3;
+            if (*abort_flag) return true;
+            continue;
+        }
         // (the V tile of position t came in on the same barrier as its K tile, which Q.K^T waited for)
         bool k_ready = false;
         if (own.has(t)) {
@@ -310,7 +353,7 @@ __device__ __forceinline__ bool tma_producer(const TcMaps& maps, const QSched& q
 // row arrive at the same new reference, rescale their half of O (64 channels each) and their partial row sum.
 // The vote also orders "both halves have read S" before "either half writes P over it".  The partial sums are
 // added at the end (exchange through TMEM).
-constexpr int TC_THREADS = 640;                     // TMA producer, 2 MMA issuers, 1 idle warp, 16 softmax warps
+constexpr int TC_THREADS = HYQ_OTPR ? 384 : 640;                     // TMA producer, 2 MMA issuers, 1 idle warp, 16 softmax warps
 constexpr float RAISE_THRESHOLD = 14.0f;            // log2 units by which a tile must exceed the reference to raise it (P stays below 2^14, inside fp16)
 
 // named barrier over `nthreads` threads with an OR reduction of `pred` (all threads of the participating warps call it)
@@ -434,7 +477,7 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
         for (int q = 0; q < QT; ++q) {
             for (int bf = 0; bf < 2; ++bf) {
                 mbar_init(&bars.s_full[q][bf], 1);
-                mbar_init(&bars.p_full[q][bf], 8);           // one arrival per softmax warp of the query tile
+                mbar_init(&bars.p_full[q][bf], HYQ_OTPR ? 4 : 8);           // one arrival per softmax warp of the query tile
                 mbar_init(&bars.o_done[q][bf], 1);
             }
         }
@@ -492,7 +535,11 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
         }
     } else if (warp >= 4) {
         // ------------------------------------------------------------------ softmax warps
+#if HYQ_OTPR
+        const int q = (warp - 4) >> 2, hsel = 0;                        // query tile (a thread owns all 64 columns of its row)
+#else
         const int q = (warp - 4) >> 3, hsel = ((warp - 4) >> 2) & 1;    // query tile, column half
+#endif
         const QSched sq = q ? qs1 : qs0;
         // named barrier of the two warps that share this warp's 32 query rows (one per query tile and lane quarter)
         const int bar_id = 1 + q * 4 + (warp & 3);
@@ -503,7 +550,7 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
         if (SPLIT && sq.live && n_total <= n0) {
             // nothing of this query tile lies in the slice: an empty partial result
             const int i = sq.i0 + (warp & 3) * 32 + lane;
-            if ((((warp - 4) >> 2) & 1) == 0 && i < L)
+            if (hsel == 0 && i < L)
                 reinterpret_cast<float2*>(p.part_ml)[((long)split * gridDim.y * gridDim.z + qhead) * L + i] = make_float2(-INFINITY, 0.0f);
         }
         if (sq.live && n_total > n0) {
@@ -542,7 +589,11 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
 #endif
             const uint32_t* vl_ptr = p.vl_bits + (long)qhead * p.mask_words + hsel;
             float nks = 0.0f;
+#if HYQ_OTPR
+            uint64_t nvl = 0u;                                  // both mask words of the tile (columns 0-31 low, 32-63 high)
+#else
             uint32_t nvl = 0u;
+#endif
             auto prefetch_tile = [&](int n) {
                 nks = 0.0f; nvl = 0u;
                 if (n >= own.a_end) return;
@@ -551,11 +602,93 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
 #else
                 nks = __ldg(ks_ptr + n);
 #endif
+#if HYQ_OTPR
+                nvl = (uint64_t)__ldg(vl_ptr + 2 * n) | ((uint64_t)__ldg(vl_ptr + 2 * n + 1) << 32);
+#else
                 nvl = __ldg(vl_ptr + 2 * n);
+#endif
             };
             prefetch_tile(n0);
             const float qs2 = q_scale * p.scale_log2;
 
+#if HYQ_OTPR
+            // one tile of the online softmax for this thread's row: all 64 columns, in two register halves.  Returns
+            // false when this warp ran into an expired wait.
+            auto do_tile = [&](auto range_tag, int n, float cs, uint64_t vl, bool int_scores, int lo_eff, unsigned span) -> bool {
+                constexpr bool NEED_RANGE = decltype(range_tag)::value;
+                const uint32_t knock = int_scores ? KNOCKOUT_S32 : KNOCKOUT_F32;
+                const int nl = n - n0;                          // tile number within this CTA's slice
+                const int buf = nl & 1;
+                const uint32_t ts = ts0 + buf * BN;
+                if (!__all_sync(0xffffffffu, mbar_wait(&bars.s_full[q][buf], (uint32_t)(nl >> 1) & 1u, WAIT_LIMIT))) {
+                    dead = true;
+                    return false;
+                }
+                tc_fence_after();
+                // vertical-line keys of a low-bit tile: -inf into their S columns before the row is read
+                if (vl != 0ull) {                                // uniform over the warp
+                    while (vl) { const int c = __ffsll((long long)vl) - 1; vl &= vl - 1; tmem_st1(ts + c, knock_lq); }
+                    tmem_wait_st();
+                }
+                uint32_t ra[32], rb[32];
+                tmem_ld32(ts, ra);
+                tmem_ld32(ts + 32, rb);
+                tmem_wait_ld();
+                if (NEED_RANGE) {
+                    mask_cols32(ra, 0, lo_eff, span, knock);
+                    mask_cols32(rb, 32, lo_eff, span, knock);
+                }
+                // integer scores become the floats 2^23 + 2^22 + s by one integer add each (knocked-out entries
+                // become -inf); the offset is taken out again by the bias of the exponent
+                if (int_scores) {
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) { ra[e] += INT_MAGIC; rb[e] += INT_MAGIC; }
+                }
+                const float f = fmaxf(row_max32(ra), row_max32(rb)) - (int_scores ? INT_MAGIC_F : 0.0f);
+                const float mt = (f == -INFINITY) ? -INFINITY : f * cs;
+                const bool raise = mt > m_used + RAISE_THRESHOLD;
+                if (__any_sync(0xffffffffu, raise)) {
+                    const float alpha = raise ? ex2f(m_used - mt) : 1.0f;      // m_used = -inf -> 0
+                    if (nl > 0) {
+                        // P.V of tile n-1 must have landed before O is rescaled.  P.V number m signals barrier m & 1;
+                        // the one before the previous is complete (the scores just read were issued after it), so
+                        // the parity wait cannot alias.
+                        if (!__all_sync(0xffffffffu, mbar_wait(&bars.o_done[q][(nl - 1) & 1], (uint32_t)((nl - 1) >> 1) & 1u, WAIT_LIMIT))) {
+                            dead = true;
+                            return false;
+                        }
+                        tc_fence_after();
+#pragma unroll 1
+                        for (int c = 0; c < 8; ++c) {
+                            uint32_t o[16];
+                            tmem_ld16(to + c * 16, o);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int e = 0; e < 16; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+                            tmem_st16(to + c * 16, o);
+                        }
+                        tmem_wait_st();
+                    }
+                    if (raise) {
+                        l_h *= alpha;
+                        m_used = mt;
+                    }
+                }
+                // ---- P = 2^(s - m) as fp16 pairs over the first 32 columns of the buffer; row sum
+                const float m_eff = (m_used == -INFINITY) ? 0.0f : m_used;
+                const float bias = int_scores ? fmaf(-INT_MAGIC_F, cs, -m_eff) : -m_eff;
+                uint32_t pa[16], pb[16];
+                l_h += row_exp32(ra, cs, bias, pa);
+                tmem_st16(ts, pa);
+                l_h += row_exp32(rb, cs, bias, pb);
+                tmem_st16(ts + 16, pb);
+                tmem_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bars.p_full[q][buf]);
+                return true;
+            };
+#else
             // one tile of the online softmax for this thread's 32 columns.  Returns false when the query tile's
             // softmax warps leave the loop together (an expired wait somewhere).
             auto do_tile = [&](auto range_tag, int n, float cs, uint32_t vl, bool int_scores, int lo_eff, unsigned span) -> bool {
@@ -668,6 +801,7 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                 }
                 return true;
             };
+#endif
 
             // ---- low-bit tiles that lie wholly below every row's window: no range mask, no bounds to compute
             const int n_plain = ragged ? 0 : min(own.a_end, max(0, (qhi(sq.i0 + off) + 1) / BN));
@@ -676,7 +810,7 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                 HYQ_TR(q * 2 + hsel, n, 2);
                 // a zero scale (all-zero tile) still has to let -inf pass through the multiply
                 const float cs = fmaxf(qs2 * nks, 1e-37f);
-                const uint32_t vl = nvl;
+                const auto vl = nvl;
                 prefetch_tile(n + 1);
                 if (!do_tile(std::false_type{}, n, cs, vl, !LOWBIT_FP8, 0, 0u)) { aborted = true; break; }
             }
@@ -687,7 +821,7 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                 HYQ_TR(q * 2 + hsel, n, 2);
                 const int t = walk_pos(n);
                 const float ks = nks;
-                const uint32_t vl = nvl;
+                const auto vl = nvl;
                 prefetch_tile(n + 1);
                 int lo = 0, hi = -1;
                 float cs;
@@ -714,6 +848,11 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
             if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars.o_done[q][(n_total - n0 - 1) & 1], (uint32_t)((n_total - n0 - 1) >> 1) & 1u, WAIT_LIMIT));
             if (!aborted) {                                     // uniform over the query tile's softmax warps
                 tc_fence_after();
+#if HYQ_OTPR
+                constexpr int NCH = 4;                          // 32-channel pieces of the row this thread writes
+                const float l_run = l_h;
+#else
+                constexpr int NCH = 2;
                 tmem_st1(ts0 + col0, __float_as_uint(l_h));     // column col0 of S buffer 0 (all MMAs are done)
                 tmem_wait_st();
                 tc_fence_before();
@@ -722,13 +861,14 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                 const float l_o = __uint_as_float(tmem_ld1(ts0 + col0_other));
                 tmem_wait_ld();
                 const float l_run = l_h + l_o;
+#endif
                 const float inv = (l_run > 0.0f) ? 1.0f / l_run : 0.0f;
                 if (SPLIT) {
                     // partial result of this slice: O as accumulated (relative to m_used), the pair (m_used, l)
                     const long prow = ((long)split * gridDim.y * gridDim.z + qhead) * L + i;
                     if (ok) {
 #pragma unroll
-                        for (int c = 0; c < 2; ++c) {
+                        for (int c = 0; c < NCH; ++c) {
                             uint32_t o[32];
                             const int ch = hsel * 64 + c * 32;
                             tmem_ld32(to + ch, o);
@@ -743,7 +883,7 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                     }
                 } else if (ok) {
 #pragma unroll
-                    for (int c = 0; c < 2; ++c) {              // this half writes channels [64 hsel, 64 hsel + 64)
+                    for (int c = 0; c < NCH; ++c) {            // this thread's channels: [64 hsel, 64 hsel + 32 NCH)
                         uint32_t o[32];
                         const int ch = hsel * 64 + c * 32;
                         tmem_ld32(to + ch, o);

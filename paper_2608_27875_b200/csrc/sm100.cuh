@@ -82,6 +82,31 @@ __device__ __forceinline__ uint32_t mbar_test_wait2(uint64_t* bar0, uint32_t par
     return done;
 }
 
+// The same operations on 32-bit shared-window addresses (for loops whose barrier addresses are a base register
+// plus a compile-time offset).
+__device__ __forceinline__ uint32_t mbar_test_wait2_a(uint32_t a0, uint32_t parity0, uint32_t a1, uint32_t parity1) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred P, Q;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 P, [%1], %2;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 Q, [%3], %4;\n\t"
+        "selp.u32 %0, 1, 0, P;\n\t@Q or.b32 %0, %0, 2;\n\t}\n"
+        : "=r"(done) : "r"(a0), "r"(parity0), "r"(a1), "r"(parity1) : "memory");
+    return done;
+}
+// bounded wait (the caller has just probed the barrier): try_wait in a loop that reads the clock
+__device__ __forceinline__ bool mbar_wait_a(uint32_t a, uint32_t parity, long long limit_cycles) {
+    const long long t0 = clock64();
+    for (;;) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred P;\n\tmbarrier.try_wait.parity.shared::cta.b64 P, [%1], %2;\n\tselp.u32 %0, 1, 0, P;\n\t}\n"
+            : "=r"(ok) : "r"(a), "r"(parity) : "memory");
+        if (ok) return true;
+        if (clock64() - t0 > limit_cycles) return false;
+    }
+}
+
 // ---- TMA --------------------------------------------------------------------------------------
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* m) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(m)) : "memory");
@@ -111,6 +136,10 @@ __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::
 // all MMAs issued so far by this thread arrive on `bar` when they have completed
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+__device__ __forceinline__ void umma_commit_a(uint32_t a) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(a) : "memory");
 }
 
 // ---- descriptors ------------------------------------------------------------------------------
