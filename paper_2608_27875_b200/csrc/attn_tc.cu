@@ -14,14 +14,17 @@
 // a walk position share one stage of a 4-stage ring (one "full" and one "free" barrier per stage) and
 // are used by both query tiles.
 //
-// Warp roles (640 threads): warp 0 lane 0 issues the TMA loads, warps 1 and 2 (lane 0) issue the
-// MMAs of query tile 0 and 1, warp 3 idles, warps 4-19 are the softmax warps: eight per query tile,
-// two threads per query row (thread (r, h) owns columns [32 h, 32 h + 32) of row r = TMEM lane r of
-// every score tile), so that each of the four schedulers hosts four softmax warps and a thread holds
-// 32 scores.  The exponentials are taken against a per-row reference maximum that is only raised when
+// Warp roles (384 threads): warp 0 lane 0 issues the TMA loads, warps 1 and 2 (lane 0) issue the
+// MMAs of query tile 0 and 1 (four tiles per trip with compile-time ring positions in the steady
+// state of the low-bit pass), warp 3 idles, warps 4-11 are the softmax warps: four per query tile,
+// one thread per query row (row r = TMEM lane r of every score tile; the thread holds the 64 scores
+// of its row in two register halves), so a row's reference maximum needs no agreement between
+// threads.  The exponentials are taken against that reference, which is only raised when
 // a tile exceeds it by more than 2^14 (the rescale of O is then rare); integer scores become floats
 // by a magic-number add.  Every mbarrier wait is bounded; when one expires the CTA records
-// HYQ_ERR_TIMEOUT in the status word and unwinds.
+// HYQ_ERR_TIMEOUT in the status word and unwinds.  (The build with a run-time block size keeps the
+// earlier layout of 640 threads with two threads per row, whose column halves can have separate
+// K scales: HYQ_OTPR = 0.)
 #include <cuda_fp16.h>
 
 #include <type_traits>
@@ -345,15 +348,19 @@ __device__ __forceinline__ bool tma_producer(const TcMaps& maps, const QSched& q
     return true;
 }
 
-// ---- softmax warps: two threads per query row ----------------------------------------------------
-// The two threads of a row must exponentiate against the same reference maximum.  Per tile they take the maximum
+// ---- softmax warps -------------------------------------------------------------------------------
+// One thread per query row (HYQ_OTPR): the thread reads its 64 scores of a tile in two register halves, raises the
+// row's reference when the tile's maximum exceeds it by more than the threshold (rescaling O and the row sum), and
+// writes the 64 probabilities as fp16 pairs over the first 32 columns of the buffer it read.
+// Two threads per query row (the layout of the run-time block-size build):
+// the two threads of a row must exponentiate against the same reference maximum.  Per tile they take the maximum
 // of their own 32 columns, and the two warps that share 32 query rows vote (named barrier of 64 threads with OR
 // reduction) whether any of these rows has to raise its reference.  In the common case none does and each half
 // proceeds on its own; otherwise every thread also reads the other half's scores from TMEM, so both threads of a
 // row arrive at the same new reference, rescale their half of O (64 channels each) and their partial row sum.
 // The vote also orders "both halves have read S" before "either half writes P over it".  The partial sums are
 // added at the end (exchange through TMEM).
-constexpr int TC_THREADS = HYQ_OTPR ? 384 : 640;                     // TMA producer, 2 MMA issuers, 1 idle warp, 16 softmax warps
+constexpr int TC_THREADS = HYQ_OTPR ? 384 : 640;   // TMA producer, 2 MMA issuers, 1 idle warp, 8 (16) softmax warps
 constexpr float RAISE_THRESHOLD = 14.0f;            // log2 units by which a tile must exceed the reference to raise it (P stays below 2^14, inside fp16)
 
 // named barrier over `nthreads` threads with an OR reduction of `pred` (all threads of the participating warps call it)
@@ -620,10 +627,12 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                 const int nl = n - n0;                          // tile number within this CTA's slice
                 const int buf = nl & 1;
                 const uint32_t ts = ts0 + buf * BN;
+                HYQ_TR(q * 2, n, 0);
                 if (!__all_sync(0xffffffffu, mbar_wait(&bars.s_full[q][buf], (uint32_t)(nl >> 1) & 1u, WAIT_LIMIT))) {
                     dead = true;
                     return false;
                 }
+                HYQ_TR(q * 2, n, 1);
                 tc_fence_after();
                 // vertical-line keys of a low-bit tile: -inf into their S columns before the row is read
                 if (vl != 0ull) {                                // uniform over the warp
@@ -634,6 +643,7 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                 tmem_ld32(ts, ra);
                 tmem_ld32(ts + 32, rb);
                 tmem_wait_ld();
+                HYQ_TR(q * 2, n, 3);
                 if (NEED_RANGE) {
                     mask_cols32(ra, 0, lo_eff, span, knock);
                     mask_cols32(rb, 32, lo_eff, span, knock);
@@ -647,6 +657,7 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                 const float f = fmaxf(row_max32(ra), row_max32(rb)) - (int_scores ? INT_MAGIC_F : 0.0f);
                 const float mt = (f == -INFINITY) ? -INFINITY : f * cs;
                 const bool raise = mt > m_used + RAISE_THRESHOLD;
+                HYQ_TR(q * 2, n, 4);
                 if (__any_sync(0xffffffffu, raise)) {
                     const float alpha = raise ? ex2f(m_used - mt) : 1.0f;      // m_used = -inf -> 0
                     if (nl > 0) {
@@ -681,11 +692,14 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                 l_h += row_exp32(ra, cs, bias, pa);
                 tmem_st16(ts, pa);
                 l_h += row_exp32(rb, cs, bias, pb);
+                HYQ_TR(q * 2, n, 5);
                 tmem_st16(ts + 16, pb);
                 tmem_wait_st();
                 tc_fence_before();
                 __syncwarp();
+                HYQ_TR(q * 2, n, 6);
                 if (lane == 0) mbar_arrive(&bars.p_full[q][buf]);
+                HYQ_TR(q * 2, n, 7);
                 return true;
             };
 #else
