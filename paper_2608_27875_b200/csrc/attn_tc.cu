@@ -854,13 +854,12 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                 }
                 const int lo_eff = (hi >= lo) ? lo : 4096;
                 const unsigned span = (hi >= lo) ? (unsigned)(hi - lo) : 0u;
-#if HYQ_OTPR
                 // tiles that every row of this warp uses in full (most window and vertical-line tiles) need no range mask
+                // (with two threads per row both warps of a pair still meet at the same named barriers)
                 if (__all_sync(0xffffffffu, lo == 0 && hi == BN - 1)) {
                     if (!do_tile(std::false_type{}, n, cs, vl, lowbit && !LOWBIT_FP8, 0, 0u)) aborted = true;
                     continue;
                 }
-#endif
                 if (!do_tile(std::true_type{}, n, cs, vl, lowbit && !LOWBIT_FP8, lo_eff, span)) aborted = true;
             }
 
