@@ -22,9 +22,8 @@
 // threads.  The exponentials are taken against that reference, which is only raised when
 // a tile exceeds it by more than 2^14 (the rescale of O is then rare); integer scores become floats
 // by a magic-number add.  Every mbarrier wait is bounded; when one expires the CTA records
-// HYQ_ERR_TIMEOUT in the status word and unwinds.  (The build with a run-time block size keeps the
-// earlier layout of 640 threads with two threads per row, whose column halves can have separate
-// K scales: HYQ_OTPR = 0.)
+// HYQ_ERR_TIMEOUT in the status word and unwinds.  (Compiled with HYQ_OTPR = 0 the file gives the
+// earlier layout of 640 threads with two threads per row and a pairwise vote per tile.)
 #include <cuda_fp16.h>
 
 #include <type_traits>
@@ -40,10 +39,11 @@
 #ifndef HYQ_TC_VARIANT_BT
 #define HYQ_TC_VARIANT_BT 0
 #endif
-// One softmax thread per query row (four warps per query tile, 64 columns per thread, no pairwise vote) in the default
-// translation unit; the run-time block-size variant keeps two threads per row (its column halves have separate K scales).
+// One softmax thread per query row (four warps per query tile, 64 columns per thread, no pairwise vote).  In the run-time
+// block-size variant the two column halves of a tile can have separate K scales (32-token blocks): the thread then
+// applies each half's own factor.  HYQ_OTPR = 0 selects the earlier layout with two threads per row.
 #ifndef HYQ_OTPR
-#define HYQ_OTPR (!HYQ_TC_VARIANT_BT)
+#define HYQ_OTPR 1
 #endif
 
 namespace hyq {
@@ -352,7 +352,7 @@ __device__ __forceinline__ bool tma_producer(const TcMaps& maps, const QSched& q
 // One thread per query row (HYQ_OTPR): the thread reads its 64 scores of a tile in two register halves, raises the
 // row's reference when the tile's maximum exceeds it by more than the threshold (rescaling O and the row sum), and
 // writes the 64 probabilities as fp16 pairs over the first 32 columns of the buffer it read.
-// Two threads per query row (the layout of the run-time block-size build):
+// Two threads per query row (HYQ_OTPR = 0, the earlier layout):
 // the two threads of a row must exponentiate against the same reference maximum.  Per tile they take the maximum
 // of their own 32 columns, and the two warps that share 32 query rows vote (named barrier of 64 threads with OR
 // reduction) whether any of these rows has to raise its reference.  In the common case none does and each half
@@ -596,6 +596,9 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
 #endif
             const uint32_t* vl_ptr = p.vl_bits + (long)qhead * p.mask_words + hsel;
             float nks = 0.0f;
+#if HYQ_TC_VARIANT_BT && HYQ_OTPR
+            float nks_b = 0.0f, cs_hi = 0.0f;                   // K scale and score factor of columns 32-63 (32-token blocks: their own block)
+#endif
 #if HYQ_OTPR
             uint64_t nvl = 0u;                                  // both mask words of the tile (columns 0-31 low, 32-63 high)
 #else
@@ -603,9 +606,15 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
 #endif
             auto prefetch_tile = [&](int n) {
                 nks = 0.0f; nvl = 0u;
+#if HYQ_TC_VARIANT_BT && HYQ_OTPR
+                nks_b = 0.0f;
+#endif
                 if (n >= own.a_end) return;
 #if HYQ_TC_VARIANT_BT
                 nks = __ldg(ks_ptr + ((n << 6) >> bsh));
+#if HYQ_OTPR
+                nks_b = (bsh == 5) ? __ldg(ks_ptr + 2 * n + 1) : nks;
+#endif
 #else
                 nks = __ldg(ks_ptr + n);
 #endif
@@ -654,8 +663,14 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
 #pragma unroll
                     for (int e = 0; e < 32; ++e) { ra[e] += INT_MAGIC; rb[e] += INT_MAGIC; }
                 }
+#if HYQ_TC_VARIANT_BT
+                const float csb = cs_hi;                        // the second half's factor (its own K scale with 32-token blocks)
+                const float fa = row_max32(ra) - (int_scores ? INT_MAGIC_F : 0.0f), fb = row_max32(rb) - (int_scores ? INT_MAGIC_F : 0.0f);
+                const float mt = fmaxf((fa == -INFINITY) ? -INFINITY : fa * cs, (fb == -INFINITY) ? -INFINITY : fb * csb);
+#else
                 const float f = fmaxf(row_max32(ra), row_max32(rb)) - (int_scores ? INT_MAGIC_F : 0.0f);
                 const float mt = (f == -INFINITY) ? -INFINITY : f * cs;
+#endif
                 const bool raise = mt > m_used + RAISE_THRESHOLD;
                 HYQ_TR(q * 2, n, 4);
                 if (__any_sync(0xffffffffu, raise)) {
@@ -691,7 +706,11 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                 uint32_t pa[16], pb[16];
                 l_h += row_exp32(ra, cs, bias, pa);
                 tmem_st16(ts, pa);
+#if HYQ_TC_VARIANT_BT
+                l_h += row_exp32(rb, csb, int_scores ? fmaf(-INT_MAGIC_F, csb, -m_eff) : -m_eff, pb);
+#else
                 l_h += row_exp32(rb, cs, bias, pb);
+#endif
                 HYQ_TR(q * 2, n, 5);
                 tmem_st16(ts + 16, pb);
                 tmem_wait_st();
@@ -824,6 +843,9 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                 HYQ_TR(q * 2 + hsel, n, 2);
                 // a zero scale (all-zero tile) still has to let -inf pass through the multiply
                 const float cs = fmaxf(qs2 * nks, 1e-37f);
+#if HYQ_TC_VARIANT_BT && HYQ_OTPR
+                cs_hi = fmaxf(qs2 * nks_b, 1e-37f);
+#endif
                 const auto vl = nvl;
                 prefetch_tile(n + 1);
                 if (!do_tile(std::false_type{}, n, cs, vl, !LOWBIT_FP8, 0, 0u)) { aborted = true; break; }
@@ -835,6 +857,9 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                 HYQ_TR(q * 2 + hsel, n, 2);
                 const int t = walk_pos(n);
                 const float ks = nks;
+#if HYQ_TC_VARIANT_BT && HYQ_OTPR
+                const float ks_b = nks_b;
+#endif
                 const auto vl = nvl;
                 prefetch_tile(n + 1);
                 int lo = 0, hi = -1;
@@ -852,6 +877,9 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                     hi = row_live ? min(ia - j0, BN - 1) : -1;
                     cs = p.scale_log2;
                 }
+#if HYQ_TC_VARIANT_BT && HYQ_OTPR
+                cs_hi = lowbit ? fmaxf(qs2 * ks_b, 1e-37f) : cs;
+#endif
                 const int lo_eff = (hi >= lo) ? lo : 4096;
                 const unsigned span = (hi >= lo) ? (unsigned)(hi - lo) : 0u;
                 // tiles that every row of this warp uses in full (most window and vertical-line tiles) need no range mask
