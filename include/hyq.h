@@ -106,7 +106,9 @@ int hyq_select_vertical(const void* q, const void* k_, int B, int Hq, int Hkv, i
  *   (8 MiB covers B*Hq*(P + 128) <= 1 Mi scores, e.g. 32 query heads at L = 32768, window 1024.)
  *
  *   The first call on each device looks up the array's device address (one runtime query, made with
- *   that device current, result cached); make that first call outside any stream capture.
+ *   that device current, result cached); make that first call outside any stream capture.  The cached
+ *   address belongs to the device's primary context: a process that destroys that context
+ *   (cudaDeviceReset) and creates a new one must not go on using this entry point.
  *   All calls on a device share the one array and each call overwrites what the previous one left
  *   (nothing in it has to start at zero): two calls whose kernels overlap on the GPU - different
  *   streams, or different host threads - race on it.  Run them one after the other.
@@ -186,6 +188,9 @@ int hyq_quantize_blocks(const void* x, int B, int H, int L, int D, int block_tok
  *   struct_size must be sizeof(hyq_attn_args).  Supported format triples (q,k,v):
  *   (INT8,INT8,INT8), (FP8_E4M3,FP8_E4M3,FP8_E4M3) - the paper's two bit widths, c_B = 127 and 448 - and
  *   (INT4,INT4,FP8_E4M3); anything else -> HYQ_ERR_UNSUPPORTED.
+ *   Value range: the value rows enter the P.V products as fp16, so |V| must stay below 65504 (attention values of
+ *   real layers do); larger magnitudes are clamped to +-65504 instead of becoming infinities.  Inputs must be
+ *   finite.
  *   vl_idx [B,Hq,k] int32, each row strictly ascending, values in [0, L); NULL iff k == 0.
  *   out [B,Hq,L,D]: fp32 (out_dtype 1) or bf16 (out_dtype 0, RNE of the fp32 result).
  *   lse: optional [B,Hq,L] fp32 natural-log-sum-exp of the scaled scores (NULL to skip).
@@ -226,6 +231,18 @@ typedef struct {
 
 int hyq_hybrid_attention_prefill_workspace(const hyq_attn_args* args, size_t* bytes /* host, out */);
 int hyq_hybrid_attention_prefill(const hyq_attn_args* args, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * hyq_test_set_attention_hooks - test hook (the paper has no counterpart): exercises the tensor-core
+ * kernel's bounded-wait unwind without faulting anything.  Process-wide, not thread-safe, meant for tests only.
+ *   wait_limit_clocks    SM clocks a single device-side barrier wait may take before the kernel gives up
+ *                        (0: the default of about two seconds)
+ *   drop_load_position   walk position (0-based key tile of a CTA) whose K/V copy the producer announces on its
+ *                        barrier but never issues, so that every wait that depends on it runs out (-1: none)
+ * With a dropped load the kernel returns normally, stores HYQ_ERR_TIMEOUT in status_word and leaves the output
+ * undefined.  Returns HYQ_ERR_INVALID_ARG for negative limits or positions below -1.
+ * ------------------------------------------------------------------------------------------- */
+int hyq_test_set_attention_hooks(long long wait_limit_clocks, int drop_load_position);
 
 #ifdef __cplusplus
 }

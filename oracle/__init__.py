@@ -129,9 +129,13 @@ def exp_det(x) -> np.ndarray:
 
 
 def select_vertical_mass(q_bits, k_bits, window: int, k: int, n_queries: int = 0, alpha: float | None = None,
-                         return_scores: bool = False):
+                         return_scores: bool = False, plain: bool = False):
     """Eq. 4-5: column mass of the softmax rows of the last n_queries queries, top-k over the non-window
-    prefix.  Returns int32 [B,Hq,k] ascending (and optionally the fp64 scores [B,Hq,P])."""
+    prefix.  Returns int32 [B,Hq,k] ascending (and optionally the fp64 scores [B,Hq,P]).
+
+    ``plain=True`` evaluates the definition itself (two-pass softmax per query with libm ``exp`` and
+    sequential sums); the default is the library's fixed-order recipe, which is pinned to the plain form
+    and which the GPU reproduces bit for bit."""
     q = _u16(q_bits, 4)
     kk = _u16(k_bits, 4)
     B, Hq, Lq, D = q.shape
@@ -142,8 +146,9 @@ def select_vertical_mass(q_bits, k_bits, window: int, k: int, n_queries: int = 0
     idx = np.zeros((B, Hq, kk_eff), dtype=np.int32)
     scores = np.zeros((B, Hq, P), dtype=np.float64) if return_scores else None
     a = 1.0 / np.sqrt(np.float64(D)) if alpha is None else float(alpha)
-    rc = _load().oracle_select_mass(_ptr(q), _ptr(kk), B, Hq, Hkv, Lq, Lk, D, window, n_queries, kk_eff,
-                                    ctypes.c_double(a), _ptr(idx), _ptr(scores) if return_scores else None)
+    fn = _load().oracle_select_mass_plain if plain else _load().oracle_select_mass
+    rc = fn(_ptr(q), _ptr(kk), B, Hq, Hkv, Lq, Lk, D, window, n_queries, kk_eff,
+            ctypes.c_double(a), _ptr(idx), _ptr(scores) if return_scores else None)
     if rc:
         raise ValueError(f"oracle_select_mass failed ({rc})")
     return (idx, scores) if return_scores else idx

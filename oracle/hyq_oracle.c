@@ -201,8 +201,11 @@ int oracle_select(const uint16_t* q, const uint16_t* k_, int B, int Hq, int Hkv,
 /* query block is end-aligned with the keys: row i sits at position            */
 /* Lk - Lq + i.  n_queries <= W, so every prefix key is visible to every t.    */
 /*                                                                             */
-/* Because the scores decide an index set that the GPU must reproduce exactly, */
-/* the arithmetic is fixed operation by operation (all fp64, round to nearest):*/
+/* This function is the library's REPRODUCIBILITY CONTRACT, not the definition: */
+/* the definition is oracle_select_mass_plain below (two-pass softmax, libm exp, */
+/* sequential sums), to which this one is pinned at 1e-12 of the largest score.  */
+/* So that the GPU can return the same set bit for bit, the arithmetic is fixed  */
+/* operation by operation (all fp64, round to nearest):                          */
 /*   s       = (fma chain over channels 0..D-1 from 0) * alpha                 */
 /*   exp     = exp_det below (range reduction by ln2 in two parts, degree-13   */
 /*             Taylor polynomial by Horner fma, exact scaling by 2^n)          */
@@ -306,6 +309,60 @@ int oracle_select_mass(const uint16_t* q, const uint16_t* k_, int B, int Hq, int
         for (int c = 0; c < k; ++c) out[c] = sc[c].p;
         qsort(out, k, sizeof(int32_t), cmp_int);
         free(S); free(srow); free(mc); free(zc); free(sc);
+    }
+    return err;
+}
+
+/* ------------------------------------------------------------------------- */
+/* Eq. 4-5 by the plain definition (the reference for oracle_select_mass and    */
+/* for the validity of any selected set): per tail query t a two-pass fp64     */
+/* softmax over the keys j <= pos(t) - libm exp, running maximum and running   */
+/* sum in ascending key order - and S(p) = sum of a_{t,p} over t in ascending  */
+/* query order.  Top-k by (score descending, position ascending), emitted      */
+/* ascending.  No blocking, no polynomial, no reordering.                      */
+/* ------------------------------------------------------------------------- */
+int oracle_select_mass_plain(const uint16_t* q, const uint16_t* k_, int B, int Hq, int Hkv, int Lq, int Lk, int D, int W,
+                             int n_queries, int k, double alpha, int32_t* idx_out, double* scores_out) {
+    if (Hkv <= 0 || Hq % Hkv) return 1;
+    const int g = Hq / Hkv;
+    const int P = (Lk - W > 0) ? Lk - W : 0;
+    if (P == 0 || k == 0) return 0;
+    if (k > P || k < 0 || Lq > Lk) return 1;
+    const int nT = n_queries ? n_queries : (W < Lq ? W : Lq);
+    if (nT <= 0 || nT > Lq || nT > W) return 1;
+    int err = 0;
+#pragma omp parallel for schedule(dynamic)
+    for (int bh = 0; bh < B * Hq; ++bh) {
+        const int b = bh / Hq, h = bh % Hq, kvh = h / g;
+        const uint16_t* kh = k_ + ((long)b * Hkv + kvh) * Lk * D;
+        double* S = (double*)calloc((size_t)P, sizeof(double));
+        double* srow = (double*)malloc(sizeof(double) * (size_t)Lk);
+        scored_t* sc = (scored_t*)malloc(sizeof(scored_t) * (size_t)P);
+        if (!S || !srow || !sc) { err = 2; free(S); free(srow); free(sc); continue; }
+        for (int i = Lq - nT; i < Lq; ++i) {
+            const int pos = Lk - Lq + i;
+            const uint16_t* qr = q + (((long)b * Hq + h) * Lq + i) * D;
+            double m = -INFINITY;
+            for (int j = 0; j <= pos; ++j) {
+                double acc = 0.0;
+                for (int d = 0; d < D; ++d) acc += (double)bf16_to_f32(qr[d]) * (double)bf16_to_f32(kh[(long)j * D + d]);
+                srow[j] = alpha * acc;
+                if (srow[j] > m) m = srow[j];
+            }
+            double Z = 0.0;
+            for (int j = 0; j <= pos; ++j) Z += exp(srow[j] - m);
+            for (int p = 0; p < P; ++p) S[p] += exp(srow[p] - m) / Z;
+        }
+        for (int p = 0; p < P; ++p) {
+            sc[p].s = S[p];
+            sc[p].p = p;
+            if (scores_out) scores_out[(long)bh * P + p] = S[p];
+        }
+        qsort(sc, P, sizeof(scored_t), cmp_scored);
+        int32_t* out = idx_out + (long)bh * k;
+        for (int c = 0; c < k; ++c) out[c] = sc[c].p;
+        qsort(out, k, sizeof(int32_t), cmp_int);
+        free(S); free(srow); free(sc);
     }
     return err;
 }

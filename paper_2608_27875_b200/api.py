@@ -20,7 +20,7 @@ WINDOW_SLIDING, WINDOW_FIXED_TAIL = 0, 1
 EXPORTS = ("hyq_status_string", "hyq_version", "hyq_paper_k", "hyq_select_vertical_workspace",
            "hyq_select_vertical", "hyq_select_vertical_static", "hyq_select_vertical_mass_workspace",
            "hyq_select_vertical_mass", "hyq_quantize_blocks", "hyq_hybrid_attention_prefill_workspace",
-           "hyq_hybrid_attention_prefill")
+           "hyq_hybrid_attention_prefill", "hyq_test_set_attention_hooks")
 
 
 class HyqError(RuntimeError):
@@ -69,6 +69,7 @@ def lib() -> ctypes.CDLL:
                                           [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p])
         L.hyq_hybrid_attention_prefill_workspace.argtypes = [ctypes.POINTER(AttnArgs), ctypes.POINTER(ctypes.c_size_t)]
         L.hyq_hybrid_attention_prefill.argtypes = [ctypes.POINTER(AttnArgs), ctypes.c_void_p]
+        L.hyq_test_set_attention_hooks.argtypes = [ctypes.c_longlong, ctypes.c_int]
         _lib = L
     return _lib
 
@@ -162,6 +163,12 @@ def hyq_select_vertical_static(q: torch.Tensor, k: torch.Tensor, window: int, k_
     _check(lib().hyq_select_vertical_static(q.data_ptr(), k.data_ptr(), B, Hq, Hkv, Lq, Lk, D, window, n_tail, k_eff,
                                             out.data_ptr(), _stream()), "hyq_select_vertical_static")
     return out
+
+
+def hyq_test_set_attention_hooks(wait_limit_clocks: int = 0, drop_load_position: int = -1) -> None:
+    """Test hook: clock limit of a device-side barrier wait (0: default) and the walk position whose K/V copy the
+    tensor-core kernel's producer leaves out (-1: none).  Process-wide; reset with the defaults."""
+    _check(lib().hyq_test_set_attention_hooks(int(wait_limit_clocks), int(drop_load_position)), "hyq_test_set_attention_hooks")
 
 
 def code_row_bytes(fmt: int, D: int) -> int:

@@ -1,7 +1,7 @@
 // C-ABI entry points of the hyq library: argument checks on the host, then kernel launches.
 #include <cmath>
 
-#include "common.cuh"
+#include "attn_common.cuh"
 
 namespace hyq {
 size_t attn_simt_workspace_bytes(const hyq_attn_args& a);
@@ -11,6 +11,11 @@ int launch_attn_tc(const hyq_attn_args& a, float alpha, cudaStream_t st);
 namespace tcbt {
 int launch_attn_tc(const hyq_attn_args& a, float alpha, cudaStream_t st);     // 32- and 128-token quantization blocks
 }
+}  // namespace hyq
+
+namespace hyq {
+static TcTestHooks g_tc_hooks = {0, -1};
+TcTestHooks tc_test_hooks() { return g_tc_hooks; }
 }  // namespace hyq
 
 using namespace hyq;
@@ -31,6 +36,13 @@ const char* hyq_status_string(int status) {
 }
 
 int hyq_version(void) { return 2; }   // 2: decode side, column-mass selector, block sizes
+
+int hyq_test_set_attention_hooks(long long wait_limit_clocks, int drop_load_position) {
+    if (wait_limit_clocks < 0 || drop_load_position < -1) return HYQ_ERR_INVALID_ARG;
+    g_tc_hooks.wait_limit = wait_limit_clocks;
+    g_tc_hooks.drop_load = drop_load_position;
+    return HYQ_OK;
+}
 
 int hyq_paper_k(int Lk, int window, double ratio) {
     const long P = (Lk - window > 0) ? (long)Lk - window : 0;

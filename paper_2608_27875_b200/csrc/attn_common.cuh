@@ -19,7 +19,7 @@ struct TcWorkspace {
     size_t part_o;      // f32  [splits][B*Hq][Lq][D]   split keys only: partial accumulators ...
     size_t part_ml;     // f32  [splits][B*Hq][Lq][2]   ... and (reference maximum, row sum) per row
     size_t total;
-    int mask_words;
+    int mask_words;     // words per head, a multiple of 4 (one 16-byte group per 128-key tile)
     int splits;         // CTAs per pair of query tiles (1: the keys are not split)
 };
 
@@ -30,6 +30,14 @@ int tc_key_splits(const hyq_attn_args& a);
 
 TcWorkspace tc_workspace_layout(const hyq_attn_args& a);
 int launch_tc_prepass(const hyq_attn_args& a, const TcWorkspace& w, cudaStream_t st);
+
+// Test hooks of the tensor-core kernel (hyq_test_set_attention_hooks): the clock limit of a single barrier wait
+// (0: the default of about two seconds) and the walk position whose K/V load the producer leaves out (-1: none).
+struct TcTestHooks {
+    long long wait_limit;
+    int drop_load;
+};
+TcTestHooks tc_test_hooks();
 
 // zero-fills bits[n_heads][mask_words] and sets one bit per vertical-line key (memset + one kernel)
 int launch_vl_bitmask(const int32_t* idx, long n_heads, int k, int L, int mask_words, uint32_t* bits, cudaStream_t st);

@@ -15,6 +15,13 @@
 
 namespace hyq {
 
+// two floats -> fp16 pair, saturated to the largest finite fp16: a value row beyond the documented range
+// (|V| < 65504) then degrades the result instead of putting an infinity, and with it NaNs, into the output
+__device__ __forceinline__ uint32_t f16x2_sat(float a, float b) {
+    const __half2 h2 = __floats2half2_rn(fminf(fmaxf(a, -65504.0f), 65504.0f), fminf(fmaxf(b, -65504.0f), 65504.0f));
+    return *reinterpret_cast<const uint32_t*>(&h2);
+}
+
 __global__ void vl_bitmask_kernel(const int32_t* __restrict__ idx, long n_heads, int k, int L, int mask_words,
                                   uint32_t* __restrict__ bits) {
     const long e = (long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -39,11 +46,9 @@ __global__ void gather_vl_kernel(const __nv_bfloat16* __restrict__ kmat, const _
     const uint2 kw = *reinterpret_cast<const uint2*>(kmat + src);
     const uint2 vw = *reinterpret_cast<const uint2*>(vmat + src);
     *reinterpret_cast<uint2*>(kvl + row * HYQ_D + lane * 4) = kw;
-    const __half2 v01 = __floats2half2_rn(bf16_lo(vw.x), bf16_hi(vw.x));
-    const __half2 v23 = __floats2half2_rn(bf16_lo(vw.y), bf16_hi(vw.y));
     uint2 o;
-    o.x = *reinterpret_cast<const uint32_t*>(&v01);
-    o.y = *reinterpret_cast<const uint32_t*>(&v23);
+    o.x = f16x2_sat(bf16_lo(vw.x), bf16_hi(vw.x));
+    o.y = f16x2_sat(bf16_lo(vw.y), bf16_hi(vw.y));
     *reinterpret_cast<uint2*>(vvl + row * HYQ_D + lane * 4) = o;
 }
 
@@ -62,10 +67,7 @@ __global__ void v_to_fp16_kernel(const uint4* __restrict__ v, const uint2* __res
     const uint32_t ws[4] = {w.x, w.y, w.z, w.w};
     uint32_t o[4], oh[4];
 #pragma unroll
-    for (int c = 0; c < 4; ++c) {
-        const __half2 h2 = __floats2half2_rn(bf16_lo(ws[c]), bf16_hi(ws[c]));
-        o[c] = *reinterpret_cast<const uint32_t*>(&h2);
-    }
+    for (int c = 0; c < 4; ++c) o[c] = f16x2_sat(bf16_lo(ws[c]), bf16_hi(ws[c]));
     const uint2 cw = __ldg(v_codes + e);
     const uint32_t cs[2] = {cw.x, cw.y};
 #pragma unroll
@@ -81,8 +83,7 @@ __global__ void v_to_fp16_kernel(const uint4* __restrict__ v, const uint2* __res
             f0 = ff.x;
             f1 = ff.y;
         }
-        const __half2 h2 = __floats2half2_rn(f0 * sc, f1 * sc);
-        oh[c] = *reinterpret_cast<const uint32_t*>(&h2);
+        oh[c] = f16x2_sat(f0 * sc, f1 * sc);
     }
     v16[e] = make_uint4(o[0], o[1], o[2], o[3]);
     vh16[e] = make_uint4(oh[0], oh[1], oh[2], oh[3]);
@@ -135,7 +136,7 @@ TcWorkspace tc_workspace_layout(const hyq_attn_args& a) {
     size_t off = 0;
     auto take = [&](size_t bytes) { const size_t o = off; off += align_up(bytes, 1024); return o; };
     const size_t kv_elems = (size_t)a.B * a.Hkv * a.L * HYQ_D, q_elems = (size_t)a.B * a.Hq * query_rows(a) * HYQ_D;
-    w.mask_words = (a.L + 31) / 32;
+    w.mask_words = (a.L + 127) / 128 * 4;
     w.vl_bits = take((size_t)a.B * a.Hq * w.mask_words * 4);
     w.v16 = take(kv_elems * 2);
     w.vh16 = take(kv_elems * 2);

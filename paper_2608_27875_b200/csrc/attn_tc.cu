@@ -22,8 +22,7 @@
 // threads.  The exponentials are taken against that reference, which is only raised when
 // a tile exceeds it by more than 2^14 (the rescale of O is then rare); integer scores become floats
 // by a magic-number add.  Every mbarrier wait is bounded; when one expires the CTA records
-// HYQ_ERR_TIMEOUT in the status word and unwinds.  (Compiled with HYQ_OTPR = 0 the file gives the
-// earlier layout of 640 threads with two threads per row and a pairwise vote per tile.)
+// HYQ_ERR_TIMEOUT in the status word, waits (bounded) for its own copies and MMAs in flight and unwinds.
 #include <cuda_fp16.h>
 
 #include <type_traits>
@@ -35,17 +34,11 @@
 // through attn_tc_bt.cu with HYQ_TC_VARIANT_BT = 1, a second time into namespace hyq::tcbt with the block size a
 // run-time parameter (32 or 128 tokens).  The kernel's loop is sensitive to every live register - compiling the
 // parameter in, even behind a compile-time-false branch, cost the 64-token path 5 % - so the default translation
-// unit is kept token for token what it was.
+// unit carries nothing of it.  With 32-token blocks the two column halves of a tile have separate K scales: the
+// softmax thread then applies each half's own factor.
 #ifndef HYQ_TC_VARIANT_BT
 #define HYQ_TC_VARIANT_BT 0
 #endif
-// One softmax thread per query row (four warps per query tile, 64 columns per thread, no pairwise vote).  In the run-time
-// block-size variant the two column halves of a tile can have separate K scales (32-token blocks): the thread then
-// applies each half's own factor.  HYQ_OTPR = 0 selects the earlier layout with two threads per row.
-#ifndef HYQ_OTPR
-#define HYQ_OTPR 1
-#endif
-
 namespace hyq {
 #if HYQ_TC_VARIANT_BT
 namespace tcbt {
@@ -54,7 +47,7 @@ using namespace sm100;
 
 constexpr int BM = 128, QT = 2;
 constexpr int RING_BYTES = 65536;                   // shared memory of the K ring and of the V ring
-constexpr long long WAIT_LIMIT = 4000000000LL;      // SM clocks (~2 s): far beyond any legitimate wait
+constexpr long long WAIT_LIMIT_DEFAULT = 4000000000LL;   // SM clocks (~2 s): far beyond any legitimate wait
 
 constexpr uint32_t Q_TILE_BYTES = BM * HYQ_D * 2, QC_TILE_BYTES = BM * HYQ_D;        // 32768, 16384
 constexpr uint32_t SQ_OFF = 0, SQC_OFF = QT * Q_TILE_BYTES, SK_OFF = SQC_OFF + QT * QC_TILE_BYTES;
@@ -83,21 +76,6 @@ constexpr float INT_MAGIC_F = 12582912.0f;
 constexpr uint32_t KNOCKOUT_F32 = 0xFF800000u;       // -inf
 constexpr uint32_t KNOCKOUT_S32 = KNOCKOUT_F32 - INT_MAGIC;   // becomes -inf after the magic add
 
-// Optional timeline trace for tuning (compiled in with -DHYQ_TRACE): SM clock stamps of one CTA's softmax warps
-// (slots 0-3: query tile, column half) and MMA issuers (slots 4, 5) for own tiles 100..163, read back by
-// hyq_debug_read_trace.
-#if defined(HYQ_TRACE) && !HYQ_TC_VARIANT_BT
-__device__ long long g_trace[6 * 64 * 8];
-#define HYQ_TR(slot, n, e)                                                                                  \
-    do {                                                                                                    \
-        if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && (threadIdx.x & 31) == 0 && (n) >= 100 && \
-            (n) < 164)                                                                                      \
-            g_trace[((slot) * 64 + ((n) - 100)) * 8 + (e)] = clock64();                                     \
-    } while (0)
-#else
-#define HYQ_TR(slot, n, e) do { } while (0)
-#endif
-
 struct TcMaps {
     CUtensorMap q, k, qc, kc, v16, vh16, kvl, vvl;
 };
@@ -121,11 +99,13 @@ struct TcParams {
     void* out;
     float* lse;
     int32_t* status;
+    long long wait_limit;        // SM clocks a single barrier wait may take
+    int drop_load;               // test hook: walk position whose K/V load the producer announces but never issues (-1: none)
 };
 
 struct TcBarriers {
     uint64_t q_full, kv_full[MAX_STAGES], kv_free[MAX_STAGES];   // ring stage = K tile and V tile of one walk position
-    uint64_t s_full[QT][2], p_full[QT][2], o_done[QT][2];
+    uint64_t s_full[QT][2], p_full[QT][2], o_done[QT][2], drain[QT];
 };
 
 // which key tiles a 128-row query tile visits in each pass (i0, i1: first and last row of the tile in the query
@@ -179,7 +159,7 @@ __device__ __forceinline__ OwnTiles own_tiles(const QSched& s, const Walk& w) {
 // The loop body is kept to waits, MMAs and commits: ring positions, parities and descriptors advance incrementally.
 template <bool LOWBIT_FP8, int TBN>
 __device__ __forceinline__ bool mma_issuer(int q, const QSched& sq, const Walk& w, TcBarriers& bars, unsigned char* smem,
-                                           uint32_t tmem, volatile int* abort_flag) {
+                                           uint32_t tmem, volatile int* abort_flag, long long limit) {
     using G = Geo<TBN>;
     constexpr int BN = TBN, NST = G::NST, NBUF = G::NBUF;
     constexpr uint32_t STAGE16 = G::STAGE_BYTES >> 4;                  // descriptor address units per ring stage
@@ -194,7 +174,7 @@ __device__ __forceinline__ bool mma_issuer(int q, const QSched& sq, const Walk& 
     const uint32_t ts0 = tmem + tm_s(q), to = tmem + tm_o(q);
     const OwnTiles own = own_tiles(sq, w);
     const int nA = w.nA;
-    if (!mbar_wait(&bars.q_full, 0, WAIT_LIMIT)) return false;
+    if (!mbar_wait(&bars.q_full, 0, limit)) return false;
 
     // Q.K^T cursor
     int tq = w.t0, kst = 0;
@@ -202,9 +182,8 @@ __device__ __forceinline__ bool mma_issuer(int q, const QSched& sq, const Walk& 
     const int T1 = w.t1;
     // (k_ready: the stage of position tq is already known to have landed)
     auto qk = [&](bool k_ready) -> bool {
-        if (!k_ready && !mbar_wait(&bars.kv_full[kst], kpar, WAIT_LIMIT)) return false;
+        if (!k_ready && !mbar_wait(&bars.kv_full[kst], kpar, limit)) return false;
         if (own.has(tq)) {
-            HYQ_TR(4 + q, (int)n_qk, 0);
             tc_fence_after();
             const uint64_t dk = dk0 + (uint64_t)(kst * STAGE16);
             const uint32_t buf = n_qk % NBUF;
@@ -222,7 +201,6 @@ __device__ __forceinline__ bool mma_issuer(int q, const QSched& sq, const Walk& 
                                 dk + ((kk >> 2) * (G::STAGE_BYTES / 32) + (kk & 3) * 2), idesc_qk, kk > 0);
             }
             umma_commit(&bars.s_full[q][buf]);
-            HYQ_TR(4 + q, (int)n_qk, 1);
             ++n_qk;
         }
         ++tq;
@@ -252,14 +230,14 @@ __device__ __forceinline__ bool mma_issuer(int q, const QSched& sq, const Walk& 
                 const uint32_t a_kf = a_bars + (uint32_t)offsetof(TcBarriers, kv_full) + ks * 8;
                 const uint32_t ppi = i < 2 ? pp : pp ^ 1u, kpi = i < 2 ? kpar : kpar ^ 1u;
                 const uint32_t done = mbar_test_wait2_a(a_p, ppi, a_kf, kpi);
-                if (!(done & 1u) && !mbar_wait_a(a_p, ppi, WAIT_LIMIT)) { ok = false; break; }
+                if (!(done & 1u) && !mbar_wait_a(a_p, ppi, limit)) { ok = false; break; }
                 tc_fence_after();
 #pragma unroll
                 for (int kk = 0; kk < BN / 16; ++kk)
                     umma_ts_f16(to, ts0 + bf * BN + kk * 8, dv0 + (uint64_t)(i * STAGE16 + kk * 128), idesc_pv, 1u);
                 umma_commit_a(a_bars + (uint32_t)offsetof(TcBarriers, o_done) + (q * 2 + bf) * 8);
                 umma_commit_a(a_bars + (uint32_t)offsetof(TcBarriers, kv_free) + i * 8);
-                if (!(done & 2u) && !mbar_wait_a(a_kf, kpi, WAIT_LIMIT)) { ok = false; break; }
+                if (!(done & 2u) && !mbar_wait_a(a_kf, kpi, limit)) { ok = false; break; }
                 tc_fence_after();
 #pragma unroll
                 for (int kk = 0; kk < 4; ++kk) {
@@ -277,22 +255,18 @@ __device__ __forceinline__ bool mma_issuer(int q, const QSched& sq, const Walk& 
         bool k_ready = false;
         if (own.has(t)) {
             const uint32_t buf = n_pv % NBUF;
-            HYQ_TR(4 + q, (int)n_pv, 4);
             // P of this tile, and in the same round trip the ring stage of the Q.K^T that follows
             const uint32_t done = mbar_test_wait2(&bars.p_full[q][buf], (n_pv / NBUF) & 1u, &bars.kv_full[kst], kpar);
             k_ready = (done & 2u) != 0u && tq < T1;
-            if (!(done & 1u) && !mbar_wait(&bars.p_full[q][buf], (n_pv / NBUF) & 1u, WAIT_LIMIT)) return false;
-            HYQ_TR(4 + q, (int)n_pv, 5);
+            if (!(done & 1u) && !mbar_wait(&bars.p_full[q][buf], (n_pv / NBUF) & 1u, limit)) return false;
             tc_fence_after();
             const uint64_t dv = dv0 + (uint64_t)(vst * STAGE16);
             const uint32_t pa = ts0 + buf * BN;
 #pragma unroll
             for (int kk = 0; kk < BN / 16; ++kk) umma_ts_f16(to, pa + kk * 8, dv + kk * 128, idesc_pv, (n_pv > 0 || kk > 0));
             umma_commit(&bars.o_done[q][n_pv & 1u]);  // P.V number n of this query tile -> barrier n & 1
-            HYQ_TR(4 + q, (int)n_pv, 6);
             ++n_pv;
             umma_commit(&bars.kv_free[vst]);        // one arrival per issuer; the ring stage is free after both
-            HYQ_TR(4 + q, (int)n_pv - 1, 7);
         } else {
             mbar_arrive(&bars.kv_free[vst]);        // nothing of this query tile reads the stage
         }
@@ -306,7 +280,8 @@ __device__ __forceinline__ bool mma_issuer(int q, const QSched& sq, const Walk& 
 // TMA producer (one thread): the two query tiles once, then the K ring and the V ring along the CTA's walk
 template <int TBN>
 __device__ __forceinline__ bool tma_producer(const TcMaps& maps, const QSched& qs0, const QSched& qs1, const Walk& w, int qhead,
-                                             int kvhead, TcBarriers& bars, unsigned char* smem, volatile int* abort_flag) {
+                                             int kvhead, TcBarriers& bars, unsigned char* smem, volatile int* abort_flag,
+                                             long long limit, int drop_load) {
     using G = Geo<TBN>;
     constexpr int BN = TBN, NST = G::NST;
     prefetch_tmap(&maps.q);
@@ -324,20 +299,24 @@ __device__ __forceinline__ bool tma_producer(const TcMaps& maps, const QSched& q
         tma_load_3d(smem + SQ_OFF + q * Q_TILE_BYTES + Q_TILE_BYTES / 2, &maps.q, &bars.q_full, 64, qi0[q], qhead);
         if (w.nA > 0) tma_load_3d(smem + SQC_OFF + q * QC_TILE_BYTES, &maps.qc, &bars.q_full, 0, qi0[q], qhead);
     }
-    for (int t = w.t0; t < w.t1 && !*abort_flag; ++t) {
+    bool ok = true;
+    int t = w.t0;
+    for (; t < w.t1 && !*abort_flag; ++t) {
         const int st = (t - w.t0) % NST, use = (t - w.t0) / NST;
         unsigned char* sk = smem + SK_OFF + st * G::STAGE_BYTES;
         unsigned char* sv = smem + SV_OFF + st * G::STAGE_BYTES;
         const bool lowbit = t < w.nA, vl = !lowbit && t < w.nA + w.nB;
         const int row = lowbit ? t * BN : (vl ? (t - w.nA) * BN : (w.tC0 + t - w.nA - w.nB) * BN);
         const int hd = vl ? qhead : kvhead;
-        if (use > 0 && !mbar_wait_sleepy(&bars.kv_free[st], (use - 1) & 1, WAIT_LIMIT)) return false;
+        if (use > 0 && !mbar_wait_sleepy(&bars.kv_free[st], (use - 1) & 1, limit)) { ok = false; break; }
         if (lowbit) {
             mbar_arrive_expect_tx(&bars.kv_full[st], G::KC_TILE_BYTES + G::STAGE_BYTES);
+            if (t == drop_load) continue;                // test hook: the announced bytes never arrive
             tma_load_3d(sk, &maps.kc, &bars.kv_full[st], 0, row, hd);
         } else {
             const CUtensorMap* m = vl ? &maps.kvl : &maps.k;
             mbar_arrive_expect_tx(&bars.kv_full[st], 2 * G::STAGE_BYTES);
+            if (t == drop_load) continue;
             tma_load_3d(sk, m, &bars.kv_full[st], 0, row, hd);
             tma_load_3d(sk + G::STAGE_BYTES / 2, m, &bars.kv_full[st], 64, row, hd);
         }
@@ -345,35 +324,20 @@ __device__ __forceinline__ bool tma_producer(const TcMaps& maps, const QSched& q
         tma_load_3d(sv, m, &bars.kv_full[st], 0, row, hd);
         tma_load_3d(sv + G::STAGE_BYTES / 2, m, &bars.kv_full[st], 64, row, hd);
     }
-    return true;
+    if (!ok || *abort_flag) {
+        // leaving early: wait (bounded) for the copies still on their way into this CTA's shared memory
+        mbar_wait_sleepy(&bars.q_full, 0, limit);
+        for (int u = max(t - w.t0 - NST, 0); u < t - w.t0; ++u) mbar_wait_sleepy(&bars.kv_full[u % NST], (u / NST) & 1, limit);
+    }
+    return ok;
 }
 
 // ---- softmax warps -------------------------------------------------------------------------------
-// One thread per query row (HYQ_OTPR): the thread reads its 64 scores of a tile in two register halves, raises the
-// row's reference when the tile's maximum exceeds it by more than the threshold (rescaling O and the row sum), and
-// writes the 64 probabilities as fp16 pairs over the first 32 columns of the buffer it read.
-// Two threads per query row (HYQ_OTPR = 0, the earlier layout):
-// the two threads of a row must exponentiate against the same reference maximum.  Per tile they take the maximum
-// of their own 32 columns, and the two warps that share 32 query rows vote (named barrier of 64 threads with OR
-// reduction) whether any of these rows has to raise its reference.  In the common case none does and each half
-// proceeds on its own; otherwise every thread also reads the other half's scores from TMEM, so both threads of a
-// row arrive at the same new reference, rescale their half of O (64 channels each) and their partial row sum.
-// The vote also orders "both halves have read S" before "either half writes P over it".  The partial sums are
-// added at the end (exchange through TMEM).
-constexpr int TC_THREADS = HYQ_OTPR ? 384 : 640;   // TMA producer, 2 MMA issuers, 1 idle warp, 8 (16) softmax warps
+// One thread per query row: the thread reads its 64 scores of a tile in two register halves, raises the row's
+// reference when the tile's maximum exceeds it by more than the threshold (rescaling O and the row sum), and writes the
+// 64 probabilities as fp16 pairs over the first 32 columns of the buffer it read.
+constexpr int TC_THREADS = 384;                     // TMA producer, 2 MMA issuers, 1 idle warp, 8 softmax warps
 constexpr float RAISE_THRESHOLD = 14.0f;            // log2 units by which a tile must exceed the reference to raise it (P stays below 2^14, inside fp16)
-
-// named barrier over `nthreads` threads with an OR reduction of `pred` (all threads of the participating warps call it)
-__device__ __forceinline__ bool bar_red_or(int id, int nthreads, bool pred) {
-    uint32_t out;
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 p, %3, 0;\n\tbar.red.or.pred q, %1, %2, p;\n\tselp.u32 %0, 1, 0, q;\n\t}\n"
-        : "=r"(out) : "r"(id), "r"(nthreads), "r"((uint32_t)pred) : "memory");
-    return out != 0;
-}
-__device__ __forceinline__ void bar_sync_named(int id, int nthreads) {
-    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
-}
 
 // row maximum of 32 float scores held in registers
 __device__ __forceinline__ float fmax3(float a, float b, float c) {
@@ -466,6 +430,7 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
     const int h = blockIdx.y, b = blockIdx.z;
     const int L = p.Lq, W = p.window, g = p.Hq / p.Hkv;     // L: rows of the query block
     const int off = QUERY_BLOCK ? p.L - p.Lq : 0;           // position of query row 0 among the keys
+    const long long limit = p.wait_limit;
     // Last low-bit-eligible key position of the row at position x: x - W with the per-row sliding window,
     // min(x, L_K - W - 1) with the fixed tail window (both as min(x, lim) - wsub).  Its window keys start right
     // after it, and the vertical keys it may use are those at or below it.
@@ -484,9 +449,10 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
         for (int q = 0; q < QT; ++q) {
             for (int bf = 0; bf < 2; ++bf) {
                 mbar_init(&bars.s_full[q][bf], 1);
-                mbar_init(&bars.p_full[q][bf], HYQ_OTPR ? 4 : 8);           // one arrival per softmax warp of the query tile
+                mbar_init(&bars.p_full[q][bf], 4);                  // one arrival per softmax warp of the query tile
                 mbar_init(&bars.o_done[q][bf], 1);
             }
+            mbar_init(&bars.drain[q], 1);
         }
         fence_mbar_init();
         abort_s = 0;
@@ -534,22 +500,22 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
 
     // the single-thread roles sit in the lowest warps (the softmax warps 4..19 keep warp % 4 = TMEM lane quarter)
     if (warp == 0) {
-        if (lane == 0 && !tma_producer<TBN>(maps, qs0, qs1, w, qhead, kvhead, bars, smem, abort_flag)) fail();
+        if (lane == 0 && !tma_producer<TBN>(maps, qs0, qs1, w, qhead, kvhead, bars, smem, abort_flag, limit, p.drop_load)) fail();
     } else if (warp == 1 || warp == 2) {
         if (lane == 0) {
             const int q = warp - 1;
-            if (!mma_issuer<LOWBIT_FP8, TBN>(q, q ? qs1 : qs0, w, bars, smem, tmem, abort_flag)) fail();
+            const bool ok = mma_issuer<LOWBIT_FP8, TBN>(q, q ? qs1 : qs0, w, bars, smem, tmem, abort_flag, limit);
+            if (!ok || *abort_flag) {
+                // leaving early: none of this thread's MMAs may be in flight when the CTA gives up its tensor memory
+                umma_commit(&bars.drain[q]);
+                mbar_wait(&bars.drain[q], 0, limit);
+            }
+            if (!ok) fail();
         }
     } else if (warp >= 4) {
         // ------------------------------------------------------------------ softmax warps
-#if HYQ_OTPR
-        const int q = (warp - 4) >> 2, hsel = 0;                        // query tile (a thread owns all 64 columns of its row)
-#else
-        const int q = (warp - 4) >> 3, hsel = ((warp - 4) >> 2) & 1;    // query tile, column half
-#endif
+        const int q = (warp - 4) >> 2;                          // query tile (a thread owns all 64 columns of its row)
         const QSched sq = q ? qs1 : qs0;
-        // named barrier of the two warps that share this warp's 32 query rows (one per query tile and lane quarter)
-        const int bar_id = 1 + q * 4 + (warp & 3);
         const OwnTiles own = own_tiles(sq, w);
         // own tiles of this CTA: numbers [n0, n_total) in the query tile's own list (all of it unless the keys are split)
         const int n0 = SPLIT ? own_before(own, w.t0) : 0;
@@ -557,7 +523,7 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
         if (SPLIT && sq.live && n_total <= n0) {
             // nothing of this query tile lies in the slice: an empty partial result
             const int i = sq.i0 + (warp & 3) * 32 + lane;
-            if (hsel == 0 && i < L)
+            if (i < L)
                 reinterpret_cast<float2*>(p.part_ml)[((long)split * gridDim.y * gridDim.z + qhead) * L + i] = make_float2(-INFINITY, 0.0f);
         }
         if (sq.live && n_total > n0) {
@@ -566,7 +532,6 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
             const int ia = i + off;                             // ... and its position among the keys
             const bool row_live = i < L;
             const bool ragged = sq.i0 + BM > L;
-            const int col0 = hsel * 32, col0_other = col0 ^ 32;
             const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
             const uint32_t to = tmem + tm_o(q) + lane_addr, ts0 = tmem + tm_s(q) + lane_addr;
 #if HYQ_TC_VARIANT_BT
@@ -590,44 +555,33 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
             // (tile n of the low-bit pass sits at walk position n; its block and mask words exist for n < a_end)
 #if HYQ_TC_VARIANT_BT
             // a 64-key tile n lies in block n / 2 (128-token blocks) or in blocks 2n and 2n + 1, one per column half (32)
-            const float* ks_ptr = p.k_scales + (long)kvhead * p.nb + (bsh == 5 ? hsel : 0);
+            const float* ks_ptr = p.k_scales + (long)kvhead * p.nb;
 #else
             const float* ks_ptr = p.k_scales + (long)kvhead * p.nb;
 #endif
-            const uint32_t* vl_ptr = p.vl_bits + (long)qhead * p.mask_words + hsel;
+            const uint32_t* vl_ptr = p.vl_bits + (long)qhead * p.mask_words;
             float nks = 0.0f;
-#if HYQ_TC_VARIANT_BT && HYQ_OTPR
+#if HYQ_TC_VARIANT_BT
             float nks_b = 0.0f, cs_hi = 0.0f;                   // K scale and score factor of columns 32-63 (32-token blocks: their own block)
 #endif
-#if HYQ_OTPR
             uint64_t nvl = 0u;                                  // both mask words of the tile (columns 0-31 low, 32-63 high)
-#else
-            uint32_t nvl = 0u;
-#endif
             auto prefetch_tile = [&](int n) {
                 nks = 0.0f; nvl = 0u;
-#if HYQ_TC_VARIANT_BT && HYQ_OTPR
+#if HYQ_TC_VARIANT_BT
                 nks_b = 0.0f;
 #endif
                 if (n >= own.a_end) return;
 #if HYQ_TC_VARIANT_BT
                 nks = __ldg(ks_ptr + ((n << 6) >> bsh));
-#if HYQ_OTPR
                 nks_b = (bsh == 5) ? __ldg(ks_ptr + 2 * n + 1) : nks;
-#endif
 #else
                 nks = __ldg(ks_ptr + n);
 #endif
-#if HYQ_OTPR
                 nvl = (uint64_t)__ldg(vl_ptr + 2 * n) | ((uint64_t)__ldg(vl_ptr + 2 * n + 1) << 32);
-#else
-                nvl = __ldg(vl_ptr + 2 * n);
-#endif
             };
             prefetch_tile(n0);
             const float qs2 = q_scale * p.scale_log2;
 
-#if HYQ_OTPR
             // one tile of the online softmax for this thread's row: all 64 columns, in two register halves.  Returns
             // false when this warp ran into an expired wait.
             auto do_tile = [&](auto range_tag, int n, float cs, uint64_t vl, bool int_scores, int lo_eff, unsigned span) -> bool {
@@ -636,12 +590,10 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                 const int nl = n - n0;                          // tile number within this CTA's slice
                 const int buf = nl & 1;
                 const uint32_t ts = ts0 + buf * BN;
-                HYQ_TR(q * 2, n, 0);
-                if (!__all_sync(0xffffffffu, mbar_wait(&bars.s_full[q][buf], (uint32_t)(nl >> 1) & 1u, WAIT_LIMIT))) {
+                if (!__all_sync(0xffffffffu, mbar_wait(&bars.s_full[q][buf], (uint32_t)(nl >> 1) & 1u, limit))) {
                     dead = true;
                     return false;
                 }
-                HYQ_TR(q * 2, n, 1);
                 tc_fence_after();
                 // vertical-line keys of a low-bit tile: -inf into their S columns before the row is read
                 if (vl != 0ull) {                                // uniform over the warp
@@ -652,7 +604,6 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                 tmem_ld32(ts, ra);
                 tmem_ld32(ts + 32, rb);
                 tmem_wait_ld();
-                HYQ_TR(q * 2, n, 3);
                 if (NEED_RANGE) {
                     mask_cols32(ra, 0, lo_eff, span, knock);
                     mask_cols32(rb, 32, lo_eff, span, knock);
@@ -672,14 +623,13 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                 const float mt = (f == -INFINITY) ? -INFINITY : f * cs;
 #endif
                 const bool raise = mt > m_used + RAISE_THRESHOLD;
-                HYQ_TR(q * 2, n, 4);
                 if (__any_sync(0xffffffffu, raise)) {
                     const float alpha = raise ? ex2f(m_used - mt) : 1.0f;      // m_used = -inf -> 0
                     if (nl > 0) {
                         // P.V of tile n-1 must have landed before O is rescaled.  P.V number m signals barrier m & 1;
                         // the one before the previous is complete (the scores just read were issued after it), so
                         // the parity wait cannot alias.
-                        if (!__all_sync(0xffffffffu, mbar_wait(&bars.o_done[q][(nl - 1) & 1], (uint32_t)((nl - 1) >> 1) & 1u, WAIT_LIMIT))) {
+                        if (!__all_sync(0xffffffffu, mbar_wait(&bars.o_done[q][(nl - 1) & 1], (uint32_t)((nl - 1) >> 1) & 1u, limit))) {
                             dead = true;
                             return false;
                         }
@@ -711,139 +661,21 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
 #else
                 l_h += row_exp32(rb, cs, bias, pb);
 #endif
-                HYQ_TR(q * 2, n, 5);
                 tmem_st16(ts + 16, pb);
                 tmem_wait_st();
                 tc_fence_before();
                 __syncwarp();
-                HYQ_TR(q * 2, n, 6);
                 if (lane == 0) mbar_arrive(&bars.p_full[q][buf]);
-                HYQ_TR(q * 2, n, 7);
                 return true;
             };
-#else
-            // one tile of the online softmax for this thread's 32 columns.  Returns false when the query tile's
-            // softmax warps leave the loop together (an expired wait somewhere).
-            auto do_tile = [&](auto range_tag, int n, float cs, uint32_t vl, bool int_scores, int lo_eff, unsigned span) -> bool {
-                constexpr bool NEED_RANGE = decltype(range_tag)::value;
-                const uint32_t knock = int_scores ? KNOCKOUT_S32 : KNOCKOUT_F32;
-                const int nl = n - n0;                          // tile number within this CTA's slice
-                const int buf = nl & 1;
-                const uint32_t ts = ts0 + buf * BN;
-                uint32_t raw[32];
-                float mt = -INFINITY;
-                HYQ_TR(q * 2 + hsel, n, 0);
-                if (!dead && !__all_sync(0xffffffffu, mbar_wait(&bars.s_full[q][buf], (uint32_t)(nl >> 1) & 1u, WAIT_LIMIT))) {
-                    dead = true;
-                }
-                __syncwarp();
-                HYQ_TR(q * 2 + hsel, n, 1);
-                if (!dead) {
-                    tc_fence_after();
-                    // vertical-line keys of a low-bit tile: -inf into their S columns before the half is read
-                    if (vl != 0u) {                              // uniform over the warp
-                        while (vl) { const int c = __ffs(vl) - 1; vl &= vl - 1; tmem_st1(ts + col0 + c, knock_lq); }
-                        tmem_wait_st();
-                    }
-                    tmem_ld32(ts + col0, raw);
-                    tmem_wait_ld();
-                    if (NEED_RANGE) mask_cols32(raw, col0, lo_eff, span, knock);
-                    // integer scores become the floats 2^23 + 2^22 + s by one integer add each (knocked-out entries
-                    // become -inf); the offset is taken out again by the bias of the exponent
-                    if (int_scores) {
-#pragma unroll
-                        for (int e = 0; e < 32; ++e) raw[e] += INT_MAGIC;
-                    }
-                    const float f = row_max32(raw) - (int_scores ? INT_MAGIC_F : 0.0f);
-                    mt = (f == -INFINITY) ? -INFINITY : f * cs;
-                }
-                // ---- vote of the two warps of these 32 rows: does any row have to raise its reference maximum?
-                // (also: both halves have read their scores before either writes P over them)
-                tc_fence_before();
-                HYQ_TR(q * 2 + hsel, n, 3);
-                const bool any_raise = bar_red_or(bar_id, 64, dead || mt > m_used + RAISE_THRESHOLD);
-                HYQ_TR(q * 2 + hsel, n, 4);
-                if (any_raise) {
-                    if (bar_red_or(bar_id, 64, dead)) return false;         // one of the two warps ran into an expired wait
-                    tc_fence_after();
-                    // the other half's maximum, from its scores in TMEM (same knock-outs, same range mask)
-                    float mo;
-                    {
-                        uint32_t oth[32];
-                        tmem_ld32(ts + col0_other, oth);
-                        tmem_wait_ld();
-                        if (NEED_RANGE) mask_cols32(oth, col0_other, lo_eff, span, knock);
-                        if (int_scores) {
-#pragma unroll
-                            for (int e = 0; e < 32; ++e) oth[e] += INT_MAGIC;
-                        }
-                        const float fo = row_max32(oth) - (int_scores ? INT_MAGIC_F : 0.0f);
-#if HYQ_TC_VARIANT_BT
-                        // 32-token blocks: the other column half of a low-bit tile has its own K scale
-                        float cs_other = cs;
-                        if (bsh == 5 && n < own.a_end) cs_other = fmaxf(qs2 * __ldg(ks_ptr + 2 * n + 1 - 2 * hsel), 1e-37f);
-                        mo = (fo == -INFINITY) ? -INFINITY : fo * cs_other;
-#else
-                        mo = (fo == -INFINITY) ? -INFINITY : fo * cs;
-#endif
-                    }
-                    tc_fence_before();
-                    bar_sync_named(bar_id, 64);                  // both halves are done reading before P is written
-                    const float m_new = fmaxf(mt, mo);
-                    const bool raise = m_new > m_used + RAISE_THRESHOLD;     // same verdict in both threads of the row
-                    const float alpha = raise ? ex2f(m_used - m_new) : 1.0f; // m_used = -inf -> 0
-                    if (nl > 0 && __any_sync(0xffffffffu, raise)) {
-                        // P.V of tile n-1 must have landed before O is rescaled.  P.V number m signals barrier m & 1;
-                        // the one before the previous is complete (the scores just read were issued after it), so
-                        // the parity wait cannot alias.
-                        if (!__all_sync(0xffffffffu, mbar_wait(&bars.o_done[q][(nl - 1) & 1], (uint32_t)((nl - 1) >> 1) & 1u, WAIT_LIMIT))) {
-                            dead = true;
-                        } else {
-                            tc_fence_after();
-#pragma unroll 1
-                            for (int c = 0; c < 4; ++c) {       // this half rescales channels [64 hsel, 64 hsel + 64)
-                                uint32_t o[16];
-                                tmem_ld16(to + hsel * 64 + c * 16, o);
-                                tmem_wait_ld();
-#pragma unroll
-                                for (int e = 0; e < 16; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-                                tmem_st16(to + hsel * 64 + c * 16, o);
-                            }
-                            tmem_wait_st();
-                        }
-                    }
-                    if (raise) {
-                        l_h *= alpha;
-                        m_used = m_new;
-                    }
-                }
-                // ---- P = 2^(s - m) as fp16 pairs over the first 32 columns of the buffer; row sum of this half
-                if (!dead) {
-                    const float m_eff = (m_used == -INFINITY) ? 0.0f : m_used;
-                    const float bias = int_scores ? fmaf(-INT_MAGIC_F, cs, -m_eff) : -m_eff;
-                    uint32_t pk[16];
-                    l_h += row_exp32(raw, cs, bias, pk);  // (integer scores were made floats above)
-                    HYQ_TR(q * 2 + hsel, n, 5);
-                    tmem_st16(ts + hsel * 16, pk);
-                    tmem_wait_st();
-                    tc_fence_before();
-                    __syncwarp();
-                    HYQ_TR(q * 2 + hsel, n, 6);
-                    if (lane == 0) mbar_arrive(&bars.p_full[q][buf]);
-                    HYQ_TR(q * 2 + hsel, n, 7);
-                }
-                return true;
-            };
-#endif
 
             // ---- low-bit tiles that lie wholly below every row's window: no range mask, no bounds to compute
             const int n_plain = ragged ? 0 : min(own.a_end, max(0, (qhi(sq.i0 + off) + 1) / BN));
             int n = n0;
             for (; n < min(n_plain, n_total); ++n) {
-                HYQ_TR(q * 2 + hsel, n, 2);
                 // a zero scale (all-zero tile) still has to let -inf pass through the multiply
                 const float cs = fmaxf(qs2 * nks, 1e-37f);
-#if HYQ_TC_VARIANT_BT && HYQ_OTPR
+#if HYQ_TC_VARIANT_BT
                 cs_hi = fmaxf(qs2 * nks_b, 1e-37f);
 #endif
                 const auto vl = nvl;
@@ -854,10 +686,9 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
             // (number of vertical-line keys this row may use: only needed from here on)
             const int cnt_r = (!aborted && sq.nB > 0 && row_live && qhi(ia) >= 0) ? count_le(idx_row, p.k, qhi(ia)) : 0;
             for (; n < n_total && !aborted; ++n) {
-                HYQ_TR(q * 2 + hsel, n, 2);
                 const int t = walk_pos(n);
                 const float ks = nks;
-#if HYQ_TC_VARIANT_BT && HYQ_OTPR
+#if HYQ_TC_VARIANT_BT
                 const float ks_b = nks_b;
 #endif
                 const auto vl = nvl;
@@ -877,7 +708,7 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                     hi = row_live ? min(ia - j0, BN - 1) : -1;
                     cs = p.scale_log2;
                 }
-#if HYQ_TC_VARIANT_BT && HYQ_OTPR
+#if HYQ_TC_VARIANT_BT
                 cs_hi = lowbit ? fmaxf(qs2 * ks_b, 1e-37f) : cs;
 #endif
                 const int lo_eff = (hi >= lo) ? lo : 4096;
@@ -893,23 +724,11 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
 
             // ---- epilogue: the last P.V (MMAs complete in order), sum of the two halves' row sums, O / l
             bool ok = !aborted && !dead;
-            if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars.o_done[q][(n_total - n0 - 1) & 1], (uint32_t)((n_total - n0 - 1) >> 1) & 1u, WAIT_LIMIT));
+            if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars.o_done[q][(n_total - n0 - 1) & 1], (uint32_t)((n_total - n0 - 1) >> 1) & 1u, limit));
             if (!aborted) {                                     // uniform over the query tile's softmax warps
                 tc_fence_after();
-#if HYQ_OTPR
                 constexpr int NCH = 4;                          // 32-channel pieces of the row this thread writes
                 const float l_run = l_h;
-#else
-                constexpr int NCH = 2;
-                tmem_st1(ts0 + col0, __float_as_uint(l_h));     // column col0 of S buffer 0 (all MMAs are done)
-                tmem_wait_st();
-                tc_fence_before();
-                bar_sync_named(bar_id, 64);
-                tc_fence_after();
-                const float l_o = __uint_as_float(tmem_ld1(ts0 + col0_other));
-                tmem_wait_ld();
-                const float l_run = l_h + l_o;
-#endif
                 const float inv = (l_run > 0.0f) ? 1.0f / l_run : 0.0f;
                 if (SPLIT) {
                     // partial result of this slice: O as accumulated (relative to m_used), the pair (m_used, l)
@@ -918,7 +737,7 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
 #pragma unroll
                         for (int c = 0; c < NCH; ++c) {
                             uint32_t o[32];
-                            const int ch = hsel * 64 + c * 32;
+                            const int ch = c * 32;
                             tmem_ld32(to + ch, o);
                             tmem_wait_ld();
                             if (row_live) {
@@ -927,13 +746,13 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                                 for (int e = 0; e < 8; ++e) dst[e] = make_uint4(o[4 * e], o[4 * e + 1], o[4 * e + 2], o[4 * e + 3]);
                             }
                         }
-                        if (row_live && hsel == 0) reinterpret_cast<float2*>(p.part_ml)[prow] = make_float2(m_used, l_run);
+                        if (row_live) reinterpret_cast<float2*>(p.part_ml)[prow] = make_float2(m_used, l_run);
                     }
                 } else if (ok) {
 #pragma unroll
-                    for (int c = 0; c < NCH; ++c) {            // this thread's channels: [64 hsel, 64 hsel + 32 NCH)
+                    for (int c = 0; c < NCH; ++c) {
                         uint32_t o[32];
-                        const int ch = hsel * 64 + c * 32;
+                        const int ch = c * 32;
                         tmem_ld32(to + ch, o);
                         tmem_wait_ld();
                         if (row_live) {
@@ -959,7 +778,7 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                             }
                         }
                     }
-                    if (p.lse && row_live && hsel == 0) p.lse[(long)qhead * L + i] = (m_used + log2f(l_run)) * 0.6931471805599453f;
+                    if (p.lse && row_live) p.lse[(long)qhead * L + i] = (m_used + log2f(l_run)) * 0.6931471805599453f;
                 }
             }
             if (!ok) fail();
@@ -1057,6 +876,9 @@ int launch_attn_tc(const hyq_attn_args& a, float alpha, cudaStream_t st) {
     p.q_scales = a.q_scales; p.k_scales = a.k_scales; p.vl_idx = a.vl_idx;
     p.vl_bits = reinterpret_cast<const uint32_t*>(base + w.vl_bits);
     p.out = a.out; p.lse = a.lse; p.status = a.status_word;
+    const TcTestHooks hooks = tc_test_hooks();
+    p.wait_limit = hooks.wait_limit > 0 ? hooks.wait_limit : WAIT_LIMIT_DEFAULT;
+    p.drop_load = hooks.drop_load;
 
     const bool blk = Lq < L || p.fixed_tail;      // the general instantiation (the other one is the whole prefill)
     // e4m3 bytes on the low-bit side: FP8 codes as they are, or INT4 codes widened by the pre-pass
@@ -1084,9 +906,3 @@ int launch_attn_tc(const hyq_attn_args& a, float alpha, cudaStream_t st) {
 }  // namespace tcbt
 #endif
 }  // namespace hyq
-
-#if defined(HYQ_TRACE) && !HYQ_TC_VARIANT_BT
-extern "C" int hyq_debug_read_trace(long long* dst) {
-    return cudaMemcpyFromSymbol(dst, hyq::g_trace, sizeof(hyq::g_trace)) == cudaSuccess ? 0 : 1;
-}
-#endif

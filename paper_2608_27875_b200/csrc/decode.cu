@@ -375,8 +375,9 @@ decode_kernel(const DecParams p) {
     long nQ = p.nQ;
     int n_vl = p.k, n_win = p.W, n_stg = p.n_s;
     if (p.lens) {                                           // ragged batch: this sequence's own row counts
+        // (clamped to the buffers' capacities: a bad length then shortens the walk instead of leaving the allocation)
         const int4 l = __ldg(p.lens + unit / p.Hkv);
-        nQ = l.x; n_vl = l.y; n_win = l.z; n_stg = l.w;
+        nQ = min(max((long)l.x, 0L), p.sQ); n_vl = min(max(l.y, 0), p.sK); n_win = min(max(l.z, 0), p.sW); n_stg = min(max(l.w, 0), p.Ws);
     }
     const long Tq = (nQ + 15) / 16;
     const int Tvl = (n_vl + 15) / 16, Ts = (n_stg + 15) / 16, Tw = (n_win + 15) / 16;

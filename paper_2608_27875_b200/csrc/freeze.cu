@@ -39,7 +39,8 @@ gather_rows_kernel(const uint4* __restrict__ k_, const uint4* __restrict__ v, co
     if (o >= k_vl + W) return;
     const int P = N - W;
     const bool vl = o < k_vl;
-    const int src = vl ? __ldg(idx + head * k_vl + o) : P + (o - k_vl);
+    // (a vertical index outside [0, N) is clamped: it then names a wrong row instead of memory outside the tensor)
+    const int src = vl ? min(max(__ldg(idx + head * k_vl + o), 0), N - 1) : P + (o - k_vl);
     const long s = (head * N + src) * 16 + c;
     const long d = vl ? (head * sK + o) * 16 + c : (head * sW + (o - k_vl)) * 16 + c;
     (vl ? k_vl_out : k_win)[d] = __ldg(k_ + s);
@@ -98,6 +99,7 @@ freeze_quantize_kernel(const uint4* __restrict__ k_, const uint4* __restrict__ v
                 if (win[mid] == 0x7fffffff || win[mid] - (j0 + mid) > p) hi = mid; else lo = mid + 1;
             }
             s = lo < FRZ_WIN ? p + j0 + lo : source_row(hidx, k_vl, p);
+            s = min(s, N - 1);                              // (only a malformed index list can reach the clamp)
         }
         src[threadIdx.x] = s;
     }

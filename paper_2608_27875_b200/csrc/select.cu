@@ -2,7 +2,7 @@
 // scores over the non-window prefix -> exact top-k per query head.
 //
 // Three kernels, all bound by memory traffic:
-//   tail_mean_kernel   qbar[b,h,:] = (1/t) sum of the last t query rows, fp64
+//   tail_mean_kernel   qbar[b,h,:] = (1/t) sum of the last t query rows, fp64, added in row order
 //   vscore_kernel      S[b,h,p] = qbar[b,h,:] . K[b,h/g,p,:], an fp64 fma chain in channel
 //                      order; each K row is read once per KV head and scored for its g query heads
 //   topk_kernel        per (b,h): MSB-first radix select of the k-th largest score on an
@@ -16,33 +16,31 @@
 
 namespace hyq {
 
-constexpr int MEAN_GROUPS = 8;       // row groups summed independently, combined in fixed order
 constexpr int SCORE_KEYS = 128;      // keys per CTA in vscore_kernel
 constexpr int SCORE_GC = 4;          // query heads scored per pass over the staged K tile
 constexpr int TOPK_THREADS = 1024;
 
 // -------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(HYQ_D * MEAN_GROUPS)
+// One thread per (b, h, channel) adds the t tail rows in ascending row order in fp64 - the order of Algorithm 1's
+// mean as it is written down, so the result is the same double for every finite input, whatever the spread of the
+// exponents (a split into partial sums would only agree while every partial sum is exact).  The loads of 16 rows
+// are issued together; only the additions form a chain.
+__global__ void __launch_bounds__(HYQ_D)
 tail_mean_kernel(const __nv_bfloat16* __restrict__ q, int Lq, int t, double* __restrict__ qbar) {
     const long bh = blockIdx.x;
-    const int d = threadIdx.x % HYQ_D, grp = threadIdx.x / HYQ_D;
+    const int d = threadIdx.x;
     const __nv_bfloat16* base = q + (bh * Lq + (Lq - t)) * (long)HYQ_D + d;
-    // rows are split into MEAN_GROUPS contiguous ranges; every partial sum and their combination
-    // are exact in fp64 for bf16 inputs of bounded exponent spread, so the order does not matter
-    const int per = (t + MEAN_GROUPS - 1) / MEAN_GROUPS;
-    const int r0 = grp * per, r1 = min(t, r0 + per);
     double s = 0.0;
-#pragma unroll 8
-    for (int r = r0; r < r1; ++r) s += (double)__bfloat162float(base[(long)r * HYQ_D]);
-    __shared__ double part[MEAN_GROUPS][HYQ_D];
-    part[grp][d] = s;
-    __syncthreads();
-    if (grp == 0) {
-        double tot = 0.0;
+    int r = 0;
+    for (; r + 16 <= t; r += 16) {
+        float v[16];
 #pragma unroll
-        for (int gi = 0; gi < MEAN_GROUPS; ++gi) tot += part[gi][d];
-        qbar[bh * HYQ_D + d] = tot / (double)t;
+        for (int j = 0; j < 16; ++j) v[j] = __bfloat162float(base[(long)(r + j) * HYQ_D]);
+#pragma unroll
+        for (int j = 0; j < 16; ++j) s += (double)v[j];
     }
+    for (; r < t; ++r) s += (double)__bfloat162float(base[(long)r * HYQ_D]);
+    qbar[bh * HYQ_D + d] = s / (double)t;
 }
 
 // -------------------------------------------------------------------------------------------
@@ -212,7 +210,7 @@ int launch_select(const void* q, const void* k, int B, int Hq, int Hkv, int Lq, 
     double* qbar = static_cast<double*>(ws);
     double* scores = reinterpret_cast<double*>(static_cast<char*>(ws) + align_up((size_t)B * Hq * HYQ_D * sizeof(double), 256));
 
-    tail_mean_kernel<<<B * Hq, HYQ_D * MEAN_GROUPS, 0, st>>>(static_cast<const __nv_bfloat16*>(q), Lq, t, qbar);
+    tail_mean_kernel<<<B * Hq, HYQ_D, 0, st>>>(static_cast<const __nv_bfloat16*>(q), Lq, t, qbar);
     if (launch_status() != HYQ_OK) return HYQ_ERR_CUDA;
 
     const size_t smem = align_up(SCORE_KEYS * KROW_WORDS * 4, 16) + (size_t)g * HYQ_D * sizeof(double);

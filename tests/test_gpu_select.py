@@ -38,6 +38,26 @@ def test_ties_duplicates_and_signed_zeros():
         _check(Q, K, W, k)
 
 
+@pytest.mark.parametrize("seed", range(4))
+def test_tail_queries_with_a_wide_exponent_spread(seed):
+    """Tail rows mixing magnitudes from 1e-30 to 3e4 and large values of alternating sign: the fp64 partial sums of
+    the tail mean are then inexact, so its value depends on the order of the additions - it has to be the row
+    order of Algorithm 1 as the oracle takes it, or the index sets near ties come out different."""
+    g = torch.Generator().manual_seed(700 + seed)
+    B, Hq, Hkv, L, W, k = 1, 4, 2, 1200, 256, 40
+    Q = torch.randn(B, Hq, L, 128, generator=g)
+    mag = 10.0 ** (torch.rand(B, Hq, L, 128, generator=g) * 34.5 - 30.0)            # 1e-30 ... 3e4
+    Q = Q.sign() * mag
+    big = 3.0e4 * (1.0 + torch.rand(B, Hq, L, 1, generator=g))
+    sign = torch.where(torch.arange(L) % 2 == 0, 1.0, -1.0).view(1, 1, L, 1)
+    Q[..., ::3] = (sign * big).expand(B, Hq, L, 128)[..., ::3]                      # cancelling large terms in every third channel
+    Q = Q.to(torch.bfloat16)
+    K = rand_bf16((B, Hkv, L, 128), seed=800 + seed)
+    K[0, :, 10:50] = K[0, :, 9:10]                                                  # equal keys: near-ties decided by the mean's last bits
+    _check(Q, K, W, k)
+    _check(Q, K, W, k, n_tail=77)
+
+
 def test_empty_problems_touch_nothing():
     ensure_built()
     Q, K = rand_bf16((1, 2, 64, 128), 3).cuda(), rand_bf16((1, 2, 64, 128), 4).cuda()

@@ -1,4 +1,8 @@
-"""GPU parity of the column-mass selector (Eq. 4-5) against the oracle: index sets bit-exact."""
+"""GPU parity of the column-mass selector (Eq. 4-5) against the oracle.  Where scores nearly tie, several sets are
+correct answers to the definition: every set the library returns is checked for VALIDITY against the
+plain-definition oracle (nothing selected scores lower than anything left out, beyond fp64 rounding), and, as a
+second and stricter assert, for bit-equality with the oracle's fixed-order recipe (the library's reproducibility
+contract)."""
 import numpy as np
 import pytest
 import torch
@@ -21,13 +25,35 @@ SHAPES = [  # B, Hq, Hkv, Lq, Lk, W, n_queries, k
 ]
 
 
+def assert_valid_for_the_definition(got, q, kk, W, k, nT, alpha=None):
+    """got [B,Hq,k]: size k, strictly ascending, inside [0, P), and no selected key scores lower under the plain
+    definition than an unselected one (tolerance: 1e-12 of the largest score, the rounding of fp64 sums)."""
+    P = max(0, kk.shape[2] - W)
+    if P == 0:
+        assert got.shape[2] == 0
+        return
+    _, sc = oracle.select_vertical_mass(wl.bits(q), wl.bits(kk), W, k, nT, alpha=alpha, return_scores=True, plain=True)
+    assert got.shape == sc.shape[:2] + (k,)
+    assert got.min() >= 0 and got.max() < P
+    assert np.all(np.diff(got, axis=-1) > 0)
+    for b in range(got.shape[0]):
+        for h in range(got.shape[1]):
+            chosen = np.zeros(P, dtype=bool)
+            chosen[got[b, h]] = True
+            if chosen.all():
+                continue
+            assert sc[b, h][chosen].min() >= sc[b, h][~chosen].max() - 1e-12 * sc[b, h].max(), (b, h)
+
+
 @pytest.mark.parametrize("B,Hq,Hkv,Lq,Lk,W,nT,k", SHAPES)
-def test_index_sets_are_bit_exact(B, Hq, Hkv, Lq, Lk, W, nT, k):
+def test_index_sets_are_valid_and_bit_exact(B, Hq, Hkv, Lq, Lk, W, nT, k):
     q, kk = rand_bf16((B, Hq, Lq, 128), 1, 1.2), rand_bf16((B, Hkv, Lk, 128), 2, 1.2)
-    want = oracle.select_vertical_mass(wl.bits(q), wl.bits(kk), W, k, nT)
     got = api.hyq_select_vertical_mass(q.cuda(), kk.cuda(), W, k, nT)
     torch.cuda.synchronize()
-    assert got.shape == want.shape and np.array_equal(got.cpu().numpy(), want)
+    got = got.cpu().numpy()
+    assert_valid_for_the_definition(got, q, kk, W, k, nT)
+    want = oracle.select_vertical_mass(wl.bits(q), wl.bits(kk), W, k, nT)
+    assert got.shape == want.shape and np.array_equal(got, want)
 
 
 def test_planted_keys_large_scores_and_a_custom_scale():
@@ -36,8 +62,9 @@ def test_planted_keys_large_scores_and_a_custom_scale():
     K[:, :, :500] = (K[:, :, :500].float() * 6).to(torch.bfloat16)          # scores in the hundreds
     for scale in (0.0, 0.05):
         want = oracle.select_vertical_mass(wl.bits(Q), wl.bits(K), w.window, w.k, 24, alpha=None if scale == 0 else np.float32(scale))
-        got = api.hyq_select_vertical_mass(Q.cuda(), K.cuda(), w.window, w.k, 24, softmax_scale=scale)
-        assert np.array_equal(got.cpu().numpy(), want)
+        got = api.hyq_select_vertical_mass(Q.cuda(), K.cuda(), w.window, w.k, 24, softmax_scale=scale).cpu().numpy()
+        assert_valid_for_the_definition(got, Q, K, w.window, w.k, 24, alpha=None if scale == 0 else np.float32(scale))
+        assert np.array_equal(got, want)
 
 
 def test_benchmark_shape_heads_and_argument_checks():
@@ -46,8 +73,9 @@ def test_benchmark_shape_heads_and_argument_checks():
     Q, K, _ = wl.make_inputs(w, heads=[0, 5])
     Qt = Q[:, :, -64:].contiguous()
     want = oracle.select_vertical_mass(wl.bits(Qt), wl.bits(K), w.window, w.k, 16)
-    got = api.hyq_select_vertical_mass(Qt.cuda(), K.cuda(), w.window, w.k, 16)
-    assert np.array_equal(got.cpu().numpy(), want)
+    got = api.hyq_select_vertical_mass(Qt.cuda(), K.cuda(), w.window, w.k, 16).cpu().numpy()
+    assert_valid_for_the_definition(got, Qt, K, w.window, w.k, 16)
+    assert np.array_equal(got, want)
     with pytest.raises(api.HyqError):
         api.hyq_select_vertical_mass(Qt.cuda(), K.cuda(), w.window, w.k, 65)       # more queries than rows given
     with pytest.raises(api.HyqError):

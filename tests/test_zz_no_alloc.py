@@ -9,8 +9,9 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from gpu_util import ensure_built, rand_bf16
-from paper_2608_27875_b200 import api
+from paper_2608_27875_b200 import api, workloads as wl
 
 pytestmark = pytest.mark.gpu
 
@@ -43,6 +44,27 @@ def test_static_scratch_matches_workspace_entry_point_on_consecutive_calls():
         ref, got = _both(Q, K, window, k)
         np.testing.assert_array_equal(got, ref)       # index sets are integers: equality, no tolerance
         assert (np.diff(got, axis=-1) > 0).all() and got.min() >= 0 and got.max() < L - window
+        np.testing.assert_array_equal(got, oracle.select_vertical(wl.bits(Q.cpu()), wl.bits(K.cpu()), window, k))
+
+
+def test_static_scratch_call_leaves_the_free_device_memory_unchanged():
+    """The point of the entry point: with the output preallocated, a call (after the first one on the device,
+    which looks up the array's address) takes nothing from the device's free memory and gives nothing back."""
+    lib = ensure_built()
+    B, Hq, Hkv, L, window, k = 1, 8, 2, 3000, 256, 55
+    Q, K = rand_bf16((B, Hq, L, 128), seed=300).cuda(), rand_bf16((B, Hkv, L, 128), seed=301).cuda()
+    out = torch.empty(B, Hq, k, dtype=torch.int32, device="cuda")
+    stream = torch.cuda.current_stream().cuda_stream
+    call = lambda: lib.hyq_select_vertical_static(Q.data_ptr(), K.data_ptr(), B, Hq, Hkv, L, L, 128, window, 0, k,   # noqa: E731
+                                                  out.data_ptr(), stream)
+    assert call() == 0
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
+    assert call() == 0
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before
+    np.testing.assert_array_equal(out.cpu().numpy(), oracle.select_vertical(wl.bits(Q.cpu()), wl.bits(K.cpu()), window, k))
 
 
 def test_static_scratch_rejects_problems_beyond_its_fixed_size():
