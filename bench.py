@@ -46,6 +46,12 @@ NCU_TRAFFIC_BYTES = {"c2": 693018624 + 500875264}
 NCU_DECODE_TRAFFIC_BYTES_B4 = 157169152 + 3803392
 
 
+def workload_config(w, world: int = 1, strong: bool = False) -> dict:
+    """The `config` object of the JSON line: the same keys and values from both arms (hyq and reference)."""
+    return {"workload": w.name, "B": w.B * (1 if strong else max(1, world)), "Hq": w.Hq, "Hkv": w.Hkv, "L": w.L, "D": w.D,
+            "window": w.window, "k": w.k, "formats": list(w.fmts)}
+
+
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -173,14 +179,51 @@ def run_reference(args, w):
         "impl": "reference", "metric": METRIC, "value": tflops, "unit": "TFLOPS", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t_tot / max(1, args.steps),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "B": w.B, "Hq": w.Hq, "Hkv": w.Hkv, "L": w.L, "D": w.D, "window": w.window,
-                   "k": w.k, "formats": list(w.fmts)},
+        "config": workload_config(w, int(os.environ.get("WORLD_SIZE", "1")), getattr(args, "strong", False)),
         "cpu_baseline": {"value": tflops, "unit": "TFLOPS", "cores": cores, "kind": "oracle", "sample": desc},
         "e2e": {"value": tflops, "unit": "TFLOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
     print(json.dumps(line))
 
+
+
+def method_error_report(w, path, Q, K, V, n_random: int = 16):
+    """Error of the METHOD against exact attention (all pairs in full precision), measured on the GPU's outputs: the
+    hybrid operator as benchmarked, the same low-bit codes with neither vertical keys nor window (uniform low-bit) and
+    with the window only.  Reference: the CPU oracle's exact attention (window >= L) on a row sample that touches
+    every structural boundary, for one (batch, KV head) group per batch element.  Sum|err| / Sum|ref| and max-abs."""
+    import oracle
+    api = path.api
+    outs = {"hybrid": path.out.clone()}
+    for name, (k_on, win) in {"uniform_lowbit": (False, 0), "window_only": (False, w.window)}.items():
+        outs[name] = api.hyq_hybrid_attention_prefill(path.Q, path.K, path.V, path.qc, path.kc, path.vc, path.qs, path.ks, path.vs,
+                                                      w.fmts, path.idx if k_on else None, win)
+    torch.cuda.synchronize()
+    rows = wl.sample_rows(w.L, w.window, n_random=n_random, edge=2)
+    g = w.Hq // w.Hkv
+    num = {n: 0.0 for n in outs}
+    mx = {n: 0.0 for n in outs}
+    den = 0.0
+    groups = []
+    for b in range(w.B):
+        kvh = b % w.Hkv
+        hs = slice(kvh * g, (kvh + 1) * g)
+        qb, kb, vb = wl.bits(Q[b:b + 1, hs]), wl.bits(K[b:b + 1, kvh:kvh + 1]), wl.bits(V[b:b + 1, kvh:kvh + 1])
+        zc = lambda h, f: np.zeros((1, h, w.L, oracle.code_row_bytes(f, w.D)), dtype=np.uint8)   # noqa: E731
+        zs = lambda h: np.zeros((1, h, -(-w.L // 64)), dtype=np.float32)                              # noqa: E731
+        exact = oracle.attention_rows(qb, kb, vb, zc(g, w.q_fmt), zc(1, w.k_fmt), zc(1, w.v_fmt), zs(g), zs(1), zs(1),
+                                      w.fmts, None, w.L, rows)          # window >= L: every pair in full precision
+        den += float(np.abs(exact).sum())
+        for n, o in outs.items():
+            d = np.abs(o[b:b + 1, hs][:, :, torch.from_numpy(rows).long().to(o.device)].double().cpu().numpy() - exact)
+            num[n] += float(d.sum())
+            mx[n] = max(mx[n], float(d.max()))
+        groups.append([b, kvh])
+    rep = {f"{n}_vs_exact": {"sum_abs_err_over_sum_abs_ref": num[n] / den, "max_abs": mx[n]} for n in outs}
+    rep["sample"] = (f"{len(rows)} rows (first/last, window edge, tile edges, {n_random} seeded random rows) of the {g} query "
+                     f"heads of one KV head per batch element: (b, kv head) = {groups}; reference = CPU oracle, exact attention in fp64")
+    return rep
 
 # ------------------------------------------------------------------------------------------------
 class DevicePath:
@@ -218,8 +261,12 @@ class DevicePath:
         self.K.copy_(K, non_blocking=True)
         self.V.copy_(V, non_blocking=True)
 
-    def step(self, timed: bool = False):
+    def step(self, timed: bool = False, kernel_events=None):
+        """One pass of the path.  kernel_events: a pair of CUDA events that the library records around the attention
+        kernel proper in this step (default: the path's own pair, overwritten every step)."""
         api, w = self.api, self.w
+        k0, k1 = kernel_events if kernel_events is not None else self.kev
+        self.args.ev_kernel_start, self.args.ev_kernel_stop = k0.cuda_event, k1.cuda_event
         if timed:
             self.ev[0].record()
         api.hyq_select_vertical(self.Q, self.K, w.window, w.k, workspace=self.sel_ws, out=self.idx)
@@ -487,6 +534,11 @@ def main():
     ap.add_argument("--staging", type=int, default=128, help="with --decode: staged rows (W_s, all filled)")
     ap.add_argument("--splits", type=int, default=0, help="with --decode: slices per KV head (0 = library's choice)")
     ap.add_argument("--kv-format", default="int4", choices=["int4", "int8", "fp8"], help="with --decode: cache code format (K4V4 / K8V8 / FP8 e4m3)")
+    ap.add_argument("--strong", action="store_true",
+                    help="strong scaling: ONE batch of the workload, its (batch, KV head) units sharded over the ranks "
+                         "(default: every rank runs its own full batch)")
+    ap.add_argument("--method-error", action="store_true",
+                    help="also report the method's error against exact attention (always on for c4)")
     ap.add_argument("--formats", default="", choices=["", *sorted(FORMAT_SETS)],
                     help="override the workload's (Q, K, V) low-bit formats (default: as the workload defines them)")
     args = ap.parse_args()
@@ -507,9 +559,33 @@ def main():
         run_decode(args, w)
         return
 
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # launched plainly: start the N ranks here (one process per GPU; NCCL only for the barrier and the max-reduction)
+        import socket
+        import torch.multiprocessing as mp
+        with socket.socket() as s_:
+            s_.bind(("127.0.0.1", 0))
+            port = s_.getsockname()[1]
+        mp.spawn(_spawned_rank, args=(args.gpus, port, sys.argv[1:]), nprocs=args.gpus, join=True)
+        return
+    run_hyq(args, w)
+
+
+def _spawned_rank(rank: int, world: int, port: int, argv):
+    os.environ.update(RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(world), MASTER_ADDR="127.0.0.1",
+                      MASTER_PORT=str(port))
+    sys.argv = [sys.argv[0]] + list(argv)
+    main()
+
+
+def run_hyq(args, w):
     import ctypes
     from paper_2608_27875_b200 import api, build, sharding
     rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+    if world != args.gpus:
+        raise SystemExit(f"bench.py: --gpus {args.gpus} but the launcher started {world} rank(s)")
+    if torch.cuda.device_count() < (world if "LOCAL_RANK" in os.environ else 1):
+        raise SystemExit(f"bench.py: {world} ranks on one node need {world} GPUs, found {torch.cuda.device_count()}")
     local = int(os.environ.get("LOCAL_RANK", "0"))
     if rank == 0 or world == 1:
         build.build()
@@ -521,6 +597,9 @@ def main():
         dist.barrier()
     api.lib()
 
+    if args.strong:
+        run_strong(args, w, api, sharding, rank, world, dev)
+        return
     # every rank runs its own full batch of the workload (units = (batch, kv head) groups; no collective)
     wr = w.scaled(seed=w.seed + 17 * rank)
     Q, K, V = wl.make_inputs(wr)
@@ -544,12 +623,19 @@ def main():
     parts = np.zeros(3)
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
+    # one pair of events per timed step for the library to record around the attention kernel proper
+    kevs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    for a_, b_ in kevs:                 # (torch creates the CUDA event at the first record)
+        a_.record()
+        b_.record()
+    barrier()
     ev0.record()
-    for _ in range(args.steps):
-        path.step(timed=True)
+    for n in range(args.steps):
+        path.step(timed=True, kernel_events=kevs[n])
     ev1.record()
     barrier()
     total_ms = ev0.elapsed_time(ev1)
+    kern_in_loop = [a_.elapsed_time(b_) for a_, b_ in kevs]
     # per-part times of the last step (events are re-recorded every step)
     parts = np.array([path.ev[n].elapsed_time(path.ev[n + 1]) for n in range(3)])
     clocks = sampler.stop()
@@ -559,6 +645,7 @@ def main():
     attn_ms, kern_ms_l = [], []
     for _ in range(max(3, min(args.steps, 10))):
         path.ev[0].record()
+        path.args.ev_kernel_start, path.args.ev_kernel_stop = (e_.cuda_event for e_ in path.kev)
         rc = api.lib().hyq_hybrid_attention_prefill(ctypes.byref(path.args), torch.cuda.current_stream().cuda_stream)
         path.ev[1].record()
         torch.cuda.synchronize()
@@ -566,7 +653,8 @@ def main():
         attn_ms.append(path.ev[0].elapsed_time(path.ev[1]))
         kern_ms_l.append(path.kev[0].elapsed_time(path.kev[1]))
     attn_call_ms = float(np.mean(attn_ms))
-    kern_ms = float(np.mean(kern_ms_l))
+    kern_ms_isolated = float(np.mean(kern_ms_l))
+    kern_ms = float(np.median(kern_in_loop))                 # the figure of record: inside the timed steps
 
     total_ms = sharding.max_over_ranks(total_ms, dev)
     ms_per_step = total_ms / args.steps
@@ -628,23 +716,32 @@ def main():
         "frac": achieved / peak_eff, "traffic": NCU_TRAFFIC_BYTES.get(w.name),
         "peak_source": f"{peaks['source']}: bf16 {peaks['bf16_tflops']} TFLOP/s for the full-precision pairs, 2x that "
                        f"(nominal 8-bit:16-bit ratio) for the low-bit pairs; peak = flops / mixed roofline time",
-        "kernel_ms": k_ms, "timed": "kernel only (events inside the library)" if kern_ms else "attention call incl. pre-pass",
+        "kernel_ms": k_ms, "kernel_ms_isolated": kern_ms_isolated,
+        "timed": "median over the timed steps of the library's own events around the attention kernel (kernel_ms_isolated: "
+                 "the same events in a separate loop with a synchronize between launches)",
         "fp_pair_share": n_fp / wr.causal_pairs, "roofline_ms_measured": t_roof_meas * 1e3,
         "roofline_ms_nominal": t_roof_nom * 1e3, "frac_nominal": (t_roof_nom * 1e3) / k_ms,
+        "frac_whole_step": (t_roof_meas * 1e3) / ms_per_step,
         "frac_nominal_whole_step": (t_roof_nom * 1e3) / ms_per_step, "min_bytes": bytes_min,
+        "nominal_definition": "the workload definition's roofline: full-precision pairs at 2250 TFLOP/s dense bf16, low-bit "
+                              "pairs at 4500 TFLOP/s dense INT8/FP8, or the minimum bytes at 8 TB/s if larger (frac_nominal); "
+                              "`frac` and `peak` use this pool's measured bf16 matmul rate instead, as the measurement "
+                              "contract asks",
     }
 
     t_cpu, pairs_cpu, desc, cores = oracle_sample(w, args.cpu_budget)
     cpu = {"value": 4 * w.D * pairs_cpu / t_cpu / 1e12, "unit": "TFLOPS", "cores": cores, "kind": "oracle", "sample": desc}
+
+    method_error = method_error_report(wr, path, Q, K, V) if (args.method_error or w.name == "c4") else None
 
     line = {
         "metric": METRIC, "value": value, "unit": "TFLOPS", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": DTYPE_NOTE[w.q_fmt],
         "data": "synthetic",
-        "config": {"workload": w.name, "B": w.B * world, "Hq": w.Hq, "Hkv": w.Hkv, "L": w.L, "D": w.D, "window": w.window,
-                   "k": w.k, "formats": list(w.fmts), "l2": "inputs larger than L2 (Q+K+V bf16 = %.0f MB per step)" % (h2d / 1e6),
-                   "step": "select + quantize Q,K,V + fused attention (pre-pass included)", "out_dtype": "fp32"},
+        "config": workload_config(w, world, args.strong),
+        "config_notes": {"l2": "inputs larger than L2 (Q+K+V bf16 = %.0f MB per step)" % (h2d / 1e6),
+                         "step": "select + quantize Q,K,V + fused attention (pre-pass included)", "out_dtype": "fp32"},
         "step_parts_ms": {"select": float(parts[0]), "quantize": float(parts[1]), "attention_call": float(parts[2])},
         "attention_only_tflops": flops / (attn_call_ms * 1e-3) / 1e12,
         "roofline": roofline, "cpu_baseline": cpu,
@@ -658,9 +755,89 @@ def main():
         "gpu_launches": path.launches_per_step * args.steps,
         "clocks": clocks,
     }
+    if method_error is not None:
+        line["method_error"] = method_error
     print(json.dumps(line))
     if world > 1:
         torch.distributed.destroy_process_group()
+
+
+def run_strong(args, w, api, sharding, rank, world, dev):
+    """`--strong`: ONE batch of the workload; its (batch, KV head) units are sharded over the ranks by
+    sharding.shard_units and every rank runs the whole path on its own units (device-resident inputs, no collective on
+    the data path).  value = the batch's FLOPs / the slowest rank's time.  The end-to-end leg goes through
+    sharding.run_sharded from pinned host tensors, every rank writing its slices of the output."""
+    import torch.distributed as dist
+    g = w.Hq // w.Hkv
+    wu = w.scaled(B=1, Hq=g, Hkv=1)
+    Q, K, V = wl.make_inputs(w)
+    mine = sharding.shard_units(w.B, w.Hkv, world, rank)
+    paths = []
+    for b, hk in mine:
+        p_ = DevicePath(wu, dev)
+        p_.load(Q[b:b + 1, hk * g:(hk + 1) * g].contiguous(), K[b:b + 1, hk:hk + 1].contiguous(), V[b:b + 1, hk:hk + 1].contiguous())
+        paths.append(p_)
+    torch.cuda.synchronize()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        for p_ in paths:
+            p_.step()
+    barrier()
+    sampler = ClockSampler(dev.index)
+    sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    ev0.record()
+    for _ in range(args.steps):
+        for p_ in paths:
+            p_.step()
+    ev1.record()
+    barrier()
+    ms = sharding.max_over_ranks(ev0.elapsed_time(ev1), dev) / args.steps
+    clocks = sampler.stop()
+    assert all(int(p_.status.item()) == 0 for p_ in paths), "attention kernel reported a device-side error"
+    # end to end: pinned host batch -> each rank's units through the public wrapper -> the rank's slices of the output
+    Qp, Kp, Vp = (t.pin_memory() for t in (Q, K, V))
+    out_host = torch.zeros(w.B, w.Hq, w.L, w.D, dtype=torch.float32).pin_memory()
+    slot = DevicePath(wu, dev)
+
+    def unit_prefill(q, k_, v, window, k_sel, fmts):
+        slot.load(q, k_, v)
+        slot.step()
+        return slot.out
+
+    e2e = []
+    for n in range(3):
+        barrier()
+        t0 = time.perf_counter()
+        sharding.run_sharded(Qp, Kp, Vp, w.window, w.k, w.fmts, prefill_fn=unit_prefill, out=out_host, world=world, rank=rank)
+        torch.cuda.synchronize()
+        if n > 0:
+            e2e.append((time.perf_counter() - t0) * 1e3)
+    e2e_ms = sharding.max_over_ranks(float(np.mean(e2e)), dev)
+    if mine:
+        b, hk = mine[-1]
+        assert torch.equal(out_host[b:b + 1, hk * g:(hk + 1) * g].to(dev), paths[-1].out), "sharded e2e differs from the device-resident run"
+    if rank == 0:
+        h2d = sum(t.numel() * t.element_size() for t in (Q, K, V))
+        print(json.dumps({
+            "metric": METRIC, "value": w.flops / (ms * 1e-3) / 1e12, "unit": "TFLOPS", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "strong", "vs_baseline": None,
+            "dtype": DTYPE_NOTE[w.q_fmt], "data": "synthetic", "config": workload_config(w, world, True),
+            "config_notes": {"sharding": f"{w.B * w.Hkv} (batch, KV head) units over {world} rank(s), contiguous balanced ranges, "
+                                         f"one launch sequence per unit, no collective on the data path",
+                             "l2": "inputs larger than L2" if h2d > 126e6 else "inputs fit L2"},
+            "e2e": {"value": w.flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOPS", "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": out_host.numel() * 4, "ms_per_step": e2e_ms,
+                    "how": "sharding.run_sharded: pinned host batch -> each rank's units H2D -> path -> D2H into the rank's output slices"},
+            "gpu_launches": sum(p_.launches_per_step for p_ in paths) * args.steps, "clocks": clocks}))
+    if world > 1:
+        dist.destroy_process_group()
 
 
 if __name__ == "__main__":

@@ -80,6 +80,50 @@ def test_two_ranks_reproduce_the_unsharded_result():
     assert ret["t_max"] == 11.0                            # max over ranks of (10, 11)
 
 
+# ---- the wrapper the product uses (sharding.run_sharded), with the oracle standing in for the device calls ---------
+def _oracle_prefill(q, k, v, window, k_sel, fmts):
+    r = oracle.hybrid_prefill(wl.bits(q), wl.bits(k), wl.bits(v), window, k_sel, fmts)
+    return torch.from_numpy(r["out"])
+
+
+def _wrapper_worker(rank, world, port, ret):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        Q, K, V = wl.make_inputs(W)
+        own = sharding.run_sharded(Q, K, V, W.window, W.k, W.fmts, prefill_fn=_oracle_prefill,
+                                   out=torch.zeros(W.B, W.Hq, W.L, W.D, dtype=torch.float64))
+        full = sharding.run_sharded(Q, K, V, W.window, W.k, W.fmts, prefill_fn=_oracle_prefill,
+                                    out=torch.zeros(W.B, W.Hq, W.L, W.D, dtype=torch.float64), gather=True)
+        ret[rank] = (own.numpy(), full.numpy())
+    finally:
+        dist.destroy_process_group()
+
+
+@pytest.mark.parametrize("world", [2, 3])
+def test_run_sharded_fills_each_ranks_slices_and_gathers_the_whole_output(world):
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    ret = mp.Manager().dict()
+    mp.spawn(_wrapper_worker, args=(world, port, ret), nprocs=world, join=True)
+    Q, K, V = wl.make_inputs(W)
+    ref = oracle.hybrid_prefill(wl.bits(Q), wl.bits(K), wl.bits(V), W.window, W.k, W.fmts)["out"]
+    g = W.Hq // W.Hkv
+    for rank in range(world):
+        own, full = ret[rank]
+        np.testing.assert_allclose(full, ref, rtol=0, atol=1e-13)               # after the gather: everything, everywhere
+        mask = np.zeros((W.B, W.Hq), dtype=bool)
+        for b, kvh in sharding.shard_units(W.B, W.Hkv, world, rank):
+            mask[b, kvh * g:(kvh + 1) * g] = True
+        np.testing.assert_allclose(own[mask], ref[mask], rtol=0, atol=1e-13)    # without it: the rank's own slices ...
+        assert not own[~mask].any()                                             # ... and nothing else touched
+    # without a process group the wrapper runs every unit itself
+    solo = sharding.run_sharded(Q, K, V, W.window, W.k, W.fmts, prefill_fn=_oracle_prefill,
+                                out=torch.zeros(W.B, W.Hq, W.L, W.D, dtype=torch.float64))
+    np.testing.assert_allclose(solo.numpy(), ref, rtol=0, atol=1e-13)
+
+
 # ---- the decode side shards by the same (batch, KV head) units ------------------------------------------------
 def _decode_inputs():
     g = torch.Generator().manual_seed(91)
