@@ -8,6 +8,7 @@
  *   hyq_select_vertical_mass       Eq. 4-5 (the same selection from accumulated softmax column mass)
  *   hyq_quantize_blocks            Algorithm 2, Stage 2 (per-tile quantization)
  *   hyq_hybrid_attention_prefill   Eq. 6-7 / Algorithm 2, Stage 3 (fused hybrid softmax attention)
+ *   hyq_*_varlen                   the same three stages over a ragged batch of prompts
  *
  * Common rules
  *   - Every tensor pointer is a DEVICE pointer to a contiguous row-major array.
@@ -231,6 +232,38 @@ typedef struct {
 
 int hyq_hybrid_attention_prefill_workspace(const hyq_attn_args* args, size_t* bytes /* host, out */);
 int hyq_hybrid_attention_prefill(const hyq_attn_args* args, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Ragged batches (several prompts of different lengths in one call; the serving shape of the paper's batching
+ * study, Section 4.3).  The three stages run per sequence exactly as the calls above define them - every sequence is
+ * its own problem with its own L, its own candidate prefix, its own quantization blocks (which restart at the
+ * sequence's first token) and its own causal / window / vertical-key predicates - so each *_varlen call returns,
+ * sequence by sequence, bit for bit what the plain call returns for that sequence alone.
+ *
+ *   Packing.  cu_seqlens is a HOST array of n_seq + 1 ascending token offsets (cu_seqlens[0] = 0; sequence s has
+ *   L_s = cu_seqlens[s+1] - cu_seqlens[s] >= 1 tokens).  A packed tensor with H heads holds the sequences one after
+ *   the other, each as a contiguous [H, L_s, D] block: sequence s starts at element H * D * cu_seqlens[s].
+ *   Packed codes follow the same rule in bytes per row (D, or D/2 for INT4).  Packed scales hold [H, nb_s] per
+ *   sequence with nb_s = ceil(L_s / block_tokens): sequence s starts at H * (sum of nb_r over r < s).  k_per_seq is
+ *   a HOST array of n_seq vertical counts (0 <= k_s <= max(0, L_s - window)); the packed index buffer holds
+ *   [Hq, k_s] per sequence, sequence s starting at Hq * (sum of k_r over r < s).
+ *
+ *   The sequences are processed one after the other on `stream` (longest first); one workspace of the size the
+ *   plain query returns for the LONGEST sequence (B = 1) serves them all.  Host arrays are read during the call
+ *   and may be freed afterwards.  Errors: as the plain calls, checked for every sequence before anything is
+ *   launched; n_seq <= 0 or a non-ascending cu_seqlens -> INVALID_ARG.
+ *
+ *   hyq_hybrid_attention_prefill_varlen takes a hyq_attn_args whose tensor pointers are the PACKED buffers and
+ *   whose B, L, Lq and k fields are ignored (whole prefills only: every sequence's queries are its L_s rows);
+ *   out [packed, Hq heads] and lse (optional, Hq * L_s floats per sequence, sequence s at Hq * cu_seqlens[s]).
+ * ------------------------------------------------------------------------------------------- */
+int hyq_select_vertical_varlen(const void* q, const void* k_, int n_seq, const int32_t* cu_seqlens /* host */,
+                               int Hq, int Hkv, int D, int window, int n_tail, const int32_t* k_per_seq /* host */,
+                               int32_t* idx_out, void* workspace, size_t workspace_bytes, void* stream);
+int hyq_quantize_blocks_varlen(const void* x, int n_seq, const int32_t* cu_seqlens /* host */, int H, int D,
+                               int block_tokens, int format, void* codes_out, float* scales_out, void* stream);
+int hyq_hybrid_attention_prefill_varlen(const hyq_attn_args* args, int n_seq, const int32_t* cu_seqlens /* host */,
+                                        const int32_t* k_per_seq /* host */, void* stream);
 
 /* ---------------------------------------------------------------------------------------------
  * hyq_test_set_attention_hooks - test hook (the paper has no counterpart): exercises the tensor-core

@@ -20,7 +20,8 @@ WINDOW_SLIDING, WINDOW_FIXED_TAIL = 0, 1
 EXPORTS = ("hyq_status_string", "hyq_version", "hyq_paper_k", "hyq_select_vertical_workspace",
            "hyq_select_vertical", "hyq_select_vertical_static", "hyq_select_vertical_mass_workspace",
            "hyq_select_vertical_mass", "hyq_quantize_blocks", "hyq_hybrid_attention_prefill_workspace",
-           "hyq_hybrid_attention_prefill", "hyq_test_set_attention_hooks")
+           "hyq_hybrid_attention_prefill", "hyq_test_set_attention_hooks", "hyq_select_vertical_varlen",
+           "hyq_quantize_blocks_varlen", "hyq_hybrid_attention_prefill_varlen")
 
 
 class HyqError(RuntimeError):
@@ -70,6 +71,12 @@ def lib() -> ctypes.CDLL:
         L.hyq_hybrid_attention_prefill_workspace.argtypes = [ctypes.POINTER(AttnArgs), ctypes.POINTER(ctypes.c_size_t)]
         L.hyq_hybrid_attention_prefill.argtypes = [ctypes.POINTER(AttnArgs), ctypes.c_void_p]
         L.hyq_test_set_attention_hooks.argtypes = [ctypes.c_longlong, ctypes.c_int]
+        i32p = ctypes.POINTER(ctypes.c_int32)
+        L.hyq_select_vertical_varlen.argtypes = ([ctypes.c_void_p] * 2 + [ctypes.c_int, i32p] + [ctypes.c_int] * 5 + [i32p] +
+                                                 [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p])
+        L.hyq_quantize_blocks_varlen.argtypes = ([ctypes.c_void_p, ctypes.c_int, i32p] + [ctypes.c_int] * 4 +
+                                                 [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p])
+        L.hyq_hybrid_attention_prefill_varlen.argtypes = [ctypes.POINTER(AttnArgs), ctypes.c_int, i32p, i32p, ctypes.c_void_p]
         _lib = L
     return _lib
 
@@ -261,3 +268,80 @@ def hybrid_prefill(q, k, v, window: int, k_sel: int, fmts=(FMT_INT8, FMT_INT8, F
     out = hyq_hybrid_attention_prefill(q, k, v, qc, kc, vc, qs, ks, vs, fmts, idx, window, impl=impl,
                                        out_dtype=out_dtype)
     return dict(idx=idx, q_codes=qc, k_codes=kc, v_codes=vc, q_scales=qs, k_scales=ks, v_scales=vs, out=out)
+
+
+# ---- ragged batches --------------------------------------------------------------------------------------------
+def _i32(xs):
+    return (ctypes.c_int32 * len(xs))(*[int(x) for x in xs])
+
+
+def pack_sequences(seqs) -> tuple[torch.Tensor, list[int]]:
+    """[H, L_s, D] tensors -> one flat packed buffer (each sequence a contiguous [H, L_s, D] block) and the token
+    offsets cu_seqlens."""
+    cu = [0]
+    for t in seqs:
+        cu.append(cu[-1] + t.shape[1])
+    return torch.cat([t.contiguous().reshape(-1) for t in seqs]), cu
+
+
+def hybrid_prefill_varlen(qs, ks, vs, window: int, k_per_seq, fmts=(FMT_INT8, FMT_INT8, FMT_INT8), block_tokens: int = 64,
+                          out_dtype=torch.float32):
+    """The whole path over a ragged batch: ``qs[s]`` is [Hq, L_s, D], ``ks[s]`` / ``vs[s]`` are [Hkv, L_s, D] (bf16,
+    CUDA).  Packs the prompts, runs the three *_varlen calls and returns per-sequence views of the results:
+    a list of dicts with idx [Hq, k_s], codes, scales and out [Hq, L_s, D]."""
+    n = len(qs)
+    Hq, _, D = qs[0].shape
+    Hkv = ks[0].shape[0]
+    dev = qs[0].device
+    qp, cu = pack_sequences(qs)
+    kp, _ = pack_sequences(ks)
+    vp, _ = pack_sequences(vs)
+    lens = [cu[s + 1] - cu[s] for s in range(n)]
+    k_per_seq = [int(k) if lens[s] - window > 0 else 0 for s, k in enumerate(k_per_seq)]
+    cu_c, k_c = _i32(cu), _i32(k_per_seq)
+    total, nbs = cu[-1], [-(-L_ // block_tokens) for L_ in lens]
+    idx = torch.empty(max(1, Hq * sum(k_per_seq)), dtype=torch.int32, device=dev)
+    need = max([hyq_select_vertical_workspace(1, Hq, Hkv, L_, L_, D, window, k_) for L_, k_ in zip(lens, k_per_seq)] + [16])
+    ws = torch.empty(need, dtype=torch.uint8, device=dev)
+    _check(lib().hyq_select_vertical_varlen(qp.data_ptr(), kp.data_ptr(), n, cu_c, Hq, Hkv, D, window, 0, k_c, idx.data_ptr(),
+                                            ws.data_ptr(), ws.numel(), _stream()), "hyq_select_vertical_varlen")
+    codes, scales = [], []
+    for x, H, f in ((qp, Hq, fmts[0]), (kp, Hkv, fmts[1]), (vp, Hkv, fmts[2])):
+        c = torch.empty(H * total * code_row_bytes(f, D), dtype=torch.uint8, device=dev)
+        sc = torch.empty(H * sum(nbs), dtype=torch.float32, device=dev)
+        _check(lib().hyq_quantize_blocks_varlen(x.data_ptr(), n, cu_c, H, D, block_tokens, f, c.data_ptr(), sc.data_ptr(), _stream()),
+               "hyq_quantize_blocks_varlen")
+        codes.append(c)
+        scales.append(sc)
+    out = torch.empty(Hq * total * D, dtype=out_dtype, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    a = AttnArgs()
+    a.struct_size = ctypes.sizeof(AttnArgs)
+    a.B, a.Hq, a.Hkv, a.L, a.D, a.Lq = 1, Hq, Hkv, max(lens), D, 0
+    a.window, a.k, a.block_tokens = window, max(k_per_seq), block_tokens
+    a.q_format, a.k_format, a.v_format = fmts
+    a.out_dtype, a.impl, a.softmax_scale, a.window_mode = (1 if out_dtype == torch.float32 else 0), IMPL_AUTO, 0.0, WINDOW_SLIDING
+    a.q, a.k_, a.v = qp.data_ptr(), kp.data_ptr(), vp.data_ptr()
+    a.q_codes, a.k_codes, a.v_codes = (c.data_ptr() for c in codes)
+    a.q_scales, a.k_scales, a.v_scales = (s_.data_ptr() for s_ in scales)
+    a.vl_idx, a.out, a.status_word = idx.data_ptr(), out.data_ptr(), status.data_ptr()
+    a.k = k_per_seq[lens.index(max(lens))]
+    wsa = torch.empty(max(16, hyq_hybrid_attention_prefill_workspace(a)), dtype=torch.uint8, device=dev)   # the longest sequence's need
+    a.workspace, a.workspace_bytes = wsa.data_ptr(), wsa.numel()
+    _check(lib().hyq_hybrid_attention_prefill_varlen(ctypes.byref(a), n, cu_c, k_c, _stream()), "hyq_hybrid_attention_prefill_varlen")
+    res, ko, no = [], 0, 0
+    for s in range(n):
+        L_, k_, nb = lens[s], k_per_seq[s], nbs[s]
+        view = lambda buf, H, row, t0=cu[s], L_=L_: buf[H * row * t0:H * row * (t0 + L_)].view(H, L_, row)   # noqa: E731
+        res.append(dict(
+            idx=idx[Hq * ko:Hq * (ko + k_)].view(Hq, k_),
+            q_codes=view(codes[0], Hq, code_row_bytes(fmts[0], D)), k_codes=view(codes[1], Hkv, code_row_bytes(fmts[1], D)),
+            v_codes=view(codes[2], Hkv, code_row_bytes(fmts[2], D)),
+            q_scales=scales[0][Hq * no:Hq * (no + nb)].view(Hq, nb), k_scales=scales[1][Hkv * no:Hkv * (no + nb)].view(Hkv, nb),
+            v_scales=scales[2][Hkv * no:Hkv * (no + nb)].view(Hkv, nb), out=view(out, Hq, D)))
+        ko += k_
+        no += nb
+    torch.cuda.synchronize()
+    if int(status.item()) != 0:
+        raise HyqError(int(status.item()), "hyq_hybrid_attention_prefill_varlen (device)")
+    return res

@@ -191,4 +191,129 @@ int hyq_hybrid_attention_prefill(const hyq_attn_args* args, void* stream) {
     return args->block_tokens == HYQ_BLOCK_TOKENS ? launch_attn_tc(*args, alpha, st) : tcbt::launch_attn_tc(*args, alpha, st);
 }
 
+// ---- ragged batches: the plain calls, sequence by sequence, on packed buffers ---------------------------------
+static int check_cu(int n_seq, const int32_t* cu) {
+    if (n_seq <= 0 || !cu || cu[0] != 0) return HYQ_ERR_INVALID_ARG;
+    for (int s = 0; s < n_seq; ++s)
+        if (cu[s + 1] <= cu[s]) return HYQ_ERR_INVALID_ARG;
+    return HYQ_OK;
+}
+
+// sequence numbers, longest first (ties by position)
+static void longest_first(int n_seq, const int32_t* cu, int* order) {
+    for (int s = 0; s < n_seq; ++s) order[s] = s;
+    for (int a = 1; a < n_seq; ++a) {                       // insertion sort: batches are small
+        const int v = order[a], lv = cu[v + 1] - cu[v];
+        int b = a - 1;
+        while (b >= 0 && cu[order[b] + 1] - cu[order[b]] < lv) { order[b + 1] = order[b]; --b; }
+        order[b + 1] = v;
+    }
+}
+
+int hyq_select_vertical_varlen(const void* q, const void* k_, int n_seq, const int32_t* cu, int Hq, int Hkv, int D,
+                               int window, int n_tail, const int32_t* k_per_seq, int32_t* idx_out, void* workspace,
+                               size_t workspace_bytes, void* stream) {
+    int rc = check_cu(n_seq, cu);
+    if (rc != HYQ_OK) return rc;
+    if (!k_per_seq) return HYQ_ERR_INVALID_ARG;
+    size_t need = 0;
+    for (int s = 0; s < n_seq; ++s) {
+        const int L = cu[s + 1] - cu[s];
+        rc = check_select(q, k_, 1, Hq, Hkv, L, L, D, window, n_tail, k_per_seq[s]);
+        if (rc != HYQ_OK) return rc;
+        const long P = L - window > 0 ? (long)L - window : 0;
+        if (P > 0 && k_per_seq[s] > 0) need = need > select_workspace_bytes(1, Hq, L, window) ? need : select_workspace_bytes(1, Hq, L, window);
+    }
+    if (need == 0) return HYQ_OK;
+    if (!q || !k_ || !idx_out || !workspace) return HYQ_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k_) || !aligned16(workspace) || (reinterpret_cast<uintptr_t>(idx_out) & 3u)) return HYQ_ERR_ALIGNMENT;
+    if (workspace_bytes < need) return HYQ_ERR_WORKSPACE;
+    int* order = new int[n_seq];
+    long* koff = new long[n_seq];
+    long acc = 0;
+    for (int s = 0; s < n_seq; ++s) { koff[s] = acc; acc += k_per_seq[s]; }
+    longest_first(n_seq, cu, order);
+    for (int n = 0; n < n_seq && rc == HYQ_OK; ++n) {
+        const int s = order[n], L = cu[s + 1] - cu[s], ks = k_per_seq[s];
+        if (ks == 0 || L - window <= 0) continue;
+        const char* qs = static_cast<const char*>(q) + (size_t)Hq * D * cu[s] * 2;
+        const char* kk = static_cast<const char*>(k_) + (size_t)Hkv * D * cu[s] * 2;
+        rc = launch_select(qs, kk, 1, Hq, Hkv, L, L, window, n_tail, ks, idx_out + (size_t)Hq * koff[s], workspace,
+                           static_cast<cudaStream_t>(stream));
+    }
+    delete[] order;
+    delete[] koff;
+    return rc;
+}
+
+int hyq_quantize_blocks_varlen(const void* x, int n_seq, const int32_t* cu, int H, int D, int block_tokens, int format,
+                               void* codes_out, float* scales_out, void* stream) {
+    int rc = check_cu(n_seq, cu);
+    if (rc != HYQ_OK) return rc;
+    if (H <= 0 || !x || !codes_out || !scales_out) return HYQ_ERR_INVALID_ARG;
+    if (D != HYQ_D || !block_tokens_ok(block_tokens)) return HYQ_ERR_UNSUPPORTED;
+    if (format != HYQ_FMT_INT8 && format != HYQ_FMT_FP8_E4M3 && format != HYQ_FMT_INT4) return HYQ_ERR_UNSUPPORTED;
+    if (!aligned16(x) || !aligned16(codes_out) || (reinterpret_cast<uintptr_t>(scales_out) & 3u)) return HYQ_ERR_ALIGNMENT;
+    const size_t row_bytes = format == HYQ_FMT_INT4 ? D / 2 : D;
+    size_t nb_before = 0;
+    for (int s = 0; s < n_seq && rc == HYQ_OK; ++s) {
+        const int L = cu[s + 1] - cu[s];
+        rc = launch_quantize(static_cast<const char*>(x) + (size_t)H * D * cu[s] * 2, H, L, block_tokens, format,
+                             static_cast<char*>(codes_out) + (size_t)H * row_bytes * cu[s], scales_out + (size_t)H * nb_before,
+                             static_cast<cudaStream_t>(stream));
+        nb_before += (size_t)(L + block_tokens - 1) / block_tokens;
+    }
+    return rc;
+}
+
+int hyq_hybrid_attention_prefill_varlen(const hyq_attn_args* args, int n_seq, const int32_t* cu, const int32_t* k_per_seq,
+                                        void* stream) {
+    int rc = check_cu(n_seq, cu);
+    if (rc != HYQ_OK) return rc;
+    if (!args || args->struct_size != sizeof(hyq_attn_args) || !k_per_seq) return HYQ_ERR_INVALID_ARG;
+    const int bt = args->block_tokens;
+    if (!block_tokens_ok(bt)) return HYQ_ERR_UNSUPPORTED;
+    const size_t q_row = args->q_format == HYQ_FMT_INT4 ? HYQ_D / 2 : HYQ_D, k_row = args->k_format == HYQ_FMT_INT4 ? HYQ_D / 2 : HYQ_D;
+    const size_t v_row = args->v_format == HYQ_FMT_INT4 ? HYQ_D / 2 : HYQ_D;
+    // one argument block per sequence, all checked before the first launch
+    hyq_attn_args* per = new hyq_attn_args[n_seq];
+    int* order = new int[n_seq];
+    size_t nb_before = 0, k_before = 0;
+    for (int s = 0; s < n_seq && rc == HYQ_OK; ++s) {
+        const int L = cu[s + 1] - cu[s];
+        hyq_attn_args a = *args;
+        a.B = 1; a.L = L; a.Lq = 0; a.k = k_per_seq[s];
+        const size_t t0 = (size_t)cu[s];
+        auto at = [](const void* base, size_t bytes) -> const void* { return base ? static_cast<const char*>(base) + bytes : nullptr; };
+        a.q = at(args->q, (size_t)args->Hq * HYQ_D * t0 * 2);
+        a.k_ = at(args->k_, (size_t)args->Hkv * HYQ_D * t0 * 2);
+        a.v = at(args->v, (size_t)args->Hkv * HYQ_D * t0 * 2);
+        a.q_codes = at(args->q_codes, (size_t)args->Hq * q_row * t0);
+        a.k_codes = at(args->k_codes, (size_t)args->Hkv * k_row * t0);
+        a.v_codes = at(args->v_codes, (size_t)args->Hkv * v_row * t0);
+        a.q_scales = args->q_scales ? args->q_scales + (size_t)args->Hq * nb_before : nullptr;
+        a.k_scales = args->k_scales ? args->k_scales + (size_t)args->Hkv * nb_before : nullptr;
+        a.v_scales = args->v_scales ? args->v_scales + (size_t)args->Hkv * nb_before : nullptr;
+        a.vl_idx = (args->vl_idx && a.k > 0) ? args->vl_idx + (size_t)args->Hq * k_before : nullptr;
+        a.out = const_cast<void*>(at(args->out, (size_t)args->Hq * HYQ_D * t0 * (args->out_dtype == 1 ? 4 : 2)));
+        a.lse = args->lse ? args->lse + (size_t)args->Hq * t0 : nullptr;
+        if (a.k < 0 || a.k > (L - a.window > 0 ? L - a.window : 0)) rc = HYQ_ERR_INVALID_ARG;
+        if (rc == HYQ_OK) rc = check_attn(&a, true);
+        if (rc == HYQ_OK) {
+            const size_t need = use_simt(&a) ? attn_simt_workspace_bytes(a) : attn_tc_workspace_bytes(a);
+            if (need > 0 && (!a.workspace || a.workspace_bytes < need)) rc = HYQ_ERR_WORKSPACE;
+        }
+        per[s] = a;
+        nb_before += (size_t)(L + bt - 1) / bt;
+        k_before += (size_t)k_per_seq[s];
+    }
+    if (rc == HYQ_OK) {
+        longest_first(n_seq, cu, order);
+        for (int n = 0; n < n_seq && rc == HYQ_OK; ++n) rc = hyq_hybrid_attention_prefill(&per[order[n]], stream);
+    }
+    delete[] per;
+    delete[] order;
+    return rc;
+}
+
 }  // extern "C"
