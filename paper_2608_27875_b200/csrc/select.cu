@@ -21,26 +21,42 @@ constexpr int SCORE_GC = 4;          // query heads scored per pass over the sta
 constexpr int TOPK_THREADS = 1024;
 
 // -------------------------------------------------------------------------------------------
-// One thread per (b, h, channel) adds the t tail rows in ascending row order in fp64 - the order of Algorithm 1's
-// mean as it is written down, so the result is the same double for every finite input, whatever the spread of the
-// exponents (a split into partial sums would only agree while every partial sum is exact).  The loads of 16 rows
-// are issued together; only the additions form a chain.
-__global__ void __launch_bounds__(HYQ_D)
+// The t tail rows are added in ascending row order in fp64, one running sum per (b, h, channel) - the order of
+// Algorithm 1's mean as it is written down, so the result is the same double for every finite input, whatever the
+// spread of the exponents (a split into partial sums would only agree while every partial sum is exact).  A CTA owns
+// 32 channels of one (b, h): all its threads stage 512 rows at a time in shared memory (the loads are what takes
+// time), then one thread per channel runs the addition chain over the staged rows.
+constexpr int MEAN_CH = 32, MEAN_ROWS = 512, MEAN_THREADS = 256;
+
+__global__ void __launch_bounds__(MEAN_THREADS)
 tail_mean_kernel(const __nv_bfloat16* __restrict__ q, int Lq, int t, double* __restrict__ qbar) {
+    __shared__ __nv_bfloat16 tile[MEAN_ROWS][MEAN_CH + 2];         // +2: the chain's column reads stay conflict-free enough
     const long bh = blockIdx.x;
-    const int d = threadIdx.x;
-    const __nv_bfloat16* base = q + (bh * Lq + (Lq - t)) * (long)HYQ_D + d;
+    const int c0 = blockIdx.y * MEAN_CH;
+    const __nv_bfloat16* base = q + (bh * Lq + (Lq - t)) * (long)HYQ_D + c0;
     double s = 0.0;
-    int r = 0;
-    for (; r + 16 <= t; r += 16) {
-        float v[16];
+    for (int r0 = 0; r0 < t; r0 += MEAN_ROWS) {
+        const int rows = min(MEAN_ROWS, t - r0);
+        __syncthreads();
+        // 16 threads per row, 4 bytes each
+        for (int e = threadIdx.x; e < rows * (MEAN_CH / 2); e += MEAN_THREADS) {
+            const int r = e / (MEAN_CH / 2), c2 = (e % (MEAN_CH / 2)) * 2;
+            *reinterpret_cast<uint32_t*>(&tile[r][c2]) = __ldg(reinterpret_cast<const uint32_t*>(base + (long)(r0 + r) * HYQ_D + c2));
+        }
+        __syncthreads();
+        if (threadIdx.x < MEAN_CH) {
+            int r = 0;
+            for (; r + 8 <= rows; r += 8) {
+                float v[8];
 #pragma unroll
-        for (int j = 0; j < 16; ++j) v[j] = __bfloat162float(base[(long)(r + j) * HYQ_D]);
+                for (int j = 0; j < 8; ++j) v[j] = __bfloat162float(tile[r + j][threadIdx.x]);
 #pragma unroll
-        for (int j = 0; j < 16; ++j) s += (double)v[j];
+                for (int j = 0; j < 8; ++j) s += (double)v[j];
+            }
+            for (; r < rows; ++r) s += (double)__bfloat162float(tile[r][threadIdx.x]);
+        }
     }
-    for (; r < t; ++r) s += (double)__bfloat162float(base[(long)r * HYQ_D]);
-    qbar[bh * HYQ_D + d] = s / (double)t;
+    if (threadIdx.x < MEAN_CH) qbar[bh * HYQ_D + c0 + threadIdx.x] = s / (double)t;
 }
 
 // -------------------------------------------------------------------------------------------
@@ -210,7 +226,7 @@ int launch_select(const void* q, const void* k, int B, int Hq, int Hkv, int Lq, 
     double* qbar = static_cast<double*>(ws);
     double* scores = reinterpret_cast<double*>(static_cast<char*>(ws) + align_up((size_t)B * Hq * HYQ_D * sizeof(double), 256));
 
-    tail_mean_kernel<<<B * Hq, HYQ_D, 0, st>>>(static_cast<const __nv_bfloat16*>(q), Lq, t, qbar);
+    tail_mean_kernel<<<dim3(B * Hq, HYQ_D / MEAN_CH), MEAN_THREADS, 0, st>>>(static_cast<const __nv_bfloat16*>(q), Lq, t, qbar);
     if (launch_status() != HYQ_OK) return HYQ_ERR_CUDA;
 
     const size_t smem = align_up(SCORE_KEYS * KROW_WORDS * 4, 16) + (size_t)g * HYQ_D * sizeof(double);
