@@ -19,6 +19,7 @@ namespace hyq {
 constexpr int SCORE_KEYS = 128;      // keys per CTA in vscore_kernel
 constexpr int SCORE_GC = 4;          // query heads scored per pass over the staged K tile
 constexpr int TOPK_THREADS = 1024;
+constexpr int TOPK_CAND = 1536;      // candidate keys that the radix select keeps in shared memory
 
 // -------------------------------------------------------------------------------------------
 // The t tail rows are added in ascending row order in fp64, one running sum per (b, h, channel) - the order of
@@ -125,7 +126,8 @@ topk_kernel(const double* __restrict__ scores, int P, int k, int32_t* __restrict
     __shared__ int hist[256];
     __shared__ int warp_gt[NW], warp_eq[NW];
     __shared__ unsigned long long sh_prefix;
-    __shared__ int sh_krem;
+    __shared__ int sh_krem, sh_bin, n_cand;
+    __shared__ unsigned long long cand[TOPK_CAND];     // the keys still in the race once few are left
     const double* row = scores + (long)blockIdx.x * P;
     int32_t* out = idx_out + (long)blockIdx.x * k;
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
@@ -134,17 +136,28 @@ topk_kernel(const double* __restrict__ scores, int P, int k, int32_t* __restrict
 
     // radix select: after the loop `prefix` is the key of the k-th largest score and k_rem how
     // many positions holding exactly that key are still to be taken
+    // Once a pass leaves no more than TOPK_CAND keys sharing the digits fixed so far, those keys are gathered into
+    // shared memory (one more sweep over the row) and the remaining passes run over that short list.
     unsigned long long prefix = 0ull;
     int k_rem = k;
+    bool gathered = false;
     for (int pass = 0; pass < 8; ++pass) {
         const int shift = 56 - 8 * pass;
 #pragma unroll
         for (int e = 0; e < 8; ++e) whist[wid][lane + 32 * e] = 0;
         __syncwarp();
-        for (int p = seg0 + lane; p < seg1; p += 32) {
-            const unsigned long long key = order_key(row[p]);
-            if (pass == 0 || (key >> (shift + 8)) == (prefix >> (shift + 8)))
-                atomicAdd(&whist[wid][(int)((key >> shift) & 0xFF)], 1);
+        if (gathered) {
+            const int nc = n_cand;
+            for (int c = threadIdx.x; c < nc; c += TOPK_THREADS) {
+                const unsigned long long key = cand[c];
+                if ((key >> (shift + 8)) == (prefix >> (shift + 8))) atomicAdd(&whist[wid][(int)((key >> shift) & 0xFF)], 1);
+            }
+        } else {
+            for (int p = seg0 + lane; p < seg1; p += 32) {
+                const unsigned long long key = order_key(row[p]);
+                if (pass == 0 || (key >> (shift + 8)) == (prefix >> (shift + 8)))
+                    atomicAdd(&whist[wid][(int)((key >> shift) & 0xFF)], 1);
+            }
         }
         __syncthreads();
         if (threadIdx.x < 256) {
@@ -176,11 +189,21 @@ topk_kernel(const double* __restrict__ scores, int P, int k, int32_t* __restrict
                 }
                 sh_prefix = prefix | ((unsigned long long)d << shift);
                 sh_krem = k_rem - above;
+                sh_bin = hist[d];                      // keys that share all digits fixed so far
+                if (!gathered) n_cand = 0;
             }
         }
         __syncthreads();
         prefix = sh_prefix;
         k_rem = sh_krem;
+        if (!gathered && pass < 6 && sh_bin <= TOPK_CAND) {
+            for (int p = seg0 + lane; p < seg1; p += 32) {
+                const unsigned long long key = order_key(row[p]);
+                if ((key >> shift) == (prefix >> shift)) cand[atomicAdd(&n_cand, 1)] = key;
+            }
+            gathered = true;                           // (uniform over the CTA: sh_bin is)
+            __syncthreads();
+        }
     }
 
     // ordered compaction: positions ascending; among keys equal to the threshold the first k_rem.
