@@ -129,7 +129,7 @@ def _run_whole_path(w):
     return {n: t.cpu().numpy() for n, t in res.items()}
 
 
-@pytest.mark.parametrize("name,kv_heads,n_random", [("c1", [0, 7], 24), ("c2", [5], 16), ("c4", [2], 12), ("c3", [6], 4)])
+@pytest.mark.parametrize("name,kv_heads,n_random", [("c1", [0, 7], 24), ("c2", [2, 5], 16), ("c4", [2], 12), ("c3", [1, 6], 8)])
 def test_full_size_workloads_in_the_benchmark_launch_configuration(name, kv_heads, n_random):
     """Full benchmark sizes, all heads launched at once; the oracle recomputes whole (batch, KV head)
     groups for selection and quantization (bit-exact) and sampled rows of the attention output."""
