@@ -16,7 +16,7 @@
 namespace hyq {
 
 constexpr int FRZ_THREADS = 128;     // gather kernel; the quantizer runs 2 * G threads (64 elements per thread)
-constexpr int FRZ_WIN = 128;         // vertical indices staged per group for the source-row search
+constexpr int FRZ_QTHREADS_PER_SM = 896;   // quantizer threads resident per SM the register budget is set for (7 CTAs of 128)
 
 // Source position of compacted row p: p + j with j the number of vertical indices below it,
 // i.e. the smallest j with idx[j] - j > p (idx ascending, so idx[j] - j never decreases).
@@ -48,7 +48,7 @@ gather_rows_kernel(const uint4* __restrict__ k_, const uint4* __restrict__ v, co
 }
 
 template <int G, int FMT>
-__global__ void __launch_bounds__(2 * G)
+__global__ void __launch_bounds__(2 * G, FRZ_QTHREADS_PER_SM / (2 * G))
 freeze_quantize_kernel(const uint4* __restrict__ k_, const uint4* __restrict__ v, const int32_t* __restrict__ idx,
                        int N, int k_vl, int nQ, long nQp, uint8_t* __restrict__ kq, uint8_t* __restrict__ vq,
                        float* __restrict__ ks, float* __restrict__ vs) {
@@ -60,45 +60,42 @@ freeze_quantize_kernel(const uint4* __restrict__ k_, const uint4* __restrict__ v
 
     constexpr int NT = 2 * G;                                  // threads of this CTA
     __shared__ int src[G];
-    __shared__ int win[FRZ_WIN], j0_sh;
     __shared__ float warp_max[NT / 32];
     constexpr bool FMT8 = FMT != HYQ_FMT_INT4;                 // byte-wide codes (INT8 or FP8 e4m3)
     constexpr int ROW_BYTES = FMT8 ? HYQ_D : HYQ_D / 2;        // code bytes per row
     constexpr int TILE_BYTES = 16 * ROW_BYTES;                 // one 16-row V tile
     constexpr float CB = FMT == HYQ_FMT_INT8 ? 127.0f : FMT == HYQ_FMT_FP8_E4M3 ? 448.0f : 7.0f;
-    __shared__ __align__(16) uint8_t vtile[(G / 16) * TILE_BYTES];
-    // Source rows of the group's G compacted rows in three dependent memory round trips instead of ten:
-    // warp 0 finds j0 = the number of vertical rows before the group's first row by a 32-way search, a window of
-    // the index list starting there goes to shared memory, and each row finishes its own search in that window
-    // (a row whose answer lies beyond the window - long runs of vertical rows - falls back to the global search).
+    // V codes are staged row-major with 16 bytes of padding per row, so that both the row-wise stores and the
+    // word loads of the fragment-major write-out below spread over the banks
+    constexpr int VSTRIDE = ROW_BYTES + 16;
+    __shared__ __align__(16) uint8_t vstage[G * VSTRIDE];
+    // Source rows of the group's G compacted rows in two dependent memory round trips and a short scan: every warp
+    // finds j0 = the number of vertical rows before the group's first row by the same 32-way search (no hand-over
+    // between warps), then each row walks on from j0 through the few indices that fall inside the group (a row
+    // behind a long run of vertical rows falls back to the binary search).
     const int p0 = grp * G;
-    if (threadIdx.x < 32) {
+    int j0;
+    {
+        const int ln = threadIdx.x & 31;
         int lo = 0, hi = k_vl;                              // smallest j in [lo, hi] with idx[j] - j > p0
         while (lo < hi) {
             const int step = (hi - lo + 31) >> 5;
-            const int pos = lo + (int)threadIdx.x * step;
+            const int pos = lo + ln * step;
             const bool below = pos < hi && __ldg(hidx + pos) - pos <= p0;      // predicate still false at pos
             const int f = __popc(__ballot_sync(0xffffffffu, below));            // falses form a prefix of the lanes
             const int new_lo = f ? lo + (f - 1) * step + 1 : lo;
             const int new_hi = f == 0 ? lo : (f < 32 && lo + f * step < hi ? lo + f * step : hi);
             lo = new_lo; hi = new_hi;
         }
-        if (threadIdx.x == 0) j0_sh = lo;
+        j0 = lo;
     }
-    __syncthreads();
-    const int j0 = j0_sh;
-    for (int i = threadIdx.x; i < FRZ_WIN; i += NT) win[i] = j0 + i < k_vl ? __ldg(hidx + j0 + i) : 0x7fffffff;
-    __syncthreads();
     if (threadIdx.x < G) {
         const int p = p0 + threadIdx.x;
         int s = -1;
         if (p < nQ) {
-            int lo = 0, hi = FRZ_WIN;                       // smallest w with win[w] - (j0 + w) > p
-            while (lo < hi) {
-                const int mid = (lo + hi) >> 1;
-                if (win[mid] == 0x7fffffff || win[mid] - (j0 + mid) > p) hi = mid; else lo = mid + 1;
-            }
-            s = lo < FRZ_WIN ? p + j0 + lo : source_row(hidx, k_vl, p);
+            int j = j0, steps = 0;                          // smallest j >= j0 with idx[j] - j > p
+            while (j < k_vl && steps < 16 && __ldg(hidx + j) - j <= p) { ++j; ++steps; }
+            s = (steps < 16) ? p + j : source_row(hidx, k_vl, p);
             s = min(s, N - 1);                              // (only a malformed index list can reach the clamp)
         }
         src[threadIdx.x] = s;
@@ -143,55 +140,68 @@ freeze_quantize_kernel(const uint4* __restrict__ k_, const uint4* __restrict__ v
         const int row = u >> 3, ch0 = (u & 7) * 16;
         const uint32_t* w = reinterpret_cast<const uint32_t*>(&r[gi][0]);
         if (FMT8) {
-            uint8_t b[16];
+            uint32_t o[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
             for (int m = 0; m < 8; ++m) {
                 const float y0 = __fmul_rn(bf16_lo(w[m]), inv), y1 = __fmul_rn(bf16_hi(w[m]), inv);
+                uint32_t two;                                // codes of channels 2m (low byte) and 2m + 1
                 if (FMT == HYQ_FMT_FP8_E4M3) {
-                    const uint32_t two = dead ? 0u : __nv_cvt_float2_to_fp8x2(make_float2(y0, y1), __NV_SATFINITE, __NV_E4M3);   // no -0 in a zero group
-                    b[2 * m] = (uint8_t)(two & 0xFF);
-                    b[2 * m + 1] = (uint8_t)(two >> 8);
+                    two = dead ? 0u : __nv_cvt_float2_to_fp8x2(make_float2(y0, y1), __NV_SATFINITE, __NV_E4M3);   // no -0 in a zero group
                 } else {
-                    b[2 * m] = (uint8_t)max(-127, min(127, __float2int_rn(y0)));
-                    b[2 * m + 1] = (uint8_t)max(-127, min(127, __float2int_rn(y1)));
+                    two = (uint32_t)(max(-127, min(127, __float2int_rn(y0))) & 0xFF) |
+                          ((uint32_t)(max(-127, min(127, __float2int_rn(y1))) & 0xFF) << 8);
                 }
+                o[m >> 1] |= (two & 0xFFFFu) << (16 * (m & 1));
             }
-            if (!is_v) {
-                uint32_t o[4];
-#pragma unroll
-                for (int c4 = 0; c4 < 4; ++c4)
-                    o[c4] = b[4 * c4] | (b[4 * c4 + 1] << 8) | (b[4 * c4 + 2] << 16) | ((uint32_t)b[4 * c4 + 3] << 24);
-                *reinterpret_cast<uint4*>(kq + ((head * nQp + grp * G + row) * ROW_BYTES + ch0)) = make_uint4(o[0], o[1], o[2], o[3]);
-            } else {
-                const int tile = row >> 4, key = row & 15;
-#pragma unroll
-                for (int m = 0; m < 16; ++m) vtile[tile * TILE_BYTES + vq8_byte_offset(key, ch0 + m)] = b[m];
-            }
+            uint4* d4 = is_v ? reinterpret_cast<uint4*>(vstage + row * VSTRIDE + ch0)
+                             : reinterpret_cast<uint4*>(kq + ((head * nQp + grp * G + row) * ROW_BYTES + ch0));
+            *d4 = make_uint4(o[0], o[1], o[2], o[3]);
         } else {
-            uint8_t b[8];
+            uint32_t o[2] = {0u, 0u};
 #pragma unroll
             for (int m = 0; m < 8; ++m) {
                 const int q0 = max(-7, min(7, __float2int_rn(__fmul_rn(bf16_lo(w[m]), inv))));
                 const int q1 = max(-7, min(7, __float2int_rn(__fmul_rn(bf16_hi(w[m]), inv))));
-                b[m] = (uint8_t)((q0 & 0xF) | ((q1 & 0xF) << 4));
+                o[m >> 2] |= (uint32_t)((q0 & 0xF) | ((q1 & 0xF) << 4)) << (8 * (m & 3));
             }
-            if (!is_v) {
-                uint32_t o0 = b[0] | (b[1] << 8) | (b[2] << 16) | ((uint32_t)b[3] << 24);
-                uint32_t o1 = b[4] | (b[5] << 8) | (b[6] << 16) | ((uint32_t)b[7] << 24);
-                *reinterpret_cast<uint2*>(kq + ((head * nQp + grp * G + row) * ROW_BYTES + ch0 / 2)) = make_uint2(o0, o1);
-            } else {
-                const int tile = row >> 4, key = row & 15;
-#pragma unroll
-                for (int m = 0; m < 8; ++m) vtile[tile * TILE_BYTES + vq_byte_offset(key, ch0 + 2 * m)] = b[m];
-            }
+            uint2* d2 = is_v ? reinterpret_cast<uint2*>(vstage + row * VSTRIDE + ch0 / 2)
+                             : reinterpret_cast<uint2*>(kq + ((head * nQp + grp * G + row) * ROW_BYTES + ch0 / 2));
+            *d2 = make_uint2(o[0], o[1]);
         }
     }
     if (is_v) {
+        // Fragment-major write-out (the layouts of vq_byte_offset / vq8_byte_offset): 16-byte piece number 32 * run + l
+        // of a tile, l = 4r + j, is made of one 4-byte load from each of the rows 2j, 2j + 1, 2j + 8, 2j + 9 and
+        // a 4 x 4 (INT4) or 2 x 2 (byte codes) transpose of their bytes.
         __syncthreads();
         uint4* dst = reinterpret_cast<uint4*>(vq + (head * (nQp / 16) + grp * (G / 16)) * (long)TILE_BYTES);
-        const uint4* s4 = reinterpret_cast<const uint4*>(vtile);
+        constexpr int PIECES = TILE_BYTES / 16;
 #pragma unroll
-        for (int i = 0; i < (G / 16) * TILE_BYTES / 16 / NT; ++i) dst[threadIdx.x + i * NT] = s4[threadIdx.x + i * NT];
+        for (int i = 0; i < (G / 16) * PIECES / NT; ++i) {
+            const int o = threadIdx.x + i * NT;
+            const int tile = o / PIECES, run = (o % PIECES) >> 5, r = (o & 31) >> 2, j = o & 3;
+            const int col = FMT8 ? 64 * (run >> 1) + 8 * r + 4 * (run & 1) : 32 * run + 4 * r;
+            const uint8_t* base = vstage + (tile * 16 + 2 * j) * VSTRIDE + col;
+            const uint32_t e0 = *reinterpret_cast<const uint32_t*>(base);                  // row 2j
+            const uint32_t o0 = *reinterpret_cast<const uint32_t*>(base + VSTRIDE);        // row 2j + 1
+            const uint32_t e1 = *reinterpret_cast<const uint32_t*>(base + 8 * VSTRIDE);    // row 2j + 8
+            const uint32_t o1 = *reinterpret_cast<const uint32_t*>(base + 9 * VSTRIDE);    // row 2j + 9
+            uint4 out;
+            if (FMT8) {
+                out.x = __byte_perm(e0, o0, 0x5140);
+                out.y = __byte_perm(e1, o1, 0x5140);
+                out.z = __byte_perm(e0, o0, 0x7362);
+                out.w = __byte_perm(e1, o1, 0x7362);
+            } else {
+                const uint32_t t0 = __byte_perm(e0, e1, 0x5140), t1 = __byte_perm(e0, e1, 0x7362);
+                const uint32_t t2 = __byte_perm(o0, o1, 0x5140), t3 = __byte_perm(o0, o1, 0x7362);
+                out.x = __byte_perm(t0, t2, 0x5410);
+                out.y = __byte_perm(t0, t2, 0x7632);
+                out.z = __byte_perm(t1, t3, 0x5410);
+                out.w = __byte_perm(t1, t3, 0x7632);
+            }
+            dst[o] = out;
+        }
     }
 }
 
