@@ -188,6 +188,14 @@ def run_reference(args, w):
 
 
 
+def launches_per_step(w) -> int:
+    """Kernels of the library launched by one pass of the path: select 3, quantize 3, the attention pre-pass (bitmask,
+    V to fp16; with vertical keys the gather and, for FP8 / INT4 scores, the vertical-line operand tiles; 2 INT4
+    widenings when used) and the attention kernel."""
+    prepass = 1 + ((2 + (1 if w.q_fmt != wl.FMT_INT8 else 0)) if w.k > 0 else 0) + (2 if w.q_fmt == wl.FMT_INT4 else 0)
+    return 3 + 3 + prepass + 1
+
+
 def method_error_report(w, path, Q, K, V, n_random: int = 16):
     """Error of the METHOD against exact attention (all pairs in full precision), measured on the GPU's outputs: the
     hybrid operator as benchmarked, the same low-bit codes with neither vertical keys nor window (uniform low-bit) and
@@ -252,9 +260,7 @@ class DevicePath:
         for e_ in self.kev:
             e_.record()
         self.args.ev_kernel_start, self.args.ev_kernel_stop = (e_.cuda_event for e_ in self.kev)
-        # kernels launched by one step: select 3, quantize 3, attention pre-pass (bitmask, gather,
-        # V to fp16, and 2 INT4 widenings when used) + the attention kernel
-        self.launches_per_step = 3 + 3 + (3 if w.k > 0 else 1) + (2 if w.q_fmt == wl.FMT_INT4 else 0) + 1
+        self.launches_per_step = launches_per_step(w)
 
     def load(self, Q, K, V):
         self.Q.copy_(Q, non_blocking=True)
@@ -413,7 +419,7 @@ def run_query_block(args, w: wl.Workload):
                      "peak": flops / t_meas / 1e12, "unit": "TFLOP/s", "frac": t_meas * 1e3 / k_ms, "traffic": None,
                      "kernel_ms": k_ms, "frac_nominal": t_nom * 1e3 / k_ms, "fp_pair_share": n_fp / pairs,
                      "peak_source": peaks["source"]},
-        "gpu_launches": (3 + 3 + (3 if w.k > 0 else 1) + (2 if w.q_fmt == wl.FMT_INT4 else 0) + 1) * args.steps,
+        "gpu_launches": launches_per_step(w) * args.steps,
         "clocks": clocks}))
 
 

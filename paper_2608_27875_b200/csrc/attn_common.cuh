@@ -16,6 +16,9 @@ struct TcWorkspace {
     size_t vvl;         // fp16 [B*Hq][k][D]            gathered vertical-line V rows
     size_t q8;          // u8   [B*Hq][Lq][D]           INT4 only: Q codes as e4m3 bytes
     size_t k8;          // u8   [B*Hkv][L][D]           INT4 only: K codes as e4m3 bytes
+    size_t vl_tiles;    // u8   [B*Hq][mask_words/2][2048]  FP8 / INT4 scores only: per 64-key tile a 64 x 32 e5m2 operand, -inf in
+                        //                              element 0 of a vertical-line key's row, zero elsewhere (two 16-byte column
+                        //                              chunks, each [64 keys][16 bytes])
     size_t part_o;      // f32  [splits][B*Hq][Lq][D]   split keys only: partial accumulators ...
     size_t part_ml;     // f32  [splits][B*Hq][Lq][2]   ... and (reference maximum, row sum) per row
     size_t total;
@@ -38,6 +41,8 @@ struct TcTestHooks {
     int drop_load;
 };
 TcTestHooks tc_test_hooks();
+
+constexpr int VL_TILE_BYTES = 2048;
 
 // zero-fills bits[n_heads][mask_words] and sets one bit per vertical-line key (memset + one kernel)
 int launch_vl_bitmask(const int32_t* idx, long n_heads, int k, int L, int mask_words, uint32_t* bits, cudaStream_t st);

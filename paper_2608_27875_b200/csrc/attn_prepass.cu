@@ -109,6 +109,16 @@ __global__ void int4_to_e4m3_kernel(const uint32_t* __restrict__ packed, long n_
     out[e] = make_uint2(o[0], o[1]);
 }
 
+// one thread per vertical-line index: the byte 0xFC (-inf in e5m2) into element 0 of the key's row of its tile's operand
+__global__ void vl_mask_tiles_kernel(const int32_t* __restrict__ idx, long n_heads, int k, int L, int tiles_per_head,
+                                     uint8_t* __restrict__ tiles) {
+    const long e = (long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= n_heads * k) return;
+    const long head = e / k;
+    const int j = __ldg(idx + e);
+    if (j >= 0 && j < L) tiles[(head * tiles_per_head + (j >> 6)) * VL_TILE_BYTES + (j & 63) * 16] = 0xFC;
+}
+
 int launch_vl_bitmask(const int32_t* idx, long n_heads, int k, int L, int mask_words, uint32_t* bits, cudaStream_t st) {
     if (cudaMemsetAsync(bits, 0, (size_t)n_heads * mask_words * 4, st) != cudaSuccess) return HYQ_ERR_CUDA;
     if (k <= 0) return HYQ_OK;
@@ -145,6 +155,7 @@ TcWorkspace tc_workspace_layout(const hyq_attn_args& a) {
     const bool int4 = a.q_format == HYQ_FMT_INT4;
     w.q8 = int4 ? take(q_elems) : 0;
     w.k8 = int4 ? take(kv_elems) : 0;
+    w.vl_tiles = (a.q_format != HYQ_FMT_INT8 && a.k > 0) ? take((size_t)a.B * a.Hq * (w.mask_words / 2) * VL_TILE_BYTES) : 0;
     w.splits = tc_key_splits(a);
     const size_t rows = (size_t)a.B * a.Hq * query_rows(a);
     w.part_o = w.splits > 1 ? take((size_t)w.splits * rows * HYQ_D * 4) : 0;
@@ -163,6 +174,13 @@ int launch_tc_prepass(const hyq_attn_args& a, const TcWorkspace& w, cudaStream_t
         gather_vl_kernel<<<(unsigned)((n * 32 + 255) / 256), 256, 0, st>>>(
             static_cast<const __nv_bfloat16*>(a.k_), static_cast<const __nv_bfloat16*>(a.v), a.vl_idx, a.Hq, a.Hkv, a.L,
             a.k, n, reinterpret_cast<__nv_bfloat16*>(base + w.kvl), reinterpret_cast<__half*>(base + w.vvl));
+        if (launch_status() != HYQ_OK) return HYQ_ERR_CUDA;
+    }
+    if (a.q_format != HYQ_FMT_INT8 && a.k > 0) {
+        uint8_t* tiles = reinterpret_cast<uint8_t*>(base + w.vl_tiles);
+        if (cudaMemsetAsync(tiles, 0, (size_t)n_heads * (w.mask_words / 2) * VL_TILE_BYTES, st) != cudaSuccess) return HYQ_ERR_CUDA;
+        const long n = n_heads * a.k;
+        vl_mask_tiles_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(a.vl_idx, n_heads, a.k, a.L, w.mask_words / 2, tiles);
         if (launch_status() != HYQ_OK) return HYQ_ERR_CUDA;
     }
     const int nb = (a.L + a.block_tokens - 1) / a.block_tokens;

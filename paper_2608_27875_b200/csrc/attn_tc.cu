@@ -21,7 +21,11 @@
 // of its row in two register halves), so a row's reference maximum needs no agreement between
 // threads.  The exponentials are taken against that reference, which is only raised when
 // a tile exceeds it by more than 2^14 (the rescale of O is then rare); integer scores become floats
-// by a magic-number add.  Every mbarrier wait is bounded; when one expires the CTA records
+// by a magic-number add.  The vertical-line keys inside a low-bit tile are taken out of pass A before the
+// softmax sees the scores: with e4m3 codes by a fifth MMA step per tile, S += ones . mask^T in e5m2 (the one
+// 8-bit format with an infinity), whose 64 x 32 operand - -inf in element 0 of a vertical key's row - is copied
+// in with the K codes; with int8 codes (no infinity) by the softmax warps, which store -inf over those columns
+// of S before they read the tile.  Every mbarrier wait is bounded; when one expires the CTA records
 // HYQ_ERR_TIMEOUT in the status word, waits (bounded) for its own copies and MMAs in flight and unwinds.
 #include <cuda_fp16.h>
 
@@ -54,6 +58,10 @@ constexpr uint32_t SQ_OFF = 0, SQC_OFF = QT * Q_TILE_BYTES, SK_OFF = SQC_OFF + Q
 constexpr uint32_t SV_OFF = SK_OFF + RING_BYTES;
 constexpr uint32_t TILE_SMEM = SV_OFF + RING_BYTES;                 // 229376
 constexpr int MAX_STAGES = 4;
+// In the low-bit pass a K ring slot holds 8 KB of codes; behind them sit the vertical-line operand of the tile
+// (64 keys x 32 e5m2 elements, copied in with the codes) and this slot's copy of the constant 128 x 32 operand whose
+// element 0 of every row is one.
+constexpr uint32_t VLT_OFF = 8192, ONES_OFF = 10240, ONES_BYTES = 4096;
 
 // geometry that follows from the keys per tile (64: 4-stage ring, two S buffers per query tile)
 template <int TBN> struct Geo {
@@ -96,6 +104,7 @@ struct TcParams {
     const float* k_scales;
     const int32_t* vl_idx;
     const uint32_t* vl_bits;
+    const uint8_t* vl_tiles;     // FP8 / INT4 scores: the vertical-line operand tiles [B*Hq][mask_words/2][2048] (null: none)
     void* out;
     float* lse;
     int32_t* status;
@@ -159,7 +168,7 @@ __device__ __forceinline__ OwnTiles own_tiles(const QSched& s, const Walk& w) {
 // The loop body is kept to waits, MMAs and commits: ring positions, parities and descriptors advance incrementally.
 template <bool LOWBIT_FP8, int TBN>
 __device__ __forceinline__ bool mma_issuer(int q, const QSched& sq, const Walk& w, TcBarriers& bars, unsigned char* smem,
-                                           uint32_t tmem, volatile int* abort_flag, long long limit) {
+                                           uint32_t tmem, volatile int* abort_flag, long long limit, bool vl_mma) {
     using G = Geo<TBN>;
     constexpr int BN = TBN, NST = G::NST, NBUF = G::NBUF;
     constexpr uint32_t STAGE16 = G::STAGE_BYTES >> 4;                  // descriptor address units per ring stage
@@ -171,6 +180,10 @@ __device__ __forceinline__ bool mma_issuer(int q, const QSched& sq, const Walk& 
     const uint64_t dqc = make_smem_desc(smem_u32(smem + SQC_OFF + q * QC_TILE_BYTES), 0, 1024);
     const uint64_t dk0 = make_smem_desc(smem_u32(smem + SK_OFF), 0, 1024);
     const uint64_t dv0 = make_smem_desc(smem_u32(smem + SV_OFF), G::STAGE_BYTES / 2, 1024);
+    // S += ones . mask^T: -inf on the columns of vertical-line keys, +0 elsewhere (e5m2 has an infinity, e4m3 has not)
+    const uint32_t idesc_vl = make_idesc(ACC_F32, FMT_E5M2, FMT_E5M2, 0, 0, BM, BN);
+    const uint64_t dones0 = make_smem_desc_plain(smem_u32(smem + SK_OFF + ONES_OFF), BM * 16, 128);
+    const uint64_t dvlt0 = make_smem_desc_plain(smem_u32(smem + SK_OFF + VLT_OFF), BN * 16, 128);
     const uint32_t ts0 = tmem + tm_s(q), to = tmem + tm_o(q);
     const OwnTiles own = own_tiles(sq, w);
     const int nA = w.nA;
@@ -194,6 +207,7 @@ __device__ __forceinline__ bool mma_issuer(int q, const QSched& sq, const Walk& 
                     if (LOWBIT_FP8) umma_ss_f8f6f4(d, dqc + kk * 2, dk + kk * 2, idesc_lq, kk > 0);
                     else umma_ss_i8(d, dqc + kk * 2, dk + kk * 2, idesc_lq, kk > 0);
                 }
+                if (LOWBIT_FP8 && vl_mma) umma_ss_f8f6f4(d, dones0 + (uint64_t)(kst * STAGE16), dvlt0 + (uint64_t)(kst * STAGE16), idesc_vl, 1u);
             } else {
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk)
@@ -244,6 +258,7 @@ __device__ __forceinline__ bool mma_issuer(int q, const QSched& sq, const Walk& 
                     if (LOWBIT_FP8) umma_ss_f8f6f4(ts0 + bf * BN, dqc + kk * 2, dk0 + (uint64_t)(ks * STAGE16 + kk * 2), idesc_lq, kk > 0);
                     else umma_ss_i8(ts0 + bf * BN, dqc + kk * 2, dk0 + (uint64_t)(ks * STAGE16 + kk * 2), idesc_lq, kk > 0);
                 }
+                if (LOWBIT_FP8 && vl_mma) umma_ss_f8f6f4(ts0 + bf * BN, dones0 + (uint64_t)(ks * STAGE16), dvlt0 + (uint64_t)(ks * STAGE16), idesc_vl, 1u);
                 umma_commit_a(a_bars + (uint32_t)offsetof(TcBarriers, s_full) + (q * 2 + bf) * 8);
             }
             if (!ok) return false;
@@ -281,7 +296,7 @@ __device__ __forceinline__ bool mma_issuer(int q, const QSched& sq, const Walk& 
 template <int TBN>
 __device__ __forceinline__ bool tma_producer(const TcMaps& maps, const QSched& qs0, const QSched& qs1, const Walk& w, int qhead,
                                              int kvhead, TcBarriers& bars, unsigned char* smem, volatile int* abort_flag,
-                                             long long limit, int drop_load) {
+                                             long long limit, int drop_load, const uint8_t* vl_tiles) {
     using G = Geo<TBN>;
     constexpr int BN = TBN, NST = G::NST;
     prefetch_tmap(&maps.q);
@@ -310,9 +325,10 @@ __device__ __forceinline__ bool tma_producer(const TcMaps& maps, const QSched& q
         const int hd = vl ? qhead : kvhead;
         if (use > 0 && !mbar_wait_sleepy(&bars.kv_free[st], (use - 1) & 1, limit)) { ok = false; break; }
         if (lowbit) {
-            mbar_arrive_expect_tx(&bars.kv_full[st], G::KC_TILE_BYTES + G::STAGE_BYTES);
+            mbar_arrive_expect_tx(&bars.kv_full[st], G::KC_TILE_BYTES + G::STAGE_BYTES + (vl_tiles ? VL_TILE_BYTES : 0));
             if (t == drop_load) continue;                // test hook: the announced bytes never arrive
             tma_load_3d(sk, &maps.kc, &bars.kv_full[st], 0, row, hd);
+            if (vl_tiles) bulk_load_1d(sk + VLT_OFF, vl_tiles + (long)t * VL_TILE_BYTES, VL_TILE_BYTES, &bars.kv_full[st]);
         } else {
             const CUtensorMap* m = vl ? &maps.kvl : &maps.k;
             mbar_arrive_expect_tx(&bars.kv_full[st], 2 * G::STAGE_BYTES);
@@ -492,6 +508,21 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
     w.t0 = SPLIT ? (int)((long)w.T * split / p.splits) : 0;
     w.t1 = SPLIT ? (int)((long)w.T * (split + 1) / p.splits) : w.T;
 
+    // vertical-line keys of the low-bit pass: with e4m3 scores an extra MMA step per tile adds -inf to their columns
+    const uint8_t* vl_tiles_head = (LOWBIT_FP8 && p.vl_tiles) ? p.vl_tiles + (long)qhead * (p.mask_words / 2) * VL_TILE_BYTES : nullptr;
+    if (vl_tiles_head) {
+        // the constant operand of that step, one copy per ring slot whose first tile is a low-bit tile (the copy of a
+        // slot is overwritten by the slot's first full-precision tile, after which the slot holds no low-bit tile again)
+        const int n_slots = min(min(w.nA, w.t1) - w.t0, NST);
+        for (int c = threadIdx.x; c < n_slots * (int)(ONES_BYTES / 16); c += TC_THREADS) {
+            const int slot = c / (int)(ONES_BYTES / 16), chunk = c % (int)(ONES_BYTES / 16);   // chunks 0..127: element 0..15 of row `chunk`
+            *reinterpret_cast<uint4*>(smem + SK_OFF + slot * G::STAGE_BYTES + ONES_OFF + chunk * 16) =
+                make_uint4(chunk < BM ? 0x3Cu : 0u, 0u, 0u, 0u);                               // 0x3C = 1.0 in e5m2
+        }
+        fence_proxy_async_smem();
+    }
+    __syncthreads();
+
     volatile int* abort_flag = &abort_s;
     auto fail = [&]() {
         *abort_flag = 1;
@@ -500,11 +531,11 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
 
     // the single-thread roles sit in the lowest warps (the softmax warps 4..19 keep warp % 4 = TMEM lane quarter)
     if (warp == 0) {
-        if (lane == 0 && !tma_producer<TBN>(maps, qs0, qs1, w, qhead, kvhead, bars, smem, abort_flag, limit, p.drop_load)) fail();
+        if (lane == 0 && !tma_producer<TBN>(maps, qs0, qs1, w, qhead, kvhead, bars, smem, abort_flag, limit, p.drop_load, vl_tiles_head)) fail();
     } else if (warp == 1 || warp == 2) {
         if (lane == 0) {
             const int q = warp - 1;
-            const bool ok = mma_issuer<LOWBIT_FP8, TBN>(q, q ? qs1 : qs0, w, bars, smem, tmem, abort_flag, limit);
+            const bool ok = mma_issuer<LOWBIT_FP8, TBN>(q, q ? qs1 : qs0, w, bars, smem, tmem, abort_flag, limit, vl_tiles_head != nullptr);
             if (!ok || *abort_flag) {
                 // leaving early: none of this thread's MMAs may be in flight when the CTA gives up its tensor memory
                 umma_commit(&bars.drain[q]);
@@ -577,7 +608,7 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
 #else
                 nks = __ldg(ks_ptr + n);
 #endif
-                nvl = (uint64_t)__ldg(vl_ptr + 2 * n) | ((uint64_t)__ldg(vl_ptr + 2 * n + 1) << 32);
+                if (!LOWBIT_FP8) nvl = (uint64_t)__ldg(vl_ptr + 2 * n) | ((uint64_t)__ldg(vl_ptr + 2 * n + 1) << 32);
             };
             prefetch_tile(n0);
             const float qs2 = q_scale * p.scale_log2;
@@ -596,7 +627,7 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                 }
                 tc_fence_after();
                 // vertical-line keys of a low-bit tile: -inf into their S columns before the row is read
-                if (vl != 0ull) {                                // uniform over the warp
+                if (!LOWBIT_FP8 && vl != 0ull) {                 // uniform over the warp (e4m3 scores: the issuer's extra MMA step did it)
                     while (vl) { const int c = __ffsll((long long)vl) - 1; vl &= vl - 1; tmem_st1(ts + c, knock_lq); }
                     tmem_wait_st();
                 }
@@ -875,6 +906,7 @@ int launch_attn_tc(const hyq_attn_args& a, float alpha, cudaStream_t st) {
     p.scale_log2 = alpha * 1.4426950408889634f;
     p.q_scales = a.q_scales; p.k_scales = a.k_scales; p.vl_idx = a.vl_idx;
     p.vl_bits = reinterpret_cast<const uint32_t*>(base + w.vl_bits);
+    p.vl_tiles = (a.q_format != HYQ_FMT_INT8 && a.k > 0) ? reinterpret_cast<const uint8_t*>(base + w.vl_tiles) : nullptr;
     p.out = a.out; p.lse = a.lse; p.status = a.status_word;
     const TcTestHooks hooks = tc_test_hooks();
     p.wait_limit = hooks.wait_limit > 0 ? hooks.wait_limit : WAIT_LIMIT_DEFAULT;
