@@ -191,9 +191,10 @@ def run_reference(args, w):
 def launches_per_step(w) -> int:
     """Kernels of the library launched by one pass of the path: select 3, quantize 3, the attention pre-pass (bitmask,
     V to fp16; with vertical keys the gather and, for FP8 / INT4 scores, the vertical-line operand tiles; 2 INT4
-    widenings when used) and the attention kernel."""
+    widenings when used) and the attention kernel (two launches with FP8 / INT4 scores)."""
     prepass = 1 + ((2 + (1 if w.q_fmt != wl.FMT_INT8 else 0)) if w.k > 0 else 0) + (2 if w.q_fmt == wl.FMT_INT4 else 0)
-    return 3 + 3 + prepass + 1
+    attention = 1 if w.q_fmt == wl.FMT_INT8 else 2      # FP8 / INT4 scores: the second launch that goes through the redo list
+    return 3 + 3 + prepass + attention
 
 
 def method_error_report(w, path, Q, K, V, n_random: int = 16):

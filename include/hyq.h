@@ -277,6 +277,16 @@ int hyq_hybrid_attention_prefill_varlen(const hyq_attn_args* args, int n_seq, co
  * ------------------------------------------------------------------------------------------- */
 int hyq_test_set_attention_hooks(long long wait_limit_clocks, int drop_load_position);
 
+/* ---------------------------------------------------------------------------------------------
+ * hyq_test_read_attention_restarts - test hook (the paper has no counterpart).  The tensor-core kernel takes the
+ * exponentials of most low-bit tiles against a row's reference as it stands and checks each tile's row sum
+ * afterwards; a CTA in which some row's sum shows an fp16 overflow (a score more than 2^16 above all the row had
+ * seen) discards its work and goes through its keys a second time with the maximum looked at in every tile.  This
+ * call synchronises the device and returns in *count_out (host) how many CTAs have done so since the library was
+ * loaded or the counter was last reset (reset != 0 clears it).  Errors: INVALID_ARG (null pointer), CUDA.
+ * ------------------------------------------------------------------------------------------- */
+int hyq_test_read_attention_restarts(unsigned long long* count_out /* host */, int reset);
+
 #ifdef __cplusplus
 }
 #endif

@@ -20,7 +20,7 @@ WINDOW_SLIDING, WINDOW_FIXED_TAIL = 0, 1
 EXPORTS = ("hyq_status_string", "hyq_version", "hyq_paper_k", "hyq_select_vertical_workspace",
            "hyq_select_vertical", "hyq_select_vertical_static", "hyq_select_vertical_mass_workspace",
            "hyq_select_vertical_mass", "hyq_quantize_blocks", "hyq_hybrid_attention_prefill_workspace",
-           "hyq_hybrid_attention_prefill", "hyq_test_set_attention_hooks", "hyq_select_vertical_varlen",
+           "hyq_hybrid_attention_prefill", "hyq_test_set_attention_hooks", "hyq_test_read_attention_restarts", "hyq_select_vertical_varlen",
            "hyq_quantize_blocks_varlen", "hyq_hybrid_attention_prefill_varlen")
 
 
@@ -71,6 +71,7 @@ def lib() -> ctypes.CDLL:
         L.hyq_hybrid_attention_prefill_workspace.argtypes = [ctypes.POINTER(AttnArgs), ctypes.POINTER(ctypes.c_size_t)]
         L.hyq_hybrid_attention_prefill.argtypes = [ctypes.POINTER(AttnArgs), ctypes.c_void_p]
         L.hyq_test_set_attention_hooks.argtypes = [ctypes.c_longlong, ctypes.c_int]
+        L.hyq_test_read_attention_restarts.argtypes = [ctypes.POINTER(ctypes.c_ulonglong), ctypes.c_int]
         i32p = ctypes.POINTER(ctypes.c_int32)
         L.hyq_select_vertical_varlen.argtypes = ([ctypes.c_void_p] * 2 + [ctypes.c_int, i32p] + [ctypes.c_int] * 5 + [i32p] +
                                                  [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p])
@@ -170,6 +171,13 @@ def hyq_select_vertical_static(q: torch.Tensor, k: torch.Tensor, window: int, k_
     _check(lib().hyq_select_vertical_static(q.data_ptr(), k.data_ptr(), B, Hq, Hkv, Lq, Lk, D, window, n_tail, k_eff,
                                             out.data_ptr(), _stream()), "hyq_select_vertical_static")
     return out
+
+
+def hyq_test_read_attention_restarts(reset: bool = False) -> int:
+    """Test hook: CTAs of the tensor-core kernel that have gone through their keys a second time (synchronises the device)."""
+    n = ctypes.c_ulonglong(0)
+    _check(lib().hyq_test_read_attention_restarts(ctypes.byref(n), 1 if reset else 0), "hyq_test_read_attention_restarts")
+    return int(n.value)
 
 
 def hyq_test_set_attention_hooks(wait_limit_clocks: int = 0, drop_load_position: int = -1) -> None:

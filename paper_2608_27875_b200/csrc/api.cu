@@ -8,8 +8,10 @@ size_t attn_simt_workspace_bytes(const hyq_attn_args& a);
 int launch_attn_simt(const hyq_attn_args& a, float alpha, cudaStream_t st);
 size_t attn_tc_workspace_bytes(const hyq_attn_args& a);
 int launch_attn_tc(const hyq_attn_args& a, float alpha, cudaStream_t st);
+int tc_restarts(unsigned long long* count, bool reset);
 namespace tcbt {
 int launch_attn_tc(const hyq_attn_args& a, float alpha, cudaStream_t st);     // 32- and 128-token quantization blocks
+int tc_restarts(unsigned long long* count, bool reset);
 }
 }  // namespace hyq
 
@@ -41,6 +43,14 @@ int hyq_test_set_attention_hooks(long long wait_limit_clocks, int drop_load_posi
     if (wait_limit_clocks < 0 || drop_load_position < -1) return HYQ_ERR_INVALID_ARG;
     g_tc_hooks.wait_limit = wait_limit_clocks;
     g_tc_hooks.drop_load = drop_load_position;
+    return HYQ_OK;
+}
+
+int hyq_test_read_attention_restarts(unsigned long long* count_out, int reset) {
+    if (!count_out) return HYQ_ERR_INVALID_ARG;
+    unsigned long long a = 0ull, b = 0ull;
+    if (tc_restarts(&a, reset != 0) != HYQ_OK || tcbt::tc_restarts(&b, reset != 0) != HYQ_OK) return HYQ_ERR_CUDA;
+    *count_out = a + b;
     return HYQ_OK;
 }
 

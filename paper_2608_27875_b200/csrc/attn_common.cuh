@@ -19,6 +19,7 @@ struct TcWorkspace {
     size_t vl_tiles;    // u8   [B*Hq][mask_words/2][2048]  FP8 / INT4 scores only: per 64-key tile a 64 x 32 e5m2 operand, -inf in
                         //                              element 0 of a vertical-line key's row, zero elsewhere (two 16-byte column
                         //                              chunks, each [64 keys][16 bytes])
+    size_t redo;        // u32  [1 + 3 * CTAs]          block indices of the CTAs whose work the second launch does again, behind their count
     size_t part_o;      // f32  [splits][B*Hq][Lq][D]   split keys only: partial accumulators ...
     size_t part_ml;     // f32  [splits][B*Hq][Lq][2]   ... and (reference maximum, row sum) per row
     size_t total;

@@ -157,6 +157,7 @@ TcWorkspace tc_workspace_layout(const hyq_attn_args& a) {
     w.k8 = int4 ? take(kv_elems) : 0;
     w.vl_tiles = (a.q_format != HYQ_FMT_INT8 && a.k > 0) ? take((size_t)a.B * a.Hq * (w.mask_words / 2) * VL_TILE_BYTES) : 0;
     w.splits = tc_key_splits(a);
+    w.redo = take((1 + 3 * (size_t)((query_rows(a) + 255) / 256) * w.splits * a.Hq * a.B) * 4);
     const size_t rows = (size_t)a.B * a.Hq * query_rows(a);
     w.part_o = w.splits > 1 ? take((size_t)w.splits * rows * HYQ_D * 4) : 0;
     w.part_ml = w.splits > 1 ? take((size_t)w.splits * rows * 2 * 4) : 0;

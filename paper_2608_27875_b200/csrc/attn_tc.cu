@@ -84,6 +84,9 @@ constexpr float INT_MAGIC_F = 12582912.0f;
 constexpr uint32_t KNOCKOUT_F32 = 0xFF800000u;       // -inf
 constexpr uint32_t KNOCKOUT_S32 = KNOCKOUT_F32 - INT_MAGIC;   // becomes -inf after the magic add
 
+// CTAs whose work was done a second time by the exact kernel (read and reset by the test hook)
+__device__ unsigned long long g_tc_restarts = 0ull;
+
 struct TcMaps {
     CUtensorMap q, k, qc, kc, v16, vh16, kvl, vvl;
 };
@@ -104,6 +107,8 @@ struct TcParams {
     const float* k_scales;
     const int32_t* vl_idx;
     const uint32_t* vl_bits;
+    uint32_t* redo;              // [0]: number of CTAs of the optimistic kernel that gave up, [1 + 3 i ...]: their block indices
+    int grid_x;                  // blockIdx.x range of the optimistic kernel (pairs of query tiles x slices)
     const uint8_t* vl_tiles;     // FP8 / INT4 scores: the vertical-line operand tiles [B*Hq][mask_words/2][2048] (null: none)
     void* out;
     float* lse;
@@ -296,7 +301,7 @@ __device__ __forceinline__ bool mma_issuer(int q, const QSched& sq, const Walk& 
 template <int TBN>
 __device__ __forceinline__ bool tma_producer(const TcMaps& maps, const QSched& qs0, const QSched& qs1, const Walk& w, int qhead,
                                              int kvhead, TcBarriers& bars, unsigned char* smem, volatile int* abort_flag,
-                                             long long limit, int drop_load, const uint8_t* vl_tiles) {
+                                             long long limit, int drop_load, const uint8_t* vl_tiles, bool settle) {
     using G = Geo<TBN>;
     constexpr int BN = TBN, NST = G::NST;
     prefetch_tmap(&maps.q);
@@ -344,6 +349,11 @@ __device__ __forceinline__ bool tma_producer(const TcMaps& maps, const QSched& q
         // leaving early: wait (bounded) for the copies still on their way into this CTA's shared memory
         mbar_wait_sleepy(&bars.q_full, 0, limit);
         for (int u = max(t - w.t0 - NST, 0); u < t - w.t0; ++u) mbar_wait_sleepy(&bars.kv_full[u % NST], (u / NST) & 1, limit);
+    } else if (settle) {
+        // every stage released for the last time: no arrival is on its way to a ring barrier any more (the CTA goes on
+        // to another piece of work on re-initialised barriers)
+        for (int u = max(t - w.t0 - NST, 0); u < t - w.t0; ++u)
+            if (!mbar_wait_sleepy(&bars.kv_free[u % NST], (u / NST) & 1, limit)) { ok = false; break; }
     }
     return ok;
 }
@@ -353,6 +363,7 @@ __device__ __forceinline__ bool tma_producer(const TcMaps& maps, const QSched& q
 // reference when the tile's maximum exceeds it by more than the threshold (rescaling O and the row sum), and writes the
 // 64 probabilities as fp16 pairs over the first 32 columns of the buffer it read.
 constexpr int TC_THREADS = 384;                     // TMA producer, 2 MMA issuers, 1 idle warp, 8 softmax warps
+constexpr float P_SUM_LIMIT = 65504.0f;             // a tile's row sum below the largest fp16 number: none of its P overflowed
 constexpr float RAISE_THRESHOLD = 14.0f;            // log2 units by which a tile must exceed the reference to raise it (P stays below 2^14, inside fp16)
 
 // row maximum of 32 float scores held in registers
@@ -427,23 +438,39 @@ __device__ __forceinline__ void mask_cols32(uint32_t (&raw)[32], int c0, int lo_
 // 2.6 % on the benchmark workload).
 // SPLIT (short query blocks only): several CTAs share a pair of query tiles, each on a contiguous slice of the
 // walk; they leave unnormalised partial results that attn_merge_kernel combines by their reference maxima.
-template <bool LOWBIT_FP8, bool QUERY_BLOCK, bool SPLIT = false>
+// EXACT = false is the kernel of the first launch: one CTA per block index.  After the first tiles of a row's low-bit pass
+// it takes the exponentials against the row's reference as it stands, without looking for the tile's maximum, and
+// every tile's row sum tells afterwards whether that was safe (no P beyond fp16).  If it was not for any row of the
+// CTA - a score more than 2^16 above everything the row had seen - the CTA writes no output and puts its block
+// index on a list.  EXACT = true is the kernel of the second launch, a small grid that goes through that list
+// (normally empty) with the maximum looked at in every tile.
+template <bool LOWBIT_FP8, bool QUERY_BLOCK, bool SPLIT = false, bool EXACT = false>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
     constexpr int TBN = 64, BN = 64;
+    if (EXACT && p.redo[0] == 0u) return;
     using G = Geo<TBN>;
     constexpr int NST = G::NST;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     __shared__ TcBarriers bars;
     __shared__ uint32_t tmem_base_s;
-    __shared__ int abort_s, cnt_b_s[QT];
+    __shared__ int abort_s, restart_s, cnt_b_s[QT];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int pt_lin = gridDim.x - 1 - blockIdx.x;           // pair of query tiles (and slice); longest rows first
+    if (warp == 0) {
+        tmem_alloc(&tmem_base_s, TM_COLS);
+        tmem_relinquish();
+    }
+    if (threadIdx.x == 0) abort_s = 0;
+    const uint32_t n_items = EXACT ? p.redo[0] : 1u;
+#pragma unroll 1
+    for (uint32_t item = EXACT ? blockIdx.x : 0u; item < n_items; item += (EXACT ? gridDim.x : 1u)) {
+    const int bx = EXACT ? (int)p.redo[1 + 3 * item] : (int)blockIdx.x;
+    const int h = EXACT ? (int)p.redo[2 + 3 * item] : (int)blockIdx.y, b = EXACT ? (int)p.redo[3 + 3 * item] : (int)blockIdx.z;
+    const int pt_lin = p.grid_x - 1 - bx;                    // pair of query tiles (and slice); longest rows first
     const int pt = SPLIT ? pt_lin / p.splits : pt_lin;
     const int split = SPLIT ? pt_lin % p.splits : 0;
-    const int h = blockIdx.y, b = blockIdx.z;
     const int L = p.Lq, W = p.window, g = p.Hq / p.Hkv;     // L: rows of the query block
     const int off = QUERY_BLOCK ? p.L - p.Lq : 0;           // position of query row 0 among the keys
     const long long limit = p.wait_limit;
@@ -471,15 +498,12 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
             mbar_init(&bars.drain[q], 1);
         }
         fence_mbar_init();
-        abort_s = 0;
+        restart_s = 0;
+        if (EXACT) atomicAdd(&g_tc_restarts, 1ull);
     }
     if (threadIdx.x < QT) {
         const int a1 = off + min(pt * QT * BM + (int)threadIdx.x * BM + BM - 1, L - 1);
         cnt_b_s[threadIdx.x] = (p.k > 0 && qhi(a1) >= 0) ? count_le(idx_row, p.k, qhi(a1)) : 0;
-    }
-    if (warp == 0) {
-        tmem_alloc(&tmem_base_s, TM_COLS);
-        tmem_relinquish();
     }
     tc_fence_before();
     __syncthreads();
@@ -524,6 +548,7 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
     __syncthreads();
 
     volatile int* abort_flag = &abort_s;
+    volatile int* restart_flag = &restart_s;
     auto fail = [&]() {
         *abort_flag = 1;
         if (p.status) atomicExch(p.status, HYQ_ERR_TIMEOUT);
@@ -531,15 +556,16 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
 
     // the single-thread roles sit in the lowest warps (the softmax warps 4..19 keep warp % 4 = TMEM lane quarter)
     if (warp == 0) {
-        if (lane == 0 && !tma_producer<TBN>(maps, qs0, qs1, w, qhead, kvhead, bars, smem, abort_flag, limit, p.drop_load, vl_tiles_head)) fail();
+        if (lane == 0 && !tma_producer<TBN>(maps, qs0, qs1, w, qhead, kvhead, bars, smem, abort_flag, limit, p.drop_load, vl_tiles_head, EXACT)) fail();
     } else if (warp == 1 || warp == 2) {
         if (lane == 0) {
             const int q = warp - 1;
             const bool ok = mma_issuer<LOWBIT_FP8, TBN>(q, q ? qs1 : qs0, w, bars, smem, tmem, abort_flag, limit, vl_tiles_head != nullptr);
-            if (!ok || *abort_flag) {
-                // leaving early: none of this thread's MMAs may be in flight when the CTA gives up its tensor memory
+            if (EXACT || !ok || *abort_flag) {
+                // leaving early, or going on to another piece of work: none of this thread's MMAs, and none of their
+                // arrivals at barriers, may be on its way when the CTA gives up its tensor memory or initialises its barriers again
                 umma_commit(&bars.drain[q]);
-                mbar_wait(&bars.drain[q], 0, limit);
+                if (!mbar_wait(&bars.drain[q], 0, limit) && ok) fail();
             }
             if (!ok) fail();
         }
@@ -548,6 +574,21 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
         const int q = (warp - 4) >> 2;                          // query tile (a thread owns all 64 columns of its row)
         const QSched sq = q ? qs1 : qs0;
         const OwnTiles own = own_tiles(sq, w);
+        // first launch: the CTA's eight softmax warps agree whether any row's exponentials overflowed; if so the CTA's
+        // block index goes on the list of the second launch and nothing is written
+        auto agree = [&](bool over_any) -> bool {
+            if (EXACT || !LOWBIT_FP8) return false;
+            if (__any_sync(0xffffffffu, over_any) && lane == 0) *restart_flag = 1;
+            bar_sync_named(1, 8 * 32);
+            const bool again = *restart_flag != 0 && *abort_flag == 0;
+            if (again && warp == 4 && lane == 0) {
+                const uint32_t slot = atomicAdd(p.redo, 1u);
+                p.redo[1 + 3 * slot] = (uint32_t)bx;
+                p.redo[2 + 3 * slot] = (uint32_t)h;
+                p.redo[3 + 3 * slot] = (uint32_t)b;
+            }
+            return again;
+        };
         // own tiles of this CTA: numbers [n0, n_total) in the query tile's own list (all of it unless the keys are split)
         const int n0 = SPLIT ? own_before(own, w.t0) : 0;
         const int n_total = SPLIT ? own_before(own, w.t1) : own.a_end + (own.b_end - own.b_beg) + (own.c_end - own.c_beg);
@@ -555,7 +596,7 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
             // nothing of this query tile lies in the slice: an empty partial result
             const int i = sq.i0 + (warp & 3) * 32 + lane;
             if (i < L)
-                reinterpret_cast<float2*>(p.part_ml)[((long)split * gridDim.y * gridDim.z + qhead) * L + i] = make_float2(-INFINITY, 0.0f);
+                reinterpret_cast<float2*>(p.part_ml)[((long)split * p.Hq * p.B + qhead) * L + i] = make_float2(-INFINITY, 0.0f);
         }
         if (sq.live && n_total > n0) {
             const int r = (warp & 3) * 32 + lane;               // query row inside the tile = TMEM lane
@@ -572,7 +613,8 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
             const float q_scale = row_live ? __ldg(p.q_scales + (long)qhead * p.nbq + i / HYQ_BLOCK_TOKENS) : 0.0f;
 #endif
             constexpr uint32_t knock_lq = LOWBIT_FP8 ? KNOCKOUT_F32 : KNOCKOUT_S32;
-            float m_used = -INFINITY, l_h = 0.0f;               // reference maximum of the row; row sum of this half
+            float m_used = -INFINITY, l_h = 0.0f;               // reference maximum of the row; row sum
+            bool over = false;                                  // a tile taken without its maximum had a row sum beyond fp16
             bool dead = false;                                  // this warp ran into an expired wait
             bool aborted = false;
 
@@ -615,7 +657,7 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
 
             // one tile of the online softmax for this thread's row: all 64 columns, in two register halves.  Returns
             // false when this warp ran into an expired wait.
-            auto do_tile = [&](auto range_tag, int n, float cs, uint64_t vl, bool int_scores, int lo_eff, unsigned span) -> bool {
+            auto do_tile = [&](auto range_tag, int n, float cs, uint64_t vl, bool int_scores, int lo_eff, unsigned span, bool skip_max = false) -> bool {
                 constexpr bool NEED_RANGE = decltype(range_tag)::value;
                 const uint32_t knock = int_scores ? KNOCKOUT_S32 : KNOCKOUT_F32;
                 const int nl = n - n0;                          // tile number within this CTA's slice
@@ -647,6 +689,9 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                 }
 #if HYQ_TC_VARIANT_BT
                 const float csb = cs_hi;                        // the second half's factor (its own K scale with 32-token blocks)
+#endif
+                if (!skip_max) {                                // (skipped: exponentials against the reference as it stands)
+#if HYQ_TC_VARIANT_BT
                 const float fa = row_max32(ra) - (int_scores ? INT_MAGIC_F : 0.0f), fb = row_max32(rb) - (int_scores ? INT_MAGIC_F : 0.0f);
                 const float mt = fmaxf((fa == -INFINITY) ? -INFINITY : fa * cs, (fb == -INFINITY) ? -INFINITY : fb * csb);
 #else
@@ -681,17 +726,20 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                         m_used = mt;
                     }
                 }
+                }
                 // ---- P = 2^(s - m) as fp16 pairs over the first 32 columns of the buffer; row sum
                 const float m_eff = (m_used == -INFINITY) ? 0.0f : m_used;
                 const float bias = int_scores ? fmaf(-INT_MAGIC_F, cs, -m_eff) : -m_eff;
                 uint32_t pa[16], pb[16];
-                l_h += row_exp32(ra, cs, bias, pa);
+                const float t_a = row_exp32(ra, cs, bias, pa);
                 tmem_st16(ts, pa);
 #if HYQ_TC_VARIANT_BT
-                l_h += row_exp32(rb, csb, int_scores ? fmaf(-INT_MAGIC_F, csb, -m_eff) : -m_eff, pb);
+                const float t_b = row_exp32(rb, csb, int_scores ? fmaf(-INT_MAGIC_F, csb, -m_eff) : -m_eff, pb);
 #else
-                l_h += row_exp32(rb, cs, bias, pb);
+                const float t_b = row_exp32(rb, cs, bias, pb);
 #endif
+                l_h += t_a + t_b;
+                if (!EXACT && LOWBIT_FP8) over |= !(t_a + t_b < P_SUM_LIMIT);               // (an overflowed or undefined sum included)
                 tmem_st16(ts + 16, pb);
                 tmem_wait_st();
                 tc_fence_before();
@@ -703,6 +751,8 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
             // ---- low-bit tiles that lie wholly below every row's window: no range mask, no bounds to compute
             const int n_plain = ragged ? 0 : min(own.a_end, max(0, (qhi(sq.i0 + off) + 1) / BN));
             int n = n0;
+            // (first launch: once every row of the warp has a finite reference, the plain tiles go without their maximum)
+            bool warm = false;
             for (; n < min(n_plain, n_total); ++n) {
                 // a zero scale (all-zero tile) still has to let -inf pass through the multiply
                 const float cs = fmaxf(qs2 * nks, 1e-37f);
@@ -711,7 +761,8 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
 #endif
                 const auto vl = nvl;
                 prefetch_tile(n + 1);
-                if (!do_tile(std::false_type{}, n, cs, vl, !LOWBIT_FP8, 0, 0u)) { aborted = true; break; }
+                if (!do_tile(std::false_type{}, n, cs, vl, !LOWBIT_FP8, 0, 0u, LOWBIT_FP8 && warm)) { aborted = true; break; }
+                if (!EXACT && LOWBIT_FP8 && !warm && n - n0 >= 1) warm = __all_sync(0xffffffffu, m_used > -INFINITY);
             }
             // ---- the remaining low-bit tiles, the vertical-line tiles and the window tiles
             // (number of vertical-line keys this row may use: only needed from here on)
@@ -756,14 +807,15 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
             // ---- epilogue: the last P.V (MMAs complete in order), sum of the two halves' row sums, O / l
             bool ok = !aborted && !dead;
             if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars.o_done[q][(n_total - n0 - 1) & 1], (uint32_t)((n_total - n0 - 1) >> 1) & 1u, limit));
-            if (!aborted) {                                     // uniform over the query tile's softmax warps
+            const bool again = agree(over);
+            if (!aborted && !again) {                           // uniform over the query tile's softmax warps
                 tc_fence_after();
                 constexpr int NCH = 4;                          // 32-channel pieces of the row this thread writes
                 const float l_run = l_h;
                 const float inv = (l_run > 0.0f) ? 1.0f / l_run : 0.0f;
                 if (SPLIT) {
                     // partial result of this slice: O as accumulated (relative to m_used), the pair (m_used, l)
-                    const long prow = ((long)split * gridDim.y * gridDim.z + qhead) * L + i;
+                    const long prow = ((long)split * p.Hq * p.B + qhead) * L + i;
                     if (ok) {
 #pragma unroll
                         for (int c = 0; c < NCH; ++c) {
@@ -813,14 +865,21 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                 }
             }
             if (!ok) fail();
+        } else {
+            agree(false);                                       // (a query tile with nothing to do still takes part)
         }
     }
 
     tc_fence_before();
     __syncthreads();
+    tc_fence_after();
+    if (EXACT && abort_s) break;
+    }
+    tc_fence_before();
+    __syncthreads();
     if (warp == 0) {
         __syncwarp();
-        tmem_dealloc(tmem, TM_COLS);
+        tmem_dealloc(tmem_base_s, TM_COLS);
     }
 }
 
@@ -860,6 +919,14 @@ attn_merge_kernel(const float* __restrict__ part_o, const float* __restrict__ pa
 
 // ---------------------------------------------------------------------------------------------
 size_t attn_tc_workspace_bytes(const hyq_attn_args& a) { return tc_workspace_layout(a).total; }
+
+// CTAs of this translation unit's kernels whose work was done a second time (synchronises the device)
+int tc_restarts(unsigned long long* count, bool reset) {
+    if (cudaMemcpyFromSymbol(count, g_tc_restarts, sizeof(*count)) != cudaSuccess) return HYQ_ERR_CUDA;
+    const unsigned long long zero = 0ull;
+    if (reset && cudaMemcpyToSymbol(g_tc_restarts, &zero, sizeof(zero)) != cudaSuccess) return HYQ_ERR_CUDA;
+    return HYQ_OK;
+}
 
 int launch_attn_tc(const hyq_attn_args& a, float alpha, cudaStream_t st) {
     constexpr int TBN = 64;                                             // keys per tile
@@ -919,12 +986,25 @@ int launch_attn_tc(const hyq_attn_args& a, float alpha, cudaStream_t st) {
     auto kern = split ? (lowbit_fp8 ? attn_tc_kernel<true, true, true> : attn_tc_kernel<false, true, true>)
               : lowbit_fp8 ? (blk ? attn_tc_kernel<true, true> : attn_tc_kernel<true, false>)
                            : (blk ? attn_tc_kernel<false, true> : attn_tc_kernel<false, false>);
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM_BYTES) != cudaSuccess)
+    // the same instantiation for the second launch (every maximum looked at; works through the first launch's list)
+    auto kern_exact = split ? (lowbit_fp8 ? attn_tc_kernel<true, true, true, true> : attn_tc_kernel<false, true, true, true>)
+                    : lowbit_fp8 ? (blk ? attn_tc_kernel<true, true, false, true> : attn_tc_kernel<true, false, false, true>)
+                                 : (blk ? attn_tc_kernel<false, true, false, true> : attn_tc_kernel<false, false, false, true>);
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM_BYTES) != cudaSuccess ||
+        cudaFuncSetAttribute(kern_exact, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM_BYTES) != cudaSuccess)
         return HYQ_ERR_CUDA;
     const dim3 grid((((int)Lq + QT * BM - 1) / (QT * BM)) * w.splits, a.Hq, a.B);
+    p.grid_x = (int)grid.x;
+    p.redo = reinterpret_cast<uint32_t*>(base + w.redo);
+    if (cudaMemsetAsync(p.redo, 0, sizeof(uint32_t), st) != cudaSuccess) return HYQ_ERR_CUDA;
     if (a.ev_kernel_start && cudaEventRecord(static_cast<cudaEvent_t>(a.ev_kernel_start), st) != cudaSuccess) return HYQ_ERR_CUDA;
     kern<<<grid, TC_THREADS, TC_SMEM_BYTES, st>>>(maps, p);
     if (launch_status() != HYQ_OK) return HYQ_ERR_CUDA;
+    const long n_ctas = (long)grid.x * grid.y * grid.z;
+    if (lowbit_fp8) {
+        kern_exact<<<(unsigned)(n_ctas < 148 ? n_ctas : 148), TC_THREADS, TC_SMEM_BYTES, st>>>(maps, p);
+        if (launch_status() != HYQ_OK) return HYQ_ERR_CUDA;
+    }
     if (split) {
         const long n_rows = (long)a.B * a.Hq * (long)Lq, n_thr = n_rows * (HYQ_D / 4);
         attn_merge_kernel<<<(unsigned)((n_thr + 255) / 256), 256, 0, st>>>(p.part_o, p.part_ml, w.splits, n_rows, a.out, p.out_fp32, a.lse);

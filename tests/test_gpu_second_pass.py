@@ -1,0 +1,79 @@
+"""The tensor-core kernel's second pass.  With e4m3 scores (FP8, or INT4 codes widened to e4m3) the first launch
+takes the exponentials of most low-bit tiles against a row's reference as it stands and checks the tile's row sum
+afterwards; a CTA that sees an fp16 overflow there - a score more than 2^16 above everything the row had seen -
+writes nothing and leaves its block index on a list, and a second launch does those CTAs again with the maximum
+looked at in every tile.  These inputs plant one such key late in the low-bit region; the result must still match
+the oracle (Eq. 6-7), and the counter of the test hook shows that the second pass ran (and only then)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from gpu_util import MAX_ABS_TOL, MEAN_REL_TOL, ensure_built, errors, gpu_attention, oracle_quant_all
+from paper_2608_27875_b200 import api, workloads as wl
+
+pytestmark = pytest.mark.gpu
+INT8, FP8, INT4FP8 = (wl.FMT_INT8,) * 3, (wl.FMT_FP8_E4M3,) * 3, (wl.FMT_INT4, wl.FMT_INT4, wl.FMT_FP8_E4M3)
+
+
+def _inputs(B, Hq, Hkv, Lq, L, W, k, j_star, seed):
+    """Gaussian Q, K, V; every query leans 6 units towards a fixed direction u, and key j_star is 30 u: its score
+    lies ~19 log2 units above the others'.  The vertical sets avoid j_star, so it is a low-bit key."""
+    g = torch.Generator().manual_seed(seed)
+    u = torch.ones(128) / 128 ** 0.5
+    Q = (torch.randn(B, Hq, Lq, 128, generator=g) + 6.0 * u).to(torch.bfloat16)
+    K = torch.randn(B, Hkv, L, 128, generator=g)
+    if j_star >= 0:
+        K[:, :, j_star] = 30.0 * u
+    V = torch.randn(B, Hkv, L, 128, generator=g).to(torch.bfloat16)
+    rng = np.random.default_rng(seed)
+    cand = np.array([j for j in range(max(0, L - W)) if j != j_star])
+    idx = np.stack([np.stack([np.sort(rng.choice(cand, k, replace=False)) for _ in range(Hq)]) for _ in range(B)]).astype(np.int32)
+    return Q, K.to(torch.bfloat16), V, idx
+
+
+@pytest.mark.parametrize("fmts,B,Hq,Hkv,L,W,k,bt,j_star,expect_second", [
+    (INT4FP8, 1, 4, 2, 2048, 128, 16, 64, 1000, True),
+    (FP8, 2, 2, 1, 1500, 100, 8, 64, 700, True),
+    (INT4FP8, 1, 2, 2, 1500, 128, 8, 32, 900, True),       # 32-token quantization blocks (the other translation unit)
+    (INT4FP8, 1, 2, 2, 1500, 128, 8, 64, -1, False),       # no such key: the first launch's result stands
+    (INT8, 1, 2, 2, 1500, 128, 8, 64, 900, False),         # integer scores: every maximum is looked at in the first place
+])
+def test_a_late_dominant_key_goes_through_the_second_pass_and_matches_the_oracle(fmts, B, Hq, Hkv, L, W, k, bt, j_star, expect_second):
+    ensure_built()
+    Q, K, V, idx = _inputs(B, Hq, Hkv, L, L, W, k, j_star, seed=L + bt)
+    qz = oracle_quant_all(Q, K, V, fmts, bt)
+    api.hyq_test_read_attention_restarts(reset=True)
+    got = gpu_attention(Q, K, V, qz, fmts, idx, W, api.IMPL_TCGEN05, block_tokens=bt).numpy()
+    n_second = api.hyq_test_read_attention_restarts(reset=True)
+    assert (n_second > 0) == expect_second, n_second
+    (qc, qs), (kc, ks), (vc, vs) = qz
+    ref = oracle.attention_rows(wl.bits(Q), wl.bits(K), wl.bits(V), qc, kc, vc, qs, ks, vs, fmts, idx, W, None, block_tokens=bt)
+    assert np.isfinite(got).all()
+    max_abs, mean_rel = errors(got, ref)
+    assert max_abs <= MAX_ABS_TOL and mean_rel <= MEAN_REL_TOL, (max_abs, mean_rel)
+
+
+def test_second_pass_of_a_short_query_block_with_split_keys():
+    """512 query rows against 16384 keys: the keys of a pair of query tiles are split over several CTAs, the slice that
+    holds the dominant key is done again, and the merge of the slices sees both launches' partial results."""
+    ensure_built()
+    fmts, B, Hq, Hkv, Lq, L, W, k, j_star = INT4FP8, 1, 2, 1, 512, 16384, 1024, 64, 9000
+    Q, K, V, idx = _inputs(B, Hq, Hkv, Lq, L, W, k, j_star, seed=77)
+    Qd, Kd, Vd = Q.cuda(), K.cuda(), V.cuda()
+    (qc, qs), (kc, ks), (vc, vs) = [api.hyq_quantize_blocks(t, f) for t, f in zip((Qd, Kd, Vd), fmts)]
+    idx_t = torch.from_numpy(idx).cuda()
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    api.hyq_test_read_attention_restarts(reset=True)
+    tc = api.hyq_hybrid_attention_prefill(Qd, Kd, Vd, qc, kc, vc, qs, ks, vs, fmts, idx_t, W, impl=api.IMPL_TCGEN05, status_word=status)
+    n_second = api.hyq_test_read_attention_restarts(reset=True)
+    simt = api.hyq_hybrid_attention_prefill(Qd, Kd, Vd, qc, kc, vc, qs, ks, vs, fmts, idx_t, W, impl=api.IMPL_SIMT)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0 and n_second > 0
+    assert torch.isfinite(tc).all()
+    assert float((tc - simt).abs().max()) <= MAX_ABS_TOL
+
+
+def test_the_counter_hook_checks_its_argument():
+    lib = ensure_built()
+    assert lib.hyq_test_read_attention_restarts(None, 0) == 1
