@@ -40,7 +40,7 @@ NOMINAL = {"bf16_tflops": 2250.0, "lowbit_tflops": 4500.0, "hbm_gbs": 8000.0}
 FALLBACK = {"bf16_tflops": 1590.0, "hbm_gbs": 6650.0}
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu
 # capture summarised under profiles/ (bytes per launch of the benchmark workload; None = no capture yet)
-NCU_TRAFFIC_BYTES = {"c2": 693018624 + 500875264}
+NCU_TRAFFIC_BYTES = {"c2": 733547008 + 503056896}
 # decode_kernel on the c2 cache shape, captured at batch 4 (157.169 MB read + 3.803 MB written); traffic grows in
 # proportion to the batch, so the bench scales it by B / 4
 NCU_DECODE_TRAFFIC_BYTES_B4 = 157169152 + 3803392
