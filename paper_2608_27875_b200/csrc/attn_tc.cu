@@ -675,8 +675,13 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                 }
                 uint32_t ra[32], rb[32];
                 tmem_ld32(ts, ra);
-                tmem_ld32(ts + 32, rb);
-                tmem_wait_ld();
+                if (skip_max) {
+                    tmem_wait_ld();                             // the second half arrives under the first half's exponentials
+                    tmem_ld32(ts + 32, rb);
+                } else {
+                    tmem_ld32(ts + 32, rb);
+                    tmem_wait_ld();
+                }
                 if (NEED_RANGE) {
                     mask_cols32(ra, 0, lo_eff, span, knock);
                     mask_cols32(rb, 32, lo_eff, span, knock);
@@ -733,6 +738,7 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                 uint32_t pa[16], pb[16];
                 const float t_a = row_exp32(ra, cs, bias, pa);
                 tmem_st16(ts, pa);
+                if (skip_max) tmem_wait_ld();
 #if HYQ_TC_VARIANT_BT
                 const float t_b = row_exp32(rb, csb, int_scores ? fmaf(-INT_MAGIC_F, csb, -m_eff) : -m_eff, pb);
 #else
