@@ -767,8 +767,57 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
 #endif
                 const auto vl = nvl;
                 prefetch_tile(n + 1);
-                if (!do_tile(std::false_type{}, n, cs, vl, !LOWBIT_FP8, 0, 0u, LOWBIT_FP8 && warm)) { aborted = true; break; }
-                if (!EXACT && LOWBIT_FP8 && !warm && n - n0 >= 1) warm = __all_sync(0xffffffffu, m_used > -INFINITY);
+                if (!do_tile(std::false_type{}, n, cs, vl, !LOWBIT_FP8, 0, 0u, false)) { aborted = true; break; }
+                if (!EXACT && LOWBIT_FP8 && n - n0 >= 1 && __all_sync(0xffffffffu, m_used > -INFINITY)) { ++n; warm = true; break; }
+            }
+            if (!EXACT && LOWBIT_FP8 && warm && !aborted) {
+                // Steady state of the first launch: exponentials against the reference as it stands.  The first half of a
+                // tile's scores is read while the previous tile's second half is still being worked on (when the scores
+                // are there by then), the second half under the first half's exponentials.
+                const int n_end = min(n_plain, n_total);
+                uint32_t ra[32], rb[32];
+                bool have_a = false;
+                for (; n < n_end; ++n) {
+                    const float cs = fmaxf(qs2 * nks, 1e-37f);
+#if HYQ_TC_VARIANT_BT
+                    const float csb = fmaxf(qs2 * nks_b, 1e-37f);
+#else
+                    const float csb = cs;
+#endif
+                    prefetch_tile(n + 1);
+                    const int nl = n - n0, buf = nl & 1;
+                    const uint32_t ts = ts0 + buf * BN;
+                    if (!have_a) {
+                        if (!__all_sync(0xffffffffu, mbar_wait(&bars.s_full[q][buf], (uint32_t)(nl >> 1) & 1u, limit))) { dead = true; aborted = true; break; }
+                        tc_fence_after();
+                        tmem_ld32(ts, ra);
+                    }
+                    tmem_wait_ld();
+                    tmem_ld32(ts + 32, rb);
+                    const float bias = -m_used;
+                    uint32_t pa[16], pb[16];
+                    const float t_a = row_exp32(ra, cs, bias, pa);
+                    tmem_st16(ts, pa);
+                    tmem_wait_ld();
+                    have_a = false;
+                    if (n + 1 < n_end) {
+                        const int nl1 = nl + 1, buf1 = nl1 & 1;
+                        if (__all_sync(0xffffffffu, mbar_test_wait(&bars.s_full[q][buf1], (uint32_t)(nl1 >> 1) & 1u))) {
+                            tc_fence_after();
+                            tmem_ld32(ts0 + buf1 * BN, ra);
+                            have_a = true;
+                        }
+                    }
+                    const float t_b = row_exp32(rb, csb, bias, pb);
+                    tmem_st16(ts + 16, pb);
+                    l_h += t_a + t_b;
+                    over |= !(t_a + t_b < P_SUM_LIMIT);
+                    tmem_wait_st();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&bars.p_full[q][buf]);
+                }
+                if (have_a) tmem_wait_ld();
             }
             // ---- the remaining low-bit tiles, the vertical-line tiles and the window tiles
             // (number of vertical-line keys this row may use: only needed from here on)
