@@ -57,7 +57,8 @@ def measured_peaks():
     if os.path.exists(path):
         with open(path) as f:
             d = json.load(f)
-        return {"bf16_tflops": float(d["bf16_tflops"]), "hbm_gbs": float(d["hbm_gbs"]), "source": "measured"}
+        return {"bf16_tflops": float(d["bf16_tflops"]), "hbm_gbs": float(d["hbm_gbs"]), "source": "measured",
+                "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", 0.0)) or None}
     return dict(FALLBACK, source="fallback")
 
 
@@ -718,6 +719,8 @@ def run_hyq(args, w):
     k_ms = kern_ms if kern_ms else attn_call_ms
     achieved = flops / (k_ms * 1e-3) / 1e12
     peak_eff = flops / t_roof_meas / 1e12
+    sus = peaks.get("bf16_tflops_sustained")
+    t_roof_sus = roofline_seconds(wr, n_fp, sus, 2 * sus, peaks["hbm_gbs"])[0] if sus else None
     roofline = {
         "bound": "tensor", "kernel": "attn_tc_kernel", "achieved": achieved, "peak": peak_eff, "unit": "TFLOP/s",
         "frac": achieved / peak_eff, "traffic": NCU_TRAFFIC_BYTES.get(w.name),
@@ -729,7 +732,12 @@ def run_hyq(args, w):
         "fp_pair_share": n_fp / wr.causal_pairs, "roofline_ms_measured": t_roof_meas * 1e3,
         "roofline_ms_nominal": t_roof_nom * 1e3, "frac_nominal": (t_roof_nom * 1e3) / k_ms,
         "frac_whole_step": (t_roof_meas * 1e3) / ms_per_step,
+        "frac_isolated": (t_roof_meas * 1e3) / kern_ms_isolated if kern_ms_isolated else None,
         "frac_nominal_whole_step": (t_roof_nom * 1e3) / ms_per_step, "min_bytes": bytes_min,
+        "frac_at_sustained_peak": (t_roof_sus * 1e3) / k_ms if t_roof_sus else None,
+        "sustained_note": "context only: the same fraction against the sustained bf16 figure of MEASURED_PEAKS.json (a matmul "
+                          "looped for seconds, at the clocks it falls to); `frac` keeps the burst figure, the larger denominator, "
+                          "because the timed region here is a fraction of a second",
         "nominal_definition": "the workload definition's roofline: full-precision pairs at 2250 TFLOP/s dense bf16, low-bit "
                               "pairs at 4500 TFLOP/s dense INT8/FP8, or the minimum bytes at 8 TB/s if larger (frac_nominal); "
                               "`frac` and `peak` use this pool's measured bf16 matmul rate instead, as the measurement "
