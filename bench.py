@@ -192,9 +192,9 @@ def run_reference(args, w):
 def launches_per_step(w) -> int:
     """Kernels of the library launched by one pass of the path: select 3, quantize 3, the attention pre-pass (bitmask,
     V to fp16; with vertical keys the gather and, for FP8 / INT4 scores, the vertical-line operand tiles; 2 INT4
-    widenings when used) and the attention kernel (two launches with FP8 / INT4 scores)."""
+    widenings when used) and the two launches of the attention kernel."""
     prepass = 1 + ((2 + (1 if w.q_fmt != wl.FMT_INT8 else 0)) if w.k > 0 else 0) + (2 if w.q_fmt == wl.FMT_INT4 else 0)
-    attention = 1 if w.q_fmt == wl.FMT_INT8 else 2      # FP8 / INT4 scores: the second launch that goes through the redo list
+    attention = 2                                       # the second launch goes through the redo list (normally empty)
     return 3 + 3 + prepass + attention
 
 

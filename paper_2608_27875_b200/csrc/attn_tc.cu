@@ -364,6 +364,8 @@ __device__ __forceinline__ bool tma_producer(const TcMaps& maps, const QSched& q
 // 64 probabilities as fp16 pairs over the first 32 columns of the buffer it read.
 constexpr int TC_THREADS = 384;                     // TMA producer, 2 MMA issuers, 1 idle warp, 8 softmax warps
 constexpr float P_SUM_LIMIT = 65504.0f;             // a tile's row sum below the largest fp16 number: none of its P overflowed
+constexpr int WARM_TILES = 8;                       // tiles at the start of a walk whose maximum is always looked at, and ...
+constexpr float WARM_SPREAD = 6.0f;                 // ... how far apart (log2 units) their maxima may lie for the rest to go without
 constexpr float RAISE_THRESHOLD = 14.0f;            // log2 units by which a tile must exceed the reference to raise it (P stays below 2^14, inside fp16)
 
 // row maximum of 32 float scores held in registers
@@ -577,7 +579,7 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
         // first launch: the CTA's eight softmax warps agree whether any row's exponentials overflowed; if so the CTA's
         // block index goes on the list of the second launch and nothing is written
         auto agree = [&](bool over_any) -> bool {
-            if (EXACT || !LOWBIT_FP8) return false;
+            if (EXACT) return false;
             if (__any_sync(0xffffffffu, over_any) && lane == 0) *restart_flag = 1;
             bar_sync_named(1, 8 * 32);
             const bool again = *restart_flag != 0 && *abort_flag == 0;
@@ -657,7 +659,8 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
 
             // one tile of the online softmax for this thread's row: all 64 columns, in two register halves.  Returns
             // false when this warp ran into an expired wait.
-            auto do_tile = [&](auto range_tag, int n, float cs, uint64_t vl, bool int_scores, int lo_eff, unsigned span, bool skip_max = false) -> bool {
+            float tile_max = -INFINITY;                         // maximum of the tile last looked at (this row, log2 units)
+            auto do_tile = [&](auto range_tag, int n, float cs, uint64_t vl, bool int_scores, int lo_eff, unsigned span) -> bool {
                 constexpr bool NEED_RANGE = decltype(range_tag)::value;
                 const uint32_t knock = int_scores ? KNOCKOUT_S32 : KNOCKOUT_F32;
                 const int nl = n - n0;                          // tile number within this CTA's slice
@@ -675,13 +678,8 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                 }
                 uint32_t ra[32], rb[32];
                 tmem_ld32(ts, ra);
-                if (skip_max) {
-                    tmem_wait_ld();                             // the second half arrives under the first half's exponentials
-                    tmem_ld32(ts + 32, rb);
-                } else {
-                    tmem_ld32(ts + 32, rb);
-                    tmem_wait_ld();
-                }
+                tmem_ld32(ts + 32, rb);
+                tmem_wait_ld();
                 if (NEED_RANGE) {
                     mask_cols32(ra, 0, lo_eff, span, knock);
                     mask_cols32(rb, 32, lo_eff, span, knock);
@@ -695,7 +693,7 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
 #if HYQ_TC_VARIANT_BT
                 const float csb = cs_hi;                        // the second half's factor (its own K scale with 32-token blocks)
 #endif
-                if (!skip_max) {                                // (skipped: exponentials against the reference as it stands)
+                {
 #if HYQ_TC_VARIANT_BT
                 const float fa = row_max32(ra) - (int_scores ? INT_MAGIC_F : 0.0f), fb = row_max32(rb) - (int_scores ? INT_MAGIC_F : 0.0f);
                 const float mt = fmaxf((fa == -INFINITY) ? -INFINITY : fa * cs, (fb == -INFINITY) ? -INFINITY : fb * csb);
@@ -703,6 +701,7 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                 const float f = fmaxf(row_max32(ra), row_max32(rb)) - (int_scores ? INT_MAGIC_F : 0.0f);
                 const float mt = (f == -INFINITY) ? -INFINITY : f * cs;
 #endif
+                tile_max = mt;
                 const bool raise = mt > m_used + RAISE_THRESHOLD;
                 if (__any_sync(0xffffffffu, raise)) {
                     const float alpha = raise ? ex2f(m_used - mt) : 1.0f;      // m_used = -inf -> 0
@@ -738,14 +737,12 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                 uint32_t pa[16], pb[16];
                 const float t_a = row_exp32(ra, cs, bias, pa);
                 tmem_st16(ts, pa);
-                if (skip_max) tmem_wait_ld();
 #if HYQ_TC_VARIANT_BT
                 const float t_b = row_exp32(rb, csb, int_scores ? fmaf(-INT_MAGIC_F, csb, -m_eff) : -m_eff, pb);
 #else
                 const float t_b = row_exp32(rb, cs, bias, pb);
 #endif
                 l_h += t_a + t_b;
-                if (!EXACT && LOWBIT_FP8) over |= !(t_a + t_b < P_SUM_LIMIT);               // (an overflowed or undefined sum included)
                 tmem_st16(ts + 16, pb);
                 tmem_wait_st();
                 tc_fence_before();
@@ -757,8 +754,12 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
             // ---- low-bit tiles that lie wholly below every row's window: no range mask, no bounds to compute
             const int n_plain = ragged ? 0 : min(own.a_end, max(0, (qhi(sq.i0 + off) + 1) / BN));
             int n = n0;
-            // (first launch: once every row of the warp has a finite reference, the plain tiles go without their maximum)
+            // First launch: the first WARM_TILES tiles are looked at in full.  If the maxima of these tiles lie close together
+            // for every row of the warp (scores without heavy tails: none of the later ones will be 2^16 above the reference),
+            // the plain tiles that follow go without their maximum; a warp with a row whose tile maxima spread out keeps
+            // looking (such rows raise their reference often, and a second pass over the whole CTA would cost more).
             bool warm = false;
+            float mt_lo = INFINITY, mt_hi = -INFINITY;
             for (; n < min(n_plain, n_total); ++n) {
                 // a zero scale (all-zero tile) still has to let -inf pass through the multiply
                 const float cs = fmaxf(qs2 * nks, 1e-37f);
@@ -767,10 +768,14 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
 #endif
                 const auto vl = nvl;
                 prefetch_tile(n + 1);
-                if (!do_tile(std::false_type{}, n, cs, vl, !LOWBIT_FP8, 0, 0u, false)) { aborted = true; break; }
-                if (!EXACT && LOWBIT_FP8 && n - n0 >= 1 && __all_sync(0xffffffffu, m_used > -INFINITY)) { ++n; warm = true; break; }
+                if (!do_tile(std::false_type{}, n, cs, vl, !LOWBIT_FP8, 0, 0u)) { aborted = true; break; }
+                if (!EXACT && n - n0 < WARM_TILES) {
+                    mt_lo = fminf(mt_lo, tile_max);
+                    mt_hi = fmaxf(mt_hi, tile_max);
+                    if (n - n0 == WARM_TILES - 1 && __all_sync(0xffffffffu, m_used > -INFINITY && mt_hi - mt_lo < WARM_SPREAD)) { ++n; warm = true; break; }
+                }
             }
-            if (!EXACT && LOWBIT_FP8 && warm && !aborted) {
+            if (!EXACT && warm && !aborted) {
                 // Steady state of the first launch: exponentials against the reference as it stands.  The first half of a
                 // tile's scores is read while the previous tile's second half is still being worked on (when the scores
                 // are there by then), the second half under the first half's exponentials.
@@ -784,17 +789,27 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
 #else
                     const float csb = cs;
 #endif
+                    uint64_t vl = nvl;                         // this tile's vertical-line columns (integer scores only)
                     prefetch_tile(n + 1);
                     const int nl = n - n0, buf = nl & 1;
                     const uint32_t ts = ts0 + buf * BN;
                     if (!have_a) {
                         if (!__all_sync(0xffffffffu, mbar_wait(&bars.s_full[q][buf], (uint32_t)(nl >> 1) & 1u, limit))) { dead = true; aborted = true; break; }
                         tc_fence_after();
+                        if (!LOWBIT_FP8 && vl != 0ull) {
+                            while (vl) { const int c = __ffsll((long long)vl) - 1; vl &= vl - 1; tmem_st1(ts + c, knock_lq); }
+                            tmem_wait_st();
+                        }
                         tmem_ld32(ts, ra);
                     }
                     tmem_wait_ld();
                     tmem_ld32(ts + 32, rb);
-                    const float bias = -m_used;
+                    if (!LOWBIT_FP8) {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) ra[e] += INT_MAGIC;
+                    }
+                    const float bias = LOWBIT_FP8 ? -m_used : fmaf(-INT_MAGIC_F, cs, -m_used);
+                    const float bias_b = LOWBIT_FP8 ? -m_used : fmaf(-INT_MAGIC_F, csb, -m_used);
                     uint32_t pa[16], pb[16];
                     const float t_a = row_exp32(ra, cs, bias, pa);
                     tmem_st16(ts, pa);
@@ -804,11 +819,20 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
                         const int nl1 = nl + 1, buf1 = nl1 & 1;
                         if (__all_sync(0xffffffffu, mbar_test_wait(&bars.s_full[q][buf1], (uint32_t)(nl1 >> 1) & 1u))) {
                             tc_fence_after();
+                            if (!LOWBIT_FP8 && nvl != 0ull) {     // (nvl: the next tile's columns by now)
+                                uint64_t v1 = nvl;
+                                while (v1) { const int c = __ffsll((long long)v1) - 1; v1 &= v1 - 1; tmem_st1(ts0 + buf1 * BN + c, knock_lq); }
+                                tmem_wait_st();
+                            }
                             tmem_ld32(ts0 + buf1 * BN, ra);
                             have_a = true;
                         }
                     }
-                    const float t_b = row_exp32(rb, csb, bias, pb);
+                    if (!LOWBIT_FP8) {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) rb[e] += INT_MAGIC;
+                    }
+                    const float t_b = row_exp32(rb, csb, bias_b, pb);
                     tmem_st16(ts + 16, pb);
                     l_h += t_a + t_b;
                     over |= !(t_a + t_b < P_SUM_LIMIT);
@@ -1056,7 +1080,7 @@ int launch_attn_tc(const hyq_attn_args& a, float alpha, cudaStream_t st) {
     kern<<<grid, TC_THREADS, TC_SMEM_BYTES, st>>>(maps, p);
     if (launch_status() != HYQ_OK) return HYQ_ERR_CUDA;
     const long n_ctas = (long)grid.x * grid.y * grid.z;
-    if (lowbit_fp8) {
+    {
         kern_exact<<<(unsigned)(n_ctas < 148 ? n_ctas : 148), TC_THREADS, TC_SMEM_BYTES, st>>>(maps, p);
         if (launch_status() != HYQ_OK) return HYQ_ERR_CUDA;
     }
