@@ -441,8 +441,8 @@ __device__ __forceinline__ void mask_cols32(uint32_t (&raw)[32], int c0, int lo_
 // SPLIT (short query blocks only): several CTAs share a pair of query tiles, each on a contiguous slice of the
 // walk; they leave unnormalised partial results that attn_merge_kernel combines by their reference maxima.
 // EXACT = false is the kernel of the first launch: one CTA per block index.  After the first tiles of a row's low-bit pass
-// it takes the exponentials against the row's reference as it stands, without looking for the tile's maximum, and
-// every tile's row sum tells afterwards whether that was safe (no P beyond fp16).  If it was not for any row of the
+// (and if their maxima lie close together) it takes the exponentials against the row's reference as it stands, without
+// looking for the tile's maximum, and every tile's row sum tells afterwards whether that was safe (no P beyond fp16).  If it was not for any row of the
 // CTA - a score more than 2^16 above everything the row had seen - the CTA writes no output and puts its block
 // index on a list.  EXACT = true is the kernel of the second launch, a small grid that goes through that list
 // (normally empty) with the maximum looked at in every tile.
@@ -759,8 +759,8 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
             // the plain tiles that follow go without their maximum; a warp with a row whose tile maxima spread out keeps
             // looking (such rows raise their reference often, and a second pass over the whole CTA would cost more).
             bool warm = false;
-            float mt_lo = INFINITY, mt_hi = -INFINITY;
-            for (; n < min(n_plain, n_total); ++n) {
+            const int n_plain_end = min(n_plain, n_total);
+            auto plain_tile = [&]() -> bool {
                 // a zero scale (all-zero tile) still has to let -inf pass through the multiply
                 const float cs = fmaxf(qs2 * nks, 1e-37f);
 #if HYQ_TC_VARIANT_BT
@@ -768,18 +768,26 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
 #endif
                 const auto vl = nvl;
                 prefetch_tile(n + 1);
-                if (!do_tile(std::false_type{}, n, cs, vl, !LOWBIT_FP8, 0, 0u)) { aborted = true; break; }
-                if (!EXACT && n - n0 < WARM_TILES) {
+                return do_tile(std::false_type{}, n, cs, vl, !LOWBIT_FP8, 0, 0u);
+            };
+            if (!EXACT && n_plain_end - n0 > WARM_TILES) {
+                float mt_lo = INFINITY, mt_hi = -INFINITY;
+                for (; n < n0 + WARM_TILES; ++n) {
+                    if (!plain_tile()) { aborted = true; break; }
                     mt_lo = fminf(mt_lo, tile_max);
                     mt_hi = fmaxf(mt_hi, tile_max);
-                    if (n - n0 == WARM_TILES - 1 && __all_sync(0xffffffffu, m_used > -INFINITY && mt_hi - mt_lo < WARM_SPREAD)) { ++n; warm = true; break; }
                 }
+                warm = !aborted && __all_sync(0xffffffffu, m_used > -INFINITY && mt_hi - mt_lo < WARM_SPREAD);
+            }
+            if (!warm) {
+                for (; n < n_plain_end && !aborted; ++n)
+                    if (!plain_tile()) { aborted = true; break; }
             }
             if (!EXACT && warm && !aborted) {
                 // Steady state of the first launch: exponentials against the reference as it stands.  The first half of a
                 // tile's scores is read while the previous tile's second half is still being worked on (when the scores
                 // are there by then), the second half under the first half's exponentials.
-                const int n_end = min(n_plain, n_total);
+                const int n_end = n_plain_end;
                 uint32_t ra[32], rb[32];
                 bool have_a = false;
                 for (; n < n_end; ++n) {
