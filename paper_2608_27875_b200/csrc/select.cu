@@ -19,6 +19,7 @@ namespace hyq {
 constexpr int SCORE_KEYS = 128;      // keys per CTA in vscore_kernel
 constexpr int SCORE_GC = 4;          // query heads scored per pass over the staged K tile
 constexpr int TOPK_THREADS = 1024;
+constexpr int SCAN_DEPTH = 8;         // loads of the score row a thread of the radix select keeps in flight
 constexpr int TOPK_CAND = 1536;      // candidate keys that the radix select keeps in shared memory
 
 // -------------------------------------------------------------------------------------------
@@ -153,10 +154,17 @@ topk_kernel(const double* __restrict__ scores, int P, int k, int32_t* __restrict
                 if ((key >> (shift + 8)) == (prefix >> (shift + 8))) atomicAdd(&whist[wid][(int)((key >> shift) & 0xFF)], 1);
             }
         } else {
-            for (int p = seg0 + lane; p < seg1; p += 32) {
-                const unsigned long long key = order_key(row[p]);
-                if (pass == 0 || (key >> (shift + 8)) == (prefix >> (shift + 8)))
-                    atomicAdd(&whist[wid][(int)((key >> shift) & 0xFF)], 1);
+            // (eight loads in flight per thread: a scan of the row is bound by their latency)
+            for (int p0 = seg0 + lane; p0 < seg1; p0 += 32 * SCAN_DEPTH) {
+                double v[SCAN_DEPTH];
+#pragma unroll
+                for (int j = 0; j < SCAN_DEPTH; ++j) v[j] = (p0 + 32 * j < seg1) ? __ldg(row + p0 + 32 * j) : 0.0;
+#pragma unroll
+                for (int j = 0; j < SCAN_DEPTH; ++j) {
+                    const unsigned long long key = order_key(v[j]);
+                    if (p0 + 32 * j < seg1 && (pass == 0 || (key >> (shift + 8)) == (prefix >> (shift + 8))))
+                        atomicAdd(&whist[wid][(int)((key >> shift) & 0xFF)], 1);
+                }
             }
         }
         __syncthreads();
@@ -197,9 +205,15 @@ topk_kernel(const double* __restrict__ scores, int P, int k, int32_t* __restrict
         prefix = sh_prefix;
         k_rem = sh_krem;
         if (!gathered && pass < 6 && sh_bin <= TOPK_CAND) {
-            for (int p = seg0 + lane; p < seg1; p += 32) {
-                const unsigned long long key = order_key(row[p]);
-                if ((key >> shift) == (prefix >> shift)) cand[atomicAdd(&n_cand, 1)] = key;
+            for (int p0 = seg0 + lane; p0 < seg1; p0 += 32 * SCAN_DEPTH) {
+                double v[SCAN_DEPTH];
+#pragma unroll
+                for (int j = 0; j < SCAN_DEPTH; ++j) v[j] = (p0 + 32 * j < seg1) ? __ldg(row + p0 + 32 * j) : 0.0;
+#pragma unroll
+                for (int j = 0; j < SCAN_DEPTH; ++j) {
+                    const unsigned long long key = order_key(v[j]);
+                    if (p0 + 32 * j < seg1 && (key >> shift) == (prefix >> shift)) cand[atomicAdd(&n_cand, 1)] = key;
+                }
             }
             gathered = true;                           // (uniform over the CTA: sh_bin is)
             __syncthreads();
@@ -210,28 +224,40 @@ topk_kernel(const double* __restrict__ scores, int P, int k, int32_t* __restrict
     // Scan 1 counts, per warp segment, the keys above and equal to the threshold; scan 2 writes: the output
     // slot of a selected position = (keys above the threshold before it) + min(keys equal before it, k_rem).
     int n_gt = 0, n_eq = 0;
-    for (int base = seg0; base < seg1; base += 32) {
-        const int p = base + lane;
-        const unsigned long long key = (p < seg1) ? order_key(row[p]) : 0ull;
-        n_gt += __popc(__ballot_sync(0xffffffffu, p < seg1 && key > prefix));
-        n_eq += __popc(__ballot_sync(0xffffffffu, p < seg1 && key == prefix));
+    for (int base = seg0; base < seg1; base += 32 * SCAN_DEPTH) {
+        double v[SCAN_DEPTH];
+#pragma unroll
+        for (int j = 0; j < SCAN_DEPTH; ++j) v[j] = (base + 32 * j + lane < seg1) ? __ldg(row + base + 32 * j + lane) : 0.0;
+#pragma unroll
+        for (int j = 0; j < SCAN_DEPTH; ++j) {
+            const bool live = base + 32 * j + lane < seg1;
+            const unsigned long long key = order_key(v[j]);
+            n_gt += __popc(__ballot_sync(0xffffffffu, live && key > prefix));
+            n_eq += __popc(__ballot_sync(0xffffffffu, live && key == prefix));
+        }
     }
     if (lane == 0) { warp_gt[wid] = n_gt; warp_eq[wid] = n_eq; }
     __syncthreads();
     int gt_run = 0, eq_run = 0;
     for (int w = 0; w < wid; ++w) { gt_run += warp_gt[w]; eq_run += warp_eq[w]; }
     const unsigned lt_mask = (1u << lane) - 1u;
-    for (int base = seg0; base < seg1; base += 32) {
-        const int p = base + lane;
-        const bool live = p < seg1;
-        const unsigned long long key = live ? order_key(row[p]) : 0ull;
-        const bool gt = live && key > prefix, eq = live && key == prefix;
-        const unsigned b_gt = __ballot_sync(0xffffffffu, gt), b_eq = __ballot_sync(0xffffffffu, eq);
-        const int eq_rank = eq_run + __popc(b_eq & lt_mask);
-        const int pos = gt_run + __popc(b_gt & lt_mask) + min(eq_rank, k_rem);
-        if ((gt || (eq && eq_rank < k_rem)) && pos < k) out[pos] = p;
-        gt_run += __popc(b_gt);
-        eq_run += __popc(b_eq);
+    for (int base = seg0; base < seg1; base += 32 * SCAN_DEPTH) {
+        double v[SCAN_DEPTH];
+#pragma unroll
+        for (int j = 0; j < SCAN_DEPTH; ++j) v[j] = (base + 32 * j + lane < seg1) ? __ldg(row + base + 32 * j + lane) : 0.0;
+#pragma unroll
+        for (int j = 0; j < SCAN_DEPTH; ++j) {
+            const int p = base + 32 * j + lane;
+            const bool live = p < seg1;
+            const unsigned long long key = order_key(v[j]);
+            const bool gt = live && key > prefix, eq = live && key == prefix;
+            const unsigned b_gt = __ballot_sync(0xffffffffu, gt), b_eq = __ballot_sync(0xffffffffu, eq);
+            const int eq_rank = eq_run + __popc(b_eq & lt_mask);
+            const int pos = gt_run + __popc(b_gt & lt_mask) + min(eq_rank, k_rem);
+            if ((gt || (eq && eq_rank < k_rem)) && pos < k) out[pos] = p;
+            gt_run += __popc(b_gt);
+            eq_run += __popc(b_eq);
+        }
     }
 }
 
