@@ -545,7 +545,7 @@ attn_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
             *reinterpret_cast<uint4*>(smem + SK_OFF + slot * G::STAGE_BYTES + ONES_OFF + chunk * 16) =
                 make_uint4(chunk < BM ? 0x3Cu : 0u, 0u, 0u, 0u);                               // 0x3C = 1.0 in e5m2
         }
-        fence_proxy_async_smem();
+        fence_proxy_async();
     }
     __syncthreads();
 
