@@ -25,7 +25,9 @@
 // softmax sees the scores: with e4m3 codes by a fifth MMA step per tile, S += ones . mask^T in e5m2 (the one
 // 8-bit format with an infinity), whose 64 x 32 operand - -inf in element 0 of a vertical key's row - is copied
 // in with the K codes; with int8 codes (no infinity) by the softmax warps, which store -inf over those columns
-// of S before they read the tile.  Every mbarrier wait is bounded; when one expires the CTA records
+// of S before they read the tile.  The attention call launches the kernel twice: the first launch takes most low-bit
+// tiles without looking for their maximum and checks the tiles' row sums instead, the second redoes the CTAs (normally
+// none) in which that check failed - see the comment at attn_tc_kernel.  Every mbarrier wait is bounded; when one expires the CTA records
 // HYQ_ERR_TIMEOUT in the status word, waits (bounded) for its own copies and MMAs in flight and unwinds.
 #include <cuda_fp16.h>
 
